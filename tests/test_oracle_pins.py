@@ -1,0 +1,324 @@
+"""Pins for the fp64 oracle: things the paper and the mathematics fix.
+
+None of these call the oracle to check the oracle: the expected values come
+from dense-mask brute force written differently (tests/bruteforce.py), from
+closed forms, or from numbers the paper prints.
+"""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from tests import bruteforce as bf
+
+RNG = np.random.default_rng
+
+
+def _qkv(rng, T, H, Hkv, d, scale=1.0):
+    return (rng.standard_normal((T, H, d)) * scale,
+            rng.standard_normal((T, Hkv, d)) * scale,
+            rng.standard_normal((T, Hkv, d)) * scale)
+
+
+def _fold(q, k, v, chunks, H, Hkv, d, base=10000.0, pos_shift=0, interleaved=False, **kw):
+    c = oracle.OracleCache(H, Hkv, d, capacity=q.shape[0], rope_base=base,
+                           interleaved=interleaved, **kw)
+    outs, lens = [], []
+    t0 = 0
+    for n in chunks:
+        outs.append(c.fold_step(q[t0:t0 + n], k[t0:t0 + n], v[t0:t0 + n], pos0=t0 + pos_shift))
+        t0 += n
+        lens.append(len(c))
+    return np.concatenate(outs, axis=0), lens, c
+
+
+# ---------------------------------------------------------------- brute force
+@pytest.mark.parametrize("H,Hkv,d,T", [(1, 1, 2, 5), (4, 1, 8, 33), (4, 2, 8, 48), (6, 3, 16, 64)])
+@pytest.mark.parametrize("interleaved", [False, True])
+def test_single_step_matches_dense_mask_bruteforce(H, Hkv, d, T, interleaved):
+    q, k, v = _qkv(RNG(1), T, H, Hkv, d)
+    ref, _ = bf.causal_attention(q, k, v, 10000.0, interleaved=interleaved)
+    got, _, _ = _fold(q, k, v, [T], H, Hkv, d, interleaved=interleaved)
+    assert np.abs(got - ref).max() <= 1e-12
+
+
+def test_rope_matches_complex_rotation():
+    rng = RNG(2)
+    x = rng.standard_normal((7, 3, 16))
+    tab = oracle.inv_freq(500000.0, 16)
+    assert np.allclose(tab, 500000.0 ** (-np.arange(8) * 2.0 / 16), rtol=1e-15, atol=0)
+    for inter in (False, True):
+        got = oracle.rope_fp64(x, 1000, tab, interleaved=inter)
+        ref = bf.rope_complex(x, np.arange(7) + 1000, 500000.0, interleaved=inter)
+        assert np.abs(got - ref).max() <= 1e-12
+
+
+def test_custom_inv_freq_table_is_honoured():
+    rng = RNG(3)
+    T, H, Hkv, d = 24, 2, 1, 8
+    q, k, v = _qkv(rng, T, H, Hkv, d)
+    tab = np.array([1.0, 0.3, 0.01, 0.0007])
+    ref, _ = bf.causal_attention(q, k, v, None, inv_freq=tab)
+    got, _, _ = _fold(q, k, v, [10, 14], H, Hkv, d, inv_freq_table=tab)
+    assert np.abs(got - ref).max() <= 1e-12
+
+
+# ------------------------------------------------- the paper's defining invariant
+def test_fold_equals_one_causal_pass_for_every_chunk_size():
+    """Folding chunk by chunk == the FULL condition's single causal pass (Section 2)."""
+    T, H, Hkv, d = 48, 4, 2, 8
+    q, k, v = _qkv(RNG(4), T, H, Hkv, d)
+    ref, _ = bf.causal_attention(q, k, v, 10000.0)
+    for C in range(1, T + 1):
+        chunks = [C] * (T // C) + ([T % C] if T % C else [])
+        got, lens, _ = _fold(q, k, v, chunks, H, Hkv, d)
+        assert np.abs(got - ref).max() <= 1e-12, C
+        assert lens == list(np.cumsum(chunks))
+
+
+def test_fold_with_mixed_chunk_lengths():
+    T, H, Hkv, d = 64, 4, 1, 16
+    q, k, v = _qkv(RNG(5), T, H, Hkv, d)
+    ref, _ = bf.causal_attention(q, k, v, 10000.0)
+    got, lens, _ = _fold(q, k, v, [17, 1, 1, 30, 8, 7], H, Hkv, d)
+    assert np.abs(got - ref).max() <= 1e-12
+    assert lens[-1] == T
+
+
+def test_tiny_config_fold_equals_monolithic():
+    """Config 1: 4 q heads / 1 KV head, d=64, C=64, 8 steps."""
+    T, H, Hkv, d, C = 512, 4, 1, 64, 64
+    q, k, v = _qkv(RNG(6), T, H, Hkv, d)
+    ref, _ = bf.causal_attention(q, k, v, 10000.0)
+    got, lens, _ = _fold(q, k, v, [C] * 8, H, Hkv, d)
+    assert np.abs(got - ref).max() <= 1e-12
+    assert lens == [C * (t + 1) for t in range(8)]      # len after t steps = t*C
+
+
+def test_isolated_condition_is_a_step_on_an_empty_cache():
+    T, H, Hkv, d = 16, 2, 2, 8
+    q, k, v = _qkv(RNG(7), T, H, Hkv, d)
+    c = oracle.OracleCache(H, Hkv, d, capacity=64)
+    c.fold_step(q, k, v)
+    c.reset()
+    assert len(c) == 0
+    got = c.fold_step(q, k, v, pos0=5)
+    ref, _ = bf.causal_attention(q, k, v, 10000.0, pos_offset=5)
+    assert np.abs(got - ref).max() <= 1e-12
+
+
+# ----------------------------------------------------------------- softmax facts
+def test_rows_sum_to_one_and_output_is_a_convex_combination():
+    T, H, Hkv, d = 96, 4, 2, 8
+    q, k, v = _qkv(RNG(8), T, H, Hkv, d, scale=3.0)
+    c = oracle.OracleCache(H, Hkv, d, capacity=T)
+    t0 = 0
+    for n in (32, 32, 32):
+        out, lse, rowsum = c.fold_step(q[t0:t0 + n], k[t0:t0 + n], v[t0:t0 + n], want_stats=True)
+        assert np.abs(rowsum - 1.0).max() <= 1e-14
+        assert np.isfinite(lse).all()
+        for i in range(n):
+            for h in range(H):
+                vis = v[:t0 + i + 1, h // 2, :]
+                assert (out[i, h] <= vis.max(axis=0) + 1e-12).all()
+                assert (out[i, h] >= vis.min(axis=0) - 1e-12).all()
+        t0 += n
+
+
+def test_lse_matches_bruteforce_logsumexp():
+    T, H, Hkv, d = 20, 2, 1, 8
+    q, k, v = _qkv(RNG(9), T, H, Hkv, d)
+    c = oracle.OracleCache(H, Hkv, d, capacity=T)
+    _, lse, _ = c.fold_step(q, k, v, want_stats=True)
+    qr = bf.rope_complex(q, np.arange(T), 10000.0)
+    kr = bf.rope_complex(k, np.arange(T), 10000.0)
+    for h in range(H):
+        s = (qr[:, h] @ kr[:, 0].T) / np.sqrt(d)
+        for i in range(T):
+            assert abs(lse[i, h] - np.log(np.exp(s[i, :i + 1]).sum())) <= 1e-12
+
+
+# ------------------------------------------------------------------ closed forms
+def test_first_token_returns_its_own_value_row():
+    q, k, v = _qkv(RNG(10), 8, 4, 2, 8)
+    out, _, _ = _fold(q, k, v, [8], 4, 2, 8)
+    for h in range(4):
+        assert np.array_equal(out[0, h], v[0, h // 2])
+
+
+def test_constant_value_rows_give_that_row():
+    rng = RNG(11)
+    q, k, _ = _qkv(rng, 40, 4, 2, 8)
+    row = rng.standard_normal((2, 8))
+    v = np.broadcast_to(row, (40, 2, 8)).copy()
+    out, _, _ = _fold(q, k, v, [16, 24], 4, 2, 8)
+    for h in range(4):
+        assert np.abs(out[:, h] - row[h // 2]).max() <= 1e-13
+
+
+def test_zero_queries_give_running_mean_of_values():
+    rng = RNG(12)
+    _, k, v = _qkv(rng, 50, 2, 1, 8)
+    q = np.zeros((50, 2, 8))
+    out, _, _ = _fold(q, k, v, [20, 30], 2, 1, 8)
+    mean = np.cumsum(v[:, 0], axis=0) / np.arange(1, 51)[:, None]
+    for h in range(2):
+        assert np.abs(out[:, h] - mean).max() <= 1e-13
+
+
+def test_position_zero_is_identity_and_rotation_keeps_pair_norms():
+    rng = RNG(13)
+    x = rng.standard_normal((1, 3, 16))
+    tab = oracle.inv_freq(10000.0, 16)
+    assert np.array_equal(oracle.rope_fp64(x, 0, tab), x)
+    y = oracle.rope_fp64(np.repeat(x, 9, axis=0), 12345, tab)
+    n_in = x[..., :8] ** 2 + x[..., 8:] ** 2
+    n_out = y[..., :8] ** 2 + y[..., 8:] ** 2
+    assert np.abs(n_out - n_in).max() <= 1e-12
+
+
+def test_shifting_all_positions_leaves_outputs_unchanged():
+    """RoPE scores depend on position differences only (continued positions, Section 2)."""
+    T, H, Hkv, d = 40, 4, 2, 16
+    q, k, v = _qkv(RNG(14), T, H, Hkv, d)
+    a, _, _ = _fold(q, k, v, [10] * 4, H, Hkv, d, base=500000.0)
+    b, _, _ = _fold(q, k, v, [10] * 4, H, Hkv, d, base=500000.0, pos_shift=100000)
+    assert np.abs(a - b).max() <= 1e-9
+    # and positions that do NOT continue across the boundary change the result
+    c = oracle.OracleCache(H, Hkv, d, capacity=T, rope_base=500000.0)
+    outs = [c.fold_step(q[t:t + 10], k[t:t + 10], v[t:t + 10], pos0=0) for t in range(0, T, 10)]
+    assert np.abs(np.concatenate(outs) - a).max() > 1e-3
+
+
+def test_gqa_equals_mha_with_replicated_kv_heads():
+    T, H, Hkv, d = 24, 4, 2, 8
+    q, k, v = _qkv(RNG(15), T, H, Hkv, d)
+    a, _, _ = _fold(q, k, v, [8] * 3, H, Hkv, d)
+    kk, vv = np.repeat(k, 2, axis=1), np.repeat(v, 2, axis=1)
+    b, _, _ = _fold(q, kk, vv, [8] * 3, H, H, d)
+    assert np.abs(a - b).max() <= 1e-14
+
+
+def test_permuting_prefix_rows_leaves_outputs_unchanged():
+    """Attention over the prefix is a set operation once keys carry their rotation."""
+    rng = RNG(16)
+    T, H, Hkv, d, P = 48, 2, 1, 8, 32
+    q, k, v = _qkv(rng, T, H, Hkv, d)
+    c1 = oracle.OracleCache(H, Hkv, d, capacity=T)
+    c1.fold_step(q[:P], k[:P], v[:P])
+    a = c1.fold_step(q[P:], k[P:], v[P:])
+    # second cache: the same prefix, fed one token at a time in a permuted order,
+    # each token at its ORIGINAL position
+    perm = rng.permutation(P)
+    c2 = oracle.OracleCache(H, Hkv, d, capacity=T)
+    for r in perm:
+        c2.fold_step(q[r:r + 1], k[r:r + 1], v[r:r + 1], pos0=int(r))
+    b = c2.fold_step(q[P:], k[P:], v[P:], pos0=P)
+    assert np.abs(a - b).max() <= 1e-12
+
+
+def test_planted_key_is_recovered_through_a_deep_chain():
+    """Kernel-level analogue of the needle test (Section 4): a key planted in chunk 0
+    dominates a late query's row and the output approaches the planted value row."""
+    rng = RNG(17)
+    T, H, Hkv, d, C = 256, 2, 1, 16, 8
+    q, k, v = _qkv(rng, T, H, Hkv, d, scale=0.1)
+    tab = oracle.inv_freq(10000.0, d)
+    needle_pos, query_pos = 3, T - 1
+    direction = rng.standard_normal(d)
+    direction /= np.linalg.norm(direction)
+    # choose pre-rotation k, q whose ROTATED versions are aligned: rotate back by -pos
+    def unrotate(vec, pos):
+        ang = pos * tab
+        z = (vec[:d // 2] + 1j * vec[d // 2:]) * np.exp(-1j * ang)
+        return np.concatenate([z.real, z.imag])
+    k[needle_pos, 0] = unrotate(direction * 30.0, needle_pos)
+    q[query_pos, :] = unrotate(direction * 30.0, query_pos)
+    out, lens, _ = _fold(q, k, v, [C] * (T // C), H, Hkv, d)
+    assert lens[-1] == T
+    for h in range(H):
+        assert np.abs(out[query_pos, h] - v[needle_pos, 0]).max() <= 1e-9
+
+
+# -------------------------------------------------------------- append / the cache
+def test_append_only_prefix_rows_are_bit_unchanged():
+    T, H, Hkv, d = 30, 2, 2, 8
+    q, k, v = _qkv(RNG(18), T, H, Hkv, d)
+    c = oracle.OracleCache(H, Hkv, d, capacity=T)
+    c.fold_step(q[:12], k[:12], v[:12])
+    k_before, v_before = c.k().copy(), c.v().copy()
+    c.fold_step(q[12:], k[12:], v[12:])
+    assert np.array_equal(c.k()[:, :12], k_before)
+    assert np.array_equal(c.v()[:, :12], v_before)
+    # values are cached as given, keys after rotation at their own positions
+    assert np.array_equal(c.v(), np.transpose(v, (1, 0, 2)))
+    kr = bf.rope_complex(k, np.arange(T), 10000.0)
+    assert np.abs(c.k() - np.transpose(kr, (1, 0, 2))).max() <= 1e-12
+
+
+def test_capacity_overflow_changes_nothing():
+    q, k, v = _qkv(RNG(19), 10, 2, 1, 8)
+    c = oracle.OracleCache(2, 1, 8, capacity=12)
+    c.fold_step(q, k, v)
+    with pytest.raises(OverflowError):
+        c.fold_step(q, k, v)
+    assert len(c) == 10
+
+
+def test_sampled_rows_equal_full_evaluation():
+    q, k, v = _qkv(RNG(20), 24, 4, 2, 8)
+    c1 = oracle.OracleCache(4, 2, 8, capacity=48)
+    c2 = oracle.OracleCache(4, 2, 8, capacity=48)
+    c1.fold_step(q, k, v)
+    c2.fold_step(q, k, v, rows=[0])
+    full = c1.fold_step(q, k, v)
+    part = c2.fold_step(q, k, v, rows=[0, 7, 23])
+    assert np.array_equal(part, full[[0, 7, 23]])
+    assert len(c1) == len(c2) == 48
+
+
+def test_cache_bytes_match_the_paper_s_printed_sizes():
+    """Section 5: 32 layers x 8 KV heads x 128 x (K,V) x 2 B per token, and the table's GB."""
+    per_token_all_layers = 32 * oracle.cache_bytes(8, 128, 1, 2)
+    assert per_token_all_layers == 131072
+    path = os.path.join(os.path.dirname(__file__), "golden", "cache_accounting.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    assert len(rows) == 4
+    for tokens, depth, gb in rows:
+        tokens, depth, gb = int(tokens), int(depth), float(gb)
+        total = 32 * oracle.cache_bytes(8, 128, tokens, 2)
+        assert abs(total / 1e9 - gb) <= 0.005 + 1e-9          # printed to 2 decimals
+        assert tokens // 256 - 1 == depth                   # chain depth at C = 256
+    assert 32 * oracle.cache_bytes(8, 128, 131072, 2) == 17179869184
+
+
+# ------------------------------------------------------- dtype-faithful rotation
+def _bf16_round(x32):
+    u = x32.astype(np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32)
+
+
+@pytest.mark.parametrize("interleaved", [False, True])
+def test_faithful_rotation_is_within_half_ulp_of_fp64(interleaved):
+    rng = RNG(21)
+    x = rng.standard_normal((64, 3, 32)).astype(np.float32)
+    tab = oracle.inv_freq(500000.0, 32)
+    exact = oracle.rope_fp64(x.astype(np.float64), 100000, tab, interleaved=interleaved)
+    y32 = oracle.rope_faithful(x, 100000, tab, interleaved=interleaved, to_bf16=False)
+    # three fp32 roundings (table value, cross product, fma): a few fp32 ulps of |x|
+    scale = np.abs(x).max()
+    assert np.abs(y32.astype(np.float64) - exact).max() <= 4 * 2.0 ** -24 * scale * 2
+    y16 = oracle.rope_faithful(x, 100000, tab, interleaved=interleaved, to_bf16=True)
+    # bf16 pattern: low 16 bits clear, and equal to RNE of the fp32 result
+    assert (y16.view(np.uint32) & 0xFFFF == 0).all()
+    assert np.array_equal(y16, _bf16_round(y32))
+    ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(exact), 1e-30))) - 7)
+    assert (np.abs(y16.astype(np.float64) - exact) <= 0.5 * ulp + 1e-6).all()
+
+
+def test_faithful_rotation_at_position_zero_is_identity():
+    x = RNG(22).standard_normal((1, 2, 16)).astype(np.float32)
+    tab = oracle.inv_freq(10000.0, 16)
+    assert np.array_equal(oracle.rope_faithful(x, 0, tab), x)
