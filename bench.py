@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the KV-Fold fold step on B200.
+
+One benchmark "step" is one whole chain of the deep-chain workload: the cache is reset to the
+empty accumulator and 131 072 tokens are folded in 512 chunks of 256 (chain depth 511), every
+chunk going through rotate+append, prefix+chunk attention and (when split) the combine kernel.
+`value` is tokens folded per second with the inputs resident in HBM; `e2e` is the same chain
+through the host-buffer entry point (pinned host q/k/v in, out back, copies inside the timing).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank folds its own
+independent sequence: there is no exchange on the data path, the only collective is the
+max-over-ranks of the elapsed time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2605_12471_b200 import workloads  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes (read + write) per attention launch measured once with ncu on a smaller chain and
+# scaled by cache rows read; None until a capture exists (see profiles/).
+NCU_TRAFFIC_BYTES_PER_CACHE_BYTE = None
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.lines = gpu_index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()          # the exact process started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower() == "active":
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_rate(w: workloads.Workload, seed: int, rows_per_step: int, repeats: int, prefix: int):
+    """Times the fp64 oracle (as it stands) on `rows_per_step` query rows of the chunk that follows
+    `prefix` cached tokens.  Returns (visible (query,key) pairs per second, seconds per repeat,
+    threads)."""
+    import numpy as np
+
+    import oracle
+    oc = oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, prefix + w.chunk * (repeats + 1),
+                            rope_base=w.rope_base)
+    gen = np.random.default_rng(seed)
+    block = 8192
+    done = 0
+    while done < prefix:                                   # fill the accumulator (not timed)
+        n = min(block, prefix - done)
+        k = gen.standard_normal((n, w.n_kv_heads, w.head_dim))
+        v = gen.standard_normal((n, w.n_kv_heads, w.head_dim))
+        q = np.zeros((n, w.n_q_heads, w.head_dim))
+        oc.fold_step(q, k, v, rows=[])
+        done += n
+    rows = sorted(set(int(x) for x in np.linspace(0, w.chunk - 1, rows_per_step)))
+    times, pairs = [], 0
+    for _ in range(repeats):
+        q = gen.standard_normal((w.chunk, w.n_q_heads, w.head_dim))
+        k = gen.standard_normal((w.chunk, w.n_kv_heads, w.head_dim))
+        v = gen.standard_normal((w.chunk, w.n_kv_heads, w.head_dim))
+        p0 = len(oc)
+        t0 = time.perf_counter()
+        oc.fold_step(q, k, v, rows=rows)
+        times.append(time.perf_counter() - t0)
+        pairs = sum(p0 + r + 1 for r in rows)
+    threads = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    return pairs / statistics.median(times), times, threads, rows
+
+
+def tokens_per_s_from_pairs(w: workloads.Workload, pairs_per_s: float) -> float:
+    """A chain of T tokens has T(T+1)/2 visible pairs: tokens/s = pairs/s / ((T+1)/2)."""
+    return pairs_per_s / ((w.tokens + 1) / 2.0)
+
+
+def run_reference(args, w):
+    """The reference arm: the CPU oracle, on a bounded sample of the same workload per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    prefix = w.tokens - w.chunk
+    import numpy as np
+
+    import oracle
+    oc = oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens + w.chunk * (args.steps + args.warmup),
+                            rope_base=w.rope_base)
+    gen = np.random.default_rng(args.seed)
+    done = 0
+    while done < prefix:
+        n = min(8192, prefix - done)
+        oc.fold_step(np.zeros((n, w.n_q_heads, w.head_dim)), gen.standard_normal((n, w.n_kv_heads, w.head_dim)),
+                     gen.standard_normal((n, w.n_kv_heads, w.head_dim)), rows=[])
+        done += n
+    rows = sorted(set(int(x) for x in np.linspace(0, w.chunk - 1, args.ref_rows)))
+    elapsed, pairs = 0.0, 0
+    for it in range(args.warmup + args.steps):
+        q = gen.standard_normal((w.chunk, w.n_q_heads, w.head_dim))
+        k = gen.standard_normal((w.chunk, w.n_kv_heads, w.head_dim))
+        v = gen.standard_normal((w.chunk, w.n_kv_heads, w.head_dim))
+        p0 = len(oc)
+        t0 = time.perf_counter()
+        oc.fold_step(q, k, v, rows=rows)
+        dt = time.perf_counter() - t0
+        if it >= args.warmup:
+            elapsed += dt
+            pairs += sum(p0 + r + 1 for r in rows)
+    value = tokens_per_s_from_pairs(w, pairs / elapsed)
+    threads = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    sample = (f"{len(rows)} query rows x {w.n_q_heads} heads per step at prefix >= {prefix} (last chunk of the "
+              f"chain), fp64 oracle; tokens/s extrapolated linearly in visible (query,key) pairs")
+    line = {
+        "impl": "reference", "metric": "fold-step tokens/s", "value": value, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * elapsed / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "tokens": w.tokens, "chunk": w.chunk, "n_q_heads": w.n_q_heads,
+                   "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--tokens", type=int, default=0, help="shorter chain (debugging; not the benchmark workload)")
+    ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--seed", type=int, default=2605)
+    ap.add_argument("--ref-rows", type=int, default=4)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--force-simt", action="store_true")
+    args = ap.parse_args()
+
+    w = workloads.DEEP_CHAIN
+    if args.tokens or args.chunk:
+        w = w.with_(name=f"deep_chain_debug_{args.tokens or w.tokens}_c{args.chunk or w.chunk}",
+                    tokens=args.tokens or w.tokens, chunk=args.chunk or w.chunk)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    from paper_2605_12471_b200 import binding, multi
+    import torch.distributed as dist
+
+    rank, world, local = multi.env_rank()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the fold step has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    lib = binding.load()
+
+    T, C, N = w.tokens, w.chunk, w.n_steps
+    H, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
+    q, k, v = workloads.sequence_inputs(w, args.seed, sequence=multi.sequence_of_rank(rank)[0], device="cuda")
+    out = torch.empty_like(q)
+    flags = binding.KVF_FORCE_SIMT if args.force_simt else 0
+    cache = binding.cache_for(w, flags=flags)
+    h = cache._h
+    stream = torch.cuda.current_stream().cuda_stream
+    eb = q.element_size()
+    qs, ks = C * H * d * eb, C * Hkv * d * eb
+    qp, kp, vp, op = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr()
+
+    def chain():
+        cache.reset()
+        for t in range(N):
+            rc = lib.kvf_fold_step(h, qp + t * qs, kp + t * ks, vp + t * ks, C, t * C, op + t * qs, None, stream)
+            if rc:
+                raise binding.KvfError(rc, "kvf_fold_step")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        a.record()
+        for _ in range(steps):
+            fn()
+        b.record()
+        barrier()
+        return multi.max_over_ranks(a.elapsed_time(b), device="cuda")
+
+    for _ in range(args.warmup):
+        chain()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    l0 = cache.launch_count()
+    ms = timed(chain, args.steps)
+    launches = cache.launch_count() - l0
+    clocks = sampler.stop() if rank == 0 else None
+    assert len(cache) == T
+    if cache.status() != binding.KVF_OK:
+        raise SystemExit("device status word reports a timed-out wait")
+    value = multi.whole_job_tokens_per_s(T, args.steps, world, ms)
+
+    # per-kernel time of the same chain, CUDA events around every launch on the launching stream
+    cache.profile(True)
+    chain()
+    kms, kcnt = cache.profile_read()
+    cache.profile(False)
+    pk = peaks()
+    attn_flops = w.flops_chain()
+    attn_tflops = attn_flops / (kms[1] * 1e-3) / 1e12
+    peak_tf = pk["bf16_tflops_sustained"]
+    cache_bytes_read = sum((t + 1) * C for t in range(N)) * w.cache_bytes_per_token()
+    traffic = None
+    if NCU_TRAFFIC_BYTES_PER_CACHE_BYTE is not None:
+        traffic = NCU_TRAFFIC_BYTES_PER_CACHE_BYTE * cache_bytes_read / kcnt[1]
+    roofline = {
+        "bound": "tensor", "kernel": "prefix+chunk attention", "achieved": attn_tflops, "peak": peak_tf,
+        "unit": "TFLOP/s", "frac": attn_tflops / peak_tf, "peak_source": pk["_source"] + " sustained bf16",
+        "traffic": traffic, "flops_per_launch": attn_flops / kcnt[1], "ms_per_launch": kms[1] / kcnt[1],
+        "launches": kcnt[1], "kernel_ms_per_chain": {"rope_append": kms[0], "attention": kms[1], "combine": kms[2]},
+        "hbm_gbs_cache_read": cache_bytes_read / (kms[1] * 1e-3) / 1e9, "hbm_peak_gbs": pk["hbm_gbs"],
+    }
+
+    e2e = None
+    if not args.no_e2e:
+        qh, kh, vh = (x.cpu().pin_memory() for x in (q, k, v))
+        oh = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        qhp, khp, vhp, ohp = qh.data_ptr(), kh.data_ptr(), vh.data_ptr(), oh.data_ptr()
+
+        def chain_host():
+            cache.reset()
+            for t in range(N):
+                rc = lib.kvf_fold_step_host(h, qhp + t * qs, khp + t * ks, vhp + t * ks, C, t * C, ohp + t * qs,
+                                            None, stream)
+                if rc:
+                    raise binding.KvfError(rc, "kvf_fold_step_host")
+
+        chain_host()
+        e2e_steps = max(1, min(args.steps, 3))
+        ems = timed(chain_host, e2e_steps)
+        e2e = {"value": world * e2e_steps * T / (ems * 1e-3), "unit": "tokens/s", "steps": e2e_steps,
+               "h2d_bytes_per_step": T * (H + 2 * Hkv) * d * eb, "d2h_bytes_per_step": T * H * d * eb,
+               "ms_per_step": ems / e2e_steps}
+
+    cpu = None
+    if rank == 0 and not args.no_cpu_baseline:
+        rate, times, threads, rows = oracle_rate(w, args.seed, rows_per_step=4, repeats=3, prefix=T - 4 * C)
+        cpu = {"value": tokens_per_s_from_pairs(w, rate), "unit": "tokens/s", "cores": threads, "kind": "oracle",
+               "sample": (f"{len(rows)} query rows x {H} heads of one chunk at prefix ~{T - 4 * C}, median of "
+                          f"{len(times)} repeats ({sum(times):.1f} s of CPU work), fp64 oracle; tokens/s "
+                          f"extrapolated linearly in visible (query,key) pairs over the chain")}
+
+    if rank == 0:
+        plan = cache.plan(C, T - C)
+        line = {
+            "metric": "fold-step tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
+            "data": "synthetic",
+            "config": {"workload": w.name, "tokens": T, "chunk": C, "fold_steps_per_step": N,
+                       "n_q_heads": H, "n_kv_heads": Hkv, "head_dim": d, "rope_base": w.rope_base,
+                       "sequences_per_gpu": 1, "l2": "inputs larger than L2 (cache grows to 512 MiB per chain)",
+                       "last_step_plan": {"tensor_core": plan[0], "splits": plan[1], "ctas": plan[2]}},
+            "attention_tflops": attn_flops * world * args.steps / (ms * 1e-3) / 1e12,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,188 @@
+/*
+ * kvfold.h - C ABI of the B200 (sm_100a) KV-Fold fold-step library.
+ *
+ * One `kvf_cache` is the accumulated K/V of ONE attention layer of ONE sequence:
+ * the accumulator of the paper's left fold (Section 2, "A recurrent view":
+ * (K,V)^(t) = F((K,V)^(t-1), x_t), started from the empty pair).  One call of
+ * kvf_fold_step is the attention part of one application of F at that layer.
+ *
+ * Conventions that hold for every entry point
+ *   - Device memory is never allocated or freed here.  The caller owns the cache
+ *     storage, the workspace, q/k/v/out and the stream; the library owns only the
+ *     host-side handle (and the TMA descriptors inside it).
+ *   - "device pointer" below means memory of the CUDA device that was current when
+ *     kvf_cache_create was called; the same device must be current at every later call.
+ *   - Calls are stream-ordered and asynchronous: they enqueue work on `cuda_stream`
+ *     (a cudaStream_t passed as void*, NULL = the default stream) and return.
+ *   - Errors are return codes.  A call that returns an error has enqueued nothing and has
+ *     changed neither the cache contents nor its length.  Nothing aborts or traps.
+ *   - A handle is not thread-safe; distinct handles are independent.  Several caches may
+ *     share one workspace if all of their calls go to the same stream.
+ *   - Results are deterministic: the same inputs, config and chunking give the same bits.
+ */
+#ifndef KVFOLD_H_
+#define KVFOLD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kvf_cache kvf_cache; /* opaque host-side handle */
+
+typedef enum {
+    KVF_OK = 0,
+    KVF_ERR_INVALID_ARG = 1, /* null / misaligned pointer, n_tokens < 1 or > max_chunk, bad config */
+    KVF_ERR_CAPACITY = 2,    /* len + n_tokens > capacity, or a buffer smaller than required     */
+    KVF_ERR_UNSUPPORTED = 3, /* head_dim / head ratio / dtype outside what the kernels cover     */
+    KVF_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed (see kvf_last_cuda_error)   */
+    KVF_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (read via kvf_cache_status)   */
+    KVF_ERR_POS = 6          /* KVF_STRICT_POS set and pos0 != current length                    */
+} kvf_status;
+
+typedef enum { KVF_BF16 = 0, KVF_F32 = 1 } kvf_dtype;
+
+enum {
+    KVF_ROPE_INTERLEAVED = 1u, /* rotate pairs (2j,2j+1) instead of (j, j+d/2)                   */
+    KVF_STRICT_POS = 2u,       /* reject pos0 != len (positions must continue across chunks)     */
+    KVF_OUT_F32 = 4u,          /* `out` is fp32 even when dtype is bf16                          */
+    KVF_FORCE_SIMT = 8u        /* use the CUDA-core attention kernel even where the tensor-core
+                                  kernel applies (bisecting aid; same results within tolerance) */
+};
+
+/*
+ * Shape and numerics of one cache.
+ *   n_q_heads (H), n_kv_heads (Hkv): grouped-query attention, query head h reads KV head
+ *       h / (H/Hkv); H % Hkv == 0 and H/Hkv a power of two <= 64.
+ *   head_dim (d): 64 or 128.
+ *   dtype: element type of q, k_new, v_new, of the cache planes and (unless KVF_OUT_F32) of out.
+ *       KVF_BF16: rotation, scores, softmax state and the output sum are fp32, probabilities
+ *       and the rotated q/k are rounded once to bf16.  KVF_F32: fp32 throughout (CUDA cores).
+ *   capacity: most tokens the cache will ever hold.
+ *   max_chunk: largest n_tokens of any later kvf_fold_step (sizes the workspace).
+ *   rope_base: theta = pos * rope_base^(-2j/d) (RoPE at continued absolute positions,
+ *       Section 2, "Position identifiers for the new tokens are continued ...").
+ *   softmax_scale: 0 means 1/sqrt(d).
+ *   inv_freq: optional HOST pointer to d/2 doubles replacing rope_base^(-2j/d)
+ *       (frequency-scaled RoPE variants); copied at create, may be freed afterwards.
+ */
+typedef struct kvf_config {
+    int32_t n_q_heads;
+    int32_t n_kv_heads;
+    int32_t head_dim;
+    int32_t dtype; /* kvf_dtype */
+    int64_t capacity;
+    int32_t max_chunk;
+    uint32_t flags;
+    double rope_base;
+    double softmax_scale;
+    const double *inv_freq;
+} kvf_config;
+
+/* Bytes of device storage one cache needs: K plane then V plane, each
+ * [n_kv_heads][capacity][head_dim] of dtype (head-major, one row = one token of one head;
+ * Section 5 gives the same count: KV heads x head_dim x (K,V) x bytes, per token).
+ * Returns 0 for an invalid config. */
+size_t kvf_cache_storage_bytes(const kvf_config *cfg);
+
+/* Bytes of device workspace: a status word, the rotated queries of one chunk, staging for
+ * kvf_fold_step_host, and the split partial results.  Returns 0 for an invalid config. */
+size_t kvf_workspace_bytes(const kvf_config *cfg);
+
+/*
+ * Create the empty accumulator (the (empty, empty) start of the fold, Section 2).
+ *   dev_storage   device pointer, 256-byte aligned, >= kvf_cache_storage_bytes(cfg); need not be
+ *                 initialised; the library writes only rows it appends (plus zeroed value rows up
+ *                 to the next multiple of 128 rows, which are not cache content).
+ *   dev_workspace device pointer, 256-byte aligned, >= kvf_workspace_bytes(cfg).
+ *   *out          receives the handle.
+ * Builds the TMA descriptors for the planes (driver entry point looked up at run time) and
+ * clears the device status word on the default stream.  Returns KVF_ERR_UNSUPPORTED for shapes
+ * outside the documented set, KVF_ERR_CAPACITY for short buffers, KVF_ERR_CUDA if no device.
+ */
+kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t storage_bytes,
+                            void *dev_workspace, size_t workspace_bytes, kvf_cache **out);
+
+/*
+ * One fold step at this layer (Section 2: queries from the new tokens, keys/values
+ * [K_0;...;K_t], positions continued from the chunk's absolute start; Figure "KV-Fold":
+ * the chunk's K/V are appended, the prefix is passed on unchanged).
+ *   q      device, [n_tokens][H][d]   dtype, contiguous, 16-byte aligned, before rotation
+ *   k_new  device, [n_tokens][Hkv][d] dtype, before rotation
+ *   v_new  device, [n_tokens][Hkv][d] dtype
+ *   pos0   absolute position of the chunk's first token (the fold passes pos0 = len); used
+ *          only for the rotation - visibility is by cache row
+ *   out    device, [n_tokens][H][d], dtype (or fp32 with KVF_OUT_F32): row i is the attention
+ *          output of token i over cache rows 0 .. len+i (all earlier chunks, then causal)
+ *   lse    device, [n_tokens][H] fp32 natural-log softmax denominators, or NULL
+ * Effects, in stream order: rotate q into the workspace; write rotated k and v as rows
+ * [len, len+n_tokens); attention; then the host-side length becomes len + n_tokens.
+ * Errors: INVALID_ARG, CAPACITY (cache full), POS, CUDA (launch failure; length unchanged).
+ */
+kvf_status kvf_fold_step(kvf_cache *c, const void *q, const void *k_new, const void *v_new,
+                         int32_t n_tokens, int64_t pos0, void *out, float *lse, void *cuda_stream);
+
+/*
+ * The same step with HOST buffers (pinned memory recommended): copies q/k/v to the workspace
+ * staging area, runs the step, copies `out` (and lse if not NULL) back, all on `cuda_stream`.
+ * The host buffers must stay valid until the stream reaches the end of the call.
+ */
+kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_host,
+                              const void *v_host, int32_t n_tokens, int64_t pos0, void *out_host,
+                              float *lse_host, void *cuda_stream);
+
+/* Tokens appended by all steps enqueued so far (host counter; after t steps of C tokens it is
+ * t*C without any synchronisation).  -1 for a null handle. */
+int64_t kvf_cache_len(const kvf_cache *c);
+
+/* Back to the empty accumulator (len = 0).  Storage is not cleared. */
+kvf_status kvf_cache_reset(kvf_cache *c);
+
+/* Reads the device status word (synchronises the default stream with a blocking copy): KVF_OK,
+ * or KVF_ERR_TIMEOUT if a bounded wait inside a kernel gave up.  Call after synchronising the
+ * streams that carried the steps. */
+kvf_status kvf_cache_status(kvf_cache *c);
+
+/* Device pointers of the planes, [n_kv_heads][capacity][head_dim] of dtype. */
+void *kvf_cache_k_plane(const kvf_cache *c);
+void *kvf_cache_v_plane(const kvf_cache *c);
+
+/*
+ * What a step of n_tokens on a prefix of prefix_len would launch:
+ *   plan[0] 1 = tensor-core (tcgen05) attention kernel, 0 = CUDA-core kernel
+ *   plan[1] number of splits over the key range (1 = none, no combine kernel)
+ *   plan[2] CTAs of the attention kernel
+ *   plan[3] kernels launched by the step
+ */
+kvf_status kvf_cache_plan(const kvf_cache *c, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]);
+
+/* Force the number of splits (0 = automatic).  Values the workspace cannot hold are clamped. */
+kvf_status kvf_cache_set_splits(kvf_cache *c, int32_t splits);
+
+/* Kernels launched through this handle since creation. */
+uint64_t kvf_cache_launch_count(const kvf_cache *c);
+
+/*
+ * Per-kernel timing.  With enable != 0 every step records CUDA events around each of its
+ * kernels on the step's stream.  kvf_cache_profile_read synchronises, then ADDS the elapsed
+ * milliseconds and launch counts since the last read to
+ *   ms[0]/launches[0] rotate+append, [1] attention, [2] split combine
+ * and forgets the recorded events.  At most 65536 launches are kept between reads.
+ */
+kvf_status kvf_cache_profile(kvf_cache *c, int32_t enable);
+kvf_status kvf_cache_profile_read(kvf_cache *c, double ms[3], uint64_t launches[3]);
+
+/* Frees the host handle (and its events); device memory stays with the caller. */
+void kvf_cache_destroy(kvf_cache *c);
+
+const char *kvf_status_str(kvf_status s);
+
+/* Text of the last CUDA error seen by this thread's calls into the library ("" if none). */
+const char *kvf_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVFOLD_H_ */

@@ -167,8 +167,10 @@ class OracleCache:
         rows_arr, rows_ptr, n_rows = None, None, 0
         if rows is not None:
             rows_arr = np.ascontiguousarray(np.asarray(rows, dtype=np.int32))
-            rows_ptr = rows_arr.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
             n_rows = rows_arr.shape[0]
+            if n_rows == 0:           # append only: keep the pointer non-null
+                rows_arr = np.zeros(1, dtype=np.int32)
+            rows_ptr = rows_arr.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
         n_out = n_rows if rows is not None else n
         out = np.empty((n_out, self.H, self.d), dtype=np.float64)
         lse = np.empty((n_out, self.H), dtype=np.float64)

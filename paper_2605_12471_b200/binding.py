@@ -1,0 +1,253 @@
+"""ctypes binding of include/kvfold.h: argument marshalling only.
+
+PyTorch appears here for device memory and streams; every step of the fold
+(rotation, append, attention, split merge) runs in the library's kernels.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkvfold.so")
+
+KVF_OK, KVF_ERR_INVALID_ARG, KVF_ERR_CAPACITY, KVF_ERR_UNSUPPORTED, KVF_ERR_CUDA, KVF_ERR_TIMEOUT, \
+    KVF_ERR_POS = range(7)
+KVF_BF16, KVF_F32 = 0, 1
+KVF_ROPE_INTERLEAVED, KVF_STRICT_POS, KVF_OUT_F32, KVF_FORCE_SIMT = 1, 2, 4, 8
+
+EXPORTS = [
+    "kvf_cache_storage_bytes", "kvf_workspace_bytes", "kvf_cache_create", "kvf_fold_step",
+    "kvf_fold_step_host", "kvf_cache_len", "kvf_cache_reset", "kvf_cache_status",
+    "kvf_cache_k_plane", "kvf_cache_v_plane", "kvf_cache_plan", "kvf_cache_set_splits",
+    "kvf_cache_launch_count", "kvf_cache_profile", "kvf_cache_profile_read", "kvf_cache_destroy",
+    "kvf_status_str", "kvf_last_cuda_error",
+]
+
+
+class kvf_config(ctypes.Structure):
+    _fields_ = [
+        ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+        ("dtype", ctypes.c_int32), ("capacity", ctypes.c_int64), ("max_chunk", ctypes.c_int32),
+        ("flags", ctypes.c_uint32), ("rope_base", ctypes.c_double), ("softmax_scale", ctypes.c_double),
+        ("inv_freq", ctypes.POINTER(ctypes.c_double)),
+    ]
+
+
+class KvfError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        lib = load()
+        msg = lib.kvf_status_str(code).decode()
+        if code == KVF_ERR_CUDA:
+            msg += ": " + lib.kvf_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg}")
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libkvfold.so; raises if the library has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2605_12471_b200.build` "
+                          "(or __graft_entry__.build()) first")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint64
+    cfgp = ctypes.POINTER(kvf_config)
+    lib.kvf_cache_storage_bytes.argtypes = [cfgp]
+    lib.kvf_cache_storage_bytes.restype = ctypes.c_size_t
+    lib.kvf_workspace_bytes.argtypes = [cfgp]
+    lib.kvf_workspace_bytes.restype = ctypes.c_size_t
+    lib.kvf_cache_create.argtypes = [cfgp, vp, ctypes.c_size_t, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
+    lib.kvf_cache_create.restype = ctypes.c_int
+    lib.kvf_fold_step.argtypes = [vp, vp, vp, vp, i32, i64, vp, vp, vp]
+    lib.kvf_fold_step.restype = ctypes.c_int
+    lib.kvf_fold_step_host.argtypes = [vp, vp, vp, vp, i32, i64, vp, vp, vp]
+    lib.kvf_fold_step_host.restype = ctypes.c_int
+    lib.kvf_cache_len.argtypes = [vp]
+    lib.kvf_cache_len.restype = i64
+    lib.kvf_cache_reset.argtypes = [vp]
+    lib.kvf_cache_reset.restype = ctypes.c_int
+    lib.kvf_cache_status.argtypes = [vp]
+    lib.kvf_cache_status.restype = ctypes.c_int
+    lib.kvf_cache_k_plane.argtypes = [vp]
+    lib.kvf_cache_k_plane.restype = vp
+    lib.kvf_cache_v_plane.argtypes = [vp]
+    lib.kvf_cache_v_plane.restype = vp
+    lib.kvf_cache_plan.argtypes = [vp, i32, i64, ctypes.POINTER(i32)]
+    lib.kvf_cache_plan.restype = ctypes.c_int
+    lib.kvf_cache_set_splits.argtypes = [vp, i32]
+    lib.kvf_cache_set_splits.restype = ctypes.c_int
+    lib.kvf_cache_launch_count.argtypes = [vp]
+    lib.kvf_cache_launch_count.restype = u64
+    lib.kvf_cache_profile.argtypes = [vp, i32]
+    lib.kvf_cache_profile.restype = ctypes.c_int
+    lib.kvf_cache_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(u64)]
+    lib.kvf_cache_profile_read.restype = ctypes.c_int
+    lib.kvf_cache_destroy.argtypes = [vp]
+    lib.kvf_cache_destroy.restype = None
+    lib.kvf_status_str.argtypes = [ctypes.c_int]
+    lib.kvf_status_str.restype = ctypes.c_char_p
+    lib.kvf_last_cuda_error.argtypes = []
+    lib.kvf_last_cuda_error.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def make_config(n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: str | int, capacity: int,
+                max_chunk: int, rope_base: float = 10000.0, softmax_scale: float = 0.0, flags: int = 0,
+                inv_freq=None) -> kvf_config:
+    cfg = kvf_config()
+    cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = n_q_heads, n_kv_heads, head_dim
+    cfg.dtype = {"bf16": KVF_BF16, "f32": KVF_F32}.get(dtype, dtype)
+    cfg.capacity, cfg.max_chunk, cfg.flags = capacity, max_chunk, flags
+    cfg.rope_base, cfg.softmax_scale = rope_base, softmax_scale
+    if inv_freq is not None:
+        arr = (ctypes.c_double * (head_dim // 2))(*[float(x) for x in inv_freq])
+        cfg._keepalive = arr
+        cfg.inv_freq = ctypes.cast(arr, ctypes.POINTER(ctypes.c_double))
+    return cfg
+
+
+def cache_storage_bytes(cfg: kvf_config) -> int:
+    return int(load().kvf_cache_storage_bytes(ctypes.byref(cfg)))
+
+
+def workspace_bytes(cfg: kvf_config) -> int:
+    return int(load().kvf_workspace_bytes(ctypes.byref(cfg)))
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+class Cache:
+    """One layer's accumulated K/V on the current CUDA device (kvf_cache_* calls)."""
+
+    def __init__(self, cfg: kvf_config, device: str | torch.device = "cuda", workspace: torch.Tensor | None = None):
+        lib = load()
+        self.cfg = cfg
+        self.device = torch.device(device)
+        sb, wb = cache_storage_bytes(cfg), workspace_bytes(cfg)
+        if sb == 0 or wb == 0:
+            # let the library name the reason
+            h = ctypes.c_void_p()
+            rc = lib.kvf_cache_create(ctypes.byref(cfg), None, 0, None, 0, ctypes.byref(h))
+            raise KvfError(rc if rc else KVF_ERR_INVALID_ARG, "kvf_cache_create")
+        self.storage = torch.empty(sb, dtype=torch.uint8, device=self.device)
+        self.workspace = workspace if workspace is not None else torch.empty(wb, dtype=torch.uint8, device=self.device)
+        h = ctypes.c_void_p()
+        with torch.cuda.device(self.device):
+            rc = lib.kvf_cache_create(ctypes.byref(cfg), self.storage.data_ptr(), sb,
+                                      self.workspace.data_ptr(), self.workspace.numel(), ctypes.byref(h))
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_cache_create")
+        self._h = h
+        self.torch_dtype = torch.bfloat16 if cfg.dtype == KVF_BF16 else torch.float32
+        self.out_dtype = torch.float32 if (cfg.flags & KVF_OUT_F32) else self.torch_dtype
+
+    def close(self):
+        if getattr(self, "_h", None):
+            load().kvf_cache_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def __len__(self) -> int:
+        return int(load().kvf_cache_len(self._h))
+
+    def reset(self):
+        rc = load().kvf_cache_reset(self._h)
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_cache_reset")
+
+    def fold_step(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                  pos0: Optional[int] = None, out: Optional[torch.Tensor] = None,
+                  lse: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """kvf_fold_step on device tensors; returns the chunk's attention output."""
+        n = q.shape[0]
+        for t in (q, k_new, v_new):
+            assert t.is_cuda and t.is_contiguous() and t.dtype == self.torch_dtype
+        if out is None:
+            out = torch.empty((n, self.cfg.n_q_heads, self.cfg.head_dim), dtype=self.out_dtype, device=q.device)
+        if pos0 is None:
+            pos0 = len(self)
+        rc = load().kvf_fold_step(self._h, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), n, int(pos0),
+                                  out.data_ptr(), lse.data_ptr() if lse is not None else None,
+                                  _stream_ptr(stream))
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_fold_step")
+        return out
+
+    def fold_step_host(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, out: torch.Tensor,
+                       pos0: Optional[int] = None, lse: Optional[torch.Tensor] = None,
+                       stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """kvf_fold_step_host on (pinned) host tensors; copies run on the stream."""
+        n = q.shape[0]
+        for t in (q, k_new, v_new, out):
+            assert not t.is_cuda and t.is_contiguous()
+        if pos0 is None:
+            pos0 = len(self)
+        rc = load().kvf_fold_step_host(self._h, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), n, int(pos0),
+                                       out.data_ptr(), lse.data_ptr() if lse is not None else None,
+                                       _stream_ptr(stream))
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_fold_step_host")
+        return out
+
+    def status(self) -> int:
+        return int(load().kvf_cache_status(self._h))
+
+    def _plane(self, ptr: int) -> torch.Tensor:
+        plane_bytes = self.storage.numel() // 2
+        off = ptr - self.storage.data_ptr()
+        flat = self.storage[off:off + plane_bytes].view(self.torch_dtype)
+        return flat.view(self.cfg.n_kv_heads, self.cfg.capacity, self.cfg.head_dim)
+
+    def k_plane(self) -> torch.Tensor:
+        """[Hkv, capacity, d] view of the rotated keys (rows >= len are not content)."""
+        return self._plane(load().kvf_cache_k_plane(self._h))
+
+    def v_plane(self) -> torch.Tensor:
+        return self._plane(load().kvf_cache_v_plane(self._h))
+
+    def plan(self, n_tokens: int, prefix_len: Optional[int] = None) -> Tuple[int, int, int, int]:
+        arr = (ctypes.c_int32 * 4)()
+        rc = load().kvf_cache_plan(self._h, n_tokens, len(self) if prefix_len is None else prefix_len, arr)
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_cache_plan")
+        return tuple(arr)
+
+    def set_splits(self, splits: int):
+        rc = load().kvf_cache_set_splits(self._h, splits)
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_cache_set_splits")
+
+    def launch_count(self) -> int:
+        return int(load().kvf_cache_launch_count(self._h))
+
+    def profile(self, enable: bool):
+        load().kvf_cache_profile(self._h, int(enable))
+
+    def profile_read(self):
+        ms = (ctypes.c_double * 3)()
+        cnt = (ctypes.c_uint64 * 3)()
+        rc = load().kvf_cache_profile_read(self._h, ms, cnt)
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_cache_profile_read")
+        return list(ms), list(cnt)
+
+
+def cache_for(w, capacity: Optional[int] = None, max_chunk: Optional[int] = None, flags: int = 0,
+              device: str | torch.device = "cuda", workspace: torch.Tensor | None = None) -> Cache:
+    """A cache shaped for a workloads.Workload."""
+    cfg = make_config(w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, capacity or w.tokens,
+                      max_chunk or w.chunk, rope_base=w.rope_base, flags=flags)
+    return Cache(cfg, device=device, workspace=workspace)

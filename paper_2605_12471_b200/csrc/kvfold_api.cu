@@ -1,0 +1,478 @@
+// Host layer of the C ABI declared in include/kvfold.h: handle, validation, workspace carving,
+// TMA descriptor creation, launch planning.  Every step of the fold runs in the kernels this file
+// launches; there is no CPU fallback.
+#include "../../include/kvfold.h"
+#include "kvfold_internal.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace kvf;
+
+namespace {
+
+thread_local char g_cuda_err[256] = "";
+
+kvf_status cuda_fail(cudaError_t e, const char *what) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+    return KVF_ERR_CUDA;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+size_t elem_bytes(int dtype) { return dtype == KVF_BF16 ? 2 : 4; }
+
+bool pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
+kvf_status check_config(const kvf_config *c) {
+    if (!c) return KVF_ERR_INVALID_ARG;
+    if (c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->capacity <= 0 || c->max_chunk <= 0)
+        return KVF_ERR_INVALID_ARG;
+    if (c->n_q_heads % c->n_kv_heads != 0) return KVF_ERR_INVALID_ARG;
+    if (c->dtype != KVF_BF16 && c->dtype != KVF_F32) return KVF_ERR_UNSUPPORTED;
+    if (c->head_dim != 64 && c->head_dim != 128) return KVF_ERR_UNSUPPORTED;
+    int G = c->n_q_heads / c->n_kv_heads;
+    if (!pow2(G) || G > 64) return KVF_ERR_UNSUPPORTED;
+    if (c->rope_base <= 0.0 && !c->inv_freq) return KVF_ERR_INVALID_ARG;
+    if (c->softmax_scale < 0.0) return KVF_ERR_INVALID_ARG;
+    if ((int64_t)c->max_chunk > c->capacity) return KVF_ERR_INVALID_ARG;
+    if (c->capacity > (int64_t)1 << 31) return KVF_ERR_UNSUPPORTED;
+    return KVF_OK;
+}
+
+struct Layout {
+    size_t status, q_rot, st_q, st_k, st_v, st_out, st_lse, part_o, part_lse, total;
+};
+
+Layout workspace_layout(const kvf_config *c) {
+    Layout l;
+    const size_t eb = elem_bytes(c->dtype);
+    const size_t qb = (size_t)c->max_chunk * c->n_q_heads * c->head_dim * eb;
+    const size_t kb = (size_t)c->max_chunk * c->n_kv_heads * c->head_dim * eb;
+    const size_t ob = (size_t)c->max_chunk * c->n_q_heads * c->head_dim *
+                      ((c->flags & KVF_OUT_F32) ? 4 : eb);
+    size_t off = 0;
+    l.status = off;   off = align_up(off + 256, 1024);
+    l.q_rot = off;    off = align_up(off + qb, 1024);
+    l.st_q = off;     off = align_up(off + qb, 1024);
+    l.st_k = off;     off = align_up(off + kb, 1024);
+    l.st_v = off;     off = align_up(off + kb, 1024);
+    l.st_out = off;   off = align_up(off + ob, 1024);
+    l.st_lse = off;   off = align_up(off + (size_t)c->max_chunk * c->n_q_heads * 4, 1024);
+    l.part_o = off;   off = align_up(off + (size_t)kPartTokens * c->n_q_heads * c->head_dim * 4, 1024);
+    l.part_lse = off; off = align_up(off + (size_t)kPartTokens * c->n_q_heads * 4, 1024);
+    l.total = off;
+    return l;
+}
+
+struct ProfRec {
+    cudaEvent_t a, b;
+    int kind;
+};
+
+}  // namespace
+
+struct kvf_cache {
+    kvf_config cfg;
+    RopeTable table;
+    int device;
+    int sm_count;
+    char *storage;
+    char *workspace;
+    size_t plane_bytes;
+    Layout lay;
+    int64_t len;
+    int G;
+    float scale_log2;
+    bool tc;
+    TcMaps maps;
+    int force_splits;
+    uint64_t launches;
+    bool profile;
+    std::vector<ProfRec> recs;
+    std::vector<cudaEvent_t> pool;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+// 3-D bf16 tensor map (x = head_dim, y, z) with a 64-element (128-byte) swizzled inner box.
+kvf_status make_map(EncodeTiledFn fn, CUtensorMap *m, void *base, uint64_t dim_y, uint64_t dim_z,
+                    uint64_t stride_y_bytes, uint64_t stride_z_bytes, int d, uint32_t box_y, uint32_t box_z) {
+    cuuint64_t dims[3] = {(cuuint64_t)d, dim_y, dim_z};
+    cuuint64_t strides[2] = {stride_y_bytes, stride_z_bytes};
+    cuuint32_t box[3] = {64u, box_y, box_z};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return KVF_ERR_CUDA;
+    }
+    return KVF_OK;
+}
+
+kvf_status build_maps(kvf_cache *c) {
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDriverEntryPoint");
+    if (qres != cudaDriverEntryPointSuccess || !sym) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "driver has no cuTensorMapEncodeTiled");
+        return KVF_ERR_CUDA;
+    }
+    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(sym);
+    const kvf_config &f = c->cfg;
+    const int d = f.head_dim;
+    const uint64_t row = (uint64_t)d * 2;
+    // rotated queries [max_chunk][H][d]: one box = (128/G tokens) x (G heads of one KV head) x 64
+    kvf_status s = make_map(fn, &c->maps.q, c->workspace + c->lay.q_rot, (uint64_t)f.n_q_heads,
+                            (uint64_t)f.max_chunk, row, row * f.n_q_heads, d, (uint32_t)c->G,
+                            (uint32_t)(128 / c->G));
+    if (s != KVF_OK) return s;
+    // planes [Hkv][capacity][d]: one box = 128 rows of one head x 64
+    s = make_map(fn, &c->maps.k, c->storage, (uint64_t)f.capacity, (uint64_t)f.n_kv_heads, row,
+                 row * f.capacity, d, (uint32_t)kKvTile, 1u);
+    if (s != KVF_OK) return s;
+    return make_map(fn, &c->maps.v, c->storage + c->plane_bytes, (uint64_t)f.capacity,
+                    (uint64_t)f.n_kv_heads, row, row * f.capacity, d, (uint32_t)kKvTile, 1u);
+}
+
+struct Plan {
+    bool tc;
+    int splits, ctas, kernels;
+};
+
+Plan make_plan(const kvf_cache *c, int n, int64_t prefix) {
+    Plan p;
+    p.tc = c->tc;
+    const int64_t L = prefix + n;
+    const int key_tile = p.tc ? kKvTile : 64;
+    const int64_t nt = (L + key_tile - 1) / key_tile;
+    const int units = p.tc ? attn_tc_ctas(n, c->G, c->cfg.n_kv_heads, 1)
+                           : attn_simt_ctas(n, c->G, c->cfg.n_kv_heads, 1);
+    const int per_sm = p.tc ? 1 : 2;
+    const int target = c->sm_count * per_sm;
+    int max_splits = kPartTokens / n;
+    if (max_splits > kMaxSplits) max_splits = kMaxSplits;
+    if (max_splits < 1) max_splits = 1;
+    int splits = 1;
+    if (c->force_splits > 0) {
+        splits = c->force_splits;
+    } else if (units < target) {
+        // fill whole waves of the machine, but keep at least 4 key tiles per split
+        int want = (target + units - 1) / units;
+        if (!p.tc) want = (2 * target + units - 1) / units;
+        int64_t cap = nt / 4;
+        if (want > cap) want = (int)cap;
+        splits = want;
+    }
+    if (splits > max_splits) splits = max_splits;
+    if ((int64_t)splits > nt) splits = (int)nt;
+    if (splits < 1) splits = 1;
+    p.splits = splits;
+    p.ctas = units * splits;
+    p.kernels = 2 + (splits > 1 ? 1 : 0);
+    return p;
+}
+
+cudaEvent_t get_event(kvf_cache *c) {
+    if (!c->pool.empty()) {
+        cudaEvent_t e = c->pool.back();
+        c->pool.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+struct ProfScope {
+    kvf_cache *c;
+    cudaStream_t s;
+    ProfRec r;
+    bool on;
+    ProfScope(kvf_cache *c_, cudaStream_t s_, int kind) : c(c_), s(s_), on(false) {
+        if (c->profile && c->recs.size() < 65536) {
+            r.a = get_event(c);
+            r.b = get_event(c);
+            r.kind = kind;
+            on = r.a && r.b;
+            if (on) cudaEventRecord(r.a, s);
+        }
+    }
+    ~ProfScope() {
+        if (on) {
+            cudaEventRecord(r.b, s);
+            c->recs.push_back(r);
+        }
+    }
+};
+
+kvf_status check_ptr(const void *p) {
+    if (!p) return KVF_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(p) & 15u) return KVF_ERR_INVALID_ARG;
+    return KVF_OK;
+}
+
+kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void *v_new, int32_t n,
+                     int64_t pos0, void *out, float *lse, cudaStream_t st) {
+    const kvf_config &f = c->cfg;
+    const int64_t P = c->len;
+    const Plan plan = make_plan(c, n, P);
+
+    RopeAppendArgs ra;
+    ra.q = q; ra.k_new = k_new; ra.v_new = v_new;
+    ra.q_rot = c->workspace + c->lay.q_rot;
+    ra.k_plane = c->storage;
+    ra.v_plane = c->storage + c->plane_bytes;
+    ra.capacity = f.capacity; ra.prefix = P; ra.pos0 = pos0;
+    ra.n = n; ra.H = f.n_q_heads; ra.Hkv = f.n_kv_heads; ra.d = f.head_dim;
+    {
+        int64_t L = P + n;
+        int64_t pad_end = (L + kKvTile - 1) / kKvTile * kKvTile;
+        if (pad_end > f.capacity) pad_end = f.capacity;
+        ra.zero_rows = (int32_t)(pad_end - L);
+    }
+    ra.table = c->table;
+
+    AttnArgs aa;
+    aa.q_rot = ra.q_rot;
+    aa.k_plane = ra.k_plane; aa.v_plane = ra.v_plane;
+    aa.out = out; aa.lse = lse;
+    aa.part_o = reinterpret_cast<float *>(c->workspace + c->lay.part_o);
+    aa.part_lse = reinterpret_cast<float *>(c->workspace + c->lay.part_lse);
+    aa.status = reinterpret_cast<int *>(c->workspace + c->lay.status);
+    aa.capacity = f.capacity; aa.prefix = P;
+    aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
+    aa.splits = plan.splits;
+    aa.out_f32 = (f.dtype == KVF_F32 || (f.flags & KVF_OUT_F32)) ? 1 : 0;
+    aa.scale_log2 = c->scale_log2;
+
+    cudaError_t e;
+    {
+        ProfScope ps(c, st, 0);
+        e = launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, st);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "rope_append launch");
+    c->launches++;
+    {
+        ProfScope ps(c, st, 1);
+        if (plan.tc) e = launch_attn_tc(aa, c->maps, st);
+        else e = launch_attn_simt(aa, f.dtype, st, nullptr);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "attention launch");
+    c->launches++;
+    if (plan.splits > 1) {
+        {
+            ProfScope ps(c, st, 2);
+            e = launch_combine(aa, f.dtype, st);
+        }
+        if (e != cudaSuccess) return cuda_fail(e, "combine launch");
+        c->launches++;
+    }
+    c->len = P + n;
+    return KVF_OK;
+}
+
+kvf_status check_step(kvf_cache *c, int32_t n, int64_t pos0) {
+    if (!c) return KVF_ERR_INVALID_ARG;
+    if (n < 1 || n > c->cfg.max_chunk) return KVF_ERR_INVALID_ARG;
+    if (pos0 < 0) return KVF_ERR_INVALID_ARG;
+    if (c->len + n > c->cfg.capacity) return KVF_ERR_CAPACITY;
+    if ((c->cfg.flags & KVF_STRICT_POS) && pos0 != c->len) return KVF_ERR_POS;
+    return KVF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t kvf_cache_storage_bytes(const kvf_config *cfg) {
+    if (check_config(cfg) != KVF_OK) return 0;
+    return 2 * (size_t)cfg->n_kv_heads * (size_t)cfg->capacity * (size_t)cfg->head_dim * elem_bytes(cfg->dtype);
+}
+
+size_t kvf_workspace_bytes(const kvf_config *cfg) {
+    if (check_config(cfg) != KVF_OK) return 0;
+    return workspace_layout(cfg).total;
+}
+
+kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t storage_bytes,
+                            void *dev_workspace, size_t workspace_bytes, kvf_cache **out) {
+    if (!out) return KVF_ERR_INVALID_ARG;
+    *out = nullptr;
+    kvf_status s = check_config(cfg);
+    if (s != KVF_OK) return s;
+    if (!dev_storage || !dev_workspace) return KVF_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(dev_storage) & 255u) || (reinterpret_cast<uintptr_t>(dev_workspace) & 255u))
+        return KVF_ERR_INVALID_ARG;
+    if (storage_bytes < kvf_cache_storage_bytes(cfg)) return KVF_ERR_CAPACITY;
+    if (workspace_bytes < kvf_workspace_bytes(cfg)) return KVF_ERR_CAPACITY;
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+
+    kvf_cache *c = new (std::nothrow) kvf_cache();
+    if (!c) return KVF_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->cfg.inv_freq = nullptr;
+    c->device = dev;
+    c->sm_count = sms;
+    c->storage = static_cast<char *>(dev_storage);
+    c->workspace = static_cast<char *>(dev_workspace);
+    c->plane_bytes = kvf_cache_storage_bytes(cfg) / 2;
+    c->lay = workspace_layout(cfg);
+    c->len = 0;
+    c->G = cfg->n_q_heads / cfg->n_kv_heads;
+    const double scale = cfg->softmax_scale > 0.0 ? cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
+    c->scale_log2 = (float)(scale * 1.4426950408889634);
+    for (int j = 0; j < cfg->head_dim / 2; ++j)
+        c->table.inv_freq[j] = cfg->inv_freq ? cfg->inv_freq[j]
+                                             : std::pow(cfg->rope_base, -2.0 * (double)j / (double)cfg->head_dim);
+    for (int j = cfg->head_dim / 2; j < kMaxHalfDim; ++j) c->table.inv_freq[j] = 0.0;
+    c->force_splits = 0;
+    c->launches = 0;
+    c->profile = false;
+    c->tc = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, c->G);
+    if (c->tc) {
+        s = build_maps(c);
+        if (s != KVF_OK) { delete c; return s; }
+    }
+    e = cudaMemset(c->workspace + c->lay.status, 0, 256);
+    if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaMemset(status)"); }
+    *out = c;
+    return KVF_OK;
+}
+
+kvf_status kvf_fold_step(kvf_cache *c, const void *q, const void *k_new, const void *v_new,
+                         int32_t n_tokens, int64_t pos0, void *out, float *lse, void *cuda_stream) {
+    kvf_status s = check_step(c, n_tokens, pos0);
+    if (s != KVF_OK) return s;
+    if (check_ptr(q) || check_ptr(k_new) || check_ptr(v_new) || check_ptr(out)) return KVF_ERR_INVALID_ARG;
+    if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return KVF_ERR_INVALID_ARG;
+    return step_impl(c, q, k_new, v_new, n_tokens, pos0, out, lse, static_cast<cudaStream_t>(cuda_stream));
+}
+
+kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_host, const void *v_host,
+                              int32_t n_tokens, int64_t pos0, void *out_host, float *lse_host,
+                              void *cuda_stream) {
+    kvf_status s = check_step(c, n_tokens, pos0);
+    if (s != KVF_OK) return s;
+    if (!q_host || !k_host || !v_host || !out_host) return KVF_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const kvf_config &f = c->cfg;
+    const size_t eb = elem_bytes(f.dtype);
+    const size_t qb = (size_t)n_tokens * f.n_q_heads * f.head_dim * eb;
+    const size_t kb = (size_t)n_tokens * f.n_kv_heads * f.head_dim * eb;
+    const size_t ob = (size_t)n_tokens * f.n_q_heads * f.head_dim * ((f.flags & KVF_OUT_F32) ? 4 : eb);
+    char *w = c->workspace;
+    cudaError_t e = cudaMemcpyAsync(w + c->lay.st_q, q_host, qb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(w + c->lay.st_k, k_host, kb, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(w + c->lay.st_v, v_host, kb, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e, "host-to-device copy");
+    float *lse_dev = lse_host ? reinterpret_cast<float *>(w + c->lay.st_lse) : nullptr;
+    s = step_impl(c, w + c->lay.st_q, w + c->lay.st_k, w + c->lay.st_v, n_tokens, pos0, w + c->lay.st_out,
+                  lse_dev, st);
+    if (s != KVF_OK) return s;
+    e = cudaMemcpyAsync(out_host, w + c->lay.st_out, ob, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && lse_host)
+        e = cudaMemcpyAsync(lse_host, lse_dev, (size_t)n_tokens * f.n_q_heads * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "device-to-host copy");
+    return KVF_OK;
+}
+
+int64_t kvf_cache_len(const kvf_cache *c) { return c ? c->len : -1; }
+
+kvf_status kvf_cache_reset(kvf_cache *c) {
+    if (!c) return KVF_ERR_INVALID_ARG;
+    c->len = 0;
+    return KVF_OK;
+}
+
+kvf_status kvf_cache_status(kvf_cache *c) {
+    if (!c) return KVF_ERR_INVALID_ARG;
+    int word = 0;
+    cudaError_t e = cudaMemcpy(&word, c->workspace + c->lay.status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
+    return word == 0 ? KVF_OK : KVF_ERR_TIMEOUT;
+}
+
+void *kvf_cache_k_plane(const kvf_cache *c) { return c ? c->storage : nullptr; }
+void *kvf_cache_v_plane(const kvf_cache *c) { return c ? c->storage + c->plane_bytes : nullptr; }
+
+kvf_status kvf_cache_plan(const kvf_cache *c, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]) {
+    if (!c || !plan || n_tokens < 1 || n_tokens > c->cfg.max_chunk || prefix_len < 0) return KVF_ERR_INVALID_ARG;
+    Plan p = make_plan(c, n_tokens, prefix_len);
+    plan[0] = p.tc ? 1 : 0;
+    plan[1] = p.splits;
+    plan[2] = p.ctas;
+    plan[3] = p.kernels;
+    return KVF_OK;
+}
+
+kvf_status kvf_cache_set_splits(kvf_cache *c, int32_t splits) {
+    if (!c || splits < 0) return KVF_ERR_INVALID_ARG;
+    c->force_splits = splits;
+    return KVF_OK;
+}
+
+uint64_t kvf_cache_launch_count(const kvf_cache *c) { return c ? c->launches : 0; }
+
+kvf_status kvf_cache_profile(kvf_cache *c, int32_t enable) {
+    if (!c) return KVF_ERR_INVALID_ARG;
+    c->profile = enable != 0;
+    return KVF_OK;
+}
+
+kvf_status kvf_cache_profile_read(kvf_cache *c, double ms[3], uint64_t launches[3]) {
+    if (!c || !ms || !launches) return KVF_ERR_INVALID_ARG;
+    kvf_status rc = KVF_OK;
+    for (ProfRec &r : c->recs) {
+        cudaError_t e = cudaEventSynchronize(r.b);
+        float t = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&t, r.a, r.b);
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaEventElapsedTime");
+        else if (r.kind >= 0 && r.kind < 3) { ms[r.kind] += t; launches[r.kind] += 1; }
+        c->pool.push_back(r.a);
+        c->pool.push_back(r.b);
+    }
+    c->recs.clear();
+    return rc;
+}
+
+void kvf_cache_destroy(kvf_cache *c) {
+    if (!c) return;
+    for (ProfRec &r : c->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (cudaEvent_t e : c->pool) cudaEventDestroy(e);
+    delete c;
+}
+
+const char *kvf_status_str(kvf_status s) {
+    switch (s) {
+        case KVF_OK: return "KVF_OK";
+        case KVF_ERR_INVALID_ARG: return "KVF_ERR_INVALID_ARG";
+        case KVF_ERR_CAPACITY: return "KVF_ERR_CAPACITY";
+        case KVF_ERR_UNSUPPORTED: return "KVF_ERR_UNSUPPORTED";
+        case KVF_ERR_CUDA: return "KVF_ERR_CUDA";
+        case KVF_ERR_TIMEOUT: return "KVF_ERR_TIMEOUT";
+        case KVF_ERR_POS: return "KVF_ERR_POS";
+    }
+    return "KVF_ERR_UNKNOWN";
+}
+
+const char *kvf_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"

@@ -1,0 +1,59 @@
+// Internal declarations shared by the host layer and the kernel launchers.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace kvf {
+
+constexpr int kMaxHalfDim = 64;       // head_dim <= 128
+constexpr int kKvTile = 128;          // key rows per tensor-core tile; V rows are zero-padded to it
+constexpr int kPartTokens = 4096;     // split partials are sized for (splits * n_tokens) <= this
+constexpr int kMaxSplits = 64;
+
+struct RopeTable {
+    double inv_freq[kMaxHalfDim];
+};
+
+// Arguments of the fused rotate + append kernel (one launch per step).
+struct RopeAppendArgs {
+    const void *q, *k_new, *v_new;   // [n][H][d], [n][Hkv][d], [n][Hkv][d]
+    void *q_rot;                     // [n][H][d]
+    void *k_plane, *v_plane;         // [Hkv][capacity][d]
+    int64_t capacity, prefix, pos0;  // prefix = rows already held
+    int32_t n, H, Hkv, d;
+    int32_t zero_rows;               // value rows [prefix+n, prefix+n+zero_rows) are cleared
+    RopeTable table;
+};
+
+// Arguments shared by the attention kernels and the combine kernel.
+struct AttnArgs {
+    const void *q_rot;               // [n][H][d]
+    const void *k_plane, *v_plane;   // [Hkv][capacity][d]
+    void *out;                       // [n][H][d], dtype or fp32
+    float *lse;                      // [n][H] or null (natural log)
+    float *part_o;                   // [splits][n][H][d] fp32, normalised per split
+    float *part_lse;                 // [splits][n][H] fp32, log2 domain; -inf = split saw no key
+    int *status;                     // device status word
+    int64_t capacity, prefix;
+    int32_t n, H, Hkv, G, d;
+    int32_t splits;
+    int32_t out_f32;
+    float scale_log2;                // softmax scale * log2(e)
+};
+
+cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interleaved, cudaStream_t s);
+cudaError_t launch_attn_simt(const AttnArgs &a, int dtype, cudaStream_t s, int *grid_out);
+cudaError_t launch_combine(const AttnArgs &a, int dtype, cudaStream_t s);
+int attn_simt_ctas(int n, int G, int Hkv, int splits);
+
+// Tensor-core path (bf16, head_dim 128).
+struct TcMaps {
+    CUtensorMap q, k, v;
+};
+bool attn_tc_supported(int dtype, int d, int G);
+int attn_tc_ctas(int n, int G, int Hkv, int splits);
+cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s);
+
+}  // namespace kvf

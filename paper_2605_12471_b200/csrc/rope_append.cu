@@ -1,0 +1,196 @@
+// Fused RoPE(q), RoPE(k) + append(k, v) for one chunk.
+//
+// Section 2 of the paper: the new tokens' position identifiers continue from the chunk's
+// absolute start, so the rotations line up with the original sequence; Figure "KV-Fold": the
+// chunk's K/V are appended to the cache and earlier rows are left as they are.
+//
+// Numerics (the cache bits are a contract): theta = pos * inv_freq[j] in fp64, cos/sin in fp64,
+// each rounded once to fp32; then per output two fp32 operations,
+//     lo' = fma(x_lo, c, -(x_hi * s))      hi' = fma(x_hi, c, x_lo * s)
+// with the cross product rounded first, and one round-to-nearest-even to the cache dtype.
+// Values are copied verbatim.  All global accesses are 16-byte vectors.
+#include "kvfold_internal.h"
+
+namespace kvf {
+namespace {
+
+constexpr int kTok = 4;        // tokens per CTA
+constexpr int kThreads = 256;
+
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void load(const float *p, float (&x)[4]) {
+        float4 v = *reinterpret_cast<const float4 *>(p);
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    }
+    static __device__ __forceinline__ void store(float *p, const float (&x)[4]) {
+        *reinterpret_cast<float4 *>(p) = make_float4(x[0], x[1], x[2], x[3]);
+    }
+};
+template <> struct Vec16<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&x)[8]) {
+        uint4 v = *reinterpret_cast<const uint4 *>(p);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            x[2 * i] = __uint_as_float(w[i] << 16);
+            x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16 *p, const float (&x)[8]) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t lo = __bfloat16_as_ushort(__float2bfloat16_rn(x[2 * i]));
+            uint32_t hi = __bfloat16_as_ushort(__float2bfloat16_rn(x[2 * i + 1]));
+            w[i] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4 *>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+__device__ __forceinline__ void rotate(float a, float b, float c, float s, float &ra, float &rb) {
+    float cross_a = __fmul_rn(b, s);
+    float cross_b = __fmul_rn(a, s);
+    ra = __fmaf_rn(a, c, -cross_a);
+    rb = __fmaf_rn(b, c, cross_b);
+}
+
+template <typename T, bool INTERLEAVED>
+__global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendArgs a) {
+    constexpr int VEC = Vec16<T>::N;
+    __shared__ float2 cs[kTok][kMaxHalfDim];   // (cos, sin) per (token, pair)
+
+    const int d = a.d, half = d / 2;
+    const int n_tok_blocks = (a.n + kTok - 1) / kTok;
+
+    if ((int)blockIdx.x >= n_tok_blocks) {
+        // Clear value rows between the new end of the cache and the next key-tile boundary,
+        // so that a zero probability never multiplies stale non-finite bits.
+        const int vec_per_row = d / VEC;
+        const int64_t total = (int64_t)a.zero_rows * a.Hkv * vec_per_row;
+        const int64_t start = ((int64_t)blockIdx.x - n_tok_blocks) * kThreads + threadIdx.x;
+        const int64_t stride = (int64_t)(gridDim.x - n_tok_blocks) * kThreads;
+        T *vp = reinterpret_cast<T *>(a.v_plane);
+        for (int64_t i = start; i < total; i += stride) {
+            int c = (int)(i % vec_per_row);
+            int64_t t = i / vec_per_row;
+            int g = (int)(t % a.Hkv);
+            int64_t row = a.prefix + a.n + t / a.Hkv;
+            *reinterpret_cast<uint4 *>(vp + ((int64_t)g * a.capacity + row) * d + c * VEC) =
+                make_uint4(0, 0, 0, 0);
+        }
+        return;
+    }
+
+    const int tok0 = blockIdx.x * kTok;
+    const int ntok = min(kTok, a.n - tok0);
+
+    for (int idx = threadIdx.x; idx < ntok * half; idx += kThreads) {
+        int t = idx / half, j = idx % half;
+        double theta = (double)(a.pos0 + tok0 + t) * a.table.inv_freq[j];
+        double sn, cn;
+        sincos(theta, &sn, &cn);
+        cs[t][j] = make_float2((float)cn, (float)sn);
+    }
+    __syncthreads();
+
+    const T *q = reinterpret_cast<const T *>(a.q);
+    const T *k = reinterpret_cast<const T *>(a.k_new);
+    const T *v = reinterpret_cast<const T *>(a.v_new);
+    T *qr = reinterpret_cast<T *>(a.q_rot);
+    T *kp = reinterpret_cast<T *>(a.k_plane);
+    T *vp = reinterpret_cast<T *>(a.v_plane);
+    const int heads = a.H + a.Hkv;
+
+    if (!INTERLEAVED) {
+        const int chunks = half / VEC;                 // vectors per half row
+        const int items = ntok * heads * chunks;
+        for (int idx = threadIdx.x; idx < items; idx += kThreads) {
+            int c = idx % chunks;
+            int hh = (idx / chunks) % heads;
+            int t = idx / (chunks * heads);
+            const T *src;
+            T *dst;
+            if (hh < a.H) {
+                src = q + ((int64_t)(tok0 + t) * a.H + hh) * d;
+                dst = qr + ((int64_t)(tok0 + t) * a.H + hh) * d;
+            } else {
+                int g = hh - a.H;
+                src = k + ((int64_t)(tok0 + t) * a.Hkv + g) * d;
+                dst = kp + ((int64_t)g * a.capacity + a.prefix + tok0 + t) * d;
+            }
+            float lo[VEC], hi[VEC], rlo[VEC], rhi[VEC];
+            Vec16<T>::load(src + c * VEC, lo);
+            Vec16<T>::load(src + half + c * VEC, hi);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+                float2 w = cs[t][c * VEC + e];
+                rotate(lo[e], hi[e], w.x, w.y, rlo[e], rhi[e]);
+            }
+            Vec16<T>::store(dst + c * VEC, rlo);
+            Vec16<T>::store(dst + half + c * VEC, rhi);
+        }
+    } else {
+        const int chunks = d / VEC;                    // vectors per row
+        const int items = ntok * heads * chunks;
+        for (int idx = threadIdx.x; idx < items; idx += kThreads) {
+            int c = idx % chunks;
+            int hh = (idx / chunks) % heads;
+            int t = idx / (chunks * heads);
+            const T *src;
+            T *dst;
+            if (hh < a.H) {
+                src = q + ((int64_t)(tok0 + t) * a.H + hh) * d;
+                dst = qr + ((int64_t)(tok0 + t) * a.H + hh) * d;
+            } else {
+                int g = hh - a.H;
+                src = k + ((int64_t)(tok0 + t) * a.Hkv + g) * d;
+                dst = kp + ((int64_t)g * a.capacity + a.prefix + tok0 + t) * d;
+            }
+            float x[VEC], r[VEC];
+            Vec16<T>::load(src + c * VEC, x);
+#pragma unroll
+            for (int e = 0; e < VEC; e += 2) {
+                float2 w = cs[t][(c * VEC + e) / 2];
+                rotate(x[e], x[e + 1], w.x, w.y, r[e], r[e + 1]);
+            }
+            Vec16<T>::store(dst + c * VEC, r);
+        }
+    }
+
+    // values: verbatim 16-byte copies
+    {
+        const int chunks = d / VEC;
+        const int items = ntok * a.Hkv * chunks;
+        for (int idx = threadIdx.x; idx < items; idx += kThreads) {
+            int c = idx % chunks;
+            int g = (idx / chunks) % a.Hkv;
+            int t = idx / (chunks * a.Hkv);
+            uint4 val = *reinterpret_cast<const uint4 *>(v + ((int64_t)(tok0 + t) * a.Hkv + g) * d + c * VEC);
+            *reinterpret_cast<uint4 *>(vp + ((int64_t)g * a.capacity + a.prefix + tok0 + t) * d + c * VEC) = val;
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interleaved, cudaStream_t s) {
+    int blocks = (a.n + kTok - 1) / kTok;
+    if (a.zero_rows > 0) {
+        int64_t vecs = (int64_t)a.zero_rows * a.Hkv * (a.d / (dtype == 0 ? 8 : 4));
+        blocks += (int)((vecs + kThreads - 1) / kThreads);
+    }
+    if (dtype == 0) {
+        if (interleaved) rope_append_kernel<__nv_bfloat16, true><<<blocks, kThreads, 0, s>>>(a);
+        else rope_append_kernel<__nv_bfloat16, false><<<blocks, kThreads, 0, s>>>(a);
+    } else {
+        if (interleaved) rope_append_kernel<float, true><<<blocks, kThreads, 0, s>>>(a);
+        else rope_append_kernel<float, false><<<blocks, kThreads, 0, s>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace kvf

@@ -1,0 +1,121 @@
+"""Host-side checks that need no GPU: the library loads, exports what the header declares,
+validates configurations before touching CUDA, and sizes buffers as documented."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2605_12471_b200 import build as kbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    kbuild.build_library()
+    from paper_2605_12471_b200 import binding as b
+    b.load()
+    return b
+
+
+def test_every_declared_symbol_is_exported(binding):
+    header = open(os.path.join(ROOT, "include", "kvfold.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(kvf_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS), declared ^ set(binding.EXPORTS)
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_struct_layout_matches_header(binding):
+    c = binding.kvf_config
+    assert ctypes.sizeof(c) == 56
+    assert c.capacity.offset == 16 and c.max_chunk.offset == 24 and c.flags.offset == 28
+    assert c.rope_base.offset == 32 and c.softmax_scale.offset == 40 and c.inv_freq.offset == 48
+
+
+def test_storage_bytes_follow_the_papers_per_token_count(binding):
+    # Section 5: 8 KV heads x 128 x (K,V) x 2 bytes per token per layer; 32 layers = 131072 B/token
+    cfg = binding.make_config(32, 8, 128, "bf16", 131072, 256, rope_base=5e5)
+    per_layer = binding.cache_storage_bytes(cfg)
+    assert per_layer == 131072 * 4096
+    assert 32 * per_layer == 17179869184
+    cfg32 = binding.make_config(32, 8, 128, "f32", 65536, 128, rope_base=5e5)
+    assert binding.cache_storage_bytes(cfg32) == 65536 * 8192
+    tiny = binding.make_config(4, 1, 64, "f32", 512, 64)
+    assert binding.cache_storage_bytes(tiny) == 512 * 1 * 64 * 4 * 2
+    assert binding.workspace_bytes(cfg) > 256 * 32 * 128 * 2
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(n_q_heads=0), "KVF_ERR_INVALID_ARG"),
+    (dict(n_q_heads=30), "KVF_ERR_INVALID_ARG"),            # not a multiple of the KV heads
+    (dict(n_q_heads=24), "KVF_ERR_UNSUPPORTED"),            # group of 3: not a power of two
+    (dict(head_dim=96), "KVF_ERR_UNSUPPORTED"),
+    (dict(dtype=7), "KVF_ERR_UNSUPPORTED"),
+    (dict(capacity=0), "KVF_ERR_INVALID_ARG"),
+    (dict(max_chunk=0), "KVF_ERR_INVALID_ARG"),
+    (dict(max_chunk=4096, capacity=1024), "KVF_ERR_INVALID_ARG"),
+    (dict(rope_base=0.0), "KVF_ERR_INVALID_ARG"),
+    (dict(softmax_scale=-1.0), "KVF_ERR_INVALID_ARG"),
+])
+def test_invalid_configs_are_rejected_before_any_cuda_call(binding, kw, code):
+    base = dict(n_q_heads=32, n_kv_heads=8, head_dim=128, dtype="bf16", capacity=1024, max_chunk=256,
+                rope_base=5e5, softmax_scale=0.0)
+    base.update(kw)
+    cfg = binding.make_config(**base)
+    lib = binding.load()
+    assert binding.cache_storage_bytes(cfg) == 0
+    assert binding.workspace_bytes(cfg) == 0
+    h = ctypes.c_void_p()
+    rc = lib.kvf_cache_create(ctypes.byref(cfg), 4096, 1 << 40, 4096, 1 << 40, ctypes.byref(h))
+    assert lib.kvf_status_str(rc).decode() == code
+    assert not h.value
+
+
+def test_create_rejects_null_and_misaligned_and_short_buffers_without_cuda(binding):
+    lib = binding.load()
+    cfg = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5)
+    sb, wb = binding.cache_storage_bytes(cfg), binding.workspace_bytes(cfg)
+    h = ctypes.c_void_p()
+    assert lib.kvf_cache_create(ctypes.byref(cfg), None, sb, 4096, wb, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_cache_create(ctypes.byref(cfg), 4096, sb, None, wb, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_cache_create(ctypes.byref(cfg), 4096 + 16, sb, 4096, wb, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_cache_create(ctypes.byref(cfg), 4096, sb - 1, 4096, wb, ctypes.byref(h)) == binding.KVF_ERR_CAPACITY
+    assert lib.kvf_cache_create(ctypes.byref(cfg), 4096, sb, 4096, wb - 1, ctypes.byref(h)) == binding.KVF_ERR_CAPACITY
+    assert lib.kvf_cache_create(None, 4096, sb, 4096, wb, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_cache_create(ctypes.byref(cfg), 4096, sb, 4096, wb, None) == binding.KVF_ERR_INVALID_ARG
+
+
+def test_null_handles_are_harmless(binding):
+    lib = binding.load()
+    assert lib.kvf_cache_len(None) == -1
+    assert lib.kvf_cache_reset(None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_fold_step(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_fold_step_host(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_cache_launch_count(None) == 0
+    lib.kvf_cache_destroy(None)
+    assert lib.kvf_status_str(0).decode() == "KVF_OK"
+    assert lib.kvf_status_str(5).decode() == "KVF_ERR_TIMEOUT"
+
+
+def test_binding_fails_loudly_without_the_library(binding, monkeypatch, tmp_path):
+    import importlib
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(ImportError):
+        binding.load()
+    monkeypatch.undo()
+    importlib.reload(binding)
+
+
+def test_product_package_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2605_12471_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".h", ".cuh")):
+                text = open(os.path.join(dirpath, f)).read()
+                for needle in ("import oracle", "from oracle", "kvfold_oracle", "okvf_"):
+                    assert needle not in text, (needle, os.path.join(dirpath, f))

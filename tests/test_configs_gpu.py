@@ -1,0 +1,77 @@
+"""Parity at the full sizes of the benchmark configurations, on sampled steps and rows.
+
+The oracle ingests every chunk (so its cache is the whole history in fp64) but evaluates only
+sampled query rows: a row over a 131 072-token prefix costs ~2 GFLOP in fp64.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_12471_b200 import binding, workloads
+from tests.chain import TOL, assert_within, run_chain, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+def _steps(n_steps, rng, extra=3):
+    fixed = {0, 1, 2, n_steps // 4, n_steps // 2, n_steps - 2, n_steps - 1}
+    fixed = {s for s in fixed if 0 <= s < n_steps}
+    fixed.update(int(x) for x in rng.integers(0, n_steps, size=extra))
+    return sorted(fixed)
+
+
+def test_config2_llama_16k_chunks_of_2048():
+    w = workloads.LLAMA_16K
+    res, cache, _, _ = run_chain(w, [w.chunk] * w.n_steps, seed=21, rows_per_step=6)
+    assert len(cache) == 16384
+    assert_within(res, "bf16", "config 2")
+    # inputs are scaled by 1/sqrt(128): outputs are ~1e-3, so the relative error is the telling one
+    assert res.rel_rms <= 2e-2, res.rel_rms
+
+
+def test_config3_deep_chain_128k_depth_511():
+    """The benchmark's launch configuration: 512 steps of 256 tokens, prefix up to 130 816."""
+    w = workloads.DEEP_CHAIN
+    steps = _steps(w.n_steps, np.random.default_rng(3), extra=2)
+    res, cache, _, _ = run_chain(w, [w.chunk] * w.n_steps, seed=22, check_steps=steps, rows_per_step=2)
+    assert len(cache) == 131072 == 512 * 256
+    assert_within(res, "bf16", "config 3")
+    assert res.rel_rms <= 2e-2, res.rel_rms
+    print("config3 drift per checked step (max abs):", {k: f"{v:.2e}" for k, v in sorted(res.per_step.items())})
+
+
+@pytest.mark.parametrize("C", [128, 512, 2048, 8192])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_config4_chunk_and_precision_sweep_64k(C, dtype):
+    w = workloads.sweep(C, dtype)
+    steps = _steps(w.n_steps, np.random.default_rng(C), extra=1)
+    res, cache, _, _ = run_chain(w, [C] * w.n_steps, seed=23, check_steps=steps, rows_per_step=1)
+    assert len(cache) == 65536
+    assert_within(res, dtype, f"config 4 C={C} {dtype}")
+    print(f"config4 C={C} {dtype}: max {res.max_abs:.2e} mean {res.mean_abs:.2e} rel_rms {res.rel_rms:.2e}")
+
+
+def test_config5_layer_stack_reduced():
+    """Config 5's structure (independent sequences x layers, each its own cache, all layers' steps
+    issued per chunk on one stream, one shared workspace) at a size the oracle can follow."""
+    w = workloads.FULL_STACK.with_(name="full_stack_reduced", tokens=4096, n_sequences=2, n_layers=3)
+    C = w.chunk
+    cfg = binding.make_config(w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.tokens, C, rope_base=w.rope_base)
+    ws = torch.empty(binding.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    caches = {(s, l): binding.Cache(cfg, workspace=ws) for s in range(w.n_sequences) for l in range(w.n_layers)}
+    oracles = {key: oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens, rope_base=w.rope_base)
+               for key in [(0, 0), (1, 2)]}
+    worst = 0.0
+    for t in range(w.n_steps):
+        outs = {}
+        for (s, l), c in caches.items():
+            q, k, v = workloads.chunk_inputs(w, 24, t, sequence=s, layer=l, device="cuda")
+            outs[(s, l)] = (c.fold_step(q, k, v), q, k, v)
+        for key, oc in oracles.items():
+            out, q, k, v = outs[key]
+            rows = [0, C // 2, C - 1]
+            ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows)
+            worst = max(worst, float(np.abs(to_f64(out[rows]) - ref).max()))
+    assert all(len(c) == w.tokens for c in caches.values())
+    assert worst <= TOL["bf16"][0]

@@ -1,0 +1,312 @@
+"""Parity of the CUDA fold step (through the C ABI) against the fp64 oracle, small and mid sizes.
+
+Every test here needs a B200; the oracle side runs on the host cores.
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_12471_b200 import binding, workloads
+from tests.chain import TOL, assert_within, run_chain, to_f64
+
+pytestmark = pytest.mark.gpu
+
+SMALL_LLAMA = workloads.Workload("small_llama_bf16", 32, 8, 128, "bf16", 256, 1024, 500000.0)
+SMALL_LLAMA_F32 = SMALL_LLAMA.with_(name="small_llama_f32", dtype="f32")
+
+
+def test_library_is_loaded_from_the_tree():
+    lib = binding.load()
+    assert lib._name == binding.LIB_PATH
+
+
+# ------------------------------------------------------------------ config 1
+def test_tiny_fold_fp32_matches_oracle_everywhere():
+    w = workloads.TINY
+    res, cache, oc, _ = run_chain(w, [w.chunk] * w.n_steps, seed=1)
+    assert len(cache) == w.tokens == len(oc)
+    assert res.count == w.tokens * w.n_q_heads * w.head_dim
+    assert_within(res, "f32", "tiny fold")
+    assert res.lse_max_abs <= 1e-5
+
+
+def test_tiny_fold_len_after_t_steps_is_t_times_c():
+    w = workloads.TINY
+    cache = binding.cache_for(w)
+    for t in range(w.n_steps):
+        q, k, v = workloads.chunk_inputs(w, 2, t, device="cuda")
+        cache.fold_step(q, k, v)
+        assert len(cache) == (t + 1) * w.chunk          # host counter, no sync needed
+    torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("C", [1, 3, 64, 100, 512])
+def test_tiny_fold_every_chunking_gives_the_same_outputs(C):
+    """fold(C) == fold(C') == one causal pass: the defining invariant, on the GPU."""
+    w = workloads.TINY
+    q, k, v = workloads.sequence_inputs(w, 3, device="cuda")
+    T = w.tokens
+    cache = binding.cache_for(w, max_chunk=T)
+    ref = cache.fold_step(q, k, v).clone()              # monolithic: one step over everything
+    cache.reset()
+    outs = []
+    for t0 in range(0, T, C):
+        outs.append(cache.fold_step(q[t0:t0 + C], k[t0:t0 + C], v[t0:t0 + C]).clone())
+    got = torch.cat(outs)
+    assert len(cache) == T
+    assert (got - ref).abs().max().item() <= 2e-6
+
+
+# ------------------------------------------------------------ cache contents
+def _ulp_diff_bf16(a: torch.Tensor, b: torch.Tensor) -> torch.Tensor:
+    ia = a.view(torch.int16).to(torch.int32)
+    ib = b.view(torch.int16).to(torch.int32)
+    # sign-magnitude -> monotone integers
+    ia = torch.where(ia < 0, -(ia & 0x7FFF), ia)
+    ib = torch.where(ib < 0, -(ib & 0x7FFF), ib)
+    return (ia - ib).abs()
+
+
+@pytest.mark.parametrize("w,chunks,flags", [
+    (workloads.TINY, [64] * 4, 0),
+    (workloads.TINY, [33, 1, 94], binding.KVF_ROPE_INTERLEAVED),
+    (SMALL_LLAMA, [256, 256, 100, 1], 0),
+    (SMALL_LLAMA, [129, 300], binding.KVF_ROPE_INTERLEAVED),
+])
+def test_appended_cache_bits_match_dtype_faithful_rotation(w, chunks, flags):
+    """K rows are the oracle's same-dtype rotation bit for bit; V rows are the inputs verbatim.
+
+    cos/sin come from the device's fp64 routines, which may differ from the host libm by an ulp
+    of fp64 and so, after rounding to fp32, in rare table entries: the contract is <= 1 ulp of
+    the cache dtype per element with at most 1e-5 of the elements differing at all.
+    """
+    total = sum(chunks)
+    pos_base = 100000                                   # large positions: worst case for the table
+    cache = binding.cache_for(w, capacity=total, max_chunk=max(chunks), flags=flags)
+    tab = oracle.inv_freq(w.rope_base, w.head_dim)
+    ks, vs = [], []
+    for t, n in enumerate(chunks):
+        q, k, v = workloads.chunk_inputs(w, 5, t, device="cuda", n_tokens=n)
+        cache.fold_step(q, k, v, pos0=pos_base + len(cache))
+        ks.append(k)
+        vs.append(v)
+    torch.cuda.synchronize()
+    k_all, v_all = torch.cat(ks).cpu(), torch.cat(vs).cpu()
+    want = oracle.rope_faithful(k_all.float().numpy(), pos_base, tab,
+                                interleaved=bool(flags & binding.KVF_ROPE_INTERLEAVED),
+                                to_bf16=(w.dtype == "bf16"))
+    want = torch.from_numpy(want).to(k_all.dtype).permute(1, 0, 2).contiguous()     # [Hkv, T, d]
+    got_k = cache.k_plane()[:, :total].cpu()
+    got_v = cache.v_plane()[:, :total].cpu()
+    assert torch.equal(got_v.view(torch.uint8), v_all.permute(1, 0, 2).contiguous().view(torch.uint8))
+    if w.dtype == "bf16":
+        diff = _ulp_diff_bf16(got_k, want)
+    else:
+        diff = (got_k.view(torch.int32).to(torch.int64) - want.view(torch.int32).to(torch.int64)).abs()
+    assert int(diff.max()) <= 1
+    assert float((diff != 0).float().mean()) <= 1e-5
+    assert len(cache) == total
+
+
+def test_prefix_rows_are_untouched_by_later_steps():
+    w = SMALL_LLAMA
+    cache = binding.cache_for(w, capacity=1024 + 128)
+    q, k, v = workloads.chunk_inputs(w, 6, 0, device="cuda", n_tokens=200)
+    cache.fold_step(q, k, v)
+    torch.cuda.synchronize()
+    k0 = cache.k_plane()[:, :200].clone()
+    v0 = cache.v_plane()[:, :200].clone()
+    for t in range(1, 4):
+        q, k, v = workloads.chunk_inputs(w, 6, t, device="cuda")
+        cache.fold_step(q, k, v)
+    torch.cuda.synchronize()
+    assert torch.equal(cache.k_plane()[:, :200], k0)
+    assert torch.equal(cache.v_plane()[:, :200], v0)
+
+
+# -------------------------------------------------------- mid-size parity, both paths
+@pytest.mark.parametrize("flags", [0, binding.KVF_FORCE_SIMT])
+def test_small_llama_bf16_matches_oracle(flags):
+    w = SMALL_LLAMA
+    res, cache, _, _ = run_chain(w, [256] * 4, seed=7, flags=flags)
+    assert_within(res, "bf16", f"small llama bf16 flags={flags}")
+    assert res.lse_max_abs <= 2e-2
+
+
+def test_small_llama_f32_matches_oracle():
+    res, _, _, _ = run_chain(SMALL_LLAMA_F32, [256] * 3, seed=8)
+    assert_within(res, "f32", "small llama f32")
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_ragged_chunk_lengths_including_single_tokens(dtype):
+    w = SMALL_LLAMA.with_(name=f"ragged_{dtype}", dtype=dtype)
+    chunks = [1, 1, 31, 32, 33, 127, 129, 255, 1, 64, 7]
+    res, cache, _, _ = run_chain(w, chunks, seed=9)
+    assert len(cache) == sum(chunks)
+    assert_within(res, dtype, "ragged")
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_out_f32_flag_and_interleaved_rotation(dtype):
+    w = SMALL_LLAMA.with_(name=f"flags_{dtype}", dtype=dtype)
+    flags = binding.KVF_OUT_F32 | binding.KVF_ROPE_INTERLEAVED
+    res, cache, _, outs = run_chain(w, [200, 56, 256], seed=10, flags=flags, keep_outputs=True)
+    assert outs[0].dtype == torch.float32
+    assert_within(res, dtype, "out_f32+interleaved")
+
+
+@pytest.mark.parametrize("dtype,flags", [("bf16", 0), ("bf16", binding.KVF_FORCE_SIMT), ("f32", 0)])
+def test_split_counts_agree_with_each_other_and_with_the_oracle(dtype, flags):
+    w = SMALL_LLAMA.with_(name=f"split_{dtype}", dtype=dtype, tokens=4096)
+    chunks = [2048, 256, 100, 1, 64]
+    ref = None
+    for splits in (1, 2, 5, 0):
+        res, cache, _, outs = run_chain(w, chunks, seed=11, flags=flags, splits=splits,
+                                        check_steps=[1, 2, 3, 4], rows_per_step=4, keep_outputs=True)
+        assert_within(res, dtype, f"splits={splits}")
+        last = torch.cat([o.float().flatten() for o in outs[1:]])
+        if ref is None:
+            ref = last
+        else:
+            assert (last - ref).abs().max().item() <= TOL[dtype][0]
+        if splits in (2, 5):
+            assert cache.plan(64)[1] == splits
+
+
+def test_results_are_bitwise_reproducible():
+    w = SMALL_LLAMA.with_(name="determinism", tokens=2048)
+    a = run_chain(w, [512, 256, 256, 3], seed=12, check_steps=[], keep_outputs=True)[3]
+    b = run_chain(w, [512, 256, 256, 3], seed=12, check_steps=[], keep_outputs=True)[3]
+    for x, y in zip(a, b):
+        assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+
+
+def test_non_continued_positions_are_honoured():
+    """pos0 is used for the rotation only; the oracle gets the same positions."""
+    w = SMALL_LLAMA.with_(name="positions")
+    res, _, _, _ = run_chain(w, [128, 128, 64], seed=13, positions=[1000, 50000, 7])
+    assert_within(res, "bf16", "free positions")
+
+
+def test_uninitialised_storage_with_nan_bits_does_not_leak():
+    """Rows past the end of the cache are not content: non-finite garbage there must not matter."""
+    w = SMALL_LLAMA.with_(name="nan_storage")
+    cache = binding.cache_for(w, capacity=1000, max_chunk=300)
+    cache.storage.view(torch.int16).fill_(0x7FC0)   # bf16 NaN
+    oc = oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, 1000, rope_base=w.rope_base)
+    for t, n in enumerate([70, 300, 1]):
+        q, k, v = workloads.chunk_inputs(w, 14, t, device="cuda", n_tokens=n)
+        out = cache.fold_step(q, k, v)
+        ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v))
+        assert torch.isfinite(out).all()
+        assert np.abs(to_f64(out) - ref).max() <= TOL["bf16"][0]
+
+
+def test_planted_key_survives_the_chain():
+    """Kernel-level needle: a key planted in chunk 0 is recovered by a query 31 chunks later."""
+    w = SMALL_LLAMA.with_(name="needle", tokens=8192)
+    H, Hkv, d, C = w.n_q_heads, w.n_kv_heads, w.head_dim, 256
+    cache = binding.cache_for(w, capacity=8192, max_chunk=C)
+    needle_v = None
+    tab = torch.from_numpy(oracle.inv_freq(w.rope_base, d))
+
+    def unrotate(vec, pos):
+        ang = pos * tab
+        lo, hi = vec[:d // 2].double(), vec[d // 2:].double()
+        return torch.cat([lo * torch.cos(ang) + hi * torch.sin(ang), hi * torch.cos(ang) - lo * torch.sin(ang)])
+
+    direction = torch.zeros(d)
+    direction[:4] = 0.5                                   # |direction| = 1
+    for t in range(32):
+        q, k, v = workloads.chunk_inputs(w, 15, t, device="cuda")
+        q, k = q * 0.05, k * 0.05
+        if t == 0:
+            k[5] = unrotate(direction * 40.0, 5).to(k.dtype).to("cuda")
+            needle_v = v[5].clone()
+        if t == 31:
+            q[200] = unrotate(direction * 40.0, 31 * C + 200).to(q.dtype).to("cuda")
+        out = cache.fold_step(q.contiguous(), k.contiguous(), v)
+    for h in range(H):
+        assert (out[200, h].float() - needle_v[h // 4].float()).abs().max().item() <= 2e-2
+
+
+# ------------------------------------------------------------------ host-side errors
+def test_errors_are_return_codes_and_change_nothing():
+    w = SMALL_LLAMA
+    cfg = binding.make_config(32, 8, 128, "bf16", 512, 256, rope_base=5e5, flags=binding.KVF_STRICT_POS)
+    cache = binding.Cache(cfg)
+    q, k, v = workloads.chunk_inputs(w, 16, 0, device="cuda")
+    lib = binding.load()
+    out = torch.empty_like(q)
+    h = cache._h
+
+    def call(qp, kp, vp, n, pos0, op):
+        return lib.kvf_fold_step(h, qp, kp, vp, n, pos0, op, None, None)
+
+    launches = cache.launch_count()
+    assert call(None, k.data_ptr(), v.data_ptr(), 256, 0, out.data_ptr()) == binding.KVF_ERR_INVALID_ARG
+    assert call(q.data_ptr() + 2, k.data_ptr(), v.data_ptr(), 256, 0, out.data_ptr()) == binding.KVF_ERR_INVALID_ARG
+    assert call(q.data_ptr(), k.data_ptr(), v.data_ptr(), 0, 0, out.data_ptr()) == binding.KVF_ERR_INVALID_ARG
+    assert call(q.data_ptr(), k.data_ptr(), v.data_ptr(), 257, 0, out.data_ptr()) == binding.KVF_ERR_INVALID_ARG
+    assert call(q.data_ptr(), k.data_ptr(), v.data_ptr(), 256, 5, out.data_ptr()) == binding.KVF_ERR_POS
+    assert len(cache) == 0 and cache.launch_count() == launches
+    cache.fold_step(q, k, v)
+    cache.fold_step(q, k, v)
+    assert len(cache) == 512
+    assert call(q.data_ptr(), k.data_ptr(), v.data_ptr(), 1, 512, out.data_ptr()) == binding.KVF_ERR_CAPACITY
+    assert len(cache) == 512
+    with pytest.raises(binding.KvfError):
+        cache.fold_step(q, k, v)
+    cache.reset()
+    assert len(cache) == 0
+    assert lib.kvf_cache_len(None) == -1
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_OK
+
+
+def test_create_rejects_short_or_misaligned_buffers():
+    lib = binding.load()
+    cfg = binding.make_config(32, 8, 128, "bf16", 512, 256, rope_base=5e5)
+    sb, wb = binding.cache_storage_bytes(cfg), binding.workspace_bytes(cfg)
+    st = torch.empty(sb + 512, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(wb + 512, dtype=torch.uint8, device="cuda")
+    h = ctypes.c_void_p()
+    assert lib.kvf_cache_create(ctypes.byref(cfg), st.data_ptr(), sb - 1, ws.data_ptr(), wb, ctypes.byref(h)) == binding.KVF_ERR_CAPACITY
+    assert lib.kvf_cache_create(ctypes.byref(cfg), st.data_ptr(), sb, ws.data_ptr(), wb - 1, ctypes.byref(h)) == binding.KVF_ERR_CAPACITY
+    assert lib.kvf_cache_create(ctypes.byref(cfg), st.data_ptr() + 16, sb, ws.data_ptr(), wb, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_cache_create(ctypes.byref(cfg), st.data_ptr(), sb, ws.data_ptr(), wb, ctypes.byref(h)) == binding.KVF_OK
+    lib.kvf_cache_destroy(h)
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    w = SMALL_LLAMA
+    a = binding.cache_for(w)
+    b = binding.cache_for(w)
+    for t in range(3):
+        q, k, v = workloads.chunk_inputs(w, 17, t, device="cuda")
+        want = a.fold_step(q, k, v)
+        qh, kh, vh = (x.cpu().pin_memory() for x in (q, k, v))
+        oh = torch.empty(want.shape, dtype=want.dtype).pin_memory()
+        lh = torch.empty((w.chunk, w.n_q_heads), dtype=torch.float32).pin_memory()
+        b.fold_step_host(qh, kh, vh, oh, lse=lh)
+        torch.cuda.synchronize()
+        assert torch.equal(oh.view(torch.int16), want.cpu().view(torch.int16))
+        assert torch.isfinite(lh).all()
+    assert len(a) == len(b) == 3 * w.chunk
+
+
+def test_profile_counters_and_launch_count():
+    w = SMALL_LLAMA
+    cache = binding.cache_for(w)
+    cache.profile(True)
+    for t in range(4):
+        q, k, v = workloads.chunk_inputs(w, 18, t, device="cuda")
+        cache.fold_step(q, k, v)
+    ms, cnt = cache.profile_read()
+    assert cnt[0] == 4 and cnt[1] == 4
+    assert cache.launch_count() == sum(cnt)
+    assert all(m >= 0 for m in ms) and ms[1] > 0

@@ -1,0 +1,62 @@
+"""The benchmark's multi-rank plumbing on two gloo ranks (CPU): each rank owns its own sequence,
+nothing is exchanged on the data path, elapsed time is reduced with max."""
+import os
+import socket
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import oracle
+from paper_2605_12471_b200 import multi, workloads
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, ret):
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    r, wsize, local = multi.env_rank()
+    assert (r, wsize, local) == (rank, world, rank)
+    w = workloads.TINY
+    seq = multi.sequence_of_rank(r)[0]
+    oc = oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens, rope_base=w.rope_base)
+    outs = []
+    for t in range(w.n_steps):
+        q, k, v = workloads.chunk_inputs(w, 7, t, sequence=seq)
+        outs.append(oc.fold_step(q.double().numpy(), k.double().numpy(), v.double().numpy()))
+    checksum = float(np.concatenate(outs).sum())
+    fake_ms = 10.0 * (rank + 1)                          # rank 1 is the slow one
+    worst = multi.max_over_ranks(fake_ms)
+    sums = [None] * world
+    dist.all_gather_object(sums, (len(oc), checksum))
+    if rank == 0:
+        ret["worst"] = worst
+        ret["sums"] = sums
+        ret["value"] = multi.whole_job_tokens_per_s(w.tokens, 2, world, worst)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_fold_independent_sequences_and_reduce_time_with_max():
+    world = 2
+    mgr = mp.Manager()
+    ret = mgr.dict()
+    mp.spawn(_worker, args=(world, _free_port(), ret), nprocs=world, join=True)
+    assert ret["worst"] == 20.0
+    (l0, c0), (l1, c1) = ret["sums"]
+    assert l0 == l1 == workloads.TINY.tokens
+    assert c0 != c1                                      # different sequences per rank
+    assert abs(ret["value"] - 2 * 2 * 512 / 0.020) < 1e-6
+
+
+def test_single_process_helpers():
+    assert multi.sequence_of_rank(3, 2) == [6, 7]
+    assert multi.max_over_ranks(3.5) == 3.5
+    assert multi.whole_job_tokens_per_s(131072, 5, 8, 1000.0) == 8 * 5 * 131072
