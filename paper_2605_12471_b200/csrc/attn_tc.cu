@@ -8,11 +8,14 @@
 //
 // One CTA = 256 query rows of one KV head (row = token * G + head-in-group, so the G query heads
 // that share a KV head share every K/V tile), processed as two 128-row tiles that take turns on
-// the tensor pipe, against 128-key tiles streamed through a 3-slot shared-memory ring by TMA.
+// the tensor pipe, against 128-key tiles streamed through a 5-slot shared-memory ring by TMA.
 //   warps 0-3 / 4-7 : softmax of row tile 0 / 1 (one thread per row; TMEM lane = row)
 //   warp 8          : TMA producer (Q once, then K(j), V(j), K(j+1), ...)
 //   warp 9          : tcgen05.mma issuer, owns the TMEM allocation
-// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each.
+// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each.  The bf16 probabilities
+// overwrite the first 64 columns of their own S tile (two per 32-bit cell) and feed the second
+// MMA straight from tensor memory; the tensor pipe runs one thread's MMAs in issue order, so the
+// next Q K^T of a row tile cannot overtake the P V that still reads those columns.
 // Split over the key range: blockIdx.z takes a contiguous range of key tiles and writes a
 // normalised partial output plus its log2 denominator; the combine kernel merges them.
 //
@@ -28,11 +31,10 @@ constexpr int kRows = 128;                    // rows of a Q tile = keys of a K/
 constexpr int kD = 128;                       // head_dim
 constexpr uint32_t kPanel = 128 * 128;        // bytes of a [128 rows][64 bf16] swizzled panel
 constexpr uint32_t kTileBytes = 2 * kPanel;   // a 128 x 128 bf16 tile = two panels
-constexpr int kSlots = 3;
+constexpr int kSlots = 5;
 constexpr int kThreads = 320;
 constexpr uint32_t kOffQ = 0;                         // 2 tiles
-constexpr uint32_t kOffP = 2 * kTileBytes;            // 2 tiles
-constexpr uint32_t kOffKV = 4 * kTileBytes;           // kSlots tiles
+constexpr uint32_t kOffKV = 2 * kTileBytes;           // kSlots tiles
 constexpr uint32_t kOffCtl = kOffKV + kSlots * kTileBytes;
 constexpr uint32_t kSmemBytes = kOffCtl + 256 + 1024; // + control block + alignment slack
 constexpr uint32_t kTmemCols = 512;
@@ -40,10 +42,11 @@ constexpr float kRescaleThreshold = 8.0f;             // log2 units
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
 // barrier indices inside the control block
-enum { B_QFULL = 0, B_FULL0 = 1, B_EMPTY0 = 4, B_SFULL0 = 7, B_PFULL0 = 9, B_OFINAL0 = 11, B_COUNT = 13 };
+enum { B_QFULL = 0, B_FULL0 = 1, B_EMPTY0 = 1 + kSlots, B_SFULL0 = 1 + 2 * kSlots, B_PFULL0 = B_SFULL0 + 2,
+       B_OFINAL0 = B_PFULL0 + 2, B_COUNT = B_OFINAL0 + 2 };
 
 struct Ctl {
-    unsigned long long bars[16];
+    unsigned long long bars[24];
     uint32_t tmem_base;
     int abort;
 };
@@ -112,6 +115,14 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// A operand from tensor memory (lane = row, each 32-bit column holds two consecutive bf16 of K)
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
 #define KVF_R32(a, o) "=r"(a[o + 0]), "=r"(a[o + 1]), "=r"(a[o + 2]), "=r"(a[o + 3]), "=r"(a[o + 4]), "=r"(a[o + 5]), "=r"(a[o + 6]), "=r"(a[o + 7]), \
@@ -254,13 +265,11 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 }
             };
             auto issue_pv = [&](int i, int slot, bool accumulate) {
-                const uint32_t pa = base + kOffP + i * kTileBytes, vb = base + kOffKV + slot * kTileBytes;
+                const uint32_t vb = base + kOffKV + slot * kTileBytes;
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t aoff = (kk >> 2) * kPanel + (kk & 3) * 32;
-                    tc_mma(tmem + 256 + i * 128, desc_kmajor(pa + aoff), desc_mnmajor(vb + kk * 2048), kIdescPV,
-                           (accumulate || kk > 0) ? 1u : 0u);
-                }
+                for (int kk = 0; kk < 8; ++kk)   // 16 keys = 8 packed columns of P per MMA
+                    tc_mma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, desc_mnmajor(vb + kk * 2048), kIdescPV,
+                              (accumulate || kk > 0) ? 1u : 0u);
             };
             for (int j = 0; j < ntiles && ok; ++j) {
                 const int tk = 2 * j, kslot = tk % kSlots;
@@ -305,8 +314,6 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         const bool valid = tok < n;
         const int64_t limit = valid ? P + tok + 1 : 0;  // keys below `limit` are visible
         const float sl2 = a.scale_log2;
-        const uint32_t p_row = base + kOffP + i * kTileBytes + r * 128;
-        const uint32_t sw = (uint32_t)(r & 7);
 
         float m_ref = -INFINITY;   // reference maximum (raw score units) the probabilities are scaled by
         float l = 0.f;
@@ -364,23 +371,20 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             const float neg = -m_safe * sl2;
             float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
-            for (int c8 = 0; c8 < 16; ++c8) {
-                float p[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) p[e] = ex2(fmaf(__uint_as_float(s[c8 * 8 + e]), sl2, neg));
-                sum0 += p[0] + p[4]; sum1 += p[1] + p[5]; sum2 += p[2] + p[6]; sum3 += p[3] + p[7];
-                uint32_t w[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    __nv_bfloat162 b = __floats2bfloat162_rn(p[2 * e], p[2 * e + 1]);
-                    w[e] = *reinterpret_cast<uint32_t *>(&b);
-                }
-                const uint32_t addr = p_row + (c8 >> 3) * kPanel + ((((uint32_t)c8 & 7u) ^ sw) << 4);
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+            for (int c4 = 0; c4 < 32; ++c4) {
+                const float p0 = ex2(fmaf(__uint_as_float(s[c4 * 4 + 0]), sl2, neg));
+                const float p1 = ex2(fmaf(__uint_as_float(s[c4 * 4 + 1]), sl2, neg));
+                const float p2 = ex2(fmaf(__uint_as_float(s[c4 * 4 + 2]), sl2, neg));
+                const float p3 = ex2(fmaf(__uint_as_float(s[c4 * 4 + 3]), sl2, neg));
+                sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+                __nv_bfloat162 b0 = __floats2bfloat162_rn(p0, p1), b1 = __floats2bfloat162_rn(p2, p3);
+                s[c4 * 2 + 0] = *reinterpret_cast<uint32_t *>(&b0);   // packed pair (2c, 2c+1) -> column c
+                s[c4 * 2 + 1] = *reinterpret_cast<uint32_t *>(&b1);
             }
             l += (sum0 + sum1) + (sum2 + sum3);
-            // P (generic-proxy writes) must be visible to the tensor core's async-proxy reads
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            KVF_TMEM_ST32(s, 0, t_s);
+            KVF_TMEM_ST32(s, 32, t_s + 32);
+            tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(B_PFULL0 + i));
         }

@@ -168,9 +168,9 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix) {
     if (c->force_splits > 0) {
         splits = c->force_splits;
     } else if (units < target) {
-        // fill whole waves of the machine, but keep at least 4 key tiles per split
-        int want = (target + units - 1) / units;
-        if (!p.tc) want = (2 * target + units - 1) / units;
+        // one wave: as many splits as still fit the machine at once (a second, partly filled
+        // wave would double the time), but keep at least 4 key tiles per split
+        int want = target / units;
         int64_t cap = nt / 4;
         if (want > cap) want = (int)cap;
         splits = want;
