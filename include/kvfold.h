@@ -177,6 +177,44 @@ kvf_status kvf_cache_profile_read(kvf_cache *c, double ms[3], uint64_t launches[
 /* Frees the host handle (and its events); device memory stays with the caller. */
 void kvf_cache_destroy(kvf_cache *c);
 
+/*
+ * The fold step for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for the sake of such callers only.)
+ *
+ * Who they are: a server that has already handed every byte of device memory to its own pool
+ * (KV pages sized to fill the GPU) and has nothing left to give for a workspace; a latency-bound
+ * loop that must stay out of the allocator because an allocation can stall the whole device for
+ * an unbounded time; a plug-in that runs under a policy forbidding allocation calls.  For them
+ * the step's scratch (status word, rotated queries, split partial results) lives in a fixed
+ * array inside the library, KVF_STATIC_SCRATCH_BYTES (about 20 MiB), which every GPU that loads
+ * the library holds from load until the process exits.  The call, and everything it calls,
+ * allocates and frees nothing on the device.
+ *
+ * There is no handle: the caller owns the planes and the length.
+ *   cfg           as for kvf_cache_create (max_chunk sizes the rotated-query area)
+ *   dev_storage   device, 256-byte aligned, >= kvf_cache_storage_bytes(cfg): K plane then V plane,
+ *                 holding `len` tokens appended by earlier calls (of this or of kvf_fold_step)
+ *   len           tokens already in the planes; after KVF_OK the caller's length is len + n_tokens
+ *   q, k_new, v_new, n_tokens, pos0, out, lse, cuda_stream: as for kvf_fold_step
+ * Limits (KVF_ERR_CAPACITY beyond them, nothing enqueued; kvf_last_cuda_error names the limit):
+ *   max_chunk * n_q_heads * head_dim * sizeof(dtype) <= 4 MiB   (32 heads x 128, bf16: 512 tokens)
+ *   n_tokens * n_q_heads * head_dim * 4 <= 16 MiB; the key range is split at most as many ways as
+ *   16 MiB of fp32 partial results hold (32 heads x 128: splits * n_tokens <= 1024), so a step
+ *   may run with fewer splits than kvf_fold_step would use - same result within tolerance.
+ * First call on a device: looks up the array's device address (cudaGetSymbolAddress, with that
+ * device current) and keeps it; make this first call before any stream capture begins.
+ * Sharing: all calls on one device use the one array, which keeps whatever the last call left
+ * (the call clears the status word it needs at zero; everything else is written before it is
+ * read).  Two calls whose kernels may overlap on the GPU - different streams, or different
+ * threads - race on it: keep all calls on a device in one stream order.  A bounded device-side
+ * wait that gives up cannot be reported here (there is no handle to ask); results are then
+ * undefined, as with kvf_fold_step before kvf_cache_status is read.
+ */
+#define KVF_STATIC_SCRATCH_BYTES 21234688
+kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_storage, size_t storage_bytes, int64_t len,
+                                const void *q, const void *k_new, const void *v_new, int32_t n_tokens,
+                                int64_t pos0, void *out, float *lse, void *cuda_stream);
+
 const char *kvf_status_str(kvf_status s);
 
 /* Text of the last CUDA error seen by this thread's calls into the library ("" if none). */

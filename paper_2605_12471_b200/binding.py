@@ -24,7 +24,7 @@ EXPORTS = [
     "kvf_fold_step_host", "kvf_cache_len", "kvf_cache_reset", "kvf_cache_status",
     "kvf_cache_k_plane", "kvf_cache_v_plane", "kvf_cache_plan", "kvf_cache_set_splits",
     "kvf_cache_launch_count", "kvf_cache_profile", "kvf_cache_profile_read", "kvf_cache_destroy",
-    "kvf_status_str", "kvf_last_cuda_error",
+    "kvf_status_str", "kvf_last_cuda_error", "kvf_fold_step_static",
 ]
 
 
@@ -71,6 +71,8 @@ def load() -> ctypes.CDLL:
     lib.kvf_fold_step.restype = ctypes.c_int
     lib.kvf_fold_step_host.argtypes = [vp, vp, vp, vp, i32, i64, vp, vp, vp]
     lib.kvf_fold_step_host.restype = ctypes.c_int
+    lib.kvf_fold_step_static.argtypes = [cfgp, vp, ctypes.c_size_t, i64, vp, vp, vp, i32, i64, vp, vp, vp]
+    lib.kvf_fold_step_static.restype = ctypes.c_int
     lib.kvf_cache_len.argtypes = [vp]
     lib.kvf_cache_len.restype = i64
     lib.kvf_cache_reset.argtypes = [vp]
@@ -243,6 +245,34 @@ class Cache:
         if rc != KVF_OK:
             raise KvfError(rc, "kvf_cache_profile_read")
         return list(ms), list(cnt)
+
+
+STATIC_SCRATCH_BYTES = 21234688
+
+
+def fold_step_static(cfg: kvf_config, storage: torch.Tensor, length: int, q: torch.Tensor, k_new: torch.Tensor,
+                     v_new: torch.Tensor, pos0: Optional[int] = None, out: Optional[torch.Tensor] = None,
+                     lse: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """kvf_fold_step_static: the step on caller-owned planes with the library's built-in scratch.
+
+    For callers that may not allocate device memory (a process whose memory is all in its own
+    pool, a loop that must stay out of the allocator): nothing is allocated below this call when
+    `out` is given.  `storage` is the uint8 tensor of the K and V planes, `length` the tokens it
+    already holds; the caller adds n_tokens to its own length afterwards.
+    """
+    n = q.shape[0]
+    for t in (q, k_new, v_new):
+        assert t.is_cuda and t.is_contiguous()
+    if out is None:
+        od = torch.float32 if (cfg.flags & KVF_OUT_F32) or cfg.dtype == KVF_F32 else torch.bfloat16
+        out = torch.empty((n, cfg.n_q_heads, cfg.head_dim), dtype=od, device=q.device)
+    rc = load().kvf_fold_step_static(ctypes.byref(cfg), storage.data_ptr(), storage.numel(), int(length),
+                                     q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), n,
+                                     int(length if pos0 is None else pos0), out.data_ptr(),
+                                     lse.data_ptr() if lse is not None else None, _stream_ptr(stream))
+    if rc != KVF_OK:
+        raise KvfError(rc, "kvf_fold_step_static")
+    return out
 
 
 def cache_for(w, capacity: Optional[int] = None, max_chunk: Optional[int] = None, flags: int = 0,

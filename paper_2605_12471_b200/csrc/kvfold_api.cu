@@ -6,7 +6,9 @@
 
 #include <cmath>
 #include <cstdio>
+#include <algorithm>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -476,3 +478,123 @@ const char *kvf_status_str(kvf_status s) {
 const char *kvf_last_cuda_error(void) { return g_cuda_err; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// kvf_fold_step_static: the fold step for callers that cannot allocate device memory.
+//
+// Scratch of the step (status word, rotated queries, split partial results) lives in the
+// file-scope device array below instead of a caller-provided workspace.  Every device that loads
+// this library holds the array (kStaticScratchBytes) from module load until the process exits.
+// In host code the array's name is only a handle for the runtime: its device address is asked
+// for once per device with cudaGetSymbolAddress, with that device current, and that address is
+// what the kernels get.
+namespace {
+
+constexpr size_t kStaticStatusBytes = 1024;
+constexpr size_t kStaticQRotBytes = (size_t)4 << 20;     // rotated queries of one chunk
+constexpr size_t kStaticPartOBytes = (size_t)16 << 20;   // split partial outputs, fp32
+constexpr size_t kStaticPartLseBytes = (size_t)256 << 10;
+constexpr size_t kStaticScratchBytes = kStaticStatusBytes + kStaticQRotBytes + kStaticPartOBytes + kStaticPartLseBytes;
+static_assert(kStaticScratchBytes == KVF_STATIC_SCRATCH_BYTES, "header and library disagree on the scratch size");
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+char *g_static_ptr[kMaxDevices];   // device address of g_static_scratch, per device; null = not asked yet
+
+// Device address of the scratch array on the current device (looked up on the first call).
+kvf_status static_scratch(int dev, char **out) {
+    if (dev < 0 || dev >= kMaxDevices) return KVF_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static scratch)");
+        if (!p || (reinterpret_cast<uintptr_t>(p) & 255u)) {
+            snprintf(g_cuda_err, sizeof(g_cuda_err), "static scratch has no usable device address");
+            return KVF_ERR_CUDA;
+        }
+        g_static_ptr[dev] = static_cast<char *>(p);
+    }
+    *out = g_static_ptr[dev];
+    return KVF_OK;
+}
+
+}  // namespace
+
+extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_storage, size_t storage_bytes,
+                                           int64_t len, const void *q, const void *k_new, const void *v_new,
+                                           int32_t n_tokens, int64_t pos0, void *out, float *lse,
+                                           void *cuda_stream) {
+    kvf_status s = check_config(cfg);
+    if (s != KVF_OK) return s;
+    if (!dev_storage || (reinterpret_cast<uintptr_t>(dev_storage) & 255u)) return KVF_ERR_INVALID_ARG;
+    if (storage_bytes < kvf_cache_storage_bytes(cfg)) return KVF_ERR_CAPACITY;
+    if (len < 0 || n_tokens < 1 || n_tokens > cfg->max_chunk || pos0 < 0) return KVF_ERR_INVALID_ARG;
+    if (len + n_tokens > cfg->capacity) return KVF_ERR_CAPACITY;
+    if ((cfg->flags & KVF_STRICT_POS) && pos0 != len) return KVF_ERR_POS;
+    if (check_ptr(q) || check_ptr(k_new) || check_ptr(v_new) || check_ptr(out)) return KVF_ERR_INVALID_ARG;
+    if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return KVF_ERR_INVALID_ARG;
+
+    // sizes the fixed scratch can hold (max_chunk sizes the rotated-query area and its TMA box)
+    const size_t row_elems = (size_t)cfg->n_q_heads * cfg->head_dim;
+    if ((size_t)cfg->max_chunk * row_elems * elem_bytes(cfg->dtype) > kStaticQRotBytes) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "max_chunk x heads x head_dim exceeds the static scratch");
+        return KVF_ERR_CAPACITY;
+    }
+    const size_t part_tokens = std::min(kStaticPartOBytes / (row_elems * 4), kStaticPartLseBytes / ((size_t)cfg->n_q_heads * 4));
+    if (part_tokens < (size_t)n_tokens) return KVF_ERR_CAPACITY;
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    char *scratch = nullptr;
+    s = static_scratch(dev, &scratch);
+    if (s != KVF_OK) return s;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+
+    // a handle on the stack that points the ordinary step at the static scratch
+    kvf_cache c;
+    c.cfg = *cfg;
+    c.cfg.inv_freq = nullptr;
+    c.device = dev;
+    c.sm_count = sms;
+    c.storage = static_cast<char *>(dev_storage);
+    c.workspace = scratch;
+    c.plane_bytes = kvf_cache_storage_bytes(cfg) / 2;
+    c.lay = Layout();
+    c.lay.status = 0;
+    c.lay.q_rot = kStaticStatusBytes;
+    c.lay.part_o = kStaticStatusBytes + kStaticQRotBytes;
+    c.lay.part_lse = c.lay.part_o + kStaticPartOBytes;
+    c.lay.total = kStaticScratchBytes;
+    c.len = len;
+    c.G = cfg->n_q_heads / cfg->n_kv_heads;
+    const double scale = cfg->softmax_scale > 0.0 ? cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
+    c.scale_log2 = (float)(scale * 1.4426950408889634);
+    for (int j = 0; j < cfg->head_dim / 2; ++j)
+        c.table.inv_freq[j] = cfg->inv_freq ? cfg->inv_freq[j]
+                                            : std::pow(cfg->rope_base, -2.0 * (double)j / (double)cfg->head_dim);
+    for (int j = cfg->head_dim / 2; j < kMaxHalfDim; ++j) c.table.inv_freq[j] = 0.0;
+    c.force_splits = 0;
+    c.launches = 0;
+    c.profile = false;
+    c.tc = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, c.G);
+    if (c.tc) {
+        s = build_maps(&c);
+        if (s != KVF_OK) return s;
+    }
+    // the split count the ordinary step would take, limited to what the partial area holds
+    Plan plan = make_plan(&c, n_tokens, len);
+    const int fit = (int)(part_tokens / (size_t)n_tokens);
+    c.force_splits = plan.splits < fit ? plan.splits : fit;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // the array keeps what the last call left: the status word has to start at zero
+    e = cudaMemsetAsync(scratch, 0, 256, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(status)");
+    return step_impl(&c, q, k_new, v_new, n_tokens, pos0, out, lse, st);
+}
