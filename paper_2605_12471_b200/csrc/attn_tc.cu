@@ -6,23 +6,39 @@
 // max / running sum softmax turns it into bf16 probabilities, and O += P V accumulates in tensor
 // memory in fp32.
 //
-// One CTA = 256 query rows of one KV head (row = token * G + head-in-group, so the G query heads
-// that share a KV head share every K/V tile), processed as two 128-row tiles that take turns on
-// the tensor pipe, against 128-key tiles streamed through a 5-slot shared-memory ring by TMA.
-//   warps 0-3 / 4-7 : softmax of row tile 0 / 1 (one thread per row; TMEM lane = row)
-//   warp 8          : TMA producer (Q once, then K(j), V(j), K(j+1), ...)
-//   warp 9          : tcgen05.mma issuer, owns the TMEM allocation
+// Work decomposition.  A row pair is 256 query rows of one KV head (row = token * G +
+// head-in-group, so the G query heads that share a KV head share every K/V tile), handled as two
+// 128-row tiles that take turns on the tensor pipe.  Keys come in 128-row tiles.  The (KV head,
+// key tile) pairs of a step are laid out on one line and cut into `ngroups` equal contiguous
+// ranges; CTA (x = row pair, y = group) runs its row pair against its group's range, which
+// touches at most two KV heads ("pieces").  The CTAs of a group stream the same tiles at the
+// same time, so a tile leaves HBM once and the other row pairs hit L2.  With ngroups == Hkv a
+// group is exactly one KV head and the CTA writes final outputs; otherwise every piece writes a
+// normalised partial output and its log2 denominator to slot (group + KV head) and the combine
+// kernel below merges the slots of each KV head in order.
+//
+// Roles (320 threads): warps 0-3 / 4-7 softmax of row tile 0 / 1 (one thread per row; TMEM lane
+// = row), warp 8 TMA producer (Q per piece, then K(j), V(j), ... through a 5-slot ring), warp 9
+// tcgen05.mma issuer and owner of the TMEM allocation.
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each.  The bf16 probabilities
-// overwrite the first 64 columns of their own S tile (two per 32-bit cell) and feed the second
-// MMA straight from tensor memory; the tensor pipe runs one thread's MMAs in issue order, so the
-// next Q K^T of a row tile cannot overtake the P V that still reads those columns.
-// Split over the key range: blockIdx.z takes a contiguous range of key tiles and writes a
-// normalised partial output plus its log2 denominator; the combine kernel merges them.
+// overwrite the first 64 columns of their own S tile, in two halves that are handed to the
+// second MMA separately, and feed it straight from tensor memory; the tensor pipe runs one
+// thread's MMAs in issue order, so the next Q K^T of a row tile cannot overtake the P V that
+// still reads those columns.
+//
+// Softmax arithmetic.  p = 2^(s * scale * log2(e) - m) with the reference maximum m moved only
+// when the tile maximum exceeds it by more than 2^8 (then the accumulator is rescaled), packed
+// two-wide fp32 multiply-adds, and, on unmasked tiles, a share of the exponentials evaluated on
+// the FMA pipe (round-to-nearest split, cubic polynomial, exponent insertion; relative error
+// 7.5e-5, below the bf16 rounding of p) because the special-function unit alone is exactly as
+// slow as the two MMAs of a tile.
 //
 // Every wait on an mbarrier is bounded (about one second): on expiry the thread raises the
 // CTA's abort flag and the device status word, all roles leave their loops, tensor memory is
 // released and the kernel returns.
 #include "kvfold_internal.h"
+
+#include <cstdlib>
 
 namespace kvf {
 namespace {
@@ -42,14 +58,15 @@ constexpr float kRescaleThreshold = 8.0f;             // log2 units
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
 // barrier indices inside the control block
-enum { B_QFULL = 0, B_FULL0 = 1, B_EMPTY0 = 1 + kSlots, B_SFULL0 = 1 + 2 * kSlots, B_PFULL0 = B_SFULL0 + 2,
-       B_OFINAL0 = B_PFULL0 + 2, B_COUNT = B_OFINAL0 + 2 };
+enum { B_QFULL = 0, B_QEMPTY = 1, B_FULL0 = 2, B_EMPTY0 = B_FULL0 + kSlots, B_SFULL0 = B_EMPTY0 + kSlots,
+       B_PA0 = B_SFULL0 + 2, B_PB0 = B_PA0 + 2, B_OFINAL0 = B_PB0 + 2, B_COUNT = B_OFINAL0 + 2 };
 
 struct Ctl {
     unsigned long long bars[24];
     uint32_t tmem_base;
     int abort;
 };
+static_assert(B_COUNT <= 24, "control block holds 24 barriers");
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -94,7 +111,9 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, Ctl *
     }
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Ctl *ctl, int *status) {
-    if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+    for (int k = 0; k < 16; ++k)
+        if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, ctl, status);
 }
 
@@ -153,6 +172,33 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&b);
+}
+
+// 2^x for two values on the FMA pipe: x = n + f with n = round(x), f in [-1/2, 1/2];
+// 2^f by a cubic (relative error 7.5e-5), n added into the exponent field.  x is clamped
+// at -126 (the result is then ~1e-38 instead of 0, which is why masked tiles do not use it).
+__device__ __forceinline__ float2 exp2_fma2(float2 x) {
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));      // 1.5 * 2^23: low bits = n
+    const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+    float2 p = __ffma2_rn(f, make_float2(0.05517132207751274f, 0.05517132207751274f),
+                          make_float2(0.24261054396629333f, 0.24261054396629333f));
+    p = __ffma2_rn(p, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
+    p = __ffma2_rn(p, f, make_float2(0.9999281167984009f, 0.9999281167984009f));
+    p.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23));
+    p.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23));
+    return p;
+}
 
 // Shared-memory matrix descriptors (128-byte swizzle, descriptor version 1).
 // K-major operand ([rows][64 bf16] panels, 8-row groups 1024 bytes apart):
@@ -170,6 +216,33 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
 
+// 32 scores of a row -> 16 packed bf16 probability pairs in p[0..15]; their sum goes to acc.
+// kEmu of every 4 pairs take the FMA-pipe exponential.  nvis_here < 32 masks the tail of the
+// chunk (those tiles use kEmu = 0, so a masked score gives exactly 0).
+template <int kEmu>
+__device__ __forceinline__ void exp_chunk(const uint32_t (&v)[32], uint32_t *p, float2 sl2v, float2 negv, int nvis_here,
+                                          float2 &acc0, float2 &acc1) {
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1])), sl2v, negv);
+        float2 e;
+        if ((c & 3) < kEmu) {
+            e = exp2_fma2(x);
+        } else {
+            if (kEmu == 0) {
+                x.x = 2 * c < nvis_here ? x.x : -INFINITY;
+                x.y = 2 * c + 1 < nvis_here ? x.y : -INFINITY;
+            }
+            e.x = ex2(x.x);
+            e.y = ex2(x.y);
+        }
+        if (c & 1) acc1 = __fadd2_rn(acc1, e);
+        else acc0 = __fadd2_rn(acc0, e);
+        p[c] = pack_bf16(e.x, e.y);
+    }
+}
+
+template <int kEmu>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v) {
@@ -180,39 +253,40 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int qpair = blockIdx.x, kvh = blockIdx.y, split = blockIdx.z;
+    const int qpair = blockIdx.x, group = blockIdx.y;
     const int G = a.G, n = a.n;
     const int64_t P = a.prefix, L = P + n;
+    const bool direct = a.ngroups == a.Hkv;
 
-    // key tiles of this CTA
+    // key tiles: this row pair needs tiles below nt_need; the group's share of the
+    // (KV head, tile) line is [lin0, lin1)
     const int row0 = qpair * 2 * kRows;
     const int tok_last = min(n - 1, (row0 + 2 * kRows - 1) / G);
     const int nt_need = (int)((P + tok_last + 1 + kRows - 1) / kRows);
     const int nt_all = (int)((L + kRows - 1) / kRows);
-    const int per = (nt_all + a.splits - 1) / a.splits;
-    const int kt0 = split * per;
-    const int kt1 = min(nt_need, kt0 + per);
-    const int ntiles = kt1 - kt0;
-
-    if (ntiles <= 0) {
-        // this split has no visible key for these rows: an empty partial
-        if (warp < 8 && a.splits > 1) {
-            int R = row0 + threadIdx.x, tok = R / G, gi = R % G;
-            if (tok < n) {
-                int64_t row = (int64_t)tok * a.H + kvh * G + gi;
-                float4 *po = reinterpret_cast<float4 *>(a.part_o + ((int64_t)split * n * a.H + row) * kD);
-#pragma unroll 4
-                for (int c = 0; c < kD / 4; ++c) po[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-                a.part_lse[(int64_t)split * n * a.H + row] = -INFINITY;
-            }
-        }
-        return;
-    }
+    const int64_t line = (int64_t)a.Hkv * nt_all;
+    const int64_t lin0 = group * line / a.ngroups, lin1 = (group + 1) * line / a.ngroups;
+    const int kvh_first = (int)(lin0 / nt_all);
+    // piece k of this CTA: KV head kvh_first + k, tiles [kt0, kt0 + ntiles)
+    auto piece = [&](int kvh, int &kt0, int &ntiles) -> bool {
+        const int64_t b = (int64_t)kvh * nt_all;
+        if (kvh >= a.Hkv || b >= lin1) return false;
+        kt0 = (int)(max(lin0, b) - b);
+        const int kt1 = (int)min(min(lin1, b + nt_all) - b, (int64_t)nt_need);
+        ntiles = kt1 - kt0;
+        return true;
+    };
 
     if (threadIdx.x == 0) {
         mbar_init(bar(B_QFULL), 1);
+        mbar_init(bar(B_QEMPTY), 1);
         for (int s = 0; s < kSlots; ++s) { mbar_init(bar(B_FULL0 + s), 1); mbar_init(bar(B_EMPTY0 + s), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_SFULL0 + i), 1); mbar_init(bar(B_PFULL0 + i), 128); mbar_init(bar(B_OFINAL0 + i), 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(B_SFULL0 + i), 1);
+            mbar_init(bar(B_PA0 + i), 4);
+            mbar_init(bar(B_PB0 + i), 4);
+            mbar_init(bar(B_OFINAL0 + i), 1);
+        }
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -225,37 +299,39 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&ctl->tmem_base);
 
-    if (warp == 8) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            mbar_expect_tx(bar(B_QFULL), 2 * kTileBytes);
-            for (int i = 0; i < 2; ++i)
-                for (int p = 0; p < 2; ++p)
-                    tma_load_3d(base + kOffQ + i * kTileBytes + p * kPanel, &map_q, bar(B_QFULL), p * 64, kvh * G,
-                                (row0 + i * kRows) / G);
-            int issued = 0;
+    if (warp >= 8) {
+        if (warp == 8 && lane == 0) {
+            // ------------------------------------------------------------------ TMA producer
+            int tg = 0, pc = 0;          // ring loads and pieces so far
             bool ok = true;
-            for (int t = 0; t < 2 * ntiles && ok; ++t) {
-                const int slot = t % kSlots, use = t / kSlots;
-                ok = mbar_wait(bar(B_EMPTY0 + slot), (use & 1) ^ 1, ctl, a.status);
+            int kt0, ntiles;
+            for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
+                if (ntiles <= 0) continue;
+                if (pc > 0) ok = mbar_wait(bar(B_QEMPTY), (pc - 1) & 1, ctl, a.status);
                 if (!ok) break;
-                const CUtensorMap *m = (t & 1) ? &map_v : &map_k;
-                const int key0 = (kt0 + (t >> 1)) * kRows;
-                mbar_expect_tx(bar(B_FULL0 + slot), kTileBytes);
-                tma_load_3d(base + kOffKV + slot * kTileBytes, m, bar(B_FULL0 + slot), 0, key0, kvh);
-                tma_load_3d(base + kOffKV + slot * kTileBytes + kPanel, m, bar(B_FULL0 + slot), 64, key0, kvh);
-                issued = t + 1;
+                mbar_expect_tx(bar(B_QFULL), 2 * kTileBytes);
+                for (int i = 0; i < 2; ++i)
+                    for (int p = 0; p < 2; ++p)
+                        tma_load_3d(base + kOffQ + i * kTileBytes + p * kPanel, &map_q, bar(B_QFULL), p * 64, kvh * G,
+                                    (row0 + i * kRows) / G);
+                ++pc;
+                for (int t = 0; t < 2 * ntiles; ++t, ++tg) {
+                    const int slot = tg % kSlots, use = tg / kSlots;
+                    ok = mbar_wait(bar(B_EMPTY0 + slot), (use & 1) ^ 1, ctl, a.status);
+                    if (!ok) break;
+                    const CUtensorMap *m = (t & 1) ? &map_v : &map_k;
+                    const int key0 = (kt0 + (t >> 1)) * kRows;
+                    mbar_expect_tx(bar(B_FULL0 + slot), kTileBytes);
+                    tma_load_3d(base + kOffKV + slot * kTileBytes, m, bar(B_FULL0 + slot), 0, key0, kvh);
+                    tma_load_3d(base + kOffKV + slot * kTileBytes + kPanel, m, bar(B_FULL0 + slot), 64, key0, kvh);
+                }
             }
             // do not leave while a copy may still be writing into this CTA's shared memory
-            mbar_wait(bar(B_QFULL), 0, ctl, a.status);
-            for (int t = max(0, issued - kSlots); t < issued; ++t)
+            if (pc > 0) mbar_wait(bar(B_QFULL), (pc - 1) & 1, ctl, a.status);
+            for (int t = max(0, tg - kSlots); t < tg; ++t)
                 mbar_wait_slow(bar(B_FULL0 + t % kSlots), (t / kSlots) & 1, ctl, a.status);
-        }
-    } else if (warp == 9) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            bool ok = mbar_wait(bar(B_QFULL), 0, ctl, a.status);
-            tc_fence_after();
+        } else if (warp == 9 && lane == 0) {
+            // ------------------------------------------------------------------ MMA issuer
             auto issue_qk = [&](int i, int slot) {
                 const uint32_t qa = base + kOffQ + i * kTileBytes, kb = base + kOffKV + slot * kTileBytes;
 #pragma unroll
@@ -264,43 +340,66 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                     tc_mma(tmem + i * 128, desc_kmajor(qa + off), desc_kmajor(kb + off), kIdescQK, kk > 0);
                 }
             };
-            auto issue_pv = [&](int i, int slot, bool accumulate) {
+            // 16 keys = 8 packed columns of P per MMA; half h covers keys 64h .. 64h+63
+            auto issue_pv_half = [&](int i, int slot, int h, bool accumulate) {
                 const uint32_t vb = base + kOffKV + slot * kTileBytes;
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)   // 16 keys = 8 packed columns of P per MMA
+                for (int kk = 4 * h; kk < 4 * h + 4; ++kk)
                     tc_mma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, desc_mnmajor(vb + kk * 2048), kIdescPV,
                               (accumulate || kk > 0) ? 1u : 0u);
             };
-            for (int j = 0; j < ntiles && ok; ++j) {
-                const int tk = 2 * j, kslot = tk % kSlots;
-                ok = mbar_wait(bar(B_FULL0 + kslot), (tk / kSlots) & 1, ctl, a.status);
+            int tg = 0, it = 0, pc = 0;   // ring loads consumed, key tiles issued, pieces so far
+            bool ok = true;
+            int kt0, ntiles;
+            for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
+                if (ntiles <= 0) continue;
+                ok = mbar_wait(bar(B_QFULL), pc & 1, ctl, a.status);
                 if (!ok) break;
                 tc_fence_after();
-                for (int i = 0; i < 2 && ok; ++i) {
-                    if (j > 0) {
-                        const int tv = 2 * (j - 1) + 1, vslot = tv % kSlots;
-                        if (i == 0) ok = mbar_wait(bar(B_FULL0 + vslot), (tv / kSlots) & 1, ctl, a.status);
-                        if (ok) ok = mbar_wait(bar(B_PFULL0 + i), (j - 1) & 1, ctl, a.status);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_pv(i, vslot, j - 1 > 0);
-                        if (i == 1) tc_commit(bar(B_EMPTY0 + vslot));
-                    }
-                    issue_qk(i, kslot);
-                    tc_commit(bar(B_SFULL0 + i));
-                    if (i == 1) tc_commit(bar(B_EMPTY0 + kslot));
-                }
-            }
-            if (ok) {
-                const int j = ntiles - 1, tv = 2 * j + 1, vslot = tv % kSlots;
-                ok = mbar_wait(bar(B_FULL0 + vslot), (tv / kSlots) & 1, ctl, a.status);
-                for (int i = 0; i < 2 && ok; ++i) {
-                    ok = mbar_wait(bar(B_PFULL0 + i), j & 1, ctl, a.status);
+                for (int j = 0; j < ntiles && ok; ++j, ++it) {
+                    const int tk = tg + 2 * j, kslot = tk % kSlots;
+                    ok = mbar_wait(bar(B_FULL0 + kslot), (tk / kSlots) & 1, ctl, a.status);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(i, vslot, j > 0);
-                    tc_commit(bar(B_OFINAL0 + i));
+                    for (int i = 0; i < 2 && ok; ++i) {
+                        if (j > 0) {
+                            const int tv = tk - 1, vslot = tv % kSlots;
+                            if (i == 0) ok = mbar_wait(bar(B_FULL0 + vslot), (tv / kSlots) & 1, ctl, a.status);
+                            if (ok) ok = mbar_wait(bar(B_PA0 + i), (it - 1) & 1, ctl, a.status);
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_pv_half(i, vslot, 0, j - 1 > 0);
+                            ok = mbar_wait(bar(B_PB0 + i), (it - 1) & 1, ctl, a.status);
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_pv_half(i, vslot, 1, true);
+                            if (i == 1) tc_commit(bar(B_EMPTY0 + vslot));
+                        }
+                        issue_qk(i, kslot);
+                        tc_commit(bar(B_SFULL0 + i));
+                        if (i == 1) tc_commit(bar(B_EMPTY0 + kslot));
+                    }
                 }
+                if (!ok) break;
+                tc_commit(bar(B_QEMPTY));          // every Q K^T of this piece has been issued
+                {
+                    const int tv = tg + 2 * ntiles - 1, vslot = tv % kSlots;
+                    ok = mbar_wait(bar(B_FULL0 + vslot), (tv / kSlots) & 1, ctl, a.status);
+                    for (int i = 0; i < 2 && ok; ++i) {
+                        ok = mbar_wait(bar(B_PA0 + i), (it - 1) & 1, ctl, a.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv_half(i, vslot, 0, ntiles > 1);
+                        ok = mbar_wait(bar(B_PB0 + i), (it - 1) & 1, ctl, a.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv_half(i, vslot, 1, true);
+                        tc_commit(bar(B_OFINAL0 + i));
+                        if (i == 1) tc_commit(bar(B_EMPTY0 + vslot));
+                    }
+                }
+                tg += 2 * ntiles;
+                ++pc;
             }
         }
     } else {
@@ -314,86 +413,136 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         const bool valid = tok < n;
         const int64_t limit = valid ? P + tok + 1 : 0;  // keys below `limit` are visible
         const float sl2 = a.scale_log2;
+        const float2 sl2v = make_float2(sl2, sl2);
+        const int64_t nG = (int64_t)n * G;
 
-        float m_ref = -INFINITY;   // reference maximum (raw score units) the probabilities are scaled by
-        float l = 0.f;
+        int it = 0, pc = 0;
         bool ok = true;
-        for (int j = 0; j < ntiles; ++j) {
-            ok = mbar_wait(bar(B_SFULL0 + i), j & 1, ctl, a.status);
+        int kt0, ntiles;
+        for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
+            const int64_t prow = (int64_t)(group + kvh) * nG + R;     // row of this piece's partial slot
+            if (ntiles <= 0) {
+                // no visible key for these rows in this range: an empty partial
+                if (!direct && valid) {
+                    float4 *po = reinterpret_cast<float4 *>(a.part_o + prow * kD);
+#pragma unroll 4
+                    for (int c = 0; c < kD / 4; ++c) po[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    a.part_lse[prow] = -INFINITY;
+                }
+                continue;
+            }
+            float m_ref = -INFINITY;   // reference maximum (raw score units) the probabilities are scaled by
+            float l = 0.f;
+            for (int j = 0; j < ntiles; ++j, ++it) {
+                ok = mbar_wait(bar(B_SFULL0 + i), it & 1, ctl, a.status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const int64_t key0 = (int64_t)(kt0 + j) * kRows;
+                const int nvis = (int)max((int64_t)0, min((int64_t)kRows, limit - key0));
+                const bool masked = __any_sync(0xffffffffu, nvis < kRows);
+
+                // ---- pass 1: row maximum, 32 columns at a time, the next load in flight
+                uint32_t va[32], vb[32];
+                float mx0 = -INFINITY, mx1 = -INFINITY;
+                auto max_chunk = [&](const uint32_t (&v)[32], int col0) {
+                    if (masked) {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4) {
+                            mx0 = max3(mx0, col0 + c < nvis ? __uint_as_float(v[c]) : -INFINITY,
+                                       col0 + c + 1 < nvis ? __uint_as_float(v[c + 1]) : -INFINITY);
+                            mx1 = max3(mx1, col0 + c + 2 < nvis ? __uint_as_float(v[c + 2]) : -INFINITY,
+                                       col0 + c + 3 < nvis ? __uint_as_float(v[c + 3]) : -INFINITY);
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4) {
+                            mx0 = max3(mx0, __uint_as_float(v[c]), __uint_as_float(v[c + 1]));
+                            mx1 = max3(mx1, __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
+                        }
+                    }
+                };
+                KVF_TMEM_LD32(va, 0, t_s);
+                tmem_wait_ld();
+                KVF_TMEM_LD32(vb, 0, t_s + 32);
+                max_chunk(va, 0);
+                tmem_wait_ld();
+                KVF_TMEM_LD32(va, 0, t_s + 64);
+                max_chunk(vb, 32);
+                tmem_wait_ld();
+                KVF_TMEM_LD32(vb, 0, t_s + 96);
+                max_chunk(va, 64);
+                tmem_wait_ld();
+                KVF_TMEM_LD32(va, 0, t_s);        // pass 2 starts while the maximum is settled
+                max_chunk(vb, 96);
+                const float m_tile = fmaxf(mx0, mx1);
+                // move the reference only when the maximum grew by more than the threshold: the
+                // probabilities then stay below 2^threshold and the accumulator is rarely rescaled
+                const bool grow = (m_tile - m_ref) * sl2 > kRescaleThreshold;   // also true when m_ref = -inf < m_tile
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float m_new = grow ? m_tile : m_ref;
+                    const float alpha = grow ? ex2((m_ref - m_new) * sl2) : 1.f;   // m_ref = -inf -> 0
+                    l *= alpha;
+                    m_ref = m_new;
+                    if (j > 0) {
+                        // the commit that completed S(j) also covers PV(j-1): O is quiescent here
+                        const float2 av = make_float2(alpha, alpha);
+#pragma unroll 1
+                        for (int c0 = 0; c0 < 128; c0 += 32) {
+                            KVF_TMEM_LD32(vb, 0, t_o + c0);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; c += 2) {
+                                const float2 v = __fmul2_rn(make_float2(__uint_as_float(vb[c]), __uint_as_float(vb[c + 1])), av);
+                                vb[c] = __float_as_uint(v.x);
+                                vb[c + 1] = __float_as_uint(v.y);
+                            }
+                            KVF_TMEM_ST32(vb, 0, t_o + c0);
+                        }
+                        tmem_wait_st();
+                    }
+                }
+                const float m_safe = m_ref == -INFINITY ? 0.f : m_ref;
+                const float neg = -m_safe * sl2;
+                const float2 negv = make_float2(neg, neg);
+                float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+
+                // ---- pass 2: probabilities; the first 64 keys are handed over before the rest
+                uint32_t p[32];
+                tmem_wait_ld();
+                KVF_TMEM_LD32(vb, 0, t_s + 32);
+                if (masked) exp_chunk<0>(va, p, sl2v, negv, nvis, acc0, acc1);
+                else exp_chunk<kEmu>(va, p, sl2v, negv, 32, acc0, acc1);
+                tmem_wait_ld();
+                KVF_TMEM_LD32(va, 0, t_s + 64);
+                if (masked) exp_chunk<0>(vb, p + 16, sl2v, negv, nvis - 32, acc0, acc1);
+                else exp_chunk<kEmu>(vb, p + 16, sl2v, negv, 32, acc0, acc1);
+                tmem_wait_ld();                      // columns 64..95 are in registers before P lands on 0..31
+                KVF_TMEM_LD32(vb, 0, t_s + 96);
+                KVF_TMEM_ST32(p, 0, t_s);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_PA0 + i));
+                if (masked) exp_chunk<0>(va, p, sl2v, negv, nvis - 64, acc0, acc1);
+                else exp_chunk<kEmu>(va, p, sl2v, negv, 32, acc0, acc1);
+                tmem_wait_ld();                      // columns 96..127 are in registers before P lands on 32..63
+                if (masked) exp_chunk<0>(vb, p + 16, sl2v, negv, nvis - 96, acc0, acc1);
+                else exp_chunk<kEmu>(vb, p + 16, sl2v, negv, 32, acc0, acc1);
+                KVF_TMEM_ST32(p, 0, t_s + 32);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_PB0 + i));
+                const float2 acc = __fadd2_rn(acc0, acc1);
+                l += acc.x + acc.y;
+            }
+            if (!ok) break;
+
+            ok = mbar_wait(bar(B_OFINAL0 + i), pc & 1, ctl, a.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            tc_fence_after();
-            uint32_t s[128];
-            KVF_TMEM_LD32(s, 0, t_s);
-            KVF_TMEM_LD32(s, 32, t_s + 32);
-            KVF_TMEM_LD32(s, 64, t_s + 64);
-            KVF_TMEM_LD32(s, 96, t_s + 96);
-            tmem_wait_ld();
-
-            const int64_t key0 = (int64_t)(kt0 + j) * kRows;
-            const int nvis = (int)max((int64_t)0, min((int64_t)kRows, limit - key0));
-            if (nvis < kRows) {
-#pragma unroll
-                for (int c = 0; c < 128; ++c) s[c] = c < nvis ? s[c] : 0xFF800000u;   // -inf
-            }
-            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 128; c += 4) {
-                mx0 = fmaxf(mx0, __uint_as_float(s[c]));
-                mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
-                mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
-                mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
-            }
-            const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-            // move the reference only when the maximum grew by more than the threshold: the
-            // probabilities then stay below 2^threshold and the accumulator is rarely rescaled
-            const bool grow = (m_tile - m_ref) * sl2 > kRescaleThreshold;   // also true when m_ref = -inf < m_tile
-            if (__any_sync(0xffffffffu, grow)) {
-                const float m_new = grow ? m_tile : m_ref;
-                const float alpha = grow ? ex2((m_ref - m_new) * sl2) : 1.f;   // m_ref = -inf -> 0
-                l *= alpha;
-                m_ref = m_new;
-                if (j > 0) {
-                    // the commit that completed S(j) also covers PV(j-1): O is quiescent here
-#pragma unroll
-                    for (int c0 = 0; c0 < 128; c0 += 32) {
-                        uint32_t o[32];
-                        KVF_TMEM_LD32(o, 0, t_o + c0);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                        KVF_TMEM_ST32(o, 0, t_o + c0);
-                    }
-                    tmem_wait_st();
-                }
-            }
-            const float m_safe = m_ref == -INFINITY ? 0.f : m_ref;
-            const float neg = -m_safe * sl2;
-            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-#pragma unroll
-            for (int c4 = 0; c4 < 32; ++c4) {
-                const float p0 = ex2(fmaf(__uint_as_float(s[c4 * 4 + 0]), sl2, neg));
-                const float p1 = ex2(fmaf(__uint_as_float(s[c4 * 4 + 1]), sl2, neg));
-                const float p2 = ex2(fmaf(__uint_as_float(s[c4 * 4 + 2]), sl2, neg));
-                const float p3 = ex2(fmaf(__uint_as_float(s[c4 * 4 + 3]), sl2, neg));
-                sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
-                __nv_bfloat162 b0 = __floats2bfloat162_rn(p0, p1), b1 = __floats2bfloat162_rn(p2, p3);
-                s[c4 * 2 + 0] = *reinterpret_cast<uint32_t *>(&b0);   // packed pair (2c, 2c+1) -> column c
-                s[c4 * 2 + 1] = *reinterpret_cast<uint32_t *>(&b1);
-            }
-            l += (sum0 + sum1) + (sum2 + sum3);
-            KVF_TMEM_ST32(s, 0, t_s);
-            KVF_TMEM_ST32(s, 32, t_s + 32);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(B_PFULL0 + i));
-        }
-
-        if (ok) {
-            ok = mbar_wait(bar(B_OFINAL0 + i), 0, ctl, a.status);
-            ok = __all_sync(0xffffffffu, ok);
-        }
-        if (ok) {
+            ++pc;
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
             const float lse2 = l > 0.f ? m_ref * sl2 + log2f(l) : -INFINITY;
@@ -404,8 +553,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 KVF_TMEM_LD32(o, 0, t_o + c0);
                 tmem_wait_ld();
                 if (!valid) continue;
-                if (a.splits > 1) {
-                    float4 *dst = reinterpret_cast<float4 *>(a.part_o + ((int64_t)split * n * a.H + row) * kD + c0);
+                if (!direct) {
+                    float4 *dst = reinterpret_cast<float4 *>(a.part_o + prow * kD + c0);
 #pragma unroll
                     for (int c = 0; c < 8; ++c)
                         dst[c] = make_float4(__uint_as_float(o[4 * c]) * inv, __uint_as_float(o[4 * c + 1]) * inv,
@@ -422,19 +571,18 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                     for (int c = 0; c < 4; ++c) {
                         uint32_t w[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(o[8 * c + 2 * e]) * inv,
-                                                                     __uint_as_float(o[8 * c + 2 * e + 1]) * inv);
-                            w[e] = *reinterpret_cast<uint32_t *>(&b);
-                        }
+                        for (int e = 0; e < 4; ++e)
+                            w[e] = pack_bf16(__uint_as_float(o[8 * c + 2 * e]) * inv, __uint_as_float(o[8 * c + 2 * e + 1]) * inv);
                         dst[c] = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
             }
             if (valid) {
-                if (a.splits > 1) a.part_lse[(int64_t)split * n * a.H + row] = lse2;
+                if (!direct) a.part_lse[prow] = lse2;
                 else if (a.lse) a.lse[row] = lse2 * 0.6931471805599453f;
             }
+            // the next piece's first P V (which overwrites O) is issued only after all 128 rows
+            // have handed over its probabilities, i.e. after these loads
         }
     }
 
@@ -446,21 +594,90 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     }
 }
 
+// Merge the pieces of each KV head.  Group g owns [g * line / ngroups, (g+1) * line / ngroups) of
+// the (KV head, key tile) line, its piece for KV head h sits in slot g + h.  With lse_s = log2 of
+// a piece's softmax denominator and O_s its normalised output,
+//   O = sum_s 2^(lse_s - M) O_s / sum_s 2^(lse_s - M),  M = max_s lse_s,  in group order.
+__global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // (row, float4 column)
+    const int64_t rows = (int64_t)a.n * a.H;
+    if (idx >= rows * (kD / 4)) return;
+    const int64_t row = idx / (kD / 4);
+    const int c = (int)(idx % (kD / 4));
+    const int tok = (int)(row / a.H), h = (int)(row % a.H), kvh = h / a.G, gi = h % a.G;
+    const int64_t nG = (int64_t)a.n * a.G, R = (int64_t)tok * a.G + gi;
+    const int nt_all = (int)((a.prefix + a.n + kRows - 1) / kRows);
+    const int64_t line = (int64_t)a.Hkv * nt_all;
+    auto start = [&](int64_t g) { return g * line / a.ngroups; };
+    auto group_of = [&](int64_t lin) {
+        int64_t g = lin * a.ngroups / line;
+        while (g > 0 && start(g) > lin) --g;
+        while (g + 1 < a.ngroups && start(g + 1) <= lin) ++g;
+        return (int)g;
+    };
+    const int g0 = group_of((int64_t)kvh * nt_all), g1 = group_of((int64_t)(kvh + 1) * nt_all - 1);
+    float M = -INFINITY;
+    for (int g = g0; g <= g1; ++g) M = fmaxf(M, a.part_lse[(int64_t)(g + kvh) * nG + R]);
+    float den = 0.f;
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int g = g0; g <= g1; ++g) {
+        const int64_t prow = (int64_t)(g + kvh) * nG + R;
+        const float ls = a.part_lse[prow];
+        if (ls == -INFINITY) continue;
+        const float w = exp2f(ls - M);
+        const float4 p = *reinterpret_cast<const float4 *>(a.part_o + prow * kD + c * 4);
+        den += w;
+        o.x = fmaf(w, p.x, o.x); o.y = fmaf(w, p.y, o.y); o.z = fmaf(w, p.z, o.z); o.w = fmaf(w, p.w, o.w);
+    }
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+    o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
+    if (a.out_f32) {
+        *reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.out) + row * kD + c * 4) = o;
+    } else {
+        uint2 pk;
+        pk.x = pack_bf16(o.x, o.y);
+        pk.y = pack_bf16(o.z, o.w);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.out) + row * kD + c * 4) = pk;
+    }
+    if (c == 0 && a.lse) a.lse[row] = (M + log2f(den)) * 0.6931471805599453f;
+}
+
+template <int kEmu>
+cudaError_t launch_t(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<kEmu>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, 1);
+    attn_tc_kernel<kEmu><<<grid, kThreads, kSmemBytes, s>>>(a, maps.q, maps.k, maps.v);
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 bool attn_tc_supported(int dtype, int d, int G) {
     return dtype == 0 && d == kD && G >= 1 && G <= 64 && (G & (G - 1)) == 0;
 }
 
-int attn_tc_ctas(int n, int G, int Hkv, int splits) { return ((n * G + 2 * kRows - 1) / (2 * kRows)) * Hkv * splits; }
+int attn_tc_row_pairs(int n, int G) { return (n * G + 2 * kRows - 1) / (2 * kRows); }
 
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
     static_assert(sizeof(Ctl) <= 256, "control block");
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    dim3 grid((a.n * a.G + 2 * kRows - 1) / (2 * kRows), a.Hkv, a.splits);
-    attn_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(a, maps.q, maps.k, maps.v);
+    static const int emu = [] {
+        const char *v = getenv("KVF_EMU");
+        return v ? atoi(v) : 1;
+    }();
+    switch (emu) {
+        case 0: return launch_t<0>(a, maps, s);
+        case 2: return launch_t<2>(a, maps, s);
+        case 3: return launch_t<3>(a, maps, s);
+        case 4: return launch_t<4>(a, maps, s);
+        default: return launch_t<1>(a, maps, s);
+    }
+}
+
+cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s) {
+    const int64_t items = (int64_t)a.n * a.H * (kD / 4);
+    combine_groups_kernel<<<(int)((items + 255) / 256), 256, 0, s>>>(a);
     return cudaGetLastError();
 }
 

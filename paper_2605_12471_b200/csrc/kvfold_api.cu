@@ -92,6 +92,7 @@ struct kvf_cache {
     bool tc;
     TcMaps maps;
     int force_splits;
+    int64_t part_rows_cap;   // rows of head_dim floats the partial area holds
     uint64_t launches;
     bool profile;
     std::vector<ProfRec> recs;
@@ -150,20 +151,44 @@ kvf_status build_maps(kvf_cache *c) {
 
 struct Plan {
     bool tc;
-    int splits, ctas, kernels;
+    int splits;    // CUDA-core path: splits of the key range; tensor-core path: ranges per KV head (rounded up)
+    int ngroups;   // tensor-core path: ranges of the (KV head, key tile) line
+    int ctas, kernels;
 };
 
 Plan make_plan(const kvf_cache *c, int n, int64_t prefix) {
     Plan p;
     p.tc = c->tc;
+    p.ngroups = 0;
     const int64_t L = prefix + n;
-    const int key_tile = p.tc ? kKvTile : 64;
-    const int64_t nt = (L + key_tile - 1) / key_tile;
-    const int units = p.tc ? attn_tc_ctas(n, c->G, c->cfg.n_kv_heads, 1)
-                           : attn_simt_ctas(n, c->G, c->cfg.n_kv_heads, 1);
-    const int per_sm = p.tc ? 1 : 2;
-    const int target = c->sm_count * per_sm;
-    int max_splits = kPartTokens / n;
+    const int Hkv = c->cfg.n_kv_heads;
+    if (p.tc) {
+        // one CTA per (row pair, group); the groups cut the Hkv * nt line of (KV head, key tile)
+        // into equal ranges.  Whole KV heads if that fills the SMs, else as many groups as give
+        // one CTA per SM, with at least 4 key tiles each and within the partial area.
+        const int64_t nt = (L + kKvTile - 1) / kKvTile;
+        const int pairs = attn_tc_row_pairs(n, c->G);
+        int64_t groups = Hkv;
+        if (c->force_splits > 0) {
+            groups = (int64_t)Hkv * c->force_splits;
+        } else if (pairs * Hkv < c->sm_count) {
+            groups = c->sm_count / pairs;
+            if (groups > Hkv * nt / 4) groups = Hkv * nt / 4;
+        }
+        const int64_t slots_cap = c->part_rows_cap / ((int64_t)n * c->G);   // slots = groups + Hkv - 1
+        if (groups + Hkv - 1 > slots_cap) groups = slots_cap - (Hkv - 1);
+        if (groups > Hkv * nt) groups = Hkv * nt;
+        if (groups < Hkv) groups = Hkv;
+        p.ngroups = (int)groups;
+        p.splits = (int)((groups + Hkv - 1) / Hkv);
+        p.ctas = pairs * p.ngroups;
+        p.kernels = 2 + (p.ngroups != Hkv ? 1 : 0);
+        return p;
+    }
+    const int64_t nt = (L + 63) / 64;
+    const int units = attn_simt_ctas(n, c->G, Hkv, 1);
+    const int target = c->sm_count * 2;
+    int64_t max_splits = c->part_rows_cap / ((int64_t)n * c->cfg.n_q_heads);
     if (max_splits > kMaxSplits) max_splits = kMaxSplits;
     if (max_splits < 1) max_splits = 1;
     int splits = 1;
@@ -177,7 +202,7 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix) {
         if (want > cap) want = (int)cap;
         splits = want;
     }
-    if (splits > max_splits) splits = max_splits;
+    if (splits > max_splits) splits = (int)max_splits;
     if ((int64_t)splits > nt) splits = (int)nt;
     if (splits < 1) splits = 1;
     p.splits = splits;
@@ -255,7 +280,8 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.status = reinterpret_cast<int *>(c->workspace + c->lay.status);
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
-    aa.splits = plan.splits;
+    aa.splits = plan.tc ? 1 : plan.splits;
+    aa.ngroups = plan.ngroups;
     aa.out_f32 = (f.dtype == KVF_F32 || (f.flags & KVF_OUT_F32)) ? 1 : 0;
     aa.scale_log2 = c->scale_log2;
 
@@ -273,10 +299,10 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     }
     if (e != cudaSuccess) return cuda_fail(e, "attention launch");
     c->launches++;
-    if (plan.splits > 1) {
+    if (plan.kernels > 2) {
         {
             ProfScope ps(c, st, 2);
-            e = launch_combine(aa, f.dtype, st);
+            e = plan.tc ? launch_combine_groups(aa, st) : launch_combine(aa, f.dtype, st);
         }
         if (e != cudaSuccess) return cuda_fail(e, "combine launch");
         c->launches++;
@@ -346,6 +372,7 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
                                              : std::pow(cfg->rope_base, -2.0 * (double)j / (double)cfg->head_dim);
     for (int j = cfg->head_dim / 2; j < kMaxHalfDim; ++j) c->table.inv_freq[j] = 0.0;
     c->force_splits = 0;
+    c->part_rows_cap = (int64_t)kPartTokens * cfg->n_q_heads;
     c->launches = 0;
     c->profile = false;
     c->tc = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, c->G);
@@ -580,6 +607,7 @@ extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_stor
                                             : std::pow(cfg->rope_base, -2.0 * (double)j / (double)cfg->head_dim);
     for (int j = cfg->head_dim / 2; j < kMaxHalfDim; ++j) c.table.inv_freq[j] = 0.0;
     c.force_splits = 0;
+    c.part_rows_cap = (int64_t)part_tokens * cfg->n_q_heads;   // the plan splits only as far as this holds
     c.launches = 0;
     c.profile = false;
     c.tc = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, c.G);
@@ -587,10 +615,6 @@ extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_stor
         s = build_maps(&c);
         if (s != KVF_OK) return s;
     }
-    // the split count the ordinary step would take, limited to what the partial area holds
-    Plan plan = make_plan(&c, n_tokens, len);
-    const int fit = (int)(part_tokens / (size_t)n_tokens);
-    c.force_splits = plan.splits < fit ? plan.splits : fit;
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     // the array keeps what the last call left: the status word has to start at zero

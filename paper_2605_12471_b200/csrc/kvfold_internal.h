@@ -9,8 +9,8 @@ namespace kvf {
 
 constexpr int kMaxHalfDim = 64;       // head_dim <= 128
 constexpr int kKvTile = 128;          // key rows per tensor-core tile; V rows are zero-padded to it
-constexpr int kPartTokens = 4096;     // split partials are sized for (splits * n_tokens) <= this
-constexpr int kMaxSplits = 64;
+constexpr int kPartTokens = 4096;     // the partial area holds kPartTokens * H rows of head_dim floats
+constexpr int kMaxSplits = 64;        // CUDA-core path: most splits of the key range
 
 struct RopeTable {
     double inv_freq[kMaxHalfDim];
@@ -33,12 +33,14 @@ struct AttnArgs {
     const void *k_plane, *v_plane;   // [Hkv][capacity][d]
     void *out;                       // [n][H][d], dtype or fp32
     float *lse;                      // [n][H] or null (natural log)
-    float *part_o;                   // [splits][n][H][d] fp32, normalised per split
-    float *part_lse;                 // [splits][n][H] fp32, log2 domain; -inf = split saw no key
+    float *part_o;                   // partial outputs, fp32, normalised per part: CUDA-core path
+                                     // [splits][n][H][d]; tensor-core path [slot][n * G][d]
+    float *part_lse;                 // log2 denominators of the parts, same order; -inf = no key seen
     int *status;                     // device status word
     int64_t capacity, prefix;
     int32_t n, H, Hkv, G, d;
-    int32_t splits;
+    int32_t splits;                  // CUDA-core path: equal splits of the key range
+    int32_t ngroups;                 // tensor-core path: contiguous ranges of the (KV head, key tile) line
     int32_t out_f32;
     float scale_log2;                // softmax scale * log2(e)
 };
@@ -53,7 +55,8 @@ struct TcMaps {
     CUtensorMap q, k, v;
 };
 bool attn_tc_supported(int dtype, int d, int G);
-int attn_tc_ctas(int n, int G, int Hkv, int splits);
-cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s);
+int attn_tc_row_pairs(int n, int G);   // 256-row pairs per KV head = grid.x
+cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s);   // grid (row pairs, ngroups)
+cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s);                // needed when ngroups != Hkv
 
 }  // namespace kvf
