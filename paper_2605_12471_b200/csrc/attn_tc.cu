@@ -17,9 +17,11 @@
 // normalised partial output and its log2 denominator to slot (group + KV head) and the combine
 // kernel below merges the slots of each KV head in order.
 //
-// Roles (320 threads): warps 0-3 / 4-7 softmax of row tile 0 / 1 (one thread per row; TMEM lane
+// Roles (384 threads): warps 0-3 / 4-7 softmax of row tile 0 / 1 (one thread per row; TMEM lane
 // = row), warp 8 TMA producer (Q per piece, then K(j), V(j), ... through a 5-slot ring), warp 9
-// tcgen05.mma issuer and owner of the TMEM allocation.
+// tcgen05.mma issuer and owner of the TMEM allocation; warps 10-11 only complete the third
+// warpgroup, which hands registers to the softmax warpgroups (setmaxnreg 72 / 216) so that a
+// whole 128-column score row stays in registers after one tensor-memory load.
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each.  The bf16 probabilities
 // overwrite the first 64 columns of their own S tile, in two halves that are handed to the
 // second MMA separately, and feed it straight from tensor memory; the tensor pipe runs one
@@ -48,7 +50,7 @@ constexpr int kD = 128;                       // head_dim
 constexpr uint32_t kPanel = 128 * 128;        // bytes of a [128 rows][64 bf16] swizzled panel
 constexpr uint32_t kTileBytes = 2 * kPanel;   // a 128 x 128 bf16 tile = two panels
 constexpr int kSlots = 5;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;
 constexpr uint32_t kOffQ = 0;                         // 2 tiles
 constexpr uint32_t kOffKV = 2 * kTileBytes;           // kSlots tiles
 constexpr uint32_t kOffCtl = kOffKV + kSlots * kTileBytes;
@@ -95,7 +97,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 
 // Bounded wait.  Returns false if the CTA is aborting or the limit ran out.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, Ctl *ctl, int *status) {
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, Ctl *ctl, int *status) {
     const unsigned long long t0 = global_ns();
     unsigned spins = 0;
     while (true) {
@@ -216,23 +218,18 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
 
-// 32 scores of a row -> 16 packed bf16 probability pairs in p[0..15]; their sum goes to acc.
-// kEmu of every 4 pairs take the FMA-pipe exponential.  nvis_here < 32 masks the tail of the
-// chunk (those tiles use kEmu = 0, so a masked score gives exactly 0).
+// 64 scores of a row -> 32 packed bf16 probability pairs in p[0..31]; their sum goes to acc.
+// kEmu of every 4 pairs take the FMA-pipe exponential (0 on masked tiles, where a masked score,
+// already set to -inf, must give exactly 0).
 template <int kEmu>
-__device__ __forceinline__ void exp_chunk(const uint32_t (&v)[32], uint32_t *p, float2 sl2v, float2 negv, int nvis_here,
-                                          float2 &acc0, float2 &acc1) {
+__device__ __forceinline__ void exp_half(const uint32_t *v, uint32_t *p, float2 sl2v, float2 negv, float2 &acc0, float2 &acc1) {
 #pragma unroll
-    for (int c = 0; c < 16; ++c) {
-        float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1])), sl2v, negv);
+    for (int c = 0; c < 32; ++c) {
+        const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1])), sl2v, negv);
         float2 e;
         if ((c & 3) < kEmu) {
             e = exp2_fma2(x);
         } else {
-            if (kEmu == 0) {
-                x.x = 2 * c < nvis_here ? x.x : -INFINITY;
-                x.y = 2 * c + 1 < nvis_here ? x.y : -INFINITY;
-            }
             e.x = ex2(x.x);
             e.y = ex2(x.y);
         }
@@ -300,6 +297,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&ctl->tmem_base);
 
     if (warp >= 8) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
         if (warp == 8 && lane == 0) {
             // ------------------------------------------------------------------ TMA producer
             int tg = 0, pc = 0;          // ring loads and pieces so far
@@ -404,6 +402,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         }
     } else {
         // ------------------------------------------------------------------ softmax, one thread per row
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         const int i = warp >> 2;                        // row tile
         const int r = (warp & 3) * 32 + lane;           // row in the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
@@ -442,39 +441,23 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 const int nvis = (int)max((int64_t)0, min((int64_t)kRows, limit - key0));
                 const bool masked = __any_sync(0xffffffffu, nvis < kRows);
 
-                // ---- pass 1: row maximum, 32 columns at a time, the next load in flight
-                uint32_t va[32], vb[32];
+                // the whole score row in registers after one load
+                uint32_t sc[128];
+                KVF_TMEM_LD32(sc, 0, t_s);
+                KVF_TMEM_LD32(sc, 32, t_s + 32);
+                KVF_TMEM_LD32(sc, 64, t_s + 64);
+                KVF_TMEM_LD32(sc, 96, t_s + 96);
+                tmem_wait_ld();
+                if (masked) {
+#pragma unroll
+                    for (int c = 0; c < 128; ++c) sc[c] = c < nvis ? sc[c] : 0xFF800000u;   // -inf
+                }
                 float mx0 = -INFINITY, mx1 = -INFINITY;
-                auto max_chunk = [&](const uint32_t (&v)[32], int col0) {
-                    if (masked) {
 #pragma unroll
-                        for (int c = 0; c < 32; c += 4) {
-                            mx0 = max3(mx0, col0 + c < nvis ? __uint_as_float(v[c]) : -INFINITY,
-                                       col0 + c + 1 < nvis ? __uint_as_float(v[c + 1]) : -INFINITY);
-                            mx1 = max3(mx1, col0 + c + 2 < nvis ? __uint_as_float(v[c + 2]) : -INFINITY,
-                                       col0 + c + 3 < nvis ? __uint_as_float(v[c + 3]) : -INFINITY);
-                        }
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 32; c += 4) {
-                            mx0 = max3(mx0, __uint_as_float(v[c]), __uint_as_float(v[c + 1]));
-                            mx1 = max3(mx1, __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
-                        }
-                    }
-                };
-                KVF_TMEM_LD32(va, 0, t_s);
-                tmem_wait_ld();
-                KVF_TMEM_LD32(vb, 0, t_s + 32);
-                max_chunk(va, 0);
-                tmem_wait_ld();
-                KVF_TMEM_LD32(va, 0, t_s + 64);
-                max_chunk(vb, 32);
-                tmem_wait_ld();
-                KVF_TMEM_LD32(vb, 0, t_s + 96);
-                max_chunk(va, 64);
-                tmem_wait_ld();
-                KVF_TMEM_LD32(va, 0, t_s);        // pass 2 starts while the maximum is settled
-                max_chunk(vb, 96);
+                for (int c = 0; c < 128; c += 4) {
+                    mx0 = max3(mx0, __uint_as_float(sc[c]), __uint_as_float(sc[c + 1]));
+                    mx1 = max3(mx1, __uint_as_float(sc[c + 2]), __uint_as_float(sc[c + 3]));
+                }
                 const float m_tile = fmaxf(mx0, mx1);
                 // move the reference only when the maximum grew by more than the threshold: the
                 // probabilities then stay below 2^threshold and the accumulator is rarely rescaled
@@ -489,15 +472,16 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                         const float2 av = make_float2(alpha, alpha);
 #pragma unroll 1
                         for (int c0 = 0; c0 < 128; c0 += 32) {
-                            KVF_TMEM_LD32(vb, 0, t_o + c0);
+                            uint32_t o[32];
+                            KVF_TMEM_LD32(o, 0, t_o + c0);
                             tmem_wait_ld();
 #pragma unroll
                             for (int c = 0; c < 32; c += 2) {
-                                const float2 v = __fmul2_rn(make_float2(__uint_as_float(vb[c]), __uint_as_float(vb[c + 1])), av);
-                                vb[c] = __float_as_uint(v.x);
-                                vb[c + 1] = __float_as_uint(v.y);
+                                const float2 v = __fmul2_rn(make_float2(__uint_as_float(o[c]), __uint_as_float(o[c + 1])), av);
+                                o[c] = __float_as_uint(v.x);
+                                o[c + 1] = __float_as_uint(v.y);
                             }
-                            KVF_TMEM_ST32(vb, 0, t_o + c0);
+                            KVF_TMEM_ST32(o, 0, t_o + c0);
                         }
                         tmem_wait_st();
                     }
@@ -507,28 +491,17 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 const float2 negv = make_float2(neg, neg);
                 float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 
-                // ---- pass 2: probabilities; the first 64 keys are handed over before the rest
+                // probabilities; the first 64 keys are handed over before the rest is computed
                 uint32_t p[32];
-                tmem_wait_ld();
-                KVF_TMEM_LD32(vb, 0, t_s + 32);
-                if (masked) exp_chunk<0>(va, p, sl2v, negv, nvis, acc0, acc1);
-                else exp_chunk<kEmu>(va, p, sl2v, negv, 32, acc0, acc1);
-                tmem_wait_ld();
-                KVF_TMEM_LD32(va, 0, t_s + 64);
-                if (masked) exp_chunk<0>(vb, p + 16, sl2v, negv, nvis - 32, acc0, acc1);
-                else exp_chunk<kEmu>(vb, p + 16, sl2v, negv, 32, acc0, acc1);
-                tmem_wait_ld();                      // columns 64..95 are in registers before P lands on 0..31
-                KVF_TMEM_LD32(vb, 0, t_s + 96);
+                if (masked) exp_half<0>(sc, p, sl2v, negv, acc0, acc1);
+                else exp_half<kEmu>(sc, p, sl2v, negv, acc0, acc1);
                 KVF_TMEM_ST32(p, 0, t_s);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B_PA0 + i));
-                if (masked) exp_chunk<0>(va, p, sl2v, negv, nvis - 64, acc0, acc1);
-                else exp_chunk<kEmu>(va, p, sl2v, negv, 32, acc0, acc1);
-                tmem_wait_ld();                      // columns 96..127 are in registers before P lands on 32..63
-                if (masked) exp_chunk<0>(vb, p + 16, sl2v, negv, nvis - 96, acc0, acc1);
-                else exp_chunk<kEmu>(vb, p + 16, sl2v, negv, 32, acc0, acc1);
+                if (masked) exp_half<0>(sc + 64, p, sl2v, negv, acc0, acc1);
+                else exp_half<kEmu>(sc + 64, p, sl2v, negv, acc0, acc1);
                 KVF_TMEM_ST32(p, 0, t_s + 32);
                 tmem_wait_st();
                 tc_fence_before();
@@ -664,7 +637,7 @@ cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
     static const int emu = [] {
         const char *v = getenv("KVF_EMU");
-        return v ? atoi(v) : 1;
+        return v ? atoi(v) : 0;
     }();
     switch (emu) {
         case 0: return launch_t<0>(a, maps, s);
