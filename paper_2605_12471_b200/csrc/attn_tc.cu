@@ -18,15 +18,16 @@
 // kernel below merges the slots of each KV head in order.
 //
 // Roles (384 threads): warps 0-3 / 4-7 softmax of row tile 0 / 1 (one thread per row; TMEM lane
-// = row), warp 8 TMA producer (Q per piece, then K(j), V(j), ... through a 5-slot ring), warp 9
-// tcgen05.mma issuer and owner of the TMEM allocation; warps 10-11 only complete the third
-// warpgroup, which hands registers to the softmax warpgroups (setmaxnreg 72 / 216) so that a
-// whole 128-column score row stays in registers after one tensor-memory load.
+// = row), warp 8 TMA producer (Q per piece, then K(j), V(j), ... through a 5-slot ring), warps 9
+// and 10 tcgen05.mma issuers of row tile 0 and 1 (warp 9 owns the TMEM allocation); warp 11 only
+// completes the third warpgroup, which hands registers to the softmax warpgroups (setmaxnreg
+// 72 / 216) so that a whole 128-column score row stays in registers after one tensor-memory load.
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each.  The bf16 probabilities
 // overwrite the first 64 columns of their own S tile, in two halves that are handed to the
 // second MMA separately, and feed it straight from tensor memory; the tensor pipe runs one
 // thread's MMAs in issue order, so the next Q K^T of a row tile cannot overtake the P V that
-// still reads those columns.
+// still reads those columns.  A single issuing thread for both tiles spends ~126 cycles per MMA
+// (measured) against 64 cycles of tensor work, hence one issuer per row tile.
 //
 // Softmax arithmetic.  p = 2^(s * scale * log2(e) - m) with the reference maximum m moved only
 // when the tile maximum exceeds it by more than 2^8 (then the accumulator is rescaled), packed
@@ -34,6 +35,10 @@
 // the FMA pipe (round-to-nearest split, cubic polynomial, exponent insertion; relative error
 // 7.5e-5, below the bf16 rounding of p) because the special-function unit alone is exactly as
 // slow as the two MMAs of a tile.
+//
+// The exponential phases of the two row tiles are sequenced per scheduler (warp w of tile 0 and
+// warp w of tile 1 alternate), which keeps the tiles in antiphase: one tile's softmax runs under
+// the other tile's MMAs.
 //
 // Every wait on an mbarrier is bounded (about one second): on expiry the thread raises the
 // CTA's abort flag and the device status word, all roles leave their loops, tensor memory is
@@ -54,21 +59,22 @@ constexpr int kThreads = 384;
 constexpr uint32_t kOffQ = 0;                         // 2 tiles
 constexpr uint32_t kOffKV = 2 * kTileBytes;           // kSlots tiles
 constexpr uint32_t kOffCtl = kOffKV + kSlots * kTileBytes;
-constexpr uint32_t kSmemBytes = kOffCtl + 256 + 1024; // + control block + alignment slack
+constexpr uint32_t kSmemBytes = kOffCtl + 512 + 1024; // + control block + alignment slack
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;             // log2 units
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
 // barrier indices inside the control block
 enum { B_QFULL = 0, B_QEMPTY = 1, B_FULL0 = 2, B_EMPTY0 = B_FULL0 + kSlots, B_SFULL0 = B_EMPTY0 + kSlots,
-       B_PA0 = B_SFULL0 + 2, B_PB0 = B_PA0 + 2, B_OFINAL0 = B_PB0 + 2, B_COUNT = B_OFINAL0 + 2 };
+       B_PA0 = B_SFULL0 + 2, B_PB0 = B_PA0 + 2, B_OFINAL0 = B_PB0 + 2, B_TURN0 = B_OFINAL0 + 2,
+       B_COUNT = B_TURN0 + 8 };
 
 struct Ctl {
-    unsigned long long bars[24];
+    unsigned long long bars[32];
     uint32_t tmem_base;
     int abort;
 };
-static_assert(B_COUNT <= 24, "control block holds 24 barriers");
+static_assert(B_COUNT <= 32, "control block holds 32 barriers");
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -276,14 +282,15 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
 
     if (threadIdx.x == 0) {
         mbar_init(bar(B_QFULL), 1);
-        mbar_init(bar(B_QEMPTY), 1);
-        for (int s = 0; s < kSlots; ++s) { mbar_init(bar(B_FULL0 + s), 1); mbar_init(bar(B_EMPTY0 + s), 1); }
+        mbar_init(bar(B_QEMPTY), 2);
+        for (int s = 0; s < kSlots; ++s) { mbar_init(bar(B_FULL0 + s), 1); mbar_init(bar(B_EMPTY0 + s), 2); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(B_SFULL0 + i), 1);
             mbar_init(bar(B_PA0 + i), 4);
             mbar_init(bar(B_PB0 + i), 4);
             mbar_init(bar(B_OFINAL0 + i), 1);
         }
+        for (int w = 0; w < 8; ++w) mbar_init(bar(B_TURN0 + w), 1);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -328,23 +335,29 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             if (pc > 0) mbar_wait(bar(B_QFULL), (pc - 1) & 1, ctl, a.status);
             for (int t = max(0, tg - kSlots); t < tg; ++t)
                 mbar_wait_slow(bar(B_FULL0 + t % kSlots), (t / kSlots) & 1, ctl, a.status);
-        } else if (warp == 9 && lane == 0) {
-            // ------------------------------------------------------------------ MMA issuer
-            auto issue_qk = [&](int i, int slot) {
-                const uint32_t qa = base + kOffQ + i * kTileBytes, kb = base + kOffKV + slot * kTileBytes;
+        } else if ((warp == 9 || warp == 10) && lane == 0) {
+            // ------------------------------------------------------------------ MMA issuer of row tile i
+            // One issuing thread per row tile: each thread's MMAs run in its issue order (P V (j)
+            // before the Q K^T (j+1) that overwrites the probabilities), the two tiles' streams
+            // interleave freely on the tensor pipe, and neither waits on the other's softmax.
+            const int i = warp - 9;
+            const uint32_t t_s = tmem + i * 128, t_o = tmem + 256 + i * 128;
+            const uint64_t qdesc = desc_kmajor(base + kOffQ + i * kTileBytes);
+            auto issue_qk = [&](int slot) {
+                const uint64_t kdesc = desc_kmajor(base + kOffKV + slot * kTileBytes);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (kk >> 2) * kPanel + (kk & 3) * 32;
-                    tc_mma(tmem + i * 128, desc_kmajor(qa + off), desc_kmajor(kb + off), kIdescQK, kk > 0);
+                    const uint64_t off = (uint64_t)(((kk >> 2) * kPanel + (kk & 3) * 32) >> 4);   // start-address field
+                    tc_mma(t_s, qdesc + off, kdesc + off, kIdescQK, kk > 0);
                 }
             };
             // 16 keys = 8 packed columns of P per MMA; half h covers keys 64h .. 64h+63
-            auto issue_pv_half = [&](int i, int slot, int h, bool accumulate) {
-                const uint32_t vb = base + kOffKV + slot * kTileBytes;
+            auto issue_pv_half = [&](int slot, int h, bool accumulate) {
+                const uint64_t vdesc = desc_mnmajor(base + kOffKV + slot * kTileBytes);
 #pragma unroll
                 for (int kk = 4 * h; kk < 4 * h + 4; ++kk)
-                    tc_mma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, desc_mnmajor(vb + kk * 2048), kIdescPV,
-                              (accumulate || kk > 0) ? 1u : 0u);
+                    tc_mma_ts(t_o, t_s + kk * 8, vdesc + (uint64_t)((kk * 2048) >> 4), kIdescPV,
+                              (accumulate || kk > 4 * h) ? 1u : 0u);
             };
             int tg = 0, it = 0, pc = 0;   // ring loads consumed, key tiles issued, pieces so far
             bool ok = true;
@@ -356,45 +369,41 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 tc_fence_after();
                 for (int j = 0; j < ntiles && ok; ++j, ++it) {
                     const int tk = tg + 2 * j, kslot = tk % kSlots;
-                    ok = mbar_wait(bar(B_FULL0 + kslot), (tk / kSlots) & 1, ctl, a.status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    for (int i = 0; i < 2 && ok; ++i) {
-                        if (j > 0) {
-                            const int tv = tk - 1, vslot = tv % kSlots;
-                            if (i == 0) ok = mbar_wait(bar(B_FULL0 + vslot), (tv / kSlots) & 1, ctl, a.status);
-                            if (ok) ok = mbar_wait(bar(B_PA0 + i), (it - 1) & 1, ctl, a.status);
-                            if (!ok) break;
-                            tc_fence_after();
-                            issue_pv_half(i, vslot, 0, j - 1 > 0);
-                            ok = mbar_wait(bar(B_PB0 + i), (it - 1) & 1, ctl, a.status);
-                            if (!ok) break;
-                            tc_fence_after();
-                            issue_pv_half(i, vslot, 1, true);
-                            if (i == 1) tc_commit(bar(B_EMPTY0 + vslot));
-                        }
-                        issue_qk(i, kslot);
-                        tc_commit(bar(B_SFULL0 + i));
-                        if (i == 1) tc_commit(bar(B_EMPTY0 + kslot));
-                    }
-                }
-                if (!ok) break;
-                tc_commit(bar(B_QEMPTY));          // every Q K^T of this piece has been issued
-                {
-                    const int tv = tg + 2 * ntiles - 1, vslot = tv % kSlots;
-                    ok = mbar_wait(bar(B_FULL0 + vslot), (tv / kSlots) & 1, ctl, a.status);
-                    for (int i = 0; i < 2 && ok; ++i) {
-                        ok = mbar_wait(bar(B_PA0 + i), (it - 1) & 1, ctl, a.status);
+                    if (j > 0) {
+                        const int tv = tk - 1, vslot = tv % kSlots;
+                        ok = mbar_wait(bar(B_FULL0 + vslot), (tv / kSlots) & 1, ctl, a.status);
+                        if (ok) ok = mbar_wait(bar(B_PA0 + i), (it - 1) & 1, ctl, a.status);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_pv_half(i, vslot, 0, ntiles > 1);
+                        issue_pv_half(vslot, 0, j - 1 > 0);
                         ok = mbar_wait(bar(B_PB0 + i), (it - 1) & 1, ctl, a.status);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_pv_half(i, vslot, 1, true);
-                        tc_commit(bar(B_OFINAL0 + i));
-                        if (i == 1) tc_commit(bar(B_EMPTY0 + vslot));
+                        issue_pv_half(vslot, 1, true);
+                        tc_commit(bar(B_EMPTY0 + vslot));
                     }
+                    ok = mbar_wait(bar(B_FULL0 + kslot), (tk / kSlots) & 1, ctl, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(kslot);
+                    tc_commit(bar(B_SFULL0 + i));
+                    tc_commit(bar(B_EMPTY0 + kslot));
+                }
+                if (!ok) break;
+                tc_commit(bar(B_QEMPTY));          // every Q K^T of this piece and row tile has been issued
+                {
+                    const int tv = tg + 2 * ntiles - 1, vslot = tv % kSlots;
+                    ok = mbar_wait(bar(B_FULL0 + vslot), (tv / kSlots) & 1, ctl, a.status);
+                    if (ok) ok = mbar_wait(bar(B_PA0 + i), (it - 1) & 1, ctl, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv_half(vslot, 0, ntiles > 1);
+                    ok = mbar_wait(bar(B_PB0 + i), (it - 1) & 1, ctl, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv_half(vslot, 1, true);
+                    tc_commit(bar(B_OFINAL0 + i));
+                    tc_commit(bar(B_EMPTY0 + vslot));
                 }
                 tg += 2 * ntiles;
                 ++pc;
@@ -452,13 +461,15 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
 #pragma unroll
                     for (int c = 0; c < 128; ++c) sc[c] = c < nvis ? sc[c] : 0xFF800000u;   // -inf
                 }
-                float mx0 = -INFINITY, mx1 = -INFINITY;
+                float mx[8];
 #pragma unroll
-                for (int c = 0; c < 128; c += 4) {
-                    mx0 = max3(mx0, __uint_as_float(sc[c]), __uint_as_float(sc[c + 1]));
-                    mx1 = max3(mx1, __uint_as_float(sc[c + 2]), __uint_as_float(sc[c + 3]));
-                }
-                const float m_tile = fmaxf(mx0, mx1);
+                for (int q = 0; q < 8; ++q) mx[q] = fmaxf(__uint_as_float(sc[2 * q]), __uint_as_float(sc[2 * q + 1]));
+#pragma unroll
+                for (int c = 16; c < 128; c += 16)
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        mx[q] = max3(mx[q], __uint_as_float(sc[c + 2 * q]), __uint_as_float(sc[c + 2 * q + 1]));
+                const float m_tile = fmaxf(max3(mx[0], mx[1], mx[2]), max3(max3(mx[3], mx[4], mx[5]), mx[6], mx[7]));
                 // move the reference only when the maximum grew by more than the threshold: the
                 // probabilities then stay below 2^threshold and the accumulator is rarely rescaled
                 const bool grow = (m_tile - m_ref) * sl2 > kRescaleThreshold;   // also true when m_ref = -inf < m_tile
@@ -491,6 +502,17 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 const float2 negv = make_float2(neg, neg);
                 float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 
+                // The two row tiles' warps that share a scheduler take turns on the exponentials:
+                // run side by side they halve each other's special-function rate and both tiles
+                // fall into step, leaving the tensor pipe idle while both are in their softmax.
+                if (i == 0) {
+                    if (it > 0) ok = mbar_wait(bar(B_TURN0 + (warp & 3)), (it - 1) & 1, ctl, a.status);
+                } else {
+                    ok = mbar_wait(bar(B_TURN0 + 4 + (warp & 3)), it & 1, ctl, a.status);
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+
                 // probabilities; the first 64 keys are handed over before the rest is computed
                 uint32_t p[32];
                 if (masked) exp_half<0>(sc, p, sl2v, negv, acc0, acc1);
@@ -506,7 +528,10 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(B_PB0 + i));
+                if (lane == 0) {
+                    mbar_arrive(bar(B_PB0 + i));
+                    mbar_arrive(bar(B_TURN0 + (i == 0 ? 4 : 0) + (warp & 3)));   // the other tile's turn
+                }
                 const float2 acc = __fadd2_rn(acc0, acc1);
                 l += acc.x + acc.y;
             }
@@ -633,7 +658,7 @@ bool attn_tc_supported(int dtype, int d, int G) {
 int attn_tc_row_pairs(int n, int G) { return (n * G + 2 * kRows - 1) / (2 * kRows); }
 
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
-    static_assert(sizeof(Ctl) <= 256, "control block");
+    static_assert(sizeof(Ctl) <= 512, "control block");
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
     static const int emu = [] {
         const char *v = getenv("KVF_EMU");
