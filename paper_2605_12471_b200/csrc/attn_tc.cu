@@ -63,6 +63,7 @@ constexpr uint32_t kSmemBytes = kOffCtl + 512 + 1024; // + control block + align
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;             // log2 units
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+constexpr uint32_t kSuspendHintNs = 20000;             // a waiting thread may sleep this long per try (woken earlier by the barrier)
 
 // barrier indices inside the control block
 enum { B_QFULL = 0, B_QEMPTY = 1, B_FULL0 = 2, B_EMPTY0 = B_FULL0 + kSlots, B_SFULL0 = B_EMPTY0 + kSlots,
@@ -91,9 +92,9 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
     return ok;
 }
 __device__ __forceinline__ unsigned long long global_ns() {
