@@ -597,48 +597,75 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
 // the (KV head, key tile) line, its piece for KV head h sits in slot g + h.  With lse_s = log2 of
 // a piece's softmax denominator and O_s its normalised output,
 //   O = sum_s 2^(lse_s - M) O_s / sum_s 2^(lse_s - M),  M = max_s lse_s,  in group order.
+// One block = kCombineTokens tokens of one KV head; one warp per row, lane = float4 column, so a
+// row of a piece is one coalesced 512-byte read and the weights are computed once per row.
+constexpr int kCombineTokens = 2;
 __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
-    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // (row, float4 column)
-    const int64_t rows = (int64_t)a.n * a.H;
-    if (idx >= rows * (kD / 4)) return;
-    const int64_t row = idx / (kD / 4);
-    const int c = (int)(idx % (kD / 4));
-    const int tok = (int)(row / a.H), h = (int)(row % a.H), kvh = h / a.G, gi = h % a.G;
-    const int64_t nG = (int64_t)a.n * a.G, R = (int64_t)tok * a.G + gi;
-    const int nt_all = (int)((a.prefix + a.n + kRows - 1) / kRows);
-    const int64_t line = (int64_t)a.Hkv * nt_all;
-    auto start = [&](int64_t g) { return g * line / a.ngroups; };
-    auto group_of = [&](int64_t lin) {
-        int64_t g = lin * a.ngroups / line;
-        while (g > 0 && start(g) > lin) --g;
-        while (g + 1 < a.ngroups && start(g + 1) <= lin) ++g;
-        return (int)g;
-    };
-    const int g0 = group_of((int64_t)kvh * nt_all), g1 = group_of((int64_t)(kvh + 1) * nt_all - 1);
-    float M = -INFINITY;
-    for (int g = g0; g <= g1; ++g) M = fmaxf(M, a.part_lse[(int64_t)(g + kvh) * nG + R]);
-    float den = 0.f;
-    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int g = g0; g <= g1; ++g) {
-        const int64_t prow = (int64_t)(g + kvh) * nG + R;
-        const float ls = a.part_lse[prow];
-        if (ls == -INFINITY) continue;
-        const float w = exp2f(ls - M);
-        const float4 p = *reinterpret_cast<const float4 *>(a.part_o + prow * kD + c * 4);
-        den += w;
-        o.x = fmaf(w, p.x, o.x); o.y = fmaf(w, p.y, o.y); o.z = fmaf(w, p.z, o.z); o.w = fmaf(w, p.w, o.w);
+    __shared__ int g_range[2];
+    const int kvh = blockIdx.y, G = a.G;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        const int nt_all = (int)((a.prefix + a.n + kRows - 1) / kRows);
+        const int64_t line = (int64_t)a.Hkv * nt_all;
+        auto start = [&](int64_t g) { return g * line / a.ngroups; };
+        auto group_of = [&](int64_t lin) {
+            int64_t g = lin * a.ngroups / line;
+            while (g > 0 && start(g) > lin) --g;
+            while (g + 1 < a.ngroups && start(g + 1) <= lin) ++g;
+            return (int)g;
+        };
+        g_range[0] = group_of((int64_t)kvh * nt_all);
+        g_range[1] = group_of((int64_t)(kvh + 1) * nt_all - 1);
     }
-    const float inv = den > 0.f ? 1.f / den : 0.f;
-    o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
-    if (a.out_f32) {
-        *reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.out) + row * kD + c * 4) = o;
-    } else {
-        uint2 pk;
-        pk.x = pack_bf16(o.x, o.y);
-        pk.y = pack_bf16(o.z, o.w);
-        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.out) + row * kD + c * 4) = pk;
+    __syncthreads();
+    const int g0 = g_range[0], np = g_range[1] - g0 + 1;     // pieces of this KV head
+    const int64_t nG = (int64_t)a.n * G;
+    const int rows = kCombineTokens * G;                      // rows of this block, row = token * G + head-in-group
+    for (int rr = warp; rr < rows; rr += 8) {
+        const int tok = blockIdx.x * kCombineTokens + rr / G, gi = rr % G;
+        if (tok >= a.n) break;
+        const int64_t R = (int64_t)tok * G + gi;
+        const int64_t row = (int64_t)tok * a.H + kvh * G + gi;
+        float M = -INFINITY;
+        for (int s0 = 0; s0 < np; s0 += 32) {
+            const float ls = s0 + lane < np ? a.part_lse[(int64_t)(g0 + s0 + lane + kvh) * nG + R] : -INFINITY;
+            M = fmaxf(M, ls);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        float den = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s0 = 0; s0 < np; s0 += 8) {                  // 8 pieces at a time, loads issued together
+            const int cnt = min(8, np - s0);
+            float4 pv[8];
+#pragma unroll
+            for (int s = 0; s < 8; ++s)
+                if (s < cnt)
+                    pv[s] = *reinterpret_cast<const float4 *>(a.part_o + ((int64_t)(g0 + s0 + s + kvh) * nG + R) * kD + lane * 4);
+            const float ls = lane < cnt ? a.part_lse[(int64_t)(g0 + s0 + lane + kvh) * nG + R] : -INFINITY;
+            const float wl = ls == -INFINITY ? 0.f : exp2f(ls - M);
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {                     // group order: deterministic
+                if (s < cnt) {
+                    const float w = __shfl_sync(0xffffffffu, wl, s);
+                    den += w;
+                    acc.x = fmaf(w, pv[s].x, acc.x); acc.y = fmaf(w, pv[s].y, acc.y);
+                    acc.z = fmaf(w, pv[s].z, acc.z); acc.w = fmaf(w, pv[s].w, acc.w);
+                }
+            }
+        }
+        const float inv = den > 0.f ? 1.f / den : 0.f;
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        if (a.out_f32) {
+            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.out) + row * kD + lane * 4) = acc;
+        } else {
+            uint2 pk;
+            pk.x = pack_bf16(acc.x, acc.y);
+            pk.y = pack_bf16(acc.z, acc.w);
+            *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.out) + row * kD + lane * 4) = pk;
+        }
+        if (lane == 0 && a.lse) a.lse[row] = (M + log2f(den)) * 0.6931471805599453f;
     }
-    if (c == 0 && a.lse) a.lse[row] = (M + log2f(den)) * 0.6931471805599453f;
 }
 
 template <int kEmu>
@@ -675,8 +702,8 @@ cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s
 }
 
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s) {
-    const int64_t items = (int64_t)a.n * a.H * (kD / 4);
-    combine_groups_kernel<<<(int)((items + 255) / 256), 256, 0, s>>>(a);
+    dim3 grid((a.n + kCombineTokens - 1) / kCombineTokens, a.Hkv, 1);
+    combine_groups_kernel<<<grid, 256, 0, s>>>(a);
     return cudaGetLastError();
 }
 

@@ -14,7 +14,7 @@
 namespace kvf {
 namespace {
 
-constexpr int kTok = 4;        // tokens per CTA
+constexpr int kTok = 2;        // tokens per CTA
 constexpr int kThreads = 256;
 
 template <typename T> struct Vec16;
