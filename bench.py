@@ -134,9 +134,10 @@ def oracle_rate(w: workloads.Workload, seed: int, rows_per_step: int, repeats: i
     return pairs / statistics.median(times), times, threads, rows
 
 
-def tokens_per_s_from_pairs(w: workloads.Workload, pairs_per_s: float) -> float:
-    """A chain of T tokens has T(T+1)/2 visible pairs: tokens/s = pairs/s / ((T+1)/2)."""
-    return pairs_per_s / ((w.tokens + 1) / 2.0)
+def tokens_per_s_from_pairs(w: workloads.Workload, pairs_per_s: float, prefill: int = 0) -> float:
+    """Tokens prefill .. T-1 see (T(T+1) - P(P+1))/2 (query, key) pairs: tokens/s = pairs/s x tokens / pairs."""
+    t, p0 = w.tokens, prefill
+    return pairs_per_s * (t - p0) / ((t * (t + 1) - p0 * (p0 + 1)) / 2.0)
 
 
 def run_reference(args, w):
@@ -170,7 +171,7 @@ def run_reference(args, w):
         if it >= args.warmup:
             elapsed += dt
             pairs += sum(p0 + r + 1 for r in rows)
-    value = tokens_per_s_from_pairs(w, pairs / elapsed)
+    value = tokens_per_s_from_pairs(w, pairs / elapsed, args.prefill)
     threads = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
     sample = (f"{len(rows)} query rows x {w.n_q_heads} heads per step at prefix >= {prefix} (last chunk of the "
               f"chain), fp64 oracle; tokens/s extrapolated linearly in visible (query,key) pairs")
@@ -179,8 +180,9 @@ def run_reference(args, w):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * elapsed / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "tokens": w.tokens, "chunk": w.chunk, "n_q_heads": w.n_q_heads,
-                   "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim},
+        "config": {"workload": w.name, "tokens": w.tokens, "chunk": w.chunk, "prefill": args.prefill,
+                   "fold_steps_per_step": (w.tokens - args.prefill) // w.chunk, "n_q_heads": w.n_q_heads,
+                   "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "rope_base": w.rope_base},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
@@ -195,16 +197,19 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--tokens", type=int, default=0, help="shorter chain (debugging; not the benchmark workload)")
     ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--prefill", type=int, default=0,
+                    help="tokens folded (in 2048-token steps, untimed) before every timed chain: the timed chain "
+                         "then runs from this prefix to --tokens (decode- and question-shaped steps at depth)")
     ap.add_argument("--seed", type=int, default=2605)
-    ap.add_argument("--ref-rows", type=int, default=4)
+    ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--force-simt", action="store_true")
     args = ap.parse_args()
 
     w = workloads.DEEP_CHAIN
-    if args.tokens or args.chunk:
-        w = w.with_(name=f"deep_chain_debug_{args.tokens or w.tokens}_c{args.chunk or w.chunk}",
+    if args.tokens or args.chunk or args.prefill:
+        w = w.with_(name=f"chain_{args.tokens or w.tokens}_c{args.chunk or w.chunk}_from_{args.prefill}",
                     tokens=args.tokens or w.tokens, chunk=args.chunk or w.chunk)
     if args.impl == "reference":
         run_reference(args, w)
@@ -221,22 +226,36 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     lib = binding.load()
 
-    T, C, N = w.tokens, w.chunk, w.n_steps
+    T, C = w.tokens, w.chunk
+    P0 = args.prefill
+    if P0 % 2048 or (T - P0) % C or P0 >= T:
+        raise SystemExit("--prefill must be a multiple of 2048 below --tokens, and (tokens - prefill) a multiple of the chunk")
+    N = (T - P0) // C                                  # timed fold steps per chain
     H, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
-    q, k, v = workloads.sequence_inputs(w, args.seed, sequence=multi.sequence_of_rank(rank)[0], device="cuda")
+    seq = multi.sequence_of_rank(rank)[0]
+    wt = w.with_(tokens=T - P0)                        # the timed part's inputs
+    q, k, v = workloads.sequence_inputs(wt, args.seed, sequence=seq, device="cuda")
     out = torch.empty_like(q)
     flags = binding.KVF_FORCE_SIMT if args.force_simt else 0
-    cache = binding.cache_for(w, flags=flags)
+    cache = binding.cache_for(w, flags=flags, max_chunk=max(C, 2048 if P0 else C))
     h = cache._h
     stream = torch.cuda.current_stream().cuda_stream
     eb = q.element_size()
     qs, ks = C * H * d * eb, C * Hkv * d * eb
     qp, kp, vp, op = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr()
+    if P0:
+        fq, fk, fv = workloads.chunk_inputs(w.with_(chunk=2048), args.seed + 1, 0, sequence=seq, device="cuda")
+        fout = torch.empty_like(fq)
 
-    def chain():
+    def prefill():
+        """Empty accumulator, then (outside every timed region) the prefix in 2048-token steps."""
         cache.reset()
-        for t in range(N):
-            rc = lib.kvf_fold_step(h, qp + t * qs, kp + t * ks, vp + t * ks, C, t * C, op + t * qs, None, stream)
+        for t in range(P0 // 2048):
+            cache.fold_step(fq, fk, fv, out=fout)
+
+    def body(first=0, last=None):
+        for t in range(first, N if last is None else last):
+            rc = lib.kvf_fold_step(h, qp + t * qs, kp + t * ks, vp + t * ks, C, P0 + t * C, op + t * qs, None, stream)
             if rc:
                 raise binding.KvfError(rc, "kvf_fold_step")
 
@@ -246,49 +265,87 @@ def main():
         torch.cuda.synchronize()
 
     def timed(fn, steps):
+        """K chains between one pair of barriers; with a prefill, one bracket per chain so that the
+        prefill stays outside."""
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        a.record()
+        if P0 == 0:
+            barrier()
+            a.record()
+            for _ in range(steps):
+                cache.reset()
+                fn()
+            b.record()
+            barrier()
+            return multi.max_over_ranks(a.elapsed_time(b), device="cuda")
+        total = 0.0
         for _ in range(steps):
+            prefill()
+            barrier()
+            a.record()
             fn()
-        b.record()
-        barrier()
-        return multi.max_over_ranks(a.elapsed_time(b), device="cuda")
+            b.record()
+            barrier()
+            total += a.elapsed_time(b)
+        return multi.max_over_ranks(total, device="cuda")
 
     for _ in range(args.warmup):
-        chain()
+        prefill()
+        body()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    l0 = cache.launch_count()
-    ms = timed(chain, args.steps)
-    launches = cache.launch_count() - l0
+    ms = timed(body, args.steps)
     clocks = sampler.stop() if rank == 0 else None
     assert len(cache) == T
     if cache.status() != binding.KVF_OK:
         raise SystemExit("device status word reports a timed-out wait")
-    value = multi.whole_job_tokens_per_s(T, args.steps, world, ms)
+    value = multi.whole_job_tokens_per_s(T - P0, args.steps, world, ms)
 
-    # per-kernel time of the same chain, CUDA events around every launch on the launching stream
+    # per-kernel time of the same chain, CUDA events around every launch on the launching stream;
+    # read out in bins of steps, which gives the latency against the prefix length
+    prefill()
+    torch.cuda.synchronize()
+    l0 = cache.launch_count()
     cache.profile(True)
-    chain()
-    kms, kcnt = cache.profile_read()
+    kms, kcnt, curve = [0.0, 0.0, 0.0], [0, 0, 0], []
+    nbins = min(16, N)
+    for bi in range(nbins):
+        first, last = bi * N // nbins, (bi + 1) * N // nbins
+        body(first, last)
+        bms, bcnt = cache.profile_read()
+        fl = sum(w.flops_step(P0 + t * C, C) for t in range(first, last))
+        by = sum(P0 + (t + 1) * C for t in range(first, last)) * w.cache_bytes_per_token()
+        curve.append({"prefix_from": P0 + first * C, "prefix_to": P0 + (last - 1) * C,
+                      "step_us": 1e3 * sum(bms) / (last - first), "attention_us": 1e3 * bms[1] / (last - first),
+                      "attention_tflops": fl / (bms[1] * 1e-3) / 1e12, "cache_read_gbs": by / (bms[1] * 1e-3) / 1e9})
+        kms = [x + y for x, y in zip(kms, bms)]
+        kcnt = [x + y for x, y in zip(kcnt, bcnt)]
     cache.profile(False)
+    launches = (cache.launch_count() - l0) * args.steps       # kernels of the timed chains
     pk = peaks()
-    attn_flops = w.flops_chain()
+    attn_flops = sum(w.flops_step(P0 + t * C, C) for t in range(N))
     attn_tflops = attn_flops / (kms[1] * 1e-3) / 1e12
-    peak_tf = pk["bf16_tflops_sustained"]
-    cache_bytes_read = sum((t + 1) * C for t in range(N)) * w.cache_bytes_per_token()
+    cache_bytes_read = sum(P0 + (t + 1) * C for t in range(N)) * w.cache_bytes_per_token()
+    hbm_gbs = cache_bytes_read / (kms[1] * 1e-3) / 1e9
     traffic = None
     if NCU_TRAFFIC_BYTES_PER_CACHE_BYTE is not None:
         traffic = NCU_TRAFFIC_BYTES_PER_CACHE_BYTE * cache_bytes_read / kcnt[1]
-    roofline = {
-        "bound": "tensor", "kernel": "prefix+chunk attention", "achieved": attn_tflops, "peak": peak_tf,
-        "unit": "TFLOP/s", "frac": attn_tflops / peak_tf, "peak_source": pk["_source"] + " sustained bf16",
-        "traffic": traffic, "flops_per_launch": attn_flops / kcnt[1], "ms_per_launch": kms[1] / kcnt[1],
-        "launches": kcnt[1], "kernel_ms_per_chain": {"rope_append": kms[0], "attention": kms[1], "combine": kms[2]},
-        "hbm_gbs_cache_read": cache_bytes_read / (kms[1] * 1e-3) / 1e9, "hbm_peak_gbs": pk["hbm_gbs"],
-    }
+    # which roof binds: arithmetic intensity G*C FLOP per cache byte against the ridge of the measured peaks
+    ridge = pk["bf16_tflops_sustained"] * 1e12 / (pk["hbm_gbs"] * 1e9)
+    intensity = attn_flops / cache_bytes_read
+    if intensity >= ridge:
+        roofline = {"bound": "tensor", "achieved": attn_tflops, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                    "frac": attn_tflops / pk["bf16_tflops_sustained"], "peak_source": pk["_source"] + " sustained bf16"}
+    else:
+        roofline = {"bound": "hbm", "achieved": hbm_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                    "frac": hbm_gbs / pk["hbm_gbs"], "peak_source": pk["_source"] + " copy bandwidth"}
+    roofline.update({
+        "kernel": "prefix+chunk attention", "traffic": traffic, "flops_per_launch": attn_flops / kcnt[1],
+        "cache_bytes_per_launch": cache_bytes_read / kcnt[1], "ms_per_launch": kms[1] / kcnt[1], "launches": kcnt[1],
+        "kernel_ms_per_chain": {"rope_append": kms[0], "attention": kms[1], "combine": kms[2]},
+        "attention_tflops": attn_tflops, "cache_read_gbs": hbm_gbs, "flop_per_cache_byte": intensity,
+        "ridge_flop_per_byte": ridge, "hbm_peak_gbs": pk["hbm_gbs"], "bf16_peak_tflops": pk["bf16_tflops_sustained"],
+    })
 
     e2e = None
     if not args.no_e2e:
@@ -296,42 +353,43 @@ def main():
         oh = torch.empty(out.shape, dtype=out.dtype).pin_memory()
         qhp, khp, vhp, ohp = qh.data_ptr(), kh.data_ptr(), vh.data_ptr(), oh.data_ptr()
 
-        def chain_host():
-            cache.reset()
+        def body_host():
             for t in range(N):
-                rc = lib.kvf_fold_step_host(h, qhp + t * qs, khp + t * ks, vhp + t * ks, C, t * C, ohp + t * qs,
+                rc = lib.kvf_fold_step_host(h, qhp + t * qs, khp + t * ks, vhp + t * ks, C, P0 + t * C, ohp + t * qs,
                                             None, stream)
                 if rc:
                     raise binding.KvfError(rc, "kvf_fold_step_host")
 
-        chain_host()
+        prefill()
+        body_host()
         e2e_steps = max(1, min(args.steps, 3))
-        ems = timed(chain_host, e2e_steps)
-        e2e = {"value": world * e2e_steps * T / (ems * 1e-3), "unit": "tokens/s", "steps": e2e_steps,
-               "h2d_bytes_per_step": T * (H + 2 * Hkv) * d * eb, "d2h_bytes_per_step": T * H * d * eb,
+        ems = timed(body_host, e2e_steps)
+        e2e = {"value": world * e2e_steps * (T - P0) / (ems * 1e-3), "unit": "tokens/s", "steps": e2e_steps,
+               "h2d_bytes_per_step": (T - P0) * (H + 2 * Hkv) * d * eb, "d2h_bytes_per_step": (T - P0) * H * d * eb,
                "ms_per_step": ems / e2e_steps}
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
-        rate, times, threads, rows = oracle_rate(w, args.seed, rows_per_step=4, repeats=3, prefix=T - 4 * C)
-        cpu = {"value": tokens_per_s_from_pairs(w, rate), "unit": "tokens/s", "cores": threads, "kind": "oracle",
+        rate, times, threads, rows = oracle_rate(w, args.seed, rows_per_step=32, repeats=4, prefix=max(0, T - 5 * C))
+        cpu = {"value": tokens_per_s_from_pairs(w, rate, P0), "unit": "tokens/s", "cores": threads, "kind": "oracle",
                "sample": (f"{len(rows)} query rows x {H} heads of one chunk at prefix ~{T - 4 * C}, median of "
                           f"{len(times)} repeats ({sum(times):.1f} s of CPU work), fp64 oracle; tokens/s "
                           f"extrapolated linearly in visible (query,key) pairs over the chain")}
 
     if rank == 0:
         plan = cache.plan(C, T - C)
+        step_flops = attn_flops * world * args.steps
         line = {
             "metric": "fold-step tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
             "data": "synthetic",
-            "config": {"workload": w.name, "tokens": T, "chunk": C, "fold_steps_per_step": N,
+            "config": {"workload": w.name, "tokens": T, "chunk": C, "prefill": P0, "fold_steps_per_step": N,
                        "n_q_heads": H, "n_kv_heads": Hkv, "head_dim": d, "rope_base": w.rope_base,
                        "sequences_per_gpu": 1, "l2": "inputs larger than L2 (cache grows to 512 MiB per chain)",
                        "last_step_plan": {"tensor_core": plan[0], "splits": plan[1], "ctas": plan[2]}},
-            "attention_tflops": attn_flops * world * args.steps / (ms * 1e-3) / 1e12,
-            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+            "attention_tflops": step_flops / (ms * 1e-3) / 1e12,
+            "roofline": roofline, "latency_vs_prefix": curve, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -31,10 +31,10 @@
 //
 // Softmax arithmetic.  p = 2^(s * scale * log2(e) - m) with the reference maximum m moved only
 // when the tile maximum exceeds it by more than 2^8 (then the accumulator is rescaled), packed
-// two-wide fp32 multiply-adds, and, on unmasked tiles, a share of the exponentials evaluated on
-// the FMA pipe (round-to-nearest split, cubic polynomial, exponent insertion; relative error
-// 7.5e-5, below the bf16 rounding of p) because the special-function unit alone is exactly as
-// slow as the two MMAs of a tile.
+// two-wide fp32 multiply-adds, one special-function exponential per score.  (The special-function
+// unit needs 1024 cycles per 128 x 128 tile and scheduler, as long as the tile's two MMAs; moving
+// a share of the exponentials to an FMA-pipe polynomial was measured and did not pay here: the
+// scheduler's issue port, not the special-function unit alone, is what the softmax saturates.)
 //
 // The exponential phases of the two row tiles are sequenced per scheduler (warp w of tile 0 and
 // warp w of tile 1 alternate), which keeps the tiles in antiphase: one tile's softmax runs under
@@ -44,8 +44,6 @@
 // CTA's abort flag and the device status word, all roles leave their loops, tensor memory is
 // released and the kernel returns.
 #include "kvfold_internal.h"
-
-#include <cstdlib>
 
 namespace kvf {
 namespace {
@@ -191,24 +189,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t *>(&b);
 }
 
-// 2^x for two values on the FMA pipe: x = n + f with n = round(x), f in [-1/2, 1/2];
-// 2^f by a cubic (relative error 7.5e-5), n added into the exponent field.  x is clamped
-// at -126 (the result is then ~1e-38 instead of 0, which is why masked tiles do not use it).
-__device__ __forceinline__ float2 exp2_fma2(float2 x) {
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
-    const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));      // 1.5 * 2^23: low bits = n
-    const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
-    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
-    float2 p = __ffma2_rn(f, make_float2(0.05517132207751274f, 0.05517132207751274f),
-                          make_float2(0.24261054396629333f, 0.24261054396629333f));
-    p = __ffma2_rn(p, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
-    p = __ffma2_rn(p, f, make_float2(0.9999281167984009f, 0.9999281167984009f));
-    p.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23));
-    p.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23));
-    return p;
-}
-
 // Shared-memory matrix descriptors (128-byte swizzle, descriptor version 1).
 // K-major operand ([rows][64 bf16] panels, 8-row groups 1024 bytes apart):
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
@@ -226,27 +206,19 @@ constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) 
 constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
 
 // 64 scores of a row -> 32 packed bf16 probability pairs in p[0..31]; their sum goes to acc.
-// kEmu of every 4 pairs take the FMA-pipe exponential (0 on masked tiles, where a masked score,
-// already set to -inf, must give exactly 0).
-template <int kEmu>
 __device__ __forceinline__ void exp_half(const uint32_t *v, uint32_t *p, float2 sl2v, float2 negv, float2 &acc0, float2 &acc1) {
 #pragma unroll
     for (int c = 0; c < 32; ++c) {
         const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1])), sl2v, negv);
         float2 e;
-        if ((c & 3) < kEmu) {
-            e = exp2_fma2(x);
-        } else {
-            e.x = ex2(x.x);
-            e.y = ex2(x.y);
-        }
+        e.x = ex2(x.x);
+        e.y = ex2(x.y);
         if (c & 1) acc1 = __fadd2_rn(acc1, e);
         else acc0 = __fadd2_rn(acc0, e);
         p[c] = pack_bf16(e.x, e.y);
     }
 }
 
-template <int kEmu>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v) {
@@ -265,6 +237,9 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     // key tiles: this row pair needs tiles below nt_need; the group's share of the
     // (KV head, tile) line is [lin0, lin1)
     const int row0 = qpair * 2 * kRows;
+    // short chunks (at most 128 / G tokens in this row pair) leave the second row tile without a
+    // valid row: its issuer and softmax warps then sit the kernel out
+    const int tiles = row0 + kRows < n * G ? 2 : 1;
     const int tok_last = min(n - 1, (row0 + 2 * kRows - 1) / G);
     const int nt_need = (int)((P + tok_last + 1 + kRows - 1) / kRows);
     const int nt_all = (int)((L + kRows - 1) / kRows);
@@ -283,8 +258,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
 
     if (threadIdx.x == 0) {
         mbar_init(bar(B_QFULL), 1);
-        mbar_init(bar(B_QEMPTY), 2);
-        for (int s = 0; s < kSlots; ++s) { mbar_init(bar(B_FULL0 + s), 1); mbar_init(bar(B_EMPTY0 + s), 2); }
+        mbar_init(bar(B_QEMPTY), tiles);
+        for (int s = 0; s < kSlots; ++s) { mbar_init(bar(B_FULL0 + s), 1); mbar_init(bar(B_EMPTY0 + s), tiles); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(B_SFULL0 + i), 1);
             mbar_init(bar(B_PA0 + i), 4);
@@ -336,7 +311,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             if (pc > 0) mbar_wait(bar(B_QFULL), (pc - 1) & 1, ctl, a.status);
             for (int t = max(0, tg - kSlots); t < tg; ++t)
                 mbar_wait_slow(bar(B_FULL0 + t % kSlots), (t / kSlots) & 1, ctl, a.status);
-        } else if ((warp == 9 || warp == 10) && lane == 0) {
+        } else if ((warp == 9 || (warp == 10 && tiles == 2)) && lane == 0) {
             // ------------------------------------------------------------------ MMA issuer of row tile i
             // One issuing thread per row tile: each thread's MMAs run in its issue order (P V (j)
             // before the Q K^T (j+1) that overwrites the probabilities), the two tiles' streams
@@ -420,13 +395,15 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         const uint32_t t_o = tmem + lane_addr + 256 + i * 128;
         const int R = row0 + i * kRows + r, tok = R / G, gi = R % G;
         const bool valid = tok < n;
-        const int64_t limit = valid ? P + tok + 1 : 0;  // keys below `limit` are visible
+        // keys below `limit` are visible; a row past the chunk's end is never written, and each
+        // row of S, P and O depends on that row alone, so such rows are left unmasked
+        const int64_t limit = valid ? P + tok + 1 : ((int64_t)1 << 62);
         const float sl2 = a.scale_log2;
         const float2 sl2v = make_float2(sl2, sl2);
         const int64_t nG = (int64_t)n * G;
 
         int it = 0, pc = 0;
-        bool ok = true;
+        bool ok = i < tiles;
         int kt0, ntiles;
         for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
             const int64_t prow = (int64_t)(group + kvh) * nG + R;     // row of this piece's partial slot
@@ -506,7 +483,9 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 // The two row tiles' warps that share a scheduler take turns on the exponentials:
                 // run side by side they halve each other's special-function rate and both tiles
                 // fall into step, leaving the tensor pipe idle while both are in their softmax.
-                if (i == 0) {
+                if (tiles == 1) {
+                    // nobody to take turns with
+                } else if (i == 0) {
                     if (it > 0) ok = mbar_wait(bar(B_TURN0 + (warp & 3)), (it - 1) & 1, ctl, a.status);
                 } else {
                     ok = mbar_wait(bar(B_TURN0 + 4 + (warp & 3)), it & 1, ctl, a.status);
@@ -516,15 +495,13 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
 
                 // probabilities; the first 64 keys are handed over before the rest is computed
                 uint32_t p[32];
-                if (masked) exp_half<0>(sc, p, sl2v, negv, acc0, acc1);
-                else exp_half<kEmu>(sc, p, sl2v, negv, acc0, acc1);
+                exp_half(sc, p, sl2v, negv, acc0, acc1);
                 KVF_TMEM_ST32(p, 0, t_s);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B_PA0 + i));
-                if (masked) exp_half<0>(sc + 64, p, sl2v, negv, acc0, acc1);
-                else exp_half<kEmu>(sc + 64, p, sl2v, negv, acc0, acc1);
+                exp_half(sc + 64, p, sl2v, negv, acc0, acc1);
                 KVF_TMEM_ST32(p, 0, t_s + 32);
                 tmem_wait_st();
                 tc_fence_before();
@@ -668,15 +645,6 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
     }
 }
 
-template <int kEmu>
-cudaError_t launch_t(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<kEmu>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, 1);
-    attn_tc_kernel<kEmu><<<grid, kThreads, kSmemBytes, s>>>(a, maps.q, maps.k, maps.v);
-    return cudaGetLastError();
-}
-
 }  // namespace
 
 bool attn_tc_supported(int dtype, int d, int G) {
@@ -688,17 +656,11 @@ int attn_tc_row_pairs(int n, int G) { return (n * G + 2 * kRows - 1) / (2 * kRow
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
     static_assert(sizeof(Ctl) <= 512, "control block");
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
-    static const int emu = [] {
-        const char *v = getenv("KVF_EMU");
-        return v ? atoi(v) : 0;
-    }();
-    switch (emu) {
-        case 0: return launch_t<0>(a, maps, s);
-        case 2: return launch_t<2>(a, maps, s);
-        case 3: return launch_t<3>(a, maps, s);
-        case 4: return launch_t<4>(a, maps, s);
-        default: return launch_t<1>(a, maps, s);
-    }
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, 1);
+    attn_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(a, maps.q, maps.k, maps.v);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s) {
