@@ -33,9 +33,11 @@ from paper_2605_12471_b200 import workloads  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes (read + write) per attention launch measured once with ncu on a smaller chain and
-# scaled by cache rows read; None until a capture exists (see profiles/).
-NCU_TRAFFIC_BYTES_PER_CACHE_BYTE = None
+# DRAM bytes (read + write) of one attention launch per algorithmic cache byte it reads, from the
+# ncu capture summarised in profiles/attn_tc_kernel_chain_64k_c256_last_steps.md (65 536-token
+# chain; traffic grows in proportion to the cache rows read, so the ratio carries over).  Set to
+# None whenever attn_tc_kernel changes after the capture.
+NCU_TRAFFIC_BYTES_PER_CACHE_BYTE = 1.033
 
 
 def peaks():
