@@ -21,7 +21,7 @@
 // = row), warp 8 TMA producer (Q per piece, then K(j), V(j), ... through a 5-slot ring), warps 9
 // and 10 tcgen05.mma issuers of row tile 0 and 1 (warp 9 owns the TMEM allocation); warp 11 only
 // completes the third warpgroup, which hands registers to the softmax warpgroups (setmaxnreg
-// 72 / 216) so that a whole 128-column score row stays in registers after one tensor-memory load.
+// 80 / 208) so that a whole 128-column score row stays in registers after one tensor-memory load.
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each.  The bf16 probabilities
 // overwrite the first 64 columns of their own S tile, in two halves that are handed to the
 // second MMA separately, and feed it straight from tensor memory; the tensor pipe runs one
@@ -64,9 +64,10 @@ constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 constexpr uint32_t kSuspendHintNs = 20000;             // a waiting thread may sleep this long per try (woken earlier by the barrier)
 
 // barrier indices inside the control block
-enum { B_QFULL = 0, B_QEMPTY = 1, B_FULL0 = 2, B_EMPTY0 = B_FULL0 + kSlots, B_SFULL0 = B_EMPTY0 + kSlots,
+constexpr int kRingBars = 6;                  // 5 slots of the shared ring, or 2 x 3 slots of the per-stream rings
+enum { B_QFULL = 0, B_QEMPTY = 1, B_FULL0 = 2, B_EMPTY0 = B_FULL0 + kRingBars, B_SFULL0 = B_EMPTY0 + kRingBars,
        B_PA0 = B_SFULL0 + 2, B_PB0 = B_PA0 + 2, B_OFINAL0 = B_PB0 + 2, B_TURN0 = B_OFINAL0 + 2,
-       B_COUNT = B_TURN0 + 8 };
+       B_DRAIN0 = B_TURN0 + 8, B_COUNT = B_DRAIN0 + 2 };
 
 struct Ctl {
     unsigned long long bars[32];
@@ -114,6 +115,19 @@ __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, Ct
                 atomicExch(status, 5);   // KVF_ERR_TIMEOUT
                 return false;
             }
+        }
+    }
+}
+// Wait used on the way out (copies or MMAs of this thread still in flight): bounded by its own
+// clock, and not cut short by the abort flag - shared and tensor memory must not be given back
+// while something still writes to them.
+__device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity, int *status) {
+    const unsigned long long t0 = global_ns();
+    unsigned spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63u) == 0 && global_ns() - t0 > kWaitLimitNs) {
+            atomicExch(status, 5);   // KVF_ERR_TIMEOUT
+            return;
         }
     }
 }
@@ -232,14 +246,18 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     const int qpair = blockIdx.x, group = blockIdx.y;
     const int G = a.G, n = a.n;
     const int64_t P = a.prefix, L = P + n;
-    const bool direct = a.ngroups == a.Hkv;
+    // streams == 2 (chunks of at most 128 / G tokens, i.e. one row tile): the two tile slots work on
+    // the SAME 128 rows and take alternate key tiles, so that one stream's softmax still runs under
+    // the other stream's MMAs; each stream leaves its own partial result.
+    const int streams = a.streams;
+    const bool direct = a.ngroups == a.Hkv && streams == 1;
 
     // key tiles: this row pair needs tiles below nt_need; the group's share of the
     // (KV head, tile) line is [lin0, lin1)
     const int row0 = qpair * 2 * kRows;
     // short chunks (at most 128 / G tokens in this row pair) leave the second row tile without a
     // valid row: its issuer and softmax warps then sit the kernel out
-    const int tiles = row0 + kRows < n * G ? 2 : 1;
+    const int tiles = (streams == 2 || row0 + kRows < n * G) ? 2 : 1;
     const int tok_last = min(n - 1, (row0 + 2 * kRows - 1) / G);
     const int nt_need = (int)((P + tok_last + 1 + kRows - 1) / kRows);
     const int nt_all = (int)((L + kRows - 1) / kRows);
@@ -258,8 +276,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
 
     if (threadIdx.x == 0) {
         mbar_init(bar(B_QFULL), 1);
-        mbar_init(bar(B_QEMPTY), tiles);
-        for (int s = 0; s < kSlots; ++s) { mbar_init(bar(B_FULL0 + s), 1); mbar_init(bar(B_EMPTY0 + s), tiles); }
+        mbar_init(bar(B_QEMPTY), tiles);                                  // both issuers read Q
+        for (int s = 0; s < kRingBars; ++s) { mbar_init(bar(B_FULL0 + s), 1); mbar_init(bar(B_EMPTY0 + s), streams == 2 ? 1 : tiles); }   // consumers of a K/V tile
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(B_SFULL0 + i), 1);
             mbar_init(bar(B_PA0 + i), 4);
@@ -267,6 +285,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             mbar_init(bar(B_OFINAL0 + i), 1);
         }
         for (int w = 0; w < 8; ++w) mbar_init(bar(B_TURN0 + w), 1);
+        mbar_init(bar(B_DRAIN0), 1);
+        mbar_init(bar(B_DRAIN0 + 1), 1);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -278,39 +298,56 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&ctl->tmem_base);
+    // K/V tile slots.  Two row tiles: one ring of 5 that both issuers walk in step.  Two streams:
+    // each stream owns a ring of 3 (the sixth slot is the second Q tile, unused there), because a
+    // parity wait is only sound for a thread that watches every use of its barrier in order.
+    auto slot_addr = [&](int sl) { return base + (sl < kSlots ? kOffKV + (uint32_t)sl * kTileBytes : kOffQ + kTileBytes); };
 
     if (warp >= 8) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
         if (warp == 8 && lane == 0) {
             // ------------------------------------------------------------------ TMA producer
             int tg = 0, pc = 0;          // ring loads and pieces so far
+            int rc[2] = {0, 0};          // loads so far into each stream's ring
             bool ok = true;
             int kt0, ntiles;
             for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
                 if (ntiles <= 0) continue;
                 if (pc > 0) ok = mbar_wait(bar(B_QEMPTY), (pc - 1) & 1, ctl, a.status);
                 if (!ok) break;
-                mbar_expect_tx(bar(B_QFULL), 2 * kTileBytes);
-                for (int i = 0; i < 2; ++i)
+                mbar_expect_tx(bar(B_QFULL), (streams == 2 ? 1 : 2) * kTileBytes);
+                for (int i = 0; i < (streams == 2 ? 1 : 2); ++i)
                     for (int p = 0; p < 2; ++p)
                         tma_load_3d(base + kOffQ + i * kTileBytes + p * kPanel, &map_q, bar(B_QFULL), p * 64, kvh * G,
                                     (row0 + i * kRows) / G);
                 ++pc;
                 for (int t = 0; t < 2 * ntiles; ++t, ++tg) {
-                    const int slot = tg % kSlots, use = tg / kSlots;
+                    int slot = tg % kSlots, use = tg / kSlots;
+                    if (streams == 2) {
+                        const int st = (t >> 1) & 1;          // key tile j goes to stream j & 1
+                        slot = st * 3 + rc[st] % 3;
+                        use = rc[st] / 3;
+                        ++rc[st];
+                    }
                     ok = mbar_wait(bar(B_EMPTY0 + slot), (use & 1) ^ 1, ctl, a.status);
                     if (!ok) break;
                     const CUtensorMap *m = (t & 1) ? &map_v : &map_k;
                     const int key0 = (kt0 + (t >> 1)) * kRows;
                     mbar_expect_tx(bar(B_FULL0 + slot), kTileBytes);
-                    tma_load_3d(base + kOffKV + slot * kTileBytes, m, bar(B_FULL0 + slot), 0, key0, kvh);
-                    tma_load_3d(base + kOffKV + slot * kTileBytes + kPanel, m, bar(B_FULL0 + slot), 64, key0, kvh);
+                    tma_load_3d(slot_addr(slot), m, bar(B_FULL0 + slot), 0, key0, kvh);
+                    tma_load_3d(slot_addr(slot) + kPanel, m, bar(B_FULL0 + slot), 64, key0, kvh);
                 }
             }
             // do not leave while a copy may still be writing into this CTA's shared memory
-            if (pc > 0) mbar_wait(bar(B_QFULL), (pc - 1) & 1, ctl, a.status);
-            for (int t = max(0, tg - kSlots); t < tg; ++t)
-                mbar_wait_slow(bar(B_FULL0 + t % kSlots), (t / kSlots) & 1, ctl, a.status);
+            if (pc > 0) mbar_wait_drain(bar(B_QFULL), (pc - 1) & 1, a.status);
+            if (streams == 2) {
+                for (int st = 0; st < 2; ++st)
+                    for (int c = max(0, rc[st] - 3); c < rc[st]; ++c)
+                        mbar_wait_drain(bar(B_FULL0 + st * 3 + c % 3), (c / 3) & 1, a.status);
+            } else {
+                for (int t = max(0, tg - kSlots); t < tg; ++t)
+                    mbar_wait_drain(bar(B_FULL0 + t % kSlots), (t / kSlots) & 1, a.status);
+            }
         } else if ((warp == 9 || (warp == 10 && tiles == 2)) && lane == 0) {
             // ------------------------------------------------------------------ MMA issuer of row tile i
             // One issuing thread per row tile: each thread's MMAs run in its issue order (P V (j)
@@ -318,9 +355,10 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             // interleave freely on the tensor pipe, and neither waits on the other's softmax.
             const int i = warp - 9;
             const uint32_t t_s = tmem + i * 128, t_o = tmem + 256 + i * 128;
-            const uint64_t qdesc = desc_kmajor(base + kOffQ + i * kTileBytes);
+            const uint64_t qdesc = desc_kmajor(base + kOffQ + (streams == 2 ? 0 : i) * kTileBytes);
+            const int j0 = streams == 2 ? i : 0, jstep = streams;    // my key tiles of a piece: j0, j0 + jstep, ...
             auto issue_qk = [&](int slot) {
-                const uint64_t kdesc = desc_kmajor(base + kOffKV + slot * kTileBytes);
+                const uint64_t kdesc = desc_kmajor(slot_addr(slot));
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint64_t off = (uint64_t)(((kk >> 2) * kPanel + (kk & 3) * 32) >> 4);   // start-address field
@@ -329,51 +367,64 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             };
             // 16 keys = 8 packed columns of P per MMA; half h covers keys 64h .. 64h+63
             auto issue_pv_half = [&](int slot, int h, bool accumulate) {
-                const uint64_t vdesc = desc_mnmajor(base + kOffKV + slot * kTileBytes);
+                const uint64_t vdesc = desc_mnmajor(slot_addr(slot));
 #pragma unroll
                 for (int kk = 4 * h; kk < 4 * h + 4; ++kk)
                     tc_mma_ts(t_o, t_s + kk * 8, vdesc + (uint64_t)((kk * 2048) >> 4), kIdescPV,
                               (accumulate || kk > 4 * h) ? 1u : 0u);
             };
-            int tg = 0, it = 0, pc = 0;   // ring loads consumed, key tiles issued, pieces so far
+            int tg = 0, it = 0, pc = 0;   // ring loads before this piece, my key tiles issued, pieces so far
             bool ok = true;
+            // load number -> slot and parity: shared ring (number counts every load) or my own ring
+            // (number counts my loads: K of my m-th tile is 2m, its V 2m + 1)
+            auto ring = [&](int num, int &slot, uint32_t &par) {
+                if (streams == 2) { slot = i * 3 + num % 3; par = (num / 3) & 1; }
+                else { slot = num % kSlots; par = (num / kSlots) & 1; }
+            };
             int kt0, ntiles;
             for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
                 if (ntiles <= 0) continue;
                 ok = mbar_wait(bar(B_QFULL), pc & 1, ctl, a.status);
                 if (!ok) break;
                 tc_fence_after();
-                for (int j = 0; j < ntiles && ok; ++j, ++it) {
-                    const int tk = tg + 2 * j, kslot = tk % kSlots;
-                    if (j > 0) {
-                        const int tv = tk - 1, vslot = tv % kSlots;
-                        ok = mbar_wait(bar(B_FULL0 + vslot), (tv / kSlots) & 1, ctl, a.status);
+                int jlast = -1;
+                for (int j = j0; j < ntiles && ok; j += jstep, ++it) {
+                    const int tk = streams == 2 ? 2 * it : tg + 2 * j;
+                    int kslot, vslot;
+                    uint32_t kpar, vpar;
+                    ring(tk, kslot, kpar);
+                    if (j > j0) {
+                        ring(tk - 1, vslot, vpar);                               // V of my previous tile
+                        ok = mbar_wait(bar(B_FULL0 + vslot), vpar, ctl, a.status);
                         if (ok) ok = mbar_wait(bar(B_PA0 + i), (it - 1) & 1, ctl, a.status);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_pv_half(vslot, 0, j - 1 > 0);
+                        issue_pv_half(vslot, 0, j - jstep > j0);
                         ok = mbar_wait(bar(B_PB0 + i), (it - 1) & 1, ctl, a.status);
                         if (!ok) break;
                         tc_fence_after();
                         issue_pv_half(vslot, 1, true);
                         tc_commit(bar(B_EMPTY0 + vslot));
                     }
-                    ok = mbar_wait(bar(B_FULL0 + kslot), (tk / kSlots) & 1, ctl, a.status);
+                    ok = mbar_wait(bar(B_FULL0 + kslot), kpar, ctl, a.status);
                     if (!ok) break;
                     tc_fence_after();
                     issue_qk(kslot);
                     tc_commit(bar(B_SFULL0 + i));
                     tc_commit(bar(B_EMPTY0 + kslot));
+                    jlast = j;
                 }
                 if (!ok) break;
-                tc_commit(bar(B_QEMPTY));          // every Q K^T of this piece and row tile has been issued
-                {
-                    const int tv = tg + 2 * ntiles - 1, vslot = tv % kSlots;
-                    ok = mbar_wait(bar(B_FULL0 + vslot), (tv / kSlots) & 1, ctl, a.status);
+                tc_commit(bar(B_QEMPTY));          // every Q K^T of mine in this piece has been issued
+                if (jlast >= 0) {
+                    int vslot;
+                    uint32_t vpar;
+                    ring(streams == 2 ? 2 * it - 1 : tg + 2 * jlast + 1, vslot, vpar);
+                    ok = mbar_wait(bar(B_FULL0 + vslot), vpar, ctl, a.status);
                     if (ok) ok = mbar_wait(bar(B_PA0 + i), (it - 1) & 1, ctl, a.status);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv_half(vslot, 0, ntiles > 1);
+                    issue_pv_half(vslot, 0, jlast > j0);
                     ok = mbar_wait(bar(B_PB0 + i), (it - 1) & 1, ctl, a.status);
                     if (!ok) break;
                     tc_fence_after();
@@ -384,17 +435,22 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 tg += 2 * ntiles;
                 ++pc;
             }
+            // whatever made this thread leave its loop, tensor memory is released only after every
+            // MMA it issued has run
+            tc_commit(bar(B_DRAIN0 + i));
+            mbar_wait_drain(bar(B_DRAIN0 + i), 0, a.status);
         }
     } else {
         // ------------------------------------------------------------------ softmax, one thread per row
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
         const int i = warp >> 2;                        // row tile
         const int r = (warp & 3) * 32 + lane;           // row in the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t t_s = tmem + lane_addr + i * 128;
         const uint32_t t_o = tmem + lane_addr + 256 + i * 128;
-        const int R = row0 + i * kRows + r, tok = R / G, gi = R % G;
+        const int R = row0 + (streams == 2 ? 0 : i * kRows) + r, tok = R / G, gi = R % G;
         const bool valid = tok < n;
+        const int j0 = streams == 2 ? i : 0, jstep = streams;        // my key tiles of a piece
         // keys below `limit` are visible; a row past the chunk's end is never written, and each
         // row of S, P and O depends on that row alone, so such rows are left unmasked
         const int64_t limit = valid ? P + tok + 1 : ((int64_t)1 << 62);
@@ -402,12 +458,18 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         const float2 sl2v = make_float2(sl2, sl2);
         const int64_t nG = (int64_t)n * G;
 
-        int it = 0, pc = 0;
+        int it = 0, oc = 0;            // my key tiles and my finished pieces so far
+        int other = 0;                 // key tiles the other tile slot has had so far
         bool ok = i < tiles;
         int kt0, ntiles;
         for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
-            const int64_t prow = (int64_t)(group + kvh) * nG + R;     // row of this piece's partial slot
-            if (ntiles <= 0) {
+            const int64_t prow = ((int64_t)(group + kvh) * streams + (streams == 2 ? i : 0)) * nG + R;   // my partial row
+            const int other_before = other;
+            {
+                const int oj0 = streams == 2 ? 1 - i : 0;            // the other slot's first key tile
+                other += ntiles > oj0 ? (ntiles - oj0 + jstep - 1) / jstep : 0;
+            }
+            if (ntiles <= j0) {
                 // no visible key for these rows in this range: an empty partial
                 if (!direct && valid) {
                     float4 *po = reinterpret_cast<float4 *>(a.part_o + prow * kD);
@@ -419,7 +481,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             }
             float m_ref = -INFINITY;   // reference maximum (raw score units) the probabilities are scaled by
             float l = 0.f;
-            for (int j = 0; j < ntiles; ++j, ++it) {
+            for (int j = j0, k = 0; j < ntiles; j += jstep, ++it, ++k) {
                 ok = mbar_wait(bar(B_SFULL0 + i), it & 1, ctl, a.status);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -456,8 +518,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                     const float alpha = grow ? ex2((m_ref - m_new) * sl2) : 1.f;   // m_ref = -inf -> 0
                     l *= alpha;
                     m_ref = m_new;
-                    if (j > 0) {
-                        // the commit that completed S(j) also covers PV(j-1): O is quiescent here
+                    if (k > 0) {
+                        // the commit that completed this S also covers my previous P V: O is quiescent here
                         const float2 av = make_float2(alpha, alpha);
 #pragma unroll 1
                         for (int c0 = 0; c0 < 128; c0 += 32) {
@@ -483,12 +545,17 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 // The two row tiles' warps that share a scheduler take turns on the exponentials:
                 // run side by side they halve each other's special-function rate and both tiles
                 // fall into step, leaving the tensor pipe idle while both are in their softmax.
+                // Slot 0's k-th tile of a piece goes after slot 1's (k-1)-th (for k = 0: after slot 1's
+                // last tile of the piece before), slot 1's k-th after slot 0's k-th; the partner's
+                // running count turns that into a barrier phase.  Neither slot can get two phases
+                // ahead of the other's wait, which a parity wait could not tell from none.
                 if (tiles == 1) {
                     // nobody to take turns with
                 } else if (i == 0) {
-                    if (it > 0) ok = mbar_wait(bar(B_TURN0 + (warp & 3)), (it - 1) & 1, ctl, a.status);
+                    if (other_before + k > 0)
+                        ok = mbar_wait(bar(B_TURN0 + (warp & 3)), (other_before + k - 1) & 1, ctl, a.status);
                 } else {
-                    ok = mbar_wait(bar(B_TURN0 + 4 + (warp & 3)), it & 1, ctl, a.status);
+                    ok = mbar_wait(bar(B_TURN0 + 4 + (warp & 3)), (other_before + k) & 1, ctl, a.status);
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -515,10 +582,10 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             }
             if (!ok) break;
 
-            ok = mbar_wait(bar(B_OFINAL0 + i), pc & 1, ctl, a.status);
+            ok = mbar_wait(bar(B_OFINAL0 + i), oc & 1, ctl, a.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            ++pc;
+            ++oc;
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
             const float lse2 = l > 0.f ? m_ref * sl2 + log2f(l) : -INFINITY;
@@ -595,7 +662,10 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
         g_range[1] = group_of((int64_t)(kvh + 1) * nt_all - 1);
     }
     __syncthreads();
-    const int g0 = g_range[0], np = g_range[1] - g0 + 1;     // pieces of this KV head
+    const int st = a.streams;
+    const int g0 = g_range[0], np = (g_range[1] - g0 + 1) * st;   // parts of this KV head: st per piece
+    // part s of the KV head sits in slot (g0 + s / st + kvh) * st + s % st
+    auto slot_of = [&](int s) { return (int64_t)(g0 + s / st + kvh) * st + s % st; };
     const int64_t nG = (int64_t)a.n * G;
     const int rows = kCombineTokens * G;                      // rows of this block, row = token * G + head-in-group
     for (int rr = warp; rr < rows; rr += 8) {
@@ -605,7 +675,7 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
         const int64_t row = (int64_t)tok * a.H + kvh * G + gi;
         float M = -INFINITY;
         for (int s0 = 0; s0 < np; s0 += 32) {
-            const float ls = s0 + lane < np ? a.part_lse[(int64_t)(g0 + s0 + lane + kvh) * nG + R] : -INFINITY;
+            const float ls = s0 + lane < np ? a.part_lse[slot_of(s0 + lane) * nG + R] : -INFINITY;
             M = fmaxf(M, ls);
         }
 #pragma unroll
@@ -618,8 +688,8 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
 #pragma unroll
             for (int s = 0; s < 8; ++s)
                 if (s < cnt)
-                    pv[s] = *reinterpret_cast<const float4 *>(a.part_o + ((int64_t)(g0 + s0 + s + kvh) * nG + R) * kD + lane * 4);
-            const float ls = lane < cnt ? a.part_lse[(int64_t)(g0 + s0 + lane + kvh) * nG + R] : -INFINITY;
+                    pv[s] = *reinterpret_cast<const float4 *>(a.part_o + (slot_of(s0 + s) * nG + R) * kD + lane * 4);
+            const float ls = lane < cnt ? a.part_lse[slot_of(s0 + lane) * nG + R] : -INFINITY;
             const float wl = ls == -INFINITY ? 0.f : exp2f(ls - M);
 #pragma unroll
             for (int s = 0; s < 8; ++s) {                     // group order: deterministic
@@ -652,6 +722,8 @@ bool attn_tc_supported(int dtype, int d, int G) {
 }
 
 int attn_tc_row_pairs(int n, int G) { return (n * G + 2 * kRows - 1) / (2 * kRows); }
+
+int attn_tc_streams(int n, int G) { return n * G <= kRows ? 2 : 1; }
 
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
     static_assert(sizeof(Ctl) <= 512, "control block");

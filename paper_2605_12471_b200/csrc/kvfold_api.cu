@@ -175,14 +175,15 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix) {
             groups = c->sm_count / pairs;
             if (groups > Hkv * nt / 4) groups = Hkv * nt / 4;
         }
-        const int64_t slots_cap = c->part_rows_cap / ((int64_t)n * c->G);   // slots = groups + Hkv - 1
+        const int streams = attn_tc_streams(n, c->G);
+        const int64_t slots_cap = c->part_rows_cap / ((int64_t)n * c->G) / streams;   // slots = streams * (groups + Hkv - 1)
         if (groups + Hkv - 1 > slots_cap) groups = slots_cap - (Hkv - 1);
         if (groups > Hkv * nt) groups = Hkv * nt;
         if (groups < Hkv) groups = Hkv;
         p.ngroups = (int)groups;
         p.splits = (int)((groups + Hkv - 1) / Hkv);
         p.ctas = pairs * p.ngroups;
-        p.kernels = 2 + (p.ngroups != Hkv ? 1 : 0);
+        p.kernels = 2 + ((p.ngroups != Hkv || streams == 2) ? 1 : 0);   // short chunks always leave two parts
         return p;
     }
     const int64_t nt = (L + 63) / 64;
@@ -282,6 +283,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
     aa.splits = plan.tc ? 1 : plan.splits;
     aa.ngroups = plan.ngroups;
+    aa.streams = plan.tc ? attn_tc_streams(n, c->G) : 1;
     aa.out_f32 = (f.dtype == KVF_F32 || (f.flags & KVF_OUT_F32)) ? 1 : 0;
     aa.scale_log2 = c->scale_log2;
 

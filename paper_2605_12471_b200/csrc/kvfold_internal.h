@@ -41,6 +41,7 @@ struct AttnArgs {
     int32_t n, H, Hkv, G, d;
     int32_t splits;                  // CUDA-core path: equal splits of the key range
     int32_t ngroups;                 // tensor-core path: contiguous ranges of the (KV head, key tile) line
+    int32_t streams;                 // tensor-core path: 2 = one row tile, its key tiles dealt to two streams
     int32_t out_f32;
     float scale_log2;                // softmax scale * log2(e)
 };
@@ -56,6 +57,7 @@ struct TcMaps {
 };
 bool attn_tc_supported(int dtype, int d, int G);
 int attn_tc_row_pairs(int n, int G);   // 256-row pairs per KV head = grid.x
+int attn_tc_streams(int n, int G);     // 2 when the chunk fits one 128-row tile
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s);   // grid (row pairs, ngroups)
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s);                // needed when ngroups != Hkv
 

@@ -310,3 +310,40 @@ def test_profile_counters_and_launch_count():
     assert cnt[0] == 4 and cnt[1] == 4
     assert cache.launch_count() == sum(cnt)
     assert all(m >= 0 for m in ms) and ms[1] > 0
+
+
+# ------------------------------------------------------------------ short chunks at depth
+def test_short_chunks_deep_in_a_chain_match_the_oracle():
+    """Decode- and question-shaped steps (1 .. 32 tokens: at most one 128-row tile) after a long
+    prefix: the kernel deals their key tiles to two streams and always merges partial results."""
+    w = SMALL_LLAMA.with_(name="short_chunks_at_depth", tokens=16384)
+    chunks = [2048] * 5 + [32] * 6 + [1] * 5 + [16, 31, 32, 7, 2, 32, 33, 64, 5]
+    check = list(range(5, len(chunks)))
+    res, cache, _, _ = run_chain(w, chunks, seed=19, check_steps=check, rows_per_step=3)
+    assert len(cache) == sum(chunks)
+    assert cache.plan(32, 10000)[3] == 3 and cache.plan(33, 10000)[1] >= 1
+    assert_within(res, "bf16", "short chunks at depth")
+    assert res.rel_rms <= 2e-2, res.rel_rms
+
+
+def test_short_chunk_chains_repeat_bitwise_without_host_synchronisation():
+    """The same chain of 32-token steps enqueued three times back to back (reset in between, no
+    synchronisation inside a chain) gives the same bits every time."""
+    w = SMALL_LLAMA.with_(name="short_chunks_async", tokens=12288 + 32 * 48)
+    cache = binding.cache_for(w, max_chunk=2048)
+    fq, fk, fv = workloads.chunk_inputs(w.with_(chunk=2048), 20, 0, device="cuda")
+    q, k, v = workloads.sequence_inputs(w.with_(tokens=32 * 48, chunk=32), 21, device="cuda")
+    outs = []
+    for rep in range(3):
+        cache.reset()
+        for _ in range(6):
+            cache.fold_step(fq, fk, fv)
+        out = torch.empty_like(q)
+        for t in range(48):
+            cache.fold_step(q[32 * t:32 * t + 32], k[32 * t:32 * t + 32], v[32 * t:32 * t + 32], out=out[32 * t:32 * t + 32])
+        outs.append(out)
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_OK
+    assert torch.isfinite(outs[0].float()).all()
+    for o in outs[1:]:
+        assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16))
