@@ -145,6 +145,12 @@ kvf_status kvf_cache_reset(kvf_cache *c);
  * streams that carried the steps. */
 kvf_status kvf_cache_status(kvf_cache *c);
 
+/* The raw device status word behind kvf_cache_status (same synchronisation): 0, or for the first
+ * bounded wait that gave up 5 + 256 * (index of the barrier in the kernel's control block)
+ * + 65536 * (waiting warp) + 2^24 * (awaited parity) - what a bug report should quote.
+ * -1 for a null handle or a failed copy. */
+int32_t kvf_cache_status_word(kvf_cache *c);
+
 /* Device pointers of the planes, [n_kv_heads][capacity][head_dim] of dtype. */
 void *kvf_cache_k_plane(const kvf_cache *c);
 void *kvf_cache_v_plane(const kvf_cache *c);

@@ -24,7 +24,7 @@ EXPORTS = [
     "kvf_fold_step_host", "kvf_cache_len", "kvf_cache_reset", "kvf_cache_status",
     "kvf_cache_k_plane", "kvf_cache_v_plane", "kvf_cache_plan", "kvf_cache_set_splits",
     "kvf_cache_launch_count", "kvf_cache_profile", "kvf_cache_profile_read", "kvf_cache_destroy",
-    "kvf_status_str", "kvf_last_cuda_error", "kvf_fold_step_static",
+    "kvf_status_str", "kvf_last_cuda_error", "kvf_fold_step_static", "kvf_cache_status_word",
 ]
 
 
@@ -79,6 +79,8 @@ def load() -> ctypes.CDLL:
     lib.kvf_cache_reset.restype = ctypes.c_int
     lib.kvf_cache_status.argtypes = [vp]
     lib.kvf_cache_status.restype = ctypes.c_int
+    lib.kvf_cache_status_word.argtypes = [vp]
+    lib.kvf_cache_status_word.restype = i32
     lib.kvf_cache_k_plane.argtypes = [vp]
     lib.kvf_cache_k_plane.restype = vp
     lib.kvf_cache_v_plane.argtypes = [vp]
@@ -206,6 +208,10 @@ class Cache:
 
     def status(self) -> int:
         return int(load().kvf_cache_status(self._h))
+
+    def status_word(self) -> int:
+        """Raw device status word (0 = no bounded wait gave up; see kvf_cache_status_word)."""
+        return int(load().kvf_cache_status_word(self._h))
 
     def _plane(self, ptr: int) -> torch.Tensor:
         plane_bytes = self.storage.numel() // 2

@@ -102,6 +102,13 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 
+// First timed-out wait of a launch leaves 5 (KVF_ERR_TIMEOUT) in the low byte of the status word,
+// the barrier's index in the control block in bits 8-15, the waiting warp in bits 16-23 and the
+// awaited parity in bit 24 (the barrier block is 1024-byte aligned, so the index is in the address).
+__device__ __forceinline__ void report_timeout(int *status, uint32_t bar, uint32_t parity) {
+    atomicCAS(status, 0, (int)(5u | (((bar & 1023u) >> 3) << 8) | ((threadIdx.x >> 5) << 16) | ((parity & 1u) << 24)));
+}
+
 // Bounded wait.  Returns false if the CTA is aborting or the limit ran out.
 __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, Ctl *ctl, int *status) {
     const unsigned long long t0 = global_ns();
@@ -112,7 +119,7 @@ __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, Ct
             if (*reinterpret_cast<volatile int *>(&ctl->abort)) return false;
             if (global_ns() - t0 > kWaitLimitNs) {
                 *reinterpret_cast<volatile int *>(&ctl->abort) = 1;
-                atomicExch(status, 5);   // KVF_ERR_TIMEOUT
+                report_timeout(status, bar, parity);
                 return false;
             }
         }
@@ -126,7 +133,7 @@ __device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity, i
     unsigned spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) == 0 && global_ns() - t0 > kWaitLimitNs) {
-            atomicExch(status, 5);   // KVF_ERR_TIMEOUT
+            report_timeout(status, bar, parity);
             return;
         }
     }
@@ -294,9 +301,11 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();   // everything above is private to the CTA; from here on the rotated chunk is read
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&ctl->tmem_base);
     // K/V tile slots.  Two row tiles: one ring of 5 that both issuers walk in step.  Two streams:
     // each stream owns a ring of 3 (the sixth slot is the second Q tile, unused there), because a
@@ -459,16 +468,36 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         const int64_t nG = (int64_t)n * G;
 
         int it = 0, oc = 0;            // my key tiles and my finished pieces so far
-        int other = 0;                 // key tiles the other tile slot has had so far
+        int turn_base = 0;             // turns (see below) both tile slots have taken before this piece
         bool ok = i < tiles;
         int kt0, ntiles;
         for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
             const int64_t prow = ((int64_t)(group + kvh) * streams + (streams == 2 ? i : 0)) * nG + R;   // my partial row
-            const int other_before = other;
-            {
-                const int oj0 = streams == 2 ? 1 - i : 0;            // the other slot's first key tile
-                other += ntiles > oj0 ? (ntiles - oj0 + jstep - 1) / jstep : 0;
-            }
+            // Turns on the exponentials: in every piece both tile slots take the same number of
+            // turns, slot 0 then slot 1, alternating strictly (a slot with fewer key tiles, which
+            // happens with two streams, passes its spare turns without doing anything).  Strict
+            // alternation is what a parity wait can follow: neither barrier is ever more than one
+            // phase away from what its waiter expects.
+            const int nturns = ntiles <= 0 ? 0 : (streams == 2 ? (ntiles + 1) / 2 : ntiles);
+            const int mine = ntiles > j0 ? (ntiles - j0 + jstep - 1) / jstep : 0;
+            auto take_turn = [&](int g) -> bool {      // wait until turn g of this slot may start
+                bool got = true;
+                if (i == 0) {
+                    if (g > 0) got = mbar_wait(bar(B_TURN0 + (warp & 3)), (g - 1) & 1, ctl, a.status);
+                } else {
+                    got = mbar_wait(bar(B_TURN0 + 4 + (warp & 3)), g & 1, ctl, a.status);
+                }
+                return __all_sync(0xffffffffu, got);
+            };
+            auto pass_spare_turns = [&]() -> bool {
+                for (int t = mine; t < nturns && tiles == 2; ++t) {
+                    if (!take_turn(turn_base + t)) return false;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(B_TURN0 + (i == 0 ? 4 : 0) + (warp & 3)));
+                }
+                turn_base += nturns;
+                return true;
+            };
             if (ntiles <= j0) {
                 // no visible key for these rows in this range: an empty partial
                 if (!direct && valid) {
@@ -477,6 +506,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                     for (int c = 0; c < kD / 4; ++c) po[c] = make_float4(0.f, 0.f, 0.f, 0.f);
                     a.part_lse[prow] = -INFINITY;
                 }
+                ok = pass_spare_turns();
                 continue;
             }
             float m_ref = -INFINITY;   // reference maximum (raw score units) the probabilities are scaled by
@@ -545,19 +575,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 // The two row tiles' warps that share a scheduler take turns on the exponentials:
                 // run side by side they halve each other's special-function rate and both tiles
                 // fall into step, leaving the tensor pipe idle while both are in their softmax.
-                // Slot 0's k-th tile of a piece goes after slot 1's (k-1)-th (for k = 0: after slot 1's
-                // last tile of the piece before), slot 1's k-th after slot 0's k-th; the partner's
-                // running count turns that into a barrier phase.  Neither slot can get two phases
-                // ahead of the other's wait, which a parity wait could not tell from none.
-                if (tiles == 1) {
-                    // nobody to take turns with
-                } else if (i == 0) {
-                    if (other_before + k > 0)
-                        ok = mbar_wait(bar(B_TURN0 + (warp & 3)), (other_before + k - 1) & 1, ctl, a.status);
-                } else {
-                    ok = mbar_wait(bar(B_TURN0 + 4 + (warp & 3)), (other_before + k) & 1, ctl, a.status);
-                }
-                ok = __all_sync(0xffffffffu, ok);
+                if (tiles == 2) ok = take_turn(turn_base + k);
                 if (!ok) break;
 
                 // probabilities; the first 64 keys are handed over before the rest is computed
@@ -580,6 +598,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 const float2 acc = __fadd2_rn(acc0, acc1);
                 l += acc.x + acc.y;
             }
+            if (!ok) break;
+            ok = pass_spare_turns();
             if (!ok) break;
 
             ok = mbar_wait(bar(B_OFINAL0 + i), oc & 1, ctl, a.status);
@@ -648,6 +668,7 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
     __shared__ int g_range[2];
     const int kvh = blockIdx.y, G = a.G;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         const int nt_all = (int)((a.prefix + a.n + kRows - 1) / kRows);
         const int64_t line = (int64_t)a.Hkv * nt_all;
@@ -662,6 +683,7 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
         g_range[1] = group_of((int64_t)(kvh + 1) * nt_all - 1);
     }
     __syncthreads();
+    pdl_wait();   // the parts are the attention kernel's output
     const int st = a.streams;
     const int g0 = g_range[0], np = (g_range[1] - g0 + 1) * st;   // parts of this KV head: st per piece
     // part s of the KV head sits in slot (g0 + s / st + kvh) * st + s % st
@@ -731,14 +753,12 @@ cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
     dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, 1);
-    attn_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(a, maps.q, maps.k, maps.v);
-    return cudaGetLastError();
+    return launch_pdl(attn_tc_kernel, grid, dim3(kThreads), kSmemBytes, s, a, maps.q, maps.k, maps.v);
 }
 
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s) {
     dim3 grid((a.n + kCombineTokens - 1) / kCombineTokens, a.Hkv, 1);
-    combine_groups_kernel<<<grid, 256, 0, s>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(combine_groups_kernel, grid, dim3(256), 0, s, a);
 }
 
 }  // namespace kvf

@@ -441,6 +441,14 @@ kvf_status kvf_cache_status(kvf_cache *c) {
     return word == 0 ? KVF_OK : KVF_ERR_TIMEOUT;
 }
 
+int32_t kvf_cache_status_word(kvf_cache *c) {
+    if (!c) return -1;
+    int word = 0;
+    cudaError_t e = cudaMemcpy(&word, c->workspace + c->lay.status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { cuda_fail(e, "cudaMemcpy(status)"); return -1; }
+    return word;
+}
+
 void *kvf_cache_k_plane(const kvf_cache *c) { return c ? c->storage : nullptr; }
 void *kvf_cache_v_plane(const kvf_cache *c) { return c ? c->storage + c->plane_bytes : nullptr; }
 

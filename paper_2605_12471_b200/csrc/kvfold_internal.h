@@ -7,6 +7,31 @@
 
 namespace kvf {
 
+// Programmatic dependent launch: a kernel launched with launch_pdl may be scheduled while the
+// kernel before it in the stream is still finishing; it must call pdl_wait() before it touches
+// anything an earlier kernel reads or writes (the wait returns when all earlier work in the
+// stream has completed and its memory is visible).  pdl_launch_dependents() lets the kernel
+// after this one be scheduled early in the same way.  Both are no-ops in a plain launch.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 constexpr int kMaxHalfDim = 64;       // head_dim <= 128
 constexpr int kKvTile = 128;          // key rows per tensor-core tile; V rows are zero-padded to it
 constexpr int kPartTokens = 4096;     // the partial area holds kPartTokens * H rows of head_dim floats

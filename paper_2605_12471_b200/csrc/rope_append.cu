@@ -66,7 +66,9 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
     const int d = a.d, half = d / 2;
     const int n_tok_blocks = (a.n + kTok - 1) / kTok;
 
+    pdl_launch_dependents();
     if ((int)blockIdx.x >= n_tok_blocks) {
+        pdl_wait();   // the attention of the step before may still be reading these rows' tile
         // Clear value rows between the new end of the cache and the next key-tile boundary,
         // so that a zero probability never multiplies stale non-finite bits.
         const int vec_per_row = d / VEC;
@@ -96,6 +98,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
         cs[t][j] = make_float2((float)cn, (float)sn);
     }
     __syncthreads();
+    pdl_wait();   // the table above needs nothing from earlier kernels; the writes below do
 
     const T *q = reinterpret_cast<const T *>(a.q);
     const T *k = reinterpret_cast<const T *>(a.k_new);
@@ -184,11 +187,11 @@ cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interlea
         blocks += (int)((vecs + kThreads - 1) / kThreads);
     }
     if (dtype == 0) {
-        if (interleaved) rope_append_kernel<__nv_bfloat16, true><<<blocks, kThreads, 0, s>>>(a);
-        else rope_append_kernel<__nv_bfloat16, false><<<blocks, kThreads, 0, s>>>(a);
+        if (interleaved) return launch_pdl(rope_append_kernel<__nv_bfloat16, true>, dim3(blocks), dim3(kThreads), 0, s, a);
+        else return launch_pdl(rope_append_kernel<__nv_bfloat16, false>, dim3(blocks), dim3(kThreads), 0, s, a);
     } else {
-        if (interleaved) rope_append_kernel<float, true><<<blocks, kThreads, 0, s>>>(a);
-        else rope_append_kernel<float, false><<<blocks, kThreads, 0, s>>>(a);
+        if (interleaved) return launch_pdl(rope_append_kernel<float, true>, dim3(blocks), dim3(kThreads), 0, s, a);
+        else return launch_pdl(rope_append_kernel<float, false>, dim3(blocks), dim3(kThreads), 0, s, a);
     }
     return cudaGetLastError();
 }

@@ -105,7 +105,7 @@ def run_chain(w: workloads.Workload, chunks: Sequence[int], seed: int = 0, flags
             res.lse_max_abs = max(res.lse_max_abs, float(np.abs(got_lse - ref_lse).max()))
         assert len(cache) == len(oc)
     torch.cuda.synchronize()
-    assert cache.status() == binding.KVF_OK
+    assert cache.status() == binding.KVF_OK, hex(cache.status_word())
     return res, cache, oc, outs
 
 
