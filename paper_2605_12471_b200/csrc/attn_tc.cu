@@ -37,12 +37,23 @@
 // scheduler's issue port, not the special-function unit alone, is what the softmax saturates.)
 //
 // The exponential phases of the two row tiles are sequenced per scheduler (warp w of tile 0 and
-// warp w of tile 1 alternate), which keeps the tiles in antiphase: one tile's softmax runs under
-// the other tile's MMAs.
+// warp w of tile 1 alternate strictly), which keeps the tiles in antiphase: one tile's softmax
+// runs under the other tile's MMAs.
+//
+// Short chunks (at most 128 / G tokens: decode, question chunk) have one row tile only.  The two
+// tile slots then work on the same 128 rows and take alternate key tiles ("two streams"), each
+// with its own accumulator, K/V ring of three slots and partial result, so the overlap of one
+// stream's softmax with the other's MMAs survives and the step runs at HBM speed.
 //
 // Every wait on an mbarrier is bounded (about one second): on expiry the thread raises the
-// CTA's abort flag and the device status word, all roles leave their loops, tensor memory is
-// released and the kernel returns.
+// CTA's abort flag and records the wait in the device status word, all roles leave their loops,
+// copies and MMAs still in flight are waited for (bounded again), tensor memory is released and
+// the kernel returns.  A parity wait is sound only for a thread that sees every phase of its
+// barrier in order and is never more than one phase away from it; the ring, the hand-over and
+// the turn protocols below are all built to that rule.
+//
+// The kernel may be launched while the kernel before it in the stream is finishing (programmatic
+// dependent launch): everything up to pdl_wait() is private to the CTA.
 #include "kvfold_internal.h"
 
 namespace kvf {
