@@ -202,6 +202,8 @@ def main():
     ap.add_argument("--prefill", type=int, default=0,
                     help="tokens folded (in 2048-token steps, untimed) before every timed chain: the timed chain "
                          "then runs from this prefix to --tokens (decode- and question-shaped steps at depth)")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"],
+                    help="cache and input dtype (f32 runs the CUDA-core path; not the benchmark workload)")
     ap.add_argument("--seed", type=int, default=2605)
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -210,9 +212,9 @@ def main():
     args = ap.parse_args()
 
     w = workloads.DEEP_CHAIN
-    if args.tokens or args.chunk or args.prefill:
-        w = w.with_(name=f"chain_{args.tokens or w.tokens}_c{args.chunk or w.chunk}_from_{args.prefill}",
-                    tokens=args.tokens or w.tokens, chunk=args.chunk or w.chunk)
+    if args.tokens or args.chunk or args.prefill or args.dtype != w.dtype:
+        w = w.with_(name=f"chain_{args.tokens or w.tokens}_c{args.chunk or w.chunk}_from_{args.prefill}_{args.dtype}",
+                    tokens=args.tokens or w.tokens, chunk=args.chunk or w.chunk, dtype=args.dtype)
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -335,7 +337,13 @@ def main():
     # which roof binds: arithmetic intensity G*C FLOP per cache byte against the ridge of the measured peaks
     ridge = pk["bf16_tflops_sustained"] * 1e12 / (pk["hbm_gbs"] * 1e9)
     intensity = attn_flops / cache_bytes_read
-    if intensity >= ridge:
+    if w.dtype == "f32":
+        # fp32 caches run on the CUDA cores (fp32 accuracy rules out single-pass tensor formats): the roof is
+        # the FFMA rate, 148 SMs x 128 lanes x 2 FLOP at the 1965 MHz maximum clock
+        alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
+        roofline = {"bound": "alu", "achieved": attn_tflops, "peak": alu_peak, "unit": "TFLOP/s",
+                    "frac": attn_tflops / alu_peak, "peak_source": "derived: 148 SMs x 128 FFMA lanes x 2 x 1.965 GHz"}
+    elif intensity >= ridge:
         roofline = {"bound": "tensor", "achieved": attn_tflops, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
                     "frac": attn_tflops / pk["bf16_tflops_sustained"], "peak_source": pk["_source"] + " sustained bf16"}
     else:
