@@ -191,6 +191,65 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_full_stack(args):
+    """Memory-scale fold (not the headline line): `--sequences` independent sequences x `--layers`
+    layers, each layer its own bf16 cache, 131 072 tokens per sequence in chunks of 1024; per chunk
+    all layers' fold steps are issued on one stream.  Every (sequence, layer) draws its chunk
+    inputs once from its own seed and reuses them for every chunk: values do not change the work,
+    and 16 384 fresh draws would not fit beside 64 GiB of cache."""
+    from paper_2605_12471_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the fold step has no CPU path")
+    torch.cuda.set_device(0)
+    w = workloads.FULL_STACK.with_(n_sequences=args.sequences, n_layers=args.layers, tokens=args.tokens or 131072)
+    C, T, N = w.chunk, w.tokens, w.n_steps
+    cfg = binding.make_config(w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, T, C, rope_base=w.rope_base)
+    ws = torch.empty(binding.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")     # one workspace, one stream
+    caches, inputs = [], []
+    for sq in range(w.n_sequences):
+        for ly in range(w.n_layers):
+            caches.append(binding.Cache(cfg, workspace=ws))
+            inputs.append(workloads.chunk_inputs(w, args.seed, 0, sequence=sq, layer=ly, device="cuda"))
+    out = torch.empty_like(inputs[0][0])
+    lib, stream = binding.load(), torch.cuda.current_stream().cuda_stream
+    ptrs = [(c._h, q.data_ptr(), k.data_ptr(), v.data_ptr()) for c, (q, k, v) in zip(caches, inputs)]
+
+    def chain():
+        for c in caches:
+            c.reset()
+        for t in range(N):
+            for h, qp, kp, vp in ptrs:
+                rc = lib.kvf_fold_step(h, qp, kp, vp, C, t * C, out.data_ptr(), None, stream)
+                if rc:
+                    raise binding.KvfError(rc, "kvf_fold_step")
+
+    sampler = ClockSampler(0)
+    chain()                                               # warm-up pass
+    torch.cuda.synchronize()
+    sampler.start()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    chain()
+    b.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = a.elapsed_time(b)
+    assert all(len(c) == T for c in caches) and all(c.status() == binding.KVF_OK for c in caches)
+    ncache = len(caches)
+    flops = ncache * w.flops_chain()
+    pk = peaks()
+    line = {"metric": "fold-step tokens/s", "value": ncache * T / (ms * 1e-3), "unit": "tokens/s (layer-tokens)", "n_gpus": 1,
+            "steps": 1, "warmup": 1, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": w.dtype, "data": "synthetic",
+            "config": {"workload": w.name, "sequences": w.n_sequences, "layers": w.n_layers, "tokens": T, "chunk": C,
+                       "caches": ncache, "cache_gib": ncache * binding.cache_storage_bytes(cfg) / 2 ** 30,
+                       "fold_steps": ncache * N, "l2": "inputs larger than L2"},
+            "attention_tflops_whole_step": flops / (ms * 1e-3) / 1e12,
+            "frac_of_sustained_bf16_peak": flops / (ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"],
+            "gpu_launches": sum(c.launch_count() for c in caches) // 2, "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -204,6 +263,10 @@ def main():
                          "then runs from this prefix to --tokens (decode- and question-shaped steps at depth)")
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"],
                     help="cache and input dtype (f32 runs the CUDA-core path; not the benchmark workload)")
+    ap.add_argument("--workload", default="deep_chain", choices=["deep_chain", "full_stack"],
+                    help="full_stack: the 4 x 32-layer memory-scale fold (64 GiB of cache; a separate, longer run)")
+    ap.add_argument("--sequences", type=int, default=4)
+    ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--seed", type=int, default=2605)
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -211,6 +274,9 @@ def main():
     ap.add_argument("--force-simt", action="store_true")
     args = ap.parse_args()
 
+    if args.workload == "full_stack" and args.impl == "ours":
+        run_full_stack(args)
+        return
     w = workloads.DEEP_CHAIN
     if args.tokens or args.chunk or args.prefill or args.dtype != w.dtype:
         w = w.with_(name=f"chain_{args.tokens or w.tokens}_c{args.chunk or w.chunk}_from_{args.prefill}_{args.dtype}",
