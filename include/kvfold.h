@@ -106,6 +106,25 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
                             void *dev_workspace, size_t workspace_bytes, kvf_cache **out);
 
 /*
+ * Paged variant of the accumulator (the paper's cache grows by appending; serving systems it
+ * cites manage such caches in fixed-size pages - Related work, "Chunked serving infrastructure").  bf16 caches
+ * with head_dim 128 only (KVF_ERR_UNSUPPORTED otherwise).
+ *   A page holds 128 consecutive tokens of every KV head: [K|V][n_kv_heads][128][head_dim].
+ *   dev_pool        device, 256-byte aligned, n_pool_pages pages (kvf_paged_pool_bytes); pages may be
+ *                   shared by many caches of the same shape
+ *   dev_page_table  device int32 array, entry i = pool page of tokens [128 i, 128 i + 128); needs
+ *                   ceil(capacity / 128) entries.  The caller owns it and may fill entries at any time
+ *                   before the step that first touches their tokens is enqueued (stream order).
+ * Everything else - workspace, steps, length, status - is as for kvf_cache_create; the plane
+ * accessors return NULL.  A step zeroes the value rows between the new end and the end of its
+ * page, so a page must not be shared between two live caches.
+ */
+size_t kvf_paged_pool_bytes(const kvf_config *cfg, int32_t n_pages);
+kvf_status kvf_paged_cache_create(const kvf_config *cfg, void *dev_pool, size_t pool_bytes, int32_t n_pool_pages,
+                                  const int32_t *dev_page_table, void *dev_workspace, size_t workspace_bytes,
+                                  kvf_cache **out);
+
+/*
  * One fold step at this layer (Section 2: queries from the new tokens, keys/values
  * [K_0;...;K_t], positions continued from the chunk's absolute start; Figure "KV-Fold":
  * the chunk's K/V are appended, the prefix is passed on unchanged).

@@ -25,6 +25,7 @@ EXPORTS = [
     "kvf_cache_k_plane", "kvf_cache_v_plane", "kvf_cache_plan", "kvf_cache_set_splits",
     "kvf_cache_launch_count", "kvf_cache_profile", "kvf_cache_profile_read", "kvf_cache_destroy",
     "kvf_status_str", "kvf_last_cuda_error", "kvf_fold_step_static", "kvf_cache_status_word",
+    "kvf_paged_pool_bytes", "kvf_paged_cache_create",
 ]
 
 
@@ -67,6 +68,10 @@ def load() -> ctypes.CDLL:
     lib.kvf_workspace_bytes.restype = ctypes.c_size_t
     lib.kvf_cache_create.argtypes = [cfgp, vp, ctypes.c_size_t, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
     lib.kvf_cache_create.restype = ctypes.c_int
+    lib.kvf_paged_pool_bytes.argtypes = [cfgp, i32]
+    lib.kvf_paged_pool_bytes.restype = ctypes.c_size_t
+    lib.kvf_paged_cache_create.argtypes = [cfgp, vp, ctypes.c_size_t, i32, vp, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
+    lib.kvf_paged_cache_create.restype = ctypes.c_int
     lib.kvf_fold_step.argtypes = [vp, vp, vp, vp, i32, i64, vp, vp, vp]
     lib.kvf_fold_step.restype = ctypes.c_int
     lib.kvf_fold_step_host.argtypes = [vp, vp, vp, vp, i32, i64, vp, vp, vp]
@@ -251,6 +256,50 @@ class Cache:
         if rc != KVF_OK:
             raise KvfError(rc, "kvf_cache_profile_read")
         return list(ms), list(cnt)
+
+
+class PagedCache(Cache):
+    """A cache whose rows live in 128-token pages of a shared pool (kvf_paged_cache_create).
+
+    `pool` is a uint8 CUDA tensor of n_pool_pages pages, `page_table` an int32 CUDA tensor with one
+    pool page number per 128 tokens of capacity; both stay owned by the caller.
+    """
+
+    def __init__(self, cfg: kvf_config, pool: torch.Tensor, n_pool_pages: int, page_table: torch.Tensor,
+                 workspace: torch.Tensor | None = None):
+        lib = load()
+        self.cfg = cfg
+        self.device = pool.device
+        assert page_table.dtype == torch.int32 and page_table.is_cuda and page_table.is_contiguous()
+        assert page_table.numel() >= (cfg.capacity + 127) // 128
+        wb = workspace_bytes(cfg)
+        self.storage, self.page_table = pool, page_table
+        self.workspace = workspace if workspace is not None else torch.empty(max(wb, 256), dtype=torch.uint8, device=pool.device)
+        h = ctypes.c_void_p()
+        with torch.cuda.device(self.device):
+            rc = lib.kvf_paged_cache_create(ctypes.byref(cfg), pool.data_ptr(), pool.numel(), n_pool_pages,
+                                            page_table.data_ptr(), self.workspace.data_ptr(), self.workspace.numel(),
+                                            ctypes.byref(h))
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_paged_cache_create")
+        self._h = h
+        self.torch_dtype = torch.bfloat16
+        self.out_dtype = torch.float32 if (cfg.flags & KVF_OUT_F32) else torch.bfloat16
+
+    def k_plane(self):
+        raise NotImplementedError("a paged cache has no planes; read rows through the page table")
+
+    v_plane = k_plane
+
+    def page_rows(self, kv: int) -> torch.Tensor:
+        """[pool pages, Hkv, 128, d] view of the K (kv = 0) or V (kv = 1) blocks of the pool."""
+        d, hkv = self.cfg.head_dim, self.cfg.n_kv_heads
+        pages = self.storage.view(torch.bfloat16).view(-1, 2, hkv, 128, d)
+        return pages[:, kv]
+
+
+def paged_pool_bytes(cfg: kvf_config, n_pages: int) -> int:
+    return int(load().kvf_paged_pool_bytes(ctypes.byref(cfg), n_pages))
 
 
 STATIC_SCRATCH_BYTES = 21234688

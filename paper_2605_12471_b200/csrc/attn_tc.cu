@@ -162,6 +162,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -329,6 +335,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             // ------------------------------------------------------------------ TMA producer
             int tg = 0, pc = 0;          // ring loads and pieces so far
             int rc[2] = {0, 0};          // loads so far into each stream's ring
+            int page = 0;                // paged cache: page of the key tile being loaded
             bool ok = true;
             int kt0, ntiles;
             for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
@@ -354,8 +361,15 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                     const CUtensorMap *m = (t & 1) ? &map_v : &map_k;
                     const int key0 = (kt0 + (t >> 1)) * kRows;
                     mbar_expect_tx(bar(B_FULL0 + slot), kTileBytes);
-                    tma_load_3d(slot_addr(slot), m, bar(B_FULL0 + slot), 0, key0, kvh);
-                    tma_load_3d(slot_addr(slot) + kPanel, m, bar(B_FULL0 + slot), 64, key0, kvh);
+                    if (a.page_table) {
+                        // paged cache: a key tile is one page; the maps are (d, row in page, KV head, page)
+                        if (!(t & 1)) page = a.page_table[kt0 + (t >> 1)];     // K then V of the same tile
+                        tma_load_4d(slot_addr(slot), m, bar(B_FULL0 + slot), 0, 0, kvh, page);
+                        tma_load_4d(slot_addr(slot) + kPanel, m, bar(B_FULL0 + slot), 64, 0, kvh, page);
+                    } else {
+                        tma_load_3d(slot_addr(slot), m, bar(B_FULL0 + slot), 0, key0, kvh);
+                        tma_load_3d(slot_addr(slot) + kPanel, m, bar(B_FULL0 + slot), 64, key0, kvh);
+                    }
                 }
             }
             // do not leave while a copy may still be writing into this CTA's shared memory

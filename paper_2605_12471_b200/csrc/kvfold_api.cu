@@ -95,6 +95,9 @@ struct kvf_cache {
     int64_t part_rows_cap;   // rows of head_dim floats the partial area holds
     uint64_t launches;
     bool profile;
+    const int32_t *page_table = nullptr;   // paged cache: device table, one page number per 128 tokens
+    int64_t page_elems = 0;                // paged cache: elements per page
+    int32_t n_pool_pages = 0;
     std::vector<ProfRec> recs;
     std::vector<cudaEvent_t> pool;
 };
@@ -123,6 +126,25 @@ kvf_status make_map(EncodeTiledFn fn, CUtensorMap *m, void *base, uint64_t dim_y
     return KVF_OK;
 }
 
+// 4-D bf16 tensor map of a page pool: (x = head_dim, row in page, KV head, page); `base` is the K or
+// the V block of page 0, consecutive pages are page_bytes apart.
+kvf_status make_page_map(EncodeTiledFn fn, CUtensorMap *m, void *base, int d, int Hkv, uint64_t n_pages,
+                         uint64_t page_bytes) {
+    const uint64_t row = (uint64_t)d * 2;
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)kKvTile, (cuuint64_t)Hkv, n_pages};
+    cuuint64_t strides[3] = {row, row * kKvTile, page_bytes};
+    cuuint32_t box[4] = {64u, (cuuint32_t)kKvTile, 1u, 1u};
+    cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled (page pool) failed with CUresult %d", (int)r);
+        return KVF_ERR_CUDA;
+    }
+    return KVF_OK;
+}
+
 kvf_status build_maps(kvf_cache *c) {
     void *sym = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -141,6 +163,13 @@ kvf_status build_maps(kvf_cache *c) {
                             (uint64_t)f.max_chunk, row, row * f.n_q_heads, d, (uint32_t)c->G,
                             (uint32_t)(128 / c->G));
     if (s != KVF_OK) return s;
+    if (c->page_table) {
+        const uint64_t page_bytes = (uint64_t)c->page_elems * 2;
+        s = make_page_map(fn, &c->maps.k, c->storage, d, f.n_kv_heads, (uint64_t)c->n_pool_pages, page_bytes);
+        if (s != KVF_OK) return s;
+        return make_page_map(fn, &c->maps.v, c->storage + c->plane_bytes, d, f.n_kv_heads, (uint64_t)c->n_pool_pages,
+                             page_bytes);
+    }
     // planes [Hkv][capacity][d]: one box = 128 rows of one head x 64
     s = make_map(fn, &c->maps.k, c->storage, (uint64_t)f.capacity, (uint64_t)f.n_kv_heads, row,
                  row * f.capacity, d, (uint32_t)kKvTile, 1u);
@@ -267,9 +296,11 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     {
         int64_t L = P + n;
         int64_t pad_end = (L + kKvTile - 1) / kKvTile * kKvTile;
-        if (pad_end > f.capacity) pad_end = f.capacity;
+        if (pad_end > f.capacity && !c->page_table) pad_end = f.capacity;   // a page always has its 128 rows
         ra.zero_rows = (int32_t)(pad_end - L);
     }
+    ra.page_table = c->page_table;
+    ra.page_elems = c->page_elems;
     ra.table = c->table;
 
     AttnArgs aa;
@@ -279,6 +310,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.part_o = reinterpret_cast<float *>(c->workspace + c->lay.part_o);
     aa.part_lse = reinterpret_cast<float *>(c->workspace + c->lay.part_lse);
     aa.status = reinterpret_cast<int *>(c->workspace + c->lay.status);
+    aa.page_table = c->page_table;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
     aa.splits = plan.tc ? 1 : plan.splits;
@@ -388,6 +420,68 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
     return KVF_OK;
 }
 
+size_t kvf_paged_pool_bytes(const kvf_config *cfg, int32_t n_pages) {
+    if (check_config(cfg) != KVF_OK || n_pages <= 0) return 0;
+    return (size_t)n_pages * 2 * (size_t)cfg->n_kv_heads * kKvTile * (size_t)cfg->head_dim * elem_bytes(cfg->dtype);
+}
+
+kvf_status kvf_paged_cache_create(const kvf_config *cfg, void *dev_pool, size_t pool_bytes, int32_t n_pool_pages,
+                                  const int32_t *dev_page_table, void *dev_workspace, size_t workspace_bytes,
+                                  kvf_cache **out) {
+    if (!out) return KVF_ERR_INVALID_ARG;
+    *out = nullptr;
+    kvf_status s = check_config(cfg);
+    if (s != KVF_OK) return s;
+    const int G = cfg->n_q_heads / cfg->n_kv_heads;
+    if ((cfg->flags & KVF_FORCE_SIMT) || !attn_tc_supported(cfg->dtype, cfg->head_dim, G)) return KVF_ERR_UNSUPPORTED;
+    if (!dev_pool || !dev_workspace || !dev_page_table || n_pool_pages <= 0) return KVF_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(dev_pool) & 255u) || (reinterpret_cast<uintptr_t>(dev_workspace) & 255u) ||
+        (reinterpret_cast<uintptr_t>(dev_page_table) & 3u))
+        return KVF_ERR_INVALID_ARG;
+    if (pool_bytes < kvf_paged_pool_bytes(cfg, n_pool_pages)) return KVF_ERR_CAPACITY;
+    if (workspace_bytes < kvf_workspace_bytes(cfg)) return KVF_ERR_CAPACITY;
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+
+    kvf_cache *c = new (std::nothrow) kvf_cache();
+    if (!c) return KVF_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->cfg.inv_freq = nullptr;
+    c->device = dev;
+    c->sm_count = sms;
+    c->storage = static_cast<char *>(dev_pool);
+    c->workspace = static_cast<char *>(dev_workspace);
+    c->page_table = dev_page_table;
+    c->n_pool_pages = n_pool_pages;
+    c->page_elems = (int64_t)2 * cfg->n_kv_heads * kKvTile * cfg->head_dim;
+    c->plane_bytes = (size_t)cfg->n_kv_heads * kKvTile * cfg->head_dim * elem_bytes(cfg->dtype);   // V block inside a page
+    c->lay = workspace_layout(cfg);
+    c->len = 0;
+    c->G = G;
+    const double scale = cfg->softmax_scale > 0.0 ? cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
+    c->scale_log2 = (float)(scale * 1.4426950408889634);
+    for (int j = 0; j < cfg->head_dim / 2; ++j)
+        c->table.inv_freq[j] = cfg->inv_freq ? cfg->inv_freq[j]
+                                             : std::pow(cfg->rope_base, -2.0 * (double)j / (double)cfg->head_dim);
+    for (int j = cfg->head_dim / 2; j < kMaxHalfDim; ++j) c->table.inv_freq[j] = 0.0;
+    c->force_splits = 0;
+    c->part_rows_cap = (int64_t)kPartTokens * cfg->n_q_heads;
+    c->launches = 0;
+    c->profile = false;
+    c->tc = true;
+    s = build_maps(c);
+    if (s != KVF_OK) { delete c; return s; }
+    e = cudaMemset(c->workspace + c->lay.status, 0, 256);
+    if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaMemset(status)"); }
+    *out = c;
+    return KVF_OK;
+}
+
 kvf_status kvf_fold_step(kvf_cache *c, const void *q, const void *k_new, const void *v_new,
                          int32_t n_tokens, int64_t pos0, void *out, float *lse, void *cuda_stream) {
     kvf_status s = check_step(c, n_tokens, pos0);
@@ -449,8 +543,8 @@ int32_t kvf_cache_status_word(kvf_cache *c) {
     return word;
 }
 
-void *kvf_cache_k_plane(const kvf_cache *c) { return c ? c->storage : nullptr; }
-void *kvf_cache_v_plane(const kvf_cache *c) { return c ? c->storage + c->plane_bytes : nullptr; }
+void *kvf_cache_k_plane(const kvf_cache *c) { return c && !c->page_table ? c->storage : nullptr; }
+void *kvf_cache_v_plane(const kvf_cache *c) { return c && !c->page_table ? c->storage + c->plane_bytes : nullptr; }
 
 kvf_status kvf_cache_plan(const kvf_cache *c, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]) {
     if (!c || !plan || n_tokens < 1 || n_tokens > c->cfg.max_chunk || prefix_len < 0) return KVF_ERR_INVALID_ARG;

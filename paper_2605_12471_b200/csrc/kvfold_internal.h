@@ -41,6 +41,24 @@ struct RopeTable {
     double inv_freq[kMaxHalfDim];
 };
 
+// Where cache row `row` of KV head `g` lives, in elements from the plane's base pointer.
+// Contiguous cache: planes are [Hkv][capacity][d].  Paged cache: a page is kKvTile tokens of every
+// KV head, K block then V block ([2][Hkv][kKvTile][d]); the K "plane" pointer is the pool's base,
+// the V one is one block further, and page_table[row / kKvTile] names the page.
+struct RowMap {
+    const int32_t *page_table;   // null = contiguous
+    int64_t capacity;            // contiguous: rows per head
+    int64_t page_elems;          // paged: elements of one page (2 * Hkv * kKvTile * d)
+    int32_t d;
+#ifdef __CUDACC__
+    __device__ __forceinline__ int64_t offset(int g, int64_t row) const {
+        if (page_table == nullptr) return ((int64_t)g * capacity + row) * d;
+        const int64_t page = page_table[row / kKvTile];
+        return page * page_elems + ((int64_t)g * kKvTile + row % kKvTile) * d;
+    }
+#endif
+};
+
 // Arguments of the fused rotate + append kernel (one launch per step).
 struct RopeAppendArgs {
     const void *q, *k_new, *v_new;   // [n][H][d], [n][Hkv][d], [n][Hkv][d]
@@ -49,6 +67,8 @@ struct RopeAppendArgs {
     int64_t capacity, prefix, pos0;  // prefix = rows already held
     int32_t n, H, Hkv, d;
     int32_t zero_rows;               // value rows [prefix+n, prefix+n+zero_rows) are cleared
+    const int32_t *page_table;       // paged cache: device table of page numbers, else null
+    int64_t page_elems;              // paged cache: elements per page
     RopeTable table;
 };
 
@@ -62,6 +82,7 @@ struct AttnArgs {
                                      // [splits][n][H][d]; tensor-core path [slot][n * G][d]
     float *part_lse;                 // log2 denominators of the parts, same order; -inf = no key seen
     int *status;                     // device status word
+    const int32_t *page_table;       // paged cache: device table of page numbers (one per key tile), else null
     int64_t capacity, prefix;
     int32_t n, H, Hkv, G, d;
     int32_t splits;                  // CUDA-core path: equal splits of the key range

@@ -65,6 +65,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
 
     const int d = a.d, half = d / 2;
     const int n_tok_blocks = (a.n + kTok - 1) / kTok;
+    const RowMap rows{a.page_table, a.capacity, a.page_elems, a.d};
 
     pdl_launch_dependents();
     if ((int)blockIdx.x >= n_tok_blocks) {
@@ -81,7 +82,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             int64_t t = i / vec_per_row;
             int g = (int)(t % a.Hkv);
             int64_t row = a.prefix + a.n + t / a.Hkv;
-            *reinterpret_cast<uint4 *>(vp + ((int64_t)g * a.capacity + row) * d + c * VEC) =
+            *reinterpret_cast<uint4 *>(vp + rows.offset(g, row) + c * VEC) =
                 make_uint4(0, 0, 0, 0);
         }
         return;
@@ -123,7 +124,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             } else {
                 int g = hh - a.H;
                 src = k + ((int64_t)(tok0 + t) * a.Hkv + g) * d;
-                dst = kp + ((int64_t)g * a.capacity + a.prefix + tok0 + t) * d;
+                dst = kp + rows.offset(g, a.prefix + tok0 + t);
             }
             float lo[VEC], hi[VEC], rlo[VEC], rhi[VEC];
             Vec16<T>::load(src + c * VEC, lo);
@@ -151,7 +152,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             } else {
                 int g = hh - a.H;
                 src = k + ((int64_t)(tok0 + t) * a.Hkv + g) * d;
-                dst = kp + ((int64_t)g * a.capacity + a.prefix + tok0 + t) * d;
+                dst = kp + rows.offset(g, a.prefix + tok0 + t);
             }
             float x[VEC], r[VEC];
             Vec16<T>::load(src + c * VEC, x);
@@ -173,7 +174,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             int g = (idx / chunks) % a.Hkv;
             int t = idx / (chunks * a.Hkv);
             uint4 val = *reinterpret_cast<const uint4 *>(v + ((int64_t)(tok0 + t) * a.Hkv + g) * d + c * VEC);
-            *reinterpret_cast<uint4 *>(vp + ((int64_t)g * a.capacity + a.prefix + tok0 + t) * d + c * VEC) = val;
+            *reinterpret_cast<uint4 *>(vp + rows.offset(g, a.prefix + tok0 + t) + c * VEC) = val;
         }
     }
 }

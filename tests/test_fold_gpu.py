@@ -347,3 +347,56 @@ def test_short_chunk_chains_repeat_bitwise_without_host_synchronisation():
     assert torch.isfinite(outs[0].float()).all()
     for o in outs[1:]:
         assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16))
+
+
+# ------------------------------------------------------------------ paged cache
+def test_paged_cache_matches_the_contiguous_cache_and_the_oracle():
+    """Rows in 128-token pages scattered over a shared pool: same bits as the contiguous cache
+    (the arithmetic does not depend on where a row lives) and within tolerance of the oracle."""
+    w = SMALL_LLAMA.with_(name="paged", tokens=4096)
+    chunks = [256, 256, 100, 1, 411, 32, 7, 1024, 33, 128, 5]
+    total = sum(chunks)
+    cfg = binding.make_config(w.n_q_heads, w.n_kv_heads, w.head_dim, "bf16", total, max(chunks), rope_base=w.rope_base)
+    n_table = (total + 127) // 128
+    n_pool = 2 * n_table + 3
+    gen = torch.Generator().manual_seed(5)
+    perm = torch.randperm(n_pool, generator=gen)[:n_table].to(torch.int32)        # scattered, not in order
+    table = perm.cuda()
+    pool = torch.empty(binding.paged_pool_bytes(cfg, n_pool), dtype=torch.uint8, device="cuda")
+    pool.view(torch.int16).fill_(0x7FC0)                                          # NaN everywhere a row was never written
+    paged = binding.PagedCache(cfg, pool, n_pool, table)
+    flat = binding.Cache(cfg)
+    oc = oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, total, rope_base=w.rope_base)
+    worst = 0.0
+    for t, n in enumerate(chunks):
+        q, k, v = workloads.chunk_inputs(w, 23, t, device="cuda", n_tokens=n)
+        got = paged.fold_step(q, k, v)
+        want = flat.fold_step(q, k, v)
+        assert torch.equal(got.view(torch.int16), want.view(torch.int16)), f"step {t}"
+        ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=[0, n - 1])
+        worst = max(worst, float(np.abs(to_f64(got[[0, n - 1]]) - ref).max()))
+    torch.cuda.synchronize()
+    assert len(paged) == total and paged.status() == binding.KVF_OK
+    assert worst <= TOL["bf16"][0]
+    # the rows are where the table says
+    kp, vp = paged.page_rows(0), paged.page_rows(1)
+    fk, fv = flat.k_plane(), flat.v_plane()
+    for i in (0, 3, n_table - 1):
+        rows = min(128, total - 128 * i)
+        assert torch.equal(kp[int(perm[i]), :, :rows], fk[:, 128 * i:128 * i + rows])
+        assert torch.equal(vp[int(perm[i]), :, :rows], fv[:, 128 * i:128 * i + rows])
+
+
+def test_paged_cache_rejects_what_it_does_not_cover():
+    lib = binding.load()
+    cfg32 = binding.make_config(32, 8, 128, "f32", 1024, 256, rope_base=5e5)
+    buf = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    table = torch.zeros(8, dtype=torch.int32, device="cuda")
+    h = ctypes.c_void_p()
+    rc = lib.kvf_paged_cache_create(ctypes.byref(cfg32), buf.data_ptr(), buf.numel(), 1, table.data_ptr(), buf.data_ptr(),
+                                    buf.numel(), ctypes.byref(h))
+    assert rc == binding.KVF_ERR_UNSUPPORTED
+    cfg = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5)
+    rc = lib.kvf_paged_cache_create(ctypes.byref(cfg), buf.data_ptr(), buf.numel(), 8, table.data_ptr(), buf.data_ptr(),
+                                    buf.numel(), ctypes.byref(h))
+    assert rc == binding.KVF_ERR_CAPACITY                     # 8 pages need 4 MiB
