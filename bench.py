@@ -272,6 +272,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--force-simt", action="store_true")
+    ap.add_argument("--paged", action="store_true", help="keep the cache in shuffled 128-token pages of a pool")
     args = ap.parse_args()
 
     if args.workload == "full_stack" and args.impl == "ours":
@@ -307,7 +308,14 @@ def main():
     q, k, v = workloads.sequence_inputs(wt, args.seed, sequence=seq, device="cuda")
     out = torch.empty_like(q)
     flags = binding.KVF_FORCE_SIMT if args.force_simt else 0
-    cache = binding.cache_for(w, flags=flags, max_chunk=max(C, 2048 if P0 else C))
+    if args.paged:
+        cfg = binding.make_config(H, Hkv, d, w.dtype, T, max(C, 2048 if P0 else C), rope_base=w.rope_base, flags=flags)
+        n_table = (T + 127) // 128
+        table = torch.randperm(n_table, generator=torch.Generator().manual_seed(args.seed)).to(torch.int32).cuda()
+        pool = torch.empty(binding.paged_pool_bytes(cfg, n_table), dtype=torch.uint8, device="cuda")
+        cache = binding.PagedCache(cfg, pool, n_table, table)
+    else:
+        cache = binding.cache_for(w, flags=flags, max_chunk=max(C, 2048 if P0 else C))
     h = cache._h
     stream = torch.cuda.current_stream().cuda_stream
     eb = q.element_size()
@@ -462,7 +470,7 @@ def main():
             "data": "synthetic",
             "config": {"workload": w.name, "tokens": T, "chunk": C, "prefill": P0, "fold_steps_per_step": N,
                        "n_q_heads": H, "n_kv_heads": Hkv, "head_dim": d, "rope_base": w.rope_base,
-                       "sequences_per_gpu": 1, "l2": "inputs larger than L2 (cache grows to 512 MiB per chain)",
+                       "sequences_per_gpu": 1, "paged": bool(args.paged), "l2": "inputs larger than L2 (cache grows to 512 MiB per chain)",
                        "last_step_plan": {"tensor_core": plan[0], "splits": plan[1], "ctas": plan[2]}},
             "attention_tflops": step_flops / (ms * 1e-3) / 1e12,
             "roofline": roofline, "latency_vs_prefix": curve, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,

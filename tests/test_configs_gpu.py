@@ -75,3 +75,49 @@ def test_config5_layer_stack_reduced():
             worst = max(worst, float(np.abs(to_f64(out[rows]) - ref).max()))
     assert all(len(c) == w.tokens for c in caches.values())
     assert worst <= TOL["bf16"][0]
+
+
+def test_config5_full_stack_64_gib_sampled_pairs():
+    """Config 5 at full size: 4 sequences x 32 layers, one 512 MiB bf16 cache each (64 GiB), 131 072
+    tokens per sequence in chunks of 1024, every chunk's 128 fold steps issued on one stream with one
+    shared workspace.  Each (sequence, layer) draws one chunk of inputs from its own seed and feeds it
+    at every chunk (the positions and the prefix still change), as the benchmark does; the oracle
+    follows two (sequence, layer) pairs and checks sampled rows at sampled chunks."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 80 * 2 ** 30:
+        pytest.skip("needs 80 GiB of free device memory")
+    w = workloads.FULL_STACK
+    C, T, N = w.chunk, w.tokens, w.n_steps
+    cfg = binding.make_config(w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, T, C, rope_base=w.rope_base)
+    ws = torch.empty(binding.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    keys = [(s, l) for s in range(w.n_sequences) for l in range(w.n_layers)]
+    caches = {key: binding.Cache(cfg, workspace=ws) for key in keys}
+    inputs = {key: workloads.chunk_inputs(w, 25, 0, sequence=key[0], layer=key[1], device="cuda") for key in keys}
+    watched = [(0, 0), (3, 17)]
+    oracles = {key: oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, T, rope_base=w.rope_base) for key in watched}
+    host_in = {key: tuple(to_f64(x) for x in inputs[key]) for key in watched}
+    check_chunks = {0, 1, N // 2, N - 1}
+    rows = [0, C // 2 - 1, C - 1]
+    outs = {key: torch.empty_like(inputs[key][0]) for key in watched}
+    scratch = torch.empty_like(inputs[keys[0]][0])
+    worst, err_sq, ref_sq = 0.0, 0.0, 0.0
+    for t in range(N):
+        for key in keys:
+            q, k, v = inputs[key]
+            caches[key].fold_step(q, k, v, out=outs[key] if key in outs else scratch)
+        for key in watched:
+            q, k, v = host_in[key]
+            if t in check_chunks:
+                ref = oracles[key].fold_step(q, k, v, rows=rows)
+                got = to_f64(outs[key][rows])
+                worst = max(worst, float(np.abs(got - ref).max()))
+                err_sq += float(((got - ref) ** 2).sum())
+                ref_sq += float((ref ** 2).sum())
+            else:
+                oracles[key].fold_step(q, k, v, rows=[])
+    torch.cuda.synchronize()
+    assert all(len(c) == T for c in caches.values())
+    assert all(c.status() == binding.KVF_OK for c in caches.values())
+    assert worst <= TOL["bf16"][0], worst
+    assert (err_sq / ref_sq) ** 0.5 <= 2e-2
+    print(f"config5 full size: max abs {worst:.2e}, rel rms {(err_sq / ref_sq) ** 0.5:.2e}")
