@@ -177,9 +177,13 @@ void *kvf_cache_v_plane(const kvf_cache *c);
 /*
  * What a step of n_tokens on a prefix of prefix_len would launch:
  *   plan[0] 1 = tensor-core (tcgen05) attention kernel, 0 = CUDA-core kernel
- *   plan[1] number of splits over the key range (1 = none, no combine kernel)
+ *   plan[1] parts the key range of one KV head is cut into (1 = none).  CUDA-core kernel: equal
+ *           splits.  Tensor-core kernel: the (KV head, key tile) pairs are cut into plan[2] /
+ *           (row pairs) contiguous ranges that need not end at KV-head boundaries; this is their
+ *           number per KV head, rounded up
  *   plan[2] CTAs of the attention kernel
- *   plan[3] kernels launched by the step
+ *   plan[3] kernels launched by the step (3 = a combine kernel merges partial results; chunks of
+ *           at most 128 / (H / Hkv) tokens always take that route on the tensor-core path)
  */
 kvf_status kvf_cache_plan(const kvf_cache *c, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]);
 

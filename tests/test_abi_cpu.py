@@ -96,9 +96,26 @@ def test_null_handles_are_harmless(binding):
     assert lib.kvf_fold_step(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_fold_step_host(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_cache_launch_count(None) == 0
+    assert lib.kvf_cache_status_word(None) == -1
+    assert lib.kvf_cache_k_plane(None) is None
     lib.kvf_cache_destroy(None)
     assert lib.kvf_status_str(0).decode() == "KVF_OK"
     assert lib.kvf_status_str(5).decode() == "KVF_ERR_TIMEOUT"
+
+
+def test_paged_entry_points_validate_before_any_cuda_call(binding):
+    import ctypes
+    lib = binding.load()
+    cfg = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5)
+    assert binding.paged_pool_bytes(cfg, 8) == 8 * 2 * 8 * 128 * 128 * 2          # pages x (K,V) x heads x rows x d x bytes
+    assert binding.paged_pool_bytes(cfg, 0) == 0
+    h = ctypes.c_void_p()
+    assert lib.kvf_paged_cache_create(ctypes.byref(cfg), None, 0, 8, None, None, 0, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
+    f32 = binding.make_config(32, 8, 128, "f32", 1024, 256, rope_base=5e5)
+    assert lib.kvf_paged_cache_create(ctypes.byref(f32), 256, 1 << 30, 8, 256, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_UNSUPPORTED
+    d64 = binding.make_config(4, 1, 64, "bf16", 1024, 256)
+    assert lib.kvf_paged_cache_create(ctypes.byref(d64), 256, 1 << 30, 8, 256, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_UNSUPPORTED
+    assert lib.kvf_paged_cache_create(ctypes.byref(cfg), 256, 1 << 30, 8, 258, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
 
 
 def test_binding_fails_loudly_without_the_library(binding, monkeypatch, tmp_path):
