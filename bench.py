@@ -273,6 +273,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--force-simt", action="store_true")
     ap.add_argument("--paged", action="store_true", help="keep the cache in shuffled 128-token pages of a pool")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="launch every fold step of the timed chains from the host instead of replaying the chain "
+                         "as one CUDA graph captured from the same kvf_fold_step calls")
     args = ap.parse_args()
 
     if args.workload == "full_stack" and args.impl == "ours":
@@ -317,7 +320,7 @@ def main():
     else:
         cache = binding.cache_for(w, flags=flags, max_chunk=max(C, 2048 if P0 else C))
     h = cache._h
-    stream = torch.cuda.current_stream().cuda_stream
+    launch_stream = [torch.cuda.current_stream().cuda_stream]
     eb = q.element_size()
     qs, ks = C * H * d * eb, C * Hkv * d * eb
     qp, kp, vp, op = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr()
@@ -333,7 +336,8 @@ def main():
 
     def body(first=0, last=None):
         for t in range(first, N if last is None else last):
-            rc = lib.kvf_fold_step(h, qp + t * qs, kp + t * ks, vp + t * ks, C, P0 + t * C, op + t * qs, None, stream)
+            rc = lib.kvf_fold_step(h, qp + t * qs, kp + t * ks, vp + t * ks, C, P0 + t * C, op + t * qs, None,
+                                   launch_stream[0])
             if rc:
                 raise binding.KvfError(rc, "kvf_fold_step")
 
@@ -369,12 +373,28 @@ def main():
     for _ in range(args.warmup):
         prefill()
         body()
+    # The chain's launches are fixed once the sizes are (every step's prefix is a kernel argument), so the
+    # timed chains replay one CUDA graph captured from the very kvf_fold_step calls of body().  The host's
+    # row count advances during the capture only; a replay needs no reset.
+    graph, run_chain = None, body
+    if not args.no_graph:
+        prefill()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            launch_stream[0] = torch.cuda.current_stream().cuda_stream
+            body()
+        launch_stream[0] = torch.cuda.current_stream().cuda_stream
+        run_chain = graph.replay
+        prefill()
+        run_chain()                                      # one untimed replay (uploads the graph)
+        torch.cuda.synchronize()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms = timed(body, args.steps)
+    ms = timed(run_chain, args.steps)
     clocks = sampler.stop() if rank == 0 else None
-    assert len(cache) == T
+    assert graph is not None or len(cache) == T
     if cache.status() != binding.KVF_OK:
         raise SystemExit("device status word reports a timed-out wait")
     value = multi.whole_job_tokens_per_s(T - P0, args.steps, world, ms)
@@ -440,7 +460,7 @@ def main():
         def body_host():
             for t in range(N):
                 rc = lib.kvf_fold_step_host(h, qhp + t * qs, khp + t * ks, vhp + t * ks, C, P0 + t * C, ohp + t * qs,
-                                            None, stream)
+                                            None, launch_stream[0])
                 if rc:
                     raise binding.KvfError(rc, "kvf_fold_step_host")
 
@@ -470,7 +490,8 @@ def main():
             "data": "synthetic",
             "config": {"workload": w.name, "tokens": T, "chunk": C, "prefill": P0, "fold_steps_per_step": N,
                        "n_q_heads": H, "n_kv_heads": Hkv, "head_dim": d, "rope_base": w.rope_base,
-                       "sequences_per_gpu": 1, "paged": bool(args.paged), "l2": "inputs larger than L2 (cache grows to 512 MiB per chain)",
+                       "sequences_per_gpu": 1, "paged": bool(args.paged),
+                       "launch": "per-step host launches" if graph is None else "one CUDA graph per chain, captured from the same calls", "l2": "inputs larger than L2 (cache grows to 512 MiB per chain)",
                        "last_step_plan": {"tensor_core": plan[0], "splits": plan[1], "ctas": plan[2]}},
             "attention_tflops": step_flops / (ms * 1e-3) / 1e12,
             "roofline": roofline, "latency_vs_prefix": curve, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
