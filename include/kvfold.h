@@ -207,6 +207,53 @@ kvf_status kvf_cache_profile_read(kvf_cache *c, double ms[3], uint64_t launches[
 void kvf_cache_destroy(kvf_cache *c);
 
 /*
+ * One launch over many caches.  The paper's fold runs once per layer (and per sequence) for every
+ * chunk, each layer with its own accumulated K/V (Section 2: the per-layer caches of chunk t are
+ * what chunk t+1 attends to); a 32-layer model folding 4 sequences has 128 caches that all stand
+ * at the same length.  A batch folds one chunk into every member with ONE launch of each kernel
+ * instead of one per cache: the members' CTAs fill the GPU together, which matters while the
+ * prefix is short or the chunk is small.
+ *
+ * Members: caches made by kvf_paged_cache_create over the SAME pool with the same configuration
+ * (they share the pool's tensor maps; each keeps its own page table), no cache twice; otherwise
+ * KVF_ERR_UNSUPPORTED (not paged) or KVF_ERR_INVALID_ARG.  The handles stay owned by the caller,
+ * stay usable on their own between batch steps, and must outlive the batch.
+ * dev_workspace: caller-owned, 256-byte aligned, kvf_batch_workspace_bytes(cfg, n_caches) bytes
+ * (0 = invalid arguments; n_caches 1..65535): the rotated chunks of all members, their partial
+ * results and one status word.  Creation copies the members' table pointers into it (blocking).
+ */
+typedef struct kvf_batch kvf_batch;
+size_t kvf_batch_workspace_bytes(const kvf_config *cfg, int32_t n_caches);
+kvf_status kvf_batch_create(kvf_cache *const *caches, int32_t n_caches, void *dev_workspace,
+                            size_t workspace_bytes, kvf_batch **out);
+
+/*
+ * kvf_fold_step for every member at once.  q, out: [n_caches][n_tokens][n_q_heads][head_dim];
+ * k_new, v_new: [n_caches][n_tokens][n_kv_heads][head_dim]; lse_or_null: [n_caches][n_tokens]
+ * [n_q_heads]; all device pointers, contiguous, member i's block at index i in the order given
+ * to kvf_batch_create.  n_tokens and pos0 are common to the members.  All members must hold the
+ * same number of rows (KVF_ERR_INVALID_ARG otherwise); each one's length advances by n_tokens.
+ * Per member the result is what kvf_fold_step gives: the same cache bits, the output within
+ * rounding of it (the key range may be cut differently, which reorders the sums).  Asynchronous
+ * on cuda_stream; errors and their effect as for kvf_fold_step.
+ */
+kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, const void *v_new,
+                               int32_t n_tokens, int64_t pos0, void *out, float *lse_or_null,
+                               void *cuda_stream);
+
+/* kvf_cache_plan for a batch step; plan[2] counts the CTAs of all members. */
+kvf_status kvf_batch_plan(const kvf_batch *b, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]);
+
+/* The batch's own device status word, encoded as kvf_cache_status_word (0 = no wait gave up). */
+int32_t kvf_batch_status_word(kvf_batch *b);
+
+/* Kernels launched through this batch since creation. */
+uint64_t kvf_batch_launch_count(const kvf_batch *b);
+
+/* Frees the host handle; the members and all device memory stay with the caller. */
+void kvf_batch_destroy(kvf_batch *b);
+
+/*
  * The fold step for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this entry point exists for the sake of such callers only.)
  *

@@ -26,6 +26,8 @@ EXPORTS = [
     "kvf_cache_launch_count", "kvf_cache_profile", "kvf_cache_profile_read", "kvf_cache_destroy",
     "kvf_status_str", "kvf_last_cuda_error", "kvf_fold_step_static", "kvf_cache_status_word",
     "kvf_paged_pool_bytes", "kvf_paged_cache_create",
+    "kvf_batch_workspace_bytes", "kvf_batch_create", "kvf_batch_fold_step", "kvf_batch_plan",
+    "kvf_batch_status_word", "kvf_batch_launch_count", "kvf_batch_destroy",
 ]
 
 
@@ -102,6 +104,20 @@ def load() -> ctypes.CDLL:
     lib.kvf_cache_profile_read.restype = ctypes.c_int
     lib.kvf_cache_destroy.argtypes = [vp]
     lib.kvf_cache_destroy.restype = None
+    lib.kvf_batch_workspace_bytes.argtypes = [cfgp, i32]
+    lib.kvf_batch_workspace_bytes.restype = ctypes.c_size_t
+    lib.kvf_batch_create.argtypes = [ctypes.POINTER(vp), i32, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
+    lib.kvf_batch_create.restype = ctypes.c_int
+    lib.kvf_batch_fold_step.argtypes = [vp, vp, vp, vp, i32, i64, vp, vp, vp]
+    lib.kvf_batch_fold_step.restype = ctypes.c_int
+    lib.kvf_batch_plan.argtypes = [vp, i32, i64, ctypes.POINTER(i32)]
+    lib.kvf_batch_plan.restype = ctypes.c_int
+    lib.kvf_batch_status_word.argtypes = [vp]
+    lib.kvf_batch_status_word.restype = i32
+    lib.kvf_batch_launch_count.argtypes = [vp]
+    lib.kvf_batch_launch_count.restype = u64
+    lib.kvf_batch_destroy.argtypes = [vp]
+    lib.kvf_batch_destroy.restype = None
     lib.kvf_status_str.argtypes = [ctypes.c_int]
     lib.kvf_status_str.restype = ctypes.c_char_p
     lib.kvf_last_cuda_error.argtypes = []
@@ -296,6 +312,67 @@ class PagedCache(Cache):
         d, hkv = self.cfg.head_dim, self.cfg.n_kv_heads
         pages = self.storage.view(torch.bfloat16).view(-1, 2, hkv, 128, d)
         return pages[:, kv]
+
+
+class Batch:
+    """Paged caches of one pool that advance together (kvf_batch_* calls): one launch of each
+    kernel folds one chunk into every member.  Tensors are [n_caches, n_tokens, heads, head_dim]."""
+
+    def __init__(self, caches, workspace: torch.Tensor | None = None):
+        lib = load()
+        self.caches = list(caches)
+        cfg = self.caches[0].cfg
+        self.cfg = cfg
+        wb = int(lib.kvf_batch_workspace_bytes(ctypes.byref(cfg), len(self.caches)))
+        self.workspace = workspace if workspace is not None else torch.empty(max(wb, 256), dtype=torch.uint8,
+                                                                             device=self.caches[0].device)
+        arr = (ctypes.c_void_p * len(self.caches))(*[c._h.value for c in self.caches])
+        h = ctypes.c_void_p()
+        with torch.cuda.device(self.caches[0].device):
+            rc = lib.kvf_batch_create(arr, len(self.caches), self.workspace.data_ptr(), self.workspace.numel(),
+                                      ctypes.byref(h))
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_batch_create")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            load().kvf_batch_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def fold_step(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, pos0: Optional[int] = None,
+                  out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                  stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        assert q.dim() == 4 and q.shape[0] == len(self.caches)
+        n = q.shape[1]
+        for t in (q, k_new, v_new):
+            assert t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16
+        if out is None:
+            od = torch.float32 if (self.cfg.flags & KVF_OUT_F32) else torch.bfloat16
+            out = torch.empty(q.shape, dtype=od, device=q.device)
+        if pos0 is None:
+            pos0 = len(self.caches[0])
+        rc = load().kvf_batch_fold_step(self._h, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), n, int(pos0),
+                                        out.data_ptr(), lse.data_ptr() if lse is not None else None,
+                                        _stream_ptr(stream))
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_batch_fold_step")
+        return out
+
+    def plan(self, n_tokens: int, prefix_len: Optional[int] = None) -> Tuple[int, int, int, int]:
+        arr = (ctypes.c_int32 * 4)()
+        rc = load().kvf_batch_plan(self._h, n_tokens, len(self.caches[0]) if prefix_len is None else prefix_len, arr)
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_batch_plan")
+        return tuple(arr)
+
+    def status_word(self) -> int:
+        return int(load().kvf_batch_status_word(self._h))
+
+    def launch_count(self) -> int:
+        return int(load().kvf_batch_launch_count(self._h))
 
 
 def paged_pool_bytes(cfg: kvf_config, n_pages: int) -> int:

@@ -268,6 +268,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qpair = blockIdx.x, group = blockIdx.y;
+    const int cb = blockIdx.z;     // cache of a batch (0 when there is one cache)
     const int G = a.G, n = a.n;
     const int64_t P = a.prefix, L = P + n;
     // streams == 2 (chunks of at most 128 / G tokens, i.e. one row tile): the two tile slots work on
@@ -336,6 +337,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             int tg = 0, pc = 0;          // ring loads and pieces so far
             int rc[2] = {0, 0};          // loads so far into each stream's ring
             int page = 0;                // paged cache: page of the key tile being loaded
+            const int32_t *page_table = a.page_tables ? a.page_tables[cb] : a.page_table;
+            const int qtok0 = cb * n;    // the caches' rotated chunks follow one another
             bool ok = true;
             int kt0, ntiles;
             for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
@@ -346,7 +349,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 for (int i = 0; i < (streams == 2 ? 1 : 2); ++i)
                     for (int p = 0; p < 2; ++p)
                         tma_load_3d(base + kOffQ + i * kTileBytes + p * kPanel, &map_q, bar(B_QFULL), p * 64, kvh * G,
-                                    (row0 + i * kRows) / G);
+                                    qtok0 + (row0 + i * kRows) / G);
                 ++pc;
                 for (int t = 0; t < 2 * ntiles; ++t, ++tg) {
                     int slot = tg % kSlots, use = tg / kSlots;
@@ -361,9 +364,9 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                     const CUtensorMap *m = (t & 1) ? &map_v : &map_k;
                     const int key0 = (kt0 + (t >> 1)) * kRows;
                     mbar_expect_tx(bar(B_FULL0 + slot), kTileBytes);
-                    if (a.page_table) {
+                    if (page_table) {
                         // paged cache: a key tile is one page; the maps are (d, row in page, KV head, page)
-                        if (!(t & 1)) page = a.page_table[kt0 + (t >> 1)];     // K then V of the same tile
+                        if (!(t & 1)) page = page_table[kt0 + (t >> 1)];       // K then V of the same tile
                         tma_load_4d(slot_addr(slot), m, bar(B_FULL0 + slot), 0, 0, kvh, page);
                         tma_load_4d(slot_addr(slot) + kPanel, m, bar(B_FULL0 + slot), 64, 0, kvh, page);
                     } else {
@@ -497,7 +500,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         bool ok = i < tiles;
         int kt0, ntiles;
         for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
-            const int64_t prow = ((int64_t)(group + kvh) * streams + (streams == 2 ? i : 0)) * nG + R;   // my partial row
+            const int64_t prow = cb * a.part_rows + ((int64_t)(group + kvh) * streams + (streams == 2 ? i : 0)) * nG + R;   // my partial row
             // Turns on the exponentials: in every piece both tile slots take the same number of
             // turns, slot 0 then slot 1, alternating strictly (a slot with fewer key tiles, which
             // happens with two streams, passes its spare turns without doing anything).  Strict
@@ -634,7 +637,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
             const float lse2 = l > 0.f ? m_ref * sl2 + log2f(l) : -INFINITY;
-            const int64_t row = (int64_t)tok * a.H + kvh * G + gi;
+            const int64_t row = ((int64_t)cb * n + tok) * a.H + kvh * G + gi;
 #pragma unroll
             for (int c0 = 0; c0 < 128; c0 += 32) {
                 uint32_t o[32];
@@ -692,6 +695,7 @@ constexpr int kCombineTokens = 2;
 __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
     __shared__ int g_range[2];
     const int kvh = blockIdx.y, G = a.G;
+    const int cb = blockIdx.z;     // cache of a batch
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
@@ -714,15 +718,17 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
     // part s of the KV head sits in slot (g0 + s / st + kvh) * st + s % st
     auto slot_of = [&](int s) { return (int64_t)(g0 + s / st + kvh) * st + s % st; };
     const int64_t nG = (int64_t)a.n * G;
+    const float *part_o = a.part_o + cb * a.part_rows * kD;
+    const float *part_lse = a.part_lse + cb * a.part_rows;
     const int rows = kCombineTokens * G;                      // rows of this block, row = token * G + head-in-group
     for (int rr = warp; rr < rows; rr += 8) {
         const int tok = blockIdx.x * kCombineTokens + rr / G, gi = rr % G;
         if (tok >= a.n) break;
         const int64_t R = (int64_t)tok * G + gi;
-        const int64_t row = (int64_t)tok * a.H + kvh * G + gi;
+        const int64_t row = ((int64_t)cb * a.n + tok) * a.H + kvh * G + gi;
         float M = -INFINITY;
         for (int s0 = 0; s0 < np; s0 += 32) {
-            const float ls = s0 + lane < np ? a.part_lse[slot_of(s0 + lane) * nG + R] : -INFINITY;
+            const float ls = s0 + lane < np ? part_lse[slot_of(s0 + lane) * nG + R] : -INFINITY;
             M = fmaxf(M, ls);
         }
 #pragma unroll
@@ -735,8 +741,8 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
 #pragma unroll
             for (int s = 0; s < 8; ++s)
                 if (s < cnt)
-                    pv[s] = *reinterpret_cast<const float4 *>(a.part_o + (slot_of(s0 + s) * nG + R) * kD + lane * 4);
-            const float ls = lane < cnt ? a.part_lse[slot_of(s0 + lane) * nG + R] : -INFINITY;
+                    pv[s] = *reinterpret_cast<const float4 *>(part_o + (slot_of(s0 + s) * nG + R) * kD + lane * 4);
+            const float ls = lane < cnt ? part_lse[slot_of(s0 + lane) * nG + R] : -INFINITY;
             const float wl = ls == -INFINITY ? 0.f : exp2f(ls - M);
 #pragma unroll
             for (int s = 0; s < 8; ++s) {                     // group order: deterministic
@@ -777,12 +783,12 @@ cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, 1);
+    dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, a.batch);
     return launch_pdl(attn_tc_kernel, grid, dim3(kThreads), kSmemBytes, s, a, maps.q, maps.k, maps.v);
 }
 
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s) {
-    dim3 grid((a.n + kCombineTokens - 1) / kCombineTokens, a.Hkv, 1);
+    dim3 grid((a.n + kCombineTokens - 1) / kCombineTokens, a.Hkv, a.batch);
     return launch_pdl(combine_groups_kernel, grid, dim3(256), 0, s, a);
 }
 

@@ -102,7 +102,40 @@ struct kvf_cache {
     std::vector<cudaEvent_t> pool;
 };
 
+// Caches that advance together: one launch of each kernel folds one chunk into every member.
+struct kvf_batch {
+    std::vector<kvf_cache *> caches;
+    char *workspace;
+    size_t off_status, off_tables, off_q_rot, off_part_o, off_part_lse;
+    int64_t part_rows;       // rows of the partial area per cache
+    CUtensorMap map_q;       // rotated chunks of all members: [n_caches * max_chunk][H][d]
+    uint64_t launches;
+};
+
 namespace {
+
+struct BatchLayout {
+    size_t status, tables, q_rot, part_o, part_lse, total;
+    int64_t part_rows;
+};
+
+BatchLayout batch_layout(const kvf_config *c, int n_caches) {
+    BatchLayout l;
+    // per cache: what two streams of a one-tile chunk can leave (2 * (2 Hkv - 1) slots of 128 rows),
+    // or its share of one cache's partial area if that is more
+    int64_t rows = (int64_t)2 * (2 * c->n_kv_heads - 1) * kKvTile;
+    const int64_t share = ((int64_t)kPartTokens * c->n_q_heads + n_caches - 1) / n_caches;
+    if (share > rows) rows = share;
+    l.part_rows = rows;
+    size_t off = 0;
+    l.status = off;   off = align_up(off + 256, 1024);
+    l.tables = off;   off = align_up(off + (size_t)n_caches * sizeof(void *), 1024);
+    l.q_rot = off;    off = align_up(off + (size_t)n_caches * c->max_chunk * c->n_q_heads * c->head_dim * elem_bytes(c->dtype), 1024);
+    l.part_o = off;   off = align_up(off + (size_t)n_caches * rows * c->head_dim * 4, 1024);
+    l.part_lse = off; off = align_up(off + (size_t)n_caches * rows * 4, 1024);
+    l.total = off;
+    return l;
+}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -145,7 +178,7 @@ kvf_status make_page_map(EncodeTiledFn fn, CUtensorMap *m, void *base, int d, in
     return KVF_OK;
 }
 
-kvf_status build_maps(kvf_cache *c) {
+kvf_status encode_fn(EncodeTiledFn *fn) {
     void *sym = nullptr;
     cudaDriverEntryPointQueryResult qres;
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres);
@@ -154,7 +187,14 @@ kvf_status build_maps(kvf_cache *c) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "driver has no cuTensorMapEncodeTiled");
         return KVF_ERR_CUDA;
     }
-    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(sym);
+    *fn = reinterpret_cast<EncodeTiledFn>(sym);
+    return KVF_OK;
+}
+
+kvf_status build_maps(kvf_cache *c) {
+    EncodeTiledFn fn = nullptr;
+    kvf_status es = encode_fn(&fn);
+    if (es != KVF_OK) return es;
     const kvf_config &f = c->cfg;
     const int d = f.head_dim;
     const uint64_t row = (uint64_t)d * 2;
@@ -185,7 +225,10 @@ struct Plan {
     int ctas, kernels;
 };
 
-Plan make_plan(const kvf_cache *c, int n, int64_t prefix) {
+// `batch` caches share the launch (their CTAs fill the SMs together) and `part_rows_cap` is the
+// partial area of ONE cache.
+Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t part_rows_cap = -1) {
+    if (part_rows_cap < 0) part_rows_cap = c->part_rows_cap;
     Plan p;
     p.tc = c->tc;
     p.ngroups = 0;
@@ -200,25 +243,25 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix) {
         int64_t groups = Hkv;
         if (c->force_splits > 0) {
             groups = (int64_t)Hkv * c->force_splits;
-        } else if (pairs * Hkv < c->sm_count) {
-            groups = c->sm_count / pairs;
+        } else if ((int64_t)pairs * Hkv * batch < c->sm_count) {
+            groups = c->sm_count / (pairs * batch);
             if (groups > Hkv * nt / 4) groups = Hkv * nt / 4;
         }
         const int streams = attn_tc_streams(n, c->G);
-        const int64_t slots_cap = c->part_rows_cap / ((int64_t)n * c->G) / streams;   // slots = streams * (groups + Hkv - 1)
+        const int64_t slots_cap = part_rows_cap / ((int64_t)n * c->G) / streams;   // slots = streams * (groups + Hkv - 1)
         if (groups + Hkv - 1 > slots_cap) groups = slots_cap - (Hkv - 1);
         if (groups > Hkv * nt) groups = Hkv * nt;
         if (groups < Hkv) groups = Hkv;
         p.ngroups = (int)groups;
         p.splits = (int)((groups + Hkv - 1) / Hkv);
-        p.ctas = pairs * p.ngroups;
+        p.ctas = pairs * p.ngroups * batch;
         p.kernels = 2 + ((p.ngroups != Hkv || streams == 2) ? 1 : 0);   // short chunks always leave two parts
         return p;
     }
     const int64_t nt = (L + 63) / 64;
     const int units = attn_simt_ctas(n, c->G, Hkv, 1);
     const int target = c->sm_count * 2;
-    int64_t max_splits = c->part_rows_cap / ((int64_t)n * c->cfg.n_q_heads);
+    int64_t max_splits = part_rows_cap / ((int64_t)n * c->cfg.n_q_heads);
     if (max_splits > kMaxSplits) max_splits = kMaxSplits;
     if (max_splits < 1) max_splits = 1;
     int splits = 1;
@@ -301,6 +344,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     }
     ra.page_table = c->page_table;
     ra.page_elems = c->page_elems;
+    ra.page_tables = nullptr;
     ra.table = c->table;
 
     AttnArgs aa;
@@ -311,6 +355,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.part_lse = reinterpret_cast<float *>(c->workspace + c->lay.part_lse);
     aa.status = reinterpret_cast<int *>(c->workspace + c->lay.status);
     aa.page_table = c->page_table;
+    aa.page_tables = nullptr; aa.part_rows = 0; aa.batch = 1;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
     aa.splits = plan.tc ? 1 : plan.splits;
@@ -322,7 +367,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     cudaError_t e;
     {
         ProfScope ps(c, st, 0);
-        e = launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, st);
+        e = launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, 1, st);
     }
     if (e != cudaSuccess) return cuda_fail(e, "rope_append launch");
     c->launches++;
@@ -592,6 +637,151 @@ void kvf_cache_destroy(kvf_cache *c) {
     for (cudaEvent_t e : c->pool) cudaEventDestroy(e);
     delete c;
 }
+
+size_t kvf_batch_workspace_bytes(const kvf_config *cfg, int32_t n_caches) {
+    if (check_config(cfg) != KVF_OK || n_caches < 1 || n_caches > 65535) return 0;
+    return batch_layout(cfg, n_caches).total;
+}
+
+kvf_status kvf_batch_create(kvf_cache *const *caches, int32_t n_caches, void *dev_workspace, size_t workspace_bytes,
+                            kvf_batch **out) {
+    if (!out) return KVF_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!caches || n_caches < 1 || n_caches > 65535 || !dev_workspace) return KVF_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(dev_workspace) & 255u) return KVF_ERR_INVALID_ARG;
+    for (int i = 0; i < n_caches; ++i)
+        if (!caches[i]) return KVF_ERR_INVALID_ARG;
+    const kvf_cache *c0 = caches[0];
+    // members: paged caches of one pool, same shape (they then share the pool's tensor maps)
+    for (int i = 0; i < n_caches; ++i) {
+        const kvf_cache *c = caches[i];
+        if (!c->page_table || !c->tc) return KVF_ERR_UNSUPPORTED;
+        const kvf_config &x = c->cfg, &y = c0->cfg;
+        if (c->storage != c0->storage || c->n_pool_pages != c0->n_pool_pages || c->device != c0->device ||
+            x.n_q_heads != y.n_q_heads || x.n_kv_heads != y.n_kv_heads || x.head_dim != y.head_dim ||
+            x.dtype != y.dtype || x.capacity != y.capacity || x.max_chunk != y.max_chunk || x.flags != y.flags ||
+            c->scale_log2 != c0->scale_log2 ||
+            std::memcmp(c->table.inv_freq, c0->table.inv_freq, sizeof(c0->table.inv_freq)) != 0)
+            return KVF_ERR_INVALID_ARG;
+        for (int j = 0; j < i; ++j)
+            if (caches[j] == c) return KVF_ERR_INVALID_ARG;
+    }
+    const BatchLayout lay = batch_layout(&c0->cfg, n_caches);
+    if (workspace_bytes < lay.total) return KVF_ERR_CAPACITY;
+
+    kvf_batch *b = new (std::nothrow) kvf_batch();
+    if (!b) return KVF_ERR_INVALID_ARG;
+    b->caches.assign(caches, caches + n_caches);
+    b->workspace = static_cast<char *>(dev_workspace);
+    b->off_status = lay.status; b->off_tables = lay.tables; b->off_q_rot = lay.q_rot;
+    b->off_part_o = lay.part_o; b->off_part_lse = lay.part_lse;
+    b->part_rows = lay.part_rows;
+    b->launches = 0;
+
+    EncodeTiledFn fn = nullptr;
+    kvf_status s = encode_fn(&fn);
+    if (s != KVF_OK) { delete b; return s; }
+    const kvf_config &f = c0->cfg;
+    const uint64_t row = (uint64_t)f.head_dim * 2;
+    s = make_map(fn, &b->map_q, b->workspace + lay.q_rot, (uint64_t)f.n_q_heads, (uint64_t)n_caches * f.max_chunk, row,
+                 row * f.n_q_heads, f.head_dim, (uint32_t)c0->G, (uint32_t)(128 / c0->G));
+    if (s != KVF_OK) { delete b; return s; }
+
+    std::vector<const int32_t *> tables(n_caches);
+    for (int i = 0; i < n_caches; ++i) tables[i] = caches[i]->page_table;
+    cudaError_t e = cudaMemcpy(b->workspace + lay.tables, tables.data(), (size_t)n_caches * sizeof(void *),
+                               cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemset(b->workspace + lay.status, 0, 256);
+    if (e != cudaSuccess) { delete b; return cuda_fail(e, "batch workspace setup"); }
+    *out = b;
+    return KVF_OK;
+}
+
+kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, const void *v_new, int32_t n,
+                               int64_t pos0, void *out, float *lse, void *cuda_stream) {
+    if (!b) return KVF_ERR_INVALID_ARG;
+    kvf_cache *c0 = b->caches[0];
+    const int64_t P = c0->len;
+    for (kvf_cache *c : b->caches)
+        if (c->len != P) return KVF_ERR_INVALID_ARG;          // the members advance together
+    kvf_status s = check_step(c0, n, pos0);
+    if (s != KVF_OK) return s;
+    if (check_ptr(q) || check_ptr(k_new) || check_ptr(v_new) || check_ptr(out)) return KVF_ERR_INVALID_ARG;
+    if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return KVF_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const kvf_config &f = c0->cfg;
+    const int B = (int)b->caches.size();
+    const Plan plan = make_plan(c0, n, P, B, b->part_rows);
+    const int32_t *const *tables = reinterpret_cast<const int32_t *const *>(b->workspace + b->off_tables);
+
+    RopeAppendArgs ra;
+    ra.q = q; ra.k_new = k_new; ra.v_new = v_new;
+    ra.q_rot = b->workspace + b->off_q_rot;
+    ra.k_plane = c0->storage;
+    ra.v_plane = c0->storage + c0->plane_bytes;
+    ra.capacity = f.capacity; ra.prefix = P; ra.pos0 = pos0;
+    ra.n = n; ra.H = f.n_q_heads; ra.Hkv = f.n_kv_heads; ra.d = f.head_dim;
+    ra.zero_rows = (int32_t)((P + n + kKvTile - 1) / kKvTile * kKvTile - (P + n));
+    ra.page_table = c0->page_table;
+    ra.page_elems = c0->page_elems;
+    ra.page_tables = tables;
+    ra.table = c0->table;
+
+    AttnArgs aa;
+    aa.q_rot = ra.q_rot;
+    aa.k_plane = ra.k_plane; aa.v_plane = ra.v_plane;
+    aa.out = out; aa.lse = lse;
+    aa.part_o = reinterpret_cast<float *>(b->workspace + b->off_part_o);
+    aa.part_lse = reinterpret_cast<float *>(b->workspace + b->off_part_lse);
+    aa.status = reinterpret_cast<int *>(b->workspace + b->off_status);
+    aa.page_table = c0->page_table;
+    aa.page_tables = tables; aa.part_rows = b->part_rows; aa.batch = B;
+    aa.capacity = f.capacity; aa.prefix = P;
+    aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c0->G; aa.d = f.head_dim;
+    aa.splits = 1;
+    aa.ngroups = plan.ngroups;
+    aa.streams = attn_tc_streams(n, c0->G);
+    aa.out_f32 = (f.flags & KVF_OUT_F32) ? 1 : 0;
+    aa.scale_log2 = c0->scale_log2;
+
+    cudaError_t e = launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, B, st);
+    if (e != cudaSuccess) return cuda_fail(e, "rope_append launch (batch)");
+    b->launches++;
+    TcMaps maps = c0->maps;
+    maps.q = b->map_q;
+    e = launch_attn_tc(aa, maps, st);
+    if (e != cudaSuccess) return cuda_fail(e, "attention launch (batch)");
+    b->launches++;
+    if (plan.kernels > 2) {
+        e = launch_combine_groups(aa, st);
+        if (e != cudaSuccess) return cuda_fail(e, "combine launch (batch)");
+        b->launches++;
+    }
+    for (kvf_cache *c : b->caches) c->len = P + n;
+    return KVF_OK;
+}
+
+kvf_status kvf_batch_plan(const kvf_batch *b, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]) {
+    if (!b || !plan || n_tokens < 1 || n_tokens > b->caches[0]->cfg.max_chunk || prefix_len < 0) return KVF_ERR_INVALID_ARG;
+    Plan p = make_plan(b->caches[0], n_tokens, prefix_len, (int)b->caches.size(), b->part_rows);
+    plan[0] = 1;
+    plan[1] = p.splits;
+    plan[2] = p.ctas;
+    plan[3] = p.kernels;
+    return KVF_OK;
+}
+
+int32_t kvf_batch_status_word(kvf_batch *b) {
+    if (!b) return -1;
+    int word = 0;
+    cudaError_t e = cudaMemcpy(&word, b->workspace + b->off_status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { cuda_fail(e, "cudaMemcpy(status)"); return -1; }
+    return word;
+}
+
+uint64_t kvf_batch_launch_count(const kvf_batch *b) { return b ? b->launches : 0; }
+
+void kvf_batch_destroy(kvf_batch *b) { delete b; }
 
 const char *kvf_status_str(kvf_status s) {
     switch (s) {

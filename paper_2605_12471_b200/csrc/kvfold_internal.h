@@ -69,6 +69,9 @@ struct RopeAppendArgs {
     int32_t zero_rows;               // value rows [prefix+n, prefix+n+zero_rows) are cleared
     const int32_t *page_table;       // paged cache: device table of page numbers, else null
     int64_t page_elems;              // paged cache: elements per page
+    // batch of caches advancing together (blockIdx.y = cache b): q, k_new, v_new, q_rot hold the
+    // caches' chunks one after the other; cache b's rows go where page_tables[b] says
+    const int32_t *const *page_tables;   // device array of device tables, or null (one cache)
     RopeTable table;
 };
 
@@ -83,6 +86,12 @@ struct AttnArgs {
     float *part_lse;                 // log2 denominators of the parts, same order; -inf = no key seen
     int *status;                     // device status word
     const int32_t *page_table;       // paged cache: device table of page numbers (one per key tile), else null
+    // batch of caches advancing together (blockIdx.z = cache b): q_rot, out, lse hold the caches'
+    // chunks one after the other, cache b's partial results start part_rows rows into the partial
+    // area per cache before it, its pages are named by page_tables[b]
+    const int32_t *const *page_tables;   // device array of device tables, or null (one cache)
+    int64_t part_rows;               // rows of the partial area per cache of a batch
+    int32_t batch;                   // caches in the launch (1 = one cache)
     int64_t capacity, prefix;
     int32_t n, H, Hkv, G, d;
     int32_t splits;                  // CUDA-core path: equal splits of the key range
@@ -92,7 +101,7 @@ struct AttnArgs {
     float scale_log2;                // softmax scale * log2(e)
 };
 
-cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interleaved, cudaStream_t s);
+cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interleaved, int batch, cudaStream_t s);
 cudaError_t launch_attn_simt(const AttnArgs &a, int dtype, cudaStream_t s, int *grid_out);
 cudaError_t launch_combine(const AttnArgs &a, int dtype, cudaStream_t s);
 int attn_simt_ctas(int n, int G, int Hkv, int splits);

@@ -65,7 +65,8 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
 
     const int d = a.d, half = d / 2;
     const int n_tok_blocks = (a.n + kTok - 1) / kTok;
-    const RowMap rows{a.page_table, a.capacity, a.page_elems, a.d};
+    const int b = blockIdx.y;      // cache of a batch (0 when there is one cache)
+    const RowMap rows{a.page_tables ? a.page_tables[b] : a.page_table, a.capacity, a.page_elems, a.d};
 
     pdl_launch_dependents();
     if ((int)blockIdx.x >= n_tok_blocks) {
@@ -101,10 +102,11 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
     __syncthreads();
     pdl_wait();   // the table above needs nothing from earlier kernels; the writes below do
 
-    const T *q = reinterpret_cast<const T *>(a.q);
-    const T *k = reinterpret_cast<const T *>(a.k_new);
-    const T *v = reinterpret_cast<const T *>(a.v_new);
-    T *qr = reinterpret_cast<T *>(a.q_rot);
+    const int64_t qoff = (int64_t)b * a.n * a.H * d, koff = (int64_t)b * a.n * a.Hkv * d;
+    const T *q = reinterpret_cast<const T *>(a.q) + qoff;
+    const T *k = reinterpret_cast<const T *>(a.k_new) + koff;
+    const T *v = reinterpret_cast<const T *>(a.v_new) + koff;
+    T *qr = reinterpret_cast<T *>(a.q_rot) + qoff;
     T *kp = reinterpret_cast<T *>(a.k_plane);
     T *vp = reinterpret_cast<T *>(a.v_plane);
     const int heads = a.H + a.Hkv;
@@ -181,18 +183,18 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
 
 }  // namespace
 
-cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interleaved, cudaStream_t s) {
+cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interleaved, int batch, cudaStream_t s) {
     int blocks = (a.n + kTok - 1) / kTok;
     if (a.zero_rows > 0) {
         int64_t vecs = (int64_t)a.zero_rows * a.Hkv * (a.d / (dtype == 0 ? 8 : 4));
         blocks += (int)((vecs + kThreads - 1) / kThreads);
     }
     if (dtype == 0) {
-        if (interleaved) return launch_pdl(rope_append_kernel<__nv_bfloat16, true>, dim3(blocks), dim3(kThreads), 0, s, a);
-        else return launch_pdl(rope_append_kernel<__nv_bfloat16, false>, dim3(blocks), dim3(kThreads), 0, s, a);
+        if (interleaved) return launch_pdl(rope_append_kernel<__nv_bfloat16, true>, dim3(blocks, batch), dim3(kThreads), 0, s, a);
+        else return launch_pdl(rope_append_kernel<__nv_bfloat16, false>, dim3(blocks, batch), dim3(kThreads), 0, s, a);
     } else {
-        if (interleaved) return launch_pdl(rope_append_kernel<float, true>, dim3(blocks), dim3(kThreads), 0, s, a);
-        else return launch_pdl(rope_append_kernel<float, false>, dim3(blocks), dim3(kThreads), 0, s, a);
+        if (interleaved) return launch_pdl(rope_append_kernel<float, true>, dim3(blocks, batch), dim3(kThreads), 0, s, a);
+        else return launch_pdl(rope_append_kernel<float, false>, dim3(blocks, batch), dim3(kThreads), 0, s, a);
     }
     return cudaGetLastError();
 }

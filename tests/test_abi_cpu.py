@@ -118,6 +118,29 @@ def test_paged_entry_points_validate_before_any_cuda_call(binding):
     assert lib.kvf_paged_cache_create(ctypes.byref(cfg), 256, 1 << 30, 8, 258, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
 
 
+def test_batch_entry_points_validate_before_any_cuda_call(binding):
+    lib = binding.load()
+    cfg = binding.make_config(32, 8, 128, "bf16", 4096, 256, rope_base=5e5)
+    one = lib.kvf_batch_workspace_bytes(ctypes.byref(cfg), 1)
+    many = lib.kvf_batch_workspace_bytes(ctypes.byref(cfg), 128)
+    # rotated chunks of all members, and at least two streams' worth of partial rows per member
+    assert one > 256 * 32 * 128 * 2 and many > 128 * 256 * 32 * 128 * 2
+    assert many >= 128 * (256 * 32 * 128 * 2 + 2 * 15 * 128 * (128 * 4 + 4))
+    assert lib.kvf_batch_workspace_bytes(ctypes.byref(cfg), 0) == 0
+    assert lib.kvf_batch_workspace_bytes(ctypes.byref(cfg), 70000) == 0
+    h = ctypes.c_void_p()
+    assert lib.kvf_batch_create(None, 1, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
+    arr = (ctypes.c_void_p * 2)(None, None)
+    assert lib.kvf_batch_create(arr, 2, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_batch_create(arr, 0, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
+    assert h.value is None
+    assert lib.kvf_batch_fold_step(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_batch_plan(None, 1, 0, (ctypes.c_int32 * 4)()) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_batch_status_word(None) == -1
+    assert lib.kvf_batch_launch_count(None) == 0
+    lib.kvf_batch_destroy(None)
+
+
 def test_binding_fails_loudly_without_the_library(binding, monkeypatch, tmp_path):
     import importlib
     monkeypatch.setattr(binding, "_lib", None)

@@ -1,0 +1,141 @@
+"""One launch over many caches (kvf_batch_*): per member the same cache bits as its own
+kvf_fold_step, outputs within tolerance of the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_12471_b200 import binding, workloads
+from tests.chain import TOL, to_f64
+
+pytestmark = pytest.mark.gpu
+
+W = workloads.Workload("batch_llama_bf16", 32, 8, 128, "bf16", 256, 1024, 500000.0)
+
+
+def make_members(n_caches, capacity, max_chunk, seed, spare_pages=3, fill=0x7FC0):
+    """n_caches paged caches over one pool, their pages dealt from one shuffled deck."""
+    cfg = binding.make_config(W.n_q_heads, W.n_kv_heads, W.head_dim, "bf16", capacity, max_chunk, rope_base=W.rope_base)
+    per = (capacity + 127) // 128
+    n_pool = n_caches * per + spare_pages
+    deck = torch.randperm(n_pool, generator=torch.Generator().manual_seed(seed))[:n_caches * per].to(torch.int32)
+    tables = deck.view(n_caches, per).cuda()
+    pool = torch.empty(binding.paged_pool_bytes(cfg, n_pool), dtype=torch.uint8, device="cuda")
+    pool.view(torch.int16).fill_(fill)                      # NaN wherever no row was ever written
+    ws = torch.empty(binding.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    caches = [binding.PagedCache(cfg, pool, n_pool, tables[i], workspace=ws) for i in range(n_caches)]
+    return cfg, pool, tables, caches
+
+
+def batch_inputs(n_caches, n, seed, step):
+    qs, ks, vs = zip(*[workloads.chunk_inputs(W, seed, step, sequence=i, device="cuda", n_tokens=n) for i in range(n_caches)])
+    return torch.stack(qs).contiguous(), torch.stack(ks).contiguous(), torch.stack(vs).contiguous()
+
+
+def test_batch_gives_each_member_its_own_fold_step():
+    """Three caches, chunks of mixed length (two row tiles, one tile, decode-shaped, ragged): the pool
+    ends up bit-identical to folding each cache by itself, outputs agree with the oracle."""
+    chunks = [256, 100, 16, 1, 300, 128, 7]
+    total = sum(chunks)
+    B = 3
+    cfg, pool, tables, caches = make_members(B, total, max(chunks), seed=11)
+    _, pool1, _, singles = make_members(B, total, max(chunks), seed=11)
+    batch = binding.Batch(caches)
+    ocs = [oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base) for _ in range(B)]
+    worst, worst_lse, worst_pair = 0.0, 0.0, 0.0
+    for t, n in enumerate(chunks):
+        q, k, v = batch_inputs(B, n, 31, t)
+        lse = torch.empty((B, n, W.n_q_heads), dtype=torch.float32, device="cuda")
+        out = batch.fold_step(q, k, v, lse=lse)
+        assert out.shape == q.shape
+        rows = sorted({0, n // 2, n - 1})
+        for i in range(B):
+            alone = singles[i].fold_step(q[i], k[i], v[i])
+            worst_pair = max(worst_pair, float((out[i].float() - alone.float()).abs().max()))
+            ref, ref_lse, _ = ocs[i].fold_step(to_f64(q[i]), to_f64(k[i]), to_f64(v[i]), rows=rows, want_stats=True)
+            worst = max(worst, float(np.abs(to_f64(out[i][rows]) - ref).max()))
+            worst_lse = max(worst_lse, float(np.abs(to_f64(lse[i][rows]) - ref_lse).max()))
+        assert all(len(c) == sum(chunks[:t + 1]) for c in caches)
+    torch.cuda.synchronize()
+    assert batch.status_word() == 0
+    assert torch.equal(pool, pool1)                          # every page, every row, same bits
+    assert worst <= TOL["bf16"][0] and worst_lse <= 2e-3, (worst, worst_lse)
+    assert worst_pair <= 2 ** -5                             # two roundings to bf16 of values below 8
+    # 3 kernels per step at most, whatever the number of members
+    assert batch.launch_count() <= 3 * len(chunks)
+
+
+def test_batch_of_two_caches_still_cuts_the_key_range():
+    """Few members on a long prefix: the plan cuts the (KV head, key tile) line into more ranges than
+    KV heads, so every member leaves partial results that the combine kernel merges per member."""
+    B, P, n = 2, 8192, 256
+    cfg, pool, tables, caches = make_members(B, P + 2 * n, 2048, seed=12)
+    batch = binding.Batch(caches)
+    ocs = [oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, P + 2 * n, rope_base=W.rope_base) for _ in range(B)]
+    for t in range(P // 2048):
+        q, k, v = batch_inputs(B, 2048, 41, t)
+        batch.fold_step(q, k, v)
+        for i in range(B):
+            ocs[i].fold_step(to_f64(q[i]), to_f64(k[i]), to_f64(v[i]), rows=[])
+    plan = batch.plan(n)
+    assert plan[3] == 3 and 4 * W.n_kv_heads * B < plan[2] <= 148      # 4 row pairs per member
+    worst = 0.0
+    for t in range(2):
+        q, k, v = batch_inputs(B, n, 42, t)
+        out = batch.fold_step(q, k, v)
+        rows = [0, 1, 127, 128, 255]
+        for i in range(B):
+            ref = ocs[i].fold_step(to_f64(q[i]), to_f64(k[i]), to_f64(v[i]), rows=rows)
+            worst = max(worst, float(np.abs(to_f64(out[i][rows]) - ref).max()))
+    torch.cuda.synchronize()
+    assert batch.status_word() == 0
+    assert worst <= TOL["bf16"][0], worst
+
+
+def test_batch_of_forty_caches_prefill_then_decode_steps():
+    """Forty members (5120 CTAs in the prefill launch), then decode-shaped steps of 1 and 8 tokens:
+    three sampled members against the oracle, all members' lengths in step."""
+    B = 40
+    chunks = [1000, 1, 1, 8, 1]
+    total = sum(chunks)
+    cfg, pool, tables, caches = make_members(B, 1152, 1024, seed=13)
+    batch = binding.Batch(caches)
+    sample = [0, 17, 39]
+    ocs = {i: oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, 1152, rope_base=W.rope_base) for i in sample}
+    worst = 0.0
+    for t, n in enumerate(chunks):
+        q, k, v = batch_inputs(B, n, 51, t)
+        out = batch.fold_step(q, k, v)
+        rows = sorted({0, n // 3, n - 1})
+        for i in sample:
+            ref = ocs[i].fold_step(to_f64(q[i]), to_f64(k[i]), to_f64(v[i]), rows=rows)
+            worst = max(worst, float(np.abs(to_f64(out[i][rows]) - ref).max()))
+    torch.cuda.synchronize()
+    assert batch.status_word() == 0 and all(len(c) == total for c in caches)
+    assert worst <= TOL["bf16"][0], worst
+
+
+def test_batch_rejects_members_it_cannot_fold_together():
+    cfg, pool, tables, caches = make_members(2, 1024, 256, seed=14)
+    flat = binding.Cache(cfg)
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.KvfError) as e:
+        binding.Batch([caches[0], flat])
+    assert e.value.code == binding.KVF_ERR_UNSUPPORTED                  # a member that is not paged
+    with pytest.raises(binding.KvfError) as e:
+        binding.Batch([caches[0], caches[0]])
+    assert e.value.code == binding.KVF_ERR_INVALID_ARG                  # the same cache twice
+    with pytest.raises(binding.KvfError) as e:
+        binding.Batch(caches, workspace=ws)
+    assert e.value.code == binding.KVF_ERR_CAPACITY                     # workspace too small
+    batch = binding.Batch(caches)
+    q, k, v = batch_inputs(2, 16, 61, 0)
+    caches[1].fold_step(q[1], k[1], v[1])                               # one member runs ahead
+    with pytest.raises(binding.KvfError) as e:
+        batch.fold_step(q, k, v)
+    assert e.value.code == binding.KVF_ERR_INVALID_ARG
+    assert len(caches[0]) == 0 and len(caches[1]) == 16                 # nothing was launched
+    caches[0].fold_step(q[0], k[0], v[0])
+    batch.fold_step(q, k, v)                                            # level again
+    torch.cuda.synchronize()
+    assert batch.status_word() == 0 and len(caches[0]) == len(caches[1]) == 32
