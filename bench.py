@@ -206,22 +206,45 @@ def run_full_stack(args):
     cfg = binding.make_config(w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, T, C, rope_base=w.rope_base)
     ws = torch.empty(binding.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")     # one workspace, one stream
     caches, inputs = [], []
-    for sq in range(w.n_sequences):
-        for ly in range(w.n_layers):
-            caches.append(binding.Cache(cfg, workspace=ws))
-            inputs.append(workloads.chunk_inputs(w, args.seed, 0, sequence=sq, layer=ly, device="cuda"))
-    out = torch.empty_like(inputs[0][0])
     lib, stream = binding.load(), torch.cuda.current_stream().cuda_stream
-    ptrs = [(c._h, q.data_ptr(), k.data_ptr(), v.data_ptr()) for c, (q, k, v) in zip(caches, inputs)]
+    keys = [(sq, ly) for sq in range(w.n_sequences) for ly in range(w.n_layers)]
+    for sq, ly in keys:
+        inputs.append(workloads.chunk_inputs(w, args.seed, 0, sequence=sq, layer=ly, device="cuda"))
+    if args.batched:
+        # every cache in 128-token pages of one pool (tables dealt from one shuffled deck); a chunk is ONE
+        # step of the batch: one launch of each kernel for all caches
+        per = (T + 127) // 128
+        n_pool = len(keys) * per
+        deck = torch.randperm(n_pool, generator=torch.Generator().manual_seed(args.seed)).to(torch.int32)
+        tables = deck.view(len(keys), per).cuda()
+        pool = torch.empty(binding.paged_pool_bytes(cfg, n_pool), dtype=torch.uint8, device="cuda")
+        caches = [binding.PagedCache(cfg, pool, n_pool, tables[i], workspace=ws) for i in range(len(keys))]
+        batch = binding.Batch(caches)
+        bq, bk, bv = (torch.stack([x[j] for x in inputs]).contiguous() for j in range(3))
+        inputs = None
+        bout = torch.empty_like(bq)
+        bh = batch._h
 
-    def chain():
-        for c in caches:
-            c.reset()
-        for t in range(N):
-            for h, qp, kp, vp in ptrs:
-                rc = lib.kvf_fold_step(h, qp, kp, vp, C, t * C, out.data_ptr(), None, stream)
+        def chain():
+            for c in caches:
+                c.reset()
+            for t in range(N):
+                rc = lib.kvf_batch_fold_step(bh, bq.data_ptr(), bk.data_ptr(), bv.data_ptr(), C, t * C, bout.data_ptr(), None, stream)
                 if rc:
-                    raise binding.KvfError(rc, "kvf_fold_step")
+                    raise binding.KvfError(rc, "kvf_batch_fold_step")
+    else:
+        caches = [binding.Cache(cfg, workspace=ws) for _ in keys]
+        out = torch.empty_like(inputs[0][0])
+        ptrs = [(c._h, q.data_ptr(), k.data_ptr(), v.data_ptr()) for c, (q, k, v) in zip(caches, inputs)]
+
+        def chain():
+            for c in caches:
+                c.reset()
+            for t in range(N):
+                for h, qp, kp, vp in ptrs:
+                    rc = lib.kvf_fold_step(h, qp, kp, vp, C, t * C, out.data_ptr(), None, stream)
+                    if rc:
+                        raise binding.KvfError(rc, "kvf_fold_step")
 
     sampler = ClockSampler(0)
     chain()                                               # warm-up pass
@@ -235,6 +258,7 @@ def run_full_stack(args):
     clocks = sampler.stop()
     ms = a.elapsed_time(b)
     assert all(len(c) == T for c in caches) and all(c.status() == binding.KVF_OK for c in caches)
+    assert not args.batched or batch.status_word() == 0
     ncache = len(caches)
     flops = ncache * w.flops_chain()
     pk = peaks()
@@ -243,10 +267,13 @@ def run_full_stack(args):
             "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": w.name, "sequences": w.n_sequences, "layers": w.n_layers, "tokens": T, "chunk": C,
                        "caches": ncache, "cache_gib": ncache * binding.cache_storage_bytes(cfg) / 2 ** 30,
-                       "fold_steps": ncache * N, "l2": "inputs larger than L2"},
+                       "fold_steps": ncache * N, "l2": "inputs larger than L2",
+                       "launch": "one batch step per chunk (one launch of each kernel for all caches, paged pool)"
+                                 if args.batched else "one fold step per cache and chunk"},
             "attention_tflops_whole_step": flops / (ms * 1e-3) / 1e12,
             "frac_of_sustained_bf16_peak": flops / (ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"],
-            "gpu_launches": sum(c.launch_count() for c in caches) // 2, "clocks": clocks}
+            "gpu_launches": (batch.launch_count() if args.batched else sum(c.launch_count() for c in caches)) // 2,
+            "clocks": clocks}
     print(json.dumps(line), flush=True)
 
 
@@ -273,6 +300,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--force-simt", action="store_true")
     ap.add_argument("--paged", action="store_true", help="keep the cache in shuffled 128-token pages of a pool")
+    ap.add_argument("--batched", action="store_true",
+                    help="full_stack only: the caches live in one paged pool and every chunk is one batch step")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every fold step of the timed chains from the host instead of replaying the chain "
                          "as one CUDA graph captured from the same kvf_fold_step calls")

@@ -77,12 +77,15 @@ def test_config5_layer_stack_reduced():
     assert worst <= TOL["bf16"][0]
 
 
-def test_config5_full_stack_64_gib_sampled_pairs():
+@pytest.mark.parametrize("batched", [False, True], ids=["per_cache_steps", "one_batch_step_per_chunk"])
+def test_config5_full_stack_64_gib_sampled_pairs(batched):
     """Config 5 at full size: 4 sequences x 32 layers, one 512 MiB bf16 cache each (64 GiB), 131 072
     tokens per sequence in chunks of 1024, every chunk's 128 fold steps issued on one stream with one
-    shared workspace.  Each (sequence, layer) draws one chunk of inputs from its own seed and feeds it
-    at every chunk (the positions and the prefix still change), as the benchmark does; the oracle
-    follows two (sequence, layer) pairs and checks sampled rows at sampled chunks."""
+    shared workspace - or, batched, as one step of a batch over 128 paged caches of one 64 GiB pool.
+    Each (sequence, layer) draws one chunk of inputs from its own seed and feeds it at every chunk
+    (the positions and the prefix still change), as the benchmark does; the oracle follows two
+    (sequence, layer) pairs and checks sampled rows at sampled chunks."""
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 80 * 2 ** 30:
         pytest.skip("needs 80 GiB of free device memory")
@@ -91,20 +94,34 @@ def test_config5_full_stack_64_gib_sampled_pairs():
     cfg = binding.make_config(w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, T, C, rope_base=w.rope_base)
     ws = torch.empty(binding.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
     keys = [(s, l) for s in range(w.n_sequences) for l in range(w.n_layers)]
-    caches = {key: binding.Cache(cfg, workspace=ws) for key in keys}
     inputs = {key: workloads.chunk_inputs(w, 25, 0, sequence=key[0], layer=key[1], device="cuda") for key in keys}
     watched = [(0, 0), (3, 17)]
     oracles = {key: oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, T, rope_base=w.rope_base) for key in watched}
     host_in = {key: tuple(to_f64(x) for x in inputs[key]) for key in watched}
     check_chunks = {0, 1, N // 2, N - 1}
     rows = [0, C // 2 - 1, C - 1]
-    outs = {key: torch.empty_like(inputs[key][0]) for key in watched}
-    scratch = torch.empty_like(inputs[keys[0]][0])
+    if batched:
+        per = T // 128
+        deck = torch.randperm(len(keys) * per, generator=torch.Generator().manual_seed(25)).to(torch.int32)
+        tables = deck.view(len(keys), per).cuda()
+        pool = torch.empty(binding.paged_pool_bytes(cfg, len(keys) * per), dtype=torch.uint8, device="cuda")
+        caches = {key: binding.PagedCache(cfg, pool, len(keys) * per, tables[i], workspace=ws) for i, key in enumerate(keys)}
+        batch = binding.Batch([caches[key] for key in keys])
+        bq, bk, bv = (torch.stack([inputs[key][j] for key in keys]).contiguous() for j in range(3))
+        bout = torch.empty_like(bq)
+        outs = {key: bout[keys.index(key)] for key in watched}
+    else:
+        caches = {key: binding.Cache(cfg, workspace=ws) for key in keys}
+        outs = {key: torch.empty_like(inputs[key][0]) for key in watched}
+        scratch = torch.empty_like(inputs[keys[0]][0])
     worst, err_sq, ref_sq = 0.0, 0.0, 0.0
     for t in range(N):
-        for key in keys:
-            q, k, v = inputs[key]
-            caches[key].fold_step(q, k, v, out=outs[key] if key in outs else scratch)
+        if batched:
+            batch.fold_step(bq, bk, bv, out=bout)
+        else:
+            for key in keys:
+                q, k, v = inputs[key]
+                caches[key].fold_step(q, k, v, out=outs[key] if key in outs else scratch)
         for key in watched:
             q, k, v = host_in[key]
             if t in check_chunks:
@@ -118,6 +135,8 @@ def test_config5_full_stack_64_gib_sampled_pairs():
     torch.cuda.synchronize()
     assert all(len(c) == T for c in caches.values())
     assert all(c.status() == binding.KVF_OK for c in caches.values())
+    if batched:
+        assert batch.status_word() == 0 and batch.launch_count() == 2 * N     # rotate+append and attention, no combine
     assert worst <= TOL["bf16"][0], worst
     assert (err_sq / ref_sq) ** 0.5 <= 2e-2
     print(f"config5 full size: max abs {worst:.2e}, rel rms {(err_sq / ref_sq) ** 0.5:.2e}")
