@@ -50,6 +50,8 @@ def _load():
     lib.okvf_cache_len.restype = ctypes.c_int64
     lib.okvf_cache_reset.argtypes = [ctypes.c_void_p]
     lib.okvf_cache_reset.restype = None
+    lib.okvf_cache_set_window.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64]
+    lib.okvf_cache_set_window.restype = None
     lib.okvf_cache_k.argtypes = [ctypes.c_void_p]
     lib.okvf_cache_k.restype = dp
     lib.okvf_cache_v.argtypes = [ctypes.c_void_p]
@@ -140,6 +142,11 @@ class OracleCache:
 
     def reset(self):
         _load().okvf_cache_reset(self._h)
+
+    def set_window(self, n_sink: int, window: int):
+        """Sink + window variant: earlier chunks' rows are visible only if among the first n_sink
+        or the last `window` before the chunk (window <= 0: all of them)."""
+        _load().okvf_cache_set_window(self._h, int(n_sink), int(window))
 
     def _plane(self, ptr) -> np.ndarray:
         a = np.ctypeslib.as_array(ptr, shape=(self.Hkv, self.capacity, self.d))

@@ -27,6 +27,15 @@
  * exponentiated, summed and normalised, and the weighted sum of value rows is
  * taken.  OpenMP is used only across independent (query row, head) pairs.
  *
+ * Sink + window variant (the paper's comparison with StreamingLLM: a few sink
+ * tokens kept from the start plus a sliding window of recent tokens, eviction
+ * that leaves the kept rows at their original positions, no RoPE re-anchoring).
+ * With okvf_cache_set_window(n_sink, window) the step behaves as if, after every
+ * chunk, all rows had been evicted except the first n_sink and the last
+ * `window`: a chunk that starts at row P sees rows r < n_sink, rows
+ * P - window <= r < P, and its own rows causally.  Nothing is deleted here (the
+ * arrays keep every row); invisible rows get weight exactly zero.
+ *
  * Readings taken where the paper is silent (each is a build-wide reading):
  *   - RoPE pairs element j with element j + d/2 (rotate-half); the
  *     "interleaved" switch pairs (2j, 2j+1) instead;
@@ -49,6 +58,7 @@
 typedef struct okvf_cache {
     int n_q_heads, n_kv_heads, head_dim, interleaved;
     int64_t capacity, len;
+    int64_t n_sink, window; /* window <= 0: every earlier row is visible */
     double scale;
     double *inv_freq; /* [head_dim/2] */
     double *K;        /* [n_kv_heads][capacity][head_dim], rotated keys */
@@ -95,6 +105,11 @@ void okvf_cache_destroy(okvf_cache *c) {
 
 int64_t okvf_cache_len(const okvf_cache *c) { return c->len; }
 void okvf_cache_reset(okvf_cache *c) { c->len = 0; }
+/* Sink + window variant (see the header); window <= 0 switches it off. */
+void okvf_cache_set_window(okvf_cache *c, int64_t n_sink, int64_t window) {
+    c->n_sink = n_sink < 0 ? 0 : n_sink;
+    c->window = window;
+}
 const double *okvf_cache_k(const okvf_cache *c) { return c->K; }
 const double *okvf_cache_v(const okvf_cache *c) { return c->V; }
 
@@ -220,6 +235,12 @@ int okvf_fold_step(okvf_cache *c, const double *q, const double *k_new, const do
             const double *Vg = c->V + (size_t)g * cap * d;
             double m = -INFINITY;
             for (int64_t r = 0; r < visible; ++r) {
+                /* sink + window: an earlier chunk's row survives eviction only as a sink or
+                 * among the last `window` rows before this chunk */
+                if (c->window > 0 && r < P && r >= c->n_sink && r < P - c->window) {
+                    s[r] = -INFINITY;
+                    continue;
+                }
                 double acc = 0.0;
                 for (int e = 0; e < d; ++e) acc += qr[e] * Kg[(size_t)r * d + e];
                 s[r] = acc * c->scale;

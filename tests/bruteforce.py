@@ -54,3 +54,50 @@ def causal_attention(q, k, v, base, scale=None, pos_offset=0, interleaved=False,
         probs[h] = p
         out[:, h, :] = p @ v[:, g, :]
     return out, probs
+
+
+def evicting_fold(q, k, v, chunks, n_sink, window, base, scale=None):
+    """Chunk-by-chunk attention over a cache that is literally evicted after every chunk.
+
+    The cache is a list of (rotated key, value) rows; a chunk attends to the rows the cache holds
+    plus its own rows causally; afterwards the chunk's rows are appended and everything except the
+    first n_sink rows ever appended and the last `window` rows is deleted.  Rows keep the rotation
+    of the position they were appended at (no re-anchoring).  Returns out [T,H,d] and the largest
+    number of rows the cache held after an eviction.
+    """
+    q, k, v = (np.asarray(a, dtype=np.float64) for a in (q, k, v))
+    T, H, d = q.shape
+    Hkv = k.shape[1]
+    G = H // Hkv
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    kept_k = [[] for _ in range(Hkv)]          # per KV head: list of rotated key rows
+    kept_v = [[] for _ in range(Hkv)]
+    kept_idx = []                              # which original rows the cache holds
+    out = np.empty_like(q)
+    held = 0
+    t0 = 0
+    for n in chunks:
+        pos = np.arange(t0, t0 + n)
+        qr = rope_complex(q[t0:t0 + n], pos, base)
+        kr = rope_complex(k[t0:t0 + n], pos, base)
+        for h in range(H):
+            g = h // G
+            for i in range(n):
+                keys = np.array(kept_k[g] + [kr[j, g] for j in range(i + 1)])
+                vals = np.array(kept_v[g] + [v[t0 + j, g] for j in range(i + 1)])
+                s = keys @ qr[i, h] * scale
+                p = np.exp(s - s.max())
+                out[t0 + i, h] = (p / p.sum()) @ vals
+        for g in range(Hkv):
+            kept_k[g] += [kr[j, g] for j in range(n)]
+            kept_v[g] += [v[t0 + j, g] for j in range(n)]
+        kept_idx += list(range(t0, t0 + n))
+        # eviction: the first n_sink rows ever seen stay, and the most recent `window`
+        keep = [x for x, idx in enumerate(kept_idx) if idx < n_sink or idx >= t0 + n - window]
+        for g in range(Hkv):
+            kept_k[g] = [kept_k[g][x] for x in keep]
+            kept_v[g] = [kept_v[g][x] for x in keep]
+        kept_idx = [kept_idx[x] for x in keep]
+        held = max(held, len(kept_idx))
+        t0 += n
+    return out, held

@@ -242,6 +242,50 @@ def test_planted_key_is_recovered_through_a_deep_chain():
 
 
 # -------------------------------------------------------------- append / the cache
+# ------------------------------------------------- sink + window variant
+@pytest.mark.parametrize("n_sink,window,chunks", [
+    (4, 12, [8] * 8), (4, 12, [5, 8, 1, 13, 7, 2, 16, 12]), (0, 9, [6] * 7), (3, 1, [4] * 6), (2, 40, [16] * 4),
+])
+def test_window_mode_equals_a_cache_that_is_literally_evicted_after_every_chunk(n_sink, window, chunks):
+    """Section 6's StreamingLLM baseline: sinks plus a sliding window, eviction that leaves the kept
+    rows at their positions.  The expected values come from a cache whose rows are deleted."""
+    T, H, Hkv, d = sum(chunks), 4, 2, 8
+    q, k, v = _qkv(RNG(31), T, H, Hkv, d)
+    ref, held = bf.evicting_fold(q, k, v, chunks, n_sink, window, 10000.0)
+    assert held <= n_sink + window                       # the cache capacity the paper quotes: 4 + 1020
+    c = oracle.OracleCache(H, Hkv, d, capacity=T)
+    c.set_window(n_sink, window)
+    outs, t0 = [], 0
+    for n in chunks:
+        o, lse, rowsum = c.fold_step(q[t0:t0 + n], k[t0:t0 + n], v[t0:t0 + n], want_stats=True)
+        assert np.abs(rowsum - 1.0).max() <= 1e-14
+        outs.append(o)
+        t0 += n
+    assert np.abs(np.concatenate(outs) - ref).max() <= 1e-12
+
+
+def test_window_that_covers_everything_is_the_plain_fold_and_a_far_key_is_lost_otherwise():
+    T, H, Hkv, d, C = 96, 2, 1, 8, 8
+    q, k, v = _qkv(RNG(32), T, H, Hkv, d)
+    plain, _, _ = _fold(q, k, v, [C] * (T // C), H, Hkv, d)
+    c = oracle.OracleCache(H, Hkv, d, capacity=T)
+    c.set_window(0, T)
+    wide = np.concatenate([c.fold_step(q[t:t + C], k[t:t + C], v[t:t + C]) for t in range(0, T, C)])
+    assert np.array_equal(wide, plain)
+    # a planted key outside sinks and window has no influence at all: changing its value row
+    # changes nothing in the last chunk's output
+    outs = []
+    for bump in (0.0, 100.0):
+        v2 = v.copy()
+        v2[20] += bump                                   # row 20: not a sink, 68 rows before the last chunk
+        c = oracle.OracleCache(H, Hkv, d, capacity=T)
+        c.set_window(4, 16)
+        for t in range(0, T, C):
+            o = c.fold_step(q[t:t + C], k[t:t + C], v2[t:t + C])
+        outs.append(o)
+    assert np.array_equal(outs[0], outs[1])
+
+
 def test_append_only_prefix_rows_are_bit_unchanged():
     T, H, Hkv, d = 30, 2, 2, 8
     q, k, v = _qkv(RNG(18), T, H, Hkv, d)
