@@ -190,6 +190,20 @@ kvf_status kvf_cache_plan(const kvf_cache *c, int32_t n_tokens, int64_t prefix_l
 /* Force the number of splits (0 = automatic).  Values the workspace cannot hold are clamped. */
 kvf_status kvf_cache_set_splits(kvf_cache *c, int32_t splits);
 
+/*
+ * Sink + window variant of the attention mask (Section 6 of the paper, the comparison with
+ * StreamingLLM at 4 sink tokens plus a window of 1020 recent ones; the rows that stay keep the
+ * positions they were appended at, no RoPE re-anchoring).  From the next step on, a chunk that starts at row P sees,
+ * of the rows before it, only rows r < n_sink and rows r >= P - window - what a cache evicted to
+ * "sinks + the last `window` rows" after every chunk would still hold - and its own rows causally.
+ * window = 0 (with n_sink = 0) restores the full prefix.  n_sink <= 64.
+ * Rows are still appended at their place and nothing is deleted: the mask alone changes, and key
+ * tiles without a visible row are never read.  With a paged cache the caller may therefore hand
+ * the pages of such tiles to another use (every page below row P - window except page 0 when
+ * n_sink > 0): their table entries are not looked at again.
+ */
+kvf_status kvf_cache_set_window(kvf_cache *c, int32_t n_sink, int64_t window);
+
 /* Kernels launched through this handle since creation. */
 uint64_t kvf_cache_launch_count(const kvf_cache *c);
 

@@ -27,7 +27,7 @@ EXPORTS = [
     "kvf_status_str", "kvf_last_cuda_error", "kvf_fold_step_static", "kvf_cache_status_word",
     "kvf_paged_pool_bytes", "kvf_paged_cache_create",
     "kvf_batch_workspace_bytes", "kvf_batch_create", "kvf_batch_fold_step", "kvf_batch_plan",
-    "kvf_batch_status_word", "kvf_batch_launch_count", "kvf_batch_destroy",
+    "kvf_batch_status_word", "kvf_batch_launch_count", "kvf_batch_destroy", "kvf_cache_set_window",
 ]
 
 
@@ -96,6 +96,8 @@ def load() -> ctypes.CDLL:
     lib.kvf_cache_plan.restype = ctypes.c_int
     lib.kvf_cache_set_splits.argtypes = [vp, i32]
     lib.kvf_cache_set_splits.restype = ctypes.c_int
+    lib.kvf_cache_set_window.argtypes = [vp, i32, i64]
+    lib.kvf_cache_set_window.restype = ctypes.c_int
     lib.kvf_cache_launch_count.argtypes = [vp]
     lib.kvf_cache_launch_count.restype = u64
     lib.kvf_cache_profile.argtypes = [vp, i32]
@@ -258,6 +260,12 @@ class Cache:
         rc = load().kvf_cache_set_splits(self._h, splits)
         if rc != KVF_OK:
             raise KvfError(rc, "kvf_cache_set_splits")
+
+    def set_window(self, n_sink: int, window: int):
+        """Sink + window mask from the next step on (kvf_cache_set_window); (0, 0) = full prefix."""
+        rc = load().kvf_cache_set_window(self._h, n_sink, window)
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_cache_set_window")
 
     def launch_count(self) -> int:
         return int(load().kvf_cache_launch_count(self._h))

@@ -61,8 +61,10 @@ __global__ void __launch_bounds__(kThreads, 2) attn_simt_kernel(const AttnArgs a
     const int row0 = tile * BM;
     const int tok_last = min(n - 1, (row0 + BM - 1) / G);
     const int64_t need = P + tok_last + 1;
-    const int nt_need = (int)((need + BN - 1) / BN);
-    const int nt_all = (int)((L + BN - 1) / BN);
+    // (virtual key tiles: without a window they are the key tiles themselves)
+    const WindowTiles wt(a.win_lo, a.n_sink, BN);
+    const int nt_need = (int)((need + BN - 1) / BN) - wt.skip;
+    const int nt_all = (int)((L + BN - 1) / BN) - wt.skip;
     const int per = (nt_all + a.splits - 1) / a.splits;
     const int kt_begin = split * per;
     const int kt_end = min(nt_need, kt_begin + per);
@@ -97,7 +99,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_simt_kernel(const AttnArgs a
     }
 
     for (int kt = kt_begin; kt < kt_end; ++kt) {
-        const int64_t key0 = (int64_t)kt * BN;
+        const int64_t key0 = (int64_t)wt.actual(kt) * BN;
         __syncthreads();   // previous iteration is done with Ks / Vs (and Q is in place)
         for (int idx = tid; idx < BN * (D / VEC); idx += kThreads) {
             int r = idx / (D / VEC), c = idx % (D / VEC);
@@ -143,7 +145,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_simt_kernel(const AttnArgs a
             float mx = -INFINITY;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                bool vis = key0 + tx + 16 * j < limit[i];
+                const int64_t key = key0 + tx + 16 * j;
+                bool vis = key < limit[i] && (key >= a.win_lo || key < a.n_sink);
                 s[i][j] = vis ? s[i][j] * a.scale_log2 : -INFINITY;
                 mx = fmaxf(mx, s[i][j]);
             }

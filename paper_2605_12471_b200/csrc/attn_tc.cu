@@ -284,8 +284,10 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     // valid row: its issuer and softmax warps then sit the kernel out
     const int tiles = (streams == 2 || row0 + kRows < n * G) ? 2 : 1;
     const int tok_last = min(n - 1, (row0 + 2 * kRows - 1) / G);
-    const int nt_need = (int)((P + tok_last + 1 + kRows - 1) / kRows);
-    const int nt_all = (int)((L + kRows - 1) / kRows);
+    // (virtual key tiles: without a window they are the key tiles themselves)
+    const WindowTiles wt(a.win_lo, a.n_sink, kRows);
+    const int nt_need = (int)((P + tok_last + 1 + kRows - 1) / kRows) - wt.skip;
+    const int nt_all = (int)((L + kRows - 1) / kRows) - wt.skip;
     const int64_t line = (int64_t)a.Hkv * nt_all;
     const int64_t lin0 = group * line / a.ngroups, lin1 = (group + 1) * line / a.ngroups;
     const int kvh_first = (int)(lin0 / nt_all);
@@ -362,11 +364,12 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                     ok = mbar_wait(bar(B_EMPTY0 + slot), (use & 1) ^ 1, ctl, a.status);
                     if (!ok) break;
                     const CUtensorMap *m = (t & 1) ? &map_v : &map_k;
-                    const int key0 = (kt0 + (t >> 1)) * kRows;
+                    const int ktile = wt.actual(kt0 + (t >> 1));
+                    const int key0 = ktile * kRows;
                     mbar_expect_tx(bar(B_FULL0 + slot), kTileBytes);
                     if (page_table) {
                         // paged cache: a key tile is one page; the maps are (d, row in page, KV head, page)
-                        if (!(t & 1)) page = page_table[kt0 + (t >> 1)];       // K then V of the same tile
+                        if (!(t & 1)) page = page_table[ktile];                // K then V of the same tile
                         tma_load_4d(slot_addr(slot), m, bar(B_FULL0 + slot), 0, 0, kvh, page);
                         tma_load_4d(slot_addr(slot) + kPanel, m, bar(B_FULL0 + slot), 64, 0, kvh, page);
                     } else {
@@ -544,9 +547,12 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                const int64_t key0 = (int64_t)(kt0 + j) * kRows;
+                const int64_t key0 = (int64_t)wt.actual(kt0 + j) * kRows;
                 const int nvis = (int)max((int64_t)0, min((int64_t)kRows, limit - key0));
-                const bool masked = __any_sync(0xffffffffu, nvis < kRows);
+                // window: columns below lo_c lie before the window and count only if they are sinks
+                const int lo_c = (int)max((int64_t)0, min((int64_t)kRows, a.win_lo - key0));
+                const int sink_c = (int)max((int64_t)0, min((int64_t)kRows, a.n_sink - key0));
+                const bool masked = __any_sync(0xffffffffu, nvis < kRows) || lo_c > sink_c;
 
                 // the whole score row in registers after one load
                 uint32_t sc[128];
@@ -557,7 +563,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 tmem_wait_ld();
                 if (masked) {
 #pragma unroll
-                    for (int c = 0; c < 128; ++c) sc[c] = c < nvis ? sc[c] : 0xFF800000u;   // -inf
+                    for (int c = 0; c < 128; ++c) sc[c] = (c < nvis && (c >= lo_c || c < sink_c)) ? sc[c] : 0xFF800000u;   // -inf
                 }
                 float mx[8];
 #pragma unroll
@@ -699,7 +705,7 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
-        const int nt_all = (int)((a.prefix + a.n + kRows - 1) / kRows);
+        const int nt_all = (int)((a.prefix + a.n + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
         const int64_t line = (int64_t)a.Hkv * nt_all;
         auto start = [&](int64_t g) { return g * line / a.ngroups; };
         auto group_of = [&](int64_t lin) {

@@ -98,6 +98,8 @@ struct kvf_cache {
     const int32_t *page_table = nullptr;   // paged cache: device table, one page number per 128 tokens
     int64_t page_elems = 0;                // paged cache: elements per page
     int32_t n_pool_pages = 0;
+    int32_t n_sink = 0;                    // sink + window variant: rows always visible
+    int64_t window = 0;                    // and the rows before the chunk that stay visible (0 = all)
     std::vector<ProfRec> recs;
     std::vector<cudaEvent_t> pool;
 };
@@ -227,6 +229,13 @@ struct Plan {
 
 // `batch` caches share the launch (their CTAs fill the SMs together) and `part_rows_cap` is the
 // partial area of ONE cache.
+// First row of the window for a chunk that starts at row `prefix` (0 = every earlier row is visible).
+int64_t window_lo(const kvf_cache *c, int64_t prefix) {
+    if (c->window <= 0) return 0;
+    const int64_t lo = prefix - c->window;
+    return lo <= c->n_sink ? 0 : lo;       // the window reaches the sinks: nothing is hidden
+}
+
 Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t part_rows_cap = -1) {
     if (part_rows_cap < 0) part_rows_cap = c->part_rows_cap;
     Plan p;
@@ -238,7 +247,7 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
         // one CTA per (row pair, group); the groups cut the Hkv * nt line of (KV head, key tile)
         // into equal ranges.  Whole KV heads if that fills the SMs, else as many groups as give
         // one CTA per SM, with at least 4 key tiles each and within the partial area.
-        const int64_t nt = (L + kKvTile - 1) / kKvTile;
+        const int64_t nt = (L + kKvTile - 1) / kKvTile - WindowTiles(window_lo(c, prefix), c->n_sink, kKvTile).skip;
         const int pairs = attn_tc_row_pairs(n, c->G);
         int64_t groups = Hkv;
         if (c->force_splits > 0) {
@@ -258,7 +267,7 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
         p.kernels = 2 + ((p.ngroups != Hkv || streams == 2) ? 1 : 0);   // short chunks always leave two parts
         return p;
     }
-    const int64_t nt = (L + 63) / 64;
+    const int64_t nt = (L + 63) / 64 - WindowTiles(window_lo(c, prefix), c->n_sink, 64).skip;
     const int units = attn_simt_ctas(n, c->G, Hkv, 1);
     const int target = c->sm_count * 2;
     int64_t max_splits = part_rows_cap / ((int64_t)n * c->cfg.n_q_heads);
@@ -356,6 +365,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.status = reinterpret_cast<int *>(c->workspace + c->lay.status);
     aa.page_table = c->page_table;
     aa.page_tables = nullptr; aa.part_rows = 0; aa.batch = 1;
+    aa.n_sink = c->n_sink; aa.win_lo = window_lo(c, P);
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
     aa.splits = plan.tc ? 1 : plan.splits;
@@ -607,6 +617,15 @@ kvf_status kvf_cache_set_splits(kvf_cache *c, int32_t splits) {
     return KVF_OK;
 }
 
+kvf_status kvf_cache_set_window(kvf_cache *c, int32_t n_sink, int64_t window) {
+    if (!c || n_sink < 0 || window < 0) return KVF_ERR_INVALID_ARG;
+    if (window == 0 && n_sink != 0) return KVF_ERR_INVALID_ARG;   // sinks mean something only beside a window
+    if (n_sink > kMaxSinks) return KVF_ERR_UNSUPPORTED;
+    c->n_sink = n_sink;
+    c->window = window;
+    return KVF_OK;
+}
+
 uint64_t kvf_cache_launch_count(const kvf_cache *c) { return c ? c->launches : 0; }
 
 kvf_status kvf_cache_profile(kvf_cache *c, int32_t enable) {
@@ -703,7 +722,8 @@ kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, c
     kvf_cache *c0 = b->caches[0];
     const int64_t P = c0->len;
     for (kvf_cache *c : b->caches)
-        if (c->len != P) return KVF_ERR_INVALID_ARG;          // the members advance together
+        if (c->len != P || c->n_sink != c0->n_sink || c->window != c0->window)
+            return KVF_ERR_INVALID_ARG;                       // the members advance together, under one mask
     kvf_status s = check_step(c0, n, pos0);
     if (s != KVF_OK) return s;
     if (check_ptr(q) || check_ptr(k_new) || check_ptr(v_new) || check_ptr(out)) return KVF_ERR_INVALID_ARG;
@@ -736,6 +756,7 @@ kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, c
     aa.status = reinterpret_cast<int *>(b->workspace + b->off_status);
     aa.page_table = c0->page_table;
     aa.page_tables = tables; aa.part_rows = b->part_rows; aa.batch = B;
+    aa.n_sink = c0->n_sink; aa.win_lo = window_lo(c0, P);
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c0->G; aa.d = f.head_dim;
     aa.splits = 1;

@@ -92,6 +92,10 @@ struct AttnArgs {
     const int32_t *const *page_tables;   // device array of device tables, or null (one cache)
     int64_t part_rows;               // rows of the partial area per cache of a batch
     int32_t batch;                   // caches in the launch (1 = one cache)
+    // sink + window variant: of the rows before the chunk only those below n_sink or from win_lo on
+    // are visible (win_lo = 0: all of them); see WindowTiles
+    int32_t n_sink;
+    int64_t win_lo;
     int64_t capacity, prefix;
     int32_t n, H, Hkv, G, d;
     int32_t splits;                  // CUDA-core path: equal splits of the key range
@@ -100,6 +104,21 @@ struct AttnArgs {
     int32_t out_f32;
     float scale_log2;                // softmax scale * log2(e)
 };
+
+// Key tiles of the sink + window variant.  Tiles that hold no visible row are never loaded: the
+// kernels walk "virtual" tiles v = 0, 1, ... and read tile actual(v).  With T0 the tile that holds
+// row win_lo, the virtual line is [tile 0, if it holds sinks and T0 > 0] followed by T0, T0 + 1, ...
+struct WindowTiles {
+    int sink_tiles;   // 1 if tile 0 is walked only for its sink rows
+    int skip;         // tiles left out between the sink tile and the window
+    __host__ __device__ WindowTiles(int64_t win_lo, int n_sink, int tile_rows) {
+        const int t0 = (int)(win_lo / tile_rows);
+        sink_tiles = (n_sink > 0 && t0 > 0) ? 1 : 0;
+        skip = t0 - sink_tiles;
+    }
+    __host__ __device__ int actual(int v) const { return v < sink_tiles ? v : v + skip; }
+};
+constexpr int kMaxSinks = 64;         // sink rows sit in the first key tile of either kernel
 
 cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interleaved, int batch, cudaStream_t s);
 cudaError_t launch_attn_simt(const AttnArgs &a, int dtype, cudaStream_t s, int *grid_out);

@@ -59,7 +59,7 @@ def test_batch_gives_each_member_its_own_fold_step():
     torch.cuda.synchronize()
     assert batch.status_word() == 0
     assert torch.equal(pool, pool1)                          # every page, every row, same bits
-    assert worst <= TOL["bf16"][0] and worst_lse <= 2e-3, (worst, worst_lse)
+    assert worst <= TOL["bf16"][0] and worst_lse <= 2e-2, (worst, worst_lse)
     assert worst_pair <= 2 ** -5                             # two roundings to bf16 of values below 8
     # 3 kernels per step at most, whatever the number of members
     assert batch.launch_count() <= 3 * len(chunks)
