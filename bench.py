@@ -300,6 +300,13 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--force-simt", action="store_true")
     ap.add_argument("--paged", action="store_true", help="keep the cache in shuffled 128-token pages of a pool")
+    ap.add_argument("--shard", default="sequences", choices=["sequences", "kv_heads"],
+                    help="with --gpus N: one sequence per rank (weak scaling), or ONE sequence whose KV heads and "
+                         "the query heads that read them are dealt to the ranks (strong scaling, no exchange)")
+    ap.add_argument("--sinks", type=int, default=0)
+    ap.add_argument("--window", type=int, default=0,
+                    help="sink + window mask (the paper's StreamingLLM comparison runs 4 + 1020); 0 = full prefix. "
+                         "FLOP and byte counts in the output line then count the visible keys only")
     ap.add_argument("--batched", action="store_true",
                     help="full_stack only: the caches live in one paged pool and every chunk is one batch step")
     ap.add_argument("--no-graph", action="store_true",
@@ -334,10 +341,15 @@ def main():
     if P0 % 2048 or (T - P0) % C or P0 >= T:
         raise SystemExit("--prefill must be a multiple of 2048 below --tokens, and (tokens - prefill) a multiple of the chunk")
     N = (T - P0) // C                                  # timed fold steps per chain
-    H, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
-    seq = multi.sequence_of_rank(rank)[0]
+    by_heads = args.shard == "kv_heads"
+    seq = 0 if by_heads else multi.sequence_of_rank(rank)[0]
     wt = w.with_(tokens=T - P0)                        # the timed part's inputs
     q, k, v = workloads.sequence_inputs(wt, args.seed, sequence=seq, device="cuda")
+    if by_heads:
+        # every rank draws the whole sequence and keeps its heads; from here on `w` is the rank's shape
+        q, k, v = multi.shard_heads(q, k, v, rank, world)
+        w = w.with_(n_q_heads=q.shape[1], n_kv_heads=k.shape[1])
+    H, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
     out = torch.empty_like(q)
     flags = binding.KVF_FORCE_SIMT if args.force_simt else 0
     if args.paged:
@@ -348,14 +360,22 @@ def main():
         cache = binding.PagedCache(cfg, pool, n_table, table)
     else:
         cache = binding.cache_for(w, flags=flags, max_chunk=max(C, 2048 if P0 else C))
+    if args.window:
+        cache.set_window(args.sinks, args.window)
     h = cache._h
     launch_stream = [torch.cuda.current_stream().cuda_stream]
     eb = q.element_size()
     qs, ks = C * H * d * eb, C * Hkv * d * eb
     qp, kp, vp, op = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr()
     if P0:
-        fq, fk, fv = workloads.chunk_inputs(w.with_(chunk=2048), args.seed + 1, 0, sequence=seq, device="cuda")
+        fq, fk, fv = workloads.chunk_inputs(w.with_(chunk=2048), args.seed + 1, 0, sequence=seq + rank, device="cuda")
         fout = torch.empty_like(fq)
+
+    def visible(prefix):
+        """Rows before a chunk that its queries see (all of them without a window)."""
+        if args.window and prefix - args.window > args.sinks:
+            return args.sinks + args.window
+        return prefix
 
     def prefill():
         """Empty accumulator, then (outside every timed region) the prefix in 2048-token steps."""
@@ -426,7 +446,7 @@ def main():
     assert graph is not None or len(cache) == T
     if cache.status() != binding.KVF_OK:
         raise SystemExit("device status word reports a timed-out wait")
-    value = multi.whole_job_tokens_per_s(T - P0, args.steps, world, ms)
+    value = multi.whole_job_tokens_per_s(T - P0, args.steps, 1 if by_heads else world, ms)
 
     # per-kernel time of the same chain, CUDA events around every launch on the launching stream;
     # read out in bins of steps, which gives the latency against the prefix length
@@ -440,8 +460,8 @@ def main():
         first, last = bi * N // nbins, (bi + 1) * N // nbins
         body(first, last)
         bms, bcnt = cache.profile_read()
-        fl = sum(w.flops_step(P0 + t * C, C) for t in range(first, last))
-        by = sum(P0 + (t + 1) * C for t in range(first, last)) * w.cache_bytes_per_token()
+        fl = sum(w.flops_step(visible(P0 + t * C), C) for t in range(first, last))
+        by = sum(visible(P0 + t * C) + C for t in range(first, last)) * w.cache_bytes_per_token()
         curve.append({"prefix_from": P0 + first * C, "prefix_to": P0 + (last - 1) * C,
                       "step_us": 1e3 * sum(bms) / (last - first), "attention_us": 1e3 * bms[1] / (last - first),
                       "attention_tflops": fl / (bms[1] * 1e-3) / 1e12, "cache_read_gbs": by / (bms[1] * 1e-3) / 1e9})
@@ -450,9 +470,9 @@ def main():
     cache.profile(False)
     launches = (cache.launch_count() - l0) * args.steps       # kernels of the timed chains
     pk = peaks()
-    attn_flops = sum(w.flops_step(P0 + t * C, C) for t in range(N))
+    attn_flops = sum(w.flops_step(visible(P0 + t * C), C) for t in range(N))
     attn_tflops = attn_flops / (kms[1] * 1e-3) / 1e12
-    cache_bytes_read = sum(P0 + (t + 1) * C for t in range(N)) * w.cache_bytes_per_token()
+    cache_bytes_read = sum(visible(P0 + t * C) + C for t in range(N)) * w.cache_bytes_per_token()
     hbm_gbs = cache_bytes_read / (kms[1] * 1e-3) / 1e9
     traffic = None
     if NCU_TRAFFIC_BYTES_PER_CACHE_BYTE is not None:
@@ -497,12 +517,12 @@ def main():
         body_host()
         e2e_steps = max(1, min(args.steps, 3))
         ems = timed(body_host, e2e_steps)
-        e2e = {"value": world * e2e_steps * (T - P0) / (ems * 1e-3), "unit": "tokens/s", "steps": e2e_steps,
+        e2e = {"value": (1 if by_heads else world) * e2e_steps * (T - P0) / (ems * 1e-3), "unit": "tokens/s", "steps": e2e_steps,
                "h2d_bytes_per_step": (T - P0) * (H + 2 * Hkv) * d * eb, "d2h_bytes_per_step": (T - P0) * H * d * eb,
                "ms_per_step": ems / e2e_steps}
 
     cpu = None
-    if rank == 0 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.window:
         rate, times, threads, rows = oracle_rate(w, args.seed, rows_per_step=32, repeats=4, prefix=max(0, T - 5 * C))
         cpu = {"value": tokens_per_s_from_pairs(w, rate, P0), "unit": "tokens/s", "cores": threads, "kind": "oracle",
                "sample": (f"{len(rows)} query rows x {H} heads of one chunk at prefix ~{T - 4 * C}, median of "
@@ -515,11 +535,11 @@ def main():
         line = {
             "metric": "fold-step tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
+            "higher_is_better": True, "scaling": "strong" if by_heads else "weak", "vs_baseline": None, "dtype": w.dtype,
             "data": "synthetic",
-            "config": {"workload": w.name, "tokens": T, "chunk": C, "prefill": P0, "fold_steps_per_step": N,
+            "config": {"workload": w.name, "shard": args.shard, "tokens": T, "chunk": C, "prefill": P0, "fold_steps_per_step": N,
                        "n_q_heads": H, "n_kv_heads": Hkv, "head_dim": d, "rope_base": w.rope_base,
-                       "sequences_per_gpu": 1, "paged": bool(args.paged),
+                       "sequences_per_gpu": 1, "paged": bool(args.paged), "sinks": args.sinks, "window": args.window,
                        "launch": "per-step host launches" if graph is None else "one CUDA graph per chain, captured from the same calls", "l2": "inputs larger than L2 (cache grows to 512 MiB per chain)",
                        "last_step_plan": {"tensor_core": plan[0], "splits": plan[1], "ctas": plan[2]}},
             "attention_tflops": step_flops / (ms * 1e-3) / 1e12,

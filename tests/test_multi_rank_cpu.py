@@ -56,7 +56,48 @@ def test_two_ranks_fold_independent_sequences_and_reduce_time_with_max():
     assert abs(ret["value"] - 2 * 2 * 512 / 0.020) < 1e-6
 
 
+def _shard_worker(rank, world, port, ret):
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    w = workloads.Workload("shard_probe", 8, 4, 16, "f32", 8, 40, 10000.0)
+    qh, kvh = multi.kv_head_shard(rank, world, w.n_q_heads, w.n_kv_heads)
+    oc = oracle.OracleCache(len(qh), len(kvh), w.head_dim, w.tokens, rope_base=w.rope_base)
+    outs = []
+    for t in range(w.n_steps):
+        q, k, v = workloads.chunk_inputs(w, 9, t)                       # every rank draws the same chunk
+        qs, ks, vs = multi.shard_heads(q, k, v, rank, world)
+        outs.append(oc.fold_step(qs.double().numpy(), ks.double().numpy(), vs.double().numpy()))
+    mine = torch.from_numpy(np.concatenate(outs))                       # [T, H / world, d]
+    parts = [torch.empty_like(mine) for _ in range(world)]
+    dist.all_gather(parts, mine)                                        # the test's check, not the data path
+    if rank == 0:
+        ret["out"] = torch.cat(parts, dim=1).numpy()
+        ret["heads"] = [(list(a), list(b)) for a, b in
+                        (multi.kv_head_shard(r, world, w.n_q_heads, w.n_kv_heads) for r in range(world))]
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_split_one_sequence_by_kv_head_without_any_exchange():
+    world = 2
+    ret = mp.Manager().dict()
+    mp.spawn(_shard_worker, args=(world, _free_port(), ret), nprocs=world, join=True)
+    assert ret["heads"] == [([0, 1, 2, 3], [0, 1]), ([4, 5, 6, 7], [2, 3])]
+    w = workloads.Workload("shard_probe", 8, 4, 16, "f32", 8, 40, 10000.0)
+    oc = oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens, rope_base=w.rope_base)
+    full = []
+    for t in range(w.n_steps):
+        q, k, v = workloads.chunk_inputs(w, 9, t)
+        full.append(oc.fold_step(q.double().numpy(), k.double().numpy(), v.double().numpy()))
+    assert np.array_equal(ret["out"], np.concatenate(full))             # head slices, nothing else
+
+
 def test_single_process_helpers():
+    assert multi.kv_head_shard(3, 4, 32, 8) == (range(24, 32), range(6, 8))
+    import pytest
+    with pytest.raises(ValueError):
+        multi.kv_head_shard(0, 3, 32, 8)
     assert multi.sequence_of_rank(3, 2) == [6, 7]
     assert multi.max_over_ranks(3.5) == 3.5
     assert multi.whole_job_tokens_per_s(131072, 5, 8, 1000.0) == 8 * 5 * 131072
