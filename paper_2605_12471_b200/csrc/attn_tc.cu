@@ -257,6 +257,8 @@ __device__ __forceinline__ void exp_half(const uint32_t *v, uint32_t *p, float2 
     }
 }
 
+// kWindow = false compiles the sink + window arithmetic out (launched whenever win_lo == 0).
+template <bool kWindow>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v) {
@@ -285,7 +287,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     const int tiles = (streams == 2 || row0 + kRows < n * G) ? 2 : 1;
     const int tok_last = min(n - 1, (row0 + 2 * kRows - 1) / G);
     // (virtual key tiles: without a window they are the key tiles themselves)
-    const WindowTiles wt(a.win_lo, a.n_sink, kRows);
+    const WindowTiles wt(kWindow ? a.win_lo : 0, kWindow ? a.n_sink : 0, kRows);
     const int nt_need = (int)((P + tok_last + 1 + kRows - 1) / kRows) - wt.skip;
     const int nt_all = (int)((L + kRows - 1) / kRows) - wt.skip;
     const int64_t line = (int64_t)a.Hkv * nt_all;
@@ -549,10 +551,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 tc_fence_after();
                 const int64_t key0 = (int64_t)wt.actual(kt0 + j) * kRows;
                 const int nvis = (int)max((int64_t)0, min((int64_t)kRows, limit - key0));
-                // window: columns below lo_c lie before the window and count only if they are sinks
-                const int lo_c = (int)max((int64_t)0, min((int64_t)kRows, a.win_lo - key0));
-                const int sink_c = (int)max((int64_t)0, min((int64_t)kRows, a.n_sink - key0));
-                const bool masked = __any_sync(0xffffffffu, nvis < kRows) || lo_c > sink_c;
+                // a tile that starts before the window holds hidden columns (the sink tile, the window's first)
+                const bool masked = __any_sync(0xffffffffu, nvis < kRows) || (kWindow && key0 < a.win_lo);
 
                 // the whole score row in registers after one load
                 uint32_t sc[128];
@@ -562,6 +562,9 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 KVF_TMEM_LD32(sc, 96, t_s + 96);
                 tmem_wait_ld();
                 if (masked) {
+                    // columns below lo_c lie before the window and count only if they are sinks
+                    const int lo_c = kWindow ? (int)max((int64_t)0, min((int64_t)kRows, a.win_lo - key0)) : 0;
+                    const int sink_c = kWindow ? (int)max((int64_t)0, min((int64_t)kRows, a.n_sink - key0)) : 0;
 #pragma unroll
                     for (int c = 0; c < 128; ++c) sc[c] = (c < nvis && (c >= lo_c || c < sink_c)) ? sc[c] : 0xFF800000u;   // -inf
                 }
@@ -787,10 +790,11 @@ int attn_tc_streams(int n, int G) { return n * G <= kRows ? 2 : 1; }
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
     static_assert(sizeof(Ctl) <= 512, "control block");
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    auto kernel = a.win_lo > 0 ? attn_tc_kernel<true> : attn_tc_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
     dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, a.batch);
-    return launch_pdl(attn_tc_kernel, grid, dim3(kThreads), kSmemBytes, s, a, maps.q, maps.k, maps.v);
+    return launch_pdl(kernel, grid, dim3(kThreads), kSmemBytes, s, a, maps.q, maps.k, maps.v);
 }
 
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s) {
