@@ -255,6 +255,17 @@ kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, c
                                int32_t n_tokens, int64_t pos0, void *out, float *lse_or_null,
                                void *cuda_stream);
 
+/*
+ * The same step for members that hold DIFFERENT numbers of rows (sequences of different length
+ * decoded together).  n_tokens is still common.  pos0_or_null: host array [n_caches] of the chunks'
+ * first positions, or null = each member's own length.  One more small launch per 64 members hands
+ * the members' row counts to the kernels; the key range is cut as the longest member needs.  Not
+ * available under a sink + window mask (KVF_ERR_UNSUPPORTED).
+ */
+kvf_status kvf_batch_fold_step_ragged(kvf_batch *b, const void *q, const void *k_new, const void *v_new,
+                                      int32_t n_tokens, const int64_t *pos0_or_null, void *out,
+                                      float *lse_or_null, void *cuda_stream);
+
 /* kvf_cache_plan for a batch step; plan[2] counts the CTAs of all members. */
 kvf_status kvf_batch_plan(const kvf_batch *b, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]);
 

@@ -28,6 +28,7 @@ EXPORTS = [
     "kvf_paged_pool_bytes", "kvf_paged_cache_create",
     "kvf_batch_workspace_bytes", "kvf_batch_create", "kvf_batch_fold_step", "kvf_batch_plan",
     "kvf_batch_status_word", "kvf_batch_launch_count", "kvf_batch_destroy", "kvf_cache_set_window",
+    "kvf_batch_fold_step_ragged",
 ]
 
 
@@ -112,6 +113,8 @@ def load() -> ctypes.CDLL:
     lib.kvf_batch_create.restype = ctypes.c_int
     lib.kvf_batch_fold_step.argtypes = [vp, vp, vp, vp, i32, i64, vp, vp, vp]
     lib.kvf_batch_fold_step.restype = ctypes.c_int
+    lib.kvf_batch_fold_step_ragged.argtypes = [vp, vp, vp, vp, i32, ctypes.POINTER(i64), vp, vp, vp]
+    lib.kvf_batch_fold_step_ragged.restype = ctypes.c_int
     lib.kvf_batch_plan.argtypes = [vp, i32, i64, ctypes.POINTER(i32)]
     lib.kvf_batch_plan.restype = ctypes.c_int
     lib.kvf_batch_status_word.argtypes = [vp]
@@ -350,9 +353,11 @@ class Batch:
 
     __del__ = close
 
-    def fold_step(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, pos0: Optional[int] = None,
+    def fold_step(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, pos0=None,
                   out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
-                  stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+                  stream: Optional[torch.cuda.Stream] = None, ragged: bool = False) -> torch.Tensor:
+        """kvf_batch_fold_step, or with ragged=True kvf_batch_fold_step_ragged (members of different
+        length; pos0 is then None or one position per member)."""
         assert q.dim() == 4 and q.shape[0] == len(self.caches)
         n = q.shape[1]
         for t in (q, k_new, v_new):
@@ -360,6 +365,14 @@ class Batch:
         if out is None:
             od = torch.float32 if (self.cfg.flags & KVF_OUT_F32) else torch.bfloat16
             out = torch.empty(q.shape, dtype=od, device=q.device)
+        if ragged:
+            arr = None if pos0 is None else (ctypes.c_int64 * len(self.caches))(*[int(p) for p in pos0])
+            rc = load().kvf_batch_fold_step_ragged(self._h, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), n, arr,
+                                                   out.data_ptr(), lse.data_ptr() if lse is not None else None,
+                                                   _stream_ptr(stream))
+            if rc != KVF_OK:
+                raise KvfError(rc, "kvf_batch_fold_step_ragged")
+            return out
         if pos0 is None:
             pos0 = len(self.caches[0])
         rc = load().kvf_batch_fold_step(self._h, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), n, int(pos0),

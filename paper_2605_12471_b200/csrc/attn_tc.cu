@@ -272,7 +272,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     const int qpair = blockIdx.x, group = blockIdx.y;
     const int cb = blockIdx.z;     // cache of a batch (0 when there is one cache)
     const int G = a.G, n = a.n;
-    const int64_t P = a.prefix, L = P + n;
+    const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix, L = P + n;
     // streams == 2 (chunks of at most 128 / G tokens, i.e. one row tile): the two tile slots work on
     // the SAME 128 rows and take alternate key tiles, so that one stream's softmax still runs under
     // the other stream's MMAs; each stream leaves its own partial result.
@@ -708,7 +708,8 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
-        const int nt_all = (int)((a.prefix + a.n + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
+        const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix;
+        const int nt_all = (int)((P + a.n + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
         const int64_t line = (int64_t)a.Hkv * nt_all;
         auto start = [&](int64_t g) { return g * line / a.ngroups; };
         auto group_of = [&](int64_t lin) {

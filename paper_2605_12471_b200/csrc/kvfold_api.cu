@@ -108,7 +108,7 @@ struct kvf_cache {
 struct kvf_batch {
     std::vector<kvf_cache *> caches;
     char *workspace;
-    size_t off_status, off_tables, off_q_rot, off_part_o, off_part_lse;
+    size_t off_status, off_tables, off_lens, off_q_rot, off_part_o, off_part_lse;
     int64_t part_rows;       // rows of the partial area per cache
     CUtensorMap map_q;       // rotated chunks of all members: [n_caches * max_chunk][H][d]
     uint64_t launches;
@@ -117,7 +117,7 @@ struct kvf_batch {
 namespace {
 
 struct BatchLayout {
-    size_t status, tables, q_rot, part_o, part_lse, total;
+    size_t status, tables, lens, q_rot, part_o, part_lse, total;
     int64_t part_rows;
 };
 
@@ -132,6 +132,7 @@ BatchLayout batch_layout(const kvf_config *c, int n_caches) {
     size_t off = 0;
     l.status = off;   off = align_up(off + 256, 1024);
     l.tables = off;   off = align_up(off + (size_t)n_caches * sizeof(void *), 1024);
+    l.lens = off;     off = align_up(off + (size_t)n_caches * 2 * sizeof(int64_t), 1024);   // row counts, then first positions
     l.q_rot = off;    off = align_up(off + (size_t)n_caches * c->max_chunk * c->n_q_heads * c->head_dim * elem_bytes(c->dtype), 1024);
     l.part_o = off;   off = align_up(off + (size_t)n_caches * rows * c->head_dim * 4, 1024);
     l.part_lse = off; off = align_up(off + (size_t)n_caches * rows * 4, 1024);
@@ -354,6 +355,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     ra.page_table = c->page_table;
     ra.page_elems = c->page_elems;
     ra.page_tables = nullptr;
+    ra.prefixes = nullptr; ra.pos0s = nullptr;
     ra.table = c->table;
 
     AttnArgs aa;
@@ -364,7 +366,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.part_lse = reinterpret_cast<float *>(c->workspace + c->lay.part_lse);
     aa.status = reinterpret_cast<int *>(c->workspace + c->lay.status);
     aa.page_table = c->page_table;
-    aa.page_tables = nullptr; aa.part_rows = 0; aa.batch = 1;
+    aa.page_tables = nullptr; aa.part_rows = 0; aa.batch = 1; aa.prefixes = nullptr;
     aa.n_sink = c->n_sink; aa.win_lo = window_lo(c, P);
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
@@ -692,7 +694,7 @@ kvf_status kvf_batch_create(kvf_cache *const *caches, int32_t n_caches, void *de
     if (!b) return KVF_ERR_INVALID_ARG;
     b->caches.assign(caches, caches + n_caches);
     b->workspace = static_cast<char *>(dev_workspace);
-    b->off_status = lay.status; b->off_tables = lay.tables; b->off_q_rot = lay.q_rot;
+    b->off_status = lay.status; b->off_tables = lay.tables; b->off_lens = lay.lens; b->off_q_rot = lay.q_rot;
     b->off_part_o = lay.part_o; b->off_part_lse = lay.part_lse;
     b->part_rows = lay.part_rows;
     b->launches = 0;
@@ -716,15 +718,42 @@ kvf_status kvf_batch_create(kvf_cache *const *caches, int32_t n_caches, void *de
     return KVF_OK;
 }
 
-kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, const void *v_new, int32_t n,
-                               int64_t pos0, void *out, float *lse, void *cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+// Per-member row counts and first positions of a ragged step, 64 members per launch, written into
+// the batch workspace by a plain (fully stream-ordered) kernel: no host-to-device copy, so a
+// ragged step can be captured into a graph like any other.
+struct LenChunk {
+    int64_t prefix[64], pos0[64];
+    int32_t base, count;
+};
+__global__ void write_lengths_kernel(const LenChunk c, int64_t *prefixes, int64_t *pos0s) {
+    const int i = threadIdx.x;
+    if (i < c.count) {
+        prefixes[c.base + i] = c.prefix[i];
+        pos0s[c.base + i] = c.pos0[i];
+    }
+}
+
+// One step of a batch.  pos0s == nullptr: every member holds the same number of rows and starts at
+// pos0; else member i starts at pos0s[i] and the members' row counts may differ.
+kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void *v_new, int32_t n,
+                      int64_t pos0, const int64_t *pos0s, void *out, float *lse, void *cuda_stream) {
     if (!b) return KVF_ERR_INVALID_ARG;
     kvf_cache *c0 = b->caches[0];
-    const int64_t P = c0->len;
-    for (kvf_cache *c : b->caches)
-        if (c->len != P || c->n_sink != c0->n_sink || c->window != c0->window)
-            return KVF_ERR_INVALID_ARG;                       // the members advance together, under one mask
-    kvf_status s = check_step(c0, n, pos0);
+    const bool ragged = pos0s != nullptr;
+    int64_t P = c0->len;                                      // ragged: the longest member, for the plan
+    for (kvf_cache *c : b->caches) {
+        if (c->n_sink != c0->n_sink || c->window != c0->window) return KVF_ERR_INVALID_ARG;   // one mask
+        if (!ragged && c->len != P) return KVF_ERR_INVALID_ARG;   // the members advance together
+        if (c->len > P) P = c->len;
+    }
+    if (ragged && c0->window > 0) return KVF_ERR_UNSUPPORTED;     // the window is placed per launch
+    kvf_status s = KVF_OK;
+    for (size_t i = 0; i < b->caches.size() && s == KVF_OK; ++i)
+        s = check_step(b->caches[i], n, ragged ? pos0s[i] : pos0);
     if (s != KVF_OK) return s;
     if (check_ptr(q) || check_ptr(k_new) || check_ptr(v_new) || check_ptr(out)) return KVF_ERR_INVALID_ARG;
     if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return KVF_ERR_INVALID_ARG;
@@ -732,6 +761,23 @@ kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, c
     const kvf_config &f = c0->cfg;
     const int B = (int)b->caches.size();
     const Plan plan = make_plan(c0, n, P, B, b->part_rows);
+    int64_t *dev_prefixes = reinterpret_cast<int64_t *>(b->workspace + b->off_lens);
+    int64_t *dev_pos0s = dev_prefixes + B;
+    if (ragged) {
+        for (int base = 0; base < B; base += 64) {
+            LenChunk ch;
+            ch.base = base;
+            ch.count = std::min(64, B - base);
+            for (int i = 0; i < ch.count; ++i) {
+                ch.prefix[i] = b->caches[base + i]->len;
+                ch.pos0[i] = pos0s[base + i];
+            }
+            write_lengths_kernel<<<1, 64, 0, st>>>(ch, dev_prefixes, dev_pos0s);
+            cudaError_t e = cudaGetLastError();
+            if (e != cudaSuccess) return cuda_fail(e, "write_lengths launch");
+            b->launches++;
+        }
+    }
     const int32_t *const *tables = reinterpret_cast<const int32_t *const *>(b->workspace + b->off_tables);
 
     RopeAppendArgs ra;
@@ -741,10 +787,13 @@ kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, c
     ra.v_plane = c0->storage + c0->plane_bytes;
     ra.capacity = f.capacity; ra.prefix = P; ra.pos0 = pos0;
     ra.n = n; ra.H = f.n_q_heads; ra.Hkv = f.n_kv_heads; ra.d = f.head_dim;
-    ra.zero_rows = (int32_t)((P + n + kKvTile - 1) / kKvTile * kKvTile - (P + n));
+    // value rows to clear up to the next page boundary; ragged: each member's own count, at most a page less one
+    ra.zero_rows = ragged ? kKvTile - 1 : (int32_t)((P + n + kKvTile - 1) / kKvTile * kKvTile - (P + n));
     ra.page_table = c0->page_table;
     ra.page_elems = c0->page_elems;
     ra.page_tables = tables;
+    ra.prefixes = ragged ? dev_prefixes : nullptr;
+    ra.pos0s = ragged ? dev_pos0s : nullptr;
     ra.table = c0->table;
 
     AttnArgs aa;
@@ -756,6 +805,7 @@ kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, c
     aa.status = reinterpret_cast<int *>(b->workspace + b->off_status);
     aa.page_table = c0->page_table;
     aa.page_tables = tables; aa.part_rows = b->part_rows; aa.batch = B;
+    aa.prefixes = ragged ? dev_prefixes : nullptr;
     aa.n_sink = c0->n_sink; aa.win_lo = window_lo(c0, P);
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c0->G; aa.d = f.head_dim;
@@ -778,8 +828,28 @@ kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, c
         if (e != cudaSuccess) return cuda_fail(e, "combine launch (batch)");
         b->launches++;
     }
-    for (kvf_cache *c : b->caches) c->len = P + n;
+    for (kvf_cache *c : b->caches) c->len += n;
     return KVF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, const void *v_new, int32_t n,
+                               int64_t pos0, void *out, float *lse, void *cuda_stream) {
+    return batch_step(b, q, k_new, v_new, n, pos0, nullptr, out, lse, cuda_stream);
+}
+
+kvf_status kvf_batch_fold_step_ragged(kvf_batch *b, const void *q, const void *k_new, const void *v_new, int32_t n,
+                                      const int64_t *pos0_or_null, void *out, float *lse, void *cuda_stream) {
+    if (!b) return KVF_ERR_INVALID_ARG;
+    std::vector<int64_t> own;
+    if (!pos0_or_null) {                                       // positions continue from each member's length
+        for (kvf_cache *c : b->caches) own.push_back(c->len);
+        pos0_or_null = own.data();
+    }
+    return batch_step(b, q, k_new, v_new, n, 0, pos0_or_null, out, lse, cuda_stream);
 }
 
 kvf_status kvf_batch_plan(const kvf_batch *b, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]) {

@@ -72,6 +72,9 @@ struct RopeAppendArgs {
     // batch of caches advancing together (blockIdx.y = cache b): q, k_new, v_new, q_rot hold the
     // caches' chunks one after the other; cache b's rows go where page_tables[b] says
     const int32_t *const *page_tables;   // device array of device tables, or null (one cache)
+    // ragged batch: cache b holds prefixes[b] rows and its chunk starts at position pos0s[b]
+    // (device arrays, or null: prefix and pos0 above hold for every cache)
+    const int64_t *prefixes, *pos0s;
     RopeTable table;
 };
 
@@ -92,6 +95,7 @@ struct AttnArgs {
     const int32_t *const *page_tables;   // device array of device tables, or null (one cache)
     int64_t part_rows;               // rows of the partial area per cache of a batch
     int32_t batch;                   // caches in the launch (1 = one cache)
+    const int64_t *prefixes;         // ragged batch: device array of the caches' row counts, else null
     // sink + window variant: of the rows before the chunk only those below n_sink or from win_lo on
     // are visible (win_lo = 0: all of them); see WindowTiles
     int32_t n_sink;

@@ -67,6 +67,10 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
     const int n_tok_blocks = (a.n + kTok - 1) / kTok;
     const int b = blockIdx.y;      // cache of a batch (0 when there is one cache)
     const RowMap rows{a.page_tables ? a.page_tables[b] : a.page_table, a.capacity, a.page_elems, a.d};
+    // (the per-cache arrays of a ragged batch were written by a kernel that had finished before
+    // this one could start)
+    const int64_t prefix = a.prefixes ? a.prefixes[b] : a.prefix;
+    const int64_t pos0 = a.pos0s ? a.pos0s[b] : a.pos0;
 
     pdl_launch_dependents();
     if ((int)blockIdx.x >= n_tok_blocks) {
@@ -74,7 +78,8 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
         // Clear value rows between the new end of the cache and the next key-tile boundary,
         // so that a zero probability never multiplies stale non-finite bits.
         const int vec_per_row = d / VEC;
-        const int64_t total = (int64_t)a.zero_rows * a.Hkv * vec_per_row;
+        const int zero_rows = a.prefixes ? (int)((kKvTile - (prefix + a.n) % kKvTile) % kKvTile) : a.zero_rows;
+        const int64_t total = (int64_t)zero_rows * a.Hkv * vec_per_row;
         const int64_t start = ((int64_t)blockIdx.x - n_tok_blocks) * kThreads + threadIdx.x;
         const int64_t stride = (int64_t)(gridDim.x - n_tok_blocks) * kThreads;
         T *vp = reinterpret_cast<T *>(a.v_plane);
@@ -82,7 +87,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             int c = (int)(i % vec_per_row);
             int64_t t = i / vec_per_row;
             int g = (int)(t % a.Hkv);
-            int64_t row = a.prefix + a.n + t / a.Hkv;
+            int64_t row = prefix + a.n + t / a.Hkv;
             *reinterpret_cast<uint4 *>(vp + rows.offset(g, row) + c * VEC) =
                 make_uint4(0, 0, 0, 0);
         }
@@ -94,7 +99,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
 
     for (int idx = threadIdx.x; idx < ntok * half; idx += kThreads) {
         int t = idx / half, j = idx % half;
-        double theta = (double)(a.pos0 + tok0 + t) * a.table.inv_freq[j];
+        double theta = (double)(pos0 + tok0 + t) * a.table.inv_freq[j];
         double sn, cn;
         sincos(theta, &sn, &cn);
         cs[t][j] = make_float2((float)cn, (float)sn);
@@ -126,7 +131,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             } else {
                 int g = hh - a.H;
                 src = k + ((int64_t)(tok0 + t) * a.Hkv + g) * d;
-                dst = kp + rows.offset(g, a.prefix + tok0 + t);
+                dst = kp + rows.offset(g, prefix + tok0 + t);
             }
             float lo[VEC], hi[VEC], rlo[VEC], rhi[VEC];
             Vec16<T>::load(src + c * VEC, lo);
@@ -154,7 +159,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             } else {
                 int g = hh - a.H;
                 src = k + ((int64_t)(tok0 + t) * a.Hkv + g) * d;
-                dst = kp + rows.offset(g, a.prefix + tok0 + t);
+                dst = kp + rows.offset(g, prefix + tok0 + t);
             }
             float x[VEC], r[VEC];
             Vec16<T>::load(src + c * VEC, x);
@@ -176,7 +181,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             int g = (idx / chunks) % a.Hkv;
             int t = idx / (chunks * a.Hkv);
             uint4 val = *reinterpret_cast<const uint4 *>(v + ((int64_t)(tok0 + t) * a.Hkv + g) * d + c * VEC);
-            *reinterpret_cast<uint4 *>(vp + rows.offset(g, a.prefix + tok0 + t) + c * VEC) = val;
+            *reinterpret_cast<uint4 *>(vp + rows.offset(g, prefix + tok0 + t) + c * VEC) = val;
         }
     }
 }

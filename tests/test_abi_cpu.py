@@ -135,6 +135,8 @@ def test_batch_entry_points_validate_before_any_cuda_call(binding):
     assert lib.kvf_batch_create(arr, 0, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
     assert h.value is None
     assert lib.kvf_batch_fold_step(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_batch_fold_step_ragged(None, None, None, None, 1, None, None, None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_cache_set_window(None, 0, 0) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_batch_plan(None, 1, 0, (ctypes.c_int32 * 4)()) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_batch_status_word(None) == -1
     assert lib.kvf_batch_launch_count(None) == 0

@@ -139,3 +139,58 @@ def test_batch_rejects_members_it_cannot_fold_together():
     batch.fold_step(q, k, v)                                            # level again
     torch.cuda.synchronize()
     assert batch.status_word() == 0 and len(caches[0]) == len(caches[1]) == 32
+
+
+def test_ragged_batch_members_of_different_length():
+    """Five sequences of different length taken forward together: a common prompt-sized step each on
+    its own first, then decode-shaped and chunk-sized batch steps; every member against its oracle,
+    and the pool bit-identical to folding every member by itself."""
+    B = 5
+    lens0 = [0, 130, 1000, 257, 4000]
+    steps = [1, 1, 16, 256, 1, 100]
+    cap = max(lens0) + sum(steps) + 128
+    cfg, pool, tables, caches = make_members(B, cap, 2048, seed=15)
+    _, pool1, _, singles = make_members(B, cap, 2048, seed=15)
+    ocs = [oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, cap, rope_base=W.rope_base) for _ in range(B)]
+    for i, L in enumerate(lens0):                              # bring the members to different lengths
+        t0 = 0
+        while t0 < L:
+            n = min(2048, L - t0)
+            q, k, v = workloads.chunk_inputs(W, 91, t0, sequence=i, device="cuda", n_tokens=n)
+            caches[i].fold_step(q, k, v)
+            singles[i].fold_step(q, k, v)
+            ocs[i].fold_step(to_f64(q), to_f64(k), to_f64(v), rows=[])
+            t0 += n
+    batch = binding.Batch(caches)
+    with pytest.raises(binding.KvfError) as e:
+        batch.fold_step(*batch_inputs(B, 1, 92, 0))            # the lock-step call refuses unequal members
+    assert e.value.code == binding.KVF_ERR_INVALID_ARG
+    worst, worst_lse = 0.0, 0.0
+    for t, n in enumerate(steps):
+        q, k, v = batch_inputs(B, n, 93, t)
+        lse = torch.empty((B, n, W.n_q_heads), dtype=torch.float32, device="cuda")
+        out = batch.fold_step(q, k, v, lse=lse, ragged=True)
+        rows = sorted({0, n // 2, n - 1})
+        for i in range(B):
+            singles[i].fold_step(q[i], k[i], v[i])
+            ref, ref_lse, _ = ocs[i].fold_step(to_f64(q[i]), to_f64(k[i]), to_f64(v[i]), rows=rows, want_stats=True)
+            worst = max(worst, float(np.abs(to_f64(out[i][rows]) - ref).max()))
+            worst_lse = max(worst_lse, float(np.abs(to_f64(lse[i][rows]) - ref_lse).max()))
+        assert [len(c) for c in caches] == [L + sum(steps[:t + 1]) for L in lens0]
+    torch.cuda.synchronize()
+    assert batch.status_word() == 0
+    assert torch.equal(pool, pool1)
+    assert worst <= TOL["bf16"][0] and worst_lse <= 2e-2, (worst, worst_lse)
+    # explicit positions: a member may be rotated from another origin than its length
+    q, k, v = batch_inputs(B, 1, 94, 0)
+    shifted = [len(c) + 7 for c in caches]
+    out = batch.fold_step(q, k, v, pos0=shifted, ragged=True)
+    for i in (0, 4):
+        ref = ocs[i].fold_step(to_f64(q[i]), to_f64(k[i]), to_f64(v[i]), pos0=shifted[i])
+        assert float(np.abs(to_f64(out[i]) - ref).max()) <= TOL["bf16"][0]
+    caches[0].set_window(4, 64)
+    for c in caches[1:]:
+        c.set_window(4, 64)
+    with pytest.raises(binding.KvfError) as e:
+        batch.fold_step(q, k, v, ragged=True)
+    assert e.value.code == binding.KVF_ERR_UNSUPPORTED
