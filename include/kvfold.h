@@ -48,8 +48,18 @@ enum {
     KVF_ROPE_INTERLEAVED = 1u, /* rotate pairs (2j,2j+1) instead of (j, j+d/2)                   */
     KVF_STRICT_POS = 2u,       /* reject pos0 != len (positions must continue across chunks)     */
     KVF_OUT_F32 = 4u,          /* `out` is fp32 even when dtype is bf16                          */
-    KVF_FORCE_SIMT = 8u        /* use the CUDA-core attention kernel even where the tensor-core
+    KVF_FORCE_SIMT = 8u,       /* use the CUDA-core attention kernel even where the tensor-core
                                   kernel applies (bisecting aid; same results within tolerance) */
+    KVF_CACHE_INT8 = 16u       /* store the cache as int8 codes with one fp32 scale per row (one token of
+                                  one KV head): d + 4 bytes per row instead of 2 d.  The paper's Discussion
+                                  perturbs the stored K/V by a round trip bf16 -> intN -> bf16 and leaves
+                                  the scheme open; here a row is quantised once, when it is appended:
+                                  scale = max|x| / 127, code = clamp(rint(x * (127 / max|x|)), +-127) in
+                                  fp32 (keys: on the rotated row before any rounding to bf16), and the
+                                  attention sees bf16(code * scale).  dtype KVF_BF16 and head_dim 128
+                                  only (KVF_ERR_UNSUPPORTED otherwise, and for paged caches and
+                                  kvf_fold_step_static); the workspace then also holds a bf16 image of
+                                  one cache that every step re-expands from the codes */
 };
 
 /*
@@ -170,9 +180,12 @@ kvf_status kvf_cache_status(kvf_cache *c);
  * -1 for a null handle or a failed copy. */
 int32_t kvf_cache_status_word(kvf_cache *c);
 
-/* Device pointers of the planes, [n_kv_heads][capacity][head_dim] of dtype. */
+/* Device pointers of the planes, [n_kv_heads][capacity][head_dim] of dtype (int8 codes under
+ * KVF_CACHE_INT8), and of the rows' fp32 scales [n_kv_heads][capacity] (NULL without that flag). */
 void *kvf_cache_k_plane(const kvf_cache *c);
 void *kvf_cache_v_plane(const kvf_cache *c);
+float *kvf_cache_k_scales(const kvf_cache *c);
+float *kvf_cache_v_scales(const kvf_cache *c);
 
 /*
  * What a step of n_tokens on a prefix of prefix_len would launch:

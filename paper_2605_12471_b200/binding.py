@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libkvfold.so")
 KVF_OK, KVF_ERR_INVALID_ARG, KVF_ERR_CAPACITY, KVF_ERR_UNSUPPORTED, KVF_ERR_CUDA, KVF_ERR_TIMEOUT, \
     KVF_ERR_POS = range(7)
 KVF_BF16, KVF_F32 = 0, 1
-KVF_ROPE_INTERLEAVED, KVF_STRICT_POS, KVF_OUT_F32, KVF_FORCE_SIMT = 1, 2, 4, 8
+KVF_ROPE_INTERLEAVED, KVF_STRICT_POS, KVF_OUT_F32, KVF_FORCE_SIMT, KVF_CACHE_INT8 = 1, 2, 4, 8, 16
 
 EXPORTS = [
     "kvf_cache_storage_bytes", "kvf_workspace_bytes", "kvf_cache_create", "kvf_fold_step",
@@ -28,7 +28,7 @@ EXPORTS = [
     "kvf_paged_pool_bytes", "kvf_paged_cache_create",
     "kvf_batch_workspace_bytes", "kvf_batch_create", "kvf_batch_fold_step", "kvf_batch_plan",
     "kvf_batch_status_word", "kvf_batch_launch_count", "kvf_batch_destroy", "kvf_cache_set_window",
-    "kvf_batch_fold_step_ragged",
+    "kvf_batch_fold_step_ragged", "kvf_cache_k_scales", "kvf_cache_v_scales",
 ]
 
 
@@ -93,6 +93,10 @@ def load() -> ctypes.CDLL:
     lib.kvf_cache_k_plane.restype = vp
     lib.kvf_cache_v_plane.argtypes = [vp]
     lib.kvf_cache_v_plane.restype = vp
+    lib.kvf_cache_k_scales.argtypes = [vp]
+    lib.kvf_cache_k_scales.restype = vp
+    lib.kvf_cache_v_scales.argtypes = [vp]
+    lib.kvf_cache_v_scales.restype = vp
     lib.kvf_cache_plan.argtypes = [vp, i32, i64, ctypes.POINTER(i32)]
     lib.kvf_cache_plan.restype = ctypes.c_int
     lib.kvf_cache_set_splits.argtypes = [vp, i32]
@@ -240,10 +244,24 @@ class Cache:
         return int(load().kvf_cache_status_word(self._h))
 
     def _plane(self, ptr: int) -> torch.Tensor:
-        plane_bytes = self.storage.numel() // 2
+        shape = (self.cfg.n_kv_heads, self.cfg.capacity, self.cfg.head_dim)
         off = ptr - self.storage.data_ptr()
+        if self.cfg.flags & KVF_CACHE_INT8:                     # int8 codes
+            n = shape[0] * shape[1] * shape[2]
+            return self.storage[off:off + n].view(torch.int8).view(shape)
+        plane_bytes = self.storage.numel() // 2
         flat = self.storage[off:off + plane_bytes].view(self.torch_dtype)
-        return flat.view(self.cfg.n_kv_heads, self.cfg.capacity, self.cfg.head_dim)
+        return flat.view(shape)
+
+    def scales(self, kv: int) -> torch.Tensor:
+        """[Hkv, capacity] fp32 row scales of the K (kv = 0) or V (kv = 1) codes (KVF_CACHE_INT8 only)."""
+        lib = load()
+        ptr = lib.kvf_cache_v_scales(self._h) if kv else lib.kvf_cache_k_scales(self._h)
+        if not ptr:
+            raise ValueError("this cache holds no scales")
+        off = ptr - self.storage.data_ptr()
+        n = self.cfg.n_kv_heads * self.cfg.capacity
+        return self.storage[off:off + 4 * n].view(torch.float32).view(self.cfg.n_kv_heads, self.cfg.capacity)
 
     def k_plane(self) -> torch.Tensor:
         """[Hkv, capacity, d] view of the rotated keys (rows >= len are not content)."""

@@ -42,11 +42,14 @@ kvf_status check_config(const kvf_config *c) {
     if (c->softmax_scale < 0.0) return KVF_ERR_INVALID_ARG;
     if ((int64_t)c->max_chunk > c->capacity) return KVF_ERR_INVALID_ARG;
     if (c->capacity > (int64_t)1 << 31) return KVF_ERR_UNSUPPORTED;
+    if ((c->flags & KVF_CACHE_INT8) &&
+        (c->dtype != KVF_BF16 || (c->flags & KVF_FORCE_SIMT) || !attn_tc_supported(c->dtype, c->head_dim, G)))
+        return KVF_ERR_UNSUPPORTED;
     return KVF_OK;
 }
 
 struct Layout {
-    size_t status, q_rot, st_q, st_k, st_v, st_out, st_lse, part_o, part_lse, total;
+    size_t status, q_rot, st_q, st_k, st_v, st_out, st_lse, part_o, part_lse, deq, total;
 };
 
 Layout workspace_layout(const kvf_config *c) {
@@ -66,6 +69,8 @@ Layout workspace_layout(const kvf_config *c) {
     l.st_lse = off;   off = align_up(off + (size_t)c->max_chunk * c->n_q_heads * 4, 1024);
     l.part_o = off;   off = align_up(off + (size_t)kPartTokens * c->n_q_heads * c->head_dim * 4, 1024);
     l.part_lse = off; off = align_up(off + (size_t)kPartTokens * c->n_q_heads * 4, 1024);
+    l.deq = off;      // quantised storage: bf16 image of one cache (K plane, then V plane)
+    if (c->flags & KVF_CACHE_INT8) off = align_up(off + 2 * (size_t)c->n_kv_heads * (size_t)c->capacity * c->head_dim * 2, 1024);
     l.total = off;
     return l;
 }
@@ -98,6 +103,8 @@ struct kvf_cache {
     const int32_t *page_table = nullptr;   // paged cache: device table, one page number per 128 tokens
     int64_t page_elems = 0;                // paged cache: elements per page
     int32_t n_pool_pages = 0;
+    bool quant = false;                    // int8 storage: codes + scales in `storage`, bf16 image in the workspace
+    QuantPlanes qp = {};
     int32_t n_sink = 0;                    // sink + window variant: rows always visible
     int64_t window = 0;                    // and the rows before the chunk that stay visible (0 = all)
     std::vector<ProfRec> recs;
@@ -213,11 +220,13 @@ kvf_status build_maps(kvf_cache *c) {
         return make_page_map(fn, &c->maps.v, c->storage + c->plane_bytes, d, f.n_kv_heads, (uint64_t)c->n_pool_pages,
                              page_bytes);
     }
-    // planes [Hkv][capacity][d]: one box = 128 rows of one head x 64
-    s = make_map(fn, &c->maps.k, c->storage, (uint64_t)f.capacity, (uint64_t)f.n_kv_heads, row,
+    // planes [Hkv][capacity][d]: one box = 128 rows of one head x 64 (quantised storage: the bf16 image)
+    char *kbase = c->quant ? c->workspace + c->lay.deq : c->storage;
+    char *vbase = c->quant ? kbase + (size_t)f.n_kv_heads * f.capacity * d * 2 : c->storage + c->plane_bytes;
+    s = make_map(fn, &c->maps.k, kbase, (uint64_t)f.capacity, (uint64_t)f.n_kv_heads, row,
                  row * f.capacity, d, (uint32_t)kKvTile, 1u);
     if (s != KVF_OK) return s;
-    return make_map(fn, &c->maps.v, c->storage + c->plane_bytes, (uint64_t)f.capacity,
+    return make_map(fn, &c->maps.v, vbase, (uint64_t)f.capacity,
                     (uint64_t)f.n_kv_heads, row, row * f.capacity, d, (uint32_t)kKvTile, 1u);
 }
 
@@ -377,7 +386,18 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.scale_log2 = c->scale_log2;
 
     cudaError_t e;
-    {
+    if (c->quant) {
+        // quantised storage: rotate + quantise + append, then the bf16 image of rows [0, L) that the
+        // attention kernel reads (its planes are in the workspace)
+        char *deq_k = c->workspace + c->lay.deq;
+        char *deq_v = deq_k + (size_t)f.n_kv_heads * f.capacity * f.head_dim * 2;
+        aa.k_plane = deq_k; aa.v_plane = deq_v;
+        ProfScope ps(c, st, 0);
+        e = launch_rope_append_q8(ra, c->qp, (f.flags & KVF_ROPE_INTERLEAVED) != 0, st);
+        if (e == cudaSuccess)
+            e = launch_expand_q8(c->qp, deq_k, deq_v, f.capacity, P + n, ra.zero_rows, f.n_kv_heads, c->sm_count, st);
+        c->launches++;
+    } else {
         ProfScope ps(c, st, 0);
         e = launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, 1, st);
     }
@@ -417,6 +437,8 @@ extern "C" {
 
 size_t kvf_cache_storage_bytes(const kvf_config *cfg) {
     if (check_config(cfg) != KVF_OK) return 0;
+    if (cfg->flags & KVF_CACHE_INT8)   // codes and one fp32 scale per row, K and V
+        return 2 * (size_t)cfg->n_kv_heads * (size_t)cfg->capacity * ((size_t)cfg->head_dim + 4);
     return 2 * (size_t)cfg->n_kv_heads * (size_t)cfg->capacity * (size_t)cfg->head_dim * elem_bytes(cfg->dtype);
 }
 
@@ -454,6 +476,15 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
     c->workspace = static_cast<char *>(dev_workspace);
     c->plane_bytes = kvf_cache_storage_bytes(cfg) / 2;
     c->lay = workspace_layout(cfg);
+    if (cfg->flags & KVF_CACHE_INT8) {
+        const size_t codes = (size_t)cfg->n_kv_heads * cfg->capacity * cfg->head_dim;
+        c->quant = true;
+        c->plane_bytes = codes;
+        c->qp.k_codes = reinterpret_cast<int8_t *>(c->storage);
+        c->qp.v_codes = c->qp.k_codes + codes;
+        c->qp.k_scales = reinterpret_cast<float *>(c->storage + 2 * codes);
+        c->qp.v_scales = c->qp.k_scales + (size_t)cfg->n_kv_heads * cfg->capacity;
+    }
     c->len = 0;
     c->G = cfg->n_q_heads / cfg->n_kv_heads;
     const double scale = cfg->softmax_scale > 0.0 ? cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
@@ -491,6 +522,7 @@ kvf_status kvf_paged_cache_create(const kvf_config *cfg, void *dev_pool, size_t 
     if (s != KVF_OK) return s;
     const int G = cfg->n_q_heads / cfg->n_kv_heads;
     if ((cfg->flags & KVF_FORCE_SIMT) || !attn_tc_supported(cfg->dtype, cfg->head_dim, G)) return KVF_ERR_UNSUPPORTED;
+    if (cfg->flags & KVF_CACHE_INT8) return KVF_ERR_UNSUPPORTED;          // pages hold bf16 rows
     if (!dev_pool || !dev_workspace || !dev_page_table || n_pool_pages <= 0) return KVF_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(dev_pool) & 255u) || (reinterpret_cast<uintptr_t>(dev_workspace) & 255u) ||
         (reinterpret_cast<uintptr_t>(dev_page_table) & 3u))
@@ -602,6 +634,8 @@ int32_t kvf_cache_status_word(kvf_cache *c) {
 
 void *kvf_cache_k_plane(const kvf_cache *c) { return c && !c->page_table ? c->storage : nullptr; }
 void *kvf_cache_v_plane(const kvf_cache *c) { return c && !c->page_table ? c->storage + c->plane_bytes : nullptr; }
+float *kvf_cache_k_scales(const kvf_cache *c) { return c && c->quant ? c->qp.k_scales : nullptr; }
+float *kvf_cache_v_scales(const kvf_cache *c) { return c && c->quant ? c->qp.v_scales : nullptr; }
 
 kvf_status kvf_cache_plan(const kvf_cache *c, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]) {
     if (!c || !plan || n_tokens < 1 || n_tokens > c->cfg.max_chunk || prefix_len < 0) return KVF_ERR_INVALID_ARG;
@@ -941,6 +975,7 @@ extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_stor
                                            void *cuda_stream) {
     kvf_status s = check_config(cfg);
     if (s != KVF_OK) return s;
+    if (cfg->flags & KVF_CACHE_INT8) return KVF_ERR_UNSUPPORTED;          // the static scratch holds no bf16 image
     if (!dev_storage || (reinterpret_cast<uintptr_t>(dev_storage) & 255u)) return KVF_ERR_INVALID_ARG;
     if (storage_bytes < kvf_cache_storage_bytes(cfg)) return KVF_ERR_CAPACITY;
     if (len < 0 || n_tokens < 1 || n_tokens > cfg->max_chunk || pos0 < 0) return KVF_ERR_INVALID_ARG;

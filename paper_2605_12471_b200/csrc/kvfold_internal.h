@@ -124,6 +124,16 @@ struct WindowTiles {
 };
 constexpr int kMaxSinks = 64;         // sink rows sit in the first key tile of either kernel
 
+// Quantised storage: int8 codes [Hkv][capacity][d] and one fp32 scale per row [Hkv][capacity].
+struct QuantPlanes {
+    int8_t *k_codes, *v_codes;
+    float *k_scales, *v_scales;
+};
+cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, cudaStream_t s);
+// stored rows [0, rows) -> bf16 planes [Hkv][capacity][128]; value rows [rows, rows + zero_rows) cleared
+cudaError_t launch_expand_q8(const QuantPlanes &qp, void *k_out, void *v_out, int64_t capacity, int64_t rows,
+                             int32_t zero_rows, int32_t Hkv, int sm_count, cudaStream_t s);
+
 cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interleaved, int batch, cudaStream_t s);
 cudaError_t launch_attn_simt(const AttnArgs &a, int dtype, cudaStream_t s, int *grid_out);
 cudaError_t launch_combine(const AttnArgs &a, int dtype, cudaStream_t s);

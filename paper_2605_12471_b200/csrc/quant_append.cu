@@ -1,0 +1,190 @@
+// Quantised cache storage: rotate + quantise + append, and the expansion of stored rows to bf16.
+//
+// The paper's Discussion perturbs the stored K/V by a round trip bf16 -> intN -> bf16 and leaves the
+// scheme open.  Here a stored row (one token of one KV head, d elements) is symmetric int8 with one
+// fp32 scale, decided once when the row is appended:
+//     amax = max |x_j|     inv = 127 / amax     scale = amax / 127        (fp32, round to nearest)
+//     code_j = clamp(rint(x_j * inv), -127, 127)                           (ties to even)
+//     value seen by the attention = bf16(code_j * scale)                   (fp32 product, one rounding)
+// For a key row x is the rotated row in fp32 (same operation order as the bf16 path, before any
+// rounding to bf16); a value row is quantised as given.  amax = 0 gives codes 0 and scale 0.
+// The cache then holds d + 4 bytes per row instead of 2 d.
+#include "kvfold_internal.h"
+
+namespace kvf {
+namespace {
+
+constexpr int kTok = 2;        // tokens per CTA
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ void rotate(float a, float b, float c, float s, float &ra, float &rb) {
+    float cross_a = __fmul_rn(b, s);
+    float cross_b = __fmul_rn(a, s);
+    ra = __fmaf_rn(a, c, -cross_a);
+    rb = __fmaf_rn(b, c, cross_b);
+}
+
+// codes of four values of a row held by one lane; the row's scale comes back in `scale`
+__device__ __forceinline__ void quantise4(const float (&x)[4], int (&code)[4], float &scale) {
+    float amax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const float inv = amax > 0.f ? __fdiv_rn(127.f, amax) : 0.f;
+    scale = __fdiv_rn(amax, 127.f);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        float r = rintf(__fmul_rn(x[e], inv));
+        r = fminf(fmaxf(r, -127.f), 127.f);
+        code[e] = (int)r;
+    }
+}
+
+// One warp per row (d = 128: four elements per lane).  Query rows are rotated and written as bf16;
+// key rows are rotated in fp32, quantised and appended; value rows are quantised and appended.
+template <bool INTERLEAVED>
+__global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppendArgs a, const QuantPlanes qp) {
+    __shared__ float2 cs[kTok][kMaxHalfDim];   // (cos, sin) per (token, pair)
+    constexpr int d = 128, half = 64;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tok0 = blockIdx.x * kTok;
+    const int ntok = min(kTok, a.n - tok0);
+
+    pdl_launch_dependents();
+    for (int idx = threadIdx.x; idx < ntok * half; idx += kThreads) {
+        int t = idx / half, j = idx % half;
+        double theta = (double)(a.pos0 + tok0 + t) * a.table.inv_freq[j];
+        double sn, cn;
+        sincos(theta, &sn, &cn);
+        cs[t][j] = make_float2((float)cn, (float)sn);
+    }
+    __syncthreads();
+    pdl_wait();   // the table above needs nothing from earlier kernels; the writes below do
+
+    const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(a.q);
+    const __nv_bfloat16 *k = reinterpret_cast<const __nv_bfloat16 *>(a.k_new);
+    const __nv_bfloat16 *v = reinterpret_cast<const __nv_bfloat16 *>(a.v_new);
+    __nv_bfloat16 *qr = reinterpret_cast<__nv_bfloat16 *>(a.q_rot);
+    const int heads = a.H + 2 * a.Hkv;         // query rows, key rows, value rows
+    for (int row = warp; row < ntok * heads; row += kThreads / 32) {
+        const int t = row / heads, hh = row % heads;
+        const int64_t tok = tok0 + t;
+        const int64_t cache_row = a.prefix + tok;
+        if (hh >= a.H + a.Hkv) {
+            // ---- value row: elements 4 lane .. 4 lane + 3
+            const int g = hh - a.H - a.Hkv;
+            const uint2 w = *reinterpret_cast<const uint2 *>(v + (tok * a.Hkv + g) * d + 4 * lane);
+            const float x[4] = {bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y)};
+            int code[4];
+            float scale;
+            quantise4(x, code, scale);
+            const int64_t r = (int64_t)g * a.capacity + cache_row;
+            const uint32_t packed = (uint32_t)(code[0] & 0xFF) | ((uint32_t)(code[1] & 0xFF) << 8) |
+                                    ((uint32_t)(code[2] & 0xFF) << 16) | ((uint32_t)(code[3] & 0xFF) << 24);
+            *reinterpret_cast<uint32_t *>(qp.v_codes + r * d + 4 * lane) = packed;
+            if (lane == 0) qp.v_scales[r] = scale;
+            continue;
+        }
+        const bool is_q = hh < a.H;
+        const __nv_bfloat16 *src = is_q ? q + (tok * a.H + hh) * d : k + (tok * a.Hkv + (hh - a.H)) * d;
+        float x[4];
+        int e0, e1;     // where x[0..1] and x[2..3] sit in the row
+        if (!INTERLEAVED) {
+            // pairs (j, j + 64) for j = 2 lane, 2 lane + 1
+            e0 = 2 * lane; e1 = half + 2 * lane;
+            const uint32_t lo = *reinterpret_cast<const uint32_t *>(src + e0);
+            const uint32_t hi = *reinterpret_cast<const uint32_t *>(src + e1);
+            const float2 w0 = cs[t][2 * lane], w1 = cs[t][2 * lane + 1];
+            rotate(bf16_lo(lo), bf16_lo(hi), w0.x, w0.y, x[0], x[2]);
+            rotate(bf16_hi(lo), bf16_hi(hi), w1.x, w1.y, x[1], x[3]);
+        } else {
+            // pairs (2 j, 2 j + 1) for j = 2 lane, 2 lane + 1
+            e0 = 4 * lane; e1 = 4 * lane + 2;
+            const uint2 w = *reinterpret_cast<const uint2 *>(src + e0);
+            const float2 w0 = cs[t][2 * lane], w1 = cs[t][2 * lane + 1];
+            rotate(bf16_lo(w.x), bf16_hi(w.x), w0.x, w0.y, x[0], x[1]);
+            rotate(bf16_lo(w.y), bf16_hi(w.y), w1.x, w1.y, x[2], x[3]);
+        }
+        if (is_q) {
+            __nv_bfloat16 *dst = qr + (tok * a.H + hh) * d;
+            __nv_bfloat162 p0 = __floats2bfloat162_rn(x[0], x[1]), p1 = __floats2bfloat162_rn(x[2], x[3]);
+            *reinterpret_cast<__nv_bfloat162 *>(dst + e0) = p0;
+            *reinterpret_cast<__nv_bfloat162 *>(dst + e1) = p1;
+        } else {
+            const int g = hh - a.H;
+            int code[4];
+            float scale;
+            quantise4(x, code, scale);
+            const int64_t r = (int64_t)g * a.capacity + cache_row;
+            *reinterpret_cast<uint16_t *>(qp.k_codes + r * d + e0) = (uint16_t)((code[0] & 0xFF) | ((code[1] & 0xFF) << 8));
+            *reinterpret_cast<uint16_t *>(qp.k_codes + r * d + e1) = (uint16_t)((code[2] & 0xFF) | ((code[3] & 0xFF) << 8));
+            if (lane == 0) qp.k_scales[r] = scale;
+        }
+    }
+}
+
+// Stored rows [0, rows) of every KV head -> bf16 planes [Hkv][capacity][128]; value rows
+// [rows, rows + zero_rows) are cleared (the attention multiplies them by zero probabilities).
+// One thread per 16 codes.
+__global__ void __launch_bounds__(256) expand_q8_kernel(const QuantPlanes qp, __nv_bfloat16 *k_out, __nv_bfloat16 *v_out,
+                                                        int64_t capacity, int64_t rows, int32_t zero_rows, int32_t Hkv) {
+    constexpr int d = 128, vecs = d / 16;
+    const int64_t per_head = (rows + zero_rows) * vecs;
+    const int64_t total = 2 * (int64_t)Hkv * per_head;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int kv = (int)(i / ((int64_t)Hkv * per_head));
+        const int64_t rest = i % ((int64_t)Hkv * per_head);
+        const int g = (int)(rest / per_head);
+        const int64_t row = (rest % per_head) / vecs;
+        const int c = (int)(rest % vecs);
+        const int64_t r = (int64_t)g * capacity + row;
+        __nv_bfloat16 *dst = (kv ? v_out : k_out) + r * d + c * 16;
+        if (row >= rows) {
+            if (kv) {
+                reinterpret_cast<uint4 *>(dst)[0] = make_uint4(0, 0, 0, 0);
+                reinterpret_cast<uint4 *>(dst)[1] = make_uint4(0, 0, 0, 0);
+            }
+            continue;
+        }
+        const uint4 w = *reinterpret_cast<const uint4 *>((kv ? qp.v_codes : qp.k_codes) + r * d + c * 16);
+        const float scale = (kv ? qp.v_scales : qp.k_scales)[r];
+        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+        uint32_t o[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float f0 = __fmul_rn((float)(int8_t)(words[j] & 0xFF), scale);
+            const float f1 = __fmul_rn((float)(int8_t)((words[j] >> 8) & 0xFF), scale);
+            const float f2 = __fmul_rn((float)(int8_t)((words[j] >> 16) & 0xFF), scale);
+            const float f3 = __fmul_rn((float)(int8_t)(words[j] >> 24), scale);
+            __nv_bfloat162 p0 = __floats2bfloat162_rn(f0, f1), p1 = __floats2bfloat162_rn(f2, f3);
+            o[2 * j] = *reinterpret_cast<uint32_t *>(&p0);
+            o[2 * j + 1] = *reinterpret_cast<uint32_t *>(&p1);
+        }
+        reinterpret_cast<uint4 *>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+        reinterpret_cast<uint4 *>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, cudaStream_t s) {
+    const int blocks = (a.n + kTok - 1) / kTok;
+    if (interleaved) return launch_pdl(rope_append_q8_kernel<true>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
+    return launch_pdl(rope_append_q8_kernel<false>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
+}
+
+cudaError_t launch_expand_q8(const QuantPlanes &qp, void *k_out, void *v_out, int64_t capacity, int64_t rows,
+                             int32_t zero_rows, int32_t Hkv, int sm_count, cudaStream_t s) {
+    const int64_t items = 2 * (int64_t)Hkv * (rows + zero_rows) * 8;
+    int64_t blocks = (items + 255) / 256;
+    const int64_t cap = (int64_t)sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    expand_q8_kernel<<<(unsigned)blocks, 256, 0, s>>>(qp, reinterpret_cast<__nv_bfloat16 *>(k_out),
+                                                      reinterpret_cast<__nv_bfloat16 *>(v_out), capacity, rows, zero_rows, Hkv);
+    return cudaGetLastError();
+}
+
+}  // namespace kvf

@@ -1,0 +1,94 @@
+"""int8 cache storage (KVF_CACHE_INT8): the stored codes and scales bit for bit against the oracle's
+round trip, and the fold against the oracle's quantised fold."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_12471_b200 import binding, workloads
+from tests.chain import TOL, to_f64
+
+pytestmark = pytest.mark.gpu
+
+W = workloads.Workload("quant_llama_bf16", 32, 8, 128, "bf16", 256, 2048, 500000.0)
+
+
+def quant_cache(total, max_chunk, flags=0):
+    cfg = binding.make_config(W.n_q_heads, W.n_kv_heads, W.head_dim, "bf16", total, max_chunk, rope_base=W.rope_base,
+                              flags=flags | binding.KVF_CACHE_INT8)
+    return cfg, binding.Cache(cfg)
+
+
+@pytest.mark.parametrize("flags", [0, binding.KVF_ROPE_INTERLEAVED], ids=["rotate_half", "interleaved"])
+def test_stored_codes_and_scales_are_the_oracles_round_trip(flags):
+    chunks = [256, 100, 1, 16, 300]
+    total = sum(chunks)
+    cfg, cache = quant_cache(total, max(chunks), flags)
+    assert binding.cache_storage_bytes(cfg) == 2 * W.n_kv_heads * total * (W.head_dim + 4)
+    tab = oracle.inv_freq(W.rope_base, W.head_dim)
+    t0 = 0
+    for t, n in enumerate(chunks):
+        q, k, v = workloads.chunk_inputs(W, 101, t, device="cuda", n_tokens=n)
+        cache.fold_step(q, k, v)
+        rot = oracle.rope_faithful(k.float().cpu().numpy(), t0, tab, interleaved=bool(flags))       # fp32, no bf16 rounding
+        kc, ks, _ = oracle.quant_rows_int8(rot)
+        vc, vs, _ = oracle.quant_rows_int8(v.float().cpu().numpy())
+        got_kc = cache.k_plane()[:, t0:t0 + n].cpu().numpy().astype(np.int32)                       # [Hkv, n, d]
+        got_vc = cache.v_plane()[:, t0:t0 + n].cpu().numpy().astype(np.int32)
+        assert np.array_equal(got_kc, np.transpose(kc, (1, 0, 2))), f"key codes, step {t}"
+        assert np.array_equal(got_vc, np.transpose(vc, (1, 0, 2))), f"value codes, step {t}"
+        assert np.array_equal(cache.scales(0)[:, t0:t0 + n].cpu().numpy().view(np.uint32), ks.T.copy().view(np.uint32))
+        assert np.array_equal(cache.scales(1)[:, t0:t0 + n].cpu().numpy().view(np.uint32), vs.T.copy().view(np.uint32))
+        t0 += n
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_OK
+
+
+def test_quantised_fold_matches_the_quantised_oracle():
+    chunks = [256, 256, 100, 1, 16, 300, 256, 1]
+    total = sum(chunks)
+    cfg, cache = quant_cache(total, max(chunks))
+    oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
+    oc.set_quant(8)
+    plain = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
+    worst, worst_lse, err_sq, ref_sq, dq_sq = 0.0, 0.0, 0.0, 0.0, 0.0
+    for t, n in enumerate(chunks):
+        q, k, v = workloads.chunk_inputs(W, 102, t, device="cuda", n_tokens=n)
+        lse = torch.empty((n, W.n_q_heads), dtype=torch.float32, device="cuda")
+        out = cache.fold_step(q, k, v, lse=lse)
+        rows = sorted({0, 1, n // 2, n - 1} & set(range(n)))
+        ref, ref_lse, _ = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows, want_stats=True)
+        unq = plain.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows)
+        got = to_f64(out[rows])
+        worst = max(worst, float(np.abs(got - ref).max()))
+        worst_lse = max(worst_lse, float(np.abs(to_f64(lse[rows]) - ref_lse).max()))
+        err_sq += float(((got - ref) ** 2).sum())
+        ref_sq += float((ref ** 2).sum())
+        dq_sq += float(((ref - unq) ** 2).sum())
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_OK and len(cache) == total
+    assert worst <= TOL["bf16"][0] and worst_lse <= 2e-2, (worst, worst_lse)
+    # the kernel's own error is well below what the quantisation itself moves the outputs by
+    assert err_sq < dq_sq, (err_sq, dq_sq)
+    print(f"int8 cache: max abs vs quantised oracle {worst:.2e}, rel rms {np.sqrt(err_sq / ref_sq):.2e}; "
+          f"quantisation moved the outputs by rel rms {np.sqrt(dq_sq / ref_sq):.2e}")
+
+
+def test_quantised_storage_rejects_what_it_does_not_cover():
+    lib = binding.load()
+    h = ctypes.c_void_p()
+    f32 = binding.make_config(32, 8, 128, "f32", 1024, 256, rope_base=5e5, flags=binding.KVF_CACHE_INT8)
+    assert binding.cache_storage_bytes(f32) == 0
+    assert lib.kvf_cache_create(ctypes.byref(f32), 256, 1 << 30, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_UNSUPPORTED
+    d64 = binding.make_config(4, 1, 64, "bf16", 1024, 256, flags=binding.KVF_CACHE_INT8)
+    assert lib.kvf_cache_create(ctypes.byref(d64), 256, 1 << 30, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_UNSUPPORTED
+    cfg = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5, flags=binding.KVF_CACHE_INT8)
+    buf = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    table = torch.zeros(8, dtype=torch.int32, device="cuda")
+    rc = lib.kvf_paged_cache_create(ctypes.byref(cfg), buf.data_ptr(), buf.numel(), 8, table.data_ptr(), buf.data_ptr(),
+                                    buf.numel(), ctypes.byref(h))
+    assert rc == binding.KVF_ERR_UNSUPPORTED
+    plain = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5)
+    assert binding.workspace_bytes(cfg) == binding.workspace_bytes(plain) + 2 * 8 * 1024 * 128 * 2   # the bf16 image
