@@ -58,8 +58,8 @@ enum {
                                   fp32 (keys: on the rotated row before any rounding to bf16), and the
                                   attention sees bf16(code * scale).  dtype KVF_BF16 and head_dim 128
                                   only (KVF_ERR_UNSUPPORTED otherwise, and for paged caches and
-                                  kvf_fold_step_static); the workspace then also holds a bf16 image of
-                                  one cache that every step re-expands from the codes */
+                                  kvf_fold_step_static); the attention kernel expands code tiles to bf16
+                                  tiles in shared memory, so a step reads d + 4 bytes per cached row */
 };
 
 /*

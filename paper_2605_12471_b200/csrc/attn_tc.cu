@@ -69,6 +69,15 @@ constexpr uint32_t kOffQ = 0;                         // 2 tiles
 constexpr uint32_t kOffKV = 2 * kTileBytes;           // kSlots tiles
 constexpr uint32_t kOffCtl = kOffKV + kSlots * kTileBytes;
 constexpr uint32_t kSmemBytes = kOffCtl + 512 + 1024; // + control block + alignment slack
+// int8 cache storage (kQuant): 512 threads (warps 12-15 expand code tiles to bf16 tiles), three
+// bf16 K/V slots, three 16 KiB slots of raw int8 tiles behind them
+constexpr int kThreadsQ8 = 512;
+constexpr int kSlotsQ8 = 3;
+constexpr int kRawSlots = 3;
+constexpr uint32_t kRawBytes = 128 * 128;             // a 128 x 128 int8 tile
+constexpr uint32_t kOffRawQ8 = kOffKV + kSlotsQ8 * kTileBytes;
+constexpr uint32_t kOffCtlQ8 = kOffRawQ8 + kRawSlots * kRawBytes;
+constexpr uint32_t kSmemBytesQ8 = kOffCtlQ8 + 512 + 1024;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;             // log2 units
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
@@ -78,14 +87,15 @@ constexpr uint32_t kSuspendHintNs = 20000;             // a waiting thread may s
 constexpr int kRingBars = 6;                  // 5 slots of the shared ring, or 2 x 3 slots of the per-stream rings
 enum { B_QFULL = 0, B_QEMPTY = 1, B_FULL0 = 2, B_EMPTY0 = B_FULL0 + kRingBars, B_SFULL0 = B_EMPTY0 + kRingBars,
        B_PA0 = B_SFULL0 + 2, B_PB0 = B_PA0 + 2, B_OFINAL0 = B_PB0 + 2, B_TURN0 = B_OFINAL0 + 2,
-       B_DRAIN0 = B_TURN0 + 8, B_COUNT = B_DRAIN0 + 2 };
+       B_DRAIN0 = B_TURN0 + 8, B_RAWFULL0 = B_DRAIN0 + 2, B_RAWEMPTY0 = B_RAWFULL0 + kRawSlots,
+       B_COUNT = B_RAWEMPTY0 + kRawSlots };
 
 struct Ctl {
-    unsigned long long bars[32];
+    unsigned long long bars[40];
     uint32_t tmem_base;
     int abort;
 };
-static_assert(B_COUNT <= 32, "control block holds 32 barriers");
+static_assert(B_COUNT <= 40, "control block holds 40 barriers");
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -257,15 +267,33 @@ __device__ __forceinline__ void exp_half(const uint32_t *v, uint32_t *p, float2 
     }
 }
 
+// Four codes (one 32-bit word, each byte already offset by 128) -> two packed bf16 pairs of
+// bf16(code * scale): byte i dropped into the mantissa of 2^23 gives 2^23 + code + 128 exactly.
+__device__ __forceinline__ void expand4(uint32_t x, float2 sc, uint32_t &lo, uint32_t &hi) {
+    const float2 off = make_float2(-8388736.f, -8388736.f);
+    float2 a = make_float2(__uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650)), __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651)));
+    float2 b = make_float2(__uint_as_float(__byte_perm(x, 0x4B000000u, 0x7652)), __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7653)));
+    a = __fmul2_rn(__fadd2_rn(a, off), sc);
+    b = __fmul2_rn(__fadd2_rn(b, off), sc);
+    lo = pack_bf16(a.x, a.y);
+    hi = pack_bf16(b.x, b.y);
+}
+
 // kWindow = false compiles the sink + window arithmetic out (launched whenever win_lo == 0).
-template <bool kWindow>
-__global__ void __launch_bounds__(kThreads, 1)
+// kQuant: map_k / map_v describe int8 code planes; the producer brings raw code tiles into their own
+// ring and warps 12-15 (one thread per key row) expand each to the swizzled bf16 tile the MMAs read,
+// value = bf16(code * row scale), which is what the FULL barriers then announce.
+template <bool kWindow, bool kQuant>
+__global__ void __launch_bounds__(kQuant ? kThreadsQ8 : kThreads, 1)
 attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v) {
+    constexpr int NS = kQuant ? kSlotsQ8 : kSlots;        // slots of the shared ring
+    constexpr int SR = kQuant ? 2 : 3;                     // slots of each stream's own ring
+    constexpr uint32_t offCtl = kQuant ? kOffCtlQ8 : kOffCtl;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    Ctl *ctl = reinterpret_cast<Ctl *>(smem_raw + (base - smem_u32(smem_raw)) + kOffCtl);
-    const uint32_t bar0 = base + kOffCtl;
+    Ctl *ctl = reinterpret_cast<Ctl *>(smem_raw + (base - smem_u32(smem_raw)) + offCtl);
+    const uint32_t bar0 = base + offCtl;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -306,7 +334,9 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     if (threadIdx.x == 0) {
         mbar_init(bar(B_QFULL), 1);
         mbar_init(bar(B_QEMPTY), tiles);                                  // both issuers read Q
-        for (int s = 0; s < kRingBars; ++s) { mbar_init(bar(B_FULL0 + s), 1); mbar_init(bar(B_EMPTY0 + s), streams == 2 ? 1 : tiles); }   // consumers of a K/V tile
+        for (int s = 0; s < kRingBars; ++s) { mbar_init(bar(B_FULL0 + s), kQuant ? 4 : 1); mbar_init(bar(B_EMPTY0 + s), streams == 2 ? 1 : tiles); }   // consumers of a K/V tile
+        if (kQuant)
+            for (int s = 0; s < kRawSlots; ++s) { mbar_init(bar(B_RAWFULL0 + s), 1); mbar_init(bar(B_RAWEMPTY0 + s), 4); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(B_SFULL0 + i), 1);
             mbar_init(bar(B_PA0 + i), 4);
@@ -332,14 +362,70 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     // K/V tile slots.  Two row tiles: one ring of 5 that both issuers walk in step.  Two streams:
     // each stream owns a ring of 3 (the sixth slot is the second Q tile, unused there), because a
     // parity wait is only sound for a thread that watches every use of its barrier in order.
-    auto slot_addr = [&](int sl) { return base + (sl < kSlots ? kOffKV + (uint32_t)sl * kTileBytes : kOffQ + kTileBytes); };
+    auto slot_addr = [&](int sl) { return base + (sl < NS ? kOffKV + (uint32_t)sl * kTileBytes : kOffQ + kTileBytes); };
 
-    if (warp >= 8) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+    if (kQuant && warp >= 12) {
+        // ------------------------------------------------------------------ int8 -> bf16 tile expansion
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+        const int t = (warp - 12) * 32 + lane;              // key row of the tile
+        const uint32_t sw = (uint32_t)(t & 7);
+        int tg = 0, rg = 0;
+        int rc[2] = {0, 0};
+        bool ok = true;
+        int kt0, ntiles;
+        for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
+            if (ntiles <= 0) continue;
+            for (int tt = 0; tt < 2 * ntiles; ++tt, ++tg, ++rg) {
+                int slot = tg % NS, use = tg / NS;
+                if (streams == 2) {
+                    const int st = (tt >> 1) & 1;
+                    slot = st * SR + rc[st] % SR;
+                    use = rc[st] / SR;
+                    ++rc[st];
+                }
+                const int r = rg % kRawSlots;
+                const int64_t key = (int64_t)wt.actual(kt0 + (tt >> 1)) * kRows + t;
+                // the row's scale comes straight from global memory, asked for before the waits
+                const float *scales = (tt & 1) ? a.v_scales : a.k_scales;
+                const float scale = key < a.capacity ? __ldg(scales + (int64_t)kvh * a.capacity + key) : 0.f;
+                ok = mbar_wait(bar(B_RAWFULL0 + r), (rg / kRawSlots) & 1, ctl, a.status);
+                if (ok) ok = mbar_wait(bar(B_EMPTY0 + slot), (use & 1) ^ 1, ctl, a.status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint32_t src = base + kOffRawQ8 + (uint32_t)r * kRawBytes + (uint32_t)t * 128u;
+                const uint32_t dst = slot_addr(slot) + (uint32_t)t * 128u;
+                const float2 sc = make_float2(scale, scale);
+#pragma unroll 2
+                for (uint32_t c = 0; c < 8; ++c) {
+                    uint32_t w0, w1, w2, w3;
+                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(src + ((c ^ sw) << 4)));
+                    uint32_t o[8];
+                    expand4(w0 ^ 0x80808080u, sc, o[0], o[1]);
+                    expand4(w1 ^ 0x80808080u, sc, o[2], o[3]);
+                    expand4(w2 ^ 0x80808080u, sc, o[4], o[5]);
+                    expand4(w3 ^ 0x80808080u, sc, o[6], o[7]);
+                    const uint32_t k0 = 2 * c, k1 = 2 * c + 1;     // 16-byte chunks of the bf16 row
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k0 >> 3) * kPanel + (((k0 & 7) ^ sw) << 4)),
+                                 "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k1 >> 3) * kPanel + (((k1 & 7) ^ sw) << 4)),
+                                 "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read through the async proxy
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(bar(B_FULL0 + slot));
+                    mbar_arrive(bar(B_RAWEMPTY0 + r));
+                }
+            }
+        }
+    } else if (warp >= 8) {
+        if (kQuant) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        else asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
         if (warp == 8 && lane == 0) {
             // ------------------------------------------------------------------ TMA producer
             int tg = 0, pc = 0;          // ring loads and pieces so far
             int rc[2] = {0, 0};          // loads so far into each stream's ring
+            int rg = 0;                  // int8 storage: loads so far into the ring of raw tiles
             int page = 0;                // paged cache: page of the key tile being loaded
             const int32_t *page_table = a.page_tables ? a.page_tables[cb] : a.page_table;
             const int qtok0 = cb * n;    // the caches' rotated chunks follow one another
@@ -356,18 +442,28 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                                     qtok0 + (row0 + i * kRows) / G);
                 ++pc;
                 for (int t = 0; t < 2 * ntiles; ++t, ++tg) {
-                    int slot = tg % kSlots, use = tg / kSlots;
+                    const CUtensorMap *m = (t & 1) ? &map_v : &map_k;
+                    const int ktile = wt.actual(kt0 + (t >> 1));
+                    const int key0 = ktile * kRows;
+                    if (kQuant) {
+                        // a raw code tile (128 rows of 128 bytes, 128-byte swizzle) into the next raw slot
+                        const int r = rg % kRawSlots;
+                        ok = mbar_wait(bar(B_RAWEMPTY0 + r), ((rg / kRawSlots) & 1) ^ 1, ctl, a.status);
+                        if (!ok) break;
+                        mbar_expect_tx(bar(B_RAWFULL0 + r), kRawBytes);
+                        tma_load_3d(base + kOffRawQ8 + (uint32_t)r * kRawBytes, m, bar(B_RAWFULL0 + r), 0, key0, kvh);
+                        ++rg;
+                        continue;
+                    }
+                    int slot = tg % NS, use = tg / NS;
                     if (streams == 2) {
                         const int st = (t >> 1) & 1;          // key tile j goes to stream j & 1
-                        slot = st * 3 + rc[st] % 3;
-                        use = rc[st] / 3;
+                        slot = st * SR + rc[st] % SR;
+                        use = rc[st] / SR;
                         ++rc[st];
                     }
                     ok = mbar_wait(bar(B_EMPTY0 + slot), (use & 1) ^ 1, ctl, a.status);
                     if (!ok) break;
-                    const CUtensorMap *m = (t & 1) ? &map_v : &map_k;
-                    const int ktile = wt.actual(kt0 + (t >> 1));
-                    const int key0 = ktile * kRows;
                     mbar_expect_tx(bar(B_FULL0 + slot), kTileBytes);
                     if (page_table) {
                         // paged cache: a key tile is one page; the maps are (d, row in page, KV head, page)
@@ -382,13 +478,16 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             }
             // do not leave while a copy may still be writing into this CTA's shared memory
             if (pc > 0) mbar_wait_drain(bar(B_QFULL), (pc - 1) & 1, a.status);
-            if (streams == 2) {
+            if (kQuant) {
+                for (int c = max(0, rg - kRawSlots); c < rg; ++c)
+                    mbar_wait_drain(bar(B_RAWFULL0 + c % kRawSlots), (c / kRawSlots) & 1, a.status);
+            } else if (streams == 2) {
                 for (int st = 0; st < 2; ++st)
-                    for (int c = max(0, rc[st] - 3); c < rc[st]; ++c)
-                        mbar_wait_drain(bar(B_FULL0 + st * 3 + c % 3), (c / 3) & 1, a.status);
+                    for (int c = max(0, rc[st] - SR); c < rc[st]; ++c)
+                        mbar_wait_drain(bar(B_FULL0 + st * SR + c % SR), (c / SR) & 1, a.status);
             } else {
-                for (int t = max(0, tg - kSlots); t < tg; ++t)
-                    mbar_wait_drain(bar(B_FULL0 + t % kSlots), (t / kSlots) & 1, a.status);
+                for (int t = max(0, tg - NS); t < tg; ++t)
+                    mbar_wait_drain(bar(B_FULL0 + t % NS), (t / NS) & 1, a.status);
             }
         } else if ((warp == 9 || (warp == 10 && tiles == 2)) && lane == 0) {
             // ------------------------------------------------------------------ MMA issuer of row tile i
@@ -420,8 +519,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             // load number -> slot and parity: shared ring (number counts every load) or my own ring
             // (number counts my loads: K of my m-th tile is 2m, its V 2m + 1)
             auto ring = [&](int num, int &slot, uint32_t &par) {
-                if (streams == 2) { slot = i * 3 + num % 3; par = (num / 3) & 1; }
-                else { slot = num % kSlots; par = (num / kSlots) & 1; }
+                if (streams == 2) { slot = i * SR + num % SR; par = (num / SR) & 1; }
+                else { slot = num % NS; par = (num / NS) & 1; }
             };
             int kt0, ntiles;
             for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
@@ -484,7 +583,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         }
     } else {
         // ------------------------------------------------------------------ softmax, one thread per row
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        if (kQuant) asm volatile("setmaxnreg.inc.sync.aligned.u32 192;");
+        else asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
         const int i = warp >> 2;                        // row tile
         const int r = (warp & 3) * 32 + lane;           // row in the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
@@ -791,11 +891,15 @@ int attn_tc_streams(int n, int G) { return n * G <= kRows ? 2 : 1; }
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
     static_assert(sizeof(Ctl) <= 512, "control block");
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
-    auto kernel = a.win_lo > 0 ? attn_tc_kernel<true> : attn_tc_kernel<false>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    static_assert(kSmemBytesQ8 <= 232448, "shared memory budget of one CTA (int8 storage)");
+    const bool quant = a.k_scales != nullptr;
+    auto kernel = quant ? (a.win_lo > 0 ? attn_tc_kernel<true, true> : attn_tc_kernel<false, true>)
+                        : (a.win_lo > 0 ? attn_tc_kernel<true, false> : attn_tc_kernel<false, false>);
+    const uint32_t smem = quant ? kSmemBytesQ8 : kSmemBytes;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, a.batch);
-    return launch_pdl(kernel, grid, dim3(kThreads), kSmemBytes, s, a, maps.q, maps.k, maps.v);
+    return launch_pdl(kernel, grid, dim3(quant ? kThreadsQ8 : kThreads), smem, s, a, maps.q, maps.k, maps.v);
 }
 
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s) {

@@ -49,7 +49,7 @@ kvf_status check_config(const kvf_config *c) {
 }
 
 struct Layout {
-    size_t status, q_rot, st_q, st_k, st_v, st_out, st_lse, part_o, part_lse, deq, total;
+    size_t status, q_rot, st_q, st_k, st_v, st_out, st_lse, part_o, part_lse, total;
 };
 
 Layout workspace_layout(const kvf_config *c) {
@@ -69,8 +69,6 @@ Layout workspace_layout(const kvf_config *c) {
     l.st_lse = off;   off = align_up(off + (size_t)c->max_chunk * c->n_q_heads * 4, 1024);
     l.part_o = off;   off = align_up(off + (size_t)kPartTokens * c->n_q_heads * c->head_dim * 4, 1024);
     l.part_lse = off; off = align_up(off + (size_t)kPartTokens * c->n_q_heads * 4, 1024);
-    l.deq = off;      // quantised storage: bf16 image of one cache (K plane, then V plane)
-    if (c->flags & KVF_CACHE_INT8) off = align_up(off + 2 * (size_t)c->n_kv_heads * (size_t)c->capacity * c->head_dim * 2, 1024);
     l.total = off;
     return l;
 }
@@ -220,9 +218,26 @@ kvf_status build_maps(kvf_cache *c) {
         return make_page_map(fn, &c->maps.v, c->storage + c->plane_bytes, d, f.n_kv_heads, (uint64_t)c->n_pool_pages,
                              page_bytes);
     }
-    // planes [Hkv][capacity][d]: one box = 128 rows of one head x 64 (quantised storage: the bf16 image)
-    char *kbase = c->quant ? c->workspace + c->lay.deq : c->storage;
-    char *vbase = c->quant ? kbase + (size_t)f.n_kv_heads * f.capacity * d * 2 : c->storage + c->plane_bytes;
+    if (c->quant) {
+        // int8 code planes [Hkv][capacity][128]: one box = 128 rows of one head x 128 bytes
+        for (int kv = 0; kv < 2; ++kv) {
+            cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)f.capacity, (cuuint64_t)f.n_kv_heads};
+            cuuint64_t strides[2] = {(cuuint64_t)d, (cuuint64_t)d * f.capacity};
+            cuuint32_t box[3] = {(cuuint32_t)d, (cuuint32_t)kKvTile, 1u};
+            cuuint32_t estr[3] = {1u, 1u, 1u};
+            CUresult r = fn(kv ? &c->maps.v : &c->maps.k, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, kv ? (void *)c->qp.v_codes : (void *)c->qp.k_codes,
+                            dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) {
+                snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled (int8 codes) failed with CUresult %d", (int)r);
+                return KVF_ERR_CUDA;
+            }
+        }
+        return KVF_OK;
+    }
+    // planes [Hkv][capacity][d]: one box = 128 rows of one head x 64
+    char *kbase = c->storage;
+    char *vbase = c->storage + c->plane_bytes;
     s = make_map(fn, &c->maps.k, kbase, (uint64_t)f.capacity, (uint64_t)f.n_kv_heads, row,
                  row * f.capacity, d, (uint32_t)kKvTile, 1u);
     if (s != KVF_OK) return s;
@@ -377,6 +392,8 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.page_table = c->page_table;
     aa.page_tables = nullptr; aa.part_rows = 0; aa.batch = 1; aa.prefixes = nullptr;
     aa.n_sink = c->n_sink; aa.win_lo = window_lo(c, P);
+    aa.k_scales = c->quant ? c->qp.k_scales : nullptr;
+    aa.v_scales = c->quant ? c->qp.v_scales : nullptr;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
     aa.splits = plan.tc ? 1 : plan.splits;
@@ -387,16 +404,9 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
 
     cudaError_t e;
     if (c->quant) {
-        // quantised storage: rotate + quantise + append, then the bf16 image of rows [0, L) that the
-        // attention kernel reads (its planes are in the workspace)
-        char *deq_k = c->workspace + c->lay.deq;
-        char *deq_v = deq_k + (size_t)f.n_kv_heads * f.capacity * f.head_dim * 2;
-        aa.k_plane = deq_k; aa.v_plane = deq_v;
+        // int8 storage: rotate + quantise + append (the attention kernel expands the code tiles itself)
         ProfScope ps(c, st, 0);
         e = launch_rope_append_q8(ra, c->qp, (f.flags & KVF_ROPE_INTERLEAVED) != 0, st);
-        if (e == cudaSuccess)
-            e = launch_expand_q8(c->qp, deq_k, deq_v, f.capacity, P + n, ra.zero_rows, f.n_kv_heads, c->sm_count, st);
-        c->launches++;
     } else {
         ProfScope ps(c, st, 0);
         e = launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, 1, st);
@@ -841,6 +851,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     aa.page_tables = tables; aa.part_rows = b->part_rows; aa.batch = B;
     aa.prefixes = ragged ? dev_prefixes : nullptr;
     aa.n_sink = c0->n_sink; aa.win_lo = window_lo(c0, P);
+    aa.k_scales = nullptr; aa.v_scales = nullptr;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c0->G; aa.d = f.head_dim;
     aa.splits = 1;

@@ -96,6 +96,8 @@ struct AttnArgs {
     int64_t part_rows;               // rows of the partial area per cache of a batch
     int32_t batch;                   // caches in the launch (1 = one cache)
     const int64_t *prefixes;         // ragged batch: device array of the caches' row counts, else null
+    const float *k_scales, *v_scales; // int8 storage: fp32 row scales [Hkv][capacity] (the tensor maps then describe
+                                     // the int8 code planes), else null
     // sink + window variant: of the rows before the chunk only those below n_sink or from win_lo on
     // are visible (win_lo = 0: all of them); see WindowTiles
     int32_t n_sink;
@@ -130,9 +132,6 @@ struct QuantPlanes {
     float *k_scales, *v_scales;
 };
 cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, cudaStream_t s);
-// stored rows [0, rows) -> bf16 planes [Hkv][capacity][128]; value rows [rows, rows + zero_rows) cleared
-cudaError_t launch_expand_q8(const QuantPlanes &qp, void *k_out, void *v_out, int64_t capacity, int64_t rows,
-                             int32_t zero_rows, int32_t Hkv, int sm_count, cudaStream_t s);
 
 cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interleaved, int batch, cudaStream_t s);
 cudaError_t launch_attn_simt(const AttnArgs &a, int dtype, cudaStream_t s, int *grid_out);

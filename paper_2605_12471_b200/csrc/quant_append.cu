@@ -1,4 +1,4 @@
-// Quantised cache storage: rotate + quantise + append, and the expansion of stored rows to bf16.
+// Quantised cache storage: rotate + quantise + append.
 //
 // The paper's Discussion perturbs the stored K/V by a round trip bf16 -> intN -> bf16 and leaves the
 // scheme open.  Here a stored row (one token of one KV head, d elements) is symmetric int8 with one
@@ -8,7 +8,8 @@
 //     value seen by the attention = bf16(code_j * scale)                   (fp32 product, one rounding)
 // For a key row x is the rotated row in fp32 (same operation order as the bf16 path, before any
 // rounding to bf16); a value row is quantised as given.  amax = 0 gives codes 0 and scale 0.
-// The cache then holds d + 4 bytes per row instead of 2 d.
+// The cache then holds d + 4 bytes per row instead of 2 d; the attention kernel expands code tiles to
+// bf16 tiles in shared memory.
 #include "kvfold_internal.h"
 
 namespace kvf {
@@ -62,6 +63,13 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
     }
     __syncthreads();
     pdl_wait();   // the table above needs nothing from earlier kernels; the writes below do
+
+    // Rows between the new end of the cache and the next key-tile boundary get value scale 0: the
+    // attention expands them to zeros whatever their codes are, so a zero probability never
+    // multiplies non-finite bits.
+    if (blockIdx.x == 0)
+        for (int i = threadIdx.x; i < a.zero_rows * a.Hkv; i += kThreads)
+            qp.v_scales[(int64_t)(i / a.zero_rows) * a.capacity + a.prefix + a.n + i % a.zero_rows] = 0.f;
 
     const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(a.q);
     const __nv_bfloat16 *k = reinterpret_cast<const __nv_bfloat16 *>(a.k_new);
@@ -125,66 +133,12 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
     }
 }
 
-// Stored rows [0, rows) of every KV head -> bf16 planes [Hkv][capacity][128]; value rows
-// [rows, rows + zero_rows) are cleared (the attention multiplies them by zero probabilities).
-// One thread per 16 codes.
-__global__ void __launch_bounds__(256) expand_q8_kernel(const QuantPlanes qp, __nv_bfloat16 *k_out, __nv_bfloat16 *v_out,
-                                                        int64_t capacity, int64_t rows, int32_t zero_rows, int32_t Hkv) {
-    constexpr int d = 128, vecs = d / 16;
-    const int64_t per_head = (rows + zero_rows) * vecs;
-    const int64_t total = 2 * (int64_t)Hkv * per_head;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int kv = (int)(i / ((int64_t)Hkv * per_head));
-        const int64_t rest = i % ((int64_t)Hkv * per_head);
-        const int g = (int)(rest / per_head);
-        const int64_t row = (rest % per_head) / vecs;
-        const int c = (int)(rest % vecs);
-        const int64_t r = (int64_t)g * capacity + row;
-        __nv_bfloat16 *dst = (kv ? v_out : k_out) + r * d + c * 16;
-        if (row >= rows) {
-            if (kv) {
-                reinterpret_cast<uint4 *>(dst)[0] = make_uint4(0, 0, 0, 0);
-                reinterpret_cast<uint4 *>(dst)[1] = make_uint4(0, 0, 0, 0);
-            }
-            continue;
-        }
-        const uint4 w = *reinterpret_cast<const uint4 *>((kv ? qp.v_codes : qp.k_codes) + r * d + c * 16);
-        const float scale = (kv ? qp.v_scales : qp.k_scales)[r];
-        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-        uint32_t o[8];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float f0 = __fmul_rn((float)(int8_t)(words[j] & 0xFF), scale);
-            const float f1 = __fmul_rn((float)(int8_t)((words[j] >> 8) & 0xFF), scale);
-            const float f2 = __fmul_rn((float)(int8_t)((words[j] >> 16) & 0xFF), scale);
-            const float f3 = __fmul_rn((float)(int8_t)(words[j] >> 24), scale);
-            __nv_bfloat162 p0 = __floats2bfloat162_rn(f0, f1), p1 = __floats2bfloat162_rn(f2, f3);
-            o[2 * j] = *reinterpret_cast<uint32_t *>(&p0);
-            o[2 * j + 1] = *reinterpret_cast<uint32_t *>(&p1);
-        }
-        reinterpret_cast<uint4 *>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
-        reinterpret_cast<uint4 *>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
-    }
-}
-
 }  // namespace
 
 cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, cudaStream_t s) {
     const int blocks = (a.n + kTok - 1) / kTok;
     if (interleaved) return launch_pdl(rope_append_q8_kernel<true>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
     return launch_pdl(rope_append_q8_kernel<false>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
-}
-
-cudaError_t launch_expand_q8(const QuantPlanes &qp, void *k_out, void *v_out, int64_t capacity, int64_t rows,
-                             int32_t zero_rows, int32_t Hkv, int sm_count, cudaStream_t s) {
-    const int64_t items = 2 * (int64_t)Hkv * (rows + zero_rows) * 8;
-    int64_t blocks = (items + 255) / 256;
-    const int64_t cap = (int64_t)sm_count * 16;
-    if (blocks > cap) blocks = cap;
-    if (blocks < 1) blocks = 1;
-    expand_q8_kernel<<<(unsigned)blocks, 256, 0, s>>>(qp, reinterpret_cast<__nv_bfloat16 *>(k_out),
-                                                      reinterpret_cast<__nv_bfloat16 *>(v_out), capacity, rows, zero_rows, Hkv);
-    return cudaGetLastError();
 }
 
 }  // namespace kvf

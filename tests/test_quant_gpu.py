@@ -91,4 +91,4 @@ def test_quantised_storage_rejects_what_it_does_not_cover():
                                     buf.numel(), ctypes.byref(h))
     assert rc == binding.KVF_ERR_UNSUPPORTED
     plain = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5)
-    assert binding.workspace_bytes(cfg) == binding.workspace_bytes(plain) + 2 * 8 * 1024 * 128 * 2   # the bf16 image
+    assert binding.workspace_bytes(cfg) == binding.workspace_bytes(plain)          # no bf16 image of the cache anywhere
