@@ -300,6 +300,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--force-simt", action="store_true")
     ap.add_argument("--paged", action="store_true", help="keep the cache in shuffled 128-token pages of a pool")
+    ap.add_argument("--cache-int8", action="store_true",
+                    help="store the cache as int8 codes + one fp32 scale per row (KVF_CACHE_INT8); byte counts in the "
+                         "output line then count 132 bytes per cached row instead of 256")
     ap.add_argument("--shard", default="sequences", choices=["sequences", "kv_heads"],
                     help="with --gpus N: one sequence per rank (weak scaling), or ONE sequence whose KV heads and "
                          "the query heads that read them are dealt to the ranks (strong scaling, no exchange)")
@@ -352,6 +355,8 @@ def main():
     H, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
     out = torch.empty_like(q)
     flags = binding.KVF_FORCE_SIMT if args.force_simt else 0
+    if args.cache_int8:
+        flags |= binding.KVF_CACHE_INT8
     if args.paged:
         cfg = binding.make_config(H, Hkv, d, w.dtype, T, max(C, 2048 if P0 else C), rope_base=w.rope_base, flags=flags)
         n_table = (T + 127) // 128
@@ -370,6 +375,9 @@ def main():
     if P0:
         fq, fk, fv = workloads.chunk_inputs(w.with_(chunk=2048), args.seed + 1, 0, sequence=seq + rank, device="cuda")
         fout = torch.empty_like(fq)
+
+    # bytes a step reads per cached token: K and V rows of every KV head (int8: d codes + one fp32 scale per row)
+    bytes_per_token = 2 * Hkv * (d + 4) if args.cache_int8 else w.cache_bytes_per_token()
 
     def visible(prefix):
         """Rows before a chunk that its queries see (all of them without a window)."""
@@ -461,7 +469,7 @@ def main():
         body(first, last)
         bms, bcnt = cache.profile_read()
         fl = sum(w.flops_step(visible(P0 + t * C), C) for t in range(first, last))
-        by = sum(visible(P0 + t * C) + C for t in range(first, last)) * w.cache_bytes_per_token()
+        by = sum(visible(P0 + t * C) + C for t in range(first, last)) * bytes_per_token
         curve.append({"prefix_from": P0 + first * C, "prefix_to": P0 + (last - 1) * C,
                       "step_us": 1e3 * sum(bms) / (last - first), "attention_us": 1e3 * bms[1] / (last - first),
                       "attention_tflops": fl / (bms[1] * 1e-3) / 1e12, "cache_read_gbs": by / (bms[1] * 1e-3) / 1e9})
@@ -472,10 +480,10 @@ def main():
     pk = peaks()
     attn_flops = sum(w.flops_step(visible(P0 + t * C), C) for t in range(N))
     attn_tflops = attn_flops / (kms[1] * 1e-3) / 1e12
-    cache_bytes_read = sum(visible(P0 + t * C) + C for t in range(N)) * w.cache_bytes_per_token()
+    cache_bytes_read = sum(visible(P0 + t * C) + C for t in range(N)) * bytes_per_token
     hbm_gbs = cache_bytes_read / (kms[1] * 1e-3) / 1e9
     traffic = None
-    if NCU_TRAFFIC_BYTES_PER_CACHE_BYTE is not None:
+    if NCU_TRAFFIC_BYTES_PER_CACHE_BYTE is not None and not args.cache_int8:
         traffic = NCU_TRAFFIC_BYTES_PER_CACHE_BYTE * cache_bytes_read / kcnt[1]
     # which roof binds: arithmetic intensity G*C FLOP per cache byte against the ridge of the measured peaks
     ridge = pk["bf16_tflops_sustained"] * 1e12 / (pk["hbm_gbs"] * 1e9)
@@ -540,6 +548,7 @@ def main():
             "config": {"workload": w.name, "shard": args.shard, "tokens": T, "chunk": C, "prefill": P0, "fold_steps_per_step": N,
                        "n_q_heads": H, "n_kv_heads": Hkv, "head_dim": d, "rope_base": w.rope_base,
                        "sequences_per_gpu": 1, "paged": bool(args.paged), "sinks": args.sinks, "window": args.window,
+                       "cache_storage": "int8 codes + fp32 row scales" if args.cache_int8 else w.dtype,
                        "launch": "per-step host launches" if graph is None else "one CUDA graph per chain, captured from the same calls", "l2": "inputs larger than L2 (cache grows to 512 MiB per chain)",
                        "last_step_plan": {"tensor_core": plan[0], "splits": plan[1], "ctas": plan[2]}},
             "attention_tflops": step_flops / (ms * 1e-3) / 1e12,

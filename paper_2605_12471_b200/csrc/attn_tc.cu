@@ -366,7 +366,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
 
     if (kQuant && warp >= 12) {
         // ------------------------------------------------------------------ int8 -> bf16 tile expansion
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
         const int t = (warp - 12) * 32 + lane;              // key row of the tile
         const uint32_t sw = (uint32_t)(t & 7);
         int tg = 0, rg = 0;
@@ -395,15 +395,20 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 const uint32_t src = base + kOffRawQ8 + (uint32_t)r * kRawBytes + (uint32_t)t * 128u;
                 const uint32_t dst = slot_addr(slot) + (uint32_t)t * 128u;
                 const float2 sc = make_float2(scale, scale);
-#pragma unroll 2
+                // all eight 16-byte chunks of the code row first, then the arithmetic: the chunks are
+                // independent, which is what gives one thread enough work in flight
+                uint32_t w[32];
+#pragma unroll
+                for (uint32_t c = 0; c < 8; ++c)
+                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3]) : "r"(src + ((c ^ sw) << 4)));
+#pragma unroll
                 for (uint32_t c = 0; c < 8; ++c) {
-                    uint32_t w0, w1, w2, w3;
-                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(src + ((c ^ sw) << 4)));
                     uint32_t o[8];
-                    expand4(w0 ^ 0x80808080u, sc, o[0], o[1]);
-                    expand4(w1 ^ 0x80808080u, sc, o[2], o[3]);
-                    expand4(w2 ^ 0x80808080u, sc, o[4], o[5]);
-                    expand4(w3 ^ 0x80808080u, sc, o[6], o[7]);
+                    expand4(w[4 * c] ^ 0x80808080u, sc, o[0], o[1]);
+                    expand4(w[4 * c + 1] ^ 0x80808080u, sc, o[2], o[3]);
+                    expand4(w[4 * c + 2] ^ 0x80808080u, sc, o[4], o[5]);
+                    expand4(w[4 * c + 3] ^ 0x80808080u, sc, o[6], o[7]);
                     const uint32_t k0 = 2 * c, k1 = 2 * c + 1;     // 16-byte chunks of the bf16 row
                     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k0 >> 3) * kPanel + (((k0 & 7) ^ sw) << 4)),
                                  "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");

@@ -92,3 +92,54 @@ def test_quantised_storage_rejects_what_it_does_not_cover():
     assert rc == binding.KVF_ERR_UNSUPPORTED
     plain = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5)
     assert binding.workspace_bytes(cfg) == binding.workspace_bytes(plain)          # no bf16 image of the cache anywhere
+
+
+def test_quantised_fold_decode_steps_at_depth_and_forced_splits():
+    """Decode-shaped steps (two streams, rings of two slots) behind a 6 144-token prefix, then the same
+    cache with the key range cut three ways per KV head: sampled rows against the quantised oracle."""
+    prefix, steps = 6144, [1, 1, 8, 32, 1, 256, 100]
+    total = prefix + sum(steps)
+    cfg, cache = quant_cache(total, 2048)
+    oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
+    oc.set_quant(8)
+    for t in range(prefix // 2048):
+        q, k, v = workloads.chunk_inputs(W, 103, t, device="cuda", n_tokens=2048)
+        cache.fold_step(q, k, v)
+        oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=[])
+    worst = 0.0
+    for t, n in enumerate(steps):
+        if t == 4:
+            cache.set_splits(3)
+        q, k, v = workloads.chunk_inputs(W, 104, t, device="cuda", n_tokens=n)
+        out = cache.fold_step(q, k, v)
+        rows = sorted({0, n // 2, n - 1})
+        ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows)
+        worst = max(worst, float(np.abs(to_f64(out[rows]) - ref).max()))
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_OK, hex(cache.status_word())
+    assert worst <= TOL["bf16"][0], worst
+
+
+def test_quantised_fold_under_a_window_and_repeated_runs_give_the_same_bits():
+    chunks = [256] * 8 + [16, 1, 256]
+    total = sum(chunks)
+    runs = []
+    for rep in range(2):
+        cfg, cache = quant_cache(total, 256)
+        cache.set_window(4, 700)
+        oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
+        oc.set_quant(8)
+        oc.set_window(4, 700)
+        outs, worst = [], 0.0
+        for t, n in enumerate(chunks):
+            q, k, v = workloads.chunk_inputs(W, 105, t, device="cuda", n_tokens=n)
+            outs.append(cache.fold_step(q, k, v))               # no synchronisation between the steps
+            if rep == 0:
+                rows = sorted({0, n // 2, n - 1})
+                ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows)
+                worst = max(worst, float(np.abs(to_f64(outs[-1][rows]) - ref).max()))
+        torch.cuda.synchronize()
+        assert cache.status() == binding.KVF_OK, hex(cache.status_word())
+        assert worst <= TOL["bf16"][0], worst
+        runs.append(torch.cat(outs))
+    assert torch.equal(runs[0].view(torch.int16), runs[1].view(torch.int16))
