@@ -51,7 +51,8 @@ enum {
     KVF_FORCE_SIMT = 8u,       /* use the CUDA-core attention kernel even where the tensor-core
                                   kernel applies (bisecting aid; same results within tolerance) */
     KVF_CACHE_INT8 = 16u       /* store the cache as int8 codes with one fp32 scale per row (one token of
-                                  one KV head): d + 4 bytes per row instead of 2 d.  The paper's Discussion
+                                  one KV head): d + 4 bytes per row instead of 2 d (kvf_cache_storage_bytes
+                                  pads each head's scales to a multiple of 16 bytes).  The paper's Discussion
                                   perturbs the stored K/V by a round trip bf16 -> intN -> bf16 and leaves
                                   the scheme open; here a row is quantised once, when it is appended:
                                   scale = max|x| / 127, code = clamp(rint(x * (127 / max|x|)), +-127) in
@@ -181,7 +182,8 @@ kvf_status kvf_cache_status(kvf_cache *c);
 int32_t kvf_cache_status_word(kvf_cache *c);
 
 /* Device pointers of the planes, [n_kv_heads][capacity][head_dim] of dtype (int8 codes under
- * KVF_CACHE_INT8), and of the rows' fp32 scales [n_kv_heads][capacity] (NULL without that flag). */
+ * KVF_CACHE_INT8), and of the rows' fp32 scales (NULL without that flag): [n_kv_heads][stride] with
+ * stride = capacity rounded up to a multiple of 4, so that every head's scales start 16-byte aligned. */
 void *kvf_cache_k_plane(const kvf_cache *c);
 void *kvf_cache_v_plane(const kvf_cache *c);
 float *kvf_cache_k_scales(const kvf_cache *c);

@@ -260,8 +260,9 @@ class Cache:
         if not ptr:
             raise ValueError("this cache holds no scales")
         off = ptr - self.storage.data_ptr()
-        n = self.cfg.n_kv_heads * self.cfg.capacity
-        return self.storage[off:off + 4 * n].view(torch.float32).view(self.cfg.n_kv_heads, self.cfg.capacity)
+        stride = (self.cfg.capacity + 3) // 4 * 4               # each head's scales start 16-byte aligned
+        n = self.cfg.n_kv_heads * stride
+        return self.storage[off:off + 4 * n].view(torch.float32).view(self.cfg.n_kv_heads, stride)[:, :self.cfg.capacity]
 
     def k_plane(self) -> torch.Tensor:
         """[Hkv, capacity, d] view of the rotated keys (rows >= len are not content)."""

@@ -70,13 +70,14 @@ constexpr uint32_t kOffKV = 2 * kTileBytes;           // kSlots tiles
 constexpr uint32_t kOffCtl = kOffKV + kSlots * kTileBytes;
 constexpr uint32_t kSmemBytes = kOffCtl + 512 + 1024; // + control block + alignment slack
 // int8 cache storage (kQuant): 512 threads (warps 12-15 expand code tiles to bf16 tiles), three
-// bf16 K/V slots, three 16 KiB slots of raw int8 tiles behind them
+// bf16 K/V slots, three 16 KiB slots of raw int8 tiles (each with its 128 row scales) behind them
 constexpr int kThreadsQ8 = 512;
 constexpr int kSlotsQ8 = 3;
 constexpr int kRawSlots = 3;
 constexpr uint32_t kRawBytes = 128 * 128;             // a 128 x 128 int8 tile
 constexpr uint32_t kOffRawQ8 = kOffKV + kSlotsQ8 * kTileBytes;
-constexpr uint32_t kOffCtlQ8 = kOffRawQ8 + kRawSlots * kRawBytes;
+constexpr uint32_t kOffScaleQ8 = kOffRawQ8 + kRawSlots * kRawBytes;      // 128 fp32 row scales per raw slot
+constexpr uint32_t kOffCtlQ8 = (kOffScaleQ8 + kRawSlots * 512 + 1023) / 1024 * 1024;
 constexpr uint32_t kSmemBytesQ8 = kOffCtlQ8 + 512 + 1024;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;             // log2 units
@@ -176,6 +177,12 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
+// plain bulk copy global -> shared (both 16-byte aligned, size a multiple of 16)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -385,13 +392,14 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 }
                 const int r = rg % kRawSlots;
                 const int64_t key = (int64_t)wt.actual(kt0 + (tt >> 1)) * kRows + t;
-                // the row's scale comes straight from global memory, asked for before the waits
-                const float *scales = (tt & 1) ? a.v_scales : a.k_scales;
-                const float scale = key < a.capacity ? __ldg(scales + (int64_t)kvh * a.capacity + key) : 0.f;
                 ok = mbar_wait(bar(B_RAWFULL0 + r), (rg / kRawSlots) & 1, ctl, a.status);
                 if (ok) ok = mbar_wait(bar(B_EMPTY0 + slot), (use & 1) ^ 1, ctl, a.status);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                // the row's scale arrived with the tile (rows past the end of the planes were not copied)
+                float scale = 0.f;
+                if (key < a.capacity)
+                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(scale) : "r"(base + kOffScaleQ8 + (uint32_t)r * 512u + (uint32_t)t * 4u));
                 const uint32_t src = base + kOffRawQ8 + (uint32_t)r * kRawBytes + (uint32_t)t * 128u;
                 const uint32_t dst = slot_addr(slot) + (uint32_t)t * 128u;
                 const float2 sc = make_float2(scale, scale);
@@ -455,8 +463,13 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                         const int r = rg % kRawSlots;
                         ok = mbar_wait(bar(B_RAWEMPTY0 + r), ((rg / kRawSlots) & 1) ^ 1, ctl, a.status);
                         if (!ok) break;
-                        mbar_expect_tx(bar(B_RAWFULL0 + r), kRawBytes);
+                        // ... and the rows' scales behind it (as many as the plane still holds)
+                        const int64_t left = a.scale_stride - key0;
+                        const uint32_t sbytes = (uint32_t)(left < kRows ? left : kRows) * 4u;
+                        const float *scales = ((t & 1) ? a.v_scales : a.k_scales) + (int64_t)kvh * a.scale_stride + key0;
+                        mbar_expect_tx(bar(B_RAWFULL0 + r), kRawBytes + sbytes);
                         tma_load_3d(base + kOffRawQ8 + (uint32_t)r * kRawBytes, m, bar(B_RAWFULL0 + r), 0, key0, kvh);
+                        bulk_load(base + kOffScaleQ8 + (uint32_t)r * 512u, scales, sbytes, bar(B_RAWFULL0 + r));
                         ++rg;
                         continue;
                     }
@@ -597,6 +610,9 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         const uint32_t t_o = tmem + lane_addr + 256 + i * 128;
         const int R = row0 + (streams == 2 ? 0 : i * kRows) + r, tok = R / G, gi = R % G;
         const bool valid = tok < n;
+        // a warp none of whose 32 rows is a row of the chunk (decode-shaped steps: most warps) keeps
+        // every barrier protocol going but skips the loads, the arithmetic and the stores
+        const bool warp_live = __any_sync(0xffffffffu, valid);
         const int j0 = streams == 2 ? i : 0, jstep = streams;        // my key tiles of a piece
         // keys below `limit` are visible; a row past the chunk's end is never written, and each
         // row of S, P and O depends on that row alone, so such rows are left unmasked
@@ -654,6 +670,18 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
+                if (!warp_live) {
+                    if (tiles == 2) ok = take_turn(turn_base + k);
+                    if (!ok) break;
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(bar(B_PA0 + i));
+                        mbar_arrive(bar(B_PB0 + i));
+                        mbar_arrive(bar(B_TURN0 + (i == 0 ? 4 : 0) + (warp & 3)));
+                    }
+                    continue;
+                }
                 const int64_t key0 = (int64_t)wt.actual(kt0 + j) * kRows;
                 const int nvis = (int)max((int64_t)0, min((int64_t)kRows, limit - key0));
                 // a tile that starts before the window holds hidden columns (the sink tile, the window's first)
@@ -749,6 +777,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             if (!ok) break;
             ++oc;
             tc_fence_after();
+            if (!warp_live) continue;
             const float inv = l > 0.f ? 1.f / l : 0.f;
             const float lse2 = l > 0.f ? m_ref * sl2 + log2f(l) : -INFINITY;
             const int64_t row = ((int64_t)cb * n + tok) * a.H + kvh * G + gi;

@@ -394,6 +394,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.n_sink = c->n_sink; aa.win_lo = window_lo(c, P);
     aa.k_scales = c->quant ? c->qp.k_scales : nullptr;
     aa.v_scales = c->quant ? c->qp.v_scales : nullptr;
+    aa.scale_stride = c->qp.scale_stride;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
     aa.splits = plan.tc ? 1 : plan.splits;
@@ -447,8 +448,8 @@ extern "C" {
 
 size_t kvf_cache_storage_bytes(const kvf_config *cfg) {
     if (check_config(cfg) != KVF_OK) return 0;
-    if (cfg->flags & KVF_CACHE_INT8)   // codes and one fp32 scale per row, K and V
-        return 2 * (size_t)cfg->n_kv_heads * (size_t)cfg->capacity * ((size_t)cfg->head_dim + 4);
+    if (cfg->flags & KVF_CACHE_INT8)   // codes and one fp32 scale per row (rows of scales padded to 16 bytes), K and V
+        return 2 * (size_t)cfg->n_kv_heads * ((size_t)cfg->capacity * cfg->head_dim + align_up((size_t)cfg->capacity, 4) * 4);
     return 2 * (size_t)cfg->n_kv_heads * (size_t)cfg->capacity * (size_t)cfg->head_dim * elem_bytes(cfg->dtype);
 }
 
@@ -493,7 +494,8 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
         c->qp.k_codes = reinterpret_cast<int8_t *>(c->storage);
         c->qp.v_codes = c->qp.k_codes + codes;
         c->qp.k_scales = reinterpret_cast<float *>(c->storage + 2 * codes);
-        c->qp.v_scales = c->qp.k_scales + (size_t)cfg->n_kv_heads * cfg->capacity;
+        c->qp.scale_stride = (int64_t)align_up((size_t)cfg->capacity, 4);
+        c->qp.v_scales = c->qp.k_scales + (size_t)cfg->n_kv_heads * c->qp.scale_stride;
     }
     c->len = 0;
     c->G = cfg->n_q_heads / cfg->n_kv_heads;
@@ -851,7 +853,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     aa.page_tables = tables; aa.part_rows = b->part_rows; aa.batch = B;
     aa.prefixes = ragged ? dev_prefixes : nullptr;
     aa.n_sink = c0->n_sink; aa.win_lo = window_lo(c0, P);
-    aa.k_scales = nullptr; aa.v_scales = nullptr;
+    aa.k_scales = nullptr; aa.v_scales = nullptr; aa.scale_stride = 0;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c0->G; aa.d = f.head_dim;
     aa.splits = 1;

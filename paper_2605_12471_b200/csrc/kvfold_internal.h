@@ -96,8 +96,9 @@ struct AttnArgs {
     int64_t part_rows;               // rows of the partial area per cache of a batch
     int32_t batch;                   // caches in the launch (1 = one cache)
     const int64_t *prefixes;         // ragged batch: device array of the caches' row counts, else null
-    const float *k_scales, *v_scales; // int8 storage: fp32 row scales [Hkv][capacity] (the tensor maps then describe
-                                     // the int8 code planes), else null
+    const float *k_scales, *v_scales; // int8 storage: fp32 row scales [Hkv][scale_stride] (the tensor maps then
+                                     // describe the int8 code planes), else null
+    int64_t scale_stride;            // capacity rounded up to a multiple of 4 (16-byte aligned rows of scales)
     // sink + window variant: of the rows before the chunk only those below n_sink or from win_lo on
     // are visible (win_lo = 0: all of them); see WindowTiles
     int32_t n_sink;
@@ -126,10 +127,12 @@ struct WindowTiles {
 };
 constexpr int kMaxSinks = 64;         // sink rows sit in the first key tile of either kernel
 
-// Quantised storage: int8 codes [Hkv][capacity][d] and one fp32 scale per row [Hkv][capacity].
+// Quantised storage: int8 codes [Hkv][capacity][d] and one fp32 scale per row [Hkv][scale_stride],
+// scale_stride = capacity rounded up to a multiple of 4.
 struct QuantPlanes {
     int8_t *k_codes, *v_codes;
     float *k_scales, *v_scales;
+    int64_t scale_stride;
 };
 cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, cudaStream_t s);
 

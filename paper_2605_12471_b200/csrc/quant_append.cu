@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
     // multiplies non-finite bits.
     if (blockIdx.x == 0)
         for (int i = threadIdx.x; i < a.zero_rows * a.Hkv; i += kThreads)
-            qp.v_scales[(int64_t)(i / a.zero_rows) * a.capacity + a.prefix + a.n + i % a.zero_rows] = 0.f;
+            qp.v_scales[(int64_t)(i / a.zero_rows) * qp.scale_stride + a.prefix + a.n + i % a.zero_rows] = 0.f;
 
     const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(a.q);
     const __nv_bfloat16 *k = reinterpret_cast<const __nv_bfloat16 *>(a.k_new);
@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
             const uint32_t packed = (uint32_t)(code[0] & 0xFF) | ((uint32_t)(code[1] & 0xFF) << 8) |
                                     ((uint32_t)(code[2] & 0xFF) << 16) | ((uint32_t)(code[3] & 0xFF) << 24);
             *reinterpret_cast<uint32_t *>(qp.v_codes + r * d + 4 * lane) = packed;
-            if (lane == 0) qp.v_scales[r] = scale;
+            if (lane == 0) qp.v_scales[(int64_t)g * qp.scale_stride + cache_row] = scale;
             continue;
         }
         const bool is_q = hh < a.H;
@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
             const int64_t r = (int64_t)g * a.capacity + cache_row;
             *reinterpret_cast<uint16_t *>(qp.k_codes + r * d + e0) = (uint16_t)((code[0] & 0xFF) | ((code[1] & 0xFF) << 8));
             *reinterpret_cast<uint16_t *>(qp.k_codes + r * d + e1) = (uint16_t)((code[2] & 0xFF) | ((code[3] & 0xFF) << 8));
-            if (lane == 0) qp.k_scales[r] = scale;
+            if (lane == 0) qp.k_scales[(int64_t)g * qp.scale_stride + cache_row] = scale;
         }
     }
 }

@@ -26,7 +26,7 @@ def test_stored_codes_and_scales_are_the_oracles_round_trip(flags):
     chunks = [256, 100, 1, 16, 300]
     total = sum(chunks)
     cfg, cache = quant_cache(total, max(chunks), flags)
-    assert binding.cache_storage_bytes(cfg) == 2 * W.n_kv_heads * total * (W.head_dim + 4)
+    assert binding.cache_storage_bytes(cfg) == 2 * W.n_kv_heads * (total * W.head_dim + (total + 3) // 4 * 4 * 4)
     tab = oracle.inv_freq(W.rope_base, W.head_dim)
     t0 = 0
     for t, n in enumerate(chunks):
