@@ -354,7 +354,7 @@ def main():
         w = w.with_(n_q_heads=q.shape[1], n_kv_heads=k.shape[1])
     H, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
     out = torch.empty_like(q)
-    flags = binding.KVF_FORCE_SIMT if args.force_simt else 0
+    flags = (binding.KVF_FORCE_SIMT if args.force_simt else 0) | binding.KVF_HOST_UPLOAD_AHEAD   # the flag touches host steps only
     if args.cache_int8:
         flags |= binding.KVF_CACHE_INT8
     if args.paged:

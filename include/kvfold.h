@@ -50,6 +50,11 @@ enum {
     KVF_OUT_F32 = 4u,          /* `out` is fp32 even when dtype is bf16                          */
     KVF_FORCE_SIMT = 8u,       /* use the CUDA-core attention kernel even where the tensor-core
                                   kernel applies (bisecting aid; same results within tolerance) */
+    KVF_HOST_UPLOAD_AHEAD = 32u, /* kvf_fold_step_host copies a step's q/k/v to the device on a stream of the
+                                  library's own, into one of two staging sets, so that the upload of step
+                                  t+1 runs while step t computes (the call's stream waits for the upload;
+                                  results and errors are as without the flag).  Needs a workspace that no
+                                  other cache's host steps use at the same time */
     KVF_CACHE_INT8 = 16u       /* store the cache as int8 codes with one fp32 scale per row (one token of
                                   one KV head): d + 4 bytes per row instead of 2 d (kvf_cache_storage_bytes
                                   pads each head's scales to a multiple of 16 bytes).  The paper's Discussion
@@ -156,8 +161,9 @@ kvf_status kvf_fold_step(kvf_cache *c, const void *q, const void *k_new, const v
 
 /*
  * The same step with HOST buffers (pinned memory recommended): copies q/k/v to the workspace
- * staging area, runs the step, copies `out` (and lse if not NULL) back, all on `cuda_stream`.
- * The host buffers must stay valid until the stream reaches the end of the call.
+ * staging area, runs the step, copies `out` (and lse if not NULL) back, all on `cuda_stream`
+ * (with KVF_HOST_UPLOAD_AHEAD the three uploads run on an internal stream that `cuda_stream` then
+ * waits for).  The host buffers must stay valid until the stream reaches the end of the call.
  */
 kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_host,
                               const void *v_host, int32_t n_tokens, int64_t pos0, void *out_host,

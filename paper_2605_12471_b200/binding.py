@@ -18,6 +18,7 @@ KVF_OK, KVF_ERR_INVALID_ARG, KVF_ERR_CAPACITY, KVF_ERR_UNSUPPORTED, KVF_ERR_CUDA
     KVF_ERR_POS = range(7)
 KVF_BF16, KVF_F32 = 0, 1
 KVF_ROPE_INTERLEAVED, KVF_STRICT_POS, KVF_OUT_F32, KVF_FORCE_SIMT, KVF_CACHE_INT8 = 1, 2, 4, 8, 16
+KVF_HOST_UPLOAD_AHEAD = 32
 
 EXPORTS = [
     "kvf_cache_storage_bytes", "kvf_workspace_bytes", "kvf_cache_create", "kvf_fold_step",

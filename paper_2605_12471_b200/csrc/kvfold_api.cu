@@ -50,6 +50,7 @@ kvf_status check_config(const kvf_config *c) {
 
 struct Layout {
     size_t status, q_rot, st_q, st_k, st_v, st_out, st_lse, part_o, part_lse, total;
+    size_t st_q2, st_k2, st_v2;   // second staging set (KVF_HOST_UPLOAD_AHEAD)
 };
 
 Layout workspace_layout(const kvf_config *c) {
@@ -65,6 +66,12 @@ Layout workspace_layout(const kvf_config *c) {
     l.st_q = off;     off = align_up(off + qb, 1024);
     l.st_k = off;     off = align_up(off + kb, 1024);
     l.st_v = off;     off = align_up(off + kb, 1024);
+    l.st_q2 = l.st_k2 = l.st_v2 = 0;
+    if (c->flags & KVF_HOST_UPLOAD_AHEAD) {
+        l.st_q2 = off; off = align_up(off + qb, 1024);
+        l.st_k2 = off; off = align_up(off + kb, 1024);
+        l.st_v2 = off; off = align_up(off + kb, 1024);
+    }
     l.st_out = off;   off = align_up(off + ob, 1024);
     l.st_lse = off;   off = align_up(off + (size_t)c->max_chunk * c->n_q_heads * 4, 1024);
     l.part_o = off;   off = align_up(off + (size_t)kPartTokens * c->n_q_heads * c->head_dim * 4, 1024);
@@ -101,6 +108,11 @@ struct kvf_cache {
     const int32_t *page_table = nullptr;   // paged cache: device table, one page number per 128 tokens
     int64_t page_elems = 0;                // paged cache: elements per page
     int32_t n_pool_pages = 0;
+    // KVF_HOST_UPLOAD_AHEAD: the library's upload stream, "upload done" and "staging set read" events
+    cudaStream_t up_stream = nullptr;
+    cudaEvent_t ev_up[2] = {nullptr, nullptr}, ev_read[2] = {nullptr, nullptr};
+    bool ev_read_set[2] = {false, false};
+    uint64_t host_steps = 0;
     bool quant = false;                    // int8 storage: codes + scales in `storage`, bf16 image in the workspace
     QuantPlanes qp = {};
     int32_t n_sink = 0;                    // sink + window variant: rows always visible
@@ -433,6 +445,36 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     return KVF_OK;
 }
 
+// What every handle starts from: shape, device, buffers, rotation table, softmax scale, counters.
+kvf_status init_handle(kvf_cache *c, const kvf_config *cfg, void *storage, void *workspace) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+    c->cfg = *cfg;
+    c->cfg.inv_freq = nullptr;
+    c->device = dev;
+    c->sm_count = sms;
+    c->storage = static_cast<char *>(storage);
+    c->workspace = static_cast<char *>(workspace);
+    c->len = 0;
+    c->G = cfg->n_q_heads / cfg->n_kv_heads;
+    const double scale = cfg->softmax_scale > 0.0 ? cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
+    c->scale_log2 = (float)(scale * 1.4426950408889634);
+    for (int j = 0; j < cfg->head_dim / 2; ++j)
+        c->table.inv_freq[j] = cfg->inv_freq ? cfg->inv_freq[j]
+                                             : std::pow(cfg->rope_base, -2.0 * (double)j / (double)cfg->head_dim);
+    for (int j = cfg->head_dim / 2; j < kMaxHalfDim; ++j) c->table.inv_freq[j] = 0.0;
+    c->force_splits = 0;
+    c->part_rows_cap = (int64_t)kPartTokens * cfg->n_q_heads;
+    c->launches = 0;
+    c->profile = false;
+    c->tc = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, c->G);
+    return KVF_OK;
+}
+
 kvf_status check_step(kvf_cache *c, int32_t n, int64_t pos0) {
     if (!c) return KVF_ERR_INVALID_ARG;
     if (n < 1 || n > c->cfg.max_chunk) return KVF_ERR_INVALID_ARG;
@@ -470,21 +512,10 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
     if (storage_bytes < kvf_cache_storage_bytes(cfg)) return KVF_ERR_CAPACITY;
     if (workspace_bytes < kvf_workspace_bytes(cfg)) return KVF_ERR_CAPACITY;
 
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
-    int sms = 0;
-    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
-
     kvf_cache *c = new (std::nothrow) kvf_cache();
     if (!c) return KVF_ERR_INVALID_ARG;
-    c->cfg = *cfg;
-    c->cfg.inv_freq = nullptr;
-    c->device = dev;
-    c->sm_count = sms;
-    c->storage = static_cast<char *>(dev_storage);
-    c->workspace = static_cast<char *>(dev_workspace);
+    s = init_handle(c, cfg, dev_storage, dev_workspace);
+    if (s != KVF_OK) { delete c; return s; }
     c->plane_bytes = kvf_cache_storage_bytes(cfg) / 2;
     c->lay = workspace_layout(cfg);
     if (cfg->flags & KVF_CACHE_INT8) {
@@ -497,24 +528,11 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
         c->qp.scale_stride = (int64_t)align_up((size_t)cfg->capacity, 4);
         c->qp.v_scales = c->qp.k_scales + (size_t)cfg->n_kv_heads * c->qp.scale_stride;
     }
-    c->len = 0;
-    c->G = cfg->n_q_heads / cfg->n_kv_heads;
-    const double scale = cfg->softmax_scale > 0.0 ? cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
-    c->scale_log2 = (float)(scale * 1.4426950408889634);
-    for (int j = 0; j < cfg->head_dim / 2; ++j)
-        c->table.inv_freq[j] = cfg->inv_freq ? cfg->inv_freq[j]
-                                             : std::pow(cfg->rope_base, -2.0 * (double)j / (double)cfg->head_dim);
-    for (int j = cfg->head_dim / 2; j < kMaxHalfDim; ++j) c->table.inv_freq[j] = 0.0;
-    c->force_splits = 0;
-    c->part_rows_cap = (int64_t)kPartTokens * cfg->n_q_heads;
-    c->launches = 0;
-    c->profile = false;
-    c->tc = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, c->G);
     if (c->tc) {
         s = build_maps(c);
         if (s != KVF_OK) { delete c; return s; }
     }
-    e = cudaMemset(c->workspace + c->lay.status, 0, 256);
+    cudaError_t e = cudaMemset(c->workspace + c->lay.status, 0, 256);
     if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaMemset(status)"); }
     *out = c;
     return KVF_OK;
@@ -542,42 +560,18 @@ kvf_status kvf_paged_cache_create(const kvf_config *cfg, void *dev_pool, size_t 
     if (pool_bytes < kvf_paged_pool_bytes(cfg, n_pool_pages)) return KVF_ERR_CAPACITY;
     if (workspace_bytes < kvf_workspace_bytes(cfg)) return KVF_ERR_CAPACITY;
 
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
-    int sms = 0;
-    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
-
     kvf_cache *c = new (std::nothrow) kvf_cache();
     if (!c) return KVF_ERR_INVALID_ARG;
-    c->cfg = *cfg;
-    c->cfg.inv_freq = nullptr;
-    c->device = dev;
-    c->sm_count = sms;
-    c->storage = static_cast<char *>(dev_pool);
-    c->workspace = static_cast<char *>(dev_workspace);
+    s = init_handle(c, cfg, dev_pool, dev_workspace);
+    if (s != KVF_OK) { delete c; return s; }
     c->page_table = dev_page_table;
     c->n_pool_pages = n_pool_pages;
     c->page_elems = (int64_t)2 * cfg->n_kv_heads * kKvTile * cfg->head_dim;
     c->plane_bytes = (size_t)cfg->n_kv_heads * kKvTile * cfg->head_dim * elem_bytes(cfg->dtype);   // V block inside a page
     c->lay = workspace_layout(cfg);
-    c->len = 0;
-    c->G = G;
-    const double scale = cfg->softmax_scale > 0.0 ? cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
-    c->scale_log2 = (float)(scale * 1.4426950408889634);
-    for (int j = 0; j < cfg->head_dim / 2; ++j)
-        c->table.inv_freq[j] = cfg->inv_freq ? cfg->inv_freq[j]
-                                             : std::pow(cfg->rope_base, -2.0 * (double)j / (double)cfg->head_dim);
-    for (int j = cfg->head_dim / 2; j < kMaxHalfDim; ++j) c->table.inv_freq[j] = 0.0;
-    c->force_splits = 0;
-    c->part_rows_cap = (int64_t)kPartTokens * cfg->n_q_heads;
-    c->launches = 0;
-    c->profile = false;
-    c->tc = true;
     s = build_maps(c);
     if (s != KVF_OK) { delete c; return s; }
-    e = cudaMemset(c->workspace + c->lay.status, 0, 256);
+    cudaError_t e = cudaMemset(c->workspace + c->lay.status, 0, 256);
     if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaMemset(status)"); }
     *out = c;
     return KVF_OK;
@@ -605,14 +599,45 @@ kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_ho
     const size_t kb = (size_t)n_tokens * f.n_kv_heads * f.head_dim * eb;
     const size_t ob = (size_t)n_tokens * f.n_q_heads * f.head_dim * ((f.flags & KVF_OUT_F32) ? 4 : eb);
     char *w = c->workspace;
-    cudaError_t e = cudaMemcpyAsync(w + c->lay.st_q, q_host, qb, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(w + c->lay.st_k, k_host, kb, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(w + c->lay.st_v, v_host, kb, cudaMemcpyHostToDevice, st);
+    cudaError_t e = cudaSuccess;
+    size_t oq = c->lay.st_q, ok_ = c->lay.st_k, ov = c->lay.st_v;
+    int set = 0;
+    if (f.flags & KVF_HOST_UPLOAD_AHEAD) {
+        // upload on the library's stream into the staging set the step before last used: it runs
+        // while the previous step computes, and starts once that set's last reader (the rotate +
+        // append kernel of two steps ago, marked by ev_read) is done
+        if (!c->up_stream) {
+            e = cudaStreamCreateWithFlags(&c->up_stream, cudaStreamNonBlocking);
+            for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+                e = cudaEventCreateWithFlags(&c->ev_up[i], cudaEventDisableTiming);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_read[i], cudaEventDisableTiming);
+            }
+            if (e != cudaSuccess) return cuda_fail(e, "upload stream setup");
+        }
+        set = (int)(c->host_steps & 1);
+        if (set) { oq = c->lay.st_q2; ok_ = c->lay.st_k2; ov = c->lay.st_v2; }
+        cudaStream_t up = c->up_stream;
+        if (c->ev_read_set[set]) e = cudaStreamWaitEvent(up, c->ev_read[set], 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(w + oq, q_host, qb, cudaMemcpyHostToDevice, up);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(w + ok_, k_host, kb, cudaMemcpyHostToDevice, up);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(w + ov, v_host, kb, cudaMemcpyHostToDevice, up);
+        if (e == cudaSuccess) e = cudaEventRecord(c->ev_up[set], up);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_up[set], 0);
+    } else {
+        e = cudaMemcpyAsync(w + oq, q_host, qb, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(w + ok_, k_host, kb, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(w + ov, v_host, kb, cudaMemcpyHostToDevice, st);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "host-to-device copy");
     float *lse_dev = lse_host ? reinterpret_cast<float *>(w + c->lay.st_lse) : nullptr;
-    s = step_impl(c, w + c->lay.st_q, w + c->lay.st_k, w + c->lay.st_v, n_tokens, pos0, w + c->lay.st_out,
-                  lse_dev, st);
+    s = step_impl(c, w + oq, w + ok_, w + ov, n_tokens, pos0, w + c->lay.st_out, lse_dev, st);
     if (s != KVF_OK) return s;
+    if (f.flags & KVF_HOST_UPLOAD_AHEAD) {
+        e = cudaEventRecord(c->ev_read[set], st);      // (after the whole step: later than needed, never too early)
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+        c->ev_read_set[set] = true;
+        c->host_steps++;
+    }
     e = cudaMemcpyAsync(out_host, w + c->lay.st_out, ob, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && lse_host)
         e = cudaMemcpyAsync(lse_host, lse_dev, (size_t)n_tokens * f.n_q_heads * 4, cudaMemcpyDeviceToHost, st);
@@ -702,6 +727,11 @@ void kvf_cache_destroy(kvf_cache *c) {
     if (!c) return;
     for (ProfRec &r : c->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (cudaEvent_t e : c->pool) cudaEventDestroy(e);
+    for (int i = 0; i < 2; ++i) {
+        if (c->ev_up[i]) cudaEventDestroy(c->ev_up[i]);
+        if (c->ev_read[i]) cudaEventDestroy(c->ev_read[i]);
+    }
+    if (c->up_stream) cudaStreamDestroy(c->up_stream);
     delete c;
 }
 
@@ -1012,18 +1042,11 @@ extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_stor
     char *scratch = nullptr;
     s = static_scratch(dev, &scratch);
     if (s != KVF_OK) return s;
-    int sms = 0;
-    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
 
     // a handle on the stack that points the ordinary step at the static scratch
     kvf_cache c;
-    c.cfg = *cfg;
-    c.cfg.inv_freq = nullptr;
-    c.device = dev;
-    c.sm_count = sms;
-    c.storage = static_cast<char *>(dev_storage);
-    c.workspace = scratch;
+    s = init_handle(&c, cfg, dev_storage, scratch);
+    if (s != KVF_OK) return s;
     c.plane_bytes = kvf_cache_storage_bytes(cfg) / 2;
     c.lay = Layout();
     c.lay.status = 0;
@@ -1032,18 +1055,7 @@ extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_stor
     c.lay.part_lse = c.lay.part_o + kStaticPartOBytes;
     c.lay.total = kStaticScratchBytes;
     c.len = len;
-    c.G = cfg->n_q_heads / cfg->n_kv_heads;
-    const double scale = cfg->softmax_scale > 0.0 ? cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
-    c.scale_log2 = (float)(scale * 1.4426950408889634);
-    for (int j = 0; j < cfg->head_dim / 2; ++j)
-        c.table.inv_freq[j] = cfg->inv_freq ? cfg->inv_freq[j]
-                                            : std::pow(cfg->rope_base, -2.0 * (double)j / (double)cfg->head_dim);
-    for (int j = cfg->head_dim / 2; j < kMaxHalfDim; ++j) c.table.inv_freq[j] = 0.0;
-    c.force_splits = 0;
     c.part_rows_cap = (int64_t)part_tokens * cfg->n_q_heads;   // the plan splits only as far as this holds
-    c.launches = 0;
-    c.profile = false;
-    c.tc = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, c.G);
     if (c.tc) {
         s = build_maps(&c);
         if (s != KVF_OK) return s;

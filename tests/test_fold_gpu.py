@@ -282,10 +282,11 @@ def test_create_rejects_short_or_misaligned_buffers():
     lib.kvf_cache_destroy(h)
 
 
-def test_host_buffer_entry_point_matches_device_entry_point():
+@pytest.mark.parametrize("flags", [0, binding.KVF_HOST_UPLOAD_AHEAD], ids=["one_stream", "upload_ahead"])
+def test_host_buffer_entry_point_matches_device_entry_point(flags):
     w = SMALL_LLAMA
     a = binding.cache_for(w)
-    b = binding.cache_for(w)
+    b = binding.cache_for(w, flags=flags)
     for t in range(3):
         q, k, v = workloads.chunk_inputs(w, 17, t, device="cuda")
         want = a.fold_step(q, k, v)
@@ -400,3 +401,26 @@ def test_paged_cache_rejects_what_it_does_not_cover():
     rc = lib.kvf_paged_cache_create(ctypes.byref(cfg), buf.data_ptr(), buf.numel(), 8, table.data_ptr(), buf.data_ptr(),
                                     buf.numel(), ctypes.byref(h))
     assert rc == binding.KVF_ERR_CAPACITY                     # 8 pages need 4 MiB
+
+
+def test_host_steps_with_upload_ahead_enqueued_back_to_back():
+    """Eight host steps enqueued without any synchronisation in between (each upload overlaps the
+    step before it, the staging sets alternate): same bits as the device entry point."""
+    w = SMALL_LLAMA.with_(name="upload_ahead", tokens=2048)
+    dev = binding.cache_for(w)
+    host = binding.cache_for(w, flags=binding.KVF_HOST_UPLOAD_AHEAD)
+    want, got, keep = [], [], []
+    for t in range(8):
+        q, k, v = workloads.chunk_inputs(w, 19, t, device="cuda")
+        want.append(dev.fold_step(q, k, v))
+        qh, kh, vh = (x.cpu().pin_memory() for x in (q, k, v))
+        oh = torch.empty(q.shape, dtype=q.dtype).pin_memory()
+        keep.append((qh, kh, vh))
+        got.append(oh)
+    torch.cuda.synchronize()
+    for t in range(8):
+        host.fold_step_host(*keep[t], got[t])
+    torch.cuda.synchronize()
+    assert host.status() == binding.KVF_OK and len(host) == 2048
+    for t in range(8):
+        assert torch.equal(got[t].view(torch.int16), want[t].cpu().view(torch.int16)), t
