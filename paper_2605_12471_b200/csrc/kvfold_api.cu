@@ -292,6 +292,18 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
         } else if ((int64_t)pairs * Hkv * batch < c->sm_count) {
             groups = c->sm_count / (pairs * batch);
             if (groups > Hkv * nt / 4) groups = Hkv * nt / 4;
+        } else {
+            // whole KV heads fill the SMs, but the last wave may be half empty (256 CTAs on 148 SMs):
+            // cut a little finer - up to twice the KV heads - if that fills the waves at least 5 %
+            // better; the price is the partial results of one chunk and the combine kernel
+            auto fill = [&](int64_t g) {
+                const int64_t ctas = (int64_t)pairs * g * batch;
+                const int64_t waves = (ctas + c->sm_count - 1) / c->sm_count;
+                return (double)ctas / (double)(waves * c->sm_count);
+            };
+            double best = fill(Hkv) + 0.05;
+            for (int64_t g = Hkv + 1; g <= 2 * Hkv && g * 4 <= Hkv * nt; ++g)
+                if (fill(g) > best) { best = fill(g); groups = g; }
         }
         const int streams = attn_tc_streams(n, c->G);
         const int64_t slots_cap = part_rows_cap / ((int64_t)n * c->G) / streams;   // slots = streams * (groups + Hkv - 1)
