@@ -102,11 +102,13 @@ def test_quantised_fold_decode_steps_at_depth_and_forced_splits():
     cfg, cache = quant_cache(total, 2048)
     oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
     oc.set_quant(8)
+    worst = 0.0
     for t in range(prefix // 2048):
         q, k, v = workloads.chunk_inputs(W, 103, t, device="cuda", n_tokens=2048)
-        cache.fold_step(q, k, v)
-        oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=[])
-    worst = 0.0
+        out = cache.fold_step(q, k, v)                       # two row tiles, 32 row pairs, whole KV heads or 9 groups
+        rows = [0, 1023, 2047]
+        ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows)
+        worst = max(worst, float(np.abs(to_f64(out[rows]) - ref).max()))
     for t, n in enumerate(steps):
         if t == 4:
             cache.set_splits(3)
@@ -143,3 +145,27 @@ def test_quantised_fold_under_a_window_and_repeated_runs_give_the_same_bits():
         assert worst <= TOL["bf16"][0], worst
         runs.append(torch.cat(outs))
     assert torch.equal(runs[0].view(torch.int16), runs[1].view(torch.int16))
+
+
+def test_quantised_deep_chain_32k_sampled_steps():
+    """The benchmark's launch shape (C = 256, 148 CTAs, pieces that straddle KV heads) on an int8 cache,
+    128 steps deep; sampled steps and rows against the quantised oracle."""
+    C, N = 256, 128
+    cfg, cache = quant_cache(C * N, C)
+    oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, C * N, rope_base=W.rope_base)
+    oc.set_quant(8)
+    check = {0, 1, 2, 31, 64, 126, 127}
+    worst, err_sq, ref_sq = 0.0, 0.0, 0.0
+    for t in range(N):
+        q, k, v = workloads.chunk_inputs(W, 106, t, device="cuda", n_tokens=C)
+        out = cache.fold_step(q, k, v)
+        rows = [0, 100, 255] if t in check else []
+        ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows)
+        if rows:
+            got = to_f64(out[rows])
+            worst = max(worst, float(np.abs(got - ref).max()))
+            err_sq += float(((got - ref) ** 2).sum())
+            ref_sq += float((ref ** 2).sum())
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_OK, hex(cache.status_word())
+    assert worst <= TOL["bf16"][0] and (err_sq / ref_sq) ** 0.5 <= 2e-2, (worst, (err_sq / ref_sq) ** 0.5)
