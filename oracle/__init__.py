@@ -52,8 +52,8 @@ def _load():
     lib.okvf_cache_reset.restype = None
     lib.okvf_cache_set_quant.argtypes = [ctypes.c_void_p, ctypes.c_int]
     lib.okvf_cache_set_quant.restype = ctypes.c_int
-    lib.okvf_quant_row_int8.argtypes = [fp, ctypes.c_int, ip, fp, fp]
-    lib.okvf_quant_row_int8.restype = None
+    lib.okvf_quant_row.argtypes = [fp, ctypes.c_int, ctypes.c_int, ip, fp, fp]
+    lib.okvf_quant_row.restype = None
     lib.okvf_cache_set_window.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64]
     lib.okvf_cache_set_window.restype = None
     lib.okvf_cache_k.argtypes = [ctypes.c_void_p]
@@ -117,7 +117,12 @@ def rope_faithful(x, pos0: int, inv_freq_table, interleaved: bool = False,
 
 
 def quant_rows_int8(x):
-    """int8 round trip of the rows of x [..., d] (fp32): (codes int32, scales fp32 [...], stored fp32)."""
+    return quant_rows(x, 8)
+
+
+def quant_rows(x, bits: int):
+    """Round trip of the rows of x [..., d] (fp32) through int8 or int4 codes:
+    (codes int32, scales fp32 [...], stored fp32)."""
     x = np.ascontiguousarray(np.asarray(x, dtype=np.float32))
     d = x.shape[-1]
     flat = x.reshape(-1, d)
@@ -129,8 +134,8 @@ def quant_rows_int8(x):
     lib = _load()
     for r in range(flat.shape[0]):
         sc = ctypes.c_float()
-        lib.okvf_quant_row_int8(flat[r].ctypes.data_as(fp), d, codes[r].ctypes.data_as(ip), ctypes.byref(sc),
-                                stored[r].ctypes.data_as(fp))
+        lib.okvf_quant_row(flat[r].ctypes.data_as(fp), d, int(bits), codes[r].ctypes.data_as(ip), ctypes.byref(sc),
+                           stored[r].ctypes.data_as(fp))
         scales[r] = sc.value
     return codes.reshape(x.shape), scales.reshape(x.shape[:-1]), stored.reshape(x.shape)
 
@@ -167,9 +172,9 @@ class OracleCache:
         _load().okvf_cache_reset(self._h)
 
     def set_quant(self, bits: int):
-        """Quantised storage: rows go through an int8 round trip when appended (bits = 8; 0 = off)."""
+        """Quantised storage: rows go through an int8 / int4 round trip when appended (bits = 8 / 4; 0 = off)."""
         if _load().okvf_cache_set_quant(self._h, int(bits)) != 0:
-            raise ValueError("only 0 or 8 bits")
+            raise ValueError("only 0, 8 or 4 bits")
 
     def set_window(self, n_sink: int, window: int):
         """Sink + window variant: earlier chunks' rows are visible only if among the first n_sink

@@ -41,10 +41,11 @@
  * Reading taken here: symmetric int8 per stored row (one token of one KV head),
  * applied once, when the row is appended (a second round trip of an already
  * quantised row would return the same codes up to ties).  With
- * okvf_cache_set_quant(c, 8) a key row is rotated in fp32 (the dtype-faithful
- * operation order), then for the row x[0..d):
- *     amax = max |x_j|      inv = 127 / amax      scale = amax / 127
- *     code_j = clamp(rint(x_j * inv), -127, 127)  (all in fp32, ties to even)
+ * okvf_cache_set_quant(c, bits) (bits = 8 or 4, the two widths the paper
+ * reports) a key row is rotated in fp32 (the dtype-faithful operation order),
+ * then for the row x[0..d), with Q = 127 for int8 and Q = 7 for int4:
+ *     amax = max |x_j|      inv = Q / amax        scale = amax / Q
+ *     code_j = clamp(rint(x_j * inv), -Q, Q)      (all in fp32, ties to even)
  *     stored value = bf16(code_j * scale)         (fp32 product, then bf16)
  * and a value row goes through the same three lines unrotated; amax = 0 gives
  * codes 0 and scale 0.  The decision that produces an integer is taken in
@@ -74,7 +75,7 @@ typedef struct okvf_cache {
     int n_q_heads, n_kv_heads, head_dim, interleaved;
     int64_t capacity, len;
     int64_t n_sink, window; /* window <= 0: every earlier row is visible */
-    int quant_bits;         /* 0: rows are stored as given; 8: int8 round trip at append */
+    int quant_bits;         /* 0: rows are stored as given; 8 / 4: int8 / int4 round trip at append */
     double scale;
     double *inv_freq; /* [head_dim/2] */
     double *K;        /* [n_kv_heads][capacity][head_dim], rotated keys */
@@ -121,9 +122,9 @@ void okvf_cache_destroy(okvf_cache *c) {
 
 int64_t okvf_cache_len(const okvf_cache *c) { return c->len; }
 void okvf_cache_reset(okvf_cache *c) { c->len = 0; }
-/* Quantised storage (see the header): bits = 0 or 8.  Returns 0, or 1 for other values. */
+/* Quantised storage (see the header): bits = 0, 8 or 4.  Returns 0, or 1 for other values. */
 int okvf_cache_set_quant(okvf_cache *c, int bits) {
-    if (bits != 0 && bits != 8) return 1;
+    if (bits != 0 && bits != 8 && bits != 4) return 1;
     c->quant_bits = bits;
     return 0;
 }
@@ -210,25 +211,30 @@ void okvf_rope_faithful(const float *x, int64_t n, int heads, int d, int64_t pos
 }
 
 /*
- * int8 round trip of one row x[0..d) (fp32 in): codes (optional, int8 as int32), the row's scale and
- * the stored values y (the bf16 values, held in fp32).  See the header for the arithmetic.
+ * Round trip of one row x[0..d) (fp32 in) through `bits`-bit codes (8 or 4): codes (optional, as
+ * int32), the row's scale and the stored values y (the bf16 values, held in fp32).  See the header
+ * for the arithmetic.
  */
-void okvf_quant_row_int8(const float *x, int d, int32_t *codes, float *scale_out, float *y) {
+void okvf_quant_row(const float *x, int d, int bits, int32_t *codes, float *scale_out, float *y) {
+    const float Q = bits == 4 ? 7.0f : 127.0f;
     float amax = 0.0f;
     for (int j = 0; j < d; ++j) {
         float a = fabsf(x[j]);
         if (a > amax) amax = a;
     }
-    float inv = amax > 0.0f ? 127.0f / amax : 0.0f;
-    float scale = amax / 127.0f;
+    float inv = amax > 0.0f ? Q / amax : 0.0f;
+    float scale = amax / Q;
     for (int j = 0; j < d; ++j) {
         float r = rintf(x[j] * inv); /* default rounding mode: to nearest, ties to even */
-        if (r > 127.0f) r = 127.0f;
-        if (r < -127.0f) r = -127.0f;
+        if (r > Q) r = Q;
+        if (r < -Q) r = -Q;
         if (codes) codes[j] = (int32_t)r;
         if (y) y[j] = round_bf16(r * scale);
     }
     if (scale_out) *scale_out = scale;
+}
+void okvf_quant_row_int8(const float *x, int d, int32_t *codes, float *scale_out, float *y) {
+    okvf_quant_row(x, d, 8, codes, scale_out, y);
 }
 
 /*
@@ -260,17 +266,17 @@ int okvf_fold_step(okvf_cache *c, const double *q, const double *k_new, const do
         for (int g = 0; g < Hkv; ++g) {
             size_t dst = ((size_t)g * cap + (size_t)(P + i)) * d;
             size_t src = ((size_t)i * Hkv + g) * d;
-            if (c->quant_bits == 8) {
+            if (c->quant_bits != 0) {
                 /* the row as the library holds it: fp32 rotation in the faithful order, int8 round
-                 * trip, bf16; the value row likewise without the rotation */
+                 * or int4 round trip, bf16; the value row likewise without the rotation */
                 float xf[512], rot[512], st[512];
                 if (d > 512) return 1;
                 for (int e = 0; e < d; ++e) xf[e] = (float)k_new[src + e];
                 okvf_rope_faithful(xf, 1, 1, d, pos0 + i, c->inv_freq, c->interleaved, 0, rot);
-                okvf_quant_row_int8(rot, d, NULL, NULL, st);
+                okvf_quant_row(rot, d, c->quant_bits, NULL, NULL, st);
                 for (int e = 0; e < d; ++e) c->K[dst + e] = (double)st[e];
                 for (int e = 0; e < d; ++e) xf[e] = (float)v_new[src + e];
-                okvf_quant_row_int8(xf, d, NULL, NULL, st);
+                okvf_quant_row(xf, d, c->quant_bits, NULL, NULL, st);
                 for (int e = 0; e < d; ++e) c->V[dst + e] = (double)st[e];
                 continue;
             }

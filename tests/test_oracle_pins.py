@@ -287,21 +287,23 @@ def test_window_that_covers_everything_is_the_plain_fold_and_a_far_key_is_lost_o
 
 
 # ------------------------------------------------- quantised storage (int8 round trip)
-def test_int8_round_trip_is_round_to_nearest_on_a_grid_of_255_levels():
-    """What 'symmetric int8 per row, round to nearest' fixes without naming an implementation:
-    integer codes within +-127, the largest element at +-127, every stored value within half a
-    grid step of the input (plus the bf16 rounding of the stored value), zero rows stay zero."""
+@pytest.mark.parametrize("bits,Q", [(8, 127), (4, 7)])
+def test_int8_round_trip_is_round_to_nearest_on_a_grid_of_255_levels(bits, Q):
+    """What 'symmetric intN per row, round to nearest' fixes without naming an implementation:
+    integer codes within +-Q (127 for int8, 7 for int4), the largest element at +-Q, every stored value
+    within half a grid step of the input (plus the bf16 rounding of the stored value), zero rows stay zero."""
     rng = RNG(41)
     x = (rng.standard_normal((64, 128)) * rng.uniform(0.01, 30.0, size=(64, 1))).astype(np.float32)
     x[7] = 0.0
-    codes, scales, stored = oracle.quant_rows_int8(x)
-    assert codes.dtype == np.int32 and np.abs(codes).max() == 127 and np.abs(codes).min() >= 0
+    codes, scales, stored = oracle.quant_rows(x, bits)
+    assert codes.dtype == np.int32 and np.abs(codes).max() == Q and np.abs(codes).min() >= 0
+    assert len(np.unique(codes)) >= (15 if bits == 4 else 200)     # the grid is used, not a coarser one
     amax = np.abs(x).max(axis=1)
     big = np.abs(x).argmax(axis=1)
     rows = np.arange(64)
-    assert np.array_equal(np.abs(codes[rows, big])[amax > 0], np.full((amax > 0).sum(), 127))
+    assert np.array_equal(np.abs(codes[rows, big])[amax > 0], np.full((amax > 0).sum(), Q))
     assert np.array_equal(np.sign(codes[rows, big]), np.sign(x[rows, big]).astype(np.int32))
-    assert np.allclose(scales, amax / 127.0, rtol=2e-7, atol=0)
+    assert np.allclose(scales, amax / float(Q), rtol=2e-7, atol=0)
     step = scales[:, None].astype(np.float64)
     exact = codes * step                                           # the grid point, before the bf16 rounding
     assert (np.abs(exact - x) <= 0.5 * step * (1 + 1e-5) + 1e-30).all()        # nearest: never more than half a step
@@ -311,21 +313,23 @@ def test_int8_round_trip_is_round_to_nearest_on_a_grid_of_255_levels():
     assert (np.abs(exact - x) > 0.25 * step).any()
 
 
-def test_int8_round_trip_symmetries():
+@pytest.mark.parametrize("bits,Q", [(8, 127), (4, 7)])
+def test_int8_round_trip_symmetries(bits, Q):
     rng = RNG(42)
     x = rng.standard_normal((16, 64)).astype(np.float32)
-    c0, s0, y0 = oracle.quant_rows_int8(x)
-    c1, s1, y1 = oracle.quant_rows_int8(-x)
+    c0, s0, y0 = oracle.quant_rows(x, bits)
+    c1, s1, y1 = oracle.quant_rows(-x, bits)
     assert np.array_equal(c1, -c0) and np.array_equal(s1, s0) and np.array_equal(y1, -y0)
-    c2, s2, y2 = oracle.quant_rows_int8(x * np.float32(2.0 ** -5))       # a power of two moves the scale only
+    c2, s2, y2 = oracle.quant_rows(x * np.float32(2.0 ** -5), bits)      # a power of two moves the scale only
     assert np.array_equal(c2, c0) and np.array_equal(s2, s0 * np.float32(2.0 ** -5)) and np.array_equal(y2, y0 * np.float32(2.0 ** -5))
-    ints = rng.integers(-127, 128, size=(8, 32)).astype(np.float32)
-    ints[:, 0] = 127.0
-    c3, s3, y3 = oracle.quant_rows_int8(ints)                            # rows already on the grid come back as they are
+    ints = rng.integers(-Q, Q + 1, size=(8, 32)).astype(np.float32)
+    ints[:, 0] = float(Q)
+    c3, s3, y3 = oracle.quant_rows(ints, bits)                           # rows already on the grid come back as they are
     assert np.array_equal(c3, ints.astype(np.int32)) and np.all(s3 == 1.0) and np.array_equal(y3, ints)
 
 
-def test_quantised_fold_is_the_plain_fold_on_rows_that_went_through_the_round_trip():
+@pytest.mark.parametrize("bits,lo,hi", [(8, 1e-4, 3e-2), (4, 2e-2, 0.5)])
+def test_quantised_fold_is_the_plain_fold_on_rows_that_went_through_the_round_trip(bits, lo, hi):
     """The cache of the quantised oracle, fed to a brute-force causal pass as already-rotated keys,
     reproduces its outputs; and against the unquantised fold the outputs move by a few per cent at
     most (noise-like perturbation, the paper's Discussion)."""
@@ -334,14 +338,14 @@ def test_quantised_fold_is_the_plain_fold_on_rows_that_went_through_the_round_tr
     q, k, v = (a.astype(np.float32).astype(np.float64) for a in (q, k, v))
     plain, _, _ = _fold(q, k, v, [C] * (T // C), H, Hkv, d)
     c = oracle.OracleCache(H, Hkv, d, capacity=T)
-    c.set_quant(8)
+    c.set_quant(bits)
     outs = [c.fold_step(q[t:t + C], k[t:t + C], v[t:t + C]) for t in range(0, T, C)]
     got = np.concatenate(outs)
     # stored keys = round trip of the fp32 rotation, stored values = round trip of v
     tab = oracle.inv_freq(10000.0, d)
     rot = oracle.rope_faithful(k.astype(np.float32), 0, tab)
-    _, _, k_st = oracle.quant_rows_int8(rot)
-    _, _, v_st = oracle.quant_rows_int8(v.astype(np.float32))
+    _, _, k_st = oracle.quant_rows(rot, bits)
+    _, _, v_st = oracle.quant_rows(v.astype(np.float32), bits)
     assert np.array_equal(c.k(), np.transpose(k_st, (1, 0, 2)).astype(np.float64))
     assert np.array_equal(c.v(), np.transpose(v_st, (1, 0, 2)).astype(np.float64))
     qr = bf.rope_complex(q, np.arange(T), 10000.0)
@@ -354,7 +358,7 @@ def test_quantised_fold_is_the_plain_fold_on_rows_that_went_through_the_round_tr
         ref[:, h] = (p / p.sum(axis=1, keepdims=True)) @ v_st[:, h // G].astype(np.float64)
     assert np.abs(got - ref).max() <= 1e-12
     rel = np.sqrt(((got - plain) ** 2).sum() / (plain ** 2).sum())
-    assert 1e-4 < rel < 3e-2, rel
+    assert lo < rel < hi, rel                                 # int4 moves the outputs an order of magnitude more
 
 
 def test_append_only_prefix_rows_are_bit_unchanged():
