@@ -303,6 +303,7 @@ def main():
     ap.add_argument("--cache-int8", action="store_true",
                     help="store the cache as int8 codes + one fp32 scale per row (KVF_CACHE_INT8); byte counts in the "
                          "output line then count 132 bytes per cached row instead of 256")
+    ap.add_argument("--cache-int4", action="store_true", help="the same with 4-bit codes (68 bytes per cached row)")
     ap.add_argument("--shard", default="sequences", choices=["sequences", "kv_heads"],
                     help="with --gpus N: one sequence per rank (weak scaling), or ONE sequence whose KV heads and "
                          "the query heads that read them are dealt to the ranks (strong scaling, no exchange)")
@@ -357,6 +358,8 @@ def main():
     flags = (binding.KVF_FORCE_SIMT if args.force_simt else 0) | binding.KVF_HOST_UPLOAD_AHEAD   # the flag touches host steps only
     if args.cache_int8:
         flags |= binding.KVF_CACHE_INT8
+    if args.cache_int4:
+        flags |= binding.KVF_CACHE_INT4
     if args.paged:
         cfg = binding.make_config(H, Hkv, d, w.dtype, T, max(C, 2048 if P0 else C), rope_base=w.rope_base, flags=flags)
         n_table = (T + 127) // 128
@@ -377,7 +380,8 @@ def main():
         fout = torch.empty_like(fq)
 
     # bytes a step reads per cached token: K and V rows of every KV head (int8: d codes + one fp32 scale per row)
-    bytes_per_token = 2 * Hkv * (d + 4) if args.cache_int8 else w.cache_bytes_per_token()
+    bytes_per_token = (2 * Hkv * (d + 4) if args.cache_int8 else 2 * Hkv * (d // 2 + 4) if args.cache_int4
+                       else w.cache_bytes_per_token())
 
     def visible(prefix):
         """Rows before a chunk that its queries see (all of them without a window)."""
@@ -483,7 +487,7 @@ def main():
     cache_bytes_read = sum(visible(P0 + t * C) + C for t in range(N)) * bytes_per_token
     hbm_gbs = cache_bytes_read / (kms[1] * 1e-3) / 1e9
     traffic = None
-    if NCU_TRAFFIC_BYTES_PER_CACHE_BYTE is not None and not args.cache_int8:
+    if NCU_TRAFFIC_BYTES_PER_CACHE_BYTE is not None and not (args.cache_int8 or args.cache_int4):
         traffic = NCU_TRAFFIC_BYTES_PER_CACHE_BYTE * cache_bytes_read / kcnt[1]
     # which roof binds: arithmetic intensity G*C FLOP per cache byte against the ridge of the measured peaks
     ridge = pk["bf16_tflops_sustained"] * 1e12 / (pk["hbm_gbs"] * 1e9)
@@ -548,7 +552,8 @@ def main():
             "config": {"workload": w.name, "shard": args.shard, "tokens": T, "chunk": C, "prefill": P0, "fold_steps_per_step": N,
                        "n_q_heads": H, "n_kv_heads": Hkv, "head_dim": d, "rope_base": w.rope_base,
                        "sequences_per_gpu": 1, "paged": bool(args.paged), "sinks": args.sinks, "window": args.window,
-                       "cache_storage": "int8 codes + fp32 row scales" if args.cache_int8 else w.dtype,
+                       "cache_storage": ("int8 codes + fp32 row scales" if args.cache_int8 else
+                                         "int4 codes + fp32 row scales" if args.cache_int4 else w.dtype),
                        "launch": "per-step host launches" if graph is None else "one CUDA graph per chain, captured from the same calls", "l2": "inputs larger than L2 (cache grows to 512 MiB per chain)",
                        "last_step_plan": {"tensor_core": plan[0], "splits": plan[1], "ctas": plan[2]}},
             "attention_tflops": step_flops / (ms * 1e-3) / 1e12,

@@ -55,7 +55,7 @@ enum {
                                   t+1 runs while step t computes (the call's stream waits for the upload;
                                   results and errors are as without the flag).  Needs a workspace that no
                                   other cache's host steps use at the same time */
-    KVF_CACHE_INT8 = 16u       /* store the cache as int8 codes with one fp32 scale per row (one token of
+    KVF_CACHE_INT8 = 16u,      /* store the cache as int8 codes with one fp32 scale per row (one token of
                                   one KV head): d + 4 bytes per row instead of 2 d (kvf_cache_storage_bytes
                                   pads each head's scales to a multiple of 16 bytes).  The paper's Discussion
                                   perturbs the stored K/V by a round trip bf16 -> intN -> bf16 and leaves
@@ -66,6 +66,10 @@ enum {
                                   only (KVF_ERR_UNSUPPORTED otherwise, and for paged caches and
                                   kvf_fold_step_static); the attention kernel expands code tiles to bf16
                                   tiles in shared memory, so a step reads d + 4 bytes per cached row */
+    KVF_CACHE_INT4 = 64u       /* the same with 4-bit codes (the other width the paper reports): scale =
+                                  max|x| / 7, codes within +-7, stored two to a byte as code + 8 (element
+                                  2i in the low nibble of byte i): d / 2 + 4 bytes per row.  Not together
+                                  with KVF_CACHE_INT8 (KVF_ERR_INVALID_ARG) */
 };
 
 /*

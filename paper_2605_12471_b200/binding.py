@@ -18,7 +18,7 @@ KVF_OK, KVF_ERR_INVALID_ARG, KVF_ERR_CAPACITY, KVF_ERR_UNSUPPORTED, KVF_ERR_CUDA
     KVF_ERR_POS = range(7)
 KVF_BF16, KVF_F32 = 0, 1
 KVF_ROPE_INTERLEAVED, KVF_STRICT_POS, KVF_OUT_F32, KVF_FORCE_SIMT, KVF_CACHE_INT8 = 1, 2, 4, 8, 16
-KVF_HOST_UPLOAD_AHEAD = 32
+KVF_HOST_UPLOAD_AHEAD, KVF_CACHE_INT4 = 32, 64
 
 EXPORTS = [
     "kvf_cache_storage_bytes", "kvf_workspace_bytes", "kvf_cache_create", "kvf_fold_step",
@@ -250,6 +250,11 @@ class Cache:
         if self.cfg.flags & KVF_CACHE_INT8:                     # int8 codes
             n = shape[0] * shape[1] * shape[2]
             return self.storage[off:off + n].view(torch.int8).view(shape)
+        if self.cfg.flags & KVF_CACHE_INT4:                     # int4 codes, unpacked to int8 (a copy)
+            n = shape[0] * shape[1] * shape[2] // 2
+            packed = self.storage[off:off + n].view(shape[0], shape[1], shape[2] // 2).to(torch.int16)
+            codes = torch.stack([packed & 15, packed >> 4], dim=-1).view(shape) - 8     # element 2i = low nibble of byte i
+            return codes.to(torch.int8)
         plane_bytes = self.storage.numel() // 2
         flat = self.storage[off:off + plane_bytes].view(self.torch_dtype)
         return flat.view(shape)

@@ -286,17 +286,32 @@ __device__ __forceinline__ void expand4(uint32_t x, float2 sc, uint32_t &lo, uin
     hi = pack_bf16(b.x, b.y);
 }
 
+// Eight 4-bit codes (one 32-bit word, each nibble = code + 8, element 2i in the low nibble of byte i)
+// -> four packed bf16 pairs of bf16(code * scale), in element order.
+__device__ __forceinline__ void expand8(uint32_t w, float2 sc, uint32_t (&o)[4]) {
+    const float2 off = make_float2(-8388616.f, -8388616.f);      // 2^23 + 8
+    const uint32_t lo = w & 0x0F0F0F0Fu, hi = (w >> 4) & 0x0F0F0F0Fu;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float2 a = make_float2(__uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7650 + i)),
+                               __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7650 + i)));
+        a = __fmul2_rn(__fadd2_rn(a, off), sc);
+        o[i] = pack_bf16(a.x, a.y);
+    }
+}
+
 // kWindow = false compiles the sink + window arithmetic out (launched whenever win_lo == 0).
-// kQuant: map_k / map_v describe int8 code planes; the producer brings raw code tiles into their own
+// kQuant (0, 8 or 4 bits): map_k / map_v describe int8 or int4 code planes; the producer brings raw code tiles into their own
 // ring and warps 12-15 (one thread per key row) expand each to the swizzled bf16 tile the MMAs read,
 // value = bf16(code * row scale), which is what the FULL barriers then announce.
-template <bool kWindow, bool kQuant>
+template <bool kWindow, int kQuant>
 __global__ void __launch_bounds__(kQuant ? kThreadsQ8 : kThreads, 1)
 attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v) {
     constexpr int NS = kQuant ? kSlotsQ8 : kSlots;        // slots of the shared ring
     constexpr int SR = kQuant ? 2 : 3;                     // slots of each stream's own ring
     constexpr uint32_t offCtl = kQuant ? kOffCtlQ8 : kOffCtl;
+    constexpr uint32_t rawBytes = kQuant == 4 ? kRawBytes / 2 : kRawBytes;   // bytes of a 128-row code tile
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     Ctl *ctl = reinterpret_cast<Ctl *>(smem_raw + (base - smem_u32(smem_raw)) + offCtl);
@@ -400,28 +415,46 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 float scale = 0.f;
                 if (key < a.capacity)
                     asm volatile("ld.shared.f32 %0, [%1];" : "=f"(scale) : "r"(base + kOffScaleQ8 + (uint32_t)r * 512u + (uint32_t)t * 4u));
-                const uint32_t src = base + kOffRawQ8 + (uint32_t)r * kRawBytes + (uint32_t)t * 128u;
                 const uint32_t dst = slot_addr(slot) + (uint32_t)t * 128u;
                 const float2 sc = make_float2(scale, scale);
-                // all eight 16-byte chunks of the code row first, then the arithmetic: the chunks are
-                // independent, which is what gives one thread enough work in flight
-                uint32_t w[32];
+                if (kQuant == 4) {
+                    // 64-byte code rows, 64-byte swizzle: chunk c of row t sits at c ^ ((t >> 1) & 3)
+                    const uint32_t src = base + kOffRawQ8 + (uint32_t)r * kRawBytes + (uint32_t)t * 64u;
+                    const uint32_t sw4 = (uint32_t)((t >> 1) & 3);
+                    uint32_t w[16];
 #pragma unroll
-                for (uint32_t c = 0; c < 8; ++c)
-                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                                 : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3]) : "r"(src + ((c ^ sw) << 4)));
+                    for (uint32_t c = 0; c < 4; ++c)
+                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3]) : "r"(src + ((c ^ sw4) << 4)));
 #pragma unroll
-                for (uint32_t c = 0; c < 8; ++c) {
-                    uint32_t o[8];
-                    expand4(w[4 * c] ^ 0x80808080u, sc, o[0], o[1]);
-                    expand4(w[4 * c + 1] ^ 0x80808080u, sc, o[2], o[3]);
-                    expand4(w[4 * c + 2] ^ 0x80808080u, sc, o[4], o[5]);
-                    expand4(w[4 * c + 3] ^ 0x80808080u, sc, o[6], o[7]);
-                    const uint32_t k0 = 2 * c, k1 = 2 * c + 1;     // 16-byte chunks of the bf16 row
-                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k0 >> 3) * kPanel + (((k0 & 7) ^ sw) << 4)),
-                                 "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k1 >> 3) * kPanel + (((k1 & 7) ^ sw) << 4)),
-                                 "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+                    for (uint32_t k = 0; k < 16; ++k) {            // word k = codes 8k .. 8k+7 = bf16 chunk k of the row
+                        uint32_t o[4];
+                        expand8(w[k], sc, o);
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k >> 3) * kPanel + (((k & 7) ^ sw) << 4)),
+                                     "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+                    }
+                } else {
+                    const uint32_t src = base + kOffRawQ8 + (uint32_t)r * kRawBytes + (uint32_t)t * 128u;
+                    // all eight 16-byte chunks of the code row first, then the arithmetic: the chunks are
+                    // independent, which is what gives one thread enough work in flight
+                    uint32_t w[32];
+#pragma unroll
+                    for (uint32_t c = 0; c < 8; ++c)
+                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3]) : "r"(src + ((c ^ sw) << 4)));
+#pragma unroll
+                    for (uint32_t c = 0; c < 8; ++c) {
+                        uint32_t o[8];
+                        expand4(w[4 * c] ^ 0x80808080u, sc, o[0], o[1]);
+                        expand4(w[4 * c + 1] ^ 0x80808080u, sc, o[2], o[3]);
+                        expand4(w[4 * c + 2] ^ 0x80808080u, sc, o[4], o[5]);
+                        expand4(w[4 * c + 3] ^ 0x80808080u, sc, o[6], o[7]);
+                        const uint32_t k0 = 2 * c, k1 = 2 * c + 1;     // 16-byte chunks of the bf16 row
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k0 >> 3) * kPanel + (((k0 & 7) ^ sw) << 4)),
+                                     "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k1 >> 3) * kPanel + (((k1 & 7) ^ sw) << 4)),
+                                     "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+                    }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read through the async proxy
                 __syncwarp();
@@ -467,7 +500,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                         const int64_t left = a.scale_stride - key0;
                         const uint32_t sbytes = (uint32_t)(left < kRows ? left : kRows) * 4u;
                         const float *scales = ((t & 1) ? a.v_scales : a.k_scales) + (int64_t)kvh * a.scale_stride + key0;
-                        mbar_expect_tx(bar(B_RAWFULL0 + r), kRawBytes + sbytes);
+                        mbar_expect_tx(bar(B_RAWFULL0 + r), rawBytes + sbytes);
                         tma_load_3d(base + kOffRawQ8 + (uint32_t)r * kRawBytes, m, bar(B_RAWFULL0 + r), 0, key0, kvh);
                         bulk_load(base + kOffScaleQ8 + (uint32_t)r * 512u, scales, sbytes, bar(B_RAWFULL0 + r));
                         ++rg;
@@ -926,9 +959,10 @@ cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s
     static_assert(sizeof(Ctl) <= 512, "control block");
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
     static_assert(kSmemBytesQ8 <= 232448, "shared memory budget of one CTA (int8 storage)");
-    const bool quant = a.k_scales != nullptr;
-    auto kernel = quant ? (a.win_lo > 0 ? attn_tc_kernel<true, true> : attn_tc_kernel<false, true>)
-                        : (a.win_lo > 0 ? attn_tc_kernel<true, false> : attn_tc_kernel<false, false>);
+    const bool quant = a.quant_bits != 0;
+    auto kernel = a.quant_bits == 8 ? (a.win_lo > 0 ? attn_tc_kernel<true, 8> : attn_tc_kernel<false, 8>)
+                : a.quant_bits == 4 ? (a.win_lo > 0 ? attn_tc_kernel<true, 4> : attn_tc_kernel<false, 4>)
+                                    : (a.win_lo > 0 ? attn_tc_kernel<true, 0> : attn_tc_kernel<false, 0>);
     const uint32_t smem = quant ? kSmemBytesQ8 : kSmemBytes;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

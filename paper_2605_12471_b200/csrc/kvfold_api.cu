@@ -42,7 +42,8 @@ kvf_status check_config(const kvf_config *c) {
     if (c->softmax_scale < 0.0) return KVF_ERR_INVALID_ARG;
     if ((int64_t)c->max_chunk > c->capacity) return KVF_ERR_INVALID_ARG;
     if (c->capacity > (int64_t)1 << 31) return KVF_ERR_UNSUPPORTED;
-    if ((c->flags & KVF_CACHE_INT8) &&
+    if ((c->flags & KVF_CACHE_INT8) && (c->flags & KVF_CACHE_INT4)) return KVF_ERR_INVALID_ARG;
+    if ((c->flags & (KVF_CACHE_INT8 | KVF_CACHE_INT4)) &&
         (c->dtype != KVF_BF16 || (c->flags & KVF_FORCE_SIMT) || !attn_tc_supported(c->dtype, c->head_dim, G)))
         return KVF_ERR_UNSUPPORTED;
     return KVF_OK;
@@ -231,14 +232,17 @@ kvf_status build_maps(kvf_cache *c) {
                              page_bytes);
     }
     if (c->quant) {
-        // int8 code planes [Hkv][capacity][128]: one box = 128 rows of one head x 128 bytes
+        // code planes [Hkv][capacity][row bytes]: one box = 128 rows of one head x 128 (int8) or 64 (int4)
+        // bytes, swizzled over the row's 16-byte chunks
+        const cuuint64_t rb = (cuuint64_t)d * c->qp.bits / 8;
         for (int kv = 0; kv < 2; ++kv) {
-            cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)f.capacity, (cuuint64_t)f.n_kv_heads};
-            cuuint64_t strides[2] = {(cuuint64_t)d, (cuuint64_t)d * f.capacity};
-            cuuint32_t box[3] = {(cuuint32_t)d, (cuuint32_t)kKvTile, 1u};
+            cuuint64_t dims[3] = {rb, (cuuint64_t)f.capacity, (cuuint64_t)f.n_kv_heads};
+            cuuint64_t strides[2] = {rb, rb * f.capacity};
+            cuuint32_t box[3] = {(cuuint32_t)rb, (cuuint32_t)kKvTile, 1u};
             cuuint32_t estr[3] = {1u, 1u, 1u};
             CUresult r = fn(kv ? &c->maps.v : &c->maps.k, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, kv ? (void *)c->qp.v_codes : (void *)c->qp.k_codes,
-                            dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            c->qp.bits == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) {
                 snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled (int8 codes) failed with CUresult %d", (int)r);
@@ -419,6 +423,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.k_scales = c->quant ? c->qp.k_scales : nullptr;
     aa.v_scales = c->quant ? c->qp.v_scales : nullptr;
     aa.scale_stride = c->qp.scale_stride;
+    aa.quant_bits = c->quant ? c->qp.bits : 0;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
     aa.splits = plan.tc ? 1 : plan.splits;
@@ -502,8 +507,11 @@ extern "C" {
 
 size_t kvf_cache_storage_bytes(const kvf_config *cfg) {
     if (check_config(cfg) != KVF_OK) return 0;
-    if (cfg->flags & KVF_CACHE_INT8)   // codes and one fp32 scale per row (rows of scales padded to 16 bytes), K and V
-        return 2 * (size_t)cfg->n_kv_heads * ((size_t)cfg->capacity * cfg->head_dim + align_up((size_t)cfg->capacity, 4) * 4);
+    if (cfg->flags & (KVF_CACHE_INT8 | KVF_CACHE_INT4)) {
+        // codes and one fp32 scale per row (rows of scales padded to 16 bytes), K and V
+        const size_t row = (cfg->flags & KVF_CACHE_INT4) ? (size_t)cfg->head_dim / 2 : (size_t)cfg->head_dim;
+        return 2 * (size_t)cfg->n_kv_heads * ((size_t)cfg->capacity * row + align_up((size_t)cfg->capacity, 4) * 4);
+    }
     return 2 * (size_t)cfg->n_kv_heads * (size_t)cfg->capacity * (size_t)cfg->head_dim * elem_bytes(cfg->dtype);
 }
 
@@ -530,8 +538,9 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
     if (s != KVF_OK) { delete c; return s; }
     c->plane_bytes = kvf_cache_storage_bytes(cfg) / 2;
     c->lay = workspace_layout(cfg);
-    if (cfg->flags & KVF_CACHE_INT8) {
-        const size_t codes = (size_t)cfg->n_kv_heads * cfg->capacity * cfg->head_dim;
+    if (cfg->flags & (KVF_CACHE_INT8 | KVF_CACHE_INT4)) {
+        c->qp.bits = (cfg->flags & KVF_CACHE_INT4) ? 4 : 8;
+        const size_t codes = (size_t)cfg->n_kv_heads * cfg->capacity * cfg->head_dim * c->qp.bits / 8;
         c->quant = true;
         c->plane_bytes = codes;
         c->qp.k_codes = reinterpret_cast<int8_t *>(c->storage);
@@ -564,7 +573,7 @@ kvf_status kvf_paged_cache_create(const kvf_config *cfg, void *dev_pool, size_t 
     if (s != KVF_OK) return s;
     const int G = cfg->n_q_heads / cfg->n_kv_heads;
     if ((cfg->flags & KVF_FORCE_SIMT) || !attn_tc_supported(cfg->dtype, cfg->head_dim, G)) return KVF_ERR_UNSUPPORTED;
-    if (cfg->flags & KVF_CACHE_INT8) return KVF_ERR_UNSUPPORTED;          // pages hold bf16 rows
+    if (cfg->flags & (KVF_CACHE_INT8 | KVF_CACHE_INT4)) return KVF_ERR_UNSUPPORTED;   // pages hold bf16 rows
     if (!dev_pool || !dev_workspace || !dev_page_table || n_pool_pages <= 0) return KVF_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(dev_pool) & 255u) || (reinterpret_cast<uintptr_t>(dev_workspace) & 255u) ||
         (reinterpret_cast<uintptr_t>(dev_page_table) & 3u))
@@ -895,7 +904,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     aa.page_tables = tables; aa.part_rows = b->part_rows; aa.batch = B;
     aa.prefixes = ragged ? dev_prefixes : nullptr;
     aa.n_sink = c0->n_sink; aa.win_lo = window_lo(c0, P);
-    aa.k_scales = nullptr; aa.v_scales = nullptr; aa.scale_stride = 0;
+    aa.k_scales = nullptr; aa.v_scales = nullptr; aa.scale_stride = 0; aa.quant_bits = 0;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c0->G; aa.d = f.head_dim;
     aa.splits = 1;
@@ -1030,7 +1039,7 @@ extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_stor
                                            void *cuda_stream) {
     kvf_status s = check_config(cfg);
     if (s != KVF_OK) return s;
-    if (cfg->flags & KVF_CACHE_INT8) return KVF_ERR_UNSUPPORTED;          // the static scratch holds no bf16 image
+    if (cfg->flags & (KVF_CACHE_INT8 | KVF_CACHE_INT4)) return KVF_ERR_UNSUPPORTED;   // contiguous bf16 / fp32 planes only
     if (!dev_storage || (reinterpret_cast<uintptr_t>(dev_storage) & 255u)) return KVF_ERR_INVALID_ARG;
     if (storage_bytes < kvf_cache_storage_bytes(cfg)) return KVF_ERR_CAPACITY;
     if (len < 0 || n_tokens < 1 || n_tokens > cfg->max_chunk || pos0 < 0) return KVF_ERR_INVALID_ARG;

@@ -99,6 +99,7 @@ struct AttnArgs {
     const float *k_scales, *v_scales; // int8 storage: fp32 row scales [Hkv][scale_stride] (the tensor maps then
                                      // describe the int8 code planes), else null
     int64_t scale_stride;            // capacity rounded up to a multiple of 4 (16-byte aligned rows of scales)
+    int32_t quant_bits;              // 0, 8 or 4
     // sink + window variant: of the rows before the chunk only those below n_sink or from win_lo on
     // are visible (win_lo = 0: all of them); see WindowTiles
     int32_t n_sink;
@@ -130,9 +131,10 @@ constexpr int kMaxSinks = 64;         // sink rows sit in the first key tile of 
 // Quantised storage: int8 codes [Hkv][capacity][d] and one fp32 scale per row [Hkv][scale_stride],
 // scale_stride = capacity rounded up to a multiple of 4.
 struct QuantPlanes {
-    int8_t *k_codes, *v_codes;
+    int8_t *k_codes, *v_codes;       // int4: two codes to a byte (code + 8, element 2i in the low nibble of byte i)
     float *k_scales, *v_scales;
     int64_t scale_stride;
+    int32_t bits;                    // 8 or 4
 };
 cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, cudaStream_t s);
 

@@ -1,15 +1,16 @@
 // Quantised cache storage: rotate + quantise + append.
 //
 // The paper's Discussion perturbs the stored K/V by a round trip bf16 -> intN -> bf16 and leaves the
-// scheme open.  Here a stored row (one token of one KV head, d elements) is symmetric int8 with one
-// fp32 scale, decided once when the row is appended:
-//     amax = max |x_j|     inv = 127 / amax     scale = amax / 127        (fp32, round to nearest)
-//     code_j = clamp(rint(x_j * inv), -127, 127)                           (ties to even)
+// scheme open.  Here a stored row (one token of one KV head, d elements) is symmetric int8 (Q = 127)
+// or int4 (Q = 7) with one fp32 scale, decided once when the row is appended:
+//     amax = max |x_j|     inv = Q / amax       scale = amax / Q          (fp32, round to nearest)
+//     code_j = clamp(rint(x_j * inv), -Q, Q)                               (ties to even)
 //     value seen by the attention = bf16(code_j * scale)                   (fp32 product, one rounding)
 // For a key row x is the rotated row in fp32 (same operation order as the bf16 path, before any
 // rounding to bf16); a value row is quantised as given.  amax = 0 gives codes 0 and scale 0.
-// The cache then holds d + 4 bytes per row instead of 2 d; the attention kernel expands code tiles to
-// bf16 tiles in shared memory.
+// The cache then holds d + 4 (int8) or d / 2 + 4 (int4: code + 8, two to a byte, element 2i in the low
+// nibble of byte i) bytes per row instead of 2 d; the attention kernel expands code tiles to bf16 tiles
+// in shared memory.
 #include "kvfold_internal.h"
 
 namespace kvf {
@@ -29,24 +30,27 @@ __device__ __forceinline__ void rotate(float a, float b, float c, float s, float
 }
 
 // codes of four values of a row held by one lane; the row's scale comes back in `scale`
+template <int BITS>
 __device__ __forceinline__ void quantise4(const float (&x)[4], int (&code)[4], float &scale) {
+    constexpr float Q = BITS == 4 ? 7.f : 127.f;
     float amax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    const float inv = amax > 0.f ? __fdiv_rn(127.f, amax) : 0.f;
-    scale = __fdiv_rn(amax, 127.f);
+    const float inv = amax > 0.f ? __fdiv_rn(Q, amax) : 0.f;
+    scale = __fdiv_rn(amax, Q);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
         float r = rintf(__fmul_rn(x[e], inv));
-        r = fminf(fmaxf(r, -127.f), 127.f);
+        r = fminf(fmaxf(r, -Q), Q);
         code[e] = (int)r;
     }
 }
 
 // One warp per row (d = 128: four elements per lane).  Query rows are rotated and written as bf16;
 // key rows are rotated in fp32, quantised and appended; value rows are quantised and appended.
-template <bool INTERLEAVED>
+template <bool INTERLEAVED, int BITS>
 __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppendArgs a, const QuantPlanes qp) {
+    constexpr int RB = 128 * BITS / 8;          // bytes of a stored row
     __shared__ float2 cs[kTok][kMaxHalfDim];   // (cos, sin) per (token, pair)
     constexpr int d = 128, half = 64;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -87,11 +91,16 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
             const float x[4] = {bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y)};
             int code[4];
             float scale;
-            quantise4(x, code, scale);
+            quantise4<BITS>(x, code, scale);
             const int64_t r = (int64_t)g * a.capacity + cache_row;
-            const uint32_t packed = (uint32_t)(code[0] & 0xFF) | ((uint32_t)(code[1] & 0xFF) << 8) |
-                                    ((uint32_t)(code[2] & 0xFF) << 16) | ((uint32_t)(code[3] & 0xFF) << 24);
-            *reinterpret_cast<uint32_t *>(qp.v_codes + r * d + 4 * lane) = packed;
+            if (BITS == 8) {
+                const uint32_t packed = (uint32_t)(code[0] & 0xFF) | ((uint32_t)(code[1] & 0xFF) << 8) |
+                                        ((uint32_t)(code[2] & 0xFF) << 16) | ((uint32_t)(code[3] & 0xFF) << 24);
+                *reinterpret_cast<uint32_t *>(qp.v_codes + r * RB + 4 * lane) = packed;
+            } else {
+                *reinterpret_cast<uint16_t *>(qp.v_codes + r * RB + 2 * lane) =
+                    (uint16_t)((code[0] + 8) | ((code[1] + 8) << 4) | ((code[2] + 8) << 8) | ((code[3] + 8) << 12));
+            }
             if (lane == 0) qp.v_scales[(int64_t)g * qp.scale_stride + cache_row] = scale;
             continue;
         }
@@ -124,10 +133,16 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
             const int g = hh - a.H;
             int code[4];
             float scale;
-            quantise4(x, code, scale);
+            quantise4<BITS>(x, code, scale);
             const int64_t r = (int64_t)g * a.capacity + cache_row;
-            *reinterpret_cast<uint16_t *>(qp.k_codes + r * d + e0) = (uint16_t)((code[0] & 0xFF) | ((code[1] & 0xFF) << 8));
-            *reinterpret_cast<uint16_t *>(qp.k_codes + r * d + e1) = (uint16_t)((code[2] & 0xFF) | ((code[3] & 0xFF) << 8));
+            if (BITS == 8) {
+                *reinterpret_cast<uint16_t *>(qp.k_codes + r * RB + e0) = (uint16_t)((code[0] & 0xFF) | ((code[1] & 0xFF) << 8));
+                *reinterpret_cast<uint16_t *>(qp.k_codes + r * RB + e1) = (uint16_t)((code[2] & 0xFF) | ((code[3] & 0xFF) << 8));
+            } else {
+                // elements e0, e0 + 1 share byte e0 / 2 (e0 and e1 are even)
+                qp.k_codes[r * RB + e0 / 2] = (int8_t)((code[0] + 8) | ((code[1] + 8) << 4));
+                qp.k_codes[r * RB + e1 / 2] = (int8_t)((code[2] + 8) | ((code[3] + 8) << 4));
+            }
             if (lane == 0) qp.k_scales[(int64_t)g * qp.scale_stride + cache_row] = scale;
         }
     }
@@ -137,8 +152,12 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
 
 cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, cudaStream_t s) {
     const int blocks = (a.n + kTok - 1) / kTok;
-    if (interleaved) return launch_pdl(rope_append_q8_kernel<true>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
-    return launch_pdl(rope_append_q8_kernel<false>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
+    if (qp.bits == 4) {
+        if (interleaved) return launch_pdl(rope_append_q8_kernel<true, 4>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
+        return launch_pdl(rope_append_q8_kernel<false, 4>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
+    }
+    if (interleaved) return launch_pdl(rope_append_q8_kernel<true, 8>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
+    return launch_pdl(rope_append_q8_kernel<false, 8>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
 }
 
 }  // namespace kvf

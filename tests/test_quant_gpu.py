@@ -15,26 +15,30 @@ pytestmark = pytest.mark.gpu
 W = workloads.Workload("quant_llama_bf16", 32, 8, 128, "bf16", 256, 2048, 500000.0)
 
 
-def quant_cache(total, max_chunk, flags=0):
+def quant_cache(total, max_chunk, flags=0, bits=8):
     cfg = binding.make_config(W.n_q_heads, W.n_kv_heads, W.head_dim, "bf16", total, max_chunk, rope_base=W.rope_base,
-                              flags=flags | binding.KVF_CACHE_INT8)
+                              flags=flags | (binding.KVF_CACHE_INT4 if bits == 4 else binding.KVF_CACHE_INT8))
     return cfg, binding.Cache(cfg)
 
 
+BITS = pytest.mark.parametrize("bits", [8, 4], ids=["int8", "int4"])
+
+
+@BITS
 @pytest.mark.parametrize("flags", [0, binding.KVF_ROPE_INTERLEAVED], ids=["rotate_half", "interleaved"])
-def test_stored_codes_and_scales_are_the_oracles_round_trip(flags):
+def test_stored_codes_and_scales_are_the_oracles_round_trip(flags, bits):
     chunks = [256, 100, 1, 16, 300]
     total = sum(chunks)
-    cfg, cache = quant_cache(total, max(chunks), flags)
-    assert binding.cache_storage_bytes(cfg) == 2 * W.n_kv_heads * (total * W.head_dim + (total + 3) // 4 * 4 * 4)
+    cfg, cache = quant_cache(total, max(chunks), flags, bits)
+    assert binding.cache_storage_bytes(cfg) == 2 * W.n_kv_heads * (total * W.head_dim * bits // 8 + (total + 3) // 4 * 4 * 4)
     tab = oracle.inv_freq(W.rope_base, W.head_dim)
     t0 = 0
     for t, n in enumerate(chunks):
         q, k, v = workloads.chunk_inputs(W, 101, t, device="cuda", n_tokens=n)
         cache.fold_step(q, k, v)
         rot = oracle.rope_faithful(k.float().cpu().numpy(), t0, tab, interleaved=bool(flags))       # fp32, no bf16 rounding
-        kc, ks, _ = oracle.quant_rows_int8(rot)
-        vc, vs, _ = oracle.quant_rows_int8(v.float().cpu().numpy())
+        kc, ks, _ = oracle.quant_rows(rot, bits)
+        vc, vs, _ = oracle.quant_rows(v.float().cpu().numpy(), bits)
         got_kc = cache.k_plane()[:, t0:t0 + n].cpu().numpy().astype(np.int32)                       # [Hkv, n, d]
         got_vc = cache.v_plane()[:, t0:t0 + n].cpu().numpy().astype(np.int32)
         assert np.array_equal(got_kc, np.transpose(kc, (1, 0, 2))), f"key codes, step {t}"
@@ -46,12 +50,13 @@ def test_stored_codes_and_scales_are_the_oracles_round_trip(flags):
     assert cache.status() == binding.KVF_OK
 
 
-def test_quantised_fold_matches_the_quantised_oracle():
+@BITS
+def test_quantised_fold_matches_the_quantised_oracle(bits):
     chunks = [256, 256, 100, 1, 16, 300, 256, 1]
     total = sum(chunks)
-    cfg, cache = quant_cache(total, max(chunks))
+    cfg, cache = quant_cache(total, max(chunks), bits=bits)
     oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
-    oc.set_quant(8)
+    oc.set_quant(bits)
     plain = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
     worst, worst_lse, err_sq, ref_sq, dq_sq = 0.0, 0.0, 0.0, 0.0, 0.0
     for t, n in enumerate(chunks):
@@ -72,13 +77,15 @@ def test_quantised_fold_matches_the_quantised_oracle():
     assert worst <= TOL["bf16"][0] and worst_lse <= 2e-2, (worst, worst_lse)
     # the kernel's own error is well below what the quantisation itself moves the outputs by
     assert err_sq < dq_sq, (err_sq, dq_sq)
-    print(f"int8 cache: max abs vs quantised oracle {worst:.2e}, rel rms {np.sqrt(err_sq / ref_sq):.2e}; "
+    print(f"int{bits} cache: max abs vs quantised oracle {worst:.2e}, rel rms {np.sqrt(err_sq / ref_sq):.2e}; "
           f"quantisation moved the outputs by rel rms {np.sqrt(dq_sq / ref_sq):.2e}")
 
 
 def test_quantised_storage_rejects_what_it_does_not_cover():
     lib = binding.load()
     h = ctypes.c_void_p()
+    both = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5, flags=binding.KVF_CACHE_INT8 | binding.KVF_CACHE_INT4)
+    assert lib.kvf_cache_create(ctypes.byref(both), 256, 1 << 30, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_INVALID_ARG
     f32 = binding.make_config(32, 8, 128, "f32", 1024, 256, rope_base=5e5, flags=binding.KVF_CACHE_INT8)
     assert binding.cache_storage_bytes(f32) == 0
     assert lib.kvf_cache_create(ctypes.byref(f32), 256, 1 << 30, 256, 1 << 30, ctypes.byref(h)) == binding.KVF_ERR_UNSUPPORTED
@@ -94,14 +101,15 @@ def test_quantised_storage_rejects_what_it_does_not_cover():
     assert binding.workspace_bytes(cfg) == binding.workspace_bytes(plain)          # no bf16 image of the cache anywhere
 
 
-def test_quantised_fold_decode_steps_at_depth_and_forced_splits():
+@BITS
+def test_quantised_fold_decode_steps_at_depth_and_forced_splits(bits):
     """Decode-shaped steps (two streams, rings of two slots) behind a 6 144-token prefix, then the same
     cache with the key range cut three ways per KV head: sampled rows against the quantised oracle."""
     prefix, steps = 6144, [1, 1, 8, 32, 1, 256, 100]
     total = prefix + sum(steps)
-    cfg, cache = quant_cache(total, 2048)
+    cfg, cache = quant_cache(total, 2048, bits=bits)
     oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
-    oc.set_quant(8)
+    oc.set_quant(bits)
     worst = 0.0
     for t in range(prefix // 2048):
         q, k, v = workloads.chunk_inputs(W, 103, t, device="cuda", n_tokens=2048)
@@ -122,15 +130,16 @@ def test_quantised_fold_decode_steps_at_depth_and_forced_splits():
     assert worst <= TOL["bf16"][0], worst
 
 
-def test_quantised_fold_under_a_window_and_repeated_runs_give_the_same_bits():
+@BITS
+def test_quantised_fold_under_a_window_and_repeated_runs_give_the_same_bits(bits):
     chunks = [256] * 8 + [16, 1, 256]
     total = sum(chunks)
     runs = []
     for rep in range(2):
-        cfg, cache = quant_cache(total, 256)
+        cfg, cache = quant_cache(total, 256, bits=bits)
         cache.set_window(4, 700)
         oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
-        oc.set_quant(8)
+        oc.set_quant(bits)
         oc.set_window(4, 700)
         outs, worst = [], 0.0
         for t, n in enumerate(chunks):
@@ -147,13 +156,14 @@ def test_quantised_fold_under_a_window_and_repeated_runs_give_the_same_bits():
     assert torch.equal(runs[0].view(torch.int16), runs[1].view(torch.int16))
 
 
-def test_quantised_deep_chain_32k_sampled_steps():
+@BITS
+def test_quantised_deep_chain_32k_sampled_steps(bits):
     """The benchmark's launch shape (C = 256, 148 CTAs, pieces that straddle KV heads) on an int8 cache,
     128 steps deep; sampled steps and rows against the quantised oracle."""
     C, N = 256, 128
-    cfg, cache = quant_cache(C * N, C)
+    cfg, cache = quant_cache(C * N, C, bits=bits)
     oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, C * N, rope_base=W.rope_base)
-    oc.set_quant(8)
+    oc.set_quant(bits)
     check = {0, 1, 2, 31, 64, 126, 127}
     worst, err_sq, ref_sq = 0.0, 0.0, 0.0
     for t in range(N):
