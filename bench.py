@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # ncu capture summarised in profiles/attn_tc_kernel_chain_64k_c256_last_steps.md (65 536-token
 # chain; traffic grows in proportion to the cache rows read, so the ratio carries over).  Set to
 # None whenever attn_tc_kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_CACHE_BYTE = 1.031
+NCU_TRAFFIC_BYTES_PER_CACHE_BYTE = 1.033
 
 
 def peaks():
