@@ -424,3 +424,17 @@ def test_host_steps_with_upload_ahead_enqueued_back_to_back():
     assert host.status() == binding.KVF_OK and len(host) == 2048
     for t in range(8):
         assert torch.equal(got[t].view(torch.int16), want[t].cpu().view(torch.int16)), t
+
+
+def test_plan_fills_the_last_wave_when_whole_kv_heads_would_leave_it_half_empty():
+    """148 SMs: 32 row pairs x 8 KV heads = 256 CTAs is 1.73 waves, 32 x 9 groups = 288 is 1.95; 128 row
+    pairs x 8 = 1024 CTAs (6.9 waves) stays with whole KV heads and needs no combine kernel."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    cache = binding.cache_for(SMALL_LLAMA.with_(name="plan_probe", tokens=65536, chunk=8192), capacity=65536, max_chunk=8192)
+    tc, parts, ctas, kernels = cache.plan(2048, 61440)
+    if sms == 148:
+        assert (tc, ctas, kernels) == (1, 288, 3) and parts == 2
+    tc, parts, ctas, kernels = cache.plan(8192, 57344)
+    assert (tc, parts, ctas, kernels) == (1, 1, 128 * 8, 2)
+    tc, parts, ctas, kernels = cache.plan(256, 130816 - 65536)      # the benchmark's chunk: one CTA per SM
+    assert tc == 1 and ctas == (sms // 4) * 4 and kernels == 3
