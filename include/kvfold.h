@@ -15,7 +15,12 @@
  *   - Calls are stream-ordered and asynchronous: they enqueue work on `cuda_stream`
  *     (a cudaStream_t passed as void*, NULL = the default stream) and return.
  *   - Errors are return codes.  A call that returns an error has enqueued nothing and has
- *     changed neither the cache contents nor its length.  Nothing aborts or traps.
+ *     changed neither the cache contents nor its length.  Nothing aborts or traps.  The one
+ *     exception is KVF_ERR_CUDA from a fold step: the launch of one of the step's kernels was
+ *     refused by the runtime after an earlier kernel of the same step (and, for the host and the
+ *     static entry points, its copies or its memset) had been enqueued, so rows [len, len+n) of
+ *     the planes may have been written; the length is unchanged, and repeating the step rewrites
+ *     those rows.
  *   - A handle is not thread-safe; distinct handles are independent.  Several caches may
  *     share one workspace if all of their calls go to the same stream.
  *   - Results are deterministic: the same inputs, config and chunking give the same bits.
@@ -82,8 +87,8 @@ enum {
  *       and the rotated q/k are rounded once to bf16.  KVF_F32: fp32 throughout (CUDA cores).
  *   capacity: most tokens the cache will ever hold.
  *   max_chunk: largest n_tokens of any later kvf_fold_step (sizes the workspace).
- *   rope_base: theta = pos * rope_base^(-2j/d) (RoPE at continued absolute positions,
- *       Section 2, "Position identifiers for the new tokens are continued ...").
+ *   rope_base: theta = pos * rope_base^(-2j/d) (RoPE at the tokens' absolute positions, which
+ *       run on across chunk boundaries: Section 2, the paragraph that defines the one-step update).
  *   softmax_scale: 0 means 1/sqrt(d).
  *   inv_freq: optional HOST pointer to d/2 doubles replacing rope_base^(-2j/d)
  *       (frequency-scaled RoPE variants); copied at create, may be freed afterwards.
@@ -173,16 +178,20 @@ kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_ho
                               const void *v_host, int32_t n_tokens, int64_t pos0, void *out_host,
                               float *lse_host, void *cuda_stream);
 
-/* Tokens appended by all steps enqueued so far (host counter; after t steps of C tokens it is
- * t*C without any synchronisation).  -1 for a null handle. */
+/* Tokens appended by all steps enqueued so far: the size of the accumulator (K,V)^(t) of Section
+ * 2's left fold after t steps, which holds the rows of chunks 0..t (host counter; after t steps
+ * of C tokens it is t*C without any synchronisation).  -1 for a null handle. */
 int64_t kvf_cache_len(const kvf_cache *c);
 
-/* Back to the empty accumulator (len = 0).  Storage is not cleared. */
+/* Back to the empty accumulator the fold starts from (Section 2: the fold's initial value is the
+ * pair of empty K and V; also the start of every chunk under the paper's ISOLATED condition,
+ * Section 2, "Three reference conditions").  len = 0; storage is not cleared. */
 kvf_status kvf_cache_reset(kvf_cache *c);
 
 /* Reads the device status word (synchronises the default stream with a blocking copy): KVF_OK,
  * or KVF_ERR_TIMEOUT if a bounded wait inside a kernel gave up.  Call after synchronising the
- * streams that carried the steps. */
+ * streams that carried the steps.  (The paper has no counterpart: this reports on the kernels'
+ * own waits, not on anything the method computes.) */
 kvf_status kvf_cache_status(kvf_cache *c);
 
 /* The raw device status word behind kvf_cache_status (same synchronisation): 0, or for the first

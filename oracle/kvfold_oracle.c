@@ -233,9 +233,6 @@ void okvf_quant_row(const float *x, int d, int bits, int32_t *codes, float *scal
     }
     if (scale_out) *scale_out = scale;
 }
-void okvf_quant_row_int8(const float *x, int d, int32_t *codes, float *scale_out, float *y) {
-    okvf_quant_row(x, d, 8, codes, scale_out, y);
-}
 
 /*
  * One fold step.

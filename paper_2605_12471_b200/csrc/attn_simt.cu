@@ -271,7 +271,7 @@ template <typename T, int D>
 cudaError_t launch_simt_t(const AttnArgs &a, cudaStream_t s, int *grid_out) {
     constexpr size_t smem = sizeof(float) * (size_t)(BM * (D + 4) + BN * (D + 4) + BN * D);
     static_assert(BM * (BN + 4) <= BN * (D + 4), "probability tile must fit in the K tile");
-    cudaError_t e = cudaFuncSetAttribute(attn_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(attn_simt_kernel<T, D>), (int)smem);
     if (e != cudaSuccess) return e;
     dim3 grid((a.n * a.G + BM - 1) / BM, a.Hkv, a.splits);
     if (grid_out) *grid_out = grid.x * grid.y * grid.z;

@@ -53,7 +53,8 @@
 // the turn protocols below are all built to that rule.
 //
 // The kernel may be launched while the kernel before it in the stream is finishing (programmatic
-// dependent launch): everything up to pdl_wait() is private to the CTA.
+// dependent launch): everything up to pdl_wait() touches only launch arguments and the CTA's own
+// shared and tensor memory (a ragged batch, whose row counts live in device memory, waits first).
 #include "kvfold_internal.h"
 
 namespace kvf {
@@ -322,6 +323,9 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     const int qpair = blockIdx.x, group = blockIdx.y;
     const int cb = blockIdx.z;     // cache of a batch (0 when there is one cache)
     const int G = a.G, n = a.n;
+    // (a ragged batch keeps its members' row counts in device memory, written by an earlier kernel
+    // of the stream: those are the one thing read before the set-up below, so wait first there)
+    if (a.prefixes) pdl_wait();
     const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix, L = P + n;
     // streams == 2 (chunks of at most 128 / G tokens, i.e. one row tile): the two tile slots work on
     // the SAME 128 rows and take alternate key tiles, so that one stream's softmax still runs under
@@ -379,7 +383,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    pdl_wait();   // everything above is private to the CTA; from here on the rotated chunk is read
+    pdl_wait();   // nothing above reads what an earlier kernel wrote; from here on the rotated chunk is read
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&ctl->tmem_base);
     // K/V tile slots.  Two row tiles: one ring of 5 that both issuers walk in step.  Two streams:
     // each stream owns a ring of 3 (the sixth slot is the second Q tile, unused there), because a
@@ -874,6 +878,7 @@ __global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
     const int cb = blockIdx.z;     // cache of a batch
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
+    if (a.prefixes) pdl_wait();   // ragged batch: the row counts were written by an earlier kernel of the stream
     if (threadIdx.x == 0) {
         const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix;
         const int nt_all = (int)((P + a.n + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
@@ -964,7 +969,7 @@ cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s
                 : a.quant_bits == 4 ? (a.win_lo > 0 ? attn_tc_kernel<true, 4> : attn_tc_kernel<false, 4>)
                                     : (a.win_lo > 0 ? attn_tc_kernel<true, 0> : attn_tc_kernel<false, 0>);
     const uint32_t smem = quant ? kSmemBytesQ8 : kSmemBytes;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(kernel), (int)smem);
     if (e != cudaSuccess) return e;
     dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, a.batch);
     return launch_pdl(kernel, grid, dim3(quant ? kThreadsQ8 : kThreads), smem, s, a, maps.q, maps.k, maps.v);

@@ -199,16 +199,23 @@ kvf_status make_page_map(EncodeTiledFn fn, CUtensorMap *m, void *base, int d, in
     return KVF_OK;
 }
 
+// cuTensorMapEncodeTiled, looked up in the driver once per process (a failed lookup is retried).
 kvf_status encode_fn(EncodeTiledFn *fn) {
-    void *sym = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDriverEntryPoint");
-    if (qres != cudaDriverEntryPointSuccess || !sym) {
-        snprintf(g_cuda_err, sizeof(g_cuda_err), "driver has no cuTensorMapEncodeTiled");
-        return KVF_ERR_CUDA;
+    static std::mutex mu;
+    static EncodeTiledFn cached = nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cached) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetDriverEntryPoint");
+        if (qres != cudaDriverEntryPointSuccess || !sym) {
+            snprintf(g_cuda_err, sizeof(g_cuda_err), "driver has no cuTensorMapEncodeTiled");
+            return KVF_ERR_CUDA;
+        }
+        cached = reinterpret_cast<EncodeTiledFn>(sym);
     }
-    *fn = reinterpret_cast<EncodeTiledFn>(sym);
+    *fn = cached;
     return KVF_OK;
 }
 
@@ -1031,6 +1038,37 @@ kvf_status static_scratch(int dev, char **out) {
     return KVF_OK;
 }
 
+// Tensor maps of recent static calls, so that a loop over the layers of a model encodes each
+// layer's maps once: keyed on the device, the planes and the shape (the rotated-query map points
+// into the static scratch, which never moves).
+struct StaticMaps {
+    int dev;
+    const void *storage;
+    int32_t H, Hkv, d, max_chunk;
+    int64_t capacity;
+    TcMaps maps;
+};
+constexpr size_t kStaticMapEntries = 128;
+std::vector<StaticMaps> g_static_maps;
+size_t g_static_maps_next = 0;
+
+kvf_status static_maps(kvf_cache *c) {
+    const kvf_config &f = c->cfg;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    for (const StaticMaps &m : g_static_maps)
+        if (m.dev == c->device && m.storage == c->storage && m.H == f.n_q_heads && m.Hkv == f.n_kv_heads &&
+            m.d == f.head_dim && m.max_chunk == f.max_chunk && m.capacity == f.capacity) {
+            c->maps = m.maps;
+            return KVF_OK;
+        }
+    kvf_status s = build_maps(c);
+    if (s != KVF_OK) return s;
+    const StaticMaps m = {c->device, c->storage, f.n_q_heads, f.n_kv_heads, f.head_dim, f.max_chunk, f.capacity, c->maps};
+    if (g_static_maps.size() < kStaticMapEntries) g_static_maps.push_back(m);
+    else g_static_maps[g_static_maps_next++ % kStaticMapEntries] = m;
+    return KVF_OK;
+}
+
 }  // namespace
 
 extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_storage, size_t storage_bytes,
@@ -1048,14 +1086,34 @@ extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_stor
     if (check_ptr(q) || check_ptr(k_new) || check_ptr(v_new) || check_ptr(out)) return KVF_ERR_INVALID_ARG;
     if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return KVF_ERR_INVALID_ARG;
 
-    // sizes the fixed scratch can hold (max_chunk sizes the rotated-query area and its TMA box)
+    // sizes the fixed scratch can hold (max_chunk sizes the rotated-query area and its TMA box);
+    // all of this is checked before the first CUDA call
     const size_t row_elems = (size_t)cfg->n_q_heads * cfg->head_dim;
     if ((size_t)cfg->max_chunk * row_elems * elem_bytes(cfg->dtype) > kStaticQRotBytes) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "max_chunk x heads x head_dim exceeds the static scratch");
         return KVF_ERR_CAPACITY;
     }
     const size_t part_tokens = std::min(kStaticPartOBytes / (row_elems * 4), kStaticPartLseBytes / ((size_t)cfg->n_q_heads * 4));
-    if (part_tokens < (size_t)n_tokens) return KVF_ERR_CAPACITY;
+    if (part_tokens < (size_t)n_tokens) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "n_tokens x heads x head_dim partial rows exceed the static scratch");
+        return KVF_ERR_CAPACITY;
+    }
+    {
+        // A chunk that fits one 128-row tile runs as two streams on the tensor-core paths and always
+        // leaves 2 * (groups + Hkv - 1) partial slots of n * G rows, with groups >= Hkv: the least the
+        // kernel will write has to fit (the plan cuts the key range no finer than the rest allows).
+        const int G = cfg->n_q_heads / cfg->n_kv_heads;
+        const bool tensor_path = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, G);
+        if (tensor_path && attn_tc_streams(n_tokens, G) == 2) {
+            const size_t least = (size_t)2 * (2 * (size_t)cfg->n_kv_heads - 1) * (size_t)n_tokens * G;
+            if (least > part_tokens * (size_t)cfg->n_q_heads) {
+                snprintf(g_cuda_err, sizeof(g_cuda_err),
+                         "a short chunk over %d KV heads leaves more partial rows than the static scratch holds",
+                         (int)cfg->n_kv_heads);
+                return KVF_ERR_CAPACITY;
+            }
+        }
+    }
 
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -1078,7 +1136,7 @@ extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_stor
     c.len = len;
     c.part_rows_cap = (int64_t)part_tokens * cfg->n_q_heads;   // the plan splits only as far as this holds
     if (c.tc) {
-        s = build_maps(&c);
+        s = static_maps(&c);
         if (s != KVF_OK) return s;
     }
 

@@ -5,6 +5,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+#include <vector>
+
 namespace kvf {
 
 // Programmatic dependent launch: a kernel launched with launch_pdl may be scheduled while the
@@ -31,6 +34,23 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #endif
+
+// Raises a kernel's dynamic shared-memory limit, once per kernel and device (the attribute
+// belongs to the device's copy of the function): launches after the first skip the runtime call.
+inline cudaError_t raise_smem_limit_once(const void *kernel, int bytes) {
+    struct Done { const void *kernel; int dev; };
+    static std::mutex mu;
+    static std::vector<Done> done;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    for (const Done &d : done)
+        if (d.kernel == kernel && d.dev == dev) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) done.push_back({kernel, dev});
+    return e;
+}
 
 constexpr int kMaxHalfDim = 64;       // head_dim <= 128
 constexpr int kKvTile = 128;          // key rows per tensor-core tile; V rows are zero-padded to it

@@ -67,8 +67,9 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
     const int n_tok_blocks = (a.n + kTok - 1) / kTok;
     const int b = blockIdx.y;      // cache of a batch (0 when there is one cache)
     const RowMap rows{a.page_tables ? a.page_tables[b] : a.page_table, a.capacity, a.page_elems, a.d};
-    // (the per-cache arrays of a ragged batch were written by a kernel that had finished before
-    // this one could start)
+    // (the per-cache arrays of a ragged batch were written by an earlier kernel of the stream: under
+    // a dependent launch they are visible only after the wait)
+    if (a.prefixes || a.pos0s) pdl_wait();
     const int64_t prefix = a.prefixes ? a.prefixes[b] : a.prefix;
     const int64_t pos0 = a.pos0s ? a.pos0s[b] : a.pos0;
 

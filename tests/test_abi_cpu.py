@@ -143,6 +143,28 @@ def test_batch_entry_points_validate_before_any_cuda_call(binding):
     lib.kvf_batch_destroy(None)
 
 
+def test_static_entry_point_refuses_what_its_fixed_scratch_cannot_hold_before_any_cuda_call(binding):
+    """The fixed scratch holds 16 MiB of partial rows.  A chunk that fits one 128-row tile runs as
+    two streams and leaves at least 2 * (2 Hkv - 1) slots of n * G rows: with 128 KV heads of 128
+    that is 65 280 rows of 512 B against 32 768, so the call must be refused (nothing is launched:
+    the pointers below are not device memory at all)."""
+    lib = binding.load()
+    cfg = binding.make_config(128, 128, 128, "bf16", 4096, 128, rope_base=5e5)
+    big = 1 << 40
+    rc = lib.kvf_fold_step_static(ctypes.byref(cfg), 4096, big, 0, 4096, 4096, 4096, 128, 0, 4096, None, None)
+    assert rc == binding.KVF_ERR_CAPACITY
+    assert b"static scratch" in lib.kvf_last_cuda_error()
+    # 64 KV heads still fit ((4 * 64 - 2) * 128 <= 512 * 64 rows): such a call passes the size checks,
+    # so ask for it with a misaligned query pointer and see the argument error instead
+    ok = binding.make_config(64, 64, 128, "bf16", 4096, 128, rope_base=5e5)
+    rc = lib.kvf_fold_step_static(ctypes.byref(ok), 4096, big, 0, 4096 + 2, 4096, 4096, 128, 0, 4096, None, None)
+    assert rc == binding.KVF_ERR_INVALID_ARG
+    # the other fixed limits: the rotated chunk (4 MiB) and the partial rows of one chunk (16 MiB)
+    wide = binding.make_config(32, 8, 128, "bf16", 4096, 1024, rope_base=5e5)
+    rc = lib.kvf_fold_step_static(ctypes.byref(wide), 4096, big, 0, 4096, 4096, 4096, 1024, 0, 4096, None, None)
+    assert rc == binding.KVF_ERR_CAPACITY and b"static scratch" in lib.kvf_last_cuda_error()
+
+
 def test_binding_fails_loudly_without_the_library(binding, monkeypatch, tmp_path):
     import importlib
     monkeypatch.setattr(binding, "_lib", None)
