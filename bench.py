@@ -33,11 +33,17 @@ from paper_2605_12471_b200 import workloads  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes (read + write) of one attention launch per algorithmic cache byte it reads, from the
-# ncu capture summarised in profiles/attn_tc_kernel_chain_64k_c256_last_steps.md (65 536-token
-# chain; traffic grows in proportion to the cache rows read, so the ratio carries over).  Set to
-# None whenever attn_tc_kernel changes after the capture.
+# DRAM bytes (read + write) of one attention launch per algorithmic cache byte it reads, from an
+# ncu capture of the last steps of a 65 536-token chain of 256-token chunks (too large to capture
+# at 131 072 tokens; traffic grows in proportion to the cache rows read, so the ratio carries
+# over).  Set to None whenever the attention kernel changes after the capture.
 NCU_TRAFFIC_BYTES_PER_CACHE_BYTE = 1.033
+NCU_TRAFFIC_SOURCE = ("ncu capture (dram__bytes_read.sum + dram__bytes_write.sum) of the attention kernel on the "
+                      "last steps of a 65 536-token chain of 256-token chunks: 1.033 DRAM bytes per algorithmic "
+                      "cache byte, scaled by the cache rows a launch of this run reads")
+NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 7700.0}      # dense bf16 and HBM3e figures of the B200 data sheet
+TENSOR_FLOP_PER_SM_CLOCK = 8192.0                         # one 128 x 128 x 16 bf16 MMA (524 288 FLOP) per 64 clocks
+N_SMS = 148
 
 
 def peaks():
@@ -100,6 +106,55 @@ class ClockSampler:
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
+
+
+class NvmlClock:
+    """Reads the SM clock of one GPU through NVML about once a millisecond (a read, nothing is set),
+    with host timestamps, so that short stretches of a run can be given their own median clock."""
+
+    def __init__(self, gpu_index: int):
+        self.samples, self._stop, self.thread, self.handle = [], threading.Event(), None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(gpu_index)
+        except Exception:            # no NVML: the per-bin clocks are simply left out
+            self.handle = None
+
+    def start(self):
+        if self.handle is None:
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        while not self._stop.is_set():
+            try:
+                mhz = self.nv.nvmlDeviceGetClockInfo(self.handle, self.nv.NVML_CLOCK_SM)
+            except Exception:
+                return
+            self.samples.append((time.perf_counter(), float(mhz)))
+            time.sleep(0.001)
+
+    def stop(self):
+        self._stop.set()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+
+    def median_between(self, t0: float, t1: float):
+        xs = [m for t, m in self.samples if t0 <= t <= t1]
+        return statistics.median(xs) if xs else None
+
+
+def set_oracle_threads(n: int) -> bool:
+    """Thread count of the oracle's OpenMP runtime (the oracle itself is left as it stands)."""
+    import ctypes
+    try:
+        ctypes.CDLL("libgomp.so.1").omp_set_num_threads(int(n))
+        return True
+    except OSError:
+        return False
 
 
 def oracle_rate(w: workloads.Workload, seed: int, rows_per_step: int, repeats: int, prefix: int):
@@ -277,7 +332,7 @@ def run_full_stack(args):
     print(json.dumps(line), flush=True)
 
 
-def main():
+def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
@@ -289,9 +344,13 @@ def main():
                     help="tokens folded (in 2048-token steps, untimed) before every timed chain: the timed chain "
                          "then runs from this prefix to --tokens (decode- and question-shaped steps at depth)")
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"],
-                    help="cache and input dtype (f32 runs the CUDA-core path; not the benchmark workload)")
-    ap.add_argument("--workload", default="deep_chain", choices=["deep_chain", "full_stack"],
-                    help="full_stack: the 4 x 32-layer memory-scale fold (64 GiB of cache; a separate, longer run)")
+                    help="cache and input dtype (not the benchmark workload)")
+    ap.add_argument("--workload", default="deep_chain", choices=["deep_chain", "llama_16k", "sweep", "full_stack"],
+                    help="deep_chain: 131 072 tokens in chunks of 256 (the headline line).  llama_16k: 16 384 tokens "
+                         "in chunks of 2048, inputs scaled by 1/sqrt(128).  sweep: 65 536 tokens at chunks of 128, "
+                         "512, 2048 and 8192, each with a bf16 and an fp32 cache, one line per combination with the "
+                         "output drift against the oracle on sampled rows.  full_stack: the 4 x 32-layer "
+                         "memory-scale fold (64 GiB of cache; a separate, longer run)")
     ap.add_argument("--sequences", type=int, default=4)
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--seed", type=int, default=2605)
@@ -316,19 +375,73 @@ def main():
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every fold step of the timed chains from the host instead of replaying the chain "
                          "as one CUDA graph captured from the same kvf_fold_step calls")
-    args = ap.parse_args()
+    return ap.parse_args()
 
+
+def main():
+    args = parse_args()
     if args.workload == "full_stack" and args.impl == "ours":
         run_full_stack(args)
         return
-    w = workloads.DEEP_CHAIN
-    if args.tokens or args.chunk or args.prefill or args.dtype != w.dtype:
-        w = w.with_(name=f"chain_{args.tokens or w.tokens}_c{args.chunk or w.chunk}_from_{args.prefill}_{args.dtype}",
-                    tokens=args.tokens or w.tokens, chunk=args.chunk or w.chunk, dtype=args.dtype)
-    if args.impl == "reference":
-        run_reference(args, w)
-        return
+    if args.workload == "sweep":
+        variants = workloads.SWEEP
+    elif args.workload == "llama_16k":
+        variants = [workloads.LLAMA_16K]
+    else:
+        variants = [workloads.DEEP_CHAIN]
+    for w in variants:
+        if args.tokens or args.chunk or args.prefill or (args.dtype != w.dtype and args.workload != "sweep"):
+            w = w.with_(name=f"chain_{args.tokens or w.tokens}_c{args.chunk or w.chunk}_from_{args.prefill}_{args.dtype}",
+                        tokens=args.tokens or w.tokens, chunk=args.chunk or w.chunk, dtype=args.dtype)
+        if args.impl == "reference":
+            run_reference(args, w)
+        else:
+            run_chain_bench(args, w, drift=(args.workload == "sweep"))
+            torch.cuda.empty_cache()                     # a sweep's next variant starts from an empty pool
+    if args.impl == "ours" and int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        import torch.distributed as dist
+        if dist.is_initialized():
+            dist.destroy_process_group()
 
+
+def oracle_drift(w, seed, q, k, v, out, C, budget_steps=15, rows_extra=10):
+    """Output drift against the fp64 oracle on sampled rows of sampled steps of one chain (the
+    oracle ingests every chunk, so it holds the same history as the cache), and the oracle's own
+    speed on those rows.  q, k, v, out hold the whole chain on the device."""
+    import numpy as np
+
+    import oracle
+    N = w.tokens // C
+    rng = np.random.default_rng(seed + C)
+    steps = {0, 1, 2, N // 4, N // 2, N - 2, N - 1}
+    steps = {t for t in steps if 0 <= t < N}
+    steps.update(int(x) for x in rng.integers(0, N, size=max(0, budget_steps - len(steps))))
+    oc = oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, w.tokens, rope_base=w.rope_base)
+    per_step, cpu_s, pairs = [], 0.0, 0
+    worst, sum_abs, count = 0.0, 0.0, 0
+    for t in range(N):
+        sl = slice(t * C, (t + 1) * C)
+        qc, kc, vc = (x[sl].to("cpu", torch.float64).numpy() for x in (q, k, v))
+        if t not in steps:
+            oc.fold_step(qc, kc, vc, rows=[])
+            continue
+        rows = sorted({r for r in (0, 1, C // 2 - 1, C // 2, C - 2, C - 1) if 0 <= r < C} |
+                      {int(x) for x in rng.integers(0, C, size=rows_extra)})
+        p0 = len(oc)
+        t0 = time.perf_counter()
+        ref = oc.fold_step(qc, kc, vc, rows=rows)
+        cpu_s += time.perf_counter() - t0
+        pairs += sum(p0 + r + 1 for r in rows)
+        got = out[sl][rows].to("cpu", torch.float64).numpy()
+        err = np.abs(got - ref)
+        per_step.append({"step": t, "prefix": t * C, "max_abs": float(err.max()), "mean_abs": float(err.mean()),
+                         "rel_rms": float(np.sqrt((err ** 2).sum() / max((ref ** 2).sum(), 1e-300)))})
+        worst, sum_abs, count = max(worst, float(err.max())), sum_abs + float(err.sum()), count + err.size
+    return {"max_abs": worst, "mean_abs": sum_abs / max(count, 1), "checked_steps": len(per_step),
+            "rows_per_step": 6 + rows_extra, "per_step": per_step}, pairs / max(cpu_s, 1e-9), cpu_s
+
+
+def run_chain_bench(args, w, drift=False):
     from paper_2605_12471_b200 import binding, multi
     import torch.distributed as dist
 
@@ -336,9 +449,10 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the fold step has no CPU path")
     torch.cuda.set_device(local)
-    if world > 1:
+    if world > 1 and not dist.is_initialized():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     lib = binding.load()
+    steps_timed = args.steps if not drift else max(1, min(args.steps, 3))
 
     T, C = w.tokens, w.chunk
     P0 = args.prefill
@@ -453,64 +567,118 @@ def main():
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms = timed(run_chain, args.steps)
+    ms = timed(run_chain, steps_timed)
     clocks = sampler.stop() if rank == 0 else None
     assert graph is not None or len(cache) == T
     if cache.status() != binding.KVF_OK:
         raise SystemExit("device status word reports a timed-out wait")
-    value = multi.whole_job_tokens_per_s(T - P0, args.steps, 1 if by_heads else world, ms)
+    value = multi.whole_job_tokens_per_s(T - P0, steps_timed, 1 if by_heads else world, ms)
 
     # per-kernel time of the same chain, CUDA events around every launch on the launching stream;
-    # read out in bins of steps, which gives the latency against the prefix length
+    # read out in bins of steps, which gives the latency against the prefix length.  The SM clock is
+    # read through NVML meanwhile, so every bin carries the clock it ran at: time x clock separates a
+    # kernel that got slower from a clock that the power cap lowered.
     prefill()
     torch.cuda.synchronize()
     l0 = cache.launch_count()
     cache.profile(True)
     kms, kcnt, curve = [0.0, 0.0, 0.0], [0, 0, 0], []
     nbins = min(16, N)
+    nvml = NvmlClock(local)
+    nvml.start()
+    t_prof0 = time.perf_counter()
+    tensor_shaped = w.dtype == "bf16" and not args.force_simt
     for bi in range(nbins):
         first, last = bi * N // nbins, (bi + 1) * N // nbins
+        t0 = time.perf_counter()
         body(first, last)
         bms, bcnt = cache.profile_read()
+        t1 = time.perf_counter()
         fl = sum(w.flops_step(visible(P0 + t * C), C) for t in range(first, last))
         by = sum(visible(P0 + t * C) + C for t in range(first, last)) * bytes_per_token
-        curve.append({"prefix_from": P0 + first * C, "prefix_to": P0 + (last - 1) * C,
-                      "step_us": 1e3 * sum(bms) / (last - first), "attention_us": 1e3 * bms[1] / (last - first),
-                      "attention_tflops": fl / (bms[1] * 1e-3) / 1e12, "cache_read_gbs": by / (bms[1] * 1e-3) / 1e9})
+        mhz = nvml.median_between(t0, t1)
+        point = {"prefix_from": P0 + first * C, "prefix_to": P0 + (last - 1) * C,
+                 "step_us": 1e3 * sum(bms) / (last - first), "attention_us": 1e3 * bms[1] / (last - first),
+                 "attention_tflops": fl / (bms[1] * 1e-3) / 1e12, "cache_read_gbs": by / (bms[1] * 1e-3) / 1e9,
+                 "sm_mhz": mhz}
+        if mhz:
+            point["attention_kilocycles"] = 1e3 * bms[1] / (last - first) * mhz / 1e3
+            if tensor_shaped:
+                point["tensor_flop_per_sm_clock_frac"] = fl / (bms[1] * 1e-3 * mhz * 1e6 * N_SMS * TENSOR_FLOP_PER_SM_CLOCK)
+        curve.append(point)
         kms = [x + y for x, y in zip(kms, bms)]
         kcnt = [x + y for x, y in zip(kcnt, bcnt)]
+    nvml.stop()
+    prof_mhz = nvml.median_between(t_prof0, time.perf_counter())
     cache.profile(False)
-    launches = (cache.launch_count() - l0) * args.steps       # kernels of the timed chains
+    launches = (cache.launch_count() - l0) * steps_timed       # kernels of the timed chains
     pk = peaks()
     attn_flops = sum(w.flops_step(visible(P0 + t * C), C) for t in range(N))
     attn_tflops = attn_flops / (kms[1] * 1e-3) / 1e12
     cache_bytes_read = sum(visible(P0 + t * C) + C for t in range(N)) * bytes_per_token
     hbm_gbs = cache_bytes_read / (kms[1] * 1e-3) / 1e9
     traffic = None
-    if NCU_TRAFFIC_BYTES_PER_CACHE_BYTE is not None and not (args.cache_int8 or args.cache_int4):
+    if NCU_TRAFFIC_BYTES_PER_CACHE_BYTE is not None and w.dtype == "bf16" and not (args.cache_int8 or args.cache_int4 or args.force_simt):
         traffic = NCU_TRAFFIC_BYTES_PER_CACHE_BYTE * cache_bytes_read / kcnt[1]
     # which roof binds: arithmetic intensity G*C FLOP per cache byte against the ridge of the measured peaks
     ridge = pk["bf16_tflops_sustained"] * 1e12 / (pk["hbm_gbs"] * 1e9)
     intensity = attn_flops / cache_bytes_read
-    if w.dtype == "f32":
-        # fp32 caches run on the CUDA cores (fp32 accuracy rules out single-pass tensor formats): the roof is
-        # the FFMA rate, 148 SMs x 128 lanes x 2 FLOP at the 1965 MHz maximum clock
-        alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
+    plan_last = cache.plan(C, T - C)
+    if w.dtype == "f32" and not plan_last[0]:
+        # CUDA-core kernel (head_dim 64, or forced): the roof is the FFMA rate, 148 SMs x 128 lanes x 2 FLOP at
+        # the 1965 MHz maximum clock
+        alu_peak = N_SMS * 128 * 2 * 1.965e9 / 1e12
         roofline = {"bound": "alu", "achieved": attn_tflops, "peak": alu_peak, "unit": "TFLOP/s",
                     "frac": attn_tflops / alu_peak, "peak_source": "derived: 148 SMs x 128 FFMA lanes x 2 x 1.965 GHz"}
+    elif w.dtype == "f32":
+        # fp32 caches on the tensor pipe: every product is three fp16 MMAs (hi x hi, hi x lo, lo x hi of operands
+        # split into two fp16 halves), so the roof is a third of the fp16/bf16 rate
+        peak = pk["bf16_tflops_sustained"] / 3.0
+        roofline = {"bound": "tensor", "achieved": attn_tflops, "peak": peak, "unit": "TFLOP/s", "frac": attn_tflops / peak,
+                    "peak_source": pk["_source"] + " sustained bf16 / 3 (three fp16 products per fp32 product)",
+                    "gate": "sustained", "frac_sustained": attn_tflops / peak,
+                    "frac_burst": attn_tflops / (pk["bf16_tflops"] / 3.0), "frac_nominal": attn_tflops / (NOMINAL["bf16_tflops"] / 3.0)}
     elif intensity >= ridge:
         roofline = {"bound": "tensor", "achieved": attn_tflops, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                    "frac": attn_tflops / pk["bf16_tflops_sustained"], "peak_source": pk["_source"] + " sustained bf16"}
+                    "frac": attn_tflops / pk["bf16_tflops_sustained"], "peak_source": pk["_source"] + " sustained bf16",
+                    # the three denominators side by side; the 60 % target is judged on the measured sustained one
+                    # (the part is power-capped: a seconds-long bf16 GEMM loop settles there)
+                    "gate": "sustained", "frac_sustained": attn_tflops / pk["bf16_tflops_sustained"],
+                    "frac_burst": attn_tflops / pk["bf16_tflops"], "frac_nominal": attn_tflops / NOMINAL["bf16_tflops"],
+                    "peaks_tflops": {"nominal": NOMINAL["bf16_tflops"], "burst": pk["bf16_tflops"],
+                                     "sustained": pk["bf16_tflops_sustained"]}}
     else:
         roofline = {"bound": "hbm", "achieved": hbm_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                    "frac": hbm_gbs / pk["hbm_gbs"], "peak_source": pk["_source"] + " copy bandwidth"}
+                    "frac": hbm_gbs / pk["hbm_gbs"], "peak_source": pk["_source"] + " copy bandwidth",
+                    "gate": "measured copy", "frac_sustained": hbm_gbs / pk["hbm_gbs"], "frac_burst": hbm_gbs / pk["hbm_gbs"],
+                    "frac_nominal": hbm_gbs / NOMINAL["hbm_gbs"]}
+    if prof_mhz and roofline["bound"] == "tensor":
+        # clock-normalised: share of the tensor pipe's per-clock rate at the clock sampled during this pass
+        per_clock = TENSOR_FLOP_PER_SM_CLOCK / (3.0 if w.dtype == "f32" else 1.0)
+        roofline["sm_mhz_during_profile"] = prof_mhz
+        roofline["frac_of_tensor_rate_at_sampled_clock"] = attn_tflops * 1e12 / (prof_mhz * 1e6 * N_SMS * per_clock)
     roofline.update({
-        "kernel": "prefix+chunk attention", "traffic": traffic, "flops_per_launch": attn_flops / kcnt[1],
+        "kernel": "prefix+chunk attention", "traffic": traffic, "traffic_source": NCU_TRAFFIC_SOURCE if traffic else None,
+        "flops_per_launch": attn_flops / kcnt[1],
         "cache_bytes_per_launch": cache_bytes_read / kcnt[1], "ms_per_launch": kms[1] / kcnt[1], "launches": kcnt[1],
         "kernel_ms_per_chain": {"rope_append": kms[0], "attention": kms[1], "combine": kms[2]},
         "attention_tflops": attn_tflops, "cache_read_gbs": hbm_gbs, "flop_per_cache_byte": intensity,
         "ridge_flop_per_byte": ridge, "hbm_peak_gbs": pk["hbm_gbs"], "bf16_peak_tflops": pk["bf16_tflops_sustained"],
     })
+
+    drift_report = None
+    cpu = None
+    if drift and rank == 0:
+        # one more eager chain whose outputs stay in `out`; the oracle follows it on sampled rows
+        cache.reset()
+        body()
+        torch.cuda.synchronize()
+        drift_report, pairs_per_s, cpu_s = oracle_drift(w, args.seed, q, k, v, out, C)
+        threads = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+        cpu = {"value": tokens_per_s_from_pairs(w, pairs_per_s, P0), "unit": "tokens/s", "cores": threads, "kind": "oracle",
+               "sample": (f"{drift_report['rows_per_step']} query rows x {H} heads at {drift_report['checked_steps']} steps "
+                          f"spread over the chain ({cpu_s:.1f} s of CPU work), fp64 oracle; tokens/s extrapolated "
+                          f"linearly in visible (query,key) pairs over the chain")}
 
     e2e = None
     if not args.no_e2e:
@@ -527,26 +695,30 @@ def main():
 
         prefill()
         body_host()
-        e2e_steps = max(1, min(args.steps, 3))
+        e2e_steps = steps_timed                              # as many chains as the device-resident leg
         ems = timed(body_host, e2e_steps)
         e2e = {"value": (1 if by_heads else world) * e2e_steps * (T - P0) / (ems * 1e-3), "unit": "tokens/s", "steps": e2e_steps,
                "h2d_bytes_per_step": (T - P0) * (H + 2 * Hkv) * d * eb, "d2h_bytes_per_step": (T - P0) * H * d * eb,
                "ms_per_step": ems / e2e_steps}
 
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.window:
+    if cpu is None and rank == 0 and world == 1 and not args.no_cpu_baseline and not args.window:
         rate, times, threads, rows = oracle_rate(w, args.seed, rows_per_step=32, repeats=4, prefix=max(0, T - 5 * C))
         cpu = {"value": tokens_per_s_from_pairs(w, rate, P0), "unit": "tokens/s", "cores": threads, "kind": "oracle",
                "sample": (f"{len(rows)} query rows x {H} heads of one chunk at prefix ~{T - 4 * C}, median of "
                           f"{len(times)} repeats ({sum(times):.1f} s of CPU work), fp64 oracle; tokens/s "
                           f"extrapolated linearly in visible (query,key) pairs over the chain")}
+        if set_oracle_threads(1):
+            # the same oracle on one thread, on a sample an eighth the size
+            rate1, times1, _, rows1 = oracle_rate(w, args.seed, rows_per_step=4, repeats=1, prefix=max(0, T - 5 * C))
+            set_oracle_threads(threads)
+            cpu["single_thread"] = {"value": tokens_per_s_from_pairs(w, rate1, P0), "unit": "tokens/s", "cores": 1,
+                                    "sample": f"{len(rows1)} query rows x {H} heads, one repeat ({sum(times1):.1f} s of CPU work)"}
 
     if rank == 0:
-        plan = cache.plan(C, T - C)
-        step_flops = attn_flops * world * args.steps
+        step_flops = attn_flops * world * steps_timed
         line = {
             "metric": "fold-step tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "steps": steps_timed, "warmup": args.warmup, "ms_per_step": ms / steps_timed,
             "higher_is_better": True, "scaling": "strong" if by_heads else "weak", "vs_baseline": None, "dtype": w.dtype,
             "data": "synthetic",
             "config": {"workload": w.name, "shard": args.shard, "tokens": T, "chunk": C, "prefill": P0, "fold_steps_per_step": N,
@@ -554,14 +726,15 @@ def main():
                        "sequences_per_gpu": 1, "paged": bool(args.paged), "sinks": args.sinks, "window": args.window,
                        "cache_storage": ("int8 codes + fp32 row scales" if args.cache_int8 else
                                          "int4 codes + fp32 row scales" if args.cache_int4 else w.dtype),
-                       "launch": "per-step host launches" if graph is None else "one CUDA graph per chain, captured from the same calls", "l2": "inputs larger than L2 (cache grows to 512 MiB per chain)",
-                       "last_step_plan": {"tensor_core": plan[0], "splits": plan[1], "ctas": plan[2]}},
+                       "launch": "per-step host launches" if graph is None else "one CUDA graph per chain, captured from the same calls",
+                       "l2": f"inputs larger than L2 (cache grows to {T * bytes_per_token / 2 ** 20:.0f} MiB per chain)",
+                       "last_step_plan": {"tensor_core": plan_last[0], "splits": plan_last[1], "ctas": plan_last[2]}},
             "attention_tflops": step_flops / (ms * 1e-3) / 1e12,
             "roofline": roofline, "latency_vs_prefix": curve, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
         }
+        if drift_report is not None:
+            line["drift_vs_oracle"] = drift_report
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -44,7 +44,9 @@ typedef enum {
     KVF_ERR_UNSUPPORTED = 3, /* head_dim / head ratio / dtype outside what the kernels cover     */
     KVF_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed (see kvf_last_cuda_error)   */
     KVF_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (read via kvf_cache_status)   */
-    KVF_ERR_POS = 6          /* KVF_STRICT_POS set and pos0 != current length                    */
+    KVF_ERR_POS = 6,         /* KVF_STRICT_POS set and pos0 != current length                    */
+    KVF_ERR_RANGE = 7        /* an fp32 cache on the tensor-core path met a rotated key, query or
+                                value above 65 504 in magnitude (read via kvf_cache_status)      */
 } kvf_status;
 
 typedef enum { KVF_BF16 = 0, KVF_F32 = 1 } kvf_dtype;
@@ -53,8 +55,9 @@ enum {
     KVF_ROPE_INTERLEAVED = 1u, /* rotate pairs (2j,2j+1) instead of (j, j+d/2)                   */
     KVF_STRICT_POS = 2u,       /* reject pos0 != len (positions must continue across chunks)     */
     KVF_OUT_F32 = 4u,          /* `out` is fp32 even when dtype is bf16                          */
-    KVF_FORCE_SIMT = 8u,       /* use the CUDA-core attention kernel even where the tensor-core
-                                  kernel applies (bisecting aid; same results within tolerance) */
+    KVF_FORCE_SIMT = 8u,       /* use the CUDA-core attention kernel even where a tensor-core
+                                  kernel applies (bisecting aid, and the path for fp32 caches whose
+                                  values leave fp16's range; same results within tolerance)      */
     KVF_HOST_UPLOAD_AHEAD = 32u, /* kvf_fold_step_host copies a step's q/k/v to the device on a stream of the
                                   library's own, into one of two staging sets, so that the upload of step
                                   t+1 runs while step t computes (the call's stream waits for the upload;
@@ -84,7 +87,13 @@ enum {
  *   head_dim (d): 64 or 128.
  *   dtype: element type of q, k_new, v_new, of the cache planes and (unless KVF_OUT_F32) of out.
  *       KVF_BF16: rotation, scores, softmax state and the output sum are fp32, probabilities
- *       and the rotated q/k are rounded once to bf16.  KVF_F32: fp32 throughout (CUDA cores).
+ *       and the rotated q/k are rounded once to bf16.  KVF_F32: fp32 throughout.  With head_dim
+ *       128 the fp32 attention runs on the tensor cores: each operand is split into two fp16
+ *       halves (22 significant bits; elements below 2^-3 to an absolute 2^-25) and each product
+ *       is three MMAs, with the output summed in round-to-nearest fp32 registers; magnitudes
+ *       must stay within fp16's 65 504 (else KVF_ERR_RANGE in the status word and non-finite
+ *       outputs).  With head_dim 64, or under KVF_FORCE_SIMT, it runs on the CUDA cores in plain
+ *       fp32 with no such limits.
  *   capacity: most tokens the cache will ever hold.
  *   max_chunk: largest n_tokens of any later kvf_fold_step (sizes the workspace).
  *   rope_base: theta = pos * rope_base^(-2j/d) (RoPE at the tokens' absolute positions, which
@@ -189,7 +198,7 @@ int64_t kvf_cache_len(const kvf_cache *c);
 kvf_status kvf_cache_reset(kvf_cache *c);
 
 /* Reads the device status word (synchronises the default stream with a blocking copy): KVF_OK,
- * or KVF_ERR_TIMEOUT if a bounded wait inside a kernel gave up.  Call after synchronising the
+ * KVF_ERR_TIMEOUT if a bounded wait inside a kernel gave up, or KVF_ERR_RANGE (see kvf_status).  Call after synchronising the
  * streams that carried the steps.  (The paper has no counterpart: this reports on the kernels'
  * own waits, not on anything the method computes.) */
 kvf_status kvf_cache_status(kvf_cache *c);
@@ -199,6 +208,14 @@ kvf_status kvf_cache_status(kvf_cache *c);
  * + 65536 * (waiting warp) + 2^24 * (awaited parity) - what a bug report should quote.
  * -1 for a null handle or a failed copy. */
 int32_t kvf_cache_status_word(kvf_cache *c);
+
+/* The SM clock the attention kernels ran at, measured by the kernels themselves.  (The paper has
+ * no counterpart: a measurement aid.)  The first CTA of every tensor-core attention launch adds the
+ * SM cycles and the nanoseconds (device timer) it was running to two sums kept beside the status
+ * word; cycles_ns[0] / cycles_ns[1] receive the sums since the cache was created, so the difference
+ * of two readings gives cycles * 1000 / ns = MHz over the launches in between.  Blocking copy, as
+ * kvf_cache_status; the CUDA-core kernel does not count.  Caches that share a workspace share the sums. */
+kvf_status kvf_cache_sm_clock(kvf_cache *c, uint64_t cycles_ns[2]);
 
 /* Device pointers of the planes, [n_kv_heads][capacity][head_dim] of dtype (int8 codes under
  * KVF_CACHE_INT8), and of the rows' fp32 scales (NULL without that flag): [n_kv_heads][stride] with
@@ -210,11 +227,11 @@ float *kvf_cache_v_scales(const kvf_cache *c);
 
 /*
  * What a step of n_tokens on a prefix of prefix_len would launch:
- *   plan[0] 1 = tensor-core (tcgen05) attention kernel, 0 = CUDA-core kernel
+ *   plan[0] 1 = a tensor-core (tcgen05) attention kernel (bf16, or fp32 with head_dim 128), 0 = CUDA-core kernel
  *   plan[1] parts the key range of one KV head is cut into (1 = none).  CUDA-core kernel: equal
  *           splits.  Tensor-core kernel: the (KV head, key tile) pairs are cut into plan[2] /
- *           (row pairs) contiguous ranges that need not end at KV-head boundaries; this is their
- *           number per KV head, rounded up
+ *           (row blocks: 256-row pairs in bf16, 128-row blocks in fp32) contiguous ranges that
+ *           need not end at KV-head boundaries; this is their number per KV head, rounded up
  *   plan[2] CTAs of the attention kernel
  *   plan[3] kernels launched by the step (3 = a combine kernel merges partial results; chunks of
  *           at most 128 / (H / Hkv) tokens always take that route on the tensor-core path)

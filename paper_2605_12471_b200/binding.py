@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkvfold.so")
 
 KVF_OK, KVF_ERR_INVALID_ARG, KVF_ERR_CAPACITY, KVF_ERR_UNSUPPORTED, KVF_ERR_CUDA, KVF_ERR_TIMEOUT, \
-    KVF_ERR_POS = range(7)
+    KVF_ERR_POS, KVF_ERR_RANGE = range(8)
 KVF_BF16, KVF_F32 = 0, 1
 KVF_ROPE_INTERLEAVED, KVF_STRICT_POS, KVF_OUT_F32, KVF_FORCE_SIMT, KVF_CACHE_INT8 = 1, 2, 4, 8, 16
 KVF_HOST_UPLOAD_AHEAD, KVF_CACHE_INT4 = 32, 64
@@ -29,7 +29,7 @@ EXPORTS = [
     "kvf_paged_pool_bytes", "kvf_paged_cache_create",
     "kvf_batch_workspace_bytes", "kvf_batch_create", "kvf_batch_fold_step", "kvf_batch_plan",
     "kvf_batch_status_word", "kvf_batch_launch_count", "kvf_batch_destroy", "kvf_cache_set_window",
-    "kvf_batch_fold_step_ragged", "kvf_cache_k_scales", "kvf_cache_v_scales",
+    "kvf_batch_fold_step_ragged", "kvf_cache_k_scales", "kvf_cache_v_scales", "kvf_cache_sm_clock",
 ]
 
 
@@ -90,6 +90,8 @@ def load() -> ctypes.CDLL:
     lib.kvf_cache_status.restype = ctypes.c_int
     lib.kvf_cache_status_word.argtypes = [vp]
     lib.kvf_cache_status_word.restype = i32
+    lib.kvf_cache_sm_clock.argtypes = [vp, ctypes.POINTER(u64)]
+    lib.kvf_cache_sm_clock.restype = ctypes.c_int
     lib.kvf_cache_k_plane.argtypes = [vp]
     lib.kvf_cache_k_plane.restype = vp
     lib.kvf_cache_v_plane.argtypes = [vp]
@@ -243,6 +245,14 @@ class Cache:
     def status_word(self) -> int:
         """Raw device status word (0 = no bounded wait gave up; see kvf_cache_status_word)."""
         return int(load().kvf_cache_status_word(self._h))
+
+    def sm_clock(self) -> Tuple[int, int]:
+        """(SM cycles, nanoseconds) summed over the first CTA of every tensor-core attention launch so far."""
+        arr = (ctypes.c_uint64 * 2)()
+        rc = load().kvf_cache_sm_clock(self._h, arr)
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_cache_sm_clock")
+        return int(arr[0]), int(arr[1])
 
     def _plane(self, ptr: int) -> torch.Tensor:
         shape = (self.cfg.n_kv_heads, self.cfg.capacity, self.cfg.head_dim)

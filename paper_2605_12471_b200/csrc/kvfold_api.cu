@@ -100,7 +100,8 @@ struct kvf_cache {
     int64_t len;
     int G;
     float scale_log2;
-    bool tc;
+    bool tc;                 // bf16, head_dim 128: the tcgen05 kernel fed by TMA
+    bool tc32;               // fp32, head_dim 128: the tcgen05 kernel on fp16 halves of the operands
     TcMaps maps;
     int force_splits;
     int64_t part_rows_cap;   // rows of head_dim floats the partial area holds
@@ -287,7 +288,7 @@ int64_t window_lo(const kvf_cache *c, int64_t prefix) {
 Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t part_rows_cap = -1) {
     if (part_rows_cap < 0) part_rows_cap = c->part_rows_cap;
     Plan p;
-    p.tc = c->tc;
+    p.tc = c->tc || c->tc32;
     p.ngroups = 0;
     const int64_t L = prefix + n;
     const int Hkv = c->cfg.n_kv_heads;
@@ -296,7 +297,8 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
         // into equal ranges.  Whole KV heads if that fills the SMs, else as many groups as give
         // one CTA per SM, with at least 4 key tiles each and within the partial area.
         const int64_t nt = (L + kKvTile - 1) / kKvTile - WindowTiles(window_lo(c, prefix), c->n_sink, kKvTile).skip;
-        const int pairs = attn_tc_row_pairs(n, c->G);
+        // (row blocks of a KV head: 256-row pairs in the bf16 kernel, 128-row blocks in the fp32 one)
+        const int pairs = c->tc32 ? attn_tc32_row_blocks(n, c->G) : attn_tc_row_pairs(n, c->G);
         int64_t groups = Hkv;
         if (c->force_splits > 0) {
             groups = (int64_t)Hkv * c->force_splits;
@@ -316,7 +318,7 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
             for (int64_t g = Hkv + 1; g <= 2 * Hkv && g * 4 <= Hkv * nt; ++g)
                 if (fill(g) > best) { best = fill(g); groups = g; }
         }
-        const int streams = attn_tc_streams(n, c->G);
+        const int streams = c->tc32 ? 1 : attn_tc_streams(n, c->G);
         const int64_t slots_cap = part_rows_cap / ((int64_t)n * c->G) / streams;   // slots = streams * (groups + Hkv - 1)
         if (groups + Hkv - 1 > slots_cap) groups = slots_cap - (Hkv - 1);
         if (groups > Hkv * nt) groups = Hkv * nt;
@@ -435,7 +437,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
     aa.splits = plan.tc ? 1 : plan.splits;
     aa.ngroups = plan.ngroups;
-    aa.streams = plan.tc ? attn_tc_streams(n, c->G) : 1;
+    aa.streams = c->tc ? attn_tc_streams(n, c->G) : 1;
     aa.out_f32 = (f.dtype == KVF_F32 || (f.flags & KVF_OUT_F32)) ? 1 : 0;
     aa.scale_log2 = c->scale_log2;
 
@@ -452,7 +454,8 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     c->launches++;
     {
         ProfScope ps(c, st, 1);
-        if (plan.tc) e = launch_attn_tc(aa, c->maps, st);
+        if (c->tc) e = launch_attn_tc(aa, c->maps, st);
+        else if (c->tc32) e = launch_attn_tc32(aa, st);
         else e = launch_attn_simt(aa, f.dtype, st, nullptr);
     }
     if (e != cudaSuccess) return cuda_fail(e, "attention launch");
@@ -496,6 +499,7 @@ kvf_status init_handle(kvf_cache *c, const kvf_config *cfg, void *storage, void 
     c->launches = 0;
     c->profile = false;
     c->tc = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, c->G);
+    c->tc32 = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc32_supported(cfg->dtype, cfg->head_dim, c->G);
     return KVF_OK;
 }
 
@@ -686,7 +690,8 @@ kvf_status kvf_cache_status(kvf_cache *c) {
     int word = 0;
     cudaError_t e = cudaMemcpy(&word, c->workspace + c->lay.status, sizeof(int), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
-    return word == 0 ? KVF_OK : KVF_ERR_TIMEOUT;
+    if (word == 0) return KVF_OK;
+    return (word & 0xFF) == KVF_ERR_RANGE ? KVF_ERR_RANGE : KVF_ERR_TIMEOUT;
 }
 
 int32_t kvf_cache_status_word(kvf_cache *c) {
@@ -695,6 +700,16 @@ int32_t kvf_cache_status_word(kvf_cache *c) {
     cudaError_t e = cudaMemcpy(&word, c->workspace + c->lay.status, sizeof(int), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) { cuda_fail(e, "cudaMemcpy(status)"); return -1; }
     return word;
+}
+
+kvf_status kvf_cache_sm_clock(kvf_cache *c, uint64_t cycles_ns[2]) {
+    if (!c || !cycles_ns) return KVF_ERR_INVALID_ARG;
+    unsigned long long ctr[2] = {0, 0};
+    cudaError_t e = cudaMemcpy(ctr, c->workspace + c->lay.status + 16, sizeof(ctr), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(clock counters)");
+    cycles_ns[0] = ctr[0];
+    cycles_ns[1] = ctr[1];
+    return KVF_OK;
 }
 
 void *kvf_cache_k_plane(const kvf_cache *c) { return c && !c->page_table ? c->storage : nullptr; }
@@ -988,6 +1003,7 @@ const char *kvf_status_str(kvf_status s) {
         case KVF_ERR_CUDA: return "KVF_ERR_CUDA";
         case KVF_ERR_TIMEOUT: return "KVF_ERR_TIMEOUT";
         case KVF_ERR_POS: return "KVF_ERR_POS";
+        case KVF_ERR_RANGE: return "KVF_ERR_RANGE";
     }
     return "KVF_ERR_UNKNOWN";
 }

@@ -173,4 +173,10 @@ int attn_tc_streams(int n, int G);     // 2 when the chunk fits one 128-row tile
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s);   // grid (row pairs, ngroups)
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s);                // needed when ngroups != Hkv
 
+// Tensor-core path for fp32 caches (head_dim 128): operands split into fp16 halves, three MMAs per
+// product; contiguous planes, read straight from global memory (no tensor maps).
+bool attn_tc32_supported(int dtype, int d, int G);
+int attn_tc32_row_blocks(int n, int G);   // 128-row blocks per KV head = grid.x
+cudaError_t launch_attn_tc32(const AttnArgs &a, cudaStream_t s);                     // grid (row blocks, ngroups)
+
 }  // namespace kvf

@@ -114,3 +114,78 @@ def assert_within(res: ChainResult, dtype: str, what: str = ""):
     assert res.count > 0
     assert res.max_abs <= mx, f"{what}: max abs {res.max_abs:.3e} > {mx} (per step {res.per_step})"
     assert res.mean_abs <= mean, f"{what}: mean abs {res.mean_abs:.3e} > {mean}"
+
+
+# ------------------------------------------------------------------ cache contents, bit for bit
+def cache_rows(cache, kv: int, start: int, n: int, table: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Rows [start, start + n) of the K (kv = 0) or V (kv = 1) side of a cache as [Hkv, n, d]:
+    a slice of the plane, or for a paged cache the rows its page table names."""
+    if table is None:
+        plane = cache.v_plane() if kv else cache.k_plane()
+        return plane[:, start:start + n]
+    assert start % 128 == 0
+    pages = cache.page_rows(kv)[table[start // 128:(start + n + 127) // 128].long()]   # [pages, Hkv, 128, d]
+    rows = pages.permute(1, 0, 2, 3).reshape(pages.shape[1], -1, pages.shape[3])
+    return rows[:, :n]
+
+
+def ulp_distance(a: torch.Tensor, b: torch.Tensor) -> torch.Tensor:
+    """Distance in units of the last place between two bf16 or fp32 tensors of finite values."""
+    if a.dtype == torch.bfloat16:
+        ia, ib = a.view(torch.int16).to(torch.int64), b.view(torch.int16).to(torch.int64)
+        mag = 0x7FFF
+    else:
+        ia, ib = a.view(torch.int32).to(torch.int64), b.view(torch.int32).to(torch.int64)
+        mag = 0x7FFFFFFF
+    ia = torch.where(ia < 0, -(ia & mag), ia)          # sign-magnitude -> monotone integers
+    ib = torch.where(ib < 0, -(ib & mag), ib)
+    return (ia - ib).abs()
+
+
+class CacheBits:
+    """Accumulates the comparison of appended rows with what the paper's append must have left:
+    V rows verbatim, K rows equal to the oracle's rotation in the cache dtype and operation order
+    (contract: at most 1 ulp apart, and at most 1e-5 of all elements different at all, because the
+    device's and the host's fp64 cos/sin may differ in their last bit)."""
+
+    def __init__(self):
+        self.elements = 0
+        self.differing = 0
+        self.max_ulp = 0
+        self.v_equal = True
+
+    def add(self, cache, w: workloads.Workload, k: torch.Tensor, v: torch.Tensor, start: int, pos0: int,
+            interleaved: bool = False, table: Optional[torch.Tensor] = None):
+        n = k.shape[0]
+        tab = oracle.inv_freq(w.rope_base, w.head_dim)
+        want = oracle.rope_faithful(k.float().cpu().numpy(), pos0, tab, interleaved=interleaved,
+                                    to_bf16=(w.dtype == "bf16"))
+        want = torch.from_numpy(want).to(k.dtype).permute(1, 0, 2).contiguous().to(k.device)     # [Hkv, n, d]
+        dist = ulp_distance(cache_rows(cache, 0, start, n, table).contiguous(), want)
+        self.elements += dist.numel()
+        self.differing += int((dist != 0).sum())
+        self.max_ulp = max(self.max_ulp, int(dist.max()))
+        got_v = cache_rows(cache, 1, start, n, table).contiguous()
+        self.v_equal = self.v_equal and bool(torch.equal(got_v.view(torch.uint8),
+                                                         v.permute(1, 0, 2).contiguous().view(torch.uint8)))
+
+    def check(self, what: str = ""):
+        assert self.elements > 0
+        assert self.v_equal, f"{what}: value rows are not the inputs verbatim"
+        assert self.max_ulp <= 1, f"{what}: a key element is {self.max_ulp} ulp from the oracle's rotation"
+        assert self.differing <= 1e-5 * self.elements, f"{what}: {self.differing} of {self.elements} key elements differ"
+
+
+def assert_chain_cache_bits(cache, w: workloads.Workload, chunks: Sequence[int], seed: int, flags: int = 0,
+                            positions: Optional[Sequence[int]] = None, what: str = ""):
+    """Every row a chain of run_chain(w, chunks, seed) appended, compared in full (the chunks'
+    inputs are drawn again from their seeds)."""
+    bits = CacheBits()
+    start = 0
+    for t, n in enumerate(chunks):
+        _, k, v = workloads.chunk_inputs(w, seed, t, device="cuda", n_tokens=n)
+        bits.add(cache, w, k, v, start, start if positions is None else positions[t],
+                 interleaved=bool(flags & binding.KVF_ROPE_INTERLEAVED))
+        start += n
+    bits.check(what)
+    return bits

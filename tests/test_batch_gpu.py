@@ -194,3 +194,23 @@ def test_ragged_batch_members_of_different_length():
     with pytest.raises(binding.KvfError) as e:
         batch.fold_step(q, k, v, ragged=True)
     assert e.value.code == binding.KVF_ERR_UNSUPPORTED
+
+
+def test_batch_status_word_written_from_the_host_is_read_back():
+    """The batch's own status word, planted by the test (no device-side wait is made to give up)."""
+    cfg, pool, tables, caches = make_members(2, 512, 256, seed=17)
+    batch = binding.Batch(caches)
+    q, k, v = batch_inputs(2, 256, 41, 0)
+    batch.fold_step(q, k, v)
+    torch.cuda.synchronize()
+    assert batch.status_word() == 0
+    word = 5 | (22 << 8) | (9 << 16) | (1 << 24)
+    batch.workspace[:4].view(torch.int32).fill_(word)
+    torch.cuda.synchronize()
+    got = batch.status_word()
+    assert got == word and (got & 0xFF) == binding.KVF_ERR_TIMEOUT
+    assert ((got >> 8) & 0xFF, (got >> 16) & 0xFF, (got >> 24) & 1) == (22, 9, 1)
+    assert all(c.status() == binding.KVF_OK for c in caches)        # the members' own words are untouched
+    batch.workspace[:4].zero_()
+    torch.cuda.synchronize()
+    assert batch.status_word() == 0

@@ -9,44 +9,59 @@ import torch
 
 import oracle
 from paper_2605_12471_b200 import binding, workloads
-from tests.chain import TOL, assert_within, run_chain, to_f64
+from tests.chain import TOL, CacheBits, assert_chain_cache_bits, assert_within, run_chain, to_f64
 
 pytestmark = pytest.mark.gpu
 
 
-def _steps(n_steps, rng, extra=3):
+def _steps(n_steps, rng, extra=8):
+    """Checked steps of a long chain: seven fixed ones and `extra` seeded-random ones."""
     fixed = {0, 1, 2, n_steps // 4, n_steps // 2, n_steps - 2, n_steps - 1}
     fixed = {s for s in fixed if 0 <= s < n_steps}
     fixed.update(int(x) for x in rng.integers(0, n_steps, size=extra))
     return sorted(fixed)
 
 
+# rows of a checked step: six fixed ones (first two, the two around the middle, last two) and ten
+# seeded-random ones (chain.sample_rows)
+ROWS_EXTRA = 10
+
+
 def test_config2_llama_16k_chunks_of_2048():
     w = workloads.LLAMA_16K
-    res, cache, _, _ = run_chain(w, [w.chunk] * w.n_steps, seed=21, rows_per_step=6)
+    chunks = [w.chunk] * w.n_steps
+    res, cache, _, _ = run_chain(w, chunks, seed=21, rows_per_step=ROWS_EXTRA)
     assert len(cache) == 16384
     assert_within(res, "bf16", "config 2")
     # inputs are scaled by 1/sqrt(128): outputs are ~1e-3, so the relative error is the telling one
     assert res.rel_rms <= 2e-2, res.rel_rms
+    # what the eight steps appended, every row of it
+    bits = assert_chain_cache_bits(cache, w, chunks, seed=21, what="config 2 cache")
+    assert bits.elements == 16384 * 8 * 128
 
 
 def test_config3_deep_chain_128k_depth_511():
     """The benchmark's launch configuration: 512 steps of 256 tokens, prefix up to 130 816."""
     w = workloads.DEEP_CHAIN
-    steps = _steps(w.n_steps, np.random.default_rng(3), extra=2)
-    res, cache, _, _ = run_chain(w, [w.chunk] * w.n_steps, seed=22, check_steps=steps, rows_per_step=2)
+    chunks = [w.chunk] * w.n_steps
+    steps = _steps(w.n_steps, np.random.default_rng(3))
+    res, cache, _, _ = run_chain(w, chunks, seed=22, check_steps=steps, rows_per_step=ROWS_EXTRA)
     assert len(cache) == 131072 == 512 * 256
     assert_within(res, "bf16", "config 3")
     assert res.rel_rms <= 2e-2, res.rel_rms
     print("config3 drift per checked step (max abs):", {k: f"{v:.2e}" for k, v in sorted(res.per_step.items())})
+    # the final cache in full: 131 072 rows x 8 KV heads, keys against the oracle's rotation, values verbatim
+    bits = assert_chain_cache_bits(cache, w, chunks, seed=22, what="config 3 cache")
+    assert bits.elements == 131072 * 8 * 128
+    print(f"config3 cache: {bits.differing} of {bits.elements} key elements differ, max {bits.max_ulp} ulp")
 
 
 @pytest.mark.parametrize("C", [128, 512, 2048, 8192])
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_config4_chunk_and_precision_sweep_64k(C, dtype):
     w = workloads.sweep(C, dtype)
-    steps = _steps(w.n_steps, np.random.default_rng(C), extra=1)
-    res, cache, _, _ = run_chain(w, [C] * w.n_steps, seed=23, check_steps=steps, rows_per_step=1)
+    steps = _steps(w.n_steps, np.random.default_rng(C))
+    res, cache, _, _ = run_chain(w, [C] * w.n_steps, seed=23, check_steps=steps, rows_per_step=ROWS_EXTRA)
     assert len(cache) == 65536
     assert_within(res, dtype, f"config 4 C={C} {dtype}")
     print(f"config4 C={C} {dtype}: max {res.max_abs:.2e} mean {res.mean_abs:.2e} rel_rms {res.rel_rms:.2e}")
@@ -115,6 +130,7 @@ def test_config5_full_stack_64_gib_sampled_pairs(batched):
         outs = {key: torch.empty_like(inputs[key][0]) for key in watched}
         scratch = torch.empty_like(inputs[keys[0]][0])
     worst, err_sq, ref_sq = 0.0, 0.0, 0.0
+    bits = {key: CacheBits() for key in watched + [keys[0], keys[-1]]}       # the two watched pairs, first and last
     for t in range(N):
         if batched:
             batch.fold_step(bq, bk, bv, out=bout)
@@ -122,6 +138,10 @@ def test_config5_full_stack_64_gib_sampled_pairs(batched):
             for key in keys:
                 q, k, v = inputs[key]
                 caches[key].fold_step(q, k, v, out=outs[key] if key in outs else scratch)
+        # the rows this chunk appended to the watched caches, every element (chunk t starts at row t * C)
+        for key, cb in bits.items():
+            _, k, v = inputs[key]
+            cb.add(caches[key], w, k, v, t * C, t * C, table=tables[keys.index(key)] if batched else None)
         for key in watched:
             q, k, v = host_in[key]
             if t in check_chunks:
@@ -139,4 +159,7 @@ def test_config5_full_stack_64_gib_sampled_pairs(batched):
         assert batch.status_word() == 0 and batch.launch_count() == 2 * N     # rotate+append and attention, no combine
     assert worst <= TOL["bf16"][0], worst
     assert (err_sq / ref_sq) ** 0.5 <= 2e-2
+    for key, cb in bits.items():
+        cb.check(f"config 5 cache of sequence {key[0]}, layer {key[1]}")
+        assert cb.elements == T * w.n_kv_heads * w.head_dim
     print(f"config5 full size: max abs {worst:.2e}, rel rms {(err_sq / ref_sq) ** 0.5:.2e}")

@@ -136,9 +136,51 @@ def test_small_llama_bf16_matches_oracle(flags):
     assert res.lse_max_abs <= 2e-2
 
 
-def test_small_llama_f32_matches_oracle():
-    res, _, _, _ = run_chain(SMALL_LLAMA_F32, [256] * 3, seed=8)
-    assert_within(res, "f32", "small llama f32")
+@pytest.mark.parametrize("flags", [0, binding.KVF_FORCE_SIMT], ids=["tensor_cores_fp16_halves", "cuda_cores"])
+def test_small_llama_f32_matches_oracle(flags):
+    """fp32 caches, head_dim 128: the tensor-core kernel on fp16 halves of the operands (three MMAs per
+    product, output summed in fp32 registers) and the CUDA-core kernel both meet 1e-5."""
+    res, cache, _, _ = run_chain(SMALL_LLAMA_F32, [256] * 3, seed=8, flags=flags)
+    assert cache.plan(256, 512)[0] == (0 if flags else 1)
+    assert_within(res, "f32", f"small llama f32 flags={flags}")
+    assert res.lse_max_abs <= 1e-5
+
+
+def test_f32_tensor_core_path_on_a_deeper_ragged_chain_with_small_and_large_inputs():
+    """Chunks that leave ragged tails in the 64-key steps and the 128-row blocks, a prefix deep enough
+    for split key ranges, and inputs scaled down (1/sqrt(128), as the 16K configuration) and up (x 2):
+    the split into fp16 halves keeps an absolute 2^-25 on small elements and 22 bits on large ones.
+    (Inputs twice as large make logits four times and values twice as large: the absolute bound is
+    scaled by that factor of eight.)"""
+    for scale, seed in ((1.0, 41), (128 ** -0.5, 42), (2.0, 43)):
+        w = SMALL_LLAMA_F32.with_(name=f"f32_ragged_{scale:.3f}", tokens=8192, input_scale=scale)
+        chunks = [2048, 1000, 333, 256, 65, 64, 63, 1, 129, 2048, 31, 700]
+        check = [1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11]
+        res, cache, _, _ = run_chain(w, chunks, seed=seed, check_steps=check, rows_per_step=6)
+        assert cache.plan(256, 4096)[0] == 1
+        tol = TOL["f32"][0] * max(1.0, scale ** 3)
+        assert res.count > 0 and res.max_abs <= tol, (scale, res.max_abs, res.per_step)
+        assert res.lse_max_abs <= 1e-5 * max(1.0, scale * scale)
+
+
+def test_f32_tensor_core_path_flags_magnitudes_beyond_fp16_range():
+    """A key element of 1e5 cannot be split into fp16 halves: the step still runs to its end and the
+    status word says KVF_ERR_RANGE; the CUDA-core kernel takes the same inputs without complaint."""
+    w = SMALL_LLAMA_F32.with_(name="f32_range")
+    q, k, v = workloads.chunk_inputs(w, 44, 0, device="cuda")
+    k[3, 2, 17] = 1.0e5
+    cache = binding.cache_for(w)
+    cache.fold_step(q, k, v)
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_ERR_RANGE and (cache.status_word() & 0xFF) == 7
+    assert binding.load().kvf_status_str(cache.status()).decode() == "KVF_ERR_RANGE"
+    simt = binding.cache_for(w, flags=binding.KVF_FORCE_SIMT)
+    out = simt.fold_step(q, k, v)
+    torch.cuda.synchronize()
+    assert simt.status() == binding.KVF_OK and torch.isfinite(out).all()
+    oc = oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, w.chunk, rope_base=w.rope_base)
+    ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v))
+    assert np.abs(to_f64(out) - ref).max() <= TOL["f32"][0]
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
@@ -159,7 +201,8 @@ def test_out_f32_flag_and_interleaved_rotation(dtype):
     assert_within(res, dtype, "out_f32+interleaved")
 
 
-@pytest.mark.parametrize("dtype,flags", [("bf16", 0), ("bf16", binding.KVF_FORCE_SIMT), ("f32", 0)])
+@pytest.mark.parametrize("dtype,flags", [("bf16", 0), ("bf16", binding.KVF_FORCE_SIMT), ("f32", 0),
+                                         ("f32", binding.KVF_FORCE_SIMT)])
 def test_split_counts_agree_with_each_other_and_with_the_oracle(dtype, flags):
     w = SMALL_LLAMA.with_(name=f"split_{dtype}", dtype=dtype, tokens=4096)
     chunks = [2048, 256, 100, 1, 64]
@@ -266,6 +309,33 @@ def test_errors_are_return_codes_and_change_nothing():
     assert lib.kvf_cache_len(None) == -1
     torch.cuda.synchronize()
     assert cache.status() == binding.KVF_OK
+
+
+def test_status_word_written_from_the_host_is_reported_as_a_timed_out_wait():
+    """The path a bounded device-side wait takes when it gives up, without making any wait give up:
+    the test itself writes the word such a wait would leave (low byte 5 = timeout, then barrier 22,
+    warp 9, parity 1) into the cache's workspace and reads it back through the two entry points."""
+    lib = binding.load()
+    cache = binding.cache_for(SMALL_LLAMA)
+    q, k, v = workloads.chunk_inputs(SMALL_LLAMA, 40, 0, device="cuda")
+    cache.fold_step(q, k, v)
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_OK and cache.status_word() == 0
+    word = 5 | (22 << 8) | (9 << 16) | (1 << 24)
+    cache.workspace[:4].view(torch.int32).fill_(word)
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_ERR_TIMEOUT
+    assert lib.kvf_status_str(cache.status()).decode() == "KVF_ERR_TIMEOUT"
+    got = cache.status_word()
+    assert got == word
+    assert (got & 0xFF, (got >> 8) & 0xFF, (got >> 16) & 0xFF, (got >> 24) & 1) == (5, 22, 9, 1)
+    # the word is sticky until the owner of the workspace clears it; steps still run
+    cache.fold_step(q, k, v)
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_ERR_TIMEOUT and len(cache) == 2 * SMALL_LLAMA.chunk
+    cache.workspace[:4].zero_()
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_OK and cache.status_word() == 0
 
 
 def test_create_rejects_short_or_misaligned_buffers():

@@ -47,10 +47,22 @@ def test_tiny_fp32_window_matches_oracle_everywhere():
     assert worst <= TOL["f32"][0] and worst_lse <= 1e-5, (worst, worst_lse)
 
 
-def test_llama_fp32_window_with_forced_splits():
+@pytest.mark.parametrize("flags", [0, binding.KVF_FORCE_SIMT], ids=["tensor_cores", "cuda_cores"])
+def test_llama_fp32_window_with_forced_splits(flags):
     w = LLAMA.with_(name="window_llama_f32", dtype="f32")
-    worst, _, _, _ = run(w, [256, 256, 100, 256, 1, 256, 256], n_sink=4, window=300, seed=72, splits=3, rows_of=some_rows)
-    assert worst <= TOL["f32"][0], worst
+    worst, worst_lse, _, _ = run(w, [256, 256, 100, 256, 1, 256, 256], n_sink=4, window=300, seed=72, splits=3,
+                                 rows_of=some_rows, flags=flags)
+    assert worst <= TOL["f32"][0] and worst_lse <= 1e-5, (worst, worst_lse)
+
+
+def test_llama_fp32_paper_window_on_the_tensor_cores():
+    """4 sinks + 1020 recent on an fp32 cache: the sink tile, skipped tiles, a window that starts inside a
+    64-key step, ragged and single-token steps behind."""
+    w = LLAMA.with_(name="window_llama_f32_paper", dtype="f32")
+    chunks = [256] * 8 + [100, 1, 16, 300, 1, 256]
+    worst, worst_lse, _, cache = run(w, chunks, n_sink=4, window=1020, seed=75, rows_of=some_rows)
+    assert cache.plan(256, 2048)[0] == 1
+    assert worst <= TOL["f32"][0] and worst_lse <= 1e-5, (worst, worst_lse)
 
 
 def test_llama_bf16_paper_window_4_sinks_1020_recent():

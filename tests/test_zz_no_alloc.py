@@ -60,6 +60,11 @@ def test_static_scratch_step_fp32_and_small_heads():
     _same_chain(w, [64, 64, 33, 1, 200], seed=32)
 
 
+def test_static_scratch_step_fp32_on_the_tensor_cores():
+    w = workloads.Workload("static_llama_f32", 32, 8, 128, "f32", 256, 2048, 500000.0)
+    _same_chain(w, [256, 256, 256, 256, 100, 1, 64], seed=33)
+
+
 def test_static_scratch_rejects_sizes_beyond_its_fixed_maximum():
     lib = binding.load()
     cfg = binding.make_config(32, 8, 128, "bf16", 4096, 1024, rope_base=5e5)      # 1024 x 32 x 128 x 2 B = 8 MiB > 4 MiB
