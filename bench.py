@@ -567,7 +567,9 @@ def run_chain_bench(args, w, drift=False):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    cyc_a, ns_a = cache.sm_clock()
     ms = timed(run_chain, steps_timed)
+    cyc_b, ns_b = cache.sm_clock()
     clocks = sampler.stop() if rank == 0 else None
     assert graph is not None or len(cache) == T
     if cache.status() != binding.KVF_OK:
@@ -587,29 +589,38 @@ def run_chain_bench(args, w, drift=False):
     nvml = NvmlClock(local)
     nvml.start()
     t_prof0 = time.perf_counter()
-    tensor_shaped = w.dtype == "bf16" and not args.force_simt
+    tensor_shaped = cache.plan(C, T - C)[0] == 1
+    per_clock_rate = TENSOR_FLOP_PER_SM_CLOCK / (3.0 if w.dtype == "f32" else 1.0)
+    clock_cycles, clock_ns = 0, 0
     for bi in range(nbins):
         first, last = bi * N // nbins, (bi + 1) * N // nbins
         t0 = time.perf_counter()
+        cy0, ns0 = cache.sm_clock()
         body(first, last)
         bms, bcnt = cache.profile_read()
+        cy1, ns1 = cache.sm_clock()
         t1 = time.perf_counter()
         fl = sum(w.flops_step(visible(P0 + t * C), C) for t in range(first, last))
         by = sum(visible(P0 + t * C) + C for t in range(first, last)) * bytes_per_token
-        mhz = nvml.median_between(t0, t1)
+        # the clock the attention kernels of this bin ran at, from the kernels' own cycle and nanosecond counters
+        # (the NVML reading is kept beside it: it lags a power-capped clock)
+        mhz_nvml = nvml.median_between(t0, t1)
+        mhz = 1e3 * (cy1 - cy0) / (ns1 - ns0) if ns1 > ns0 else mhz_nvml
+        clock_cycles += cy1 - cy0
+        clock_ns += ns1 - ns0
         point = {"prefix_from": P0 + first * C, "prefix_to": P0 + (last - 1) * C,
                  "step_us": 1e3 * sum(bms) / (last - first), "attention_us": 1e3 * bms[1] / (last - first),
                  "attention_tflops": fl / (bms[1] * 1e-3) / 1e12, "cache_read_gbs": by / (bms[1] * 1e-3) / 1e9,
-                 "sm_mhz": mhz}
+                 "sm_mhz": mhz, "sm_mhz_nvml": mhz_nvml}
         if mhz:
             point["attention_kilocycles"] = 1e3 * bms[1] / (last - first) * mhz / 1e3
             if tensor_shaped:
-                point["tensor_flop_per_sm_clock_frac"] = fl / (bms[1] * 1e-3 * mhz * 1e6 * N_SMS * TENSOR_FLOP_PER_SM_CLOCK)
+                point["tensor_flop_per_sm_clock_frac"] = fl / (bms[1] * 1e-3 * mhz * 1e6 * N_SMS * per_clock_rate)
         curve.append(point)
         kms = [x + y for x, y in zip(kms, bms)]
         kcnt = [x + y for x, y in zip(kcnt, bcnt)]
     nvml.stop()
-    prof_mhz = nvml.median_between(t_prof0, time.perf_counter())
+    prof_mhz = 1e3 * clock_cycles / clock_ns if clock_ns else nvml.median_between(t_prof0, time.perf_counter())
     cache.profile(False)
     launches = (cache.launch_count() - l0) * steps_timed       # kernels of the timed chains
     pk = peaks()
@@ -657,6 +668,13 @@ def run_chain_bench(args, w, drift=False):
         per_clock = TENSOR_FLOP_PER_SM_CLOCK / (3.0 if w.dtype == "f32" else 1.0)
         roofline["sm_mhz_during_profile"] = prof_mhz
         roofline["frac_of_tensor_rate_at_sampled_clock"] = attn_tflops * 1e12 / (prof_mhz * 1e6 * N_SMS * per_clock)
+    if ns_b > ns_a:
+        # the attention kernels inside the timed chains themselves (no events between the kernels there): time and
+        # cycles the first CTA of every launch was running, from the kernels' own counters
+        in_ms = (ns_b - ns_a) * 1e-6 / steps_timed
+        roofline["in_timed_chains"] = {"attention_ms_per_chain": in_ms, "sm_mhz": 1e3 * (cyc_b - cyc_a) / (ns_b - ns_a),
+                                       "attention_tflops": attn_flops / (in_ms * 1e-3) / 1e12,
+                                       "other_ms_per_chain": ms / steps_timed - in_ms}
     roofline.update({
         "kernel": "prefix+chunk attention", "traffic": traffic, "traffic_source": NCU_TRAFFIC_SOURCE if traffic else None,
         "flops_per_launch": attn_flops / kcnt[1],

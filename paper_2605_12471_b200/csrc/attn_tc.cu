@@ -732,66 +732,78 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
 // a piece's softmax denominator and O_s its normalised output,
 //   O = sum_s 2^(lse_s - M) O_s / sum_s 2^(lse_s - M),  M = max_s lse_s,  in group order.
 // One block = kCombineTokens tokens of one KV head; one warp per row, lane = float4 column, so a
-// row of a piece is one coalesced 512-byte read and the weights are computed once per row.
-constexpr int kCombineTokens = 2;
-__global__ void __launch_bounds__(256) combine_groups_kernel(const AttnArgs a) {
+// row of a piece is one coalesced 512-byte read and the weights are computed once per row.  The
+// groups that touch a KV head come with the launch arguments when the host knows the row count
+// (AttnArgs::g_first / g_last); a ragged batch works them out per cache.  Up to eight pieces (the
+// usual case) are fetched together with their denominators, so a row costs one trip to memory.
+// (64 registers per thread: four blocks per SM, so that the blocks of a 256-token chunk - 512 of them -
+// are all resident at once instead of taking turns in waves)
+constexpr int kCombineTokens = 4;
+template <bool kFew>   // kFew: every KV head has at most eight parts (known on the host), the loops below run once
+__global__ void __launch_bounds__(256, kFew ? 4 : 2) combine_groups_kernel(const __grid_constant__ AttnArgs a) {
     __shared__ int g_range[2];
     const int kvh = blockIdx.y, G = a.G;
     const int cb = blockIdx.z;     // cache of a batch
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
-    if (a.prefixes) pdl_wait();   // ragged batch: the row counts were written by an earlier kernel of the stream
-    if (threadIdx.x == 0) {
-        const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix;
-        const int nt_all = (int)((P + a.n + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
-        const int64_t line = (int64_t)a.Hkv * nt_all;
-        auto start = [&](int64_t g) { return g * line / a.ngroups; };
-        auto group_of = [&](int64_t lin) {
-            int64_t g = lin * a.ngroups / line;
-            while (g > 0 && start(g) > lin) --g;
-            while (g + 1 < a.ngroups && start(g + 1) <= lin) ++g;
-            return (int)g;
-        };
-        g_range[0] = group_of((int64_t)kvh * nt_all);
-        g_range[1] = group_of((int64_t)(kvh + 1) * nt_all - 1);
+    int g0, g1;
+    if (a.range_valid && kvh < kRangeHeads) {
+        g0 = a.g_first[kvh];
+        g1 = a.g_last[kvh];
+    } else {
+        if (a.prefixes) pdl_wait();   // ragged batch: the row counts were written by an earlier kernel of the stream
+        if (threadIdx.x == 0) {
+            const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix;
+            const int nt_all = (int)((P + a.n + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
+            group_range(a.Hkv, nt_all, a.ngroups, kvh, g_range[0], g_range[1]);
+        }
+        __syncthreads();
+        g0 = g_range[0];
+        g1 = g_range[1];
     }
-    __syncthreads();
     pdl_wait();   // the parts are the attention kernel's output
     const int st = a.streams;
-    const int g0 = g_range[0], np = (g_range[1] - g0 + 1) * st;   // parts of this KV head: st per piece
-    // part s of the KV head sits in slot (g0 + s / st + kvh) * st + s % st
-    auto slot_of = [&](int s) { return (int64_t)(g0 + s / st + kvh) * st + s % st; };
+    const int np = (g1 - g0 + 1) * st;   // parts of this KV head: st per piece
+    // part s of the KV head sits in slot (g0 + s / st + kvh) * st + s % st = (g0 + kvh) * st + s
     const int64_t nG = (int64_t)a.n * G;
-    const float *part_o = a.part_o + cb * a.part_rows * kD;
-    const float *part_lse = a.part_lse + cb * a.part_rows;
+    const int64_t slot0 = (int64_t)(g0 + kvh) * st;
+    const float *part_o = a.part_o + (cb * a.part_rows + slot0 * nG) * kD + lane * 4;
+    const float *part_lse = a.part_lse + cb * a.part_rows + slot0 * nG;
     const int rows = kCombineTokens * G;                      // rows of this block, row = token * G + head-in-group
     for (int rr = warp; rr < rows; rr += 8) {
         const int tok = blockIdx.x * kCombineTokens + rr / G, gi = rr % G;
         if (tok >= a.n) break;
         const int64_t R = (int64_t)tok * G + gi;
         const int64_t row = ((int64_t)cb * a.n + tok) * a.H + kvh * G + gi;
-        float M = -INFINITY;
-        for (int s0 = 0; s0 < np; s0 += 32) {
-            const float ls = s0 + lane < np ? part_lse[slot_of(s0 + lane) * nG + R] : -INFINITY;
-            M = fmaxf(M, ls);
-        }
+        const float *po = part_o + R * kD;                    // part s: po + s * nG * kD
+        const float *pl = part_lse + R;                       //         pl + s * nG
+        // the first eight pieces (usually all of them) are fetched together with the denominators,
+        // so a row costs one trip to memory
+        float4 pv[8];
+#pragma unroll
+        for (int s = 0; s < 8; ++s)
+            if (s < np) pv[s] = *reinterpret_cast<const float4 *>(po + s * nG * kD);
+        float ls = lane < np ? pl[lane * nG] : -INFINITY;     // lane s holds the denominator of piece s (s < 32)
+        float M = ls;
+        if (!kFew)
+            for (int s = 32 + lane; s < np; s += 32) M = fmaxf(M, pl[s * nG]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
         float den = 0.f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s0 = 0; s0 < np; s0 += 8) {                  // 8 pieces at a time, loads issued together
+        for (int s0 = 0; s0 < (kFew ? 1 : np); s0 += 8) {     // 8 pieces at a time, in group order: deterministic
             const int cnt = min(8, np - s0);
-            float4 pv[8];
+            if (!kFew && s0 > 0) {
 #pragma unroll
-            for (int s = 0; s < 8; ++s)
-                if (s < cnt)
-                    pv[s] = *reinterpret_cast<const float4 *>(part_o + (slot_of(s0 + s) * nG + R) * kD + lane * 4);
-            const float ls = lane < cnt ? part_lse[slot_of(s0 + lane) * nG + R] : -INFINITY;
+                for (int s = 0; s < 8; ++s)
+                    if (s < cnt) pv[s] = *reinterpret_cast<const float4 *>(po + (s0 + s) * nG * kD);
+                if ((s0 & 31) == 0) ls = s0 + lane < np ? pl[(s0 + lane) * nG] : -INFINITY;
+            }
             const float wl = ls == -INFINITY ? 0.f : exp2f(ls - M);
 #pragma unroll
-            for (int s = 0; s < 8; ++s) {                     // group order: deterministic
+            for (int s = 0; s < 8; ++s) {
                 if (s < cnt) {
-                    const float w = __shfl_sync(0xffffffffu, wl, s);
+                    const float w = __shfl_sync(0xffffffffu, wl, (s0 + s) & 31);
                     den += w;
                     acc.x = fmaf(w, pv[s].x, acc.x); acc.y = fmaf(w, pv[s].y, acc.y);
                     acc.z = fmaf(w, pv[s].z, acc.z); acc.w = fmaf(w, pv[s].w, acc.w);
@@ -839,7 +851,12 @@ cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s
 
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s) {
     dim3 grid((a.n + kCombineTokens - 1) / kCombineTokens, a.Hkv, a.batch);
-    return launch_pdl(combine_groups_kernel, grid, dim3(256), 0, s, a);
+    // at most eight parts per KV head (two streams x four pieces, or eight pieces)?  The host knows when it
+    // worked out the groups of each head.
+    bool few = a.range_valid != 0 && a.Hkv <= kRangeHeads;
+    for (int h = 0; few && h < a.Hkv; ++h) few = (a.g_last[h] - a.g_first[h] + 1) * a.streams <= 8;
+    if (few) return launch_pdl(combine_groups_kernel<true>, grid, dim3(256), 0, s, a);
+    return launch_pdl(combine_groups_kernel<false>, grid, dim3(256), 0, s, a);
 }
 
 }  // namespace kvf

@@ -394,6 +394,19 @@ kvf_status check_ptr(const void *p) {
     return KVF_OK;
 }
 
+// The groups that touch each KV head, worked out once on the host for the combine kernel.
+void fill_group_ranges(AttnArgs &aa, int64_t nt_all) {
+    aa.range_valid = 0;
+    if (aa.ngroups <= 0 || aa.ngroups > 32767 || nt_all <= 0 || nt_all > (int64_t)1 << 30) return;
+    for (int h = 0; h < aa.Hkv && h < kRangeHeads; ++h) {
+        int g0, g1;
+        group_range(aa.Hkv, (int)nt_all, aa.ngroups, h, g0, g1);
+        aa.g_first[h] = (int16_t)g0;
+        aa.g_last[h] = (int16_t)g1;
+    }
+    aa.range_valid = 1;
+}
+
 kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void *v_new, int32_t n,
                      int64_t pos0, void *out, float *lse, cudaStream_t st) {
     const kvf_config &f = c->cfg;
@@ -440,6 +453,9 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.streams = c->tc ? attn_tc_streams(n, c->G) : 1;
     aa.out_f32 = (f.dtype == KVF_F32 || (f.flags & KVF_OUT_F32)) ? 1 : 0;
     aa.scale_log2 = c->scale_log2;
+    aa.range_valid = 0;
+    if (plan.tc && plan.kernels > 2)
+        fill_group_ranges(aa, (P + n + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip);
 
     cudaError_t e;
     if (c->quant) {
@@ -934,6 +950,9 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     aa.streams = attn_tc_streams(n, c0->G);
     aa.out_f32 = (f.flags & KVF_OUT_F32) ? 1 : 0;
     aa.scale_log2 = c0->scale_log2;
+    aa.range_valid = 0;
+    if (!ragged && plan.kernels > 2)
+        fill_group_ranges(aa, (P + n + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip);
 
     cudaError_t e = launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, B, st);
     if (e != cudaSuccess) return cuda_fail(e, "rope_append launch (batch)");

