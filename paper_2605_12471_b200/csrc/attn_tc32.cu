@@ -10,15 +10,15 @@
 // Here every fp32 operand x is split into two fp16 numbers, hi = fp16(x) and lo = fp16(x - hi),
 // which together carry 22 significant bits (elements below 2^-3 are kept to an absolute 2^-25,
 // the spacing of fp16 subnormals), and every product A B becomes three MMAs,
-//     A_hi B_lo + A_lo B_hi + A_hi B_hi          (the dropped A_lo B_lo term is below 2^-22),
-// issued in that order into one fp32 accumulator, so that the two small terms are summed before
-// the large one.  The accumulator of a tensor-core MMA is not rounded to nearest when it is
+//     A_hi B_hi + A_hi B_lo + A_lo B_hi          (the dropped A_lo B_lo term is below 2^-22),
+// each sum over a 64-key step only (scores) or over its 64 keys (output), in fp32 accumulators.  The accumulator of a tensor-core MMA is not rounded to nearest when it is
 // updated, which matters once thousands of updates pile up: O = P V is therefore accumulated in
 // tensor memory over ONE 64-key step only and then added, in round-to-nearest fp32, to the
-// running output row that the softmax thread keeps in registers.  Scores take 24 MMA updates
-// per 64-key step, the output 12.  fp16 holds magnitudes up to 65 504: a larger rotated key,
-// query or value sets code 7 (KVF_ERR_RANGE) in the device status word; such caches belong on
-// the CUDA-core kernel (KVF_FORCE_SIMT).
+// running output row that the softmax thread keeps in registers.  Scores take 16 MMA updates
+// per 64-key step, the output 12.  fp16 holds magnitudes up to 65 504: the rotate + append kernel
+// checks every rotated key and query and every value it writes for such a cache and sets code 7
+// (KVF_ERR_RANGE) in the device status word when one is larger; such caches belong on the
+// CUDA-core kernel (KVF_FORCE_SIMT).
 //
 // Work decomposition (as for the bf16 kernel, with 128-row blocks instead of 256-row pairs): row
 // = token * G + head-in-group; the (KV head, 128-key tile) pairs of a step form one line that is
@@ -33,15 +33,23 @@
 //               written back to tensor memory, the step's P V added to the 128 output registers
 //   warps 4-7   K converters: 16 rows of the step's K tile per warp, fp32 from global memory (one
 //               coalesced 512-byte row per warp instruction), split, written as 128-byte-swizzled
-//               K-major fp16 tiles (hi, lo) into a ring of three slots
-//   warps 8-11  V converters: the same for V (ring of two slots; a V tile is read MN-major, so its
-//               shared-memory image is that of a K tile); both converter groups also split the
-//               piece's 128 x 128 Q tile
-//   warp 12     MMA issuer (one thread) and owner of the tensor-memory allocation
-// Tensor memory: S0 | S1 (64 fp32 columns each) | P0 | P1 (hi: 32 columns, lo: 32 columns) | O (128).
-// Issue order QK(0) QK(1) PV(0) QK(2) PV(1) ...: the next step's scores are computed while the
-// softmax of the current step runs, and a step's P V is in flight while the softmax adds the
-// previous one.
+//               K-major fp16 tiles into a ring of three slots; in a slot the 64 rows of K_lo follow
+//               the 64 rows of K_hi inside each 64-column panel, so [K_hi; K_lo] is ONE 128-row operand
+//   warps 8-11  V converters: the same for V (ring of two slots, V_hi then V_lo; a V tile is read
+//               MN-major, so its rows are laid out as a K tile's); both converter groups also split
+//               the piece's 128 x 128 Q tile
+//   warp 12     issuer of the score MMAs (one thread) and owner of the tensor-memory allocation
+//   warp 13     issuer of the output MMAs (one thread)
+// One tcgen05.mma costs its issuing thread about as long as a 128 x 128 x 16 MMA runs, whatever its
+// N, so the kernel is built to issue few, wide MMAs from two threads: per 64-key step and 16
+// elements of d, Q_hi [K_hi; K_lo]^T is one MMA with N = 128 (its columns 0-63 are Q_hi K_hi, 64-127
+// the small term Q_hi K_lo) and Q_lo K_hi^T one with N = 64 added onto columns 0-63; the softmax
+// adds the two halves of a score.  16 score MMAs and 12 output MMAs per step (a first version with
+// 24 + 12 from one thread spent ~120 cycles per MMA on issue alone and left the tensor pipe 70 % idle).
+// Tensor memory: S0 | S1 (128 fp32 columns each: 64 scores + 64 small terms) | P0 | P1 (hi: 32
+// columns, lo: 32 columns) | O (128).  The score issuer runs ahead of the softmax by one step (S is
+// double-buffered), the output issuer starts a step's P V as soon as its probabilities are
+// written and the previous P V has been added to the registers.
 //
 // Every wait on an mbarrier is bounded and reports through the status word, as in the bf16 kernel.
 #include "kvfold_internal.h"
@@ -69,13 +77,13 @@ constexpr uint32_t kOffV = kOffK + kKSlots * kKSlot;
 constexpr uint32_t kOffCtl = kOffV + kVSlots * kKSlot;
 constexpr uint32_t kSmemBytes = kOffCtl + 512 + 1024;          // + control block + alignment slack
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColP = 128, kColO = 256;        // S0|S1 at 0, 64; P0|P1 at 128, 192; O at 256
+constexpr uint32_t kColS = 0, kColP = 256, kColO = 384;        // S0|S1 at 0, 128; P0|P1 at 256, 320; O at 384
+constexpr uint32_t kKOperand = 2 * kKPanel;                    // one 64-column panel of [K_hi; K_lo]: 128 rows
 constexpr float kRescaleThreshold = 8.0f;                      // log2 units
-constexpr float kHalfMax = 65504.0f;
 
 enum { B_QFULL = 0, B_QEMPTY = 1, B_KFULL0 = 2, B_KEMPTY0 = B_KFULL0 + kKSlots, B_VFULL0 = B_KEMPTY0 + kKSlots,
        B_VEMPTY0 = B_VFULL0 + kVSlots, B_SFULL0 = B_VEMPTY0 + kVSlots, B_SFREE0 = B_SFULL0 + 2, B_PFULL0 = B_SFREE0 + 2,
-       B_OFULL = B_PFULL0 + 2, B_OFREE = B_OFULL + 1, B_DRAIN = B_OFREE + 1, B_COUNT = B_DRAIN + 1 };
+       B_OFULL = B_PFULL0 + 2, B_OFREE = B_OFULL + 1, B_DRAIN0 = B_OFREE + 1, B_COUNT = B_DRAIN0 + 2 };
 
 struct Ctl {
     unsigned long long bars[32];
@@ -99,7 +107,8 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
 }
 // Instruction descriptors: D fp32, A and B fp16 (format 0), M = 128; scores N = 64, output N = 128
 // with B MN-major (bit 16).
-constexpr uint32_t kIdescQK = (1u << 4) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescQK64 = (1u << 4) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescQK128 = (1u << 4) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescPV = (1u << 4) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
 __device__ __forceinline__ uint32_t half2_bits(__half2 h) { return *reinterpret_cast<uint32_t *>(&h); }
@@ -114,18 +123,16 @@ __device__ __forceinline__ void split2(float a, float b, uint32_t &hi, uint32_t 
 
 // One fp32 row segment of four elements -> 8 bytes of hi and 8 bytes of lo at the swizzled place
 // of (row r, elements 4 * lane .. 4 * lane + 3) in a K-major tile whose panels hold `panel` bytes.
-__device__ __forceinline__ void store_split4(uint32_t part_hi, uint32_t part_lo, uint32_t panel, int r, int lane, float4 x) {
+// (Plain stores: the rows of a tile are independent, and the compiler may interleave their
+// conversions; the proxy fence and the barrier arrive behind the tile order them for the MMAs.)
+__device__ __forceinline__ void store_split4(uint8_t *part_hi, uint8_t *part_lo, uint32_t panel, int r, int lane, float4 x) {
     uint32_t h0, l0, h1, l1;
     split2(x.x, x.y, h0, l0);
     split2(x.z, x.w, h1, l1);
     const uint32_t off = (uint32_t)(lane >> 4) * panel + (uint32_t)r * 128u +
                          ((((uint32_t)(lane & 15) >> 1) ^ ((uint32_t)r & 7u)) << 4) + ((uint32_t)lane & 1u) * 8u;
-    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(part_hi + off), "r"(h0), "r"(h1) : "memory");
-    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(part_lo + off), "r"(l0), "r"(l1) : "memory");
-}
-
-__device__ __forceinline__ float amax4(float m, float4 x) {
-    return fmaxf(fmaxf(m, fmaxf(fabsf(x.x), fabsf(x.y))), fmaxf(fabsf(x.z), fabsf(x.w)));
+    *reinterpret_cast<uint2 *>(part_hi + off) = make_uint2(h0, h1);
+    *reinterpret_cast<uint2 *>(part_lo + off) = make_uint2(l0, l1);
 }
 
 // 16 columns x (32-bit) of this thread's TMEM lane <-> registers
@@ -139,14 +146,6 @@ __device__ __forceinline__ float amax4(float m, float4 x) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};" \
                  ::"r"(a[o + 0]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]), "r"(a[o + 5]), "r"(a[o + 6]), "r"(a[o + 7]), \
                    "r"(taddr) : "memory")
-
-// fp16 A and B: the same instruction as the bf16 kernel's with another instruction descriptor
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    tc_mma(d_tmem, a_desc, b_desc, idesc, accumulate);
-}
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    tc_mma_ts(d_tmem, a_tmem, b_desc, idesc, accumulate);
-}
 
 template <bool kWindow>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a) {
@@ -200,7 +199,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
         }
         mbar_init(bar(B_OFULL), 1);
         mbar_init(bar(B_OFREE), 4);
-        mbar_init(bar(B_DRAIN), 1);
+        mbar_init(bar(B_DRAIN0), 1);
+        mbar_init(bar(B_DRAIN0 + 1), 1);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -222,83 +222,79 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
     }
 
     if (warp >= 12) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
         if (warp == 12 && lane == 0) {
-            // ------------------------------------------------------------------ MMA issuer
-            const uint32_t q_hi = base + kOffQ, q_lo = q_hi + kQPart;
-            int g = 0;                   // steps issued so far (scores), all pieces
-            int gp = 0;                  // steps whose P V has been issued
+            // ------------------------------------------------------------------ issuer of the score MMAs
+            const uint64_t dqh = desc_kmajor(base + kOffQ), dql = desc_kmajor(base + kOffQ + kQPart);
+            int g = 0;                   // steps so far, all pieces = load number of the K ring
             int pc = 0;                  // pieces so far
             bool ok = true;
-            // scores of the step that is load number kc of the K ring, into S[g & 1]
-            auto issue_qk = [&](int kc) -> bool {
-                const int b = g & 1, slot = kc % kKSlots;
-                if (!mbar_wait(bar(B_SFREE0 + b), ((g >> 1) & 1) ^ 1, ctl, a.status)) return false;
-                if (!mbar_wait(bar(B_KFULL0 + slot), (kc / kKSlots) & 1, ctl, a.status)) return false;
-                tc_fence_after();
-                const uint32_t k_hi = base + kOffK + (uint32_t)slot * kKSlot, k_lo = k_hi + kKPart;
-                const uint32_t t_s = tmem + kColS + 64u * (uint32_t)b;
-                const uint64_t dqh = desc_kmajor(q_hi), dql = desc_kmajor(q_lo), dkh = desc_kmajor(k_hi), dkl = desc_kmajor(k_lo);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {          // 16 elements of d per MMA: the two small terms first
-                    const uint64_t qo = (uint64_t)(((kk >> 2) * kQPanel + (kk & 3) * 32) >> 4);
-                    const uint64_t ko = (uint64_t)(((kk >> 2) * kKPanel + (kk & 3) * 32) >> 4);
-                    mma_ss(t_s, dqh + qo, dkl + ko, kIdescQK, kk > 0);
-                    mma_ss(t_s, dql + qo, dkh + ko, kIdescQK, 1);
-                }
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint64_t qo = (uint64_t)(((kk >> 2) * kQPanel + (kk & 3) * 32) >> 4);
-                    const uint64_t ko = (uint64_t)(((kk >> 2) * kKPanel + (kk & 3) * 32) >> 4);
-                    mma_ss(t_s, dqh + qo, dkh + ko, kIdescQK, 1);
-                }
-                tc_commit(bar(B_SFULL0 + b));
-                tc_commit(bar(B_KEMPTY0 + slot));
-                ++g;
-                return true;
-            };
-            // O = P V of step number gp (V ring load number gp), fresh accumulator
-            auto issue_pv = [&]() -> bool {
-                const int b = gp & 1, slot = gp % kVSlots;
-                if (!mbar_wait(bar(B_VFULL0 + slot), (gp / kVSlots) & 1, ctl, a.status)) return false;
-                if (!mbar_wait(bar(B_PFULL0 + b), (gp >> 1) & 1, ctl, a.status)) return false;
-                if (gp > 0 && !mbar_wait(bar(B_OFREE), (gp - 1) & 1, ctl, a.status)) return false;
-                tc_fence_after();
-                const uint32_t v_hi = base + kOffV + (uint32_t)slot * kKSlot, v_lo = v_hi + kKPart;
-                const uint32_t p_hi = tmem + kColP + 64u * (uint32_t)b, p_lo = p_hi + 32u, t_o = tmem + kColO;
-                const uint64_t dvh = desc_mnmajor(v_hi), dvl = desc_mnmajor(v_lo);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {          // 16 keys = 8 packed columns of P per MMA
-                    const uint64_t vo = (uint64_t)((kk * 2048) >> 4);
-                    mma_ts(t_o, p_hi + kk * 8, dvl + vo, kIdescPV, kk > 0);
-                    mma_ts(t_o, p_lo + kk * 8, dvh + vo, kIdescPV, 1);
-                }
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    mma_ts(t_o, p_hi + kk * 8, dvh + (uint64_t)((kk * 2048) >> 4), kIdescPV, 1);
-                tc_commit(bar(B_OFULL));
-                tc_commit(bar(B_VEMPTY0 + slot));
-                ++gp;
-                return true;
-            };
             int kt0, ntiles, nsteps;
             for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles, nsteps); ++kvh) {
                 if (nsteps <= 0) continue;
                 ok = mbar_wait(bar(B_QFULL), pc & 1, ctl, a.status);
                 if (!ok) break;
-                tc_fence_after();
-                const int g0 = g;                      // K ring load number = step number (one K tile per step)
-                ok = issue_qk(g0);
-                for (int j = 0; j < nsteps && ok; ++j) {
-                    if (j + 1 < nsteps) ok = issue_qk(g0 + j + 1);
-                    if (j + 1 == nsteps) tc_commit(bar(B_QEMPTY));      // every Q K^T of this piece has been issued
-                    if (ok) ok = issue_pv();
+                for (int j = 0; j < nsteps; ++j, ++g) {
+                    const int b = g & 1, slot = g % kKSlots;
+                    ok = mbar_wait(bar(B_SFREE0 + b), ((g >> 1) & 1) ^ 1, ctl, a.status);
+                    if (ok) ok = mbar_wait(bar(B_KFULL0 + slot), (g / kKSlots) & 1, ctl, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t dk = desc_kmajor(base + kOffK + (uint32_t)slot * kKSlot);
+                    const uint32_t t_s = tmem + kColS + 128u * (uint32_t)b;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {          // 16 elements of d per MMA: Q_hi [K_hi; K_lo]^T, 128 columns
+                        const uint64_t qo = (uint64_t)(((kk >> 2) * kQPanel + (kk & 3) * 32) >> 4);
+                        const uint64_t ko = (uint64_t)(((kk >> 2) * kKOperand + (kk & 3) * 32) >> 4);
+                        tc_mma(t_s, dqh + qo, dk + ko, kIdescQK128, kk > 0);
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {          // Q_lo K_hi^T onto columns 0-63
+                        const uint64_t qo = (uint64_t)(((kk >> 2) * kQPanel + (kk & 3) * 32) >> 4);
+                        const uint64_t ko = (uint64_t)(((kk >> 2) * kKOperand + (kk & 3) * 32) >> 4);
+                        tc_mma(t_s, dql + qo, dk + ko, kIdescQK64, 1);
+                    }
+                    tc_commit(bar(B_SFULL0 + b));
+                    tc_commit(bar(B_KEMPTY0 + slot));
                 }
+                if (!ok) break;
+                tc_commit(bar(B_QEMPTY));                     // every Q K^T of this piece has been issued
                 ++pc;
             }
             // tensor memory is released only after every MMA issued here has run
-            tc_commit(bar(B_DRAIN));
-            mbar_wait_drain(bar(B_DRAIN), 0, a.status);
+            tc_commit(bar(B_DRAIN0));
+            mbar_wait_drain(bar(B_DRAIN0), 0, a.status);
+        } else if (warp == 13 && lane == 0) {
+            // ------------------------------------------------------------------ issuer of the output MMAs
+            int g = 0;                   // steps so far, all pieces = load number of the V ring
+            bool ok = true;
+            int kt0, ntiles, nsteps;
+            for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles, nsteps); ++kvh) {
+                for (int j = 0; j < nsteps; ++j, ++g) {
+                    const int b = g & 1, slot = g % kVSlots;
+                    ok = mbar_wait(bar(B_VFULL0 + slot), (g / kVSlots) & 1, ctl, a.status);
+                    if (ok) ok = mbar_wait(bar(B_PFULL0 + b), (g >> 1) & 1, ctl, a.status);
+                    if (ok && g > 0) ok = mbar_wait(bar(B_OFREE), (g - 1) & 1, ctl, a.status);   // the previous P V has been added
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t v_hi = base + kOffV + (uint32_t)slot * kKSlot;
+                    const uint32_t p_hi = tmem + kColP + 64u * (uint32_t)b, p_lo = p_hi + 32u, t_o = tmem + kColO;
+                    const uint64_t dvh = desc_mnmajor(v_hi), dvl = desc_mnmajor(v_hi + kKPart);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {          // 16 keys = 8 packed columns of P per MMA; small terms first
+                        const uint64_t vo = (uint64_t)((kk * 2048) >> 4);
+                        tc_mma_ts(t_o, p_hi + kk * 8, dvl + vo, kIdescPV, kk > 0);
+                        tc_mma_ts(t_o, p_lo + kk * 8, dvh + vo, kIdescPV, 1);
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        tc_mma_ts(t_o, p_hi + kk * 8, dvh + (uint64_t)((kk * 2048) >> 4), kIdescPV, 1);
+                    tc_commit(bar(B_OFULL));
+                    tc_commit(bar(B_VEMPTY0 + slot));
+                }
+            }
+            tc_commit(bar(B_DRAIN0 + 1));
+            mbar_wait_drain(bar(B_DRAIN0 + 1), 0, a.status);
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ converters: fp32 rows -> fp16 hi / lo tiles
@@ -309,10 +305,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
         const float *plane = reinterpret_cast<const float *>(is_v ? a.v_plane : a.k_plane);
         const float *q_rot = reinterpret_cast<const float *>(a.q_rot);
         const int nslots = is_v ? kVSlots : kKSlots;
-        const uint32_t ring = base + (is_v ? kOffV : kOffK);
+        const uint32_t ring = is_v ? kOffV : kOffK;
+        uint8_t *smem = smem_raw + (base - smem_u32(smem_raw));        // the 1024-byte aligned tile area
         const int b_full = is_v ? B_VFULL0 : B_KFULL0, b_empty = is_v ? B_VEMPTY0 : B_KEMPTY0;
         int lc = 0, pc = 0;                                  // ring loads and pieces so far
-        float amax = 0.f;
         bool ok = true;
         int kt0, ntiles, nsteps;
         for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles, nsteps); ++kvh) {
@@ -331,8 +327,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
                 if (!ok) break;
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    amax = amax4(amax, x[i]);
-                    store_split4(base + kOffQ, base + kOffQ + kQPart, kQPanel, w8 * 16 + i, lane, x[i]);
+                    store_split4(smem + kOffQ, smem + kOffQ + kQPart, kQPanel, w8 * 16 + i, lane, x[i]);
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read through the async proxy
                 __syncwarp();
@@ -354,22 +349,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
                 ok = mbar_wait(bar(b_empty + slot), ((lc / nslots) & 1) ^ 1, ctl, a.status);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                const uint32_t dst = ring + (uint32_t)slot * kKSlot;
+                // K: lo rows behind the hi rows inside each panel (one 128-row operand); V: hi tile, then lo tile
+                uint8_t *dst = smem + ring + (uint32_t)slot * kKSlot;
+                uint8_t *dst_lo = dst + (is_v ? kKPart : kKPanel);
+                const uint32_t panel = is_v ? kKPanel : kKOperand;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    amax = amax4(amax, x[i]);
-                    store_split4(dst, dst + kKPart, kKPanel, w4 * 16 + i, lane, x[i]);
-                }
+                for (int i = 0; i < 16; ++i) store_split4(dst, dst_lo, panel, w4 * 16 + i, lane, x[i]);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(b_full + slot));
             }
         }
-        // a magnitude fp16 cannot hold went into the split as infinity: say so
-        if (amax > kHalfMax) atomicCAS(a.status, 0, 7);
     } else {
         // ------------------------------------------------------------------ softmax and output rows, one thread per row
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 248;");
         const int r = warp * 32 + lane;                  // row of the CTA = TMEM lane
         const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
         const int R = row0 + r, tok = R / G, gi = R % G;
@@ -409,13 +402,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
                 got = __all_sync(0xffffffffu, got);
                 if (!got) return false;
                 tc_fence_after();
+                const bool rescale = __any_sync(0xffffffffu, scale != 1.f);      // rare: the reference moved at this step
+                const float2 sv = make_float2(scale, scale);
 #pragma unroll
-                for (int c0 = 0; c0 < kD; c0 += 16) {
-                    uint32_t t[16];
-                    KVF_TMEM_LD16(t, 0, t_o + c0);
+                for (int c0 = 0; c0 < kD; c0 += 32) {
+                    uint32_t t[32];
+                    KVF_TMEM_LD32(t, 0, t_o + c0);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) o[c0 + c] = (o[c0 + c] + __uint_as_float(t[c])) * scale;
+                    for (int c = 0; c < 32; c += 2) {
+                        float2 v = __fadd2_rn(make_float2(o[c0 + c], o[c0 + c + 1]), make_float2(__uint_as_float(t[c]), __uint_as_float(t[c + 1])));
+                        if (rescale) v = __fmul2_rn(v, sv);
+                        o[c0 + c] = v.x;
+                        o[c0 + c + 1] = v.y;
+                    }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -425,7 +425,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
 
             for (int j = 0; j < nsteps; ++j, ++g) {
                 const int b = g & 1;
-                const uint32_t t_s = tmem + lane_addr + kColS + 64u * (uint32_t)b;
+                const uint32_t t_s = tmem + lane_addr + kColS + 128u * (uint32_t)b;     // 64 scores, then their 64 small terms
                 const uint32_t t_p = tmem + lane_addr + kColP + 64u * (uint32_t)b;
                 ok = mbar_wait(bar(B_SFULL0 + b), (g >> 1) & 1, ctl, a.status);
                 ok = __all_sync(0xffffffffu, ok);
@@ -439,28 +439,38 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
                 const int sink_c = kWindow ? (int)max((int64_t)0, min((int64_t)kKeys, (int64_t)a.n_sink - key0)) : 0;
 
                 // first reading of the scores: the row maximum
-                float m_tile = -INFINITY;
+                // the step's 64 scores (columns c and 64 + c added up) into registers, and the row maximum
+                float v[64];
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    uint32_t sc[32];
+                    uint32_t sc[32], sx[32];
                     KVF_TMEM_LD32(sc, 0, t_s + 32 * h);
+                    KVF_TMEM_LD32(sx, 0, t_s + 64 + 32 * h);
                     tmem_wait_ld();
-                    if (masked) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            const int cc = 32 * h + c;
-                            sc[c] = (cc < nvis && (cc >= lo_c || cc < sink_c)) ? sc[c] : 0xFF800000u;   // -inf
-                        }
+                    for (int c = 0; c < 32; c += 2) {
+                        const float2 t = __fadd2_rn(make_float2(__uint_as_float(sc[c]), __uint_as_float(sc[c + 1])),
+                                                    make_float2(__uint_as_float(sx[c]), __uint_as_float(sx[c + 1])));
+                        v[32 * h + c] = t.x;
+                        v[32 * h + c + 1] = t.y;
                     }
-                    float mx[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) mx[q] = fmaxf(__uint_as_float(sc[2 * q]), __uint_as_float(sc[2 * q + 1]));
-#pragma unroll
-                    for (int c = 8; c < 32; c += 8)
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) mx[q] = max3(mx[q], __uint_as_float(sc[c + 2 * q]), __uint_as_float(sc[c + 2 * q + 1]));
-                    m_tile = fmaxf(m_tile, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])));
                 }
+                // the scores are in registers: the issuer may overwrite them with the step after next
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_SFREE0 + b));
+                if (masked) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) v[c] = (c < nvis && (c >= lo_c || c < sink_c)) ? v[c] : -INFINITY;
+                }
+                float mx[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) mx[q] = fmaxf(v[2 * q], v[2 * q + 1]);
+#pragma unroll
+                for (int c = 16; c < 64; c += 16)
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) mx[q] = max3(mx[q], v[c + 2 * q], v[c + 2 * q + 1]);
+                const float m_tile = fmaxf(max3(mx[0], mx[1], mx[2]), max3(max3(mx[3], mx[4], mx[5]), mx[6], mx[7]));
                 // move the reference only when the maximum grew by more than the threshold: the
                 // probabilities then stay below 2^threshold and the output row is rarely rescaled
                 const bool grow = (m_tile - m_ref) * sl2 > kRescaleThreshold;   // also true when m_ref = -inf < m_tile
@@ -473,39 +483,29 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
                 const float m_safe = m_ref == -INFINITY ? 0.f : m_ref;
                 const float neg = -m_safe * sl2;
 
-                // second reading: probabilities, split into fp16 hi / lo, 16 keys at a time
-                float acc0 = 0.f, acc1 = 0.f;
+                // probabilities, split into fp16 hi / lo, written 16 keys at a time
+                float2 acc = make_float2(0.f, 0.f);
+                const float2 sl2v = make_float2(sl2, sl2), negv = make_float2(neg, neg);
 #pragma unroll
                 for (int h = 0; h < 4; ++h) {
-                    uint32_t sc[16];
-                    KVF_TMEM_LD16(sc, 0, t_s + 16 * h);
-                    tmem_wait_ld();
-                    if (h == 3) {
-                        // the scores are in registers: the issuer may overwrite them with the step after next
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar(B_SFREE0 + b));
-                    }
-                    if (masked) {
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const int cc = 16 * h + c;
-                            sc[c] = (cc < nvis && (cc >= lo_c || cc < sink_c)) ? sc[c] : 0xFF800000u;
-                        }
-                    }
                     uint32_t ph[8], pl[8];
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
-                        const float e0 = ex2(fmaf(__uint_as_float(sc[2 * c]), sl2, neg));
-                        const float e1 = ex2(fmaf(__uint_as_float(sc[2 * c + 1]), sl2, neg));
-                        acc0 += e0;
-                        acc1 += e1;
-                        split2(e0, e1, ph[c], pl[c]);
+                        const float2 x = __ffma2_rn(make_float2(v[16 * h + 2 * c], v[16 * h + 2 * c + 1]), sl2v, negv);
+                        float2 e;
+                        e.x = ex2(x.x);
+                        e.y = ex2(x.y);
+                        acc = __fadd2_rn(acc, e);
+                        const __half2 hh = __floats2half2_rn(e.x, e.y);
+                        const float2 back = __half22float2(hh);
+                        const float2 rest = __fadd2_rn(e, make_float2(-back.x, -back.y));
+                        ph[c] = half2_bits(hh);
+                        pl[c] = half2_bits(__floats2half2_rn(rest.x, rest.y));
                     }
                     KVF_TMEM_ST8(ph, 0, t_p + 8 * h);
                     KVF_TMEM_ST8(pl, 0, t_p + 32 + 8 * h);
                 }
-                l += acc0 + acc1;
+                l += acc.x + acc.y;
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();

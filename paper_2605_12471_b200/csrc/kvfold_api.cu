@@ -430,6 +430,8 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     ra.page_elems = c->page_elems;
     ra.page_tables = nullptr;
     ra.prefixes = nullptr; ra.pos0s = nullptr;
+    ra.status = reinterpret_cast<int *>(c->workspace + c->lay.status);
+    ra.range_limit = c->tc32 ? 65504.f : 0.f;      // the fp32 tensor-core kernel computes on fp16 halves
     ra.table = c->table;
 
     AttnArgs aa;
@@ -929,6 +931,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     ra.page_tables = tables;
     ra.prefixes = ragged ? dev_prefixes : nullptr;
     ra.pos0s = ragged ? dev_pos0s : nullptr;
+    ra.status = nullptr; ra.range_limit = 0.f;
     ra.table = c0->table;
 
     AttnArgs aa;

@@ -95,6 +95,10 @@ struct RopeAppendArgs {
     // ragged batch: cache b holds prefixes[b] rows and its chunk starts at position pos0s[b]
     // (device arrays, or null: prefix and pos0 above hold for every cache)
     const int64_t *prefixes, *pos0s;
+    // fp32 cache whose attention runs on fp16 halves of its operands: a rotated query or key or a value
+    // above range_limit in magnitude sets code 7 in *status (range_limit = 0: no check)
+    int *status;
+    float range_limit;
     RopeTable table;
 };
 

@@ -123,6 +123,8 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
     const int rot_items = ntok * heads * rot_chunks;
     const int v_chunks = d / VEC;
     const int items = rot_items + ntok * a.Hkv * v_chunks;
+    float amax = 0.f;               // largest magnitude written (tracked only under a range limit, fp32 caches)
+    const bool ranged = sizeof(T) == 4 && a.range_limit > 0.f;
     for (int idx = threadIdx.x; idx < items; idx += kThreads) {
         if (idx >= rot_items) {
             const int i = idx - rot_items;
@@ -131,6 +133,9 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             const int t = i / (v_chunks * a.Hkv);
             const uint4 val = *reinterpret_cast<const uint4 *>(v + ((int64_t)(tok0 + t) * a.Hkv + g) * d + c * VEC);
             *reinterpret_cast<uint4 *>(vp + rows.offset(g, prefix + tok0 + t) + c * VEC) = val;
+            if (ranged)
+                amax = fmaxf(fmaxf(amax, fmaxf(fabsf(__uint_as_float(val.x)), fabsf(__uint_as_float(val.y)))),
+                             fmaxf(fabsf(__uint_as_float(val.z)), fabsf(__uint_as_float(val.w))));
             continue;
         }
         const int c = idx % rot_chunks;
@@ -157,6 +162,10 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             }
             Vec16<T>::store(dst + c * VEC, rlo);
             Vec16<T>::store(dst + half + c * VEC, rhi);
+            if (ranged) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) amax = fmaxf(amax, fmaxf(fabsf(rlo[e]), fabsf(rhi[e])));
+            }
         } else {
             float x[VEC], r[VEC];
             Vec16<T>::load(src + c * VEC, x);
@@ -166,8 +175,13 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
                 rotate(x[e], x[e + 1], w.x, w.y, r[e], r[e + 1]);
             }
             Vec16<T>::store(dst + c * VEC, r);
+            if (ranged) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) amax = fmaxf(amax, fabsf(r[e]));
+            }
         }
     }
+    if (ranged && amax > a.range_limit) atomicCAS(a.status, 0, 7);
 }
 
 }  // namespace
