@@ -469,7 +469,8 @@ def run_chain_bench(args, w, drift=False):
         w = w.with_(n_q_heads=q.shape[1], n_kv_heads=k.shape[1])
     H, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
     out = torch.empty_like(q)
-    flags = (binding.KVF_FORCE_SIMT if args.force_simt else 0) | binding.KVF_HOST_UPLOAD_AHEAD   # the flag touches host steps only
+    # (the two host-step flags touch kvf_fold_step_host only: uploads ahead of, result copies behind the steps)
+    flags = (binding.KVF_FORCE_SIMT if args.force_simt else 0) | binding.KVF_HOST_UPLOAD_AHEAD | binding.KVF_HOST_DOWNLOAD_BEHIND
     if args.cache_int8:
         flags |= binding.KVF_CACHE_INT8
     if args.cache_int4:
@@ -710,6 +711,7 @@ def run_chain_bench(args, w, drift=False):
                                             None, launch_stream[0])
                 if rc:
                     raise binding.KvfError(rc, "kvf_fold_step_host")
+            cache.host_flush()                               # the chain ends when its last results are in host memory
 
         prefill()
         body_host()

@@ -63,6 +63,14 @@ enum {
                                   t+1 runs while step t computes (the call's stream waits for the upload;
                                   results and errors are as without the flag).  Needs a workspace that no
                                   other cache's host steps use at the same time */
+    KVF_HOST_DOWNLOAD_BEHIND = 128u, /* kvf_fold_step_host copies a step's results (out, lse) back on a stream of
+                                  the library's own, behind the step, from one of two result staging sets, so
+                                  that the copy of step t runs while step t+1 computes instead of standing in
+                                  front of it on the caller's stream.  The contract on the results relaxes:
+                                  those of call t are in host memory once the caller's stream has passed the
+                                  end of call t+1, or of a kvf_cache_host_flush made after call t - not
+                                  already at the end of call t.  Can be combined with KVF_HOST_UPLOAD_AHEAD;
+                                  needs a workspace that no other cache's host steps use at the same time */
     KVF_CACHE_INT8 = 16u,      /* store the cache as int8 codes with one fp32 scale per row (one token of
                                   one KV head): d + 4 bytes per row instead of 2 d (kvf_cache_storage_bytes
                                   pads each head's scales to a multiple of 16 bytes).  The paper's Discussion
@@ -181,11 +189,18 @@ kvf_status kvf_fold_step(kvf_cache *c, const void *q, const void *k_new, const v
  * The same step with HOST buffers (pinned memory recommended): copies q/k/v to the workspace
  * staging area, runs the step, copies `out` (and lse if not NULL) back, all on `cuda_stream`
  * (with KVF_HOST_UPLOAD_AHEAD the three uploads run on an internal stream that `cuda_stream` then
- * waits for).  The host buffers must stay valid until the stream reaches the end of the call.
+ * waits for; with KVF_HOST_DOWNLOAD_BEHIND the results are copied back on an internal stream, see
+ * that flag for when they are there).  The host buffers must stay valid until the stream reaches
+ * the end of the call (result buffers under KVF_HOST_DOWNLOAD_BEHIND: until the results are there).
  */
 kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_host,
                               const void *v_host, int32_t n_tokens, int64_t pos0, void *out_host,
                               float *lse_host, void *cuda_stream);
+
+/* With KVF_HOST_DOWNLOAD_BEHIND: makes `cuda_stream` wait for the result copies of every host step
+ * enqueued so far (synchronising that stream afterwards means "all results are in host memory").
+ * Without the flag, or with nothing outstanding, it does nothing.  Enqueues waits only; returns at once. */
+kvf_status kvf_cache_host_flush(kvf_cache *c, void *cuda_stream);
 
 /* Tokens appended by all steps enqueued so far: the size of the accumulator (K,V)^(t) of Section
  * 2's left fold after t steps, which holds the rows of chunks 0..t (host counter; after t steps

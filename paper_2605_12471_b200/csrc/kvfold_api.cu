@@ -52,6 +52,7 @@ kvf_status check_config(const kvf_config *c) {
 struct Layout {
     size_t status, q_rot, st_q, st_k, st_v, st_out, st_lse, part_o, part_lse, total;
     size_t st_q2, st_k2, st_v2;   // second staging set (KVF_HOST_UPLOAD_AHEAD)
+    size_t st_out2, st_lse2;      // second result staging set (KVF_HOST_DOWNLOAD_BEHIND)
 };
 
 Layout workspace_layout(const kvf_config *c) {
@@ -75,6 +76,11 @@ Layout workspace_layout(const kvf_config *c) {
     }
     l.st_out = off;   off = align_up(off + ob, 1024);
     l.st_lse = off;   off = align_up(off + (size_t)c->max_chunk * c->n_q_heads * 4, 1024);
+    l.st_out2 = l.st_lse2 = 0;
+    if (c->flags & KVF_HOST_DOWNLOAD_BEHIND) {
+        l.st_out2 = off; off = align_up(off + ob, 1024);
+        l.st_lse2 = off; off = align_up(off + (size_t)c->max_chunk * c->n_q_heads * 4, 1024);
+    }
     l.part_o = off;   off = align_up(off + (size_t)kPartTokens * c->n_q_heads * c->head_dim * 4, 1024);
     l.part_lse = off; off = align_up(off + (size_t)kPartTokens * c->n_q_heads * 4, 1024);
     l.total = off;
@@ -115,6 +121,12 @@ struct kvf_cache {
     cudaEvent_t ev_up[2] = {nullptr, nullptr}, ev_read[2] = {nullptr, nullptr};
     bool ev_read_set[2] = {false, false};
     uint64_t host_steps = 0;
+    // KVF_HOST_DOWNLOAD_BEHIND: the library's download stream, "step done" (caller's stream) and "results
+    // copied" (download stream) events of the two result staging sets
+    cudaStream_t down_stream = nullptr;
+    cudaEvent_t ev_step[2] = {nullptr, nullptr}, ev_down[2] = {nullptr, nullptr};
+    bool ev_down_set[2] = {false, false};
+    uint64_t host_down_steps = 0;
     bool quant = false;                    // int8 storage: codes + scales in `storage`, bf16 image in the workspace
     QuantPlanes qp = {};
     int32_t n_sink = 0;                    // sink + window variant: rows always visible
@@ -305,6 +317,15 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
         } else if ((int64_t)pairs * Hkv * batch < c->sm_count) {
             groups = c->sm_count / (pairs * batch);
             if (groups > Hkv * nt / 4) groups = Hkv * nt / 4;
+            // A group count that is a multiple of the KV heads keeps every CTA inside one KV head: one Q load
+            // and one set of partial rows instead of two.  Measured at C = 256 (Llama shape): the second
+            // piece costs a CTA about as long as 3.3 key tiles, so while the line is short - here below
+            // ~12 K tokens - 128 aligned CTAs beat 148 that straddle KV heads.
+            const int64_t aligned = groups / Hkv * Hkv;
+            if (aligned >= Hkv && aligned < groups) {
+                const double line = (double)Hkv * (double)nt;
+                if (line / (double)aligned - line / (double)groups < 3.3) groups = aligned;
+            }
         } else {
             // whole KV heads fill the SMs, but the last wave may be half empty (256 CTAs on 148 SMs):
             // cut a little finer - up to twice the KV heads - if that fills the waves at least 5 %
@@ -679,8 +700,28 @@ kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_ho
         if (e == cudaSuccess) e = cudaMemcpyAsync(w + ov, v_host, kb, cudaMemcpyHostToDevice, st);
     }
     if (e != cudaSuccess) return cuda_fail(e, "host-to-device copy");
-    float *lse_dev = lse_host ? reinterpret_cast<float *>(w + c->lay.st_lse) : nullptr;
-    s = step_impl(c, w + oq, w + ok_, w + ov, n_tokens, pos0, w + c->lay.st_out, lse_dev, st);
+    const bool behind = (f.flags & KVF_HOST_DOWNLOAD_BEHIND) != 0;
+    int oset = 0;
+    size_t o_out = c->lay.st_out, o_lse = c->lay.st_lse;
+    if (behind) {
+        if (!c->down_stream) {
+            e = cudaStreamCreateWithFlags(&c->down_stream, cudaStreamNonBlocking);
+            for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+                e = cudaEventCreateWithFlags(&c->ev_step[i], cudaEventDisableTiming);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_down[i], cudaEventDisableTiming);
+            }
+            if (e != cudaSuccess) return cuda_fail(e, "download stream setup");
+        }
+        oset = (int)(c->host_down_steps & 1);
+        if (oset) { o_out = c->lay.st_out2; o_lse = c->lay.st_lse2; }
+        // this result set was last copied out two steps ago: the step must not overwrite it before that copy is done
+        if (c->ev_down_set[oset]) {
+            e = cudaStreamWaitEvent(st, c->ev_down[oset], 0);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaStreamWaitEvent(download)");
+        }
+    }
+    float *lse_dev = lse_host ? reinterpret_cast<float *>(w + o_lse) : nullptr;
+    s = step_impl(c, w + oq, w + ok_, w + ov, n_tokens, pos0, w + o_out, lse_dev, st);
     if (s != KVF_OK) return s;
     if (f.flags & KVF_HOST_UPLOAD_AHEAD) {
         e = cudaEventRecord(c->ev_read[set], st);      // (after the whole step: later than needed, never too early)
@@ -688,10 +729,41 @@ kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_ho
         c->ev_read_set[set] = true;
         c->host_steps++;
     }
-    e = cudaMemcpyAsync(out_host, w + c->lay.st_out, ob, cudaMemcpyDeviceToHost, st);
+    cudaStream_t ds = behind ? c->down_stream : st;
+    if (behind) {
+        // the copies of this step's results run on the library's stream, behind the step, while the caller's
+        // stream goes on with the next step
+        e = cudaEventRecord(c->ev_step[oset], st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ds, c->ev_step[oset], 0);
+        if (e != cudaSuccess) return cuda_fail(e, "download stream hand-over");
+    }
+    e = cudaMemcpyAsync(out_host, w + o_out, ob, cudaMemcpyDeviceToHost, ds);
     if (e == cudaSuccess && lse_host)
-        e = cudaMemcpyAsync(lse_host, lse_dev, (size_t)n_tokens * f.n_q_heads * 4, cudaMemcpyDeviceToHost, st);
+        e = cudaMemcpyAsync(lse_host, lse_dev, (size_t)n_tokens * f.n_q_heads * 4, cudaMemcpyDeviceToHost, ds);
     if (e != cudaSuccess) return cuda_fail(e, "device-to-host copy");
+    if (behind) {
+        e = cudaEventRecord(c->ev_down[oset], ds);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord(download)");
+        c->ev_down_set[oset] = true;
+        c->host_down_steps++;
+        // the step BEFORE this one has had this whole step to copy its results out: from here on the
+        // caller's stream is behind them
+        if (c->ev_down_set[oset ^ 1]) {
+            e = cudaStreamWaitEvent(st, c->ev_down[oset ^ 1], 0);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaStreamWaitEvent(previous download)");
+        }
+    }
+    return KVF_OK;
+}
+
+kvf_status kvf_cache_host_flush(kvf_cache *c, void *cuda_stream) {
+    if (!c) return KVF_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    for (int i = 0; i < 2; ++i) {
+        if (!c->ev_down_set[i]) continue;
+        cudaError_t e = cudaStreamWaitEvent(st, c->ev_down[i], 0);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaStreamWaitEvent(flush)");
+    }
     return KVF_OK;
 }
 
@@ -793,6 +865,11 @@ void kvf_cache_destroy(kvf_cache *c) {
         if (c->ev_read[i]) cudaEventDestroy(c->ev_read[i]);
     }
     if (c->up_stream) cudaStreamDestroy(c->up_stream);
+    for (int i = 0; i < 2; ++i) {
+        if (c->ev_step[i]) cudaEventDestroy(c->ev_step[i]);
+        if (c->ev_down[i]) cudaEventDestroy(c->ev_down[i]);
+    }
+    if (c->down_stream) cudaStreamDestroy(c->down_stream);
     delete c;
 }
 

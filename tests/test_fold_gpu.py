@@ -499,6 +499,44 @@ def test_host_steps_with_upload_ahead_enqueued_back_to_back():
         assert torch.equal(got[t].view(torch.int16), want[t].cpu().view(torch.int16)), t
 
 
+@pytest.mark.parametrize("flags", [binding.KVF_HOST_DOWNLOAD_BEHIND,
+                                   binding.KVF_HOST_DOWNLOAD_BEHIND | binding.KVF_HOST_UPLOAD_AHEAD],
+                         ids=["download_behind", "upload_ahead_and_download_behind"])
+def test_host_steps_with_results_copied_behind_the_next_step(flags):
+    """Eight host steps enqueued back to back with the result copies on the library's own stream (two
+    result staging sets, the copy of step t behind step t+1): the same bits as the device entry point,
+    and the relaxed contract - step t's results are there once the stream has passed call t+1, the last
+    step's after a flush."""
+    w = SMALL_LLAMA.with_(name="download_behind", tokens=2048)
+    dev = binding.cache_for(w)
+    host = binding.cache_for(w, flags=flags)
+    want, got, lses, keep = [], [], [], []
+    for t in range(8):
+        q, k, v = workloads.chunk_inputs(w, 19, t, device="cuda")
+        want.append(dev.fold_step(q, k, v))
+        keep.append(tuple(x.cpu().pin_memory() for x in (q, k, v)))
+        got.append(torch.zeros(q.shape, dtype=q.dtype).pin_memory())
+        lses.append(torch.zeros((w.chunk, w.n_q_heads), dtype=torch.float32).pin_memory())
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+    for t in range(7):
+        host.fold_step_host(*keep[t], got[t], lse=lses[t])
+    stream.synchronize()                     # the stream has passed the end of call 6: steps 0 .. 5 are there
+    for t in range(6):
+        assert torch.equal(got[t].view(torch.int16), want[t].cpu().view(torch.int16)), t
+    host.fold_step_host(*keep[7], got[7], lse=lses[7])
+    host.host_flush()
+    stream.synchronize()
+    assert host.status() == binding.KVF_OK and len(host) == 2048
+    for t in range(8):
+        assert torch.equal(got[t].view(torch.int16), want[t].cpu().view(torch.int16)), t
+        assert torch.isfinite(lses[t]).all() and float(lses[t].abs().max()) > 0
+    # a flush with nothing outstanding, and on a cache without the flag, is harmless
+    host.host_flush()
+    dev.host_flush()
+    torch.cuda.synchronize()
+
+
 def test_plan_fills_the_last_wave_when_whole_kv_heads_would_leave_it_half_empty():
     """148 SMs: 32 row pairs x 8 KV heads = 256 CTAs is 1.73 waves, 32 x 9 groups = 288 is 1.95; 128 row
     pairs x 8 = 1024 CTAs (6.9 waves) stays with whole KV heads and needs no combine kernel."""
@@ -511,3 +549,7 @@ def test_plan_fills_the_last_wave_when_whole_kv_heads_would_leave_it_half_empty(
     assert (tc, parts, ctas, kernels) == (1, 1, 128 * 8, 2)
     tc, parts, ctas, kernels = cache.plan(256, 130816 - 65536)      # the benchmark's chunk: one CTA per SM
     assert tc == 1 and ctas == (sms // 4) * 4 and kernels == 3
+    # a short line: 32 groups (4 per KV head, every CTA inside one KV head) instead of 37 that straddle heads
+    tc, parts, ctas, kernels = cache.plan(256, 2048)
+    if sms == 148:
+        assert (tc, parts, ctas, kernels) == (1, 4, 128, 3)
