@@ -79,9 +79,10 @@ enum {
                                   scale = max|x| / 127, code = clamp(rint(x * (127 / max|x|)), +-127) in
                                   fp32 (keys: on the rotated row before any rounding to bf16), and the
                                   attention sees bf16(code * scale).  dtype KVF_BF16 and head_dim 128
-                                  only (KVF_ERR_UNSUPPORTED otherwise, and for paged caches and
-                                  kvf_fold_step_static); the attention kernel expands code tiles to bf16
-                                  tiles in shared memory, so a step reads d + 4 bytes per cached row */
+                                  only (KVF_ERR_UNSUPPORTED otherwise, and for kvf_fold_step_static);
+                                  the attention kernel expands code tiles to bf16 tiles in shared
+                                  memory, so a step reads d + 4 bytes per cached row.  Paged caches and
+                                  batches of them take the flag too (see kvf_paged_cache_create) */
     KVF_CACHE_INT4 = 64u       /* the same with 4-bit codes (the other width the paper reports): scale =
                                   max|x| / 7, codes within +-7, stored two to a byte as code + 8 (element
                                   2i in the low nibble of byte i): d / 2 + 4 bytes per row.  Not together
@@ -150,8 +151,11 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
 /*
  * Paged variant of the accumulator (the paper's cache grows by appending; serving systems it
  * cites manage such caches in fixed-size pages - Related work, "Chunked serving infrastructure").  bf16 caches
- * with head_dim 128 only (KVF_ERR_UNSUPPORTED otherwise).
- *   A page holds 128 consecutive tokens of every KV head: [K|V][n_kv_heads][128][head_dim].
+ * with head_dim 128 only (KVF_ERR_UNSUPPORTED otherwise), stored as bf16 or, under KVF_CACHE_INT8 /
+ * KVF_CACHE_INT4, as codes and row scales.
+ *   A page holds 128 consecutive tokens of every KV head: [K|V][n_kv_heads][128][head_dim]; quantised:
+ *   [K codes|V codes][n_kv_heads][128][head_dim or head_dim / 2 bytes], then [K scales|V scales]
+ *   [n_kv_heads][128] fp32 (kvf_paged_pool_bytes counts both; the scale accessors return NULL).
  *   dev_pool        device, 256-byte aligned, n_pool_pages pages (kvf_paged_pool_bytes); pages may be
  *                   shared by many caches of the same shape
  *   dev_page_table  device int32 array, entry i = pool page of tokens [128 i, 128 i + 128); needs

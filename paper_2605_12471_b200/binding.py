@@ -363,10 +363,34 @@ class PagedCache(Cache):
     v_plane = k_plane
 
     def page_rows(self, kv: int) -> torch.Tensor:
-        """[pool pages, Hkv, 128, d] view of the K (kv = 0) or V (kv = 1) blocks of the pool."""
+        """[pool pages, Hkv, 128, d] view of the K (kv = 0) or V (kv = 1) blocks of the pool (bf16 pages)."""
         d, hkv = self.cfg.head_dim, self.cfg.n_kv_heads
         pages = self.storage.view(torch.bfloat16).view(-1, 2, hkv, 128, d)
         return pages[:, kv]
+
+    def _quant_page_bytes(self) -> Tuple[int, int]:
+        """(bytes of a page, bytes of one block of codes) of a quantised pool."""
+        d, hkv = self.cfg.head_dim, self.cfg.n_kv_heads
+        rb = d // 2 if self.cfg.flags & KVF_CACHE_INT4 else d
+        return 2 * hkv * 128 * rb + 2 * hkv * 128 * 4, hkv * 128 * rb
+
+    def page_codes(self, kv: int) -> torch.Tensor:
+        """[pool pages, Hkv, 128, d] int8 codes of the K (kv = 0) or V (kv = 1) blocks of a quantised pool
+        (a copy; int4 codes unpacked: element 2i is the low nibble of byte i, stored as code + 8)."""
+        d, hkv = self.cfg.head_dim, self.cfg.n_kv_heads
+        page, block = self._quant_page_bytes()
+        raw = self.storage.view(-1, page)[:, kv * block:(kv + 1) * block]
+        if self.cfg.flags & KVF_CACHE_INT4:
+            packed = raw.reshape(-1, hkv, 128, d // 2).to(torch.int16)
+            return (torch.stack([packed & 15, packed >> 4], dim=-1).reshape(-1, hkv, 128, d) - 8).to(torch.int8)
+        return raw.reshape(-1, hkv, 128, d).view(torch.int8).clone()
+
+    def page_scales(self, kv: int) -> torch.Tensor:
+        """[pool pages, Hkv, 128] fp32 row scales of the K (kv = 0) or V (kv = 1) rows of a quantised pool (a copy)."""
+        hkv = self.cfg.n_kv_heads
+        page, block = self._quant_page_bytes()
+        raw = self.storage.view(-1, page)[:, 2 * block + kv * hkv * 512:2 * block + (kv + 1) * hkv * 512]
+        return raw.contiguous().view(torch.float32).view(-1, hkv, 128)
 
 
 class Batch:

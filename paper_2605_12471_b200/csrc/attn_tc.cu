@@ -362,6 +362,16 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                         ok = mbar_wait(bar(B_RAWEMPTY0 + r), ((rg / kRawSlots) & 1) ^ 1, ctl, a.status);
                         if (!ok) break;
                         // ... and the rows' scales behind it (as many as the plane still holds)
+                        if (page_table) {
+                            // paged cache: a key tile is one page, which always holds its 128 rows and their scales
+                            if (!(t & 1)) page = page_table[ktile];                // K then V of the same tile
+                            const float *scales = ((t & 1) ? a.v_scales : a.k_scales) + (int64_t)page * a.scale_page_stride + kvh * kRows;
+                            mbar_expect_tx(bar(B_RAWFULL0 + r), rawBytes + kRows * 4u);
+                            tma_load_4d(base + kOffRawQ8 + (uint32_t)r * kRawBytes, m, bar(B_RAWFULL0 + r), 0, 0, kvh, page);
+                            bulk_load(base + kOffScaleQ8 + (uint32_t)r * 512u, scales, kRows * 4u, bar(B_RAWFULL0 + r));
+                            ++rg;
+                            continue;
+                        }
                         const int64_t left = a.scale_stride - key0;
                         const uint32_t sbytes = (uint32_t)(left < kRows ? left : kRows) * 4u;
                         const float *scales = ((t & 1) ? a.v_scales : a.k_scales) + (int64_t)kvh * a.scale_stride + key0;

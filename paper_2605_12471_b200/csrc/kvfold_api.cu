@@ -244,6 +244,25 @@ kvf_status build_maps(kvf_cache *c) {
                             (uint64_t)f.max_chunk, row, row * f.n_q_heads, d, (uint32_t)c->G,
                             (uint32_t)(128 / c->G));
     if (s != KVF_OK) return s;
+    if (c->page_table && c->quant) {
+        // pages of codes: (row bytes, row in page, KV head, page), the K and the V block of a page apart
+        const cuuint64_t rb = (cuuint64_t)d * c->qp.bits / 8;
+        for (int kv = 0; kv < 2; ++kv) {
+            cuuint64_t dims[4] = {rb, (cuuint64_t)kKvTile, (cuuint64_t)f.n_kv_heads, (cuuint64_t)c->n_pool_pages};
+            cuuint64_t strides[3] = {rb, rb * kKvTile, (cuuint64_t)c->qp.page_bytes};
+            cuuint32_t box[4] = {(cuuint32_t)rb, (cuuint32_t)kKvTile, 1u, 1u};
+            cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+            CUresult r = fn(kv ? &c->maps.v : &c->maps.k, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, kv ? (void *)c->qp.v_codes : (void *)c->qp.k_codes,
+                            dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            c->qp.bits == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) {
+                snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled (paged codes) failed with CUresult %d", (int)r);
+                return KVF_ERR_CUDA;
+            }
+        }
+        return KVF_OK;
+    }
     if (c->page_table) {
         const uint64_t page_bytes = (uint64_t)c->page_elems * 2;
         s = make_page_map(fn, &c->maps.k, c->storage, d, f.n_kv_heads, (uint64_t)c->n_pool_pages, page_bytes);
@@ -468,6 +487,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.k_scales = c->quant ? c->qp.k_scales : nullptr;
     aa.v_scales = c->quant ? c->qp.v_scales : nullptr;
     aa.scale_stride = c->qp.scale_stride;
+    aa.scale_page_stride = c->qp.page_bytes / 4;
     aa.quant_bits = c->quant ? c->qp.bits : 0;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
@@ -484,7 +504,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     if (c->quant) {
         // int8 storage: rotate + quantise + append (the attention kernel expands the code tiles itself)
         ProfScope ps(c, st, 0);
-        e = launch_rope_append_q8(ra, c->qp, (f.flags & KVF_ROPE_INTERLEAVED) != 0, st);
+        e = launch_rope_append_q8(ra, c->qp, (f.flags & KVF_ROPE_INTERLEAVED) != 0, 1, st);
     } else {
         ProfScope ps(c, st, 0);
         e = launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, 1, st);
@@ -540,6 +560,15 @@ kvf_status init_handle(kvf_cache *c, const kvf_config *cfg, void *storage, void 
     c->tc = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, c->G);
     c->tc32 = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc32_supported(cfg->dtype, cfg->head_dim, c->G);
     return KVF_OK;
+}
+
+// Bytes of one page: 128 tokens of every KV head, K block then V block; quantised caches keep the rows'
+// codes there and behind them one fp32 scale per row, K then V.
+size_t page_bytes_of(const kvf_config *cfg) {
+    const size_t rows = 2 * (size_t)cfg->n_kv_heads * kKvTile;
+    if (cfg->flags & (KVF_CACHE_INT8 | KVF_CACHE_INT4))
+        return rows * ((cfg->flags & KVF_CACHE_INT4) ? (size_t)cfg->head_dim / 2 : (size_t)cfg->head_dim) + rows * 4;
+    return rows * (size_t)cfg->head_dim * elem_bytes(cfg->dtype);
 }
 
 kvf_status check_step(kvf_cache *c, int32_t n, int64_t pos0) {
@@ -611,7 +640,7 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
 
 size_t kvf_paged_pool_bytes(const kvf_config *cfg, int32_t n_pages) {
     if (check_config(cfg) != KVF_OK || n_pages <= 0) return 0;
-    return (size_t)n_pages * 2 * (size_t)cfg->n_kv_heads * kKvTile * (size_t)cfg->head_dim * elem_bytes(cfg->dtype);
+    return (size_t)n_pages * page_bytes_of(cfg);
 }
 
 kvf_status kvf_paged_cache_create(const kvf_config *cfg, void *dev_pool, size_t pool_bytes, int32_t n_pool_pages,
@@ -623,7 +652,6 @@ kvf_status kvf_paged_cache_create(const kvf_config *cfg, void *dev_pool, size_t 
     if (s != KVF_OK) return s;
     const int G = cfg->n_q_heads / cfg->n_kv_heads;
     if ((cfg->flags & KVF_FORCE_SIMT) || !attn_tc_supported(cfg->dtype, cfg->head_dim, G)) return KVF_ERR_UNSUPPORTED;
-    if (cfg->flags & (KVF_CACHE_INT8 | KVF_CACHE_INT4)) return KVF_ERR_UNSUPPORTED;   // pages hold bf16 rows
     if (!dev_pool || !dev_workspace || !dev_page_table || n_pool_pages <= 0) return KVF_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(dev_pool) & 255u) || (reinterpret_cast<uintptr_t>(dev_workspace) & 255u) ||
         (reinterpret_cast<uintptr_t>(dev_page_table) & 3u))
@@ -639,6 +667,19 @@ kvf_status kvf_paged_cache_create(const kvf_config *cfg, void *dev_pool, size_t 
     c->n_pool_pages = n_pool_pages;
     c->page_elems = (int64_t)2 * cfg->n_kv_heads * kKvTile * cfg->head_dim;
     c->plane_bytes = (size_t)cfg->n_kv_heads * kKvTile * cfg->head_dim * elem_bytes(cfg->dtype);   // V block inside a page
+    if (cfg->flags & (KVF_CACHE_INT8 | KVF_CACHE_INT4)) {
+        // quantised pages: [K codes | V codes][Hkv][128][row bytes], then [K scales | V scales][Hkv][128] fp32
+        c->quant = true;
+        c->qp.bits = (cfg->flags & KVF_CACHE_INT4) ? 4 : 8;
+        const size_t codes = (size_t)cfg->n_kv_heads * kKvTile * cfg->head_dim * c->qp.bits / 8;   // one block of codes
+        c->plane_bytes = codes;
+        c->qp.page_bytes = (int64_t)page_bytes_of(cfg);
+        c->qp.k_codes = reinterpret_cast<int8_t *>(c->storage);
+        c->qp.v_codes = c->qp.k_codes + codes;
+        c->qp.k_scales = reinterpret_cast<float *>(c->storage + 2 * codes);
+        c->qp.v_scales = c->qp.k_scales + (size_t)cfg->n_kv_heads * kKvTile;
+        c->qp.scale_stride = 0;
+    }
     c->lay = workspace_layout(cfg);
     s = build_maps(c);
     if (s != KVF_OK) { delete c; return s; }
@@ -804,8 +845,8 @@ kvf_status kvf_cache_sm_clock(kvf_cache *c, uint64_t cycles_ns[2]) {
 
 void *kvf_cache_k_plane(const kvf_cache *c) { return c && !c->page_table ? c->storage : nullptr; }
 void *kvf_cache_v_plane(const kvf_cache *c) { return c && !c->page_table ? c->storage + c->plane_bytes : nullptr; }
-float *kvf_cache_k_scales(const kvf_cache *c) { return c && c->quant ? c->qp.k_scales : nullptr; }
-float *kvf_cache_v_scales(const kvf_cache *c) { return c && c->quant ? c->qp.v_scales : nullptr; }
+float *kvf_cache_k_scales(const kvf_cache *c) { return c && c->quant && !c->page_table ? c->qp.k_scales : nullptr; }
+float *kvf_cache_v_scales(const kvf_cache *c) { return c && c->quant && !c->page_table ? c->qp.v_scales : nullptr; }
 
 kvf_status kvf_cache_plan(const kvf_cache *c, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]) {
     if (!c || !plan || n_tokens < 1 || n_tokens > c->cfg.max_chunk || prefix_len < 0) return KVF_ERR_INVALID_ARG;
@@ -1022,7 +1063,11 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     aa.page_tables = tables; aa.part_rows = b->part_rows; aa.batch = B;
     aa.prefixes = ragged ? dev_prefixes : nullptr;
     aa.n_sink = c0->n_sink; aa.win_lo = window_lo(c0, P);
-    aa.k_scales = nullptr; aa.v_scales = nullptr; aa.scale_stride = 0; aa.quant_bits = 0;
+    aa.k_scales = c0->quant ? c0->qp.k_scales : nullptr;
+    aa.v_scales = c0->quant ? c0->qp.v_scales : nullptr;
+    aa.scale_stride = 0;
+    aa.scale_page_stride = c0->qp.page_bytes / 4;
+    aa.quant_bits = c0->quant ? c0->qp.bits : 0;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c0->G; aa.d = f.head_dim;
     aa.splits = 1;
@@ -1034,7 +1079,8 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     if (!ragged && plan.kernels > 2)
         fill_group_ranges(aa, (P + n + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip);
 
-    cudaError_t e = launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, B, st);
+    cudaError_t e = c0->quant ? launch_rope_append_q8(ra, c0->qp, (f.flags & KVF_ROPE_INTERLEAVED) != 0, B, st)
+                              : launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, B, st);
     if (e != cudaSuccess) return cuda_fail(e, "rope_append launch (batch)");
     b->launches++;
     TcMaps maps = c0->maps;

@@ -121,8 +121,9 @@ struct AttnArgs {
     int32_t batch;                   // caches in the launch (1 = one cache)
     const int64_t *prefixes;         // ragged batch: device array of the caches' row counts, else null
     const float *k_scales, *v_scales; // int8 storage: fp32 row scales [Hkv][scale_stride] (the tensor maps then
-                                     // describe the int8 code planes), else null
+                                     // describe the int8 code planes), else null; paged: the scale blocks of page 0
     int64_t scale_stride;            // capacity rounded up to a multiple of 4 (16-byte aligned rows of scales)
+    int64_t scale_page_stride;       // paged quantised cache: floats from one page's scale block to the next page's
     int32_t quant_bits;              // 0, 8 or 4
     // sink + window variant: of the rows before the chunk only those below n_sink or from win_lo on
     // are visible (win_lo = 0: all of them); see WindowTiles
@@ -174,13 +175,16 @@ constexpr int kMaxSinks = 64;         // sink rows sit in the first key tile of 
 
 // Quantised storage: int8 codes [Hkv][capacity][d] and one fp32 scale per row [Hkv][scale_stride],
 // scale_stride = capacity rounded up to a multiple of 4.
+// Paged: a page is kKvTile tokens of every KV head, [K codes | V codes][Hkv][kKvTile][row bytes] followed
+// by [K scales | V scales][Hkv][kKvTile] fp32; the pointers below are those blocks of page 0.
 struct QuantPlanes {
     int8_t *k_codes, *v_codes;       // int4: two codes to a byte (code + 8, element 2i in the low nibble of byte i)
     float *k_scales, *v_scales;
     int64_t scale_stride;
     int32_t bits;                    // 8 or 4
+    int64_t page_bytes;              // paged: bytes of one page (0 = contiguous planes)
 };
-cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, cudaStream_t s);
+cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, int batch, cudaStream_t s);
 
 cudaError_t launch_rope_append(const RopeAppendArgs &a, int dtype, bool interleaved, int batch, cudaStream_t s);
 cudaError_t launch_attn_simt(const AttnArgs &a, int dtype, cudaStream_t s, int *grid_out);

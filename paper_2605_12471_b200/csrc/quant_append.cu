@@ -10,7 +10,8 @@
 // rounding to bf16); a value row is quantised as given.  amax = 0 gives codes 0 and scale 0.
 // The cache then holds d + 4 (int8) or d / 2 + 4 (int4: code + 8, two to a byte, element 2i in the low
 // nibble of byte i) bytes per row instead of 2 d; the attention kernel expands code tiles to bf16 tiles
-// in shared memory.
+// in shared memory.  Paged caches keep codes and scales of 128 tokens of every KV head in one page
+// (see QuantPlanes); a batch of paged caches is one launch (blockIdx.y = cache).
 #include "kvfold_internal.h"
 
 namespace kvf {
@@ -56,11 +57,27 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tok0 = blockIdx.x * kTok;
     const int ntok = min(kTok, a.n - tok0);
+    const int b = blockIdx.y;      // cache of a batch (0 when there is one cache)
 
     pdl_launch_dependents();
+    // (the per-cache arrays of a ragged batch were written by an earlier kernel of the stream: under
+    // a dependent launch they are visible only after the wait)
+    if (a.prefixes || a.pos0s) pdl_wait();
+    const int64_t prefix = a.prefixes ? a.prefixes[b] : a.prefix;
+    const int64_t pos0 = a.pos0s ? a.pos0s[b] : a.pos0;
+    const int32_t *page_table = a.page_tables ? a.page_tables[b] : a.page_table;
+    // where row `row` of KV head g lives: byte offset of its codes from the code block, index of its scale
+    auto code_off = [&](int g, int64_t row) -> int64_t {
+        if (qp.page_bytes == 0) return ((int64_t)g * a.capacity + row) * RB;
+        return (int64_t)page_table[row / kKvTile] * qp.page_bytes + ((int64_t)g * kKvTile + row % kKvTile) * RB;
+    };
+    auto scale_idx = [&](int g, int64_t row) -> int64_t {
+        if (qp.page_bytes == 0) return (int64_t)g * qp.scale_stride + row;
+        return (int64_t)page_table[row / kKvTile] * (qp.page_bytes / 4) + (int64_t)g * kKvTile + row % kKvTile;
+    };
     for (int idx = threadIdx.x; idx < ntok * half; idx += kThreads) {
         int t = idx / half, j = idx % half;
-        double theta = (double)(a.pos0 + tok0 + t) * a.table.inv_freq[j];
+        double theta = (double)(pos0 + tok0 + t) * a.table.inv_freq[j];
         double sn, cn;
         sincos(theta, &sn, &cn);
         cs[t][j] = make_float2((float)cn, (float)sn);
@@ -71,19 +88,22 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
     // Rows between the new end of the cache and the next key-tile boundary get value scale 0: the
     // attention expands them to zeros whatever their codes are, so a zero probability never
     // multiplies non-finite bits.
-    if (blockIdx.x == 0)
-        for (int i = threadIdx.x; i < a.zero_rows * a.Hkv; i += kThreads)
-            qp.v_scales[(int64_t)(i / a.zero_rows) * qp.scale_stride + a.prefix + a.n + i % a.zero_rows] = 0.f;
+    if (blockIdx.x == 0) {
+        const int zero_rows = a.prefixes ? (int)((kKvTile - (prefix + a.n) % kKvTile) % kKvTile) : a.zero_rows;
+        for (int i = threadIdx.x; i < zero_rows * a.Hkv; i += kThreads)
+            qp.v_scales[scale_idx(i / zero_rows, prefix + a.n + i % zero_rows)] = 0.f;
+    }
 
-    const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(a.q);
-    const __nv_bfloat16 *k = reinterpret_cast<const __nv_bfloat16 *>(a.k_new);
-    const __nv_bfloat16 *v = reinterpret_cast<const __nv_bfloat16 *>(a.v_new);
-    __nv_bfloat16 *qr = reinterpret_cast<__nv_bfloat16 *>(a.q_rot);
+    const int64_t qoff = (int64_t)b * a.n * a.H * d, koff = (int64_t)b * a.n * a.Hkv * d;
+    const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(a.q) + qoff;
+    const __nv_bfloat16 *k = reinterpret_cast<const __nv_bfloat16 *>(a.k_new) + koff;
+    const __nv_bfloat16 *v = reinterpret_cast<const __nv_bfloat16 *>(a.v_new) + koff;
+    __nv_bfloat16 *qr = reinterpret_cast<__nv_bfloat16 *>(a.q_rot) + qoff;
     const int heads = a.H + 2 * a.Hkv;         // query rows, key rows, value rows
     for (int row = warp; row < ntok * heads; row += kThreads / 32) {
         const int t = row / heads, hh = row % heads;
         const int64_t tok = tok0 + t;
-        const int64_t cache_row = a.prefix + tok;
+        const int64_t cache_row = prefix + tok;
         if (hh >= a.H + a.Hkv) {
             // ---- value row: elements 4 lane .. 4 lane + 3
             const int g = hh - a.H - a.Hkv;
@@ -92,16 +112,16 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
             int code[4];
             float scale;
             quantise4<BITS>(x, code, scale);
-            const int64_t r = (int64_t)g * a.capacity + cache_row;
+            const int64_t r = code_off(g, cache_row);
             if (BITS == 8) {
                 const uint32_t packed = (uint32_t)(code[0] & 0xFF) | ((uint32_t)(code[1] & 0xFF) << 8) |
                                         ((uint32_t)(code[2] & 0xFF) << 16) | ((uint32_t)(code[3] & 0xFF) << 24);
-                *reinterpret_cast<uint32_t *>(qp.v_codes + r * RB + 4 * lane) = packed;
+                *reinterpret_cast<uint32_t *>(qp.v_codes + r + 4 * lane) = packed;
             } else {
-                *reinterpret_cast<uint16_t *>(qp.v_codes + r * RB + 2 * lane) =
+                *reinterpret_cast<uint16_t *>(qp.v_codes + r + 2 * lane) =
                     (uint16_t)((code[0] + 8) | ((code[1] + 8) << 4) | ((code[2] + 8) << 8) | ((code[3] + 8) << 12));
             }
-            if (lane == 0) qp.v_scales[(int64_t)g * qp.scale_stride + cache_row] = scale;
+            if (lane == 0) qp.v_scales[scale_idx(g, cache_row)] = scale;
             continue;
         }
         const bool is_q = hh < a.H;
@@ -134,30 +154,30 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
             int code[4];
             float scale;
             quantise4<BITS>(x, code, scale);
-            const int64_t r = (int64_t)g * a.capacity + cache_row;
+            const int64_t r = code_off(g, cache_row);
             if (BITS == 8) {
-                *reinterpret_cast<uint16_t *>(qp.k_codes + r * RB + e0) = (uint16_t)((code[0] & 0xFF) | ((code[1] & 0xFF) << 8));
-                *reinterpret_cast<uint16_t *>(qp.k_codes + r * RB + e1) = (uint16_t)((code[2] & 0xFF) | ((code[3] & 0xFF) << 8));
+                *reinterpret_cast<uint16_t *>(qp.k_codes + r + e0) = (uint16_t)((code[0] & 0xFF) | ((code[1] & 0xFF) << 8));
+                *reinterpret_cast<uint16_t *>(qp.k_codes + r + e1) = (uint16_t)((code[2] & 0xFF) | ((code[3] & 0xFF) << 8));
             } else {
                 // elements e0, e0 + 1 share byte e0 / 2 (e0 and e1 are even)
-                qp.k_codes[r * RB + e0 / 2] = (int8_t)((code[0] + 8) | ((code[1] + 8) << 4));
-                qp.k_codes[r * RB + e1 / 2] = (int8_t)((code[2] + 8) | ((code[3] + 8) << 4));
+                qp.k_codes[r + e0 / 2] = (int8_t)((code[0] + 8) | ((code[1] + 8) << 4));
+                qp.k_codes[r + e1 / 2] = (int8_t)((code[2] + 8) | ((code[3] + 8) << 4));
             }
-            if (lane == 0) qp.k_scales[(int64_t)g * qp.scale_stride + cache_row] = scale;
+            if (lane == 0) qp.k_scales[scale_idx(g, cache_row)] = scale;
         }
     }
 }
 
 }  // namespace
 
-cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, cudaStream_t s) {
-    const int blocks = (a.n + kTok - 1) / kTok;
+cudaError_t launch_rope_append_q8(const RopeAppendArgs &a, const QuantPlanes &qp, bool interleaved, int batch, cudaStream_t s) {
+    const dim3 grid((a.n + kTok - 1) / kTok, batch);
     if (qp.bits == 4) {
-        if (interleaved) return launch_pdl(rope_append_q8_kernel<true, 4>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
-        return launch_pdl(rope_append_q8_kernel<false, 4>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
+        if (interleaved) return launch_pdl(rope_append_q8_kernel<true, 4>, grid, dim3(kThreads), 0, s, a, qp);
+        return launch_pdl(rope_append_q8_kernel<false, 4>, grid, dim3(kThreads), 0, s, a, qp);
     }
-    if (interleaved) return launch_pdl(rope_append_q8_kernel<true, 8>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
-    return launch_pdl(rope_append_q8_kernel<false, 8>, dim3(blocks), dim3(kThreads), 0, s, a, qp);
+    if (interleaved) return launch_pdl(rope_append_q8_kernel<true, 8>, grid, dim3(kThreads), 0, s, a, qp);
+    return launch_pdl(rope_append_q8_kernel<false, 8>, grid, dim3(kThreads), 0, s, a, qp);
 }
 
 }  // namespace kvf

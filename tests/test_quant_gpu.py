@@ -94,9 +94,14 @@ def test_quantised_storage_rejects_what_it_does_not_cover():
     cfg = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5, flags=binding.KVF_CACHE_INT8)
     buf = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
     table = torch.zeros(8, dtype=torch.int32, device="cuda")
-    rc = lib.kvf_paged_cache_create(ctypes.byref(cfg), buf.data_ptr(), buf.numel(), 8, table.data_ptr(), buf.data_ptr(),
-                                    buf.numel(), ctypes.byref(h))
-    assert rc == binding.KVF_ERR_UNSUPPORTED
+    ws = torch.empty(binding.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    rc = lib.kvf_paged_cache_create(ctypes.byref(cfg), buf.data_ptr(), buf.numel(), 8, table.data_ptr(), ws.data_ptr(),
+                                    ws.numel(), ctypes.byref(h))
+    assert rc == binding.KVF_OK                     # quantised rows may live in pages (8 pages of 264 KiB fit 64 MiB)
+    lib.kvf_cache_destroy(h)
+    rc = lib.kvf_paged_cache_create(ctypes.byref(cfg), buf.data_ptr(), 8 * 270336 - 1, 8, table.data_ptr(), ws.data_ptr(),
+                                    ws.numel(), ctypes.byref(h))
+    assert rc == binding.KVF_ERR_CAPACITY           # a page holds 2 x 8 x 128 rows of 128 codes + 2 x 8 x 128 scales
     plain = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5)
     assert binding.workspace_bytes(cfg) == binding.workspace_bytes(plain)          # no bf16 image of the cache anywhere
 
@@ -179,3 +184,91 @@ def test_quantised_deep_chain_32k_sampled_steps(bits):
     torch.cuda.synchronize()
     assert cache.status() == binding.KVF_OK, hex(cache.status_word())
     assert worst <= TOL["bf16"][0] and (err_sq / ref_sq) ** 0.5 <= 2e-2, (worst, (err_sq / ref_sq) ** 0.5)
+
+
+# ------------------------------------------------------------------ quantised rows in pages, and batches of them
+def quant_paged_members(n_caches, capacity, max_chunk, bits, seed):
+    """n_caches paged caches with quantised storage over one pool, pages dealt from one shuffled deck."""
+    cfg = binding.make_config(W.n_q_heads, W.n_kv_heads, W.head_dim, "bf16", capacity, max_chunk, rope_base=W.rope_base,
+                              flags=binding.KVF_CACHE_INT4 if bits == 4 else binding.KVF_CACHE_INT8)
+    per = (capacity + 127) // 128
+    n_pool = n_caches * per + 2
+    deck = torch.randperm(n_pool, generator=torch.Generator().manual_seed(seed))[:n_caches * per].to(torch.int32)
+    tables = deck.view(n_caches, per).cuda()
+    pool = torch.empty(binding.paged_pool_bytes(cfg, n_pool), dtype=torch.uint8, device="cuda")
+    pool.fill_(0xFF)                                        # scale bits 0xFFFFFFFF = NaN wherever no row was written
+    ws = torch.empty(binding.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    caches = [binding.PagedCache(cfg, pool, n_pool, tables[i], workspace=ws) for i in range(n_caches)]
+    return cfg, pool, tables, caches
+
+
+@BITS
+def test_paged_quantised_cache_holds_the_same_codes_and_gives_the_same_bits(bits):
+    """Codes and scales in 128-token pages scattered over a pool: the same codes, scales and output bits as
+    the contiguous quantised cache (whose codes are the oracle's), ragged and single-token steps included."""
+    chunks = [256, 100, 1, 16, 300, 128, 33]
+    total = sum(chunks)
+    cfg, pool, tables, (paged,) = quant_paged_members(1, total, max(chunks), bits, seed=3)
+    assert binding.paged_pool_bytes(cfg, 4) == 4 * (2 * 8 * 128 * (128 * bits // 8) + 2 * 8 * 128 * 4)
+    _, flat = quant_cache(total, max(chunks), bits=bits)
+    for t, n in enumerate(chunks):
+        q, k, v = workloads.chunk_inputs(W, 105, t, device="cuda", n_tokens=n)
+        got = paged.fold_step(q, k, v)
+        want = flat.fold_step(q, k, v)
+        assert torch.equal(got.view(torch.int16), want.view(torch.int16)), f"step {t}"
+    torch.cuda.synchronize()
+    assert paged.status() == binding.KVF_OK and len(paged) == total
+    table = tables[0].cpu()
+    for kv in (0, 1):
+        codes, scales = paged.page_codes(kv), paged.page_scales(kv)
+        flat_codes = flat.k_plane() if kv == 0 else flat.v_plane()
+        flat_scales = flat.scales(kv)
+        for i in range((total + 127) // 128):
+            rows = min(128, total - 128 * i)
+            page = int(table[i])
+            assert torch.equal(codes[page, :, :rows], flat_codes[:, 128 * i:128 * i + rows]), (kv, i)
+            assert torch.equal(scales[page, :, :rows].view(torch.int32), flat_scales[:, 128 * i:128 * i + rows].contiguous().view(torch.int32)), (kv, i)
+
+
+@BITS
+def test_batch_of_paged_quantised_caches(bits):
+    """One launch over three quantised paged caches: per member the bits of its own step, outputs within
+    tolerance of the oracle's quantised fold; lock-step chunks, then a ragged step."""
+    chunks = [256, 100, 16, 1, 300]
+    total = sum(chunks) + 64 + 32
+    B = 3
+    cfg, pool, tables, caches = quant_paged_members(B, total, max(chunks), bits, seed=5)
+    _, pool1, _, singles = quant_paged_members(B, total, max(chunks), bits, seed=5)
+    batch = binding.Batch(caches)
+    ocs = [oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base) for _ in range(B)]
+    for oc in ocs:
+        oc.set_quant(bits)
+    worst, worst_pair = 0.0, 0.0
+    for t, n in enumerate(chunks):
+        qs, ks, vs = zip(*[workloads.chunk_inputs(W, 106, t, sequence=i, device="cuda", n_tokens=n) for i in range(B)])
+        q, k, v = (torch.stack(x).contiguous() for x in (qs, ks, vs))
+        out = batch.fold_step(q, k, v)
+        rows = sorted({0, n // 2, n - 1})
+        for i in range(B):
+            alone = singles[i].fold_step(q[i], k[i], v[i])
+            worst_pair = max(worst_pair, float((out[i].float() - alone.float()).abs().max()))
+            ref = ocs[i].fold_step(to_f64(q[i]), to_f64(k[i]), to_f64(v[i]), rows=rows)
+            worst = max(worst, float(np.abs(to_f64(out[i][rows]) - ref).max()))
+    # members of different length: one member gets 64 rows more on its own, then a ragged step over all three
+    q1, k1, v1 = workloads.chunk_inputs(W, 107, 0, sequence=1, device="cuda", n_tokens=64)
+    caches[1].fold_step(q1, k1, v1)
+    singles[1].fold_step(q1, k1, v1)
+    ocs[1].fold_step(to_f64(q1), to_f64(k1), to_f64(v1), rows=[])
+    qs, ks, vs = zip(*[workloads.chunk_inputs(W, 108, 0, sequence=i, device="cuda", n_tokens=32) for i in range(B)])
+    q, k, v = (torch.stack(x).contiguous() for x in (qs, ks, vs))
+    out = batch.fold_step(q, k, v, ragged=True)
+    for i in range(B):
+        alone = singles[i].fold_step(q[i], k[i], v[i])
+        worst_pair = max(worst_pair, float((out[i].float() - alone.float()).abs().max()))
+        ref = ocs[i].fold_step(to_f64(q[i]), to_f64(k[i]), to_f64(v[i]), rows=[0, 31])
+        worst = max(worst, float(np.abs(to_f64(out[i][[0, 31]]) - ref).max()))
+    torch.cuda.synchronize()
+    assert batch.status_word() == 0 and all(c.status() == binding.KVF_OK for c in caches)
+    assert [len(c) for c in caches] == [sum(chunks) + 32, sum(chunks) + 96, sum(chunks) + 32]
+    assert torch.equal(pool, pool1)                         # every code and every scale, page for page
+    assert worst <= TOL["bf16"][0] and worst_pair <= TOL["bf16"][0], (worst, worst_pair)
