@@ -336,6 +336,21 @@ kvf_status kvf_batch_fold_step_ragged(kvf_batch *b, const void *q, const void *k
                                       int32_t n_tokens, const int64_t *pos0_or_null, void *out,
                                       float *lse_or_null, void *cuda_stream);
 
+/*
+ * The ragged step for members whose CHUNKS differ in length as well (the paper's trials end with a
+ * question chunk and up to 30 decoded tokens each - Section 4, the needle protocol - so sequences
+ * that are served together take steps of different length, and finish at different times).
+ *   n_tokens    host array [n_caches]: member i folds n_tokens[i] tokens, 0 <= n_tokens[i] <= max_tokens;
+ *               0 = the member sits this step out (its cache, length and block of `out` are untouched)
+ *   max_tokens  1 .. max_chunk: the stride of the members' blocks - q, out: [n_caches][max_tokens][n_q_heads]
+ *               [head_dim], k_new, v_new: [n_caches][max_tokens][n_kv_heads][head_dim], lse_or_null:
+ *               [n_caches][max_tokens][n_q_heads]; member i uses the first n_tokens[i] rows of its blocks
+ * Everything else as kvf_batch_fold_step_ragged; at least one member must take part.
+ */
+kvf_status kvf_batch_fold_step_varlen(kvf_batch *b, const void *q, const void *k_new, const void *v_new,
+                                      const int32_t *n_tokens, int32_t max_tokens, const int64_t *pos0_or_null,
+                                      void *out, float *lse_or_null, void *cuda_stream);
+
 /* kvf_cache_plan for a batch step; plan[2] counts the CTAs of all members. */
 kvf_status kvf_batch_plan(const kvf_batch *b, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]);
 

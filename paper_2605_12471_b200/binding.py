@@ -30,7 +30,7 @@ EXPORTS = [
     "kvf_batch_workspace_bytes", "kvf_batch_create", "kvf_batch_fold_step", "kvf_batch_plan",
     "kvf_batch_status_word", "kvf_batch_launch_count", "kvf_batch_destroy", "kvf_cache_set_window",
     "kvf_batch_fold_step_ragged", "kvf_cache_k_scales", "kvf_cache_v_scales", "kvf_cache_sm_clock",
-    "kvf_cache_host_flush",
+    "kvf_cache_host_flush", "kvf_batch_fold_step_varlen",
 ]
 
 
@@ -125,6 +125,8 @@ def load() -> ctypes.CDLL:
     lib.kvf_batch_fold_step.restype = ctypes.c_int
     lib.kvf_batch_fold_step_ragged.argtypes = [vp, vp, vp, vp, i32, ctypes.POINTER(i64), vp, vp, vp]
     lib.kvf_batch_fold_step_ragged.restype = ctypes.c_int
+    lib.kvf_batch_fold_step_varlen.argtypes = [vp, vp, vp, vp, ctypes.POINTER(i32), i32, ctypes.POINTER(i64), vp, vp, vp]
+    lib.kvf_batch_fold_step_varlen.restype = ctypes.c_int
     lib.kvf_batch_plan.argtypes = [vp, i32, i64, ctypes.POINTER(i32)]
     lib.kvf_batch_plan.restype = ctypes.c_int
     lib.kvf_batch_status_word.argtypes = [vp]
@@ -448,6 +450,25 @@ class Batch:
                                         _stream_ptr(stream))
         if rc != KVF_OK:
             raise KvfError(rc, "kvf_batch_fold_step")
+        return out
+
+    def fold_step_varlen(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, n_tokens, pos0=None,
+                         out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                         stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """kvf_batch_fold_step_varlen: member i folds the first n_tokens[i] rows of its block (0 = sits out)."""
+        assert q.dim() == 4 and q.shape[0] == len(self.caches) == len(n_tokens)
+        for t in (q, k_new, v_new):
+            assert t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16
+        if out is None:
+            od = torch.float32 if (self.cfg.flags & KVF_OUT_F32) else torch.bfloat16
+            out = torch.empty(q.shape, dtype=od, device=q.device)
+        ns = (ctypes.c_int32 * len(self.caches))(*[int(x) for x in n_tokens])
+        arr = None if pos0 is None else (ctypes.c_int64 * len(self.caches))(*[int(p) for p in pos0])
+        rc = load().kvf_batch_fold_step_varlen(self._h, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), ns, q.shape[1],
+                                               arr, out.data_ptr(), lse.data_ptr() if lse is not None else None,
+                                               _stream_ptr(stream))
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_batch_fold_step_varlen")
         return out
 
     def plan(self, n_tokens: int, prefix_len: Optional[int] = None) -> Tuple[int, int, int, int]:

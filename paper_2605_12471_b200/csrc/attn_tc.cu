@@ -177,10 +177,13 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qpair = blockIdx.x, group = blockIdx.y;
     const int cb = blockIdx.z;     // cache of a batch (0 when there is one cache)
-    const int G = a.G, n = a.n;
+    const int G = a.G;
     // (a ragged batch keeps its members' row counts in device memory, written by an earlier kernel
     // of the stream: those are the one thing read before the set-up below, so wait first there)
     if (a.prefixes) pdl_wait();
+    // tokens this cache folds; a.n is the longest chunk of the launch and the stride of the caches' blocks
+    const int n = a.ns ? (int)a.ns[cb] : a.n, nmax = a.n;
+    if (blockIdx.x * 2 * kRows >= n * G) return;          // a shorter member of a batch: no row of this row pair exists
     const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix, L = P + n;
     // streams == 2 (chunks of at most 128 / G tokens, i.e. one row tile): the two tile slots work on
     // the SAME 128 rows and take alternate key tiles, so that one stream's softmax still runs under
@@ -339,7 +342,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             int rg = 0;                  // int8 storage: loads so far into the ring of raw tiles
             int page = 0;                // paged cache: page of the key tile being loaded
             const int32_t *page_table = a.page_tables ? a.page_tables[cb] : a.page_table;
-            const int qtok0 = cb * n;    // the caches' rotated chunks follow one another
+            const int qtok0 = cb * nmax; // the caches' rotated chunks follow one another
             bool ok = true;
             int kt0, ntiles;
             for (int kvh = kvh_first; ok && piece(kvh, kt0, ntiles); ++kvh) {
@@ -527,7 +530,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         const int64_t limit = valid ? P + tok + 1 : ((int64_t)1 << 62);
         const float sl2 = a.scale_log2;
         const float2 sl2v = make_float2(sl2, sl2);
-        const int64_t nG = (int64_t)n * G;
+        const int64_t nG = (int64_t)nmax * G;                 // rows of a partial slot
 
         int it = 0, oc = 0;            // my key tiles and my finished pieces so far
         int turn_base = 0;             // turns (see below) both tile slots have taken before this piece
@@ -688,7 +691,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             if (!warp_live) continue;
             const float inv = l > 0.f ? 1.f / l : 0.f;
             const float lse2 = l > 0.f ? m_ref * sl2 + log2f(l) : -INFINITY;
-            const int64_t row = ((int64_t)cb * n + tok) * a.H + kvh * G + gi;
+            const int64_t row = ((int64_t)cb * nmax + tok) * a.H + kvh * G + gi;
 #pragma unroll
             for (int c0 = 0; c0 < 128; c0 += 32) {
                 uint32_t o[32];
@@ -757,14 +760,16 @@ __global__ void __launch_bounds__(256, kFew ? 4 : 2) combine_groups_kernel(const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     int g0, g1;
-    if (a.range_valid && kvh < kRangeHeads) {
+    if (kFew || (a.range_valid && kvh < kRangeHeads)) {      // (kFew is chosen only when the host worked the ranges out)
         g0 = a.g_first[kvh];
         g1 = a.g_last[kvh];
     } else {
         if (a.prefixes) pdl_wait();   // ragged batch: the row counts were written by an earlier kernel of the stream
+        const int n_b = a.ns ? (int)a.ns[cb] : a.n;
+        if (n_b == 0) return;         // this cache sat the step out
         if (threadIdx.x == 0) {
             const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix;
-            const int nt_all = (int)((P + a.n + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
+            const int nt_all = (int)((P + n_b + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
             group_range(a.Hkv, nt_all, a.ngroups, kvh, g_range[0], g_range[1]);
         }
         __syncthreads();
@@ -772,6 +777,9 @@ __global__ void __launch_bounds__(256, kFew ? 4 : 2) combine_groups_kernel(const
         g1 = g_range[1];
     }
     pdl_wait();   // the parts are the attention kernel's output
+    // tokens this cache folded (a.n: the longest chunk, the stride); members of different length come
+    // with a ragged batch only, which never takes the kFew variant
+    const int n = (!kFew && a.ns) ? (int)a.ns[cb] : a.n;
     const int st = a.streams;
     const int np = (g1 - g0 + 1) * st;   // parts of this KV head: st per piece
     // part s of the KV head sits in slot (g0 + s / st + kvh) * st + s % st = (g0 + kvh) * st + s
@@ -782,7 +790,7 @@ __global__ void __launch_bounds__(256, kFew ? 4 : 2) combine_groups_kernel(const
     const int rows = kCombineTokens * G;                      // rows of this block, row = token * G + head-in-group
     for (int rr = warp; rr < rows; rr += 8) {
         const int tok = blockIdx.x * kCombineTokens + rr / G, gi = rr % G;
-        if (tok >= a.n) break;
+        if (tok >= n) break;
         const int64_t R = (int64_t)tok * G + gi;
         const int64_t row = ((int64_t)cb * a.n + tok) * a.H + kvh * G + gi;
         const float *po = part_o + R * kD;                    // part s: po + s * nG * kD

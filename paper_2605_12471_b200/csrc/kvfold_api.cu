@@ -163,7 +163,7 @@ BatchLayout batch_layout(const kvf_config *c, int n_caches) {
     size_t off = 0;
     l.status = off;   off = align_up(off + 256, 1024);
     l.tables = off;   off = align_up(off + (size_t)n_caches * sizeof(void *), 1024);
-    l.lens = off;     off = align_up(off + (size_t)n_caches * 2 * sizeof(int64_t), 1024);   // row counts, then first positions
+    l.lens = off;     off = align_up(off + (size_t)n_caches * 3 * sizeof(int64_t), 1024);   // row counts, first positions, chunk lengths
     l.q_rot = off;    off = align_up(off + (size_t)n_caches * c->max_chunk * c->n_q_heads * c->head_dim * elem_bytes(c->dtype), 1024);
     l.part_o = off;   off = align_up(off + (size_t)n_caches * rows * c->head_dim * 4, 1024);
     l.part_lse = off; off = align_up(off + (size_t)n_caches * rows * 4, 1024);
@@ -469,7 +469,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     ra.page_table = c->page_table;
     ra.page_elems = c->page_elems;
     ra.page_tables = nullptr;
-    ra.prefixes = nullptr; ra.pos0s = nullptr;
+    ra.prefixes = nullptr; ra.pos0s = nullptr; ra.ns = nullptr;
     ra.status = reinterpret_cast<int *>(c->workspace + c->lay.status);
     ra.range_limit = c->tc32 ? 65504.f : 0.f;      // the fp32 tensor-core kernel computes on fp16 halves
     ra.table = c->table;
@@ -482,7 +482,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.part_lse = reinterpret_cast<float *>(c->workspace + c->lay.part_lse);
     aa.status = reinterpret_cast<int *>(c->workspace + c->lay.status);
     aa.page_table = c->page_table;
-    aa.page_tables = nullptr; aa.part_rows = 0; aa.batch = 1; aa.prefixes = nullptr;
+    aa.page_tables = nullptr; aa.part_rows = 0; aa.batch = 1; aa.prefixes = nullptr; aa.ns = nullptr;
     aa.n_sink = c->n_sink; aa.win_lo = window_lo(c, P);
     aa.k_scales = c->quant ? c->qp.k_scales : nullptr;
     aa.v_scales = c->quant ? c->qp.v_scales : nullptr;
@@ -982,20 +982,24 @@ namespace {
 // ragged step can be captured into a graph like any other.
 struct LenChunk {
     int64_t prefix[64], pos0[64];
+    int32_t n[64];
     int32_t base, count;
 };
-__global__ void write_lengths_kernel(const LenChunk c, int64_t *prefixes, int64_t *pos0s) {
+__global__ void write_lengths_kernel(const LenChunk c, int64_t *prefixes, int64_t *pos0s, int64_t *ns) {
     const int i = threadIdx.x;
     if (i < c.count) {
         prefixes[c.base + i] = c.prefix[i];
         pos0s[c.base + i] = c.pos0[i];
+        ns[c.base + i] = c.n[i];
     }
 }
 
 // One step of a batch.  pos0s == nullptr: every member holds the same number of rows and starts at
-// pos0; else member i starts at pos0s[i] and the members' row counts may differ.
+// pos0; else member i starts at pos0s[i] and the members' row counts may differ.  ns != nullptr
+// (ragged only): member i folds ns[i] <= n tokens (0 = it sits the step out) out of blocks of n.
 kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void *v_new, int32_t n,
-                      int64_t pos0, const int64_t *pos0s, void *out, float *lse, void *cuda_stream) {
+                      int64_t pos0, const int64_t *pos0s, const int32_t *ns, void *out, float *lse,
+                      void *cuda_stream) {
     if (!b) return KVF_ERR_INVALID_ARG;
     kvf_cache *c0 = b->caches[0];
     const bool ragged = pos0s != nullptr;
@@ -1007,9 +1011,15 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     }
     if (ragged && c0->window > 0) return KVF_ERR_UNSUPPORTED;     // the window is placed per launch
     kvf_status s = KVF_OK;
-    for (size_t i = 0; i < b->caches.size() && s == KVF_OK; ++i)
-        s = check_step(b->caches[i], n, ragged ? pos0s[i] : pos0);
+    bool any = ns == nullptr;
+    for (size_t i = 0; i < b->caches.size() && s == KVF_OK; ++i) {
+        if (ns && (ns[i] < 0 || ns[i] > n)) return KVF_ERR_INVALID_ARG;
+        if (ns && ns[i] == 0) continue;                         // sits the step out: nothing to check
+        any = true;
+        s = check_step(b->caches[i], ns ? ns[i] : n, ragged ? pos0s[i] : pos0);
+    }
     if (s != KVF_OK) return s;
+    if (n < 1 || n > c0->cfg.max_chunk || !any) return KVF_ERR_INVALID_ARG;   // (a step nobody takes part in)
     if (check_ptr(q) || check_ptr(k_new) || check_ptr(v_new) || check_ptr(out)) return KVF_ERR_INVALID_ARG;
     if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return KVF_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -1018,6 +1028,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     const Plan plan = make_plan(c0, n, P, B, b->part_rows);
     int64_t *dev_prefixes = reinterpret_cast<int64_t *>(b->workspace + b->off_lens);
     int64_t *dev_pos0s = dev_prefixes + B;
+    int64_t *dev_ns = dev_pos0s + B;
     if (ragged) {
         for (int base = 0; base < B; base += 64) {
             LenChunk ch;
@@ -1026,8 +1037,9 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
             for (int i = 0; i < ch.count; ++i) {
                 ch.prefix[i] = b->caches[base + i]->len;
                 ch.pos0[i] = pos0s[base + i];
+                ch.n[i] = ns ? ns[base + i] : n;
             }
-            write_lengths_kernel<<<1, 64, 0, st>>>(ch, dev_prefixes, dev_pos0s);
+            write_lengths_kernel<<<1, 64, 0, st>>>(ch, dev_prefixes, dev_pos0s, dev_ns);
             cudaError_t e = cudaGetLastError();
             if (e != cudaSuccess) return cuda_fail(e, "write_lengths launch");
             b->launches++;
@@ -1049,6 +1061,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     ra.page_tables = tables;
     ra.prefixes = ragged ? dev_prefixes : nullptr;
     ra.pos0s = ragged ? dev_pos0s : nullptr;
+    ra.ns = ns ? dev_ns : nullptr;
     ra.status = nullptr; ra.range_limit = 0.f;
     ra.table = c0->table;
 
@@ -1062,6 +1075,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     aa.page_table = c0->page_table;
     aa.page_tables = tables; aa.part_rows = b->part_rows; aa.batch = B;
     aa.prefixes = ragged ? dev_prefixes : nullptr;
+    aa.ns = ns ? dev_ns : nullptr;
     aa.n_sink = c0->n_sink; aa.win_lo = window_lo(c0, P);
     aa.k_scales = c0->quant ? c0->qp.k_scales : nullptr;
     aa.v_scales = c0->quant ? c0->qp.v_scales : nullptr;
@@ -1093,7 +1107,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
         if (e != cudaSuccess) return cuda_fail(e, "combine launch (batch)");
         b->launches++;
     }
-    for (kvf_cache *c : b->caches) c->len += n;
+    for (size_t i = 0; i < b->caches.size(); ++i) b->caches[i]->len += ns ? ns[i] : n;
     return KVF_OK;
 }
 
@@ -1103,7 +1117,7 @@ extern "C" {
 
 kvf_status kvf_batch_fold_step(kvf_batch *b, const void *q, const void *k_new, const void *v_new, int32_t n,
                                int64_t pos0, void *out, float *lse, void *cuda_stream) {
-    return batch_step(b, q, k_new, v_new, n, pos0, nullptr, out, lse, cuda_stream);
+    return batch_step(b, q, k_new, v_new, n, pos0, nullptr, nullptr, out, lse, cuda_stream);
 }
 
 kvf_status kvf_batch_fold_step_ragged(kvf_batch *b, const void *q, const void *k_new, const void *v_new, int32_t n,
@@ -1114,7 +1128,19 @@ kvf_status kvf_batch_fold_step_ragged(kvf_batch *b, const void *q, const void *k
         for (kvf_cache *c : b->caches) own.push_back(c->len);
         pos0_or_null = own.data();
     }
-    return batch_step(b, q, k_new, v_new, n, 0, pos0_or_null, out, lse, cuda_stream);
+    return batch_step(b, q, k_new, v_new, n, 0, pos0_or_null, nullptr, out, lse, cuda_stream);
+}
+
+kvf_status kvf_batch_fold_step_varlen(kvf_batch *b, const void *q, const void *k_new, const void *v_new,
+                                      const int32_t *n_tokens, int32_t max_tokens, const int64_t *pos0_or_null,
+                                      void *out, float *lse, void *cuda_stream) {
+    if (!b || !n_tokens) return KVF_ERR_INVALID_ARG;
+    std::vector<int64_t> own;
+    if (!pos0_or_null) {                                       // positions continue from each member's length
+        for (kvf_cache *c : b->caches) own.push_back(c->len);
+        pos0_or_null = own.data();
+    }
+    return batch_step(b, q, k_new, v_new, max_tokens, 0, pos0_or_null, n_tokens, out, lse, cuda_stream);
 }
 
 kvf_status kvf_batch_plan(const kvf_batch *b, int32_t n_tokens, int64_t prefix_len, int32_t plan[4]) {

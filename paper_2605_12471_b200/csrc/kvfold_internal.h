@@ -95,6 +95,9 @@ struct RopeAppendArgs {
     // ragged batch: cache b holds prefixes[b] rows and its chunk starts at position pos0s[b]
     // (device arrays, or null: prefix and pos0 above hold for every cache)
     const int64_t *prefixes, *pos0s;
+    // ... and, if its members' chunks differ in length too, cache b folds ns[b] tokens (0 = it sits the step
+    // out); n above is then the longest chunk and the stride of the members' blocks in q, k_new, v_new, q_rot
+    const int64_t *ns;
     // fp32 cache whose attention runs on fp16 halves of its operands: a rotated query or key or a value
     // above range_limit in magnitude sets code 7 in *status (range_limit = 0: no check)
     int *status;
@@ -120,6 +123,8 @@ struct AttnArgs {
     int64_t part_rows;               // rows of the partial area per cache of a batch
     int32_t batch;                   // caches in the launch (1 = one cache)
     const int64_t *prefixes;         // ragged batch: device array of the caches' row counts, else null
+    const int64_t *ns;               // ragged batch with chunks of different length: device array of the caches'
+                                     // token counts (n below is then the longest chunk = stride of the blocks), else null
     const float *k_scales, *v_scales; // int8 storage: fp32 row scales [Hkv][scale_stride] (the tensor maps then
                                      // describe the int8 code planes), else null; paged: the scale blocks of page 0
     int64_t scale_stride;            // capacity rounded up to a multiple of 4 (16-byte aligned rows of scales)

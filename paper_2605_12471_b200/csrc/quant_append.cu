@@ -56,7 +56,6 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
     constexpr int d = 128, half = 64;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tok0 = blockIdx.x * kTok;
-    const int ntok = min(kTok, a.n - tok0);
     const int b = blockIdx.y;      // cache of a batch (0 when there is one cache)
 
     pdl_launch_dependents();
@@ -65,6 +64,8 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
     if (a.prefixes || a.pos0s) pdl_wait();
     const int64_t prefix = a.prefixes ? a.prefixes[b] : a.prefix;
     const int64_t pos0 = a.pos0s ? a.pos0s[b] : a.pos0;
+    const int n = a.ns ? (int)a.ns[b] : a.n;               // tokens this cache folds (a.n: the longest chunk, the stride)
+    const int ntok = max(0, min(kTok, n - tok0));
     const int32_t *page_table = a.page_tables ? a.page_tables[b] : a.page_table;
     // where row `row` of KV head g lives: byte offset of its codes from the code block, index of its scale
     auto code_off = [&](int g, int64_t row) -> int64_t {
@@ -88,10 +89,10 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
     // Rows between the new end of the cache and the next key-tile boundary get value scale 0: the
     // attention expands them to zeros whatever their codes are, so a zero probability never
     // multiplies non-finite bits.
-    if (blockIdx.x == 0) {
-        const int zero_rows = a.prefixes ? (int)((kKvTile - (prefix + a.n) % kKvTile) % kKvTile) : a.zero_rows;
+    if (blockIdx.x == 0 && n > 0) {
+        const int zero_rows = a.prefixes ? (int)((kKvTile - (prefix + n) % kKvTile) % kKvTile) : a.zero_rows;
         for (int i = threadIdx.x; i < zero_rows * a.Hkv; i += kThreads)
-            qp.v_scales[scale_idx(i / zero_rows, prefix + a.n + i % zero_rows)] = 0.f;
+            qp.v_scales[scale_idx(i / zero_rows, prefix + n + i % zero_rows)] = 0.f;
     }
 
     const int64_t qoff = (int64_t)b * a.n * a.H * d, koff = (int64_t)b * a.n * a.Hkv * d;

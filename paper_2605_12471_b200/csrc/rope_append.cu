@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
     __shared__ float2 cs[kTok][kMaxHalfDim];   // (cos, sin) per (token, pair)
 
     const int d = a.d, half = d / 2;
-    const int n_tok_blocks = (a.n + kTok - 1) / kTok;
+    const int n_tok_blocks = (a.n + kTok - 1) / kTok;      // (a.n: the longest chunk of the launch)
     const int b = blockIdx.y;      // cache of a batch (0 when there is one cache)
     const RowMap rows{a.page_tables ? a.page_tables[b] : a.page_table, a.capacity, a.page_elems, a.d};
     // (the per-cache arrays of a ragged batch were written by an earlier kernel of the stream: under
@@ -72,6 +72,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
     if (a.prefixes || a.pos0s) pdl_wait();
     const int64_t prefix = a.prefixes ? a.prefixes[b] : a.prefix;
     const int64_t pos0 = a.pos0s ? a.pos0s[b] : a.pos0;
+    const int n = a.ns ? (int)a.ns[b] : a.n;               // tokens this cache folds
 
     pdl_launch_dependents();
     if ((int)blockIdx.x >= n_tok_blocks) {
@@ -79,7 +80,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
         // Clear value rows between the new end of the cache and the next key-tile boundary,
         // so that a zero probability never multiplies stale non-finite bits.
         const int vec_per_row = d / VEC;
-        const int zero_rows = a.prefixes ? (int)((kKvTile - (prefix + a.n) % kKvTile) % kKvTile) : a.zero_rows;
+        const int zero_rows = n == 0 ? 0 : a.prefixes ? (int)((kKvTile - (prefix + n) % kKvTile) % kKvTile) : a.zero_rows;
         const int64_t total = (int64_t)zero_rows * a.Hkv * vec_per_row;
         const int64_t start = ((int64_t)blockIdx.x - n_tok_blocks) * kThreads + threadIdx.x;
         const int64_t stride = (int64_t)(gridDim.x - n_tok_blocks) * kThreads;
@@ -88,7 +89,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
             int c = (int)(i % vec_per_row);
             int64_t t = i / vec_per_row;
             int g = (int)(t % a.Hkv);
-            int64_t row = prefix + a.n + t / a.Hkv;
+            int64_t row = prefix + n + t / a.Hkv;
             *reinterpret_cast<uint4 *>(vp + rows.offset(g, row) + c * VEC) =
                 make_uint4(0, 0, 0, 0);
         }
@@ -96,7 +97,8 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
     }
 
     const int tok0 = blockIdx.x * kTok;
-    const int ntok = min(kTok, a.n - tok0);
+    const int ntok = min(kTok, n - tok0);
+    if (ntok <= 0) return;                                  // a shorter member of a batch
 
     for (int idx = threadIdx.x; idx < ntok * half; idx += kThreads) {
         int t = idx / half, j = idx % half;

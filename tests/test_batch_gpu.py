@@ -1,5 +1,7 @@
 """One launch over many caches (kvf_batch_*): per member the same cache bits as its own
 kvf_fold_step, outputs within tolerance of the fp64 oracle."""
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -214,3 +216,61 @@ def test_batch_status_word_written_from_the_host_is_read_back():
     batch.workspace[:4].zero_()
     torch.cuda.synchronize()
     assert batch.status_word() == 0
+
+
+def test_members_take_steps_of_different_length_and_sit_steps_out():
+    """kvf_batch_fold_step_varlen: sequences served together end at different times - one still folds a
+    question chunk while others decode single tokens or have finished (n = 0).  Per member the pool ends
+    up bit-identical to folding that member by itself, outputs agree with the oracle, blocks of members
+    that sit a step out are left alone."""
+    B = 4
+    total = 1024
+    cfg, pool, tables, caches = make_members(B, total, 256, seed=19)
+    _, pool1, _, singles = make_members(B, total, 256, seed=19)
+    batch = binding.Batch(caches)
+    ocs = [oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base) for _ in range(B)]
+    # (max_tokens of the step, tokens of each member)
+    steps = [(256, [256, 200, 256, 130]),      # ragged prefill: two row tiles for some, one and a bit for others
+             (100, [100, 1, 0, 33]),           # a question chunk, a decoded token, a finished sequence, a short chunk
+             (1, [1, 1, 0, 1]),                # decode
+             (40, [0, 40, 0, 7]),
+             (256, [1, 0, 256, 0]),            # a long chunk beside a single token
+             (30, [30, 30, 30, 30])]
+    worst, worst_lse, worst_pair = 0.0, 0.0, 0.0
+    for t, (mx, ns) in enumerate(steps):
+        q, k, v = batch_inputs(B, mx, 43, t)
+        out = torch.full(q.shape, 7.0, dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((B, mx, W.n_q_heads), 7.0, dtype=torch.float32, device="cuda")
+        before = [len(c) for c in caches]
+        batch.fold_step_varlen(q, k, v, ns, out=out, lse=lse)
+        for i, n in enumerate(ns):
+            assert len(caches[i]) == before[i] + n
+            # rows past a member's own count (and the whole block of a member that sat out) are untouched
+            assert bool((out[i, n:] == 7.0).all()) and bool((lse[i, n:] == 7.0).all())
+            if n == 0:
+                continue
+            alone = singles[i].fold_step(q[i, :n].contiguous(), k[i, :n].contiguous(), v[i, :n].contiguous())
+            worst_pair = max(worst_pair, float((out[i, :n].float() - alone.float()).abs().max()))
+            rows = sorted({0, n // 2, n - 1})
+            ref, ref_lse, _ = ocs[i].fold_step(to_f64(q[i, :n]), to_f64(k[i, :n]), to_f64(v[i, :n]), rows=rows, want_stats=True)
+            worst = max(worst, float(np.abs(to_f64(out[i, :n][rows]) - ref).max()))
+            worst_lse = max(worst_lse, float(np.abs(to_f64(lse[i, :n][rows]) - ref_lse).max()))
+    torch.cuda.synchronize()
+    assert batch.status_word() == 0 and all(c.status() == binding.KVF_OK for c in caches)
+    assert torch.equal(pool.view(torch.int16), pool1.view(torch.int16))            # every appended row, page for page
+    assert worst <= TOL["bf16"][0] and worst_pair <= TOL["bf16"][0] and worst_lse <= 2e-2, (worst, worst_pair, worst_lse)
+    # argument checks: a count above the stride, a negative count, a step nobody takes
+    lib = binding.load()
+    q, k, v = batch_inputs(B, 8, 43, 99)
+    out = torch.empty_like(q)
+
+    def call(ns, mx):
+        arr = (ctypes.c_int32 * B)(*ns)
+        return lib.kvf_batch_fold_step_varlen(batch._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), arr, mx, None,
+                                              out.data_ptr(), None, None)
+    lens = [len(c) for c in caches]
+    assert call([9, 1, 1, 1], 8) == binding.KVF_ERR_INVALID_ARG
+    assert call([-1, 1, 1, 1], 8) == binding.KVF_ERR_INVALID_ARG
+    assert call([0, 0, 0, 0], 8) == binding.KVF_ERR_INVALID_ARG
+    assert call([1, 1, 1, 1], 0) == binding.KVF_ERR_INVALID_ARG
+    assert [len(c) for c in caches] == lens
