@@ -36,6 +36,18 @@ def test_struct_layout_matches_header(binding):
     assert c.rope_base.offset == 32 and c.softmax_scale.offset == 40 and c.inv_freq.offset == 48
 
 
+def test_quantised_pages_and_result_staging_are_counted(binding):
+    # a quantised page: 2 x 8 KV heads x 128 rows of 128 (int8) or 64 (int4) code bytes, then 2 x 8 x 128 fp32 scales
+    q8 = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5, flags=binding.KVF_CACHE_INT8)
+    q4 = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5, flags=binding.KVF_CACHE_INT4)
+    assert binding.paged_pool_bytes(q8, 3) == 3 * (2 * 8 * 128 * 128 + 2 * 8 * 128 * 4)
+    assert binding.paged_pool_bytes(q4, 3) == 3 * (2 * 8 * 128 * 64 + 2 * 8 * 128 * 4)
+    # the second result staging set of KVF_HOST_DOWNLOAD_BEHIND: one more chunk of outputs and of lse
+    plain = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5)
+    behind = binding.make_config(32, 8, 128, "bf16", 1024, 256, rope_base=5e5, flags=binding.KVF_HOST_DOWNLOAD_BEHIND)
+    assert binding.workspace_bytes(behind) - binding.workspace_bytes(plain) == 256 * 32 * 128 * 2 + 256 * 32 * 4
+
+
 def test_storage_bytes_follow_the_papers_per_token_count(binding):
     # Section 5: 8 KV heads x 128 x (K,V) x 2 bytes per token per layer; 32 layers = 131072 B/token
     cfg = binding.make_config(32, 8, 128, "bf16", 131072, 256, rope_base=5e5)
@@ -97,6 +109,10 @@ def test_null_handles_are_harmless(binding):
     assert lib.kvf_fold_step_host(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_cache_launch_count(None) == 0
     assert lib.kvf_cache_status_word(None) == -1
+    assert lib.kvf_cache_host_flush(None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_cache_sm_clock(None, (ctypes.c_uint64 * 2)()) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_batch_fold_step_varlen(None, None, None, None, None, 1, None, None, None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_status_str(7).decode() == "KVF_ERR_RANGE"
     assert lib.kvf_cache_k_plane(None) is None
     lib.kvf_cache_destroy(None)
     assert lib.kvf_status_str(0).decode() == "KVF_OK"

@@ -386,6 +386,25 @@ def test_profile_counters_and_launch_count():
     assert all(m >= 0 for m in ms) and ms[1] > 0
 
 
+def test_attention_kernels_report_the_clock_they_ran_at():
+    """kvf_cache_sm_clock: the first CTA of every tensor-core attention launch adds its SM cycles and its
+    nanoseconds to two sums; their ratio is a clock between idle and the part's maximum."""
+    for w in (SMALL_LLAMA.with_(name="clock_bf16", tokens=4096), SMALL_LLAMA_F32.with_(name="clock_f32", tokens=4096)):
+        cache = binding.cache_for(w)
+        assert cache.sm_clock() == (0, 0)
+        q, k, v = workloads.chunk_inputs(w, 45, 0, device="cuda")
+        for t in range(8):
+            cache.fold_step(q, k, v)
+        cycles, ns = cache.sm_clock()                      # a blocking copy: the steps are done when it returns
+        assert cycles > 0 and ns > 0
+        mhz = 1e3 * cycles / ns
+        assert 300.0 < mhz < 2200.0, mhz                  # (a B200's SM clock tops out at 1965 MHz)
+    tiny = binding.cache_for(workloads.TINY)              # CUDA-core kernel: it does not count
+    q, k, v = workloads.chunk_inputs(workloads.TINY, 46, 0, device="cuda")
+    tiny.fold_step(q, k, v)
+    assert tiny.sm_clock() == (0, 0)
+
+
 # ------------------------------------------------------------------ short chunks at depth
 def test_short_chunks_deep_in_a_chain_match_the_oracle():
     """Decode- and question-shaped steps (1 .. 32 tokens: at most one 128-row tile) after a long
