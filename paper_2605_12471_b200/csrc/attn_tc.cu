@@ -57,6 +57,7 @@
 // shared and tensor memory (a ragged batch, whose row counts live in device memory, waits first).
 #include "kvfold_internal.h"
 #include "sm100_ptx.cuh"
+#include "quant_expand.cuh"
 
 namespace kvf {
 namespace {
@@ -127,32 +128,6 @@ __device__ __forceinline__ void exp_half(const uint32_t *v, uint32_t *p, float2 
         if (c & 1) acc1 = __fadd2_rn(acc1, e);
         else acc0 = __fadd2_rn(acc0, e);
         p[c] = pack_bf16(e.x, e.y);
-    }
-}
-
-// Four codes (one 32-bit word, each byte already offset by 128) -> two packed bf16 pairs of
-// bf16(code * scale): byte i dropped into the mantissa of 2^23 gives 2^23 + code + 128 exactly.
-__device__ __forceinline__ void expand4(uint32_t x, float2 sc, uint32_t &lo, uint32_t &hi) {
-    const float2 off = make_float2(-8388736.f, -8388736.f);
-    float2 a = make_float2(__uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650)), __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651)));
-    float2 b = make_float2(__uint_as_float(__byte_perm(x, 0x4B000000u, 0x7652)), __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7653)));
-    a = __fmul2_rn(__fadd2_rn(a, off), sc);
-    b = __fmul2_rn(__fadd2_rn(b, off), sc);
-    lo = pack_bf16(a.x, a.y);
-    hi = pack_bf16(b.x, b.y);
-}
-
-// Eight 4-bit codes (one 32-bit word, each nibble = code + 8, element 2i in the low nibble of byte i)
-// -> four packed bf16 pairs of bf16(code * scale), in element order.
-__device__ __forceinline__ void expand8(uint32_t w, float2 sc, uint32_t (&o)[4]) {
-    const float2 off = make_float2(-8388616.f, -8388616.f);      // 2^23 + 8
-    const uint32_t lo = w & 0x0F0F0F0Fu, hi = (w >> 4) & 0x0F0F0F0Fu;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float2 a = make_float2(__uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7650 + i)),
-                               __uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7650 + i)));
-        a = __fmul2_rn(__fadd2_rn(a, off), sc);
-        o[i] = pack_bf16(a.x, a.y);
     }
 }
 

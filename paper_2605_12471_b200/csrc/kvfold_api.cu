@@ -301,6 +301,7 @@ kvf_status build_maps(kvf_cache *c) {
 }
 
 struct Plan {
+    bool qdec;     // quantised cache, a few query rows: the decode kernel that expands codes in registers
     bool tc;
     int splits;    // CUDA-core path: splits of the key range; tensor-core path: ranges per KV head (rounded up)
     int ngroups;   // tensor-core path: ranges of the (KV head, key tile) line
@@ -317,12 +318,31 @@ int64_t window_lo(const kvf_cache *c, int64_t prefix) {
 }
 
 Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t part_rows_cap = -1) {
+    const bool single = part_rows_cap < 0;      // a step of one cache through its own handle (not a batch of one)
     if (part_rows_cap < 0) part_rows_cap = c->part_rows_cap;
     Plan p;
+    p.qdec = false;
     p.tc = c->tc || c->tc32;
     p.ngroups = 0;
     const int64_t L = prefix + n;
     const int Hkv = c->cfg.n_kv_heads;
+    if (c->quant && single && c->window <= 0 && n * c->G <= attn_q8_decode_max_rows()) {
+        // one CTA per SM, each inside one KV head (a multiple of the KV heads), at least two key tiles each;
+        // a forced split count is the number of ranges per KV head
+        const int64_t nt = (L + kKvTile - 1) / kKvTile;
+        int64_t per_head = c->force_splits > 0 ? c->force_splits : c->sm_count / Hkv;
+        if (c->force_splits <= 0 && per_head > nt / 2) per_head = nt / 2;
+        if (per_head > nt) per_head = nt;
+        const int64_t slots_cap = part_rows_cap / ((int64_t)n * c->G);            // slots = groups + Hkv - 1
+        if (per_head * Hkv + Hkv - 1 > slots_cap) per_head = (slots_cap - (Hkv - 1)) / Hkv;
+        if (per_head < 1) per_head = 1;
+        p.qdec = true;
+        p.ngroups = (int)(per_head * Hkv);
+        p.splits = (int)per_head;
+        p.ctas = p.ngroups;
+        p.kernels = 2 + (per_head > 1 ? 1 : 0);
+        return p;
+    }
     if (p.tc) {
         // one CTA per (row pair, group); the groups cut the Hkv * nt line of (KV head, key tile)
         // into equal ranges.  Whole KV heads if that fills the SMs, else as many groups as give
@@ -493,7 +513,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
     aa.splits = plan.tc ? 1 : plan.splits;
     aa.ngroups = plan.ngroups;
-    aa.streams = c->tc ? attn_tc_streams(n, c->G) : 1;
+    aa.streams = (c->tc && !plan.qdec) ? attn_tc_streams(n, c->G) : 1;
     aa.out_f32 = (f.dtype == KVF_F32 || (f.flags & KVF_OUT_F32)) ? 1 : 0;
     aa.scale_log2 = c->scale_log2;
     aa.range_valid = 0;
@@ -513,7 +533,8 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     c->launches++;
     {
         ProfScope ps(c, st, 1);
-        if (c->tc) e = launch_attn_tc(aa, c->maps, st);
+        if (plan.qdec) e = launch_attn_q8_decode(aa, c->maps, st);
+        else if (c->tc) e = launch_attn_tc(aa, c->maps, st);
         else if (c->tc32) e = launch_attn_tc32(aa, st);
         else e = launch_attn_simt(aa, f.dtype, st, nullptr);
     }

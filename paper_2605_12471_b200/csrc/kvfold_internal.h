@@ -206,6 +206,12 @@ int attn_tc_streams(int n, int G);     // 2 when the chunk fits one 128-row tile
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s);   // grid (row pairs, ngroups)
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s);                // needed when ngroups != Hkv
 
+// Decode-shaped steps (at most attn_q8_decode_max_rows() query rows) on a quantised cache: codes are
+// expanded into mma.sync register fragments, shared memory is all ring.  Grid = ngroups CTAs, ngroups a
+// multiple of the KV heads; partial results as for the other tensor-core kernels (streams = 1).
+int attn_q8_decode_max_rows();
+cudaError_t launch_attn_q8_decode(const AttnArgs &a, const TcMaps &maps, cudaStream_t s);
+
 // Tensor-core path for fp32 caches (head_dim 128): operands split into fp16 halves, three MMAs per
 // product; contiguous planes, read straight from global memory (no tensor maps).
 bool attn_tc32_supported(int dtype, int d, int G);

@@ -272,3 +272,37 @@ def test_batch_of_paged_quantised_caches(bits):
     assert [len(c) for c in caches] == [sum(chunks) + 32, sum(chunks) + 96, sum(chunks) + 32]
     assert torch.equal(pool, pool1)                         # every code and every scale, page for page
     assert worst <= TOL["bf16"][0] and worst_pair <= TOL["bf16"][0], (worst, worst_pair)
+
+
+@BITS
+@pytest.mark.parametrize("paged", [False, True], ids=["contiguous", "paged"])
+def test_decode_shaped_steps_on_a_quantised_cache_at_depth(bits, paged):
+    """One to four tokens per step (at most 16 query rows) after a long prefix: the kernel that expands codes
+    straight into MMA register fragments, every row of every step against the oracle's quantised fold; then
+    longer chunks again (the other kernel) on the same cache, and forced range counts."""
+    chunks = [2048] * 4 + [1, 1, 2, 3, 4, 1, 4] + [256, 5, 1] + [1] * 6
+    total = sum(chunks)
+    if paged:
+        cfg, pool, tables, (cache,) = quant_paged_members(1, total, max(chunks), bits, seed=9)
+    else:
+        cfg, cache = quant_cache(total, max(chunks), bits=bits)
+    oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
+    oc.set_quant(bits)
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert cache.plan(1, 8192) == (1, 18, 144, 3)            # 18 key ranges per KV head, one CTA each
+        assert cache.plan(4, 8192) == (1, 18, 144, 3) and cache.plan(5, 8192)[2] != 144      # 16 rows is the limit
+    worst, worst_lse = 0.0, 0.0
+    for t, n in enumerate(chunks):
+        q, k, v = workloads.chunk_inputs(W, 109, t, device="cuda", n_tokens=n)
+        if t >= len(chunks) - 6:
+            cache.set_splits([1, 2, 3, 7, 18, 0][t - (len(chunks) - 6)])      # one range per KV head (direct output) ... many
+        lse = torch.empty((n, W.n_q_heads), dtype=torch.float32, device="cuda")
+        out = cache.fold_step(q, k, v, lse=lse)
+        rows = list(range(n)) if n <= 4 else []
+        ref, ref_lse, _ = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows, want_stats=True)
+        if rows:
+            worst = max(worst, float(np.abs(to_f64(out) - ref).max()))
+            worst_lse = max(worst_lse, float(np.abs(to_f64(lse) - ref_lse).max()))
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_OK and len(cache) == total
+    assert worst <= TOL["bf16"][0] and worst_lse <= 2e-2, (worst, worst_lse)
