@@ -10,19 +10,24 @@
 // tensor-core kernel for long chunks expands every code tile into a bf16 tile in shared memory,
 // which costs it the shared memory it would need to keep enough bytes in flight, and runs the
 // expansion on four warps.  Here the codes never get a bf16 image in shared memory: the whole of
-// it is a ring of raw code tiles (K codes, V codes and their row scales: 33 KiB a stage for int8,
-// six stages; 17 KiB and ten stages for int4) filled by TMA, with one consumer warp per stage:
-// warp w takes every tile that lands in stage w (so it sees every phase of that stage's barriers, which
-// is what a parity wait needs), expands codes straight into the register fragments of mma.sync
-// m16n8k16 (bf16 in, fp32 accumulate) and keeps its own running softmax and output; the warps'
-// results are merged at the end.  Both contractions are free in how they number what they sum
-// over or put out, which is what makes the expansion cheap:
-//   S = Q K^T sums over d: thread (g, q) of a warp (g = lane / 4, q = lane % 4) takes the 32 codes
-//     d = 32 q .. 32 q + 31 of key row g of an 8-key block - one contiguous 32 bytes - as its
-//     B elements of the eight k-steps, and Q's fragments are loaded once in the same order;
-//   O = P V puts out d: the same 32 codes of a V row become, after one 8 x 8 register transpose
-//     (movmatrix) per fragment, the B elements of sixteen 8-column blocks whose columns are, for
-//     thread q, again d = 32 q .. 32 q + 31; P comes straight from the score accumulators.
+// it is a ring of raw code tiles (K codes, V codes and their row scales of 128 keys: 33 KiB a
+// stage for int8, 17 KiB for int4) filled by TMA, and two consumer warps per stage, each taking
+// 64 of the tile's keys (a warp always reads the same stage, so it sees every phase of that
+// stage's barriers, which is what a parity wait needs).  A warp expands codes straight into the
+// register fragments of mma.sync m16n8k16 (bf16 in, fp32 accumulate) and keeps its own running
+// softmax and output; the warps' results are merged at the end.
+//
+// With so few query rows the KEYS take the 16-row side of the MMA and the query rows the 8-column
+// side (one or two column blocks), so no MMA row is wasted on padding and V needs no transpose:
+//   S^T = K Q^T (16 keys x 8 rows, summed over d): thread (g, t) of a warp (g = lane / 4,
+//     t = lane % 4) takes the 32 codes d = 32 t .. 32 t + 31 of key rows g and g + 8 of a 16-key
+//     block - contiguous bytes - as its A elements of the eight k-steps; the contraction is free in
+//     how it numbers d, and Q's B fragments are loaded once in the same order;
+//   O^T = V^T P^T (128 d x 8 rows, summed over 16 keys): an A element pairs two KEYS of one d, and
+//     since every code is expanded on its own, thread (g, t) builds its pairs from the 16 codes
+//     d = 16 g .. 16 g + 15 of key rows 2 t, 2 t + 1, 2 t + 8, 2 t + 9 (the MMA's row index is
+//     free in how it numbers d as well).  P^T's B fragment is the transposed score fragment:
+//     two 8 x 8 register transposes (movmatrix) per 16 keys.
 //
 // Work: the key tiles (128 keys) of each KV head are cut into ngroups / Hkv ranges (the group
 // count is a multiple of the KV heads, so a CTA stays inside one head); every CTA leaves a
@@ -38,26 +43,29 @@ namespace {
 
 constexpr int kKeysPerTile = 128;
 constexpr int kD = 128;
-constexpr int kMaxRows = 16;                   // one m16 tile of query rows
+constexpr int kMaxRows = 16;                   // two 8-column blocks of query rows
 
 struct Ctl {
     unsigned long long full[12], empty[12];
     int abort;
 };
 
-template <int BITS> struct Geo {
+// NB = 8-row blocks of query rows (1: up to 8 rows, 2: up to 16).  A scheduler of the SM holds 16 K
+// registers: with 13 warps one of them has four (128 registers a thread, enough for one block of
+// rows), with 11 none has more than three (168, what two blocks need without spilling).
+template <int BITS, int NB> struct Geo {
     static constexpr int RB = kD * BITS / 8;                       // bytes of a row of codes
     static constexpr uint32_t kCodes = kKeysPerTile * RB;          // one tile of codes
     static constexpr uint32_t kStage = 2 * kCodes + 1024;          // K codes, V codes, K scales, V scales
-    static constexpr int kStages = BITS == 4 ? 10 : 6;
+    static constexpr int kStages = NB == 2 ? 5 : 6;
     static constexpr uint32_t kOffCtl = kStages * kStage;
     static constexpr uint32_t kSmem = kOffCtl + 1024 + 1024;       // + control block + alignment slack
-    static constexpr int kWarps = kStages;                         // consumer warps, one per stage; one more warp produces
+    static constexpr int kWarps = 2 * kStages;                     // consumer warps, two per stage; one more warp produces
     static constexpr int kThreads = (kWarps + 1) * 32;
 };
 // what the warps leave for the merge: 16 rows x 128 fp32 and per row a maximum and a sum
 constexpr uint32_t kMergeWarp = kMaxRows * kD * 4 + kMaxRows * 8;
-static_assert(Geo<4>::kWarps * kMergeWarp <= Geo<4>::kOffCtl && Geo<8>::kWarps * kMergeWarp <= Geo<8>::kOffCtl, "the merge area reuses the ring");
+static_assert(Geo<4, 1>::kWarps * kMergeWarp <= Geo<4, 1>::kOffCtl && Geo<4, 2>::kWarps * kMergeWarp <= Geo<4, 2>::kOffCtl, "the merge area reuses the ring");
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     // (not volatile: a pure function of its register operands, so the compiler may interleave independent chains)
@@ -71,41 +79,104 @@ __device__ __forceinline__ uint32_t transpose8x8(uint32_t x) {
     asm("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
     return y;
 }
+// (volatile, here and below: the tiles are rewritten by later TMA copies)
+__device__ __forceinline__ void lds128(uint32_t addr, uint32_t (&w)[4]) {
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr));
+}
+__device__ __forceinline__ void lds64(uint32_t addr, uint32_t (&w)[2]) {
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "r"(addr));
+}
 
-// The 32 codes d = 32 q .. 32 q + 31 of code row `row` of a tile at shared address `tile`
-// (rows of RB bytes, swizzled over their 16-byte chunks as the TMA left them) -> 16 registers of
-// two bf16 each, bf16(code * scale), in element order.
+// A fragments of S^T = K Q^T for one 16-key block: the 32 codes d = 32 t .. 32 t + 31 of key rows
+// `row` and `row + 8` of the code tile at shared address `tile` (rows swizzled over their 16-byte
+// chunks as the TMA left them).  k-step s covers d = 32 t + 4 s .. + 3: a0 / a2 from the first row,
+// a1 / a3 from the second, each bf16(code * scale) in element order.
 template <int BITS>
-__device__ __forceinline__ void expand_segment(uint32_t tile, int row, int q, float scale, uint32_t (&out)[16]) {
-    const float2 sc = make_float2(scale, scale);
-    if (BITS == 8) {
-        // 128-byte rows, 128-byte swizzle: chunk c of row r sits at c ^ (r & 7); my chunks are 2 q and 2 q + 1
-        const uint32_t base = tile + (uint32_t)row * 128u, sw = (uint32_t)row & 7u;
-        uint32_t w[8];
+__device__ __forceinline__ void key_fragments(uint32_t tile, int row, int t, float sc_a, float sc_b, uint32_t (&ka)[8][4]) {
 #pragma unroll
-        for (uint32_t c = 0; c < 2; ++c)
-            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3]) : "r"(base + (((2u * (uint32_t)q + c) ^ sw) << 4)));   // (volatile: the tile is rewritten by later TMA copies)
+    for (int h = 0; h < 2; ++h) {
+        const int r = row + 8 * h;
+        const float s1 = h ? sc_b : sc_a;
+        const float2 sc = make_float2(s1, s1);
+        if (BITS == 8) {
+            // 128-byte rows, 128-byte swizzle: chunk c of row r sits at c ^ (r & 7); my chunks are 2 t and 2 t + 1
+            const uint32_t base = tile + (uint32_t)r * 128u, sw = (uint32_t)r & 7u;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) expand4(w[i] ^ 0x80808080u, sc, out[2 * i], out[2 * i + 1]);
-    } else {
-        // 64-byte rows, 64-byte swizzle: chunk c of row r sits at c ^ ((r >> 1) & 3); my chunk is q
-        const uint32_t base = tile + (uint32_t)row * 64u, sw = ((uint32_t)row >> 1) & 3u;
-        uint32_t w[4];
-        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(base + (((uint32_t)q ^ sw) << 4)));
+            for (uint32_t c = 0; c < 2; ++c) {
+                uint32_t w[4];
+                lds128(base + (((2u * (uint32_t)t + c) ^ sw) << 4), w);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            uint32_t o[4];
-            expand8(w[i], sc, o);
-            out[4 * i] = o[0]; out[4 * i + 1] = o[1]; out[4 * i + 2] = o[2]; out[4 * i + 3] = o[3];
+                for (int i = 0; i < 4; ++i) expand4(w[i] ^ 0x80808080u, sc, ka[4 * c + i][h], ka[4 * c + i][2 + h]);
+            }
+        } else {
+            // 64-byte rows, 64-byte swizzle: chunk c of row r sits at c ^ ((r >> 1) & 3); my chunk is t
+            const uint32_t base = tile + (uint32_t)r * 64u, sw = ((uint32_t)r >> 1) & 3u;
+            uint32_t w[4];
+            lds128(base + (((uint32_t)t ^ sw) << 4), w);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t o[4];
+                expand8(w[i], sc, o);
+                ka[2 * i][h] = o[0]; ka[2 * i][2 + h] = o[1];
+                ka[2 * i + 1][h] = o[2]; ka[2 * i + 1][2 + h] = o[3];
+            }
         }
     }
 }
 
+// bf16 pair (x(wa), x(wb)) * sc of byte `byte` of two words whose bytes hold code + `bias`
+// (2^23 + byte is exact in fp32, as is the difference that follows)
+__device__ __forceinline__ uint32_t pair_of_rows(uint32_t wa, uint32_t wb, int byte, float2 off, float2 sc) {
+    float2 x = make_float2(__uint_as_float(__byte_perm(wa, 0x4B000000u, 0x7650 + byte)),
+                           __uint_as_float(__byte_perm(wb, 0x4B000000u, 0x7650 + byte)));
+    x = __fmul2_rn(__fadd2_rn(x, off), sc);
+    return pack_bf16_pair(x.x, x.y);
+}
+
+// The codes d = 16 g .. 16 g + 15 of key rows row0 + 2 t + {0, 1, 8, 9} of the V code tile, ready
+// for pair_of_rows: int8 as four words of four codes (each byte code + 128), int4 as two words of
+// low nibbles (elements 16 g + 2 i) and two of high nibbles (elements 16 g + 2 i + 1), each code + 8.
 template <int BITS>
-__global__ void __launch_bounds__(Geo<BITS>::kThreads, 1)
+__device__ __forceinline__ void value_codes(uint32_t tile, int row0, int g, int t, uint32_t (&w)[4][4]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = row0 + 2 * t + (i & 1) + 8 * (i >> 1);
+        if (BITS == 8) {
+            lds128(tile + (uint32_t)r * 128u + (((uint32_t)g ^ ((uint32_t)r & 7u)) << 4), w[i]);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) w[i][k] ^= 0x80808080u;
+        } else {
+            uint32_t x[2];
+            lds64(tile + (uint32_t)r * 64u + (((((uint32_t)g >> 1) ^ (((uint32_t)r >> 1) & 3u)) << 4) | (((uint32_t)g & 1u) << 3)), x);
+            w[i][0] = x[0] & 0x0F0F0F0Fu; w[i][1] = x[1] & 0x0F0F0F0Fu;
+            w[i][2] = (x[0] >> 4) & 0x0F0F0F0Fu; w[i][3] = (x[1] >> 4) & 0x0F0F0F0Fu;
+        }
+    }
+}
+// A fragment jp of O^T = V^T P^T: MMA rows g / g + 8 are d = 16 g + 2 jp / + 1, columns the 16 keys.
+template <int BITS>
+__device__ __forceinline__ void value_fragment(const uint32_t (&w)[4][4], int jp, float2 sc01, float2 sc89, uint32_t (&va)[4]) {
+    if (BITS == 8) {
+        const float2 off = make_float2(-8388736.f, -8388736.f);          // 2^23 + 128
+        const int word = jp >> 1, b = 2 * (jp & 1);
+        va[0] = pair_of_rows(w[0][word], w[1][word], b, off, sc01);
+        va[1] = pair_of_rows(w[0][word], w[1][word], b + 1, off, sc01);
+        va[2] = pair_of_rows(w[2][word], w[3][word], b, off, sc89);
+        va[3] = pair_of_rows(w[2][word], w[3][word], b + 1, off, sc89);
+    } else {
+        const float2 off = make_float2(-8388616.f, -8388616.f);          // 2^23 + 8
+        const int word = jp >> 2, b = jp & 3;
+        va[0] = pair_of_rows(w[0][word], w[1][word], b, off, sc01);
+        va[1] = pair_of_rows(w[0][2 + word], w[1][2 + word], b, off, sc01);
+        va[2] = pair_of_rows(w[2][word], w[3][word], b, off, sc89);
+        va[3] = pair_of_rows(w[2][2 + word], w[3][2 + word], b, off, sc89);
+    }
+}
+
+template <int BITS, int NB>
+__global__ void __launch_bounds__(Geo<BITS, NB>::kThreads, 1)
 attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
-    using Gm = Geo<BITS>;
+    using Gm = Geo<BITS, NB>;
     constexpr int NST = Gm::kStages, kWarps = Gm::kWarps;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -114,7 +185,7 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     const uint32_t bar_full = base + Gm::kOffCtl, bar_empty = bar_full + 12 * 8;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = lane >> 2, q = lane & 3;
+    const int g = lane >> 2, t4 = lane & 3;
     const int group = blockIdx.x;
     const int G = a.G, n = a.n, nG = n * G;
     const int64_t P = a.prefix, L = P + n;
@@ -131,7 +202,7 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     if (threadIdx.x == 0) {
         for (int s = 0; s < NST; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 2);       // the stage's two consumer warps
         }
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -140,14 +211,20 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     __syncthreads();
     pdl_wait();   // nothing above reads what an earlier kernel wrote; from here on the rotated chunk and the cache are read
 
-    // what a consumer warp carries through its tiles (declared here so that every warp reaches the
-    // merge below by the same path)
-    float o[16][4];            // output: 8-column block vb, rows g / g + 8; columns d = 32 q + 2 vb + {0, 1}
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};      // rows g and g + 8; log2 units
+    // what a consumer warp carries through its keys (declared here so that every warp reaches the
+    // merge below by the same path): O^T[d = 16 g + 2 jp + {0, 1}][row 8 nb + 2 t + {0, 1}] as
+    // ot[nb][jp][{0, 1}] (first d) and [{2, 3}] (second d); maxima and sums of rows 8 nb + 2 t + {0, 1}
+    float ot[NB][8][4];
+    float m_run[NB][2], l_run[NB][2];
 #pragma unroll
-    for (int vb = 0; vb < 16; ++vb)
+    for (int nb = 0; nb < NB; ++nb) {
+        m_run[nb][0] = m_run[nb][1] = -INFINITY;
+        l_run[nb][0] = l_run[nb][1] = 0.f;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) o[vb][e] = 0.f;
+        for (int jp = 0; jp < 8; ++jp)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) ot[nb][jp][e] = 0.f;
+    }
 
     if (warp == kWarps) {
         if (lane == 0) {
@@ -184,135 +261,141 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             for (int t = max(0, ntiles - NST); t < ntiles; ++t) mbar_wait_drain(bar_full + 8 * (t % NST), (t / NST) & 1, a.status);
         }
     } else {
-        // ------------------------------------------------------------------ consumers: whole key tiles, one warp each
-        // Q fragments of the eight k-steps, in the order the key codes are taken: k-step s of thread q
-        // covers d = 32 q + 4 s .. + 3 (first pair: a0 / a1 for rows g / g + 8, second pair: a2 / a3)
-        uint32_t aq[8][4];
+        // ------------------------------------------------------------------ consumers: 64 keys of every tile of one stage
+        const int s = warp >> 1, half = warp & 1;
+        // Q^T's B fragments of the eight k-steps, in the order the key codes are taken: k-step ks of
+        // thread t covers d = 32 t + 4 ks .. + 3 of query row 8 nb + g
+        uint32_t bq[NB][8][2];
         {
             const __nv_bfloat16 *q_rot = reinterpret_cast<const __nv_bfloat16 *>(a.q_rot);
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int R = g + 8 * h, tok = R / G, gi = R % G;
-                const __nv_bfloat16 *src = q_rot + ((int64_t)tok * a.H + kvh * G + gi) * kD + 32 * q;
+            for (int nb = 0; nb < NB; ++nb) {
+                const int R = g + 8 * nb, tok = R / G, gi = R % G;
+                const __nv_bfloat16 *src = q_rot + ((int64_t)tok * a.H + kvh * G + gi) * kD + 32 * t4;
 #pragma unroll
-                for (int s = 0; s < 8; ++s) {
+                for (int ks = 0; ks < 8; ++ks) {
                     uint2 w = make_uint2(0u, 0u);
-                    if (R < nG) w = *reinterpret_cast<const uint2 *>(src + 4 * s);
-                    aq[s][h] = w.x;
-                    aq[s][2 + h] = w.y;
+                    if (R < nG) w = *reinterpret_cast<const uint2 *>(src + 4 * ks);
+                    bq[nb][ks][0] = w.x;
+                    bq[nb][ks][1] = w.y;
                 }
             }
         }
         // keys below the limit are visible (rows past the chunk's end are never written; each row of S, P
         // and O depends on that row alone, so they are left unmasked)
-        int64_t limit[2];
+        // (counted from the chunk's first key, P)
+        int limit[NB][2];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int R = g + 8 * h;
-            limit[h] = R < nG ? P + R / G + 1 : ((int64_t)1 << 62);
-        }
+        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int R = 8 * nb + 2 * t4 + e;
+                limit[nb][e] = R < nG ? R / G + 1 : (1 << 30);
+            }
         const float sl2 = a.scale_log2;
         bool ok = true;
-        for (int t = warp; t < ntiles && ok; t += kWarps) {
-            const int s = warp;          // = t % NST: this warp is the only reader of its stage
+        for (int t = s; t < ntiles && ok; t += NST) {
             ok = mbar_wait(bar_full + 8 * s, (t / NST) & 1, ctl, a.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const uint32_t k_tile = base + (uint32_t)s * Gm::kStage, v_tile = k_tile + Gm::kCodes;
             const float *k_sc = reinterpret_cast<const float *>(smem + (uint32_t)s * Gm::kStage + 2 * Gm::kCodes);
             const float *v_sc = k_sc + 128;
-            const int64_t key_base = (int64_t)(kt0 + t) * kKeysPerTile;
-#pragma unroll 1
-            for (int half = 0; half < 2; ++half) {
-                // ---- scores of 64 keys: eight 8-key blocks, S[kb] = rows g / g + 8, keys 2 q, 2 q + 1 of the block
-                float sacc[8][4];
+            const int64_t key_h = (int64_t)(kt0 + t) * kKeysPerTile + half * 64;      // my 64 keys
+            // (rows past the end of the planes were not copied: they count as zero)
+            const int in_planes = (int)min((int64_t)64, a.capacity - key_h);
+
+            // ---- scores of the 64 keys: four 16-key blocks, sacc[j][nb] = keys g / g + 8 of block j, rows 8 nb + 2 t + {0, 1}
+            float sacc[4][NB][4];
 #pragma unroll
-                for (int kb = 0; kb < 8; kb += 2) {
-                    // two key blocks at a time, each with a second accumulator for its odd k-steps: four
-                    // independent chains of four MMAs instead of one chain of eight per block
-                    float odd[2][4];
-                    uint32_t b[2][16];
+            for (int j = 0; j < 4; ++j) {
+                const int rl = 16 * j + g;                       // my first key row within the 64
+                uint32_t ka[8][4];
+                key_fragments<BITS>(k_tile, half * 64 + rl, t4, rl < in_planes ? k_sc[half * 64 + rl] : 0.f,
+                                    rl + 8 < in_planes ? k_sc[half * 64 + rl + 8] : 0.f, ka);
 #pragma unroll
-                    for (int i = 0; i < 2; ++i) {
+                for (int nb = 0; nb < NB; ++nb) {
+                    // a second accumulator for the odd k-steps: two chains of four MMAs instead of one of eight
+                    float odd[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) { sacc[kb + i][e] = 0.f; odd[i][e] = 0.f; }
-                        const int row = half * 64 + (kb + i) * 8 + g;
-                        // (rows past the end of the planes were not copied: they count as zero)
-                        const float scale = key_base + row < a.capacity ? k_sc[row] : 0.f;
-                        expand_segment<BITS>(k_tile, row, q, scale, b[i]);
+                    for (int e = 0; e < 4; ++e) { sacc[j][nb][e] = 0.f; odd[e] = 0.f; }
+#pragma unroll
+                    for (int ks = 0; ks < 8; ks += 2) {
+                        mma_bf16(sacc[j][nb], ka[ks], bq[nb][ks][0], bq[nb][ks][1]);
+                        mma_bf16(odd, ka[ks + 1], bq[nb][ks + 1][0], bq[nb][ks + 1][1]);
                     }
 #pragma unroll
-                    for (int ks = 0; ks < 8; ks += 2)
-#pragma unroll
-                        for (int i = 0; i < 2; ++i) {
-                            mma_bf16(sacc[kb + i], aq[ks], b[i][2 * ks], b[i][2 * ks + 1]);
-                            mma_bf16(odd[i], aq[ks + 1], b[i][2 * ks + 2], b[i][2 * ks + 3]);
-                        }
-#pragma unroll
-                    for (int i = 0; i < 2; ++i)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) sacc[kb + i][e] += odd[i][e];
+                    for (int e = 0; e < 4; ++e) sacc[j][nb][e] += odd[e];
                 }
-                // ---- mask, running maximum, probabilities
-                const int64_t key_h = key_base + half * 64;
+            }
+            // ---- mask (only where the chunk's own keys are near), running maximum, probabilities
+            const bool masked = key_h + 64 > P;
+            const int rel = masked ? (int)(key_h - P) + g : 0;      // my first key, counted from P (> -64 where it matters)
+            uint32_t pb[4][NB][2];         // P^T as B fragments of the four 16-key steps
+            float alpha[NB][2];
+            bool rescale = false;
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb) {
                 float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-                for (int kb = 0; kb < 8; ++kb)
+                for (int j = 0; j < 4; ++j)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const int64_t key = key_h + kb * 8 + 2 * q + (e & 1);
-                        const float v = key < limit[e >> 1] ? sacc[kb][e] * sl2 : -INFINITY;
-                        sacc[kb][e] = v;
-                        mx[e >> 1] = fmaxf(mx[e >> 1], v);
+                        float v = sacc[j][nb][e] * sl2;
+                        if (masked && rel + 16 * j + 8 * (e >> 1) >= limit[nb][e & 1]) v = -INFINITY;
+                        sacc[j][nb][e] = v;
+                        mx[e & 1] = fmaxf(mx[e & 1], v);
                     }
-                float alpha[2], m_safe[2];
+                float m_safe[2];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
-                    mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
-                    const float m_new = fmaxf(m_run[h], mx[h]);
-                    m_safe[h] = m_new == -INFINITY ? 0.f : m_new;
-                    alpha[h] = ex2(m_run[h] - m_safe[h]);                   // m_run = -inf -> 0
-                    m_run[h] = m_new;
-                    l_run[h] *= alpha[h];
+                for (int e = 0; e < 2; ++e) {
+                    mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 4));
+                    mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 8));
+                    mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 16));
+                    const float m_new = fmaxf(m_run[nb][e], mx[e]);
+                    m_safe[e] = m_new == -INFINITY ? 0.f : m_new;
+                    alpha[nb][e] = ex2(m_run[nb][e] - m_safe[e]);                   // m_run = -inf -> 0
+                    m_run[nb][e] = m_new;
+                    l_run[nb][e] *= alpha[nb][e];
+                    rescale = rescale || alpha[nb][e] != 1.f;
                 }
-                uint32_t pa[4][4];         // P as A fragments of the four 16-key steps
-#pragma unroll
-                for (int kb = 0; kb < 8; ++kb) {
-                    const float p0 = ex2(sacc[kb][0] - m_safe[0]), p1 = ex2(sacc[kb][1] - m_safe[0]);
-                    const float p2 = ex2(sacc[kb][2] - m_safe[1]), p3 = ex2(sacc[kb][3] - m_safe[1]);
-                    l_run[0] += p0 + p1;
-                    l_run[1] += p2 + p3;
-                    pa[kb >> 1][2 * (kb & 1)] = pack_bf16_pair(p0, p1);           // a0 / a2: row g
-                    pa[kb >> 1][2 * (kb & 1) + 1] = pack_bf16_pair(p2, p3);       // a1 / a3: row g + 8
-                }
-                if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
-#pragma unroll
-                    for (int vb = 0; vb < 16; ++vb) {
-                        o[vb][0] *= alpha[0]; o[vb][1] *= alpha[0];
-                        o[vb][2] *= alpha[1]; o[vb][3] *= alpha[1];
-                    }
-                }
-                // ---- O += P V, 16 keys at a time
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    uint32_t bt0[16], bt1[16];
+                    const float p0 = ex2(sacc[j][nb][0] - m_safe[0]), p1 = ex2(sacc[j][nb][1] - m_safe[1]);
+                    const float p2 = ex2(sacc[j][nb][2] - m_safe[0]), p3 = ex2(sacc[j][nb][3] - m_safe[1]);
+                    l_run[nb][0] += p0 + p2;
+                    l_run[nb][1] += p1 + p3;
+                    // (key g, rows 2 t, 2 t + 1) transposed: (keys 2 t, 2 t + 1; row g) - P^T's b0; keys + 8: b1
+                    pb[j][nb][0] = transpose8x8(pack_bf16_pair(p0, p1));
+                    pb[j][nb][1] = transpose8x8(pack_bf16_pair(p2, p3));
+                }
+            }
+            if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll
-                    for (int blk = 0; blk < 2; ++blk) {
-                        const int row = half * 64 + j * 16 + blk * 8 + g;
-                        const float scale = key_base + row < a.capacity ? v_sc[row] : 0.f;
-                        uint32_t b[16];
-                        expand_segment<BITS>(v_tile, row, q, scale, b);
-                        // register i holds V[key g of the block][d = 32 q + 2 i, + 1]: block i of eight columns
-                        // as an 8 x 8 matrix [key][column 2 q, 2 q + 1]; transposed it is that block's B fragment
+                for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const uint32_t tr = transpose8x8(b[i]);
-                            if (blk == 0) bt0[i] = tr; else bt1[i] = tr;
-                        }
+                    for (int jp = 0; jp < 8; ++jp) {
+                        ot[nb][jp][0] *= alpha[nb][0]; ot[nb][jp][1] *= alpha[nb][1];
+                        ot[nb][jp][2] *= alpha[nb][0]; ot[nb][jp][3] *= alpha[nb][1];
                     }
+            }
+            // ---- O^T += V^T P^T, 16 keys at a time
 #pragma unroll
-                    for (int vb = 0; vb < 16; ++vb) mma_bf16(o[vb], pa[j], bt0[vb], bt1[vb]);
+            for (int j = 0; j < 4; ++j) {
+                const int r0 = 16 * j + 2 * t4;                  // my first key row within the 64
+                float2 sc01, sc89;
+                sc01.x = r0 < in_planes ? v_sc[half * 64 + r0] : 0.f;
+                sc01.y = r0 + 1 < in_planes ? v_sc[half * 64 + r0 + 1] : 0.f;
+                sc89.x = r0 + 8 < in_planes ? v_sc[half * 64 + r0 + 8] : 0.f;
+                sc89.y = r0 + 9 < in_planes ? v_sc[half * 64 + r0 + 9] : 0.f;
+                uint32_t w[4][4];
+                value_codes<BITS>(v_tile, half * 64 + 16 * j, g, t4, w);
+#pragma unroll
+                for (int jp = 0; jp < 8; ++jp) {
+                    uint32_t va[4];
+                    value_fragment<BITS>(w, jp, sc01, sc89, va);
+#pragma unroll
+                    for (int nb = 0; nb < NB; ++nb) mma_bf16(ot[nb][jp], va, pb[j][nb][0], pb[j][nb][1]);
                 }
             }
             __syncwarp();
@@ -329,19 +412,22 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         float *mo = mrg + (size_t)warp * (kMergeWarp / 4);
         float *mm = mo + kMaxRows * kD;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            float l = l_run[h];
-            l += __shfl_xor_sync(0xffffffffu, l, 1);
-            l += __shfl_xor_sync(0xffffffffu, l, 2);
-            const int r = g + 8 * h;
+        for (int nb = 0; nb < NB; ++nb)
 #pragma unroll
-            for (int vb = 0; vb < 16; ++vb)
-                *reinterpret_cast<float2 *>(mo + r * kD + 32 * q + 2 * vb) = make_float2(o[vb][2 * h], o[vb][2 * h + 1]);
-            if (q == 0) {
-                mm[2 * r] = m_run[h];
-                mm[2 * r + 1] = l;
+            for (int e = 0; e < 2; ++e) {
+                float l = l_run[nb][e];          // my keys' share; the other keys sit in the threads of the other g
+                l += __shfl_xor_sync(0xffffffffu, l, 4);
+                l += __shfl_xor_sync(0xffffffffu, l, 8);
+                l += __shfl_xor_sync(0xffffffffu, l, 16);
+                const int r = 8 * nb + 2 * t4 + e;
+#pragma unroll
+                for (int jp = 0; jp < 8; ++jp)
+                    *reinterpret_cast<float2 *>(mo + r * kD + 16 * g + 2 * jp) = make_float2(ot[nb][jp][e], ot[nb][jp][2 + e]);
+                if (g == 0) {
+                    mm[2 * r] = m_run[nb][e];
+                    mm[2 * r + 1] = l;
+                }
             }
-        }
     }
     __syncthreads();
     for (int item = threadIdx.x; item < kMaxRows * 16; item += kWarps * 32) {
@@ -398,13 +484,15 @@ int attn_q8_decode_max_rows() { return kMaxRows; }
 
 cudaError_t launch_attn_q8_decode(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
     static_assert(sizeof(Ctl) <= 1024, "control block");
-    static_assert(Geo<8>::kSmem <= 232448 && Geo<4>::kSmem <= 232448, "shared memory budget of one CTA");
-    static_assert(Geo<8>::kStages <= 12 && Geo<4>::kStages <= 12, "control block holds 12 stages");
-    auto kernel = a.quant_bits == 4 ? attn_q8_decode_kernel<4> : attn_q8_decode_kernel<8>;
-    const uint32_t smem = a.quant_bits == 4 ? Geo<4>::kSmem : Geo<8>::kSmem;
+    static_assert(Geo<8, 1>::kSmem <= 232448 && Geo<8, 2>::kSmem <= 232448, "shared memory budget of one CTA");
+    static_assert(Geo<8, 1>::kStages <= 12, "control block holds 12 stages");
+    const bool wide = a.n * a.G > 8, four = a.quant_bits == 4;
+    auto kernel = four ? (wide ? attn_q8_decode_kernel<4, 2> : attn_q8_decode_kernel<4, 1>)
+                       : (wide ? attn_q8_decode_kernel<8, 2> : attn_q8_decode_kernel<8, 1>);
+    const uint32_t smem = four ? (wide ? Geo<4, 2>::kSmem : Geo<4, 1>::kSmem) : (wide ? Geo<8, 2>::kSmem : Geo<8, 1>::kSmem);
     cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(kernel), (int)smem);
     if (e != cudaSuccess) return e;
-    const int threads = a.quant_bits == 4 ? Geo<4>::kThreads : Geo<8>::kThreads;
+    const int threads = wide ? Geo<8, 2>::kThreads : Geo<8, 1>::kThreads;
     return launch_pdl(kernel, dim3(a.ngroups), dim3(threads), smem, s, a, maps.k, maps.v);
 }
 
