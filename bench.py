@@ -372,6 +372,8 @@ def parse_args():
                          "FLOP and byte counts in the output line then count the visible keys only")
     ap.add_argument("--batched", action="store_true",
                     help="full_stack only: the caches live in one paged pool and every chunk is one batch step")
+    ap.add_argument("--no-combine-behind", action="store_true",
+                    help="leave the merge of a step's partial results on the caller's stream (no KVF_COMBINE_BEHIND)")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every fold step of the timed chains from the host instead of replaying the chain "
                          "as one CUDA graph captured from the same kvf_fold_step calls")
@@ -469,8 +471,12 @@ def run_chain_bench(args, w, drift=False):
         w = w.with_(n_q_heads=q.shape[1], n_kv_heads=k.shape[1])
     H, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
     out = torch.empty_like(q)
-    # (the two host-step flags touch kvf_fold_step_host only: uploads ahead of, result copies behind the steps)
+    # (the two host-step flags touch kvf_fold_step_host only: uploads ahead of, result copies behind the steps;
+    # KVF_COMBINE_BEHIND puts the merge of a step's partial results beside the next step's rotate + append
+    # kernel - a chain ends with kvf_cache_flush, inside the timed region)
     flags = (binding.KVF_FORCE_SIMT if args.force_simt else 0) | binding.KVF_HOST_UPLOAD_AHEAD | binding.KVF_HOST_DOWNLOAD_BEHIND
+    if not args.no_combine_behind:
+        flags |= binding.KVF_COMBINE_BEHIND
     if args.cache_int8:
         flags |= binding.KVF_CACHE_INT8
     if args.cache_int4:
@@ -492,7 +498,7 @@ def run_chain_bench(args, w, drift=False):
     qp, kp, vp, op = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr()
     if P0:
         fq, fk, fv = workloads.chunk_inputs(w.with_(chunk=2048), args.seed + 1, 0, sequence=seq + rank, device="cuda")
-        fout = torch.empty_like(fq)
+        fout = [torch.empty_like(fq), torch.empty_like(fq)]       # (a step's results stay the library's until the next step ends)
 
     # bytes a step reads per cached token: K and V rows of every KV head (int8: d codes + one fp32 scale per row)
     bytes_per_token = (2 * Hkv * (d + 4) if args.cache_int8 else 2 * Hkv * (d // 2 + 4) if args.cache_int4
@@ -508,7 +514,8 @@ def run_chain_bench(args, w, drift=False):
         """Empty accumulator, then (outside every timed region) the prefix in 2048-token steps."""
         cache.reset()
         for t in range(P0 // 2048):
-            cache.fold_step(fq, fk, fv, out=fout)
+            cache.fold_step(fq, fk, fv, out=fout[t & 1])
+        cache.flush()
 
     def body(first=0, last=None):
         for t in range(first, N if last is None else last):
@@ -516,6 +523,9 @@ def run_chain_bench(args, w, drift=False):
                                    launch_stream[0])
             if rc:
                 raise binding.KvfError(rc, "kvf_fold_step")
+        rc = lib.kvf_cache_flush(h, launch_stream[0])      # the last step's merge, if it runs on the library's stream
+        if rc:
+            raise binding.KvfError(rc, "kvf_cache_flush")
 
     def barrier():
         if world > 1:
@@ -711,7 +721,7 @@ def run_chain_bench(args, w, drift=False):
                                             None, launch_stream[0])
                 if rc:
                     raise binding.KvfError(rc, "kvf_fold_step_host")
-            cache.host_flush()                               # the chain ends when its last results are in host memory
+            cache.flush()                                    # the chain ends when its last results are in host memory
 
         prefill()
         body_host()
@@ -747,6 +757,7 @@ def run_chain_bench(args, w, drift=False):
                        "cache_storage": ("int8 codes + fp32 row scales" if args.cache_int8 else
                                          "int4 codes + fp32 row scales" if args.cache_int4 else w.dtype),
                        "launch": "per-step host launches" if graph is None else "one CUDA graph per chain, captured from the same calls",
+                       "combine": "on the caller's stream" if args.no_combine_behind else "behind the attention kernel on the library's stream (KVF_COMBINE_BEHIND), chain closed by kvf_cache_flush",
                        "l2": f"inputs larger than L2 (cache grows to {T * bytes_per_token / 2 ** 20:.0f} MiB per chain)",
                        "last_step_plan": {"tensor_core": plan_last[0], "splits": plan_last[1], "ctas": plan_last[2]}},
             "attention_tflops": step_flops / (ms * 1e-3) / 1e12,

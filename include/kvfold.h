@@ -71,6 +71,22 @@ enum {
                                   end of call t+1, or of a kvf_cache_host_flush made after call t - not
                                   already at the end of call t.  Can be combined with KVF_HOST_UPLOAD_AHEAD;
                                   needs a workspace that no other cache's host steps use at the same time */
+    KVF_COMBINE_BEHIND = 256u, /* kvf_fold_step and kvf_fold_step_host launch the kernel that merges the key
+                                  ranges' partial results (the last kernel of a step whose plan has three)
+                                  on a stream of the library's own, behind the attention kernel, and keep two
+                                  sets of partial results, so that the merge of step t runs beside the rotate
+                                  + append and the attention kernel of step t+1 instead of in front of them.
+                                  The contract on the results relaxes: `out` and `lse` of call t are complete
+                                  on the caller's stream once that stream has passed the end of call t+1 on
+                                  this cache, or of a kvf_cache_flush made after call t - not already at the
+                                  end of call t - and until then they belong to the library (call t+1 must
+                                  be given other result buffers).  Same values as without the flag.  A
+                                  stream capture has to hold whole chains: a step or a flush that meets a
+                                  merge left open outside its own capture returns KVF_ERR_INVALID_ARG and
+                                  enqueues nothing - flush before a capture begins and before it ends.  The
+                                  stream and its events are made by kvf_cache_create /
+                                  kvf_paged_cache_create, and kvf_workspace_bytes grows by the second set;
+                                  batches and kvf_fold_step_static ignore the flag */
     KVF_CACHE_INT8 = 16u,      /* store the cache as int8 codes with one fp32 scale per row (one token of
                                   one KV head): d + 4 bytes per row instead of 2 d (kvf_cache_storage_bytes
                                   pads each head's scales to a multiple of 16 bytes).  The paper's Discussion
@@ -201,9 +217,15 @@ kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_ho
                               const void *v_host, int32_t n_tokens, int64_t pos0, void *out_host,
                               float *lse_host, void *cuda_stream);
 
-/* With KVF_HOST_DOWNLOAD_BEHIND: makes `cuda_stream` wait for the result copies of every host step
- * enqueued so far (synchronising that stream afterwards means "all results are in host memory").
- * Without the flag, or with nothing outstanding, it does nothing.  Enqueues waits only; returns at once. */
+/* Makes `cuda_stream` wait for whatever part of the steps enqueued so far runs on a stream of the
+ * library's own: the merge of the last step under KVF_COMBINE_BEHIND, the result copies of the host
+ * steps under KVF_HOST_DOWNLOAD_BEHIND (synchronising that stream afterwards means "all results are
+ * there").  Without those flags, or with nothing outstanding, it does nothing.  Enqueues waits only;
+ * returns at once.  No counterpart in the paper: it closes the two relaxed contracts above.
+ * KVF_ERR_INVALID_ARG for a null handle, or when the open merge belongs to another stream capture
+ * than `cuda_stream` (or to none while `cuda_stream` is being captured). */
+kvf_status kvf_cache_flush(kvf_cache *c, void *cuda_stream);
+/* The same call under its earlier name. */
 kvf_status kvf_cache_host_flush(kvf_cache *c, void *cuda_stream);
 
 /* Tokens appended by all steps enqueued so far: the size of the accumulator (K,V)^(t) of Section

@@ -18,7 +18,7 @@ KVF_OK, KVF_ERR_INVALID_ARG, KVF_ERR_CAPACITY, KVF_ERR_UNSUPPORTED, KVF_ERR_CUDA
     KVF_ERR_POS, KVF_ERR_RANGE = range(8)
 KVF_BF16, KVF_F32 = 0, 1
 KVF_ROPE_INTERLEAVED, KVF_STRICT_POS, KVF_OUT_F32, KVF_FORCE_SIMT, KVF_CACHE_INT8 = 1, 2, 4, 8, 16
-KVF_HOST_UPLOAD_AHEAD, KVF_CACHE_INT4, KVF_HOST_DOWNLOAD_BEHIND = 32, 64, 128
+KVF_HOST_UPLOAD_AHEAD, KVF_CACHE_INT4, KVF_HOST_DOWNLOAD_BEHIND, KVF_COMBINE_BEHIND = 32, 64, 128, 256
 
 EXPORTS = [
     "kvf_cache_storage_bytes", "kvf_workspace_bytes", "kvf_cache_create", "kvf_fold_step",
@@ -30,7 +30,7 @@ EXPORTS = [
     "kvf_batch_workspace_bytes", "kvf_batch_create", "kvf_batch_fold_step", "kvf_batch_plan",
     "kvf_batch_status_word", "kvf_batch_launch_count", "kvf_batch_destroy", "kvf_cache_set_window",
     "kvf_batch_fold_step_ragged", "kvf_cache_k_scales", "kvf_cache_v_scales", "kvf_cache_sm_clock",
-    "kvf_cache_host_flush", "kvf_batch_fold_step_varlen",
+    "kvf_cache_host_flush", "kvf_batch_fold_step_varlen", "kvf_cache_flush",
 ]
 
 
@@ -85,6 +85,8 @@ def load() -> ctypes.CDLL:
     lib.kvf_fold_step_static.restype = ctypes.c_int
     lib.kvf_cache_host_flush.argtypes = [vp, vp]
     lib.kvf_cache_host_flush.restype = ctypes.c_int
+    lib.kvf_cache_flush.argtypes = [vp, vp]
+    lib.kvf_cache_flush.restype = ctypes.c_int
     lib.kvf_cache_len.argtypes = [vp]
     lib.kvf_cache_len.restype = i64
     lib.kvf_cache_reset.argtypes = [vp]
@@ -243,6 +245,13 @@ class Cache:
         if rc != KVF_OK:
             raise KvfError(rc, "kvf_fold_step_host")
         return out
+
+    def flush(self, stream: Optional[torch.cuda.Stream] = None):
+        """kvf_cache_flush: the stream waits for the merge (KVF_COMBINE_BEHIND) and the result copies
+        (KVF_HOST_DOWNLOAD_BEHIND) the steps so far left on the library's streams."""
+        rc = load().kvf_cache_flush(self._h, _stream_ptr(stream))
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_cache_flush")
 
     def host_flush(self, stream: Optional[torch.cuda.Stream] = None):
         """kvf_cache_host_flush: the stream waits for the result copies of all host steps so far."""

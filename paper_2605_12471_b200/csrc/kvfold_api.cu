@@ -53,6 +53,7 @@ struct Layout {
     size_t status, q_rot, st_q, st_k, st_v, st_out, st_lse, part_o, part_lse, total;
     size_t st_q2, st_k2, st_v2;   // second staging set (KVF_HOST_UPLOAD_AHEAD)
     size_t st_out2, st_lse2;      // second result staging set (KVF_HOST_DOWNLOAD_BEHIND)
+    size_t part_o2, part_lse2;    // second set of partial results (KVF_COMBINE_BEHIND)
 };
 
 Layout workspace_layout(const kvf_config *c) {
@@ -83,6 +84,11 @@ Layout workspace_layout(const kvf_config *c) {
     }
     l.part_o = off;   off = align_up(off + (size_t)kPartTokens * c->n_q_heads * c->head_dim * 4, 1024);
     l.part_lse = off; off = align_up(off + (size_t)kPartTokens * c->n_q_heads * 4, 1024);
+    l.part_o2 = l.part_lse2 = 0;
+    if (c->flags & KVF_COMBINE_BEHIND) {
+        l.part_o2 = off;   off = align_up(off + (size_t)kPartTokens * c->n_q_heads * c->head_dim * 4, 1024);
+        l.part_lse2 = off; off = align_up(off + (size_t)kPartTokens * c->n_q_heads * 4, 1024);
+    }
     l.total = off;
     return l;
 }
@@ -127,6 +133,14 @@ struct kvf_cache {
     cudaEvent_t ev_step[2] = {nullptr, nullptr}, ev_down[2] = {nullptr, nullptr};
     bool ev_down_set[2] = {false, false};
     uint64_t host_down_steps = 0;
+    // KVF_COMBINE_BEHIND: the library's stream for the merge of the partial results, "attention launched"
+    // (caller's stream) and "merged" (that stream) events, which capture, if any, the open merge belongs to,
+    // and which of the two sets of partial results the next step with a merge writes
+    cudaStream_t comb_stream = nullptr;
+    cudaEvent_t ev_attn = nullptr, ev_comb = nullptr;
+    bool comb_pending = false;
+    unsigned long long comb_capture = 0;
+    int part_set = 0;
     bool quant = false;                    // int8 storage: codes + scales in `storage`, bf16 image in the workspace
     QuantPlanes qp = {};
     int32_t n_sink = 0;                    // sink + window variant: rows always visible
@@ -467,11 +481,38 @@ void fill_group_ranges(AttnArgs &aa, int64_t nt_all) {
     aa.range_valid = 1;
 }
 
+// The capture `st` is part of (0: none).  An event recorded in one capture cannot be waited for
+// from outside it or from another one.
+kvf_status capture_of(cudaStream_t st, unsigned long long *id) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    unsigned long long cid = 0;
+    cudaError_t e = cudaStreamGetCaptureInfo(st, &cs, &cid);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamGetCaptureInfo");
+    *id = cs == cudaStreamCaptureStatusActive ? cid : 0;
+    return KVF_OK;
+}
+
+// Makes `st` wait for a merge that still runs on the library's stream.
+kvf_status join_combine(kvf_cache *c, cudaStream_t st) {
+    if (!c->comb_pending) return KVF_OK;
+    cudaError_t e = cudaStreamWaitEvent(st, c->ev_comb, 0);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamWaitEvent(merge)");
+    c->comb_pending = false;
+    return KVF_OK;
+}
+
 kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void *v_new, int32_t n,
                      int64_t pos0, void *out, float *lse, cudaStream_t st) {
     const kvf_config &f = c->cfg;
     const int64_t P = c->len;
     const Plan plan = make_plan(c, n, P);
+    const bool behind = c->comb_stream != nullptr;
+    unsigned long long capture = 0;
+    if (behind) {
+        kvf_status s = capture_of(st, &capture);
+        if (s != KVF_OK) return s;
+        if (c->comb_pending && capture != c->comb_capture) return KVF_ERR_INVALID_ARG;    // flush first
+    }
 
     RopeAppendArgs ra;
     ra.q = q; ra.k_new = k_new; ra.v_new = v_new;
@@ -498,8 +539,11 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.q_rot = ra.q_rot;
     aa.k_plane = ra.k_plane; aa.v_plane = ra.v_plane;
     aa.out = out; aa.lse = lse;
-    aa.part_o = reinterpret_cast<float *>(c->workspace + c->lay.part_o);
-    aa.part_lse = reinterpret_cast<float *>(c->workspace + c->lay.part_lse);
+    // (with the merge behind the step, this step's attention kernel fills one set of partial results while
+    // the merge of the step before may still read the other)
+    const bool second = behind && c->part_set == 1;
+    aa.part_o = reinterpret_cast<float *>(c->workspace + (second ? c->lay.part_o2 : c->lay.part_o));
+    aa.part_lse = reinterpret_cast<float *>(c->workspace + (second ? c->lay.part_lse2 : c->lay.part_lse));
     aa.status = reinterpret_cast<int *>(c->workspace + c->lay.status);
     aa.page_table = c->page_table;
     aa.page_tables = nullptr; aa.part_rows = 0; aa.batch = 1; aa.prefixes = nullptr; aa.ns = nullptr;
@@ -540,13 +584,35 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     }
     if (e != cudaSuccess) return cuda_fail(e, "attention launch");
     c->launches++;
+    if (behind && plan.kernels > 2) {
+        // the merge goes behind the attention kernel on the library's stream; the caller's stream
+        // meets it again at the end of the next step, or in kvf_cache_flush
+        e = cudaEventRecord(c->ev_attn, st);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord(attention)");
+    }
+    // the merge of the step before: behind this step's attention kernel on the caller's stream, which by
+    // now has had that whole kernel to hide under (its set of partial results is written again in the next step)
+    if (kvf_status s = join_combine(c, st)) return s;
     if (plan.kernels > 2) {
+        cudaStream_t cs = st;
+        if (behind) {
+            cs = c->comb_stream;
+            e = cudaStreamWaitEvent(cs, c->ev_attn, 0);
+            if (e != cudaSuccess) return cuda_fail(e, "merge stream hand-over");
+        }
         {
-            ProfScope ps(c, st, 2);
-            e = plan.tc ? launch_combine_groups(aa, st) : launch_combine(aa, f.dtype, st);
+            ProfScope ps(c, cs, 2);
+            e = plan.tc ? launch_combine_groups(aa, cs) : launch_combine(aa, f.dtype, cs);
         }
         if (e != cudaSuccess) return cuda_fail(e, "combine launch");
         c->launches++;
+        if (behind) {
+            e = cudaEventRecord(c->ev_comb, cs);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord(merge)");
+            c->comb_pending = true;
+            c->comb_capture = capture;
+            c->part_set ^= 1;
+        }
     }
     c->len = P + n;
     return KVF_OK;
@@ -581,6 +647,16 @@ kvf_status init_handle(kvf_cache *c, const kvf_config *cfg, void *storage, void 
     c->tc = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, c->G);
     c->tc32 = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc32_supported(cfg->dtype, cfg->head_dim, c->G);
     return KVF_OK;
+}
+
+// KVF_COMBINE_BEHIND: the stream and the events are made with the handle, so that a step inside a
+// stream capture creates nothing.
+kvf_status setup_combine_behind(kvf_cache *c) {
+    if (!(c->cfg.flags & KVF_COMBINE_BEHIND)) return KVF_OK;
+    cudaError_t e = cudaStreamCreateWithFlags(&c->comb_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_attn, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_comb, cudaEventDisableTiming);
+    return e == cudaSuccess ? KVF_OK : cuda_fail(e, "merge stream setup");
 }
 
 // Bytes of one page: 128 tokens of every KV head, K block then V block; quantised caches keep the rows'
@@ -655,6 +731,8 @@ kvf_status kvf_cache_create(const kvf_config *cfg, void *dev_storage, size_t sto
     }
     cudaError_t e = cudaMemset(c->workspace + c->lay.status, 0, 256);
     if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaMemset(status)"); }
+    s = setup_combine_behind(c);
+    if (s != KVF_OK) { kvf_cache_destroy(c); return s; }
     *out = c;
     return KVF_OK;
 }
@@ -706,6 +784,8 @@ kvf_status kvf_paged_cache_create(const kvf_config *cfg, void *dev_pool, size_t 
     if (s != KVF_OK) { delete c; return s; }
     cudaError_t e = cudaMemset(c->workspace + c->lay.status, 0, 256);
     if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaMemset(status)"); }
+    s = setup_combine_behind(c);
+    if (s != KVF_OK) { kvf_cache_destroy(c); return s; }
     *out = c;
     return KVF_OK;
 }
@@ -797,7 +877,10 @@ kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_ho
         // stream goes on with the next step
         e = cudaEventRecord(c->ev_step[oset], st);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(ds, c->ev_step[oset], 0);
+        if (e == cudaSuccess && c->comb_pending) e = cudaStreamWaitEvent(ds, c->ev_comb, 0);   // the merge writes the results
         if (e != cudaSuccess) return cuda_fail(e, "download stream hand-over");
+    } else if (kvf_status js = join_combine(c, st)) {
+        return js;
     }
     e = cudaMemcpyAsync(out_host, w + o_out, ob, cudaMemcpyDeviceToHost, ds);
     if (e == cudaSuccess && lse_host)
@@ -818,9 +901,17 @@ kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_ho
     return KVF_OK;
 }
 
-kvf_status kvf_cache_host_flush(kvf_cache *c, void *cuda_stream) {
+kvf_status kvf_cache_flush(kvf_cache *c, void *cuda_stream) {
     if (!c) return KVF_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (c->comb_pending) {
+        unsigned long long capture = 0;
+        kvf_status s = capture_of(st, &capture);
+        if (s != KVF_OK) return s;
+        if (capture != c->comb_capture) return KVF_ERR_INVALID_ARG;
+        s = join_combine(c, st);
+        if (s != KVF_OK) return s;
+    }
     for (int i = 0; i < 2; ++i) {
         if (!c->ev_down_set[i]) continue;
         cudaError_t e = cudaStreamWaitEvent(st, c->ev_down[i], 0);
@@ -828,6 +919,8 @@ kvf_status kvf_cache_host_flush(kvf_cache *c, void *cuda_stream) {
     }
     return KVF_OK;
 }
+
+kvf_status kvf_cache_host_flush(kvf_cache *c, void *cuda_stream) { return kvf_cache_flush(c, cuda_stream); }
 
 int64_t kvf_cache_len(const kvf_cache *c) { return c ? c->len : -1; }
 
@@ -932,6 +1025,9 @@ void kvf_cache_destroy(kvf_cache *c) {
         if (c->ev_down[i]) cudaEventDestroy(c->ev_down[i]);
     }
     if (c->down_stream) cudaStreamDestroy(c->down_stream);
+    if (c->ev_attn) cudaEventDestroy(c->ev_attn);
+    if (c->ev_comb) cudaEventDestroy(c->ev_comb);
+    if (c->comb_stream) cudaStreamDestroy(c->comb_stream);
     delete c;
 }
 

@@ -110,6 +110,7 @@ def test_null_handles_are_harmless(binding):
     assert lib.kvf_cache_launch_count(None) == 0
     assert lib.kvf_cache_status_word(None) == -1
     assert lib.kvf_cache_host_flush(None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_cache_flush(None, None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_cache_sm_clock(None, (ctypes.c_uint64 * 2)()) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_batch_fold_step_varlen(None, None, None, None, None, 1, None, None, None, None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_status_str(7).decode() == "KVF_ERR_RANGE"

@@ -556,6 +556,109 @@ def test_host_steps_with_results_copied_behind_the_next_step(flags):
     torch.cuda.synchronize()
 
 
+def _merge_behind_chain(flags, chunks, seed=23):
+    """The same chain on a plain cache and on one with KVF_COMBINE_BEHIND (+ flags); steps enqueued back to back."""
+    total = sum(chunks)
+    w = SMALL_LLAMA.with_(name="merge_behind", tokens=total)
+    plain = binding.cache_for(w, capacity=total, max_chunk=max(chunks), flags=flags)
+    behind = binding.cache_for(w, capacity=total, max_chunk=max(chunks), flags=flags | binding.KVF_COMBINE_BEHIND)
+    ins = [workloads.chunk_inputs(w, seed, t, device="cuda", n_tokens=n) for t, n in enumerate(chunks)]
+    want, want_lse = [], []
+    for q, k, v in ins:
+        lse = torch.empty((q.shape[0], w.n_q_heads), dtype=torch.float32, device="cuda")
+        want.append(plain.fold_step(q, k, v, lse=lse))
+        want_lse.append(lse)
+    torch.cuda.synchronize()
+    return w, behind, ins, want, want_lse
+
+
+@pytest.mark.parametrize("flags", [0, binding.KVF_CACHE_INT8], ids=["bf16", "int8"])
+def test_merge_behind_the_attention_kernel_gives_the_same_bits(flags):
+    """KVF_COMBINE_BEHIND: the merge of step t runs on the library's stream beside the rotate + append kernel
+    of step t+1.  Same bits as without the flag; step t's results are there once the stream has passed call
+    t+1, the last step's after a flush.  Chunks of 256 and of one token, at prefixes where the plan has a
+    merge kernel and where it has none."""
+    chunks = [256] * 6 + [1, 1, 3, 256, 1, 1]
+    w, cache, ins, want, want_lse = _merge_behind_chain(flags, chunks)
+    kernels = [cache.plan(n, sum(chunks[:t]))[3] for t, n in enumerate(chunks)]
+    assert 3 in kernels
+    got = [torch.zeros_like(x) for x in want]
+    got_lse = [torch.zeros_like(x) for x in want_lse]
+    stream = torch.cuda.current_stream()
+    last = len(chunks) - 1
+    for t in range(last):
+        cache.fold_step(*ins[t], out=got[t], lse=got_lse[t])
+    stream.synchronize()                     # the stream has passed the end of call last - 1
+    for t in range(last - 1):
+        assert torch.equal(got[t].view(torch.int16), want[t].view(torch.int16)), t
+    cache.fold_step(*ins[last], out=got[last], lse=got_lse[last])
+    cache.flush()
+    stream.synchronize()
+    assert cache.status() == binding.KVF_OK and len(cache) == sum(chunks)
+    for t in range(len(chunks)):
+        assert torch.equal(got[t].view(torch.int16), want[t].view(torch.int16)), t
+        assert torch.equal(got_lse[t], want_lse[t]), t
+    cache.flush()                            # nothing outstanding: harmless
+    torch.cuda.synchronize()
+
+
+def test_merge_behind_inside_a_stream_capture():
+    """A chain with KVF_COMBINE_BEHIND captured into a CUDA graph (the library's stream joins the capture
+    through its events and is joined again by the flush) and replayed: the same bits.  A step that meets a
+    merge left open outside its capture is refused and enqueues nothing."""
+    chunks = [256] * 8
+    w, cache, ins, want, _ = _merge_behind_chain(0, chunks)
+    got = [torch.zeros_like(x) for x in want]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for t in range(len(chunks)):
+            cache.fold_step(*ins[t], out=got[t])
+        cache.flush()
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    for t in range(len(chunks)):
+        assert torch.equal(got[t].view(torch.int16), want[t].view(torch.int16)), t
+    # an open merge from before the capture
+    cache.reset()
+    first = next(t for t in range(len(chunks)) if cache.plan(256, 256 * t)[3] == 3)     # the first step with a merge kernel
+    assert first < len(chunks) - 1
+    for t in range(first + 1):
+        cache.fold_step(*ins[t], out=got[t])
+    launches = cache.launch_count()
+    refused = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(refused):
+        with pytest.raises(binding.KvfError) as err:
+            cache.fold_step(*ins[first + 1], out=got[first + 1])
+        with pytest.raises(binding.KvfError):
+            cache.flush()
+    assert err.value.code == binding.KVF_ERR_INVALID_ARG
+    assert len(cache) == 256 * (first + 1) and cache.launch_count() == launches
+    cache.flush()
+    torch.cuda.synchronize()
+    assert torch.equal(got[first].view(torch.int16), want[first].view(torch.int16))
+    assert cache.status() == binding.KVF_OK
+
+
+def test_merge_behind_with_host_steps_and_results_copied_behind():
+    """KVF_COMBINE_BEHIND together with the two host-step flags: the result copy of a step waits for its merge."""
+    flags = binding.KVF_HOST_DOWNLOAD_BEHIND | binding.KVF_HOST_UPLOAD_AHEAD
+    chunks = [256] * 8
+    w, cache, ins, want, want_lse = _merge_behind_chain(flags, chunks)
+    keep = [tuple(x.cpu().pin_memory() for x in qkv) for qkv in ins]
+    got = [torch.zeros(x.shape, dtype=x.dtype).pin_memory() for x in want]
+    lses = [torch.zeros(x.shape, dtype=torch.float32).pin_memory() for x in want_lse]
+    torch.cuda.synchronize()
+    for t in range(len(chunks)):
+        cache.fold_step_host(*keep[t], got[t], lse=lses[t])
+    cache.flush()
+    torch.cuda.current_stream().synchronize()
+    assert cache.status() == binding.KVF_OK
+    for t in range(len(chunks)):
+        assert torch.equal(got[t].view(torch.int16), want[t].cpu().view(torch.int16)), t
+        assert torch.equal(lses[t], want_lse[t].cpu()), t
+
+
 def test_plan_fills_the_last_wave_when_whole_kv_heads_would_leave_it_half_empty():
     """148 SMs: 32 row pairs x 8 KV heads = 256 CTAs is 1.73 waves, 32 x 9 groups = 288 is 1.95; 128 row
     pairs x 8 = 1024 CTAs (6.9 waves) stays with whole KV heads and needs no combine kernel."""
