@@ -97,7 +97,9 @@ enum {
                                   attention sees bf16(code * scale).  dtype KVF_BF16 and head_dim 128
                                   only (KVF_ERR_UNSUPPORTED otherwise, and for kvf_fold_step_static);
                                   the attention kernel expands code tiles to bf16 tiles in shared
-                                  memory, so a step reads d + 4 bytes per cached row.  Paged caches and
+                                  memory - or, for steps of at most 16 query rows (n_tokens * H/Hkv) on
+                                  a cache without a window, straight into the register fragments of its
+                                  MMAs - so a step reads d + 4 bytes per cached row.  Paged caches and
                                   batches of them take the flag too (see kvf_paged_cache_create) */
     KVF_CACHE_INT4 = 64u       /* the same with 4-bit codes (the other width the paper reports): scale =
                                   max|x| / 7, codes within +-7, stored two to a byte as code + 8 (element

@@ -17,8 +17,10 @@
 namespace kvf {
 namespace {
 
-constexpr int kTok = 2;        // tokens per CTA
-constexpr int kThreads = 256;
+// One token per CTA of 16 warps: a warp then has three of the token's 48 rows to do, one after the
+// other (each a load, a warp reduction and a store), instead of twelve.
+constexpr int kTok = 1;        // tokens per CTA
+constexpr int kThreads = 512;
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }

@@ -306,3 +306,29 @@ def test_decode_shaped_steps_on_a_quantised_cache_at_depth(bits, paged):
     torch.cuda.synchronize()
     assert cache.status() == binding.KVF_OK and len(cache) == total
     assert worst <= TOL["bf16"][0] and worst_lse <= 2e-2, (worst, worst_lse)
+
+
+def test_decode_steps_on_an_int8_cache_at_the_benchmark_prefix():
+    """The decode benchmark's launch configuration: prefix 129 024 (63 steps of 2048), then steps of one, two and
+    four tokens, every row of them against the oracle's quantised fold; 144 CTAs of the decode kernel."""
+    chunks = [2048] * 63 + [1, 1, 2, 4, 1]
+    total = sum(chunks)
+    cfg, cache = quant_cache(total, 2048, bits=8)
+    oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
+    oc.set_quant(8)
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert cache.plan(1, 129024) == (1, 18, 144, 3)
+    worst, worst_lse = 0.0, 0.0
+    for t, n in enumerate(chunks):
+        q, k, v = workloads.chunk_inputs(W, 131, t, device="cuda", n_tokens=n)
+        lse = torch.empty((n, W.n_q_heads), dtype=torch.float32, device="cuda")
+        out = cache.fold_step(q, k, v, lse=lse)
+        rows = list(range(n)) if n <= 4 else []
+        ref, ref_lse, _ = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows, want_stats=True)
+        if rows:
+            worst = max(worst, float(np.abs(to_f64(out) - ref).max()))
+            worst_lse = max(worst_lse, float(np.abs(to_f64(lse) - ref_lse).max()))
+    torch.cuda.synchronize()
+    assert cache.status() == binding.KVF_OK and len(cache) == total
+    assert worst <= TOL["bf16"][0] and worst_lse <= 2e-2, (worst, worst_lse)
+
