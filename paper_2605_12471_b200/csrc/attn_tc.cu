@@ -135,7 +135,12 @@ __device__ __forceinline__ void exp_half(const uint32_t *v, uint32_t *p, float2 
 // kQuant (0, 8 or 4 bits): map_k / map_v describe int8 or int4 code planes; the producer brings raw code tiles into their own
 // ring and warps 12-15 (one thread per key row) expand each to the swizzled bf16 tile the MMAs read,
 // value = bf16(code * row scale), which is what the FULL barriers then announce.
-template <bool kWindow, int kQuant>
+// kPair (quantised caches only): the CTAs of row pairs 2k and 2k + 1 form a cluster of two that walks
+// the same key tiles.  Each expands 64 of a tile's 128 key rows into its own slot and, with a bulk copy that
+// completes on the partner's FULL barrier, into the partner's; a slot is free once the issuers of BOTH CTAs
+// have committed their reads of it.  Each SM then expands half the codes.  The host launches this variant only
+// when both row pairs of every cluster need the same key tiles and have two row tiles.
+template <bool kWindow, int kQuant, bool kPair = false>
 __global__ void __launch_bounds__(kQuant ? kThreadsQ8 : kThreads, 1)
 attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v) {
@@ -149,8 +154,10 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     const uint32_t bar0 = base + offCtl;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
+    static_assert(!kPair || (kQuant != 0 && !kWindow), "the paired variant is for quantised caches without a window");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qpair = blockIdx.x, group = blockIdx.y;
+    const uint32_t rank = kPair ? cluster_cta_rank() : 0u;     // which of K (0) and V (1) this CTA expands
     const int cb = blockIdx.z;     // cache of a batch (0 when there is one cache)
     const int G = a.G;
     // (a ragged batch keeps its members' row counts in device memory, written by an earlier kernel
@@ -193,7 +200,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     if (threadIdx.x == 0) {
         mbar_init(bar(B_QFULL), 1);
         mbar_init(bar(B_QEMPTY), tiles);                                  // both issuers read Q
-        for (int s = 0; s < kRingBars; ++s) { mbar_init(bar(B_FULL0 + s), kQuant ? 4 : 1); mbar_init(bar(B_EMPTY0 + s), streams == 2 ? 1 : tiles); }   // consumers of a K/V tile
+        for (int s = 0; s < kRingBars; ++s) { mbar_init(bar(B_FULL0 + s), kQuant ? 4 : 1); mbar_init(bar(B_EMPTY0 + s), kPair ? 2 * tiles : streams == 2 ? 1 : tiles); }   // consumers of a K/V tile
         if (kQuant)
             for (int s = 0; s < kRawSlots; ++s) { mbar_init(bar(B_RAWFULL0 + s), 1); mbar_init(bar(B_RAWEMPTY0 + s), 4); }
         for (int i = 0; i < 2; ++i) {
@@ -215,6 +222,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
+    if (kPair) cluster_sync_all();      // the partner's barriers exist before anything is sent to them
     tc_fence_after();
     pdl_wait();   // nothing above reads what an earlier kernel wrote; from here on the rotated chunk is read
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&ctl->tmem_base);
@@ -232,7 +240,10 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     if (kQuant && warp >= 12) {
         // ------------------------------------------------------------------ int8 -> bf16 tile expansion
         asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-        const int t = (warp - 12) * 32 + lane;              // key row of the tile
+        // One thread per key row; in the paired variant two threads per row (64 codes each: the thread's
+        // half of d is one panel of the bf16 tile) and this CTA's 64 of the tile's 128 rows.
+        const int t = kPair ? (int)rank * 64 + (warp - 12) * 16 + (lane >> 1) : (warp - 12) * 32 + lane;   // key row of the tile
+        const uint32_t hd = kPair ? (uint32_t)(lane & 1) : 0u;                                           // my half of d
         const uint32_t sw = (uint32_t)(t & 7);
         int tg = 0, rg = 0;
         int rc[2] = {0, 0};
@@ -258,51 +269,69 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 float scale = 0.f;
                 if (key < a.capacity)
                     asm volatile("ld.shared.f32 %0, [%1];" : "=f"(scale) : "r"(base + kOffScaleQ8 + (uint32_t)r * 512u + (uint32_t)t * 4u));
-                const uint32_t dst = slot_addr(slot) + (uint32_t)t * 128u;
+                const uint32_t dst = slot_addr(slot) + (uint32_t)t * 128u + hd * kPanel;
                 const float2 sc = make_float2(scale, scale);
                 if (kQuant == 4) {
                     // 64-byte code rows, 64-byte swizzle: chunk c of row t sits at c ^ ((t >> 1) & 3)
+                    constexpr uint32_t NC = kPair ? 2 : 4;               // 16-byte chunks of codes I expand
                     const uint32_t src = base + kOffRawQ8 + (uint32_t)r * kRawBytes + (uint32_t)t * 64u;
                     const uint32_t sw4 = (uint32_t)((t >> 1) & 3);
-                    uint32_t w[16];
+                    uint32_t w[4 * NC];
 #pragma unroll
-                    for (uint32_t c = 0; c < 4; ++c)
+                    for (uint32_t c = 0; c < NC; ++c)
                         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                                     : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3]) : "r"(src + ((c ^ sw4) << 4)));
+                                     : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3]) : "r"(src + (((c + NC * hd) ^ sw4) << 4)));
 #pragma unroll
-                    for (uint32_t k = 0; k < 16; ++k) {            // word k = codes 8k .. 8k+7 = bf16 chunk k of the row
+                    for (uint32_t k = 0; k < 4 * NC; ++k) {        // word k = 8 codes = one 16-byte chunk of the bf16 row
                         uint32_t o[4];
                         expand8(w[k], sc, o);
                         asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k >> 3) * kPanel + (((k & 7) ^ sw) << 4)),
                                      "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
                     }
                 } else {
+                    constexpr uint32_t NC = kPair ? 4 : 8;               // 16-byte chunks of codes I expand
                     const uint32_t src = base + kOffRawQ8 + (uint32_t)r * kRawBytes + (uint32_t)t * 128u;
-                    // all eight 16-byte chunks of the code row first, then the arithmetic: the chunks are
+                    // all 16-byte chunks of the code row first, then the arithmetic: the chunks are
                     // independent, which is what gives one thread enough work in flight
-                    uint32_t w[32];
+                    uint32_t w[4 * NC];
 #pragma unroll
-                    for (uint32_t c = 0; c < 8; ++c)
+                    for (uint32_t c = 0; c < NC; ++c)
                         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                                     : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3]) : "r"(src + ((c ^ sw) << 4)));
+                                     : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3]) : "r"(src + (((c + NC * hd) ^ sw) << 4)));
 #pragma unroll
-                    for (uint32_t c = 0; c < 8; ++c) {
+                    for (uint32_t c = 0; c < NC; ++c) {
                         uint32_t o[8];
                         expand4(w[4 * c] ^ 0x80808080u, sc, o[0], o[1]);
                         expand4(w[4 * c + 1] ^ 0x80808080u, sc, o[2], o[3]);
                         expand4(w[4 * c + 2] ^ 0x80808080u, sc, o[4], o[5]);
                         expand4(w[4 * c + 3] ^ 0x80808080u, sc, o[6], o[7]);
-                        const uint32_t k0 = 2 * c, k1 = 2 * c + 1;     // 16-byte chunks of the bf16 row
+                        const uint32_t k0 = 2 * c, k1 = 2 * c + 1;     // 16-byte chunks of the bf16 row (of my panel, when paired)
                         asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k0 >> 3) * kPanel + (((k0 & 7) ^ sw) << 4)),
                                      "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
                         asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (k1 >> 3) * kPanel + (((k1 & 7) ^ sw) << 4)),
                                      "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
                     }
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read through the async proxy
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs (and the copy below) read through the async proxy
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(bar(B_FULL0 + slot));
+                    if (kPair) {
+                        // The partner's 64 rows are on their way: my warp's arrival on the FULL barrier of MY slot
+                        // (one of them also books the 16 KiB), then my warp's 16 rows of both panels to the same place
+                        // in the partner's slot, completing on the partner's barrier.  The slot is free in both CTAs
+                        // (the EMPTY barrier counts the issuers of both), and neither rewrites it before the other's
+                        // issuers have committed, which they do after these bytes have landed.
+                        if (warp == 12) mbar_expect_tx(bar(B_FULL0 + slot), kTileBytes / 2);
+                        else mbar_arrive(bar(B_FULL0 + slot));
+                        const uint32_t peer_bar = peer_smem(bar(B_FULL0 + slot), rank ^ 1u);
+#pragma unroll
+                        for (uint32_t p = 0; p < 2; ++p) {
+                            const uint32_t src = slot_addr(slot) + p * kPanel + ((uint32_t)rank * 64u + (uint32_t)(warp - 12) * 16u) * 128u;
+                            bulk_push(peer_smem(src, rank ^ 1u), src, 16u * 128u, peer_bar);
+                        }
+                    } else {
+                        mbar_arrive(bar(B_FULL0 + slot));
+                    }
                     mbar_arrive(bar(B_RAWEMPTY0 + r));
                 }
             }
@@ -342,7 +371,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                         // ... and the rows' scales behind it (as many as the plane still holds)
                         if (page_table) {
                             // paged cache: a key tile is one page, which always holds its 128 rows and their scales
-                            if (!(t & 1)) page = page_table[ktile];                // K then V of the same tile
+                            if (kPair || !(t & 1)) page = page_table[ktile];       // K then V of the same tile
                             const float *scales = ((t & 1) ? a.v_scales : a.k_scales) + (int64_t)page * a.scale_page_stride + kvh * kRows;
                             mbar_expect_tx(bar(B_RAWFULL0 + r), rawBytes + kRows * 4u);
                             tma_load_4d(base + kOffRawQ8 + (uint32_t)r * kRawBytes, m, bar(B_RAWFULL0 + r), 0, 0, kvh, page);
@@ -418,6 +447,12 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                     tc_mma_ts(t_o, t_s + kk * 8, vdesc + (uint64_t)((kk * 2048) >> 4), kIdescPV,
                               (accumulate || kk > 4 * h) ? 1u : 0u);
             };
+            // a K/V slot is free once its readers have run: in the paired variant the partner's expansion warps
+            // wait for my reads as well (they write my slot), so the commit goes to both CTAs' barriers
+            auto commit_empty = [&](int slot) {
+                if (kPair) tc_commit_pair(bar(B_EMPTY0 + slot));
+                else tc_commit(bar(B_EMPTY0 + slot));
+            };
             int tg = 0, it = 0, pc = 0;   // ring loads before this piece, my key tiles issued, pieces so far
             bool ok = true;
             // load number -> slot and parity: shared ring (number counts every load) or my own ring
@@ -449,14 +484,14 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                         if (!ok) break;
                         tc_fence_after();
                         issue_pv_half(vslot, 1, true);
-                        tc_commit(bar(B_EMPTY0 + vslot));
+                        commit_empty(vslot);
                     }
                     ok = mbar_wait(bar(B_FULL0 + kslot), kpar, ctl, a.status);
                     if (!ok) break;
                     tc_fence_after();
                     issue_qk(kslot);
                     tc_commit(bar(B_SFULL0 + i));
-                    tc_commit(bar(B_EMPTY0 + kslot));
+                    commit_empty(kslot);
                     jlast = j;
                 }
                 if (!ok) break;
@@ -475,7 +510,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                     tc_fence_after();
                     issue_pv_half(vslot, 1, true);
                     tc_commit(bar(B_OFINAL0 + i));
-                    tc_commit(bar(B_EMPTY0 + vslot));
+                    commit_empty(vslot);
                 }
                 tg += 2 * ntiles;
                 ++pc;
@@ -708,6 +743,8 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
 
     tc_fence_before();
     __syncthreads();
+    // (paired variant: neither CTA leaves while the partner may still send tiles or commits its way)
+    if (kPair) cluster_sync_all();
     if (warp == 9) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -827,6 +864,45 @@ int attn_tc_row_pairs(int n, int G) { return (n * G + 2 * kRows - 1) / (2 * kRow
 
 int attn_tc_streams(int n, int G) { return n * G <= kRows ? 2 : 1; }
 
+// Can the row pairs 2k and 2k + 1 of this launch share their expansions (paired variant)?  Every row pair
+// must have both row tiles, and the two of a cluster must need the same key tiles.
+static bool pair_launch_ok(const AttnArgs &a) {
+    if (!a.quant_bits || a.win_lo > 0 || a.streams != 1 || a.prefixes || a.ns || a.page_tables) return false;
+    const int64_t rows = (int64_t)a.n * a.G;
+    if (rows % (4 * kRows)) return false;
+    for (int64_t r0 = 0; r0 < rows; r0 += 4 * kRows) {
+        const int64_t last0 = (r0 + 2 * kRows - 1) / a.G, last1 = (r0 + 4 * kRows - 1) / a.G;
+        if ((a.prefix + last0 + kRows) / kRows != (a.prefix + last1 + kRows) / kRows) return false;   // ceil((P + last + 1) / 128)
+    }
+    return true;
+}
+
+// Do the clusters of two fill the device as single CTAs do (queried once per device)?
+static bool pair_clusters_fit(const void *kernel, uint32_t smem) {
+    static std::mutex mu;
+    static std::vector<std::pair<int, bool>> seen;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    for (auto &d : seen)
+        if (d.first == dev) return d.second;
+    int sms = 0, clusters = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2, 1024, 1);
+    cfg.blockDim = dim3(kThreadsQ8);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    bool fit = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+               cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) == cudaSuccess && 2 * clusters >= sms - sms % 2;
+    if (!fit) cudaGetLastError();
+    seen.push_back({dev, fit});
+    return fit;
+}
+
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
     static_assert(sizeof(Ctl) <= 512, "control block");
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
@@ -836,9 +912,16 @@ cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s
                 : a.quant_bits == 4 ? (a.win_lo > 0 ? attn_tc_kernel<true, 4> : attn_tc_kernel<false, 4>)
                                     : (a.win_lo > 0 ? attn_tc_kernel<true, 0> : attn_tc_kernel<false, 0>);
     const uint32_t smem = quant ? kSmemBytesQ8 : kSmemBytes;
+    dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, a.batch);
+    if (pair_launch_ok(a)) {
+        auto paired = a.quant_bits == 8 ? attn_tc_kernel<false, 8, true> : attn_tc_kernel<false, 4, true>;
+        cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(paired), (int)smem);
+        if (e != cudaSuccess) return e;
+        if (pair_clusters_fit(reinterpret_cast<const void *>(paired), smem))
+            return launch_pdl_cluster2(paired, grid, dim3(kThreadsQ8), smem, s, a, maps.q, maps.k, maps.v);
+    }
     cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(kernel), (int)smem);
     if (e != cudaSuccess) return e;
-    dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, a.batch);
     return launch_pdl(kernel, grid, dim3(quant ? kThreadsQ8 : kThreads), smem, s, a, maps.q, maps.k, maps.v);
 }
 

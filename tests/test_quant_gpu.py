@@ -231,6 +231,38 @@ def test_paged_quantised_cache_holds_the_same_codes_and_gives_the_same_bits(bits
 
 
 @BITS
+def test_two_ctas_sharing_their_expansions_give_the_bits_of_ctas_on_their_own(bits):
+    """Chunks whose row pairs come in twos that need the same key tiles (256, 512, 1024 tokens at prefixes that are
+    multiples of 128) run as clusters of two CTAs, each expanding half of every code tile for both.  A batch of one
+    cache never does.  Wherever both cut the key range alike the outputs are the same bits; everywhere they agree
+    within the tolerance, and with the oracle's quantised fold on sampled rows."""
+    chunks = [256] * 9 + [512, 1024, 256, 128, 256]
+    total = sum(chunks)
+    _, _, _, (alone,) = quant_paged_members(1, total, max(chunks), bits, seed=11)
+    _, _, _, (member,) = quant_paged_members(1, total, max(chunks), bits, seed=11)
+    batch = binding.Batch([member])
+    oc = oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base)
+    oc.set_quant(bits)
+    same_plan, worst, worst_oracle = 0, 0.0, 0.0
+    for t, n in enumerate(chunks):
+        q, k, v = workloads.chunk_inputs(W, 113, t, device="cuda", n_tokens=n)
+        prefix = len(alone)
+        got = alone.fold_step(q, k, v)
+        want = batch.fold_step(q[None].contiguous(), k[None].contiguous(), v[None].contiguous())[0]
+        if alone.plan(n, prefix)[1:] == batch.plan(n, prefix)[1:]:
+            same_plan += 1
+            assert torch.equal(got.view(torch.int16), want.view(torch.int16)), f"step {t}"
+        worst = max(worst, float((got.float() - want.float()).abs().max()))
+        rows = sorted({0, n // 2, n - 1})
+        ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows)
+        worst_oracle = max(worst_oracle, float(np.abs(to_f64(got[rows]) - ref).max()))
+    torch.cuda.synchronize()
+    assert alone.status() == binding.KVF_OK and batch.status_word() == 0
+    assert same_plan >= len(chunks) // 2, same_plan
+    assert worst <= TOL["bf16"][0] and worst_oracle <= TOL["bf16"][0], (worst, worst_oracle)
+
+
+@BITS
 def test_batch_of_paged_quantised_caches(bits):
     """One launch over three quantised paged caches: per member the bits of its own step, outputs within
     tolerance of the oracle's quantised fold; lock-step chunks, then a ragged step."""
