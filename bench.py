@@ -681,7 +681,7 @@ def run_chain_bench(args, w, drift=False):
         roofline["frac_of_tensor_rate_at_sampled_clock"] = attn_tflops * 1e12 / (prof_mhz * 1e6 * N_SMS * per_clock)
     if ns_b > ns_a:
         # the attention kernels inside the timed chains themselves (no events between the kernels there): time and
-        # cycles the first CTA of every launch was running, from the kernels' own counters
+        # cycles one CTA of every launch (its last row block) was running, from the kernels' own counters
         in_ms = (ns_b - ns_a) * 1e-6 / steps_timed
         roofline["in_timed_chains"] = {"attention_ms_per_chain": in_ms, "sm_mhz": 1e3 * (cyc_b - cyc_a) / (ns_b - ns_a),
                                        "attention_tflops": attn_flops / (in_ms * 1e-3) / 1e12,

@@ -253,7 +253,7 @@ kvf_status kvf_cache_status(kvf_cache *c);
 int32_t kvf_cache_status_word(kvf_cache *c);
 
 /* The SM clock the attention kernels ran at, measured by the kernels themselves.  (The paper has
- * no counterpart: a measurement aid.)  The first CTA of every tensor-core attention launch adds the
+ * no counterpart: a measurement aid.)  One CTA of every tensor-core attention launch (the last row block of the first key range) adds the
  * SM cycles and the nanoseconds (device timer) it was running to two sums kept beside the status
  * word; cycles_ns[0] / cycles_ns[1] receive the sums since the cache was created, so the difference
  * of two readings gives cycles * 1000 / ns = MHz over the launches in between.  Blocking copy, as

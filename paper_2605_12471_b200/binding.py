@@ -267,7 +267,7 @@ class Cache:
         return int(load().kvf_cache_status_word(self._h))
 
     def sm_clock(self) -> Tuple[int, int]:
-        """(SM cycles, nanoseconds) summed over the first CTA of every tensor-core attention launch so far."""
+        """(SM cycles, nanoseconds) summed over one CTA (last row block, first key range) of every tensor-core attention launch so far."""
         arr = (ctypes.c_uint64 * 2)()
         rc = load().kvf_cache_sm_clock(self._h, arr)
         if rc != KVF_OK:

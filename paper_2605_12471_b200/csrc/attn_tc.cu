@@ -96,7 +96,7 @@ struct Ctl {
     unsigned long long bars[40];
     uint32_t tmem_base;
     int abort;
-    long long clk0;                // start of the CTA in SM cycles and in nanoseconds (first CTA only)
+    long long clk0;                // start of the CTA in SM cycles and in nanoseconds (the timed CTA only)
     unsigned long long ns0;
 };
 static_assert(B_COUNT <= 40, "control block holds 40 barriers");
@@ -226,8 +226,9 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     tc_fence_after();
     pdl_wait();   // nothing above reads what an earlier kernel wrote; from here on the rotated chunk is read
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&ctl->tmem_base);
-    // CTA (0, 0, 0) times itself in SM cycles and in nanoseconds: the ratio is the clock the launch ran at
-    const bool clocked = (blockIdx.x | blockIdx.y | blockIdx.z) == 0 && threadIdx.x == 0;
+    // One CTA times itself in SM cycles and in nanoseconds: the ratio is the clock the launch ran at
+    // (the last row pair: it sees the most keys of the chunk itself, so no CTA of the launch runs longer)
+    const bool clocked = blockIdx.x == gridDim.x - 1 && (blockIdx.y | blockIdx.z) == 0 && threadIdx.x == 0;
     if (clocked) {
         ctl->clk0 = clock64();
         ctl->ns0 = global_ns();

@@ -89,7 +89,7 @@ struct Ctl {
     unsigned long long bars[32];
     uint32_t tmem_base;
     int abort;
-    long long clk0;                // start of the CTA in SM cycles and in nanoseconds (first CTA only)
+    long long clk0;                // start of the CTA in SM cycles and in nanoseconds (the timed CTA only)
     unsigned long long ns0;
 };
 static_assert(B_COUNT <= 32, "control block holds 32 barriers");
@@ -147,7 +147,12 @@ __device__ __forceinline__ void store_split4(uint8_t *part_hi, uint8_t *part_lo,
                  ::"r"(a[o + 0]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]), "r"(a[o + 5]), "r"(a[o + 6]), "r"(a[o + 7]), \
                    "r"(taddr) : "memory")
 
-template <bool kWindow>
+// kPair: the CTAs of row blocks 2k and 2k + 1 form a cluster of two that walks the same 64-key steps.  Each
+// converts 32 of a step's 64 key rows (K and V) into its own slot and, with bulk copies that complete on the
+// partner's FULL barrier, into the partner's; a slot is free once the issuers of BOTH CTAs have committed their
+// reads of it.  Each SM then loads and converts half the fp32 rows.  The host launches this variant only when
+// both row blocks of every cluster take the same steps.
+template <bool kWindow, bool kPair = false>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -157,6 +162,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rblock = blockIdx.x, group = blockIdx.y;
+    const uint32_t rank = kPair ? cluster_cta_rank() : 0u;
     const int G = a.G, n = a.n;
     const int64_t P = a.prefix, L = P + n;
     const bool direct = a.ngroups == a.Hkv;
@@ -190,8 +196,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
     if (threadIdx.x == 0) {
         mbar_init(bar(B_QFULL), 8);
         mbar_init(bar(B_QEMPTY), 1);
-        for (int s = 0; s < kKSlots; ++s) { mbar_init(bar(B_KFULL0 + s), 4); mbar_init(bar(B_KEMPTY0 + s), 1); }
-        for (int s = 0; s < kVSlots; ++s) { mbar_init(bar(B_VFULL0 + s), 4); mbar_init(bar(B_VEMPTY0 + s), 1); }
+        for (int s = 0; s < kKSlots; ++s) { mbar_init(bar(B_KFULL0 + s), 4); mbar_init(bar(B_KEMPTY0 + s), kPair ? 2 : 1); }
+        for (int s = 0; s < kVSlots; ++s) { mbar_init(bar(B_VFULL0 + s), 4); mbar_init(bar(B_VEMPTY0 + s), kPair ? 2 : 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(B_SFULL0 + i), 1);
             mbar_init(bar(B_SFREE0 + i), 4);
@@ -211,11 +217,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
     pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
+    if (kPair) cluster_sync_all();      // the partner's barriers exist before anything is sent to them
     tc_fence_after();
     pdl_wait();   // nothing above reads what an earlier kernel wrote; from here on the rotated chunk and the cache are read
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&ctl->tmem_base);
-    // CTA (0, 0) times itself in SM cycles and in nanoseconds: the ratio is the clock the launch ran at
-    const bool clocked = (blockIdx.x | blockIdx.y) == 0 && threadIdx.x == 0;
+    // One CTA times itself in SM cycles and in nanoseconds: the ratio is the clock the launch ran at
+    // (the last row block: it sees the most keys of the chunk itself, so no CTA of the launch runs longer)
+    const bool clocked = blockIdx.x == gridDim.x - 1 && blockIdx.y == 0 && threadIdx.x == 0;
     if (clocked) {
         ctl->clk0 = clock64();
         ctl->ns0 = global_ns();
@@ -255,7 +263,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
                         tc_mma(t_s, dql + qo, dk + ko, kIdescQK64, 1);
                     }
                     tc_commit(bar(B_SFULL0 + b));
-                    tc_commit(bar(B_KEMPTY0 + slot));
+                    if (kPair) tc_commit_pair(bar(B_KEMPTY0 + slot));     // the partner's converters write my slot too
+                    else tc_commit(bar(B_KEMPTY0 + slot));
                 }
                 if (!ok) break;
                 tc_commit(bar(B_QEMPTY));                     // every Q K^T of this piece has been issued
@@ -290,7 +299,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
                     for (int kk = 0; kk < 4; ++kk)
                         tc_mma_ts(t_o, p_hi + kk * 8, dvh + (uint64_t)((kk * 2048) >> 4), kIdescPV, 1);
                     tc_commit(bar(B_OFULL));
-                    tc_commit(bar(B_VEMPTY0 + slot));
+                    if (kPair) tc_commit_pair(bar(B_VEMPTY0 + slot));
+                    else tc_commit(bar(B_VEMPTY0 + slot));
                 }
             }
             tc_commit(bar(B_DRAIN0 + 1));
@@ -335,13 +345,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
                 ++pc;
             }
             const float *head = plane + (int64_t)kvh * a.capacity * kD;
+            // rows of a step this warp converts: 16 of the 64, or 8 of this CTA's 32 in the paired variant
+            constexpr int NR = kPair ? 8 : 16;
+            const int r0 = kPair ? (int)rank * 32 + w4 * 8 : w4 * 16;
             for (int s = 0; s < nsteps; ++s, ++lc) {
                 const int64_t key0 = step_key0(kt0, s);
                 // rows past the end of the cache are not content (and may hold anything): they count as zero
-                float4 x[16];
+                float4 x[NR];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int64_t key = key0 + w4 * 16 + i;
+                for (int i = 0; i < NR; ++i) {
+                    const int64_t key = key0 + r0 + i;
                     x[i] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (key < L) x[i] = *reinterpret_cast<const float4 *>(head + key * kD + lane * 4);
                 }
@@ -354,10 +367,30 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
                 uint8_t *dst_lo = dst + (is_v ? kKPart : kKPanel);
                 const uint32_t panel = is_v ? kKPanel : kKOperand;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) store_split4(dst, dst_lo, panel, w4 * 16 + i, lane, x[i]);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                for (int i = 0; i < NR; ++i) store_split4(dst, dst_lo, panel, r0 + i, lane, x[i]);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs (and the copies below) read through the async proxy
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(b_full + slot));
+                if (lane == 0) {
+                    if (kPair) {
+                        // The partner's 32 rows are on their way: my warp's arrival on the FULL barrier of MY slot (one
+                        // of them also books the 16 KiB), then my warp's 8 rows of the four blocks (hi and lo of both
+                        // panels) to the same place in the partner's slot, completing on the partner's barrier.  The slot
+                        // is free in both CTAs (the EMPTY barrier counts the issuers of both), and neither rewrites it
+                        // before the other's issuer has committed, which it does after these bytes have landed.
+                        if (w4 == 0) mbar_expect_tx(bar(b_full + slot), kKSlot / 2);
+                        else mbar_arrive(bar(b_full + slot));
+                        const uint32_t peer_bar = peer_smem(bar(b_full + slot), rank ^ 1u);
+                        const uint32_t s_hi = base + ring + (uint32_t)slot * kKSlot + (uint32_t)r0 * 128u;
+                        const uint32_t s_lo = s_hi + (is_v ? kKPart : kKPanel);
+#pragma unroll
+                        for (uint32_t pnl = 0; pnl < 2; ++pnl) {
+                            bulk_push(peer_smem(s_hi + pnl * panel, rank ^ 1u), s_hi + pnl * panel, 8u * 128u, peer_bar);
+                            bulk_push(peer_smem(s_lo + pnl * panel, rank ^ 1u), s_lo + pnl * panel, 8u * 128u, peer_bar);
+                        }
+                    } else {
+                        mbar_arrive(bar(b_full + slot));
+                    }
+                }
             }
         }
     } else {
@@ -539,6 +572,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
 
     tc_fence_before();
     __syncthreads();
+    // (paired variant: neither CTA leaves while the partner may still send tiles or commits its way)
+    if (kPair) cluster_sync_all();
     if (warp == 12) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -554,13 +589,62 @@ bool attn_tc32_supported(int dtype, int d, int G) {
 
 int attn_tc32_row_blocks(int n, int G) { return (n * G + kRows - 1) / kRows; }
 
+// Can the row blocks 2k and 2k + 1 of this launch share their conversions (paired variant)?  The two of a
+// cluster must take the same 64-key steps of every piece (the same arithmetic as the kernel's piece()).
+static bool pair_launch_ok32(const AttnArgs &a) {
+    if (a.win_lo > 0) return false;
+    const int64_t rows = (int64_t)a.n * a.G;
+    if (rows % (2 * kRows)) return false;
+    for (int64_t r0 = 0; r0 < rows; r0 += 2 * kRows) {
+        const int64_t need0 = a.prefix + (r0 + kRows - 1) / a.G + 1, need1 = a.prefix + (r0 + 2 * kRows - 1) / a.G + 1;
+        // tiles needed, and whether the second half of the last one is
+        if ((need0 + kTileKeys - 1) / kTileKeys != (need1 + kTileKeys - 1) / kTileKeys) return false;
+        const int64_t last_half = ((need1 + kTileKeys - 1) / kTileKeys - 1) * kTileKeys + kKeys;
+        if ((last_half >= need0) != (last_half >= need1)) return false;
+    }
+    return true;
+}
+
+// Do the clusters of two fill the device as single CTAs do (queried once per device)?
+static bool pair_clusters_fit32(const void *kernel) {
+    static std::mutex mu;
+    static std::vector<std::pair<int, bool>> seen;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    for (auto &d : seen)
+        if (d.first == dev) return d.second;
+    int sms = 0, clusters = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2, 1024, 1);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    bool fit = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+               cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) == cudaSuccess && 2 * clusters >= sms - sms % 2;
+    if (!fit) cudaGetLastError();
+    seen.push_back({dev, fit});
+    return fit;
+}
+
 cudaError_t launch_attn_tc32(const AttnArgs &a, cudaStream_t s) {
     static_assert(sizeof(Ctl) <= 512, "control block");
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
+    dim3 grid(attn_tc32_row_blocks(a.n, a.G), a.ngroups, 1);
+    if (pair_launch_ok32(a)) {
+        auto paired = attn_tc32_kernel<false, true>;
+        cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(paired), (int)kSmemBytes);
+        if (e != cudaSuccess) return e;
+        if (pair_clusters_fit32(reinterpret_cast<const void *>(paired)))
+            return launch_pdl_cluster2(paired, grid, dim3(kThreads), kSmemBytes, s, a);
+    }
     auto kernel = a.win_lo > 0 ? attn_tc32_kernel<true> : attn_tc32_kernel<false>;
     cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(kernel), (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    dim3 grid(attn_tc32_row_blocks(a.n, a.G), a.ngroups, 1);
     return launch_pdl(kernel, grid, dim3(kThreads), kSmemBytes, s, a);
 }
 

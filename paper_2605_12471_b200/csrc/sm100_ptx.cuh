@@ -38,7 +38,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 
 // The 256-byte status block of a workspace: word 0 is the status word; bytes 16-31 hold two running
-// sums, SM cycles and nanoseconds that the first CTA of every tensor-core attention launch spent
+// sums, SM cycles and nanoseconds that one CTA (the last row block of the first key range) of every tensor-core attention launch spent
 // (one thread of one CTA per launch writes them, and launches of a stream do not overlap).
 __device__ __forceinline__ void add_clock_counters(int *status, long long cycles, unsigned long long ns) {
     unsigned long long *ctr = reinterpret_cast<unsigned long long *>(status) + 2;
