@@ -85,7 +85,9 @@ enum {
                                   merge left open outside its own capture returns KVF_ERR_INVALID_ARG and
                                   enqueues nothing - flush before a capture begins and before it ends.  The
                                   stream and its events are made by kvf_cache_create /
-                                  kvf_paged_cache_create, and kvf_workspace_bytes grows by the second set;
+                                  kvf_paged_cache_create, and kvf_workspace_bytes grows by the second set.
+                                  Needs a workspace that no other cache's steps use while a merge is open
+                                  (the merge reads its partial results there behind the caller's stream);
                                   batches and kvf_fold_step_static ignore the flag */
     KVF_CACHE_INT8 = 16u,      /* store the cache as int8 codes with one fp32 scale per row (one token of
                                   one KV head): d + 4 bytes per row instead of 2 d (kvf_cache_storage_bytes
