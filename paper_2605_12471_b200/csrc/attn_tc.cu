@@ -139,7 +139,7 @@ __device__ __forceinline__ void exp_half(const uint32_t *v, uint32_t *p, float2 
 // the same key tiles.  Each expands 64 of a tile's 128 key rows into its own slot and, with a bulk copy that
 // completes on the partner's FULL barrier, into the partner's; a slot is free once the issuers of BOTH CTAs
 // have committed their reads of it.  Each SM then expands half the codes.  The host launches this variant only
-// when both row pairs of every cluster need the same key tiles and have two row tiles.
+// when every row pair has two row tiles (a chunk of a multiple of 512 / G tokens).
 template <bool kWindow, int kQuant, bool kPair = false>
 __global__ void __launch_bounds__(kQuant ? kThreadsQ8 : kThreads, 1)
 attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -179,7 +179,9 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     // short chunks (at most 128 / G tokens in this row pair) leave the second row tile without a
     // valid row: its issuer and softmax warps then sit the kernel out
     const int tiles = (streams == 2 || row0 + kRows < n * G) ? 2 : 1;
-    const int tok_last = min(n - 1, (row0 + 2 * kRows - 1) / G);
+    // (paired variant: both CTAs of a cluster walk the key tiles the later row pair needs; the earlier one
+    // finds nothing visible in the last of them, and its rows' limits mask that tile out)
+    const int tok_last = min(n - 1, ((kPair ? (qpair | 1) * 2 * kRows : row0) + 2 * kRows - 1) / G);
     // (virtual key tiles: without a window they are the key tiles themselves)
     const WindowTiles wt(kWindow ? a.win_lo : 0, kWindow ? a.n_sink : 0, kRows);
     const int nt_need = (int)((P + tok_last + 1 + kRows - 1) / kRows) - wt.skip;
@@ -866,16 +868,10 @@ int attn_tc_row_pairs(int n, int G) { return (n * G + 2 * kRows - 1) / (2 * kRow
 int attn_tc_streams(int n, int G) { return n * G <= kRows ? 2 : 1; }
 
 // Can the row pairs 2k and 2k + 1 of this launch share their expansions (paired variant)?  Every row pair
-// must have both row tiles, and the two of a cluster must need the same key tiles.
+// must have both row tiles (the two of a cluster then walk the key tiles of the later one).
 static bool pair_launch_ok(const AttnArgs &a) {
     if (!a.quant_bits || a.win_lo > 0 || a.streams != 1 || a.prefixes || a.ns || a.page_tables) return false;
-    const int64_t rows = (int64_t)a.n * a.G;
-    if (rows % (4 * kRows)) return false;
-    for (int64_t r0 = 0; r0 < rows; r0 += 4 * kRows) {
-        const int64_t last0 = (r0 + 2 * kRows - 1) / a.G, last1 = (r0 + 4 * kRows - 1) / a.G;
-        if ((a.prefix + last0 + kRows) / kRows != (a.prefix + last1 + kRows) / kRows) return false;   // ceil((P + last + 1) / 128)
-    }
-    return true;
+    return ((int64_t)a.n * a.G) % (4 * kRows) == 0;
 }
 
 // Do the clusters of two fill the device as single CTAs do (queried once per device)?

@@ -151,7 +151,7 @@ __device__ __forceinline__ void store_split4(uint8_t *part_hi, uint8_t *part_lo,
 // converts 32 of a step's 64 key rows (K and V) into its own slot and, with bulk copies that complete on the
 // partner's FULL barrier, into the partner's; a slot is free once the issuers of BOTH CTAs have committed their
 // reads of it.  Each SM then loads and converts half the fp32 rows.  The host launches this variant only when
-// both row blocks of every cluster take the same steps.
+// the row blocks come in twos (a chunk of a multiple of 256 / G tokens).
 template <bool kWindow, bool kPair = false>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a) {
     extern __shared__ uint8_t smem_raw[];
@@ -167,7 +167,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
     const int64_t P = a.prefix, L = P + n;
     const bool direct = a.ngroups == a.Hkv;
     const int row0 = rblock * kRows;
-    const int tok_last = min(n - 1, (row0 + kRows - 1) / G);
+    // (paired variant: both CTAs of a cluster take the steps the later row block needs; the earlier one finds
+    // nothing visible in the last of them, and its rows' limits mask those keys out)
+    const int tok_last = min(n - 1, ((kPair ? (rblock | 1) * kRows : row0) + kRows - 1) / G);
     const int64_t need = P + tok_last + 1;            // keys below `need` are visible to some row of this CTA
     // (virtual key tiles: without a window they are the key tiles themselves)
     const WindowTiles wt(kWindow ? a.win_lo : 0, kWindow ? a.n_sink : 0, kTileKeys);
@@ -589,20 +591,10 @@ bool attn_tc32_supported(int dtype, int d, int G) {
 
 int attn_tc32_row_blocks(int n, int G) { return (n * G + kRows - 1) / kRows; }
 
-// Can the row blocks 2k and 2k + 1 of this launch share their conversions (paired variant)?  The two of a
-// cluster must take the same 64-key steps of every piece (the same arithmetic as the kernel's piece()).
+// Can the row blocks 2k and 2k + 1 of this launch share their conversions (paired variant)?  The row blocks
+// must come in twos (the two of a cluster then take the steps of the later one).
 static bool pair_launch_ok32(const AttnArgs &a) {
-    if (a.win_lo > 0) return false;
-    const int64_t rows = (int64_t)a.n * a.G;
-    if (rows % (2 * kRows)) return false;
-    for (int64_t r0 = 0; r0 < rows; r0 += 2 * kRows) {
-        const int64_t need0 = a.prefix + (r0 + kRows - 1) / a.G + 1, need1 = a.prefix + (r0 + 2 * kRows - 1) / a.G + 1;
-        // tiles needed, and whether the second half of the last one is
-        if ((need0 + kTileKeys - 1) / kTileKeys != (need1 + kTileKeys - 1) / kTileKeys) return false;
-        const int64_t last_half = ((need1 + kTileKeys - 1) / kTileKeys - 1) * kTileKeys + kKeys;
-        if ((last_half >= need0) != (last_half >= need1)) return false;
-    }
-    return true;
+    return a.win_lo <= 0 && ((int64_t)a.n * a.G) % (2 * kRows) == 0;
 }
 
 // Do the clusters of two fill the device as single CTAs do (queried once per device)?

@@ -232,11 +232,12 @@ def test_paged_quantised_cache_holds_the_same_codes_and_gives_the_same_bits(bits
 
 @BITS
 def test_two_ctas_sharing_their_expansions_give_the_bits_of_ctas_on_their_own(bits):
-    """Chunks whose row pairs come in twos that need the same key tiles (256, 512, 1024 tokens at prefixes that are
-    multiples of 128) run as clusters of two CTAs, each expanding half of every code tile for both.  A batch of one
-    cache never does.  Wherever both cut the key range alike the outputs are the same bits; everywhere they agree
-    within the tolerance, and with the oracle's quantised fold on sampled rows."""
-    chunks = [256] * 9 + [512, 1024, 256, 128, 256]
+    """Chunks whose row pairs come in twos (128, 256, 512, 1024 tokens) run as clusters of two CTAs, each expanding
+    half of every code tile for both, at any prefix: the two walk the key tiles of the later row pair, and the
+    earlier one masks what it does not see (the chunks after the 100-token one start off the tile grid).  A batch
+    of one cache never does.  Wherever both cut the key range alike the outputs are the same bits; everywhere they
+    agree within the tolerance, and with the oracle's quantised fold on sampled rows."""
+    chunks = [256] * 5 + [100] + [256] * 4 + [512, 1024, 256, 128, 256]
     total = sum(chunks)
     _, _, _, (alone,) = quant_paged_members(1, total, max(chunks), bits, seed=11)
     _, _, _, (member,) = quant_paged_members(1, total, max(chunks), bits, seed=11)
@@ -253,7 +254,7 @@ def test_two_ctas_sharing_their_expansions_give_the_bits_of_ctas_on_their_own(bi
             same_plan += 1
             assert torch.equal(got.view(torch.int16), want.view(torch.int16)), f"step {t}"
         worst = max(worst, float((got.float() - want.float()).abs().max()))
-        rows = sorted({0, n // 2, n - 1})
+        rows = sorted({0, 1, n // 4, n // 2 - 1, n // 2, n - 1})     # rows of both CTAs of a cluster
         ref = oc.fold_step(to_f64(q), to_f64(k), to_f64(v), rows=rows)
         worst_oracle = max(worst_oracle, float(np.abs(to_f64(got[rows]) - ref).max()))
     torch.cuda.synchronize()
