@@ -100,8 +100,9 @@ enum {
                                   only (KVF_ERR_UNSUPPORTED otherwise, and for kvf_fold_step_static);
                                   the attention kernel expands code tiles to bf16 tiles in shared
                                   memory - or, for steps of at most 16 query rows (n_tokens * H/Hkv) on
-                                  a cache without a window, straight into the register fragments of its
-                                  MMAs - so a step reads d + 4 bytes per cached row.  Paged caches and
+                                  a cache (or a batch of caches) without a window, straight into the
+                                  register fragments of its MMAs - so a step reads d + 4 bytes per
+                                  cached row.  Paged caches and
                                   batches of them take the flag too (see kvf_paged_cache_create) */
     KVF_CACHE_INT4 = 64u       /* the same with 4-bit codes (the other width the paper reports): scale =
                                   max|x| / 7, codes within +-7, stored two to a byte as code + 8 (element

@@ -198,7 +198,8 @@ class Cache:
         self.out_dtype = torch.float32 if (cfg.flags & KVF_OUT_F32) else self.torch_dtype
 
     def close(self):
-        if getattr(self, "_h", None):
+        # (at interpreter shutdown the module's globals may already be gone: then the process ends anyway)
+        if getattr(self, "_h", None) and load is not None:
             load().kvf_cache_destroy(self._h)
             self._h = None
 
@@ -426,7 +427,7 @@ class Batch:
         self._h = h
 
     def close(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and load is not None:
             load().kvf_batch_destroy(self._h)
             self._h = None
 

@@ -187,9 +187,17 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t4 = lane & 3;
     const int group = blockIdx.x;
-    const int G = a.G, n = a.n, nG = n * G;
-    const int64_t P = a.prefix, L = P + n;
+    const int cb = blockIdx.y;     // cache of a batch (0 when there is one cache)
+    const int G = a.G;
+    // (a ragged batch keeps its members' row counts in device memory, written by an earlier kernel of the
+    // stream: those are the one thing read before the set-up below, so wait first there)
+    if (a.prefixes) pdl_wait();
+    // tokens this cache folds; a.n is the longest chunk of the launch and the stride of the caches' blocks
+    const int n = a.ns ? (int)a.ns[cb] : a.n, nmax = a.n, nG = n * G;
+    if (n <= 0) return;                                   // a member that sits the step out
+    const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix, L = P + n;
     const bool direct = a.ngroups == a.Hkv;
+    const int64_t slot_rows = (int64_t)nmax * G;          // rows of a partial slot
 
     // this CTA's range of its KV head's key tiles (the same line arithmetic as the other kernels)
     const int nt_all = (int)((L + kKeysPerTile - 1) / kKeysPerTile);
@@ -198,6 +206,19 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     const int kvh = (int)(lin0 / nt_all);
     const int kt0 = (int)(lin0 - (int64_t)kvh * nt_all);
     const int ntiles = (int)(lin1 - lin0);         // a multiple of the KV heads cuts the line inside heads
+    if (ntiles <= 0) {
+        // A shorter member of a ragged batch (or a forced split count) can leave a range without a tile: an
+        // empty partial, for the merge reads every slot between a head's first and last range.
+        pdl_wait();   // (the partial area may still be read by the merge of the step before)
+        if (!direct && kvh < a.Hkv)
+            for (int item = threadIdx.x; item < nG * (kD / 4); item += blockDim.x) {
+                const int r = item / (kD / 4), c4 = item % (kD / 4);
+                const int64_t prow = (int64_t)cb * a.part_rows + (int64_t)(group + kvh) * slot_rows + r;
+                reinterpret_cast<float4 *>(a.part_o + prow * kD)[c4] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (c4 == 0) a.part_lse[prow] = -INFINITY;
+            }
+        return;
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NST; ++s) {
@@ -230,7 +251,7 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         if (lane == 0) {
             // ------------------------------------------------------------------ TMA producer
             bool ok = true;
-            const int32_t *page_table = a.page_table;
+            const int32_t *page_table = a.page_tables ? a.page_tables[cb] : a.page_table;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int s = t % NST;
                 ok = mbar_wait(bar_empty + 8 * s, ((t / NST) & 1) ^ 1, ctl, a.status);
@@ -271,7 +292,7 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb) {
                 const int R = g + 8 * nb, tok = R / G, gi = R % G;
-                const __nv_bfloat16 *src = q_rot + ((int64_t)tok * a.H + kvh * G + gi) * kD + 32 * t4;
+                const __nv_bfloat16 *src = q_rot + (((int64_t)cb * nmax + tok) * a.H + kvh * G + gi) * kD + 32 * t4;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     uint2 w = make_uint2(0u, 0u);
@@ -454,9 +475,9 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             const float inv = den > 0.f ? 1.f / den : 0.f;
             const float lse2 = den > 0.f ? M + log2f(den) : -INFINITY;
             const int tok = r / G, gi = r % G;
-            const int64_t row = (int64_t)tok * a.H + kvh * G + gi;
+            const int64_t row = ((int64_t)cb * nmax + tok) * a.H + kvh * G + gi;
             if (!direct) {
-                const int64_t prow = (int64_t)(group + kvh) * nG + r;
+                const int64_t prow = (int64_t)cb * a.part_rows + (int64_t)(group + kvh) * slot_rows + r;
                 float4 *dst = reinterpret_cast<float4 *>(a.part_o + prow * kD + c0);
                 dst[0] = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
                 dst[1] = make_float4(acc[4] * inv, acc[5] * inv, acc[6] * inv, acc[7] * inv);
@@ -493,7 +514,7 @@ cudaError_t launch_attn_q8_decode(const AttnArgs &a, const TcMaps &maps, cudaStr
     cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(kernel), (int)smem);
     if (e != cudaSuccess) return e;
     const int threads = wide ? Geo<8, 2>::kThreads : Geo<8, 1>::kThreads;
-    return launch_pdl(kernel, dim3(a.ngroups), dim3(threads), smem, s, a, maps.k, maps.v);
+    return launch_pdl(kernel, dim3(a.ngroups, a.batch), dim3(threads), smem, s, a, maps.k, maps.v);
 }
 
 }  // namespace kvf

@@ -332,7 +332,6 @@ int64_t window_lo(const kvf_cache *c, int64_t prefix) {
 }
 
 Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t part_rows_cap = -1) {
-    const bool single = part_rows_cap < 0;      // a step of one cache through its own handle (not a batch of one)
     if (part_rows_cap < 0) part_rows_cap = c->part_rows_cap;
     Plan p;
     p.qdec = false;
@@ -340,11 +339,11 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
     p.ngroups = 0;
     const int64_t L = prefix + n;
     const int Hkv = c->cfg.n_kv_heads;
-    if (c->quant && single && c->window <= 0 && n * c->G <= attn_q8_decode_max_rows()) {
-        // one CTA per SM, each inside one KV head (a multiple of the KV heads), at least two key tiles each;
-        // a forced split count is the number of ranges per KV head
+    if (c->quant && c->window <= 0 && n * c->G <= attn_q8_decode_max_rows()) {
+        // one CTA per SM (all caches of a batch together), each inside one KV head (a multiple of the KV heads),
+        // at least two key tiles each; a forced split count is the number of ranges per KV head
         const int64_t nt = (L + kKvTile - 1) / kKvTile;
-        int64_t per_head = c->force_splits > 0 ? c->force_splits : c->sm_count / Hkv;
+        int64_t per_head = c->force_splits > 0 ? c->force_splits : c->sm_count / (Hkv * batch);
         if (c->force_splits <= 0 && per_head > nt / 2) per_head = nt / 2;
         if (per_head > nt) per_head = nt;
         const int64_t slots_cap = part_rows_cap / ((int64_t)n * c->G);            // slots = groups + Hkv - 1
@@ -353,7 +352,7 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
         p.qdec = true;
         p.ngroups = (int)(per_head * Hkv);
         p.splits = (int)per_head;
-        p.ctas = p.ngroups;
+        p.ctas = p.ngroups * batch;
         p.kernels = 2 + (per_head > 1 ? 1 : 0);
         return p;
     }
@@ -1203,7 +1202,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c0->G; aa.d = f.head_dim;
     aa.splits = 1;
     aa.ngroups = plan.ngroups;
-    aa.streams = attn_tc_streams(n, c0->G);
+    aa.streams = plan.qdec ? 1 : attn_tc_streams(n, c0->G);
     aa.out_f32 = (f.flags & KVF_OUT_F32) ? 1 : 0;
     aa.scale_log2 = c0->scale_log2;
     aa.range_valid = 0;
@@ -1216,7 +1215,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     b->launches++;
     TcMaps maps = c0->maps;
     maps.q = b->map_q;
-    e = launch_attn_tc(aa, maps, st);
+    e = plan.qdec ? launch_attn_q8_decode(aa, maps, st) : launch_attn_tc(aa, maps, st);
     if (e != cudaSuccess) return cuda_fail(e, "attention launch (batch)");
     b->launches++;
     if (plan.kernels > 2) {

@@ -308,6 +308,85 @@ def test_batch_of_paged_quantised_caches(bits):
 
 
 @BITS
+def test_batch_of_quantised_caches_decoding_together(bits):
+    """Decode-shaped steps of a batch (at most 16 query rows per member) take the decode kernel with the cache in
+    the grid: members in lock step, members of different length (one far shorter than the key ranges the longest
+    one is cut into), members that take fewer tokens or sit a step out.  Per member the pool ends up bit-identical
+    to folding it by itself; every row of every step against the oracle's quantised fold."""
+    B = 5
+    extra = [0, 40, 700, 3, 1300]                      # tokens the members fold on their own after the common prefix
+    total = 2 * 2048 + max(extra) + 64
+    cfg, pool, tables, caches = quant_paged_members(B, total, 2048, bits, seed=21)
+    _, pool1, _, singles = quant_paged_members(B, total, 2048, bits, seed=21)
+    batch = binding.Batch(caches)
+    ocs = [oracle.OracleCache(W.n_q_heads, W.n_kv_heads, W.head_dim, total, rope_base=W.rope_base) for _ in range(B)]
+    for oc in ocs:
+        oc.set_quant(bits)
+
+    def inputs(n, seed, t):
+        qs, ks, vs = zip(*[workloads.chunk_inputs(W, seed, t, sequence=i, device="cuda", n_tokens=n) for i in range(B)])
+        return tuple(torch.stack(x).contiguous() for x in (qs, ks, vs))
+
+    worst, worst_lse, worst_pair = 0.0, 0.0, 0.0
+
+    def check(out, lse, q, k, v, ns):
+        nonlocal worst, worst_lse, worst_pair
+        for i, n in enumerate(ns):
+            if n == 0:
+                continue
+            qi, ki, vi = (x[i, :n].contiguous() for x in (q, k, v))
+            alone = singles[i].fold_step(qi, ki, vi)
+            worst_pair = max(worst_pair, float((out[i, :n].float() - alone.float()).abs().max()))
+            rows = list(range(n)) if n <= 4 else []
+            ref, ref_lse, _ = ocs[i].fold_step(to_f64(qi), to_f64(ki), to_f64(vi), rows=rows, want_stats=True)
+            if rows:
+                worst = max(worst, float(np.abs(to_f64(out[i, :n]) - ref).max()))
+                worst_lse = max(worst_lse, float(np.abs(to_f64(lse[i, :n]) - ref_lse).max()))
+
+    # the common prefix, in lock step (the long-chunk kernel), and two lock-step decode steps
+    for t, n in enumerate([2048, 2048, 1, 4]):
+        q, k, v = inputs(n, 141, t)
+        lse = torch.empty((B, n, W.n_q_heads), dtype=torch.float32, device="cuda")
+        if n <= 4 and torch.cuda.get_device_properties(0).multi_processor_count == 148:
+            assert batch.plan(n) == (1, 3, 120, 3)             # 148 / (8 KV heads x 5 caches) = 3 ranges per head and cache
+        out = batch.fold_step(q, k, v, lse=lse)
+        check(out, lse, q, k, v, [n] * B)
+    # members of different length
+    for i, n in enumerate(extra):
+        if n:
+            q1, k1, v1 = workloads.chunk_inputs(W, 142, 0, sequence=i, device="cuda", n_tokens=n)
+            caches[i].fold_step(q1, k1, v1)
+            singles[i].fold_step(q1, k1, v1)
+            ocs[i].fold_step(to_f64(q1), to_f64(k1), to_f64(v1), rows=[])
+    for t, n in enumerate([1, 2, 4, 1]):
+        q, k, v = inputs(n, 143, t)
+        lse = torch.empty((B, n, W.n_q_heads), dtype=torch.float32, device="cuda")
+        out = batch.fold_step(q, k, v, lse=lse, ragged=True)
+        check(out, lse, q, k, v, [n] * B)
+    # more key ranges per KV head than the members have key tiles: ranges without a tile leave empty partials
+    caches[0].set_splits(48)
+    q, k, v = inputs(1, 145, 0)
+    lse = torch.empty((B, 1, W.n_q_heads), dtype=torch.float32, device="cuda")
+    out = batch.fold_step(q, k, v, lse=lse, ragged=True)
+    check(out, lse, q, k, v, [1] * B)
+    caches[0].set_splits(0)
+    # fewer tokens for some, none for others
+    for t, (mx, ns) in enumerate([(2, [1, 0, 2, 1, 2]), (4, [4, 3, 0, 0, 1]), (1, [0, 1, 0, 1, 1])]):
+        q, k, v = inputs(mx, 144, t)
+        out = torch.full(q.shape, 7.0, dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((B, mx, W.n_q_heads), 7.0, dtype=torch.float32, device="cuda")
+        batch.fold_step_varlen(q, k, v, ns, out=out, lse=lse)
+        for i, n in enumerate(ns):
+            assert bool((out[i, n:] == 7.0).all()) and bool((lse[i, n:] == 7.0).all())
+        check(out, lse, q, k, v, ns)
+    torch.cuda.synchronize()
+    assert batch.status_word() == 0 and all(c.status() == binding.KVF_OK for c in caches)
+    assert [len(c) for c in caches] == [len(c) for c in singles] == [len(oc) for oc in ocs]
+    assert torch.equal(pool, pool1)                        # every code and every scale, page for page
+    assert worst <= TOL["bf16"][0] and worst_pair <= TOL["bf16"][0] and worst_lse <= 2e-2, (worst, worst_pair, worst_lse)
+
+
+@BITS
 @pytest.mark.parametrize("paged", [False, True], ids=["contiguous", "paged"])
 def test_decode_shaped_steps_on_a_quantised_cache_at_depth(bits, paged):
     """One to four tokens per step (at most 16 query rows) after a long prefix: the kernel that expands codes
