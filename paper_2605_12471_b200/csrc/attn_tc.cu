@@ -870,7 +870,8 @@ int attn_tc_streams(int n, int G) { return n * G <= kRows ? 2 : 1; }
 // Can the row pairs 2k and 2k + 1 of this launch share their expansions (paired variant)?  Every row pair
 // must have both row tiles (the two of a cluster then walk the key tiles of the later one).
 static bool pair_launch_ok(const AttnArgs &a) {
-    if (!a.quant_bits || a.win_lo > 0 || a.streams != 1 || a.prefixes || a.ns || a.page_tables) return false;
+    // (members of a batch that take fewer tokens than the launch's chunk may lack a row tile: no pairs then)
+    if (!a.quant_bits || a.win_lo > 0 || a.streams != 1 || a.ns) return false;
     return ((int64_t)a.n * a.G) % (4 * kRows) == 0;
 }
 

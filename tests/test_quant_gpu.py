@@ -234,8 +234,9 @@ def test_paged_quantised_cache_holds_the_same_codes_and_gives_the_same_bits(bits
 def test_two_ctas_sharing_their_expansions_give_the_bits_of_ctas_on_their_own(bits):
     """Chunks whose row pairs come in twos (128, 256, 512, 1024 tokens) run as clusters of two CTAs, each expanding
     half of every code tile for both, at any prefix: the two walk the key tiles of the later row pair, and the
-    earlier one masks what it does not see (the chunks after the 100-token one start off the tile grid).  A batch
-    of one cache never does.  Wherever both cut the key range alike the outputs are the same bits; everywhere they
+    earlier one masks what it does not see (the chunks after the 100-token one start off the tile grid).  A step
+    whose members may take fewer tokens than the chunk (kvf_batch_fold_step_varlen, here a batch of one cache
+    taking all of them) never does.  Wherever both cut the key range alike the outputs are the same bits; everywhere they
     agree within the tolerance, and with the oracle's quantised fold on sampled rows."""
     chunks = [256] * 5 + [100] + [256] * 4 + [512, 1024, 256, 128, 256]
     total = sum(chunks)
@@ -249,7 +250,7 @@ def test_two_ctas_sharing_their_expansions_give_the_bits_of_ctas_on_their_own(bi
         q, k, v = workloads.chunk_inputs(W, 113, t, device="cuda", n_tokens=n)
         prefix = len(alone)
         got = alone.fold_step(q, k, v)
-        want = batch.fold_step(q[None].contiguous(), k[None].contiguous(), v[None].contiguous())[0]
+        want = batch.fold_step_varlen(q[None].contiguous(), k[None].contiguous(), v[None].contiguous(), [n])[0]
         if alone.plan(n, prefix)[1:] == batch.plan(n, prefix)[1:]:
             same_plan += 1
             assert torch.equal(got.view(torch.int16), want.view(torch.int16)), f"step {t}"
