@@ -332,6 +332,88 @@ def run_full_stack(args):
     print(json.dumps(line), flush=True)
 
 
+def run_batch_decode(args):
+    """Sequences decoded together (not the headline line): `--caches` paged caches of one pool, each holding
+    `--prefill` tokens (folded in lock step, 2048 at a time, outside the timed region), then `--steps` timed
+    batch steps of `--chunk` tokens per member (default one), every member with inputs of its own.  The step is
+    bound by the cache read: value = tokens/s over all members, roofline = cache bytes read per second."""
+    from paper_2605_12471_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the fold step has no CPU path")
+    torch.cuda.set_device(0)
+    B, P, n = args.caches, args.prefill or 16384, args.chunk or 1
+    if P % 2048:
+        raise SystemExit("--prefill must be a multiple of 2048")
+    w = workloads.DEEP_CHAIN
+    H, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
+    steps = max(args.steps, 1) * 400                             # a timed stretch of about half a second
+    cap = P + (args.warmup + 1) * steps * n + 128
+    flags = binding.KVF_CACHE_INT8 if args.cache_int8 else binding.KVF_CACHE_INT4 if args.cache_int4 else 0
+    cfg = binding.make_config(H, Hkv, d, "bf16", cap, 2048, rope_base=w.rope_base, flags=flags)
+    per = (cap + 127) // 128
+    n_pool = B * per
+    deck = torch.randperm(n_pool, generator=torch.Generator().manual_seed(args.seed)).to(torch.int32)
+    tables = deck.view(B, per).cuda()
+    pool = torch.zeros(binding.paged_pool_bytes(cfg, n_pool), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(binding.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    caches = [binding.PagedCache(cfg, pool, n_pool, tables[i], workspace=ws) for i in range(B)]
+    batch = binding.Batch(caches)
+    gen = torch.Generator(device="cuda").manual_seed(args.seed)
+
+    def draw(tokens, heads):
+        return torch.randn((B, tokens, heads, d), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+
+    fq, fk, fv = draw(2048, H), draw(2048, Hkv), draw(2048, Hkv)
+    for _ in range(P // 2048):
+        batch.fold_step(fq, fk, fv)
+    del fq, fk, fv
+    q, k, v = draw(n, H), draw(n, Hkv), draw(n, Hkv)
+    out = torch.empty_like(q)
+    lib, bh, stream = binding.load(), batch._h, torch.cuda.current_stream().cuda_stream
+
+    def run(count):
+        for _ in range(count):
+            rc = lib.kvf_batch_fold_step(bh, q.data_ptr(), k.data_ptr(), v.data_ptr(), n, len(caches[0]), out.data_ptr(),
+                                         None, stream)
+            if rc:
+                raise binding.KvfError(rc, "kvf_batch_fold_step")
+
+    for _ in range(max(args.warmup, 1)):
+        run(steps)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    first = len(caches[0])
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    run(steps)
+    b.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = a.elapsed_time(b)
+    assert batch.status_word() == 0 and all(c.status() == binding.KVF_OK for c in caches)
+    row_bytes = 2 * Hkv * ((d + 4) if args.cache_int8 else (d // 2 + 4) if args.cache_int4 else 2 * d)
+    mean_rows = first + (steps * n + n) / 2.0                    # rows a step reads per cache, averaged over the stretch
+    gbs = B * mean_rows * row_bytes * steps / (ms * 1e-3) / 1e9
+    pk = peaks()
+    line = {"metric": "fold-step tokens/s", "value": B * n * steps / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+            "steps": steps, "warmup": max(args.warmup, 1), "ms_per_step": ms / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "batch_decode", "caches": B, "prefix": first, "tokens_per_member": n,
+                       "n_q_heads": H, "n_kv_heads": Hkv, "head_dim": d,
+                       "cache_storage": "int8 codes + fp32 row scales" if args.cache_int8 else
+                                        "int4 codes + fp32 row scales" if args.cache_int4 else "bf16 rows",
+                       "paged": True, "plan": dict(zip(("tensor_core", "splits", "ctas", "kernels"), batch.plan(n))),
+                       "launch": "one batch step per token (one launch of each kernel for all caches)",
+                       "l2": "inputs larger than L2 (%.2f GB of cache rows per step)" % (B * mean_rows * row_bytes / 1e9)},
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": gbs / pk["hbm_gbs"],
+                         "peak_source": "measured copy bandwidth" if pk["_source"] == "measured" else "fallback copy bandwidth", "traffic": None,
+                         "kernel": "whole step (rotate + append, attention, merge)",
+                         "cache_bytes_per_step": B * mean_rows * row_bytes},
+            "cpu_baseline": None, "e2e": None, "gpu_launches": batch.launch_count(), "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -345,12 +427,15 @@ def parse_args():
                          "then runs from this prefix to --tokens (decode- and question-shaped steps at depth)")
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"],
                     help="cache and input dtype (not the benchmark workload)")
-    ap.add_argument("--workload", default="deep_chain", choices=["deep_chain", "llama_16k", "sweep", "full_stack"],
+    ap.add_argument("--workload", default="deep_chain", choices=["deep_chain", "llama_16k", "sweep", "full_stack", "batch_decode"],
                     help="deep_chain: 131 072 tokens in chunks of 256 (the headline line).  llama_16k: 16 384 tokens "
                          "in chunks of 2048, inputs scaled by 1/sqrt(128).  sweep: 65 536 tokens at chunks of 128, "
                          "512, 2048 and 8192, each with a bf16 and an fp32 cache, one line per combination with the "
                          "output drift against the oracle on sampled rows.  full_stack: the 4 x 32-layer "
-                         "memory-scale fold (64 GiB of cache; a separate, longer run)")
+                         "memory-scale fold (64 GiB of cache; a separate, longer run).  batch_decode: --caches paged "
+                         "caches of --prefill tokens each decoding --chunk tokens per batch step (with --cache-int8 / "
+                         "--cache-int4 on quantised pages)")
+    ap.add_argument("--caches", type=int, default=32, help="batch_decode: sequences decoded together")
     ap.add_argument("--sequences", type=int, default=4)
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--seed", type=int, default=2605)
@@ -384,6 +469,9 @@ def main():
     args = parse_args()
     if args.workload == "full_stack" and args.impl == "ours":
         run_full_stack(args)
+        return
+    if args.workload == "batch_decode" and args.impl == "ours":
+        run_batch_decode(args)
         return
     if args.workload == "sweep":
         variants = workloads.SWEEP
