@@ -53,11 +53,14 @@ struct Ctl {
 // NB = 8-row blocks of query rows (1: up to 8 rows, 2: up to 16).  A scheduler of the SM holds 16 K
 // registers: with 13 warps one of them has four (128 registers a thread, enough for one block of
 // rows), with 11 none has more than three (168, what two blocks need without spilling).
+// BITS = 16 stands for a cache of plain bf16 rows: the same kernel without the expansion (a tile is then two
+// 128-byte-swizzled panels of 64 columns, 32 KiB; three stages of 64 KiB, six consumer warps).
 template <int BITS, int NB> struct Geo {
     static constexpr int RB = kD * BITS / 8;                       // bytes of a row of codes
     static constexpr uint32_t kCodes = kKeysPerTile * RB;          // one tile of codes
-    static constexpr uint32_t kStage = 2 * kCodes + 1024;          // K codes, V codes, K scales, V scales
-    static constexpr int kStages = NB == 2 ? 5 : 6;
+    static constexpr uint32_t kScales = BITS == 16 ? 0 : 1024;     // K scales, V scales
+    static constexpr uint32_t kStage = 2 * kCodes + kScales;       // K codes, V codes, scales
+    static constexpr int kStages = BITS == 16 ? 3 : NB == 2 ? 5 : 6;
     static constexpr uint32_t kOffCtl = kStages * kStage;
     static constexpr uint32_t kSmem = kOffCtl + 1024 + 1024;       // + control block + alignment slack
     static constexpr int kWarps = 2 * kStages;                     // consumer warps, two per stage; one more warp produces
@@ -96,6 +99,19 @@ __device__ __forceinline__ void key_fragments(uint32_t tile, int row, int t, flo
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int r = row + 8 * h;
+        if (BITS == 16) {
+            // bf16 rows: two panels of [128 rows][64 columns], 128-byte swizzle; my 32 columns are four 16-byte
+            // chunks (t & 1) * 4 .. + 3 of panel t >> 1, each two k-steps' worth
+            const uint32_t base = tile + (uint32_t)(t >> 1) * (kKeysPerTile * 128u) + (uint32_t)r * 128u, sw = (uint32_t)r & 7u;
+#pragma unroll
+            for (uint32_t c = 0; c < 4; ++c) {
+                uint32_t w[4];
+                lds128(base + (((((uint32_t)t & 1u) << 2) + c) ^ sw) * 16u, w);
+                ka[2 * c][h] = w[0]; ka[2 * c][2 + h] = w[1];
+                ka[2 * c + 1][h] = w[2]; ka[2 * c + 1][2 + h] = w[3];
+            }
+            continue;
+        }
         const float s1 = h ? sc_b : sc_a;
         const float2 sc = make_float2(s1, s1);
         if (BITS == 8) {
@@ -136,12 +152,23 @@ __device__ __forceinline__ uint32_t pair_of_rows(uint32_t wa, uint32_t wb, int b
 // The codes d = 16 g .. 16 g + 15 of key rows row0 + 2 t + {0, 1, 8, 9} of the V code tile, ready
 // for pair_of_rows: int8 as four words of four codes (each byte code + 128), int4 as two words of
 // low nibbles (elements 16 g + 2 i) and two of high nibbles (elements 16 g + 2 i + 1), each code + 8.
+// (bf16 rows: the 16 values themselves, eight words of two.)
 template <int BITS>
-__device__ __forceinline__ void value_codes(uint32_t tile, int row0, int g, int t, uint32_t (&w)[4][4]) {
+__device__ __forceinline__ void value_codes(uint32_t tile, int row0, int g, int t, uint32_t (&w)[4][BITS == 16 ? 8 : 4]) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int r = row0 + 2 * t + (i & 1) + 8 * (i >> 1);
-        if (BITS == 8) {
+        if constexpr (BITS == 16) {
+            // columns 16 g .. 16 g + 15: chunks (g & 3) * 2, + 1 of panel g >> 2
+            const uint32_t base = tile + (uint32_t)(g >> 2) * (kKeysPerTile * 128u) + (uint32_t)r * 128u, sw = (uint32_t)r & 7u;
+#pragma unroll
+            for (uint32_t c = 0; c < 2; ++c) {
+                uint32_t x[4];
+                lds128(base + (((((uint32_t)g & 3u) << 1) + c) ^ sw) * 16u, x);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) w[i][4 * c + k] = x[k];
+            }
+        } else if constexpr (BITS == 8) {
             lds128(tile + (uint32_t)r * 128u + (((uint32_t)g ^ ((uint32_t)r & 7u)) << 4), w[i]);
 #pragma unroll
             for (int k = 0; k < 4; ++k) w[i][k] ^= 0x80808080u;
@@ -155,8 +182,14 @@ __device__ __forceinline__ void value_codes(uint32_t tile, int row0, int g, int 
 }
 // A fragment jp of O^T = V^T P^T: MMA rows g / g + 8 are d = 16 g + 2 jp / + 1, columns the 16 keys.
 template <int BITS>
-__device__ __forceinline__ void value_fragment(const uint32_t (&w)[4][4], int jp, float2 sc01, float2 sc89, uint32_t (&va)[4]) {
-    if (BITS == 8) {
+__device__ __forceinline__ void value_fragment(const uint32_t (&w)[4][BITS == 16 ? 8 : 4], int jp, float2 sc01, float2 sc89, uint32_t (&va)[4]) {
+    if constexpr (BITS == 16) {
+        // word jp of a row holds the row's values at d = 16 g + 2 jp (low half) and + 1 (high half)
+        va[0] = __byte_perm(w[0][jp], w[1][jp], 0x5410);
+        va[1] = __byte_perm(w[0][jp], w[1][jp], 0x7632);
+        va[2] = __byte_perm(w[2][jp], w[3][jp], 0x5410);
+        va[3] = __byte_perm(w[2][jp], w[3][jp], 0x7632);
+    } else if constexpr (BITS == 8) {
         const float2 off = make_float2(-8388736.f, -8388736.f);          // 2^23 + 128
         const int word = jp >> 1, b = 2 * (jp & 1);
         va[0] = pair_of_rows(w[0][word], w[1][word], b, off, sc01);
@@ -259,7 +292,23 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 const int ktile = kt0 + t;
                 const int key0 = ktile * kKeysPerTile;
                 const uint32_t dst = base + (uint32_t)s * Gm::kStage;
-                if (page_table) {
+                if (BITS == 16) {
+                    // bf16 rows: each tile as two panels of 64 columns (rows past the end of a plane are filled with zeros)
+                    constexpr uint32_t kPanel = kKeysPerTile * 128u;
+                    mbar_expect_tx(bar_full + 8 * s, 2 * Gm::kCodes);
+                    if (page_table) {
+                        const int page = page_table[ktile];
+                        tma_load_4d(dst, &map_k, bar_full + 8 * s, 0, 0, kvh, page);
+                        tma_load_4d(dst + kPanel, &map_k, bar_full + 8 * s, 64, 0, kvh, page);
+                        tma_load_4d(dst + Gm::kCodes, &map_v, bar_full + 8 * s, 0, 0, kvh, page);
+                        tma_load_4d(dst + Gm::kCodes + kPanel, &map_v, bar_full + 8 * s, 64, 0, kvh, page);
+                    } else {
+                        tma_load_3d(dst, &map_k, bar_full + 8 * s, 0, key0, kvh);
+                        tma_load_3d(dst + kPanel, &map_k, bar_full + 8 * s, 64, key0, kvh);
+                        tma_load_3d(dst + Gm::kCodes, &map_v, bar_full + 8 * s, 0, key0, kvh);
+                        tma_load_3d(dst + Gm::kCodes + kPanel, &map_v, bar_full + 8 * s, 64, key0, kvh);
+                    }
+                } else if (page_table) {
                     // paged cache: a key tile is one page, which always holds its 128 rows and their scales
                     const int page = page_table[ktile];
                     mbar_expect_tx(bar_full + 8 * s, 2 * Gm::kCodes + 1024u);
@@ -320,6 +369,7 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const uint32_t k_tile = base + (uint32_t)s * Gm::kStage, v_tile = k_tile + Gm::kCodes;
+            // (bf16 rows have no scales: the pointers are then never read)
             const float *k_sc = reinterpret_cast<const float *>(smem + (uint32_t)s * Gm::kStage + 2 * Gm::kCodes);
             const float *v_sc = k_sc + 128;
             const int64_t key_h = (int64_t)(kt0 + t) * kKeysPerTile + half * 64;      // my 64 keys
@@ -332,8 +382,8 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             for (int j = 0; j < 4; ++j) {
                 const int rl = 16 * j + g;                       // my first key row within the 64
                 uint32_t ka[8][4];
-                key_fragments<BITS>(k_tile, half * 64 + rl, t4, rl < in_planes ? k_sc[half * 64 + rl] : 0.f,
-                                    rl + 8 < in_planes ? k_sc[half * 64 + rl + 8] : 0.f, ka);
+                key_fragments<BITS>(k_tile, half * 64 + rl, t4, BITS != 16 && rl < in_planes ? k_sc[half * 64 + rl] : 0.f,
+                                    BITS != 16 && rl + 8 < in_planes ? k_sc[half * 64 + rl + 8] : 0.f, ka);
 #pragma unroll
                 for (int nb = 0; nb < NB; ++nb) {
                     // a second accumulator for the odd k-steps: two chains of four MMAs instead of one of eight
@@ -405,11 +455,11 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             for (int j = 0; j < 4; ++j) {
                 const int r0 = 16 * j + 2 * t4;                  // my first key row within the 64
                 float2 sc01, sc89;
-                sc01.x = r0 < in_planes ? v_sc[half * 64 + r0] : 0.f;
-                sc01.y = r0 + 1 < in_planes ? v_sc[half * 64 + r0 + 1] : 0.f;
-                sc89.x = r0 + 8 < in_planes ? v_sc[half * 64 + r0 + 8] : 0.f;
-                sc89.y = r0 + 9 < in_planes ? v_sc[half * 64 + r0 + 9] : 0.f;
-                uint32_t w[4][4];
+                sc01.x = BITS != 16 && r0 < in_planes ? v_sc[half * 64 + r0] : 0.f;
+                sc01.y = BITS != 16 && r0 + 1 < in_planes ? v_sc[half * 64 + r0 + 1] : 0.f;
+                sc89.x = BITS != 16 && r0 + 8 < in_planes ? v_sc[half * 64 + r0 + 8] : 0.f;
+                sc89.y = BITS != 16 && r0 + 9 < in_planes ? v_sc[half * 64 + r0 + 9] : 0.f;
+                uint32_t w[4][BITS == 16 ? 8 : 4];
                 value_codes<BITS>(v_tile, half * 64 + 16 * j, g, t4, w);
 #pragma unroll
                 for (int jp = 0; jp < 8; ++jp) {
@@ -505,15 +555,19 @@ int attn_q8_decode_max_rows() { return kMaxRows; }
 
 cudaError_t launch_attn_q8_decode(const AttnArgs &a, const TcMaps &maps, cudaStream_t s) {
     static_assert(sizeof(Ctl) <= 1024, "control block");
-    static_assert(Geo<8, 1>::kSmem <= 232448 && Geo<8, 2>::kSmem <= 232448, "shared memory budget of one CTA");
+    static_assert(Geo<8, 1>::kSmem <= 232448 && Geo<8, 2>::kSmem <= 232448 && Geo<16, 1>::kSmem <= 232448, "shared memory budget of one CTA");
     static_assert(Geo<8, 1>::kStages <= 12, "control block holds 12 stages");
-    const bool wide = a.n * a.G > 8, four = a.quant_bits == 4;
-    auto kernel = four ? (wide ? attn_q8_decode_kernel<4, 2> : attn_q8_decode_kernel<4, 1>)
-                       : (wide ? attn_q8_decode_kernel<8, 2> : attn_q8_decode_kernel<8, 1>);
-    const uint32_t smem = four ? (wide ? Geo<4, 2>::kSmem : Geo<4, 1>::kSmem) : (wide ? Geo<8, 2>::kSmem : Geo<8, 1>::kSmem);
+    static_assert(Geo<16, 1>::kWarps * kMergeWarp <= Geo<16, 1>::kOffCtl, "the merge area reuses the ring");
+    const bool wide = a.n * a.G > 8;
+    const int bits = a.quant_bits ? a.quant_bits : 16;              // 16: plain bf16 rows
+    auto kernel = bits == 4 ? (wide ? attn_q8_decode_kernel<4, 2> : attn_q8_decode_kernel<4, 1>)
+                : bits == 8 ? (wide ? attn_q8_decode_kernel<8, 2> : attn_q8_decode_kernel<8, 1>)
+                            : (wide ? attn_q8_decode_kernel<16, 2> : attn_q8_decode_kernel<16, 1>);
+    const uint32_t smem = bits == 4 ? (wide ? Geo<4, 2>::kSmem : Geo<4, 1>::kSmem)
+                        : bits == 8 ? (wide ? Geo<8, 2>::kSmem : Geo<8, 1>::kSmem) : (wide ? Geo<16, 2>::kSmem : Geo<16, 1>::kSmem);
     cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(kernel), (int)smem);
     if (e != cudaSuccess) return e;
-    const int threads = wide ? Geo<8, 2>::kThreads : Geo<8, 1>::kThreads;
+    const int threads = bits == 16 ? Geo<16, 1>::kThreads : wide ? Geo<8, 2>::kThreads : Geo<8, 1>::kThreads;
     return launch_pdl(kernel, dim3(a.ngroups, a.batch), dim3(threads), smem, s, a, maps.k, maps.v);
 }
 

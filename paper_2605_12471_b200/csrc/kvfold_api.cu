@@ -315,7 +315,7 @@ kvf_status build_maps(kvf_cache *c) {
 }
 
 struct Plan {
-    bool qdec;     // quantised cache, a few query rows: the decode kernel that expands codes in registers
+    bool qdec;     // a few query rows on a bf16 or quantised cache: the decode kernel that feeds MMAs from registers
     bool tc;
     int splits;    // CUDA-core path: splits of the key range; tensor-core path: ranges per KV head (rounded up)
     int ngroups;   // tensor-core path: ranges of the (KV head, key tile) line
@@ -339,7 +339,7 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
     p.ngroups = 0;
     const int64_t L = prefix + n;
     const int Hkv = c->cfg.n_kv_heads;
-    if (c->quant && c->window <= 0 && n * c->G <= attn_q8_decode_max_rows()) {
+    if ((c->quant || c->tc) && c->window <= 0 && n * c->G <= attn_q8_decode_max_rows()) {
         // one CTA per SM (all caches of a batch together), each inside one KV head (a multiple of the KV heads),
         // at least two key tiles each; a forced split count is the number of ranges per KV head
         const int64_t nt = (L + kKvTile - 1) / kKvTile;
