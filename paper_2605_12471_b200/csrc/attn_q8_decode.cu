@@ -1,5 +1,6 @@
-// Decode-shaped steps on a quantised cache: at most 16 query rows (n_tokens * G <= 16, i.e. one to
-// four tokens at the Llama group size) against a long prefix stored as int8 or int4 codes.
+// Decode-shaped steps: at most 16 query rows (n_tokens * G <= 16, i.e. one to four tokens at the
+// Llama group size) against a long prefix stored as int8 or int4 codes - or as plain bf16 rows, which
+// take the same kernel without the expansion (BITS = 16 below).
 //
 // Section 2 of the paper: the chunk's queries attend to every row of the earlier chunks and,
 // causally, to the chunk itself; query head h reads KV head h / G.  The trials of Section 4 end
