@@ -243,6 +243,23 @@ int64_t kvf_cache_len(const kvf_cache *c);
  * Section 2, "Three reference conditions").  len = 0; storage is not cleared. */
 kvf_status kvf_cache_reset(kvf_cache *c);
 
+/* Sets the number of rows the accumulator holds, 0 <= len <= capacity (else KVF_ERR_CAPACITY);
+ * host counter only, nothing is enqueued and no row is touched.
+ * Section 2 states that the cache IS the whole state of the fold, so a fold can be taken back to
+ * an earlier accumulator (K,V)^(t') by forgetting the rows behind it.  The paper's multi-needle
+ * protocol ("Multi-needle retrieval", in the section on scaling) asks K questions about ONE folded
+ * haystack, each queried separately: fold the haystack once, then per key a question chunk and the
+ * decoded tokens, then kvf_cache_set_len(c, haystack_len) - instead of folding 128 K tokens K times.
+ * len <= kvf_cache_len: rows [len, old len) are forgotten; the next step appends at row len (and
+ *   rotates at the pos0 the caller passes).  Steps enqueued before the call are not affected.
+ * len >  kvf_cache_len: resuming from restored storage.  The caller vouches that the planes hold what a
+ *   cache of at least len rows held (a byte copy of the storage of a live cache, taken when its
+ *   length was >= len, is that); rows the library never wrote may hold non-finite bits, which a
+ *   masked key tile would turn into NaN outputs.
+ * With KVF_COMBINE_BEHIND / KVF_HOST_DOWNLOAD_BEHIND the results of the last step are still on their
+ * way as after any step; this call does not wait for them. */
+kvf_status kvf_cache_set_len(kvf_cache *c, int64_t len);
+
 /* Reads the device status word (synchronises the default stream with a blocking copy): KVF_OK,
  * KVF_ERR_TIMEOUT if a bounded wait inside a kernel gave up, or KVF_ERR_RANGE (see kvf_status).  Call after synchronising the
  * streams that carried the steps.  (The paper has no counterpart: this reports on the kernels'

@@ -22,7 +22,7 @@ KVF_HOST_UPLOAD_AHEAD, KVF_CACHE_INT4, KVF_HOST_DOWNLOAD_BEHIND, KVF_COMBINE_BEH
 
 EXPORTS = [
     "kvf_cache_storage_bytes", "kvf_workspace_bytes", "kvf_cache_create", "kvf_fold_step",
-    "kvf_fold_step_host", "kvf_cache_len", "kvf_cache_reset", "kvf_cache_status",
+    "kvf_fold_step_host", "kvf_cache_len", "kvf_cache_reset", "kvf_cache_set_len", "kvf_cache_status",
     "kvf_cache_k_plane", "kvf_cache_v_plane", "kvf_cache_plan", "kvf_cache_set_splits",
     "kvf_cache_launch_count", "kvf_cache_profile", "kvf_cache_profile_read", "kvf_cache_destroy",
     "kvf_status_str", "kvf_last_cuda_error", "kvf_fold_step_static", "kvf_cache_status_word",
@@ -91,6 +91,8 @@ def load() -> ctypes.CDLL:
     lib.kvf_cache_len.restype = i64
     lib.kvf_cache_reset.argtypes = [vp]
     lib.kvf_cache_reset.restype = ctypes.c_int
+    lib.kvf_cache_set_len.argtypes = [vp, i64]
+    lib.kvf_cache_set_len.restype = ctypes.c_int
     lib.kvf_cache_status.argtypes = [vp]
     lib.kvf_cache_status.restype = ctypes.c_int
     lib.kvf_cache_status_word.argtypes = [vp]
@@ -212,6 +214,12 @@ class Cache:
         rc = load().kvf_cache_reset(self._h)
         if rc != KVF_OK:
             raise KvfError(rc, "kvf_cache_reset")
+
+    def set_len(self, n: int):
+        """kvf_cache_set_len: forget the rows behind row n (or resume from restored storage)."""
+        rc = load().kvf_cache_set_len(self._h, int(n))
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_cache_set_len")
 
     def fold_step(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
                   pos0: Optional[int] = None, out: Optional[torch.Tensor] = None,

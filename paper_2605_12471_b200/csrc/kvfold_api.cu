@@ -929,6 +929,13 @@ kvf_status kvf_cache_reset(kvf_cache *c) {
     return KVF_OK;
 }
 
+kvf_status kvf_cache_set_len(kvf_cache *c, int64_t len) {
+    if (!c) return KVF_ERR_INVALID_ARG;
+    if (len < 0 || len > c->cfg.capacity) return KVF_ERR_CAPACITY;
+    c->len = len;
+    return KVF_OK;
+}
+
 kvf_status kvf_cache_status(kvf_cache *c) {
     if (!c) return KVF_ERR_INVALID_ARG;
     int word = 0;

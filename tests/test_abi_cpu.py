@@ -105,6 +105,7 @@ def test_null_handles_are_harmless(binding):
     lib = binding.load()
     assert lib.kvf_cache_len(None) == -1
     assert lib.kvf_cache_reset(None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_cache_set_len(None, 0) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_fold_step(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_fold_step_host(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_cache_launch_count(None) == 0
