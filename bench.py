@@ -414,6 +414,92 @@ def run_batch_decode(args):
     print(json.dumps(line), flush=True)
 
 
+def run_multi_needle(args):
+    """Several questions about one folded haystack (not the headline line).  The paper's multi-needle protocol
+    queries K keys separately on the same context: the haystack (`--prefill` tokens, default 129 024) is folded
+    ONCE, outside the timed region; the timed region is `--needles` questions, each a question chunk of `--chunk`
+    tokens (default 32) and 30 tokens decoded one at a time, after which kvf_cache_set_len takes the cache back to
+    the haystack.  Every step is bound by the cache read; value = tokens folded per second in the timed region."""
+    from paper_2605_12471_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the fold step has no CPU path")
+    torch.cuda.set_device(0)
+    w = workloads.DEEP_CHAIN
+    H, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
+    P, nq, ndec, K = args.prefill or 129024, args.chunk or 32, 30, args.needles
+    if P % 2048:
+        raise SystemExit("--prefill must be a multiple of 2048")
+    flags = binding.KVF_CACHE_INT8 if args.cache_int8 else binding.KVF_CACHE_INT4 if args.cache_int4 else 0
+    cfg = binding.make_config(H, Hkv, d, "bf16", P + nq + ndec, 2048, rope_base=w.rope_base, flags=flags)
+    cache = binding.Cache(cfg)
+    gen = torch.Generator(device="cuda").manual_seed(args.seed)
+
+    def draw(tokens, heads):
+        return torch.randn((tokens, heads, d), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+
+    fq, fk, fv = draw(2048, H), draw(2048, Hkv), draw(2048, Hkv)
+    fout = torch.empty_like(fq)
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0.record()
+    for _ in range(P // 2048):
+        cache.fold_step(fq, fk, fv, out=fout)
+    h1.record()
+    torch.cuda.synchronize()
+    haystack_ms = h0.elapsed_time(h1)
+    del fq, fk, fv, fout
+    qs = [(draw(nq, H), draw(nq, Hkv), draw(nq, Hkv)) for _ in range(K)]
+    dq, dk, dv = draw(1, H), draw(1, Hkv), draw(1, Hkv)
+    out_q, out_d = torch.empty((nq, H, d), dtype=torch.bfloat16, device="cuda"), torch.empty((1, H, d), dtype=torch.bfloat16, device="cuda")
+
+    def questions():
+        for q, k, v in qs:
+            cache.fold_step(q, k, v, out=out_q)
+            for _ in range(ndec):
+                cache.fold_step(dq, dk, dv, out=out_d)
+            cache.set_len(P)
+
+    for _ in range(max(args.warmup, 3)):
+        questions()
+    torch.cuda.synchronize()
+    launches0 = cache.launch_count()
+    sampler = ClockSampler(0)
+    sampler.start()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    reps = max(args.steps, 1) * 4                                    # a timed stretch of about half a second
+    for _ in range(reps):
+        questions()
+    b.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = a.elapsed_time(b) / reps
+    assert cache.status() == binding.KVF_OK, hex(cache.status_word())
+    row_bytes = 2 * Hkv * ((d + 4) if args.cache_int8 else (d // 2 + 4) if args.cache_int4 else 2 * d)
+    rows = (P + nq) + sum(P + nq + i + 1 for i in range(ndec))       # cache rows the steps of one question read
+    gbs = K * rows * row_bytes / (ms * 1e-3) / 1e9
+    pk = peaks()
+    line = {"metric": "fold-step tokens/s", "value": K * (nq + ndec) / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+            "steps": reps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "multi_needle", "haystack_tokens": P, "questions_per_step": K, "question_tokens": nq,
+                       "decoded_tokens": ndec, "n_q_heads": H, "n_kv_heads": Hkv, "head_dim": d,
+                       "cache_storage": "int8 codes + fp32 row scales" if args.cache_int8 else
+                                        "int4 codes + fp32 row scales" if args.cache_int4 else "bf16 rows",
+                       "launch": "one kvf_fold_step per question chunk and per decoded token, kvf_cache_set_len back to "
+                                 "the haystack after every question",
+                       "l2": "inputs larger than L2 (%.0f MB of cache rows per step)" % (P * row_bytes / 1e6)},
+            "ms_per_question": ms / K,
+            "haystack_fold_ms": haystack_ms,
+            "haystack_fold_note": "the haystack folded once in chunks of 2048, outside the timed region: what every "
+                                  "further question would cost again without kvf_cache_set_len",
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": gbs / pk["hbm_gbs"],
+                         "peak_source": "measured copy bandwidth" if pk["_source"] == "measured" else "fallback copy bandwidth",
+                         "traffic": None, "kernel": "whole steps (rotate + append, attention, merge)",
+                         "cache_bytes_per_question": rows * row_bytes},
+            "cpu_baseline": None, "e2e": None, "gpu_launches": cache.launch_count() - launches0, "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -427,7 +513,7 @@ def parse_args():
                          "then runs from this prefix to --tokens (decode- and question-shaped steps at depth)")
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"],
                     help="cache and input dtype (not the benchmark workload)")
-    ap.add_argument("--workload", default="deep_chain", choices=["deep_chain", "llama_16k", "sweep", "full_stack", "batch_decode"],
+    ap.add_argument("--workload", default="deep_chain", choices=["deep_chain", "llama_16k", "sweep", "full_stack", "batch_decode", "multi_needle"],
                     help="deep_chain: 131 072 tokens in chunks of 256 (the headline line).  llama_16k: 16 384 tokens "
                          "in chunks of 2048, inputs scaled by 1/sqrt(128).  sweep: 65 536 tokens at chunks of 128, "
                          "512, 2048 and 8192, each with a bf16 and an fp32 cache, one line per combination with the "
@@ -436,6 +522,9 @@ def parse_args():
                          "caches of --prefill tokens each decoding --chunk tokens per batch step (with --cache-int8 / "
                          "--cache-int4 on quantised pages)")
     ap.add_argument("--caches", type=int, default=32, help="batch_decode: sequences decoded together")
+    ap.add_argument("--needles", type=int, default=8,
+                    help="multi_needle: questions asked one after the other about one folded haystack (--prefill tokens), "
+                         "each a chunk of --chunk tokens and 30 decoded tokens, with kvf_cache_set_len back in between")
     ap.add_argument("--sequences", type=int, default=4)
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--seed", type=int, default=2605)
@@ -472,6 +561,9 @@ def main():
         return
     if args.workload == "batch_decode" and args.impl == "ours":
         run_batch_decode(args)
+        return
+    if args.workload == "multi_needle" and args.impl == "ours":
+        run_multi_needle(args)
         return
     if args.workload == "sweep":
         variants = workloads.SWEEP
