@@ -406,6 +406,21 @@ def test_attention_kernels_report_the_clock_they_ran_at():
 
 
 # ------------------------------------------------------------------ short chunks at depth
+@pytest.mark.parametrize("splits", [0, 1], ids=["merged_ranges", "one_range_per_head"])
+def test_decode_shaped_steps_with_fp32_output(splits):
+    """One to four tokens per step take the decode kernel; with one key range per KV head it writes the outputs
+    and log-sum-exps itself (no merge), otherwise the merge kernel does: both in fp32 under KVF_OUT_F32."""
+    w = SMALL_LLAMA.with_(name="decode_out_f32", tokens=4096)
+    chunks = [2048, 300, 1, 1, 2, 3, 4, 1]
+    res, cache, _, outs = run_chain(w, chunks, seed=23, flags=binding.KVF_OUT_F32, splits=splits,
+                                    check_steps=list(range(2, len(chunks))), keep_outputs=True)
+    assert outs[-1].dtype == torch.float32
+    if splits:
+        assert cache.plan(1)[1] == 1
+    assert_within(res, "bf16", "decode, fp32 output")
+    assert res.lse_max_abs <= 2e-2, res.lse_max_abs
+
+
 def test_short_chunks_deep_in_a_chain_match_the_oracle():
     """Decode- and question-shaped steps (1 .. 32 tokens: at most one 128-row tile) after a long
     prefix: the kernel deals their key tiles to two streams and always merges partial results."""
