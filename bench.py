@@ -521,6 +521,10 @@ def parse_args():
                          "memory-scale fold (64 GiB of cache; a separate, longer run).  batch_decode: --caches paged "
                          "caches of --prefill tokens each decoding --chunk tokens per batch step (with --cache-int8 / "
                          "--cache-int4 on quantised pages)")
+    ap.add_argument("--q-heads", type=int, default=0,
+                    help="query heads of the layer (with --kv-heads: another model's attention shape, e.g. 28 / 4 for "
+                         "Qwen2.5-7B; not the benchmark workload)")
+    ap.add_argument("--kv-heads", type=int, default=0)
     ap.add_argument("--caches", type=int, default=32, help="batch_decode: sequences decoded together")
     ap.add_argument("--needles", type=int, default=8,
                     help="multi_needle: questions asked one after the other about one folded haystack (--prefill tokens), "
@@ -575,6 +579,9 @@ def main():
         if args.tokens or args.chunk or args.prefill or (args.dtype != w.dtype and args.workload != "sweep"):
             w = w.with_(name=f"chain_{args.tokens or w.tokens}_c{args.chunk or w.chunk}_from_{args.prefill}_{args.dtype}",
                         tokens=args.tokens or w.tokens, chunk=args.chunk or w.chunk, dtype=args.dtype)
+        if args.q_heads or args.kv_heads:
+            w = w.with_(name=f"{w.name}_heads_{args.q_heads or w.n_q_heads}_{args.kv_heads or w.n_kv_heads}",
+                        n_q_heads=args.q_heads or w.n_q_heads, n_kv_heads=args.kv_heads or w.n_kv_heads)
         if args.impl == "reference":
             run_reference(args, w)
         else:

@@ -113,7 +113,11 @@ enum {
 /*
  * Shape and numerics of one cache.
  *   n_q_heads (H), n_kv_heads (Hkv): grouped-query attention, query head h reads KV head
- *       h / (H/Hkv); H % Hkv == 0 and H/Hkv a power of two <= 64.
+ *       h / (H/Hkv); H % Hkv == 0 and H/Hkv <= 64 (the models of the paper's experiments have
+ *       groups of 4 (Llama-3.1-8B: 32/8), 7 (Qwen2.5-7B: 28/4), 6 (Qwen2.5-1.5B: 12/2) and 1
+ *       (OLMoE: 16/16)).  The tensor-core kernels lay a group that is no power of two out as
+ *       the next power of two, so 1/8 (groups of 7) or 1/4 (groups of 6) of their tensor-core
+ *       work is spent on padding rows.
  *   head_dim (d): 64 or 128.
  *   dtype: element type of q, k_new, v_new, of the cache planes and (unless KVF_OUT_F32) of out.
  *       KVF_BF16: rotation, scores, softmax state and the output sum are fp32, probabilities

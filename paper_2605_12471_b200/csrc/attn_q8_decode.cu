@@ -231,7 +231,9 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     if (n <= 0) return;                                   // a member that sits the step out
     const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix, L = P + n;
     const bool direct = a.ngroups == a.Hkv;
-    const int64_t slot_rows = (int64_t)nmax * G;          // rows of a partial slot
+    // rows of a partial slot; the slots keep the row layout of the tensor-core kernels, row = token * Gp +
+    // head-in-group with Gp = G rounded up to a power of two, because the same merge kernel reads both
+    const int64_t slot_rows = (int64_t)nmax * a.Gp;
 
     // this CTA's range of its KV head's key tiles (the same line arithmetic as the other kernels)
     const int nt_all = (int)((L + kKeysPerTile - 1) / kKeysPerTile);
@@ -247,7 +249,7 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         if (!direct && kvh < a.Hkv)
             for (int item = threadIdx.x; item < nG * (kD / 4); item += blockDim.x) {
                 const int r = item / (kD / 4), c4 = item % (kD / 4);
-                const int64_t prow = (int64_t)cb * a.part_rows + (int64_t)(group + kvh) * slot_rows + r;
+                const int64_t prow = (int64_t)cb * a.part_rows + (int64_t)(group + kvh) * slot_rows + (r / G) * a.Gp + r % G;
                 reinterpret_cast<float4 *>(a.part_o + prow * kD)[c4] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (c4 == 0) a.part_lse[prow] = -INFINITY;
             }
@@ -528,7 +530,7 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             const int tok = r / G, gi = r % G;
             const int64_t row = ((int64_t)cb * nmax + tok) * a.H + kvh * G + gi;
             if (!direct) {
-                const int64_t prow = (int64_t)cb * a.part_rows + (int64_t)(group + kvh) * slot_rows + r;
+                const int64_t prow = (int64_t)cb * a.part_rows + (int64_t)(group + kvh) * slot_rows + (r / G) * a.Gp + r % G;
                 float4 *dst = reinterpret_cast<float4 *>(a.part_o + prow * kD + c0);
                 dst[0] = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
                 dst[1] = make_float4(acc[4] * inv, acc[5] * inv, acc[6] * inv, acc[7] * inv);

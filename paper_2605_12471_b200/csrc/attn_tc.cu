@@ -7,7 +7,9 @@
 // memory in fp32.
 //
 // Work decomposition.  A row pair is 256 query rows of one KV head (row = token * G +
-// head-in-group, so the G query heads that share a KV head share every K/V tile), handled as two
+// head-in-group, so the G query heads that share a KV head share every K/V tile; a group size that
+// is no power of two - the 28 / 4 heads of Qwen2.5-7B - is laid out with G rounded up, the padding
+// rows computed and never written), handled as two
 // 128-row tiles that take turns on the tensor pipe.  Keys come in 128-row tiles.  The (KV head,
 // key tile) pairs of a step are laid out on one line and cut into `ngroups` equal contiguous
 // ranges; CTA (x = row pair, y = group) runs its row pair against its group's range, which
@@ -159,7 +161,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     const int qpair = blockIdx.x, group = blockIdx.y;
     const uint32_t rank = kPair ? cluster_cta_rank() : 0u;     // which of K (0) and V (1) this CTA expands
     const int cb = blockIdx.z;     // cache of a batch (0 when there is one cache)
-    const int G = a.G;
+    const int G = a.Gp;     // rows per token in the row layout (a power of two >= a.G, the query heads per KV head)
     // (a ragged batch keeps its members' row counts in device memory, written by an earlier kernel
     // of the stream: those are the one thing read before the set-up below, so wait first there)
     if (a.prefixes) pdl_wait();
@@ -359,7 +361,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
                 mbar_expect_tx(bar(B_QFULL), (streams == 2 ? 1 : 2) * kTileBytes);
                 for (int i = 0; i < (streams == 2 ? 1 : 2); ++i)
                     for (int p = 0; p < 2; ++p)
-                        tma_load_3d(base + kOffQ + i * kTileBytes + p * kPanel, &map_q, bar(B_QFULL), p * 64, kvh * G,
+                        tma_load_3d(base + kOffQ + i * kTileBytes + p * kPanel, &map_q, bar(B_QFULL), p * 64, kvh * a.G,
                                     qtok0 + (row0 + i * kRows) / G);
                 ++pc;
                 for (int t = 0; t < 2 * ntiles; ++t, ++tg) {
@@ -533,7 +535,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         const uint32_t t_s = tmem + lane_addr + i * 128;
         const uint32_t t_o = tmem + lane_addr + 256 + i * 128;
         const int R = row0 + (streams == 2 ? 0 : i * kRows) + r, tok = R / G, gi = R % G;
-        const bool valid = tok < n;
+        const bool valid = tok < n && gi < a.G;     // (gi >= a.G: padding of a group that is no power of two)
         // a warp none of whose 32 rows is a row of the chunk (decode-shaped steps: most warps) keeps
         // every barrier protocol going but skips the loads, the arithmetic and the stores
         const bool warp_live = __any_sync(0xffffffffu, valid);
@@ -704,7 +706,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
             if (!warp_live) continue;
             const float inv = l > 0.f ? 1.f / l : 0.f;
             const float lse2 = l > 0.f ? m_ref * sl2 + log2f(l) : -INFINITY;
-            const int64_t row = ((int64_t)cb * nmax + tok) * a.H + kvh * G + gi;
+            const int64_t row = ((int64_t)cb * nmax + tok) * a.H + kvh * a.G + gi;
 #pragma unroll
             for (int c0 = 0; c0 < 128; c0 += 32) {
                 uint32_t o[32];
@@ -770,7 +772,7 @@ constexpr int kCombineTokens = 4;
 template <bool kFew>   // kFew: every KV head has at most eight parts (known on the host), the loops below run once
 __global__ void __launch_bounds__(256, kFew ? 4 : 2) combine_groups_kernel(const __grid_constant__ AttnArgs a) {
     __shared__ int g_range[2];
-    const int kvh = blockIdx.y, G = a.G;
+    const int kvh = blockIdx.y, G = a.G;     // (a.Gp >= G: rows a token takes in the slots)
     const int cb = blockIdx.z;     // cache of a batch
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
@@ -798,15 +800,18 @@ __global__ void __launch_bounds__(256, kFew ? 4 : 2) combine_groups_kernel(const
     const int st = a.streams;
     const int np = (g1 - g0 + 1) * st;   // parts of this KV head: st per piece
     // part s of the KV head sits in slot (g0 + s / st + kvh) * st + s % st = (g0 + kvh) * st + s
-    const int64_t nG = (int64_t)a.n * G;
+    const int64_t nG = (int64_t)a.n * a.Gp;
     const int64_t slot0 = (int64_t)(g0 + kvh) * st;
     const float *part_o = a.part_o + (cb * a.part_rows + slot0 * nG) * kD + lane * 4;
     const float *part_lse = a.part_lse + cb * a.part_rows + slot0 * nG;
-    const int rows = kCombineTokens * G;                      // rows of this block, row = token * G + head-in-group
+    const int Gp = a.Gp;                                      // rows a token takes in the slots (>= G: the rest is padding)
+    const int rows = kCombineTokens * Gp;                     // rows of this block, row = token * Gp + head-in-group
+    const int lgp = __ffs(Gp) - 1;
     for (int rr = warp; rr < rows; rr += 8) {
-        const int tok = blockIdx.x * kCombineTokens + rr / G, gi = rr % G;
+        const int tok = blockIdx.x * kCombineTokens + (rr >> lgp), gi = rr & (Gp - 1);     // (Gp is a power of two)
         if (tok >= n) break;
-        const int64_t R = (int64_t)tok * G + gi;
+        if (gi >= G) continue;
+        const int64_t R = (int64_t)tok * Gp + gi;
         const int64_t row = ((int64_t)cb * a.n + tok) * a.H + kvh * G + gi;
         const float *po = part_o + R * kD;                    // part s: po + s * nG * kD
         const float *pl = part_lse + R;                       //         pl + s * nG
@@ -859,8 +864,17 @@ __global__ void __launch_bounds__(256, kFew ? 4 : 2) combine_groups_kernel(const
 
 }  // namespace
 
+// Any group size up to 64: the kernels lay rows out with the group rounded up to a power of two
+// (attn_tc_padded_group), so that a 128-row tile holds whole tokens; the rows of the padding cost
+// tensor-core work (1/8 of it for the 28 / 4 heads of Qwen2.5-7B) and are never written.
 bool attn_tc_supported(int dtype, int d, int G) {
-    return dtype == 0 && d == kD && G >= 1 && G <= 64 && (G & (G - 1)) == 0;
+    return dtype == 0 && d == kD && G >= 1 && G <= 64;
+}
+
+int attn_tc_padded_group(int G) {
+    int p = 1;
+    while (p < G) p *= 2;
+    return p;
 }
 
 int attn_tc_row_pairs(int n, int G) { return (n * G + 2 * kRows - 1) / (2 * kRows); }
@@ -872,7 +886,7 @@ int attn_tc_streams(int n, int G) { return n * G <= kRows ? 2 : 1; }
 static bool pair_launch_ok(const AttnArgs &a) {
     // (members of a batch that take fewer tokens than the launch's chunk may lack a row tile: no pairs then)
     if (!a.quant_bits || a.win_lo > 0 || a.streams != 1 || a.ns) return false;
-    return ((int64_t)a.n * a.G) % (4 * kRows) == 0;
+    return ((int64_t)a.n * a.Gp) % (4 * kRows) == 0;
 }
 
 // Do the clusters of two fill the device as single CTAs do (queried once per device)?
@@ -910,7 +924,7 @@ cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s
                 : a.quant_bits == 4 ? (a.win_lo > 0 ? attn_tc_kernel<true, 4> : attn_tc_kernel<false, 4>)
                                     : (a.win_lo > 0 ? attn_tc_kernel<true, 0> : attn_tc_kernel<false, 0>);
     const uint32_t smem = quant ? kSmemBytesQ8 : kSmemBytes;
-    dim3 grid(attn_tc_row_pairs(a.n, a.G), a.ngroups, a.batch);
+    dim3 grid(attn_tc_row_pairs(a.n, a.Gp), a.ngroups, a.batch);
     if (pair_launch_ok(a)) {
         auto paired = a.quant_bits == 8 ? attn_tc_kernel<false, 8, true> : attn_tc_kernel<false, 4, true>;
         cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(paired), (int)smem);

@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rblock = blockIdx.x, group = blockIdx.y;
     const uint32_t rank = kPair ? cluster_cta_rank() : 0u;
-    const int G = a.G, n = a.n;
+    const int G = a.Gp, Gq = a.G, n = a.n;      // rows per token in the row layout (a power of two), query heads per KV head
     const int64_t P = a.prefix, L = P + n;
     const bool direct = a.ngroups == a.Hkv;
     const int row0 = rblock * kRows;
@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
                 for (int i = 0; i < 16; ++i) {
                     const int R = row0 + w8 * 16 + i, tok = R / G, gi = R % G;
                     x[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (tok < n) x[i] = *reinterpret_cast<const float4 *>(q_rot + ((int64_t)tok * a.H + kvh * G + gi) * kD + lane * 4);
+                    if (tok < n && gi < Gq) x[i] = *reinterpret_cast<const float4 *>(q_rot + ((int64_t)tok * a.H + kvh * Gq + gi) * kD + lane * 4);
                 }
                 if (pc > 0) ok = mbar_wait(bar(B_QEMPTY), (pc - 1) & 1, ctl, a.status);
                 ok = __all_sync(0xffffffffu, ok);
@@ -401,7 +401,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
         const int r = warp * 32 + lane;                  // row of the CTA = TMEM lane
         const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
         const int R = row0 + r, tok = R / G, gi = R % G;
-        const bool valid = tok < n;
+        const bool valid = tok < n && gi < Gq;       // (gi >= Gq: padding of a group that is no power of two)
         // keys below `limit` are visible; a row past the chunk's end is never written, and each
         // row of S, P and O depends on that row alone, so such rows are left unmasked
         const int64_t limit = valid ? P + tok + 1 : ((int64_t)1 << 62);
@@ -560,7 +560,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
             const float inv = l > 0.f ? 1.f / l : 0.f;
             const float lse2 = l > 0.f ? m_ref * sl2 + log2f(l) : -INFINITY;
             if (valid) {
-                const int64_t row = (int64_t)tok * a.H + kvh * G + gi;
+                const int64_t row = (int64_t)tok * a.H + kvh * Gq + gi;
                 float4 *dst = direct ? reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.out) + row * kD)
                                      : reinterpret_cast<float4 *>(a.part_o + prow * kD);
 #pragma unroll
@@ -586,7 +586,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
 }  // namespace
 
 bool attn_tc32_supported(int dtype, int d, int G) {
-    return dtype == 1 && d == kD && G >= 1 && G <= 64 && (G & (G - 1)) == 0;
+    return dtype == 1 && d == kD && G >= 1 && G <= 64;     // (any group size: rows are laid out with the padded group)
 }
 
 int attn_tc32_row_blocks(int n, int G) { return (n * G + kRows - 1) / kRows; }
@@ -594,7 +594,7 @@ int attn_tc32_row_blocks(int n, int G) { return (n * G + kRows - 1) / kRows; }
 // Can the row blocks 2k and 2k + 1 of this launch share their conversions (paired variant)?  The row blocks
 // must come in twos (the two of a cluster then take the steps of the later one).
 static bool pair_launch_ok32(const AttnArgs &a) {
-    return a.win_lo <= 0 && ((int64_t)a.n * a.G) % (2 * kRows) == 0;
+    return a.win_lo <= 0 && ((int64_t)a.n * a.Gp) % (2 * kRows) == 0;
 }
 
 // Do the clusters of two fill the device as single CTAs do (queried once per device)?
@@ -626,7 +626,7 @@ static bool pair_clusters_fit32(const void *kernel) {
 cudaError_t launch_attn_tc32(const AttnArgs &a, cudaStream_t s) {
     static_assert(sizeof(Ctl) <= 512, "control block");
     static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
-    dim3 grid(attn_tc32_row_blocks(a.n, a.G), a.ngroups, 1);
+    dim3 grid(attn_tc32_row_blocks(a.n, a.Gp), a.ngroups, 1);
     if (pair_launch_ok32(a)) {
         auto paired = attn_tc32_kernel<false, true>;
         cudaError_t e = raise_smem_limit_once(reinterpret_cast<const void *>(paired), (int)kSmemBytes);

@@ -37,7 +37,7 @@ kvf_status check_config(const kvf_config *c) {
     if (c->dtype != KVF_BF16 && c->dtype != KVF_F32) return KVF_ERR_UNSUPPORTED;
     if (c->head_dim != 64 && c->head_dim != 128) return KVF_ERR_UNSUPPORTED;
     int G = c->n_q_heads / c->n_kv_heads;
-    if (!pow2(G) || G > 64) return KVF_ERR_UNSUPPORTED;
+    if (G > 64) return KVF_ERR_UNSUPPORTED;
     if (c->rope_base <= 0.0 && !c->inv_freq) return KVF_ERR_INVALID_ARG;
     if (c->softmax_scale < 0.0) return KVF_ERR_INVALID_ARG;
     if ((int64_t)c->max_chunk > c->capacity) return KVF_ERR_INVALID_ARG;
@@ -110,7 +110,8 @@ struct kvf_cache {
     size_t plane_bytes;
     Layout lay;
     int64_t len;
-    int G;
+    int G;                   // query heads per KV head
+    int Gp;                  // rows a token takes in the tcgen05 kernels' row layout: G rounded up to a power of two
     float scale_log2;
     bool tc;                 // bf16, head_dim 128: the tcgen05 kernel fed by TMA
     bool tc32;               // fp32, head_dim 128: the tcgen05 kernel on fp16 halves of the operands
@@ -253,10 +254,11 @@ kvf_status build_maps(kvf_cache *c) {
     const kvf_config &f = c->cfg;
     const int d = f.head_dim;
     const uint64_t row = (uint64_t)d * 2;
-    // rotated queries [max_chunk][H][d]: one box = (128/G tokens) x (G heads of one KV head) x 64
+    // rotated queries [max_chunk][H][d]: one box = (128/Gp tokens) x (Gp heads from the first of one KV head on) x 64
+    // (Gp > G: the box runs into the next KV head's queries, or past the last head, where it reads zeros - padding rows)
     kvf_status s = make_map(fn, &c->maps.q, c->workspace + c->lay.q_rot, (uint64_t)f.n_q_heads,
-                            (uint64_t)f.max_chunk, row, row * f.n_q_heads, d, (uint32_t)c->G,
-                            (uint32_t)(128 / c->G));
+                            (uint64_t)f.max_chunk, row, row * f.n_q_heads, d, (uint32_t)c->Gp,
+                            (uint32_t)(128 / c->Gp));
     if (s != KVF_OK) return s;
     if (c->page_table && c->quant) {
         // pages of codes: (row bytes, row in page, KV head, page), the K and the V block of a page apart
@@ -346,7 +348,7 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
         int64_t per_head = c->force_splits > 0 ? c->force_splits : c->sm_count / (Hkv * batch);
         if (c->force_splits <= 0 && per_head > nt / 2) per_head = nt / 2;
         if (per_head > nt) per_head = nt;
-        const int64_t slots_cap = part_rows_cap / ((int64_t)n * c->G);            // slots = groups + Hkv - 1
+        const int64_t slots_cap = part_rows_cap / ((int64_t)n * c->Gp);           // slots = groups + Hkv - 1
         if (per_head * Hkv + Hkv - 1 > slots_cap) per_head = (slots_cap - (Hkv - 1)) / Hkv;
         if (per_head < 1) per_head = 1;
         p.qdec = true;
@@ -362,7 +364,7 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
         // one CTA per SM, with at least 4 key tiles each and within the partial area.
         const int64_t nt = (L + kKvTile - 1) / kKvTile - WindowTiles(window_lo(c, prefix), c->n_sink, kKvTile).skip;
         // (row blocks of a KV head: 256-row pairs in the bf16 kernel, 128-row blocks in the fp32 one)
-        const int pairs = c->tc32 ? attn_tc32_row_blocks(n, c->G) : attn_tc_row_pairs(n, c->G);
+        const int pairs = c->tc32 ? attn_tc32_row_blocks(n, c->Gp) : attn_tc_row_pairs(n, c->Gp);
         int64_t groups = Hkv;
         if (c->force_splits > 0) {
             groups = (int64_t)Hkv * c->force_splits;
@@ -391,8 +393,8 @@ Plan make_plan(const kvf_cache *c, int n, int64_t prefix, int batch = 1, int64_t
             for (int64_t g = Hkv + 1; g <= 2 * Hkv && g * 4 <= Hkv * nt; ++g)
                 if (fill(g) > best) { best = fill(g); groups = g; }
         }
-        const int streams = c->tc32 ? 1 : attn_tc_streams(n, c->G);
-        const int64_t slots_cap = part_rows_cap / ((int64_t)n * c->G) / streams;   // slots = streams * (groups + Hkv - 1)
+        const int streams = c->tc32 ? 1 : attn_tc_streams(n, c->Gp);
+        const int64_t slots_cap = part_rows_cap / ((int64_t)n * c->Gp) / streams;   // slots = streams * (groups + Hkv - 1)
         if (groups + Hkv - 1 > slots_cap) groups = slots_cap - (Hkv - 1);
         if (groups > Hkv * nt) groups = Hkv * nt;
         if (groups < Hkv) groups = Hkv;
@@ -554,9 +556,10 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.quant_bits = c->quant ? c->qp.bits : 0;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c->G; aa.d = f.head_dim;
+    aa.Gp = c->Gp;
     aa.splits = plan.tc ? 1 : plan.splits;
     aa.ngroups = plan.ngroups;
-    aa.streams = (c->tc && !plan.qdec) ? attn_tc_streams(n, c->G) : 1;
+    aa.streams = (c->tc && !plan.qdec) ? attn_tc_streams(n, c->Gp) : 1;
     aa.out_f32 = (f.dtype == KVF_F32 || (f.flags & KVF_OUT_F32)) ? 1 : 0;
     aa.scale_log2 = c->scale_log2;
     aa.range_valid = 0;
@@ -633,6 +636,7 @@ kvf_status init_handle(kvf_cache *c, const kvf_config *cfg, void *storage, void 
     c->workspace = static_cast<char *>(workspace);
     c->len = 0;
     c->G = cfg->n_q_heads / cfg->n_kv_heads;
+    c->Gp = attn_tc_padded_group(c->G);
     const double scale = cfg->softmax_scale > 0.0 ? cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
     c->scale_log2 = (float)(scale * 1.4426950408889634);
     for (int j = 0; j < cfg->head_dim / 2; ++j)
@@ -1083,7 +1087,7 @@ kvf_status kvf_batch_create(kvf_cache *const *caches, int32_t n_caches, void *de
     const kvf_config &f = c0->cfg;
     const uint64_t row = (uint64_t)f.head_dim * 2;
     s = make_map(fn, &b->map_q, b->workspace + lay.q_rot, (uint64_t)f.n_q_heads, (uint64_t)n_caches * f.max_chunk, row,
-                 row * f.n_q_heads, f.head_dim, (uint32_t)c0->G, (uint32_t)(128 / c0->G));
+                 row * f.n_q_heads, f.head_dim, (uint32_t)c0->Gp, (uint32_t)(128 / c0->Gp));
     if (s != KVF_OK) { delete b; return s; }
 
     std::vector<const int32_t *> tables(n_caches);
@@ -1207,9 +1211,10 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     aa.quant_bits = c0->quant ? c0->qp.bits : 0;
     aa.capacity = f.capacity; aa.prefix = P;
     aa.n = n; aa.H = f.n_q_heads; aa.Hkv = f.n_kv_heads; aa.G = c0->G; aa.d = f.head_dim;
+    aa.Gp = c0->Gp;
     aa.splits = 1;
     aa.ngroups = plan.ngroups;
-    aa.streams = plan.qdec ? 1 : attn_tc_streams(n, c0->G);
+    aa.streams = plan.qdec ? 1 : attn_tc_streams(n, c0->Gp);
     aa.out_f32 = (f.flags & KVF_OUT_F32) ? 1 : 0;
     aa.scale_log2 = c0->scale_log2;
     aa.range_valid = 0;
@@ -1414,8 +1419,9 @@ extern "C" kvf_status kvf_fold_step_static(const kvf_config *cfg, void *dev_stor
         // kernel will write has to fit (the plan cuts the key range no finer than the rest allows).
         const int G = cfg->n_q_heads / cfg->n_kv_heads;
         const bool tensor_path = !(cfg->flags & KVF_FORCE_SIMT) && attn_tc_supported(cfg->dtype, cfg->head_dim, G);
-        if (tensor_path && attn_tc_streams(n_tokens, G) == 2) {
-            const size_t least = (size_t)2 * (2 * (size_t)cfg->n_kv_heads - 1) * (size_t)n_tokens * G;
+        const int Gp = attn_tc_padded_group(G);      // rows a token takes in the partial slots
+        if (tensor_path && attn_tc_streams(n_tokens, Gp) == 2) {
+            const size_t least = (size_t)2 * (2 * (size_t)cfg->n_kv_heads - 1) * (size_t)n_tokens * Gp;
             if (least > part_tokens * (size_t)cfg->n_q_heads) {
                 snprintf(g_cuda_err, sizeof(g_cuda_err),
                          "a short chunk over %d KV heads leaves more partial rows than the static scratch holds",

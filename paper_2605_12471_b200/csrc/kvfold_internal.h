@@ -131,7 +131,7 @@ struct AttnArgs {
     void *out;                       // [n][H][d], dtype or fp32
     float *lse;                      // [n][H] or null (natural log)
     float *part_o;                   // partial outputs, fp32, normalised per part: CUDA-core path
-                                     // [splits][n][H][d]; tensor-core path [slot][n * G][d]
+                                     // [splits][n][H][d]; tensor-core path [slot][n * Gp][d]
     float *part_lse;                 // log2 denominators of the parts, same order; -inf = no key seen
     int *status;                     // device status word
     const int32_t *page_table;       // paged cache: device table of page numbers (one per key tile), else null
@@ -155,6 +155,10 @@ struct AttnArgs {
     int64_t win_lo;
     int64_t capacity, prefix;
     int32_t n, H, Hkv, G, d;
+    int32_t Gp;                      // rows a token takes in the row layout of the tensor-core kernels and of the partial
+                                     // slots (row = token * Gp + head-in-group): G, or for the tcgen05 kernels G rounded up
+                                     // to a power of two so that a 128-row tile holds whole tokens (rows with
+                                     // head-in-group >= G are padding: computed, never written)
     int32_t splits;                  // CUDA-core path: equal splits of the key range
     int32_t ngroups;                 // tensor-core path: contiguous ranges of the (KV head, key tile) line
     int32_t streams;                 // tensor-core path: 2 = one row tile, its key tiles dealt to two streams
@@ -220,7 +224,8 @@ struct TcMaps {
     CUtensorMap q, k, v;
 };
 bool attn_tc_supported(int dtype, int d, int G);
-int attn_tc_row_pairs(int n, int G);   // 256-row pairs per KV head = grid.x
+int attn_tc_padded_group(int G);       // G rounded up to a power of two: rows a token takes in the tcgen05 kernels' row layout
+int attn_tc_row_pairs(int n, int G);   // 256-row pairs per KV head = grid.x (G: the padded group, as below)
 int attn_tc_streams(int n, int G);     // 2 when the chunk fits one 128-row tile
 cudaError_t launch_attn_tc(const AttnArgs &a, const TcMaps &maps, cudaStream_t s);   // grid (row pairs, ngroups)
 cudaError_t launch_combine_groups(const AttnArgs &a, cudaStream_t s);                // needed when ngroups != Hkv

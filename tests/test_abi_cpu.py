@@ -64,7 +64,7 @@ def test_storage_bytes_follow_the_papers_per_token_count(binding):
 @pytest.mark.parametrize("kw,code", [
     (dict(n_q_heads=0), "KVF_ERR_INVALID_ARG"),
     (dict(n_q_heads=30), "KVF_ERR_INVALID_ARG"),            # not a multiple of the KV heads
-    (dict(n_q_heads=24), "KVF_ERR_UNSUPPORTED"),            # group of 3: not a power of two
+    (dict(n_q_heads=520), "KVF_ERR_UNSUPPORTED"),           # 65 query heads per KV head: more than 64
     (dict(head_dim=96), "KVF_ERR_UNSUPPORTED"),
     (dict(dtype=7), "KVF_ERR_UNSUPPORTED"),
     (dict(capacity=0), "KVF_ERR_INVALID_ARG"),
