@@ -866,7 +866,8 @@ def run_chain_bench(args, w, drift=False):
         per_clock = TENSOR_FLOP_PER_SM_CLOCK / (3.0 if w.dtype == "f32" else 1.0)
         roofline["sm_mhz_during_profile"] = prof_mhz
         roofline["frac_of_tensor_rate_at_sampled_clock"] = attn_tflops * 1e12 / (prof_mhz * 1e6 * N_SMS * per_clock)
-    if ns_b > ns_a:
+    if ns_b > ns_a and roofline["bound"] == "tensor":
+        # (only the tcgen05 kernels for long chunks keep these counters: not reported for decode-shaped runs)
         # the attention kernels inside the timed chains themselves (no events between the kernels there): time and
         # cycles one CTA of every launch (its last row block) was running, from the kernels' own counters
         in_ms = (ns_b - ns_a) * 1e-6 / steps_timed
