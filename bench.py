@@ -37,9 +37,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # ncu capture of the last steps of a 65 536-token chain of 256-token chunks (too large to capture
 # at 131 072 tokens; traffic grows in proportion to the cache rows read, so the ratio carries
 # over).  Set to None whenever the attention kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_CACHE_BYTE = 1.034
+NCU_TRAFFIC_BYTES_PER_CACHE_BYTE = 1.033
 NCU_TRAFFIC_SOURCE = ("ncu capture (dram__bytes_read.sum + dram__bytes_write.sum) of the attention kernel on the "
-                      "last steps of a 65 536-token chain of 256-token chunks: 1.034 DRAM bytes per algorithmic "
+                      "last steps of a 65 536-token chain of 256-token chunks: 1.033 DRAM bytes per algorithmic "
                       "cache byte, scaled by the cache rows a launch of this run reads")
 NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 7700.0}      # dense bf16 and HBM3e figures of the B200 data sheet
 TENSOR_FLOP_PER_SM_CLOCK = 8192.0                         # one 128 x 128 x 16 bf16 MMA (524 288 FLOP) per 64 clocks
