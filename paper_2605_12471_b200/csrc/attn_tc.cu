@@ -188,15 +188,18 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     const WindowTiles wt(kWindow ? a.win_lo : 0, kWindow ? a.n_sink : 0, kRows);
     const int nt_need = (int)((P + tok_last + 1 + kRows - 1) / kRows) - wt.skip;
     const int nt_all = (int)((L + kRows - 1) / kRows) - wt.skip;
-    const int64_t line = (int64_t)a.Hkv * nt_all;
+    // (the line holds a.piece_cost virtual tiles in front of every KV head's key tiles: a range that runs into the
+    // next head spends them on what its second piece costs and takes that many key tiles fewer)
+    const int pcost = a.piece_cost, ntv = nt_all + pcost;
+    const int64_t line = (int64_t)a.Hkv * ntv;
     const int64_t lin0 = group * line / a.ngroups, lin1 = (group + 1) * line / a.ngroups;
-    const int kvh_first = (int)(lin0 / nt_all);
+    const int kvh_first = (int)(lin0 / ntv);
     // piece k of this CTA: KV head kvh_first + k, tiles [kt0, kt0 + ntiles)
     auto piece = [&](int kvh, int &kt0, int &ntiles) -> bool {
-        const int64_t b = (int64_t)kvh * nt_all;
+        const int64_t b = (int64_t)kvh * ntv;
         if (kvh >= a.Hkv || b >= lin1) return false;
-        kt0 = (int)(max(lin0, b) - b);
-        const int kt1 = (int)min(min(lin1, b + nt_all) - b, (int64_t)nt_need);
+        kt0 = max((int)(max(lin0, b) - b) - pcost, 0);
+        const int kt1 = min(max((int)(min(lin1, b + ntv) - b) - pcost, 0), nt_need);
         ntiles = kt1 - kt0;
         return true;
     };
@@ -787,7 +790,7 @@ __global__ void __launch_bounds__(256, kFew ? 4 : 2) combine_groups_kernel(const
         if (threadIdx.x == 0) {
             const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix;
             const int nt_all = (int)((P + n_b + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
-            group_range(a.Hkv, nt_all, a.ngroups, kvh, g_range[0], g_range[1]);
+            group_range(a.Hkv, nt_all + a.piece_cost, a.ngroups, kvh, g_range[0], g_range[1]);
         }
         __syncthreads();
         g0 = g_range[0];

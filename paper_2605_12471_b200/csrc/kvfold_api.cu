@@ -469,6 +469,19 @@ kvf_status check_ptr(const void *p) {
     return KVF_OK;
 }
 
+// What a second piece costs a CTA of the bf16 / quantised tcgen05 kernel, in key tiles (measured at C = 256 on
+// the Llama shape: ~3.3): the line the groups cut carries that many virtual tiles in front of every KV head, so a
+// CTA whose range runs into the next head takes as many key tiles fewer and all CTAs of a launch finish
+// together.  Only where ranges do run across heads (a group count that is no multiple of the KV heads) and for
+// chunks of two row tiles; the fp32 kernel and the decode kernel cut the plain line.
+#ifndef KVF_PIECE_COST
+#define KVF_PIECE_COST 3
+#endif
+int piece_cost_of(const kvf_cache *c, const Plan &plan, int streams) {
+    if (!c->tc || plan.qdec || streams != 1 || plan.ngroups % c->cfg.n_kv_heads == 0) return 0;
+    return KVF_PIECE_COST;
+}
+
 // The groups that touch each KV head, worked out once on the host for the combine kernel.
 void fill_group_ranges(AttnArgs &aa, int64_t nt_all) {
     aa.range_valid = 0;
@@ -563,8 +576,9 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.out_f32 = (f.dtype == KVF_F32 || (f.flags & KVF_OUT_F32)) ? 1 : 0;
     aa.scale_log2 = c->scale_log2;
     aa.range_valid = 0;
+    aa.piece_cost = piece_cost_of(c, plan, aa.streams);
     if (plan.tc && plan.kernels > 2)
-        fill_group_ranges(aa, (P + n + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip);
+        fill_group_ranges(aa, (P + n + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip + aa.piece_cost);
 
     cudaError_t e;
     if (c->quant) {
@@ -1218,8 +1232,9 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     aa.out_f32 = (f.flags & KVF_OUT_F32) ? 1 : 0;
     aa.scale_log2 = c0->scale_log2;
     aa.range_valid = 0;
+    aa.piece_cost = piece_cost_of(c0, plan, aa.streams);
     if (!ragged && plan.kernels > 2)
-        fill_group_ranges(aa, (P + n + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip);
+        fill_group_ranges(aa, (P + n + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip + aa.piece_cost);
 
     cudaError_t e = c0->quant ? launch_rope_append_q8(ra, c0->qp, (f.flags & KVF_ROPE_INTERLEAVED) != 0, B, st)
                               : launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, B, st);

@@ -162,6 +162,10 @@ struct AttnArgs {
     int32_t splits;                  // CUDA-core path: equal splits of the key range
     int32_t ngroups;                 // tensor-core path: contiguous ranges of the (KV head, key tile) line
     int32_t streams;                 // tensor-core path: 2 = one row tile, its key tiles dealt to two streams
+    int32_t piece_cost;              // tensor-core path: the line the groups cut holds, in front of every KV head's key
+                                     // tiles, this many virtual tiles that stand for what a second piece costs a CTA
+                                     // (another Q load, another drain and set of partial rows): a CTA whose range
+                                     // runs into the next KV head gets that many key tiles fewer (0: plain line)
     int32_t out_f32;
     float scale_log2;                // softmax scale * log2(e)
     // tensor-core paths, when the host knows the row count (no ragged batch): first and last group whose
@@ -173,6 +177,8 @@ constexpr int kRangeHeads = 64;
 
 // Groups cut the line of Hkv * nt_all (KV head, key tile) pairs into ngroups ranges, group g owning
 // [g * line / ngroups, (g + 1) * line / ngroups).  First and last group that own a tile of KV head kvh.
+// (With AttnArgs::piece_cost the line holds nt_all + piece_cost entries per KV head: callers pass that sum,
+// and a group that owns only virtual tiles of a head still counts - it leaves an empty partial.)
 __host__ __device__ inline void group_range(int Hkv, int nt_all, int ngroups, int kvh, int &g_first, int &g_last) {
     const int64_t line = (int64_t)Hkv * nt_all;
     auto start = [&](int64_t g) { return g * line / ngroups; };
