@@ -500,6 +500,80 @@ def run_multi_needle(args):
     print(json.dumps(line), flush=True)
 
 
+def run_row_range(args):
+    """One sequence whose cache rows are dealt to the ranks chunk by chunk (not the headline line; strong
+    scaling: the whole job is one chain).  Every step: the rank that takes the chunk folds it, the others let the
+    same queries attend to the rows they hold (kvf_attend), one all-gather of (out, lse) and kvf_merge_partials
+    (multi.row_range_fold_step).  On one GPU the owner is always rank 0 and the gather is the identity: the line
+    then shows what the split costs a step (the log-sum-exp output, fp32 parts and the merge kernel)."""
+    import torch.distributed as dist
+    from paper_2605_12471_b200 import binding, multi
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the fold step has no CPU path")
+    rank, world, local = multi.env_rank()
+    torch.cuda.set_device(local)
+    if world > 1 and not dist.is_initialized():
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    w = workloads.DEEP_CHAIN
+    if args.tokens or args.chunk:
+        w = w.with_(tokens=args.tokens or w.tokens, chunk=args.chunk or w.chunk)
+    T, C, H, Hkv, d = w.tokens, w.chunk, w.n_q_heads, w.n_kv_heads, w.head_dim
+    N = T // C
+    mine = (N + world - 1 - rank) // world * C + C           # rows this rank will hold, rounded up
+    flags = binding.KVF_OUT_F32                               # parts travel in fp32: no second rounding in the merge
+    cfg = binding.make_config(H, Hkv, d, "bf16", min(T, mine), C, rope_base=w.rope_base, flags=flags)
+    cache = binding.Cache(cfg)
+    q, k, v = workloads.sequence_inputs(w, args.seed, sequence=0, device="cuda")      # every rank draws the same sequence
+
+    def chain():
+        cache.reset()
+        for t in range(N):
+            sl = slice(t * C, (t + 1) * C)
+            multi.row_range_fold_step(cache, q[sl], k[sl], v[sl], t, t * C, rank, world)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(3):
+        chain()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    a.record()
+    for _ in range(args.steps):
+        chain()
+    b.record()
+    barrier()
+    ms = multi.max_over_ranks(a.elapsed_time(b), device="cuda") / args.steps
+    clocks = sampler.stop() if rank == 0 else None
+    assert cache.status() == binding.KVF_OK, hex(cache.status_word())
+    if rank == 0:
+        pk = peaks()
+        tf = w.flops_chain() / (ms * 1e-3) / 1e12
+        line = {"metric": "fold-step tokens/s", "value": T / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
+                "steps": args.steps, "warmup": 3, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "row_range_" + w.name, "shard": "cache rows, chunk t on rank t % world", "tokens": T,
+                           "chunk": C, "n_q_heads": H, "n_kv_heads": Hkv, "head_dim": d,
+                           "exchange": "all-gather of fp32 (out, lse): %d bytes per rank and step" % (C * H * (d + 1) * 4),
+                           "launch": "every step from the host", "l2": "inputs larger than L2 at full size"},
+                "attention_tflops": tf,
+                "roofline": {"bound": "tensor", "achieved": tf, "peak": pk["bf16_tflops_sustained"] * world,
+                             "unit": "TFLOP/s", "frac": tf / (pk["bf16_tflops_sustained"] * world),
+                             "peak_source": "measured sustained bf16 x ranks" if pk["_source"] == "measured" else "fallback x ranks",
+                             "kernel": "whole chain (all kernels, exchange and merge)", "traffic": None},
+                "cpu_baseline": None, "e2e": None, "gpu_launches": cache.launch_count() // (args.steps + 3) + N,
+                "clocks": clocks}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -513,7 +587,7 @@ def parse_args():
                          "then runs from this prefix to --tokens (decode- and question-shaped steps at depth)")
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"],
                     help="cache and input dtype (not the benchmark workload)")
-    ap.add_argument("--workload", default="deep_chain", choices=["deep_chain", "llama_16k", "sweep", "full_stack", "batch_decode", "multi_needle"],
+    ap.add_argument("--workload", default="deep_chain", choices=["deep_chain", "llama_16k", "sweep", "full_stack", "batch_decode", "multi_needle", "row_range"],
                     help="deep_chain: 131 072 tokens in chunks of 256 (the headline line).  llama_16k: 16 384 tokens "
                          "in chunks of 2048, inputs scaled by 1/sqrt(128).  sweep: 65 536 tokens at chunks of 128, "
                          "512, 2048 and 8192, each with a bf16 and an fp32 cache, one line per combination with the "
@@ -568,6 +642,9 @@ def main():
         return
     if args.workload == "multi_needle" and args.impl == "ours":
         run_multi_needle(args)
+        return
+    if args.workload == "row_range" and args.impl == "ours":
+        run_row_range(args)
         return
     if args.workload == "sweep":
         variants = workloads.SWEEP

@@ -222,6 +222,37 @@ kvf_status kvf_fold_step(kvf_cache *c, const void *q, const void *k_new, const v
  * that flag for when they are there).  The host buffers must stay valid until the stream reaches
  * the end of the call (result buffers under KVF_HOST_DOWNLOAD_BEHIND: until the results are there).
  */
+/*
+ * Queries only: the n_tokens query rows are rotated at positions pos0, pos0+1, ... and attend to ALL
+ * rows the cache holds (no causal limit: none of them is a row of this chunk); nothing is appended
+ * and kvf_cache_len does not change.  out and lse as in kvf_fold_step; pass lse whenever the result
+ * is to be merged with others.  (Section 2: a chunk's queries attend to the concatenation of the
+ * rows of all chunks so far; when those rows are spread over several caches - one sequence split
+ * by row range over GPUs, Section 5's single-GPU memory limit being what such a split lifts - the
+ * cache that takes the chunk runs kvf_fold_step and every other one kvf_attend, and
+ * kvf_merge_partials puts the results together.)  KVF_ERR_INVALID_ARG on an empty cache (there is
+ * nothing to attend to: leave that part out of the merge, or give it lse = -inf),
+ * KVF_ERR_UNSUPPORTED under a sink + window mask.  Same stream semantics, workspace use and error
+ * contract as kvf_fold_step.
+ */
+kvf_status kvf_attend(kvf_cache *c, const void *q, int32_t n_tokens, int64_t pos0, void *out, float *lse,
+                      void *cuda_stream);
+
+/*
+ * Merges n_parts attention results over disjoint sets of rows into the result over their union:
+ *     lse = log sum_r exp(lse_r),   out = sum_r exp(lse_r - lse) * out_r     (parts in index order).
+ * parts_out: device, [n_parts][n_rows][head_dim], elements of `dtype` (KVF_BF16 or KVF_F32: what the
+ * steps wrote - fp32 under KVF_OUT_F32, which keeps the merged result free of a second rounding);
+ * parts_lse: device, [n_parts][n_rows] fp32 natural-log values as kvf_fold_step / kvf_attend return
+ * them (-inf: that part saw no row and is skipped); n_rows = tokens * query heads; out: device,
+ * [n_rows][head_dim] of `dtype`; lse: device [n_rows] or null.  This layout is what an all-gather of
+ * every rank's (out, lse) produces.  head_dim 64 or 128; pointers 16-byte (lse: 4-byte) aligned.
+ * Stateless: needs no cache handle and no workspace; one kernel on cuda_stream.  (The paper runs on one
+ * GPU and has no counterpart; the identity is the softmax over a union of key sets, Section 2.)
+ */
+kvf_status kvf_merge_partials(int32_t n_parts, int64_t n_rows, int32_t head_dim, kvf_dtype dtype, const void *parts_out,
+                              const float *parts_lse, void *out, float *lse_or_null, void *cuda_stream);
+
 kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_host,
                               const void *v_host, int32_t n_tokens, int64_t pos0, void *out_host,
                               float *lse_host, void *cuda_stream);

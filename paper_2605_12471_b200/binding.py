@@ -22,7 +22,7 @@ KVF_HOST_UPLOAD_AHEAD, KVF_CACHE_INT4, KVF_HOST_DOWNLOAD_BEHIND, KVF_COMBINE_BEH
 
 EXPORTS = [
     "kvf_cache_storage_bytes", "kvf_workspace_bytes", "kvf_cache_create", "kvf_fold_step",
-    "kvf_fold_step_host", "kvf_cache_len", "kvf_cache_reset", "kvf_cache_set_len", "kvf_cache_status",
+    "kvf_fold_step_host", "kvf_attend", "kvf_merge_partials", "kvf_cache_len", "kvf_cache_reset", "kvf_cache_set_len", "kvf_cache_status",
     "kvf_cache_k_plane", "kvf_cache_v_plane", "kvf_cache_plan", "kvf_cache_set_splits",
     "kvf_cache_launch_count", "kvf_cache_profile", "kvf_cache_profile_read", "kvf_cache_destroy",
     "kvf_status_str", "kvf_last_cuda_error", "kvf_fold_step_static", "kvf_cache_status_word",
@@ -91,6 +91,10 @@ def load() -> ctypes.CDLL:
     lib.kvf_cache_len.restype = i64
     lib.kvf_cache_reset.argtypes = [vp]
     lib.kvf_cache_reset.restype = ctypes.c_int
+    lib.kvf_attend.argtypes = [vp, vp, i32, i64, vp, vp, vp]
+    lib.kvf_attend.restype = ctypes.c_int
+    lib.kvf_merge_partials.argtypes = [i32, i64, i32, ctypes.c_int, vp, vp, vp, vp, vp]
+    lib.kvf_merge_partials.restype = ctypes.c_int
     lib.kvf_cache_set_len.argtypes = [vp, i64]
     lib.kvf_cache_set_len.restype = ctypes.c_int
     lib.kvf_cache_status.argtypes = [vp]
@@ -237,6 +241,19 @@ class Cache:
                                   _stream_ptr(stream))
         if rc != KVF_OK:
             raise KvfError(rc, "kvf_fold_step")
+        return out
+
+    def attend(self, q: torch.Tensor, pos0: Optional[int] = None, out: Optional[torch.Tensor] = None,
+               lse: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """kvf_attend: the queries attend to every row the cache holds; nothing is appended."""
+        n = q.shape[0]
+        assert q.is_cuda and q.is_contiguous() and q.dtype == self.torch_dtype
+        if out is None:
+            out = torch.empty((n, self.cfg.n_q_heads, self.cfg.head_dim), dtype=self.out_dtype, device=q.device)
+        rc = load().kvf_attend(self._h, q.data_ptr(), n, int(len(self) if pos0 is None else pos0), out.data_ptr(),
+                               lse.data_ptr() if lse is not None else None, _stream_ptr(stream))
+        if rc != KVF_OK:
+            raise KvfError(rc, "kvf_attend")
         return out
 
     def fold_step_host(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, out: torch.Tensor,
@@ -508,6 +525,26 @@ def paged_pool_bytes(cfg: kvf_config, n_pages: int) -> int:
 
 
 STATIC_SCRATCH_BYTES = 21234688
+
+
+def merge_partials(parts_out: torch.Tensor, parts_lse: torch.Tensor, out: Optional[torch.Tensor] = None,
+                   lse: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """kvf_merge_partials on [parts, tokens, heads, head_dim] outputs (bf16 or fp32) and [parts, tokens, heads]
+    log-sum-exps; returns (out, lse)."""
+    assert parts_out.is_cuda and parts_out.is_contiguous() and parts_out.dim() == 4
+    assert parts_lse.is_cuda and parts_lse.is_contiguous() and parts_lse.dtype == torch.float32
+    assert parts_lse.shape == parts_out.shape[:3] and parts_out.dtype in (torch.bfloat16, torch.float32)
+    r, n, h, d = parts_out.shape
+    if out is None:
+        out = torch.empty((n, h, d), dtype=parts_out.dtype, device=parts_out.device)
+    if lse is None:
+        lse = torch.empty((n, h), dtype=torch.float32, device=parts_out.device)
+    rc = load().kvf_merge_partials(r, n * h, d, KVF_F32 if parts_out.dtype == torch.float32 else KVF_BF16,
+                                   parts_out.data_ptr(), parts_lse.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                   _stream_ptr(stream))
+    if rc != KVF_OK:
+        raise KvfError(rc, "kvf_merge_partials")
+    return out, lse
 
 
 def fold_step_static(cfg: kvf_config, storage: torch.Tensor, length: int, q: torch.Tensor, k_new: torch.Tensor,

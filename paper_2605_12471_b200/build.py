@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libkvfold.so")
-SOURCES = ["kvfold_api.cu", "rope_append.cu", "quant_append.cu", "attn_simt.cu", "attn_tc.cu", "attn_tc32.cu", "attn_q8_decode.cu"]
+SOURCES = ["kvfold_api.cu", "rope_append.cu", "quant_append.cu", "attn_simt.cu", "attn_tc.cu", "attn_tc32.cu", "attn_q8_decode.cu", "merge_parts.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -229,7 +229,7 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     // tokens this cache folds; a.n is the longest chunk of the launch and the stride of the caches' blocks
     const int n = a.ns ? (int)a.ns[cb] : a.n, nmax = a.n, nG = n * G;
     if (n <= 0) return;                                   // a member that sits the step out
-    const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix, L = P + n;
+    const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix, L = P + n * a.self_rows;
     const bool direct = a.ngroups == a.Hkv;
     // rows of a partial slot; the slots keep the row layout of the tensor-core kernels, row = token * Gp +
     // head-in-group with Gp = G rounded up to a power of two, because the same merge kernel reads both
@@ -363,7 +363,7 @@ attn_q8_decode_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const int R = 8 * nb + 2 * t4 + e;
-                limit[nb][e] = R < nG ? R / G + 1 : (1 << 30);
+                limit[nb][e] = R < nG ? (R / G + 1) * a.self_rows : (1 << 30);
             }
         const float sl2 = a.scale_log2;
         bool ok = true;

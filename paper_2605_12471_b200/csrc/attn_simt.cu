@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_simt_kernel(const AttnArgs a
     const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
     const int tile = blockIdx.x, kvh = blockIdx.y, split = blockIdx.z;
     const int G = a.G, n = a.n;
-    const int64_t P = a.prefix, L = P + n;
+    const int64_t P = a.prefix, L = P + n * a.self_rows;
     const T *q = reinterpret_cast<const T *>(a.q_rot);
     const T *Kp = reinterpret_cast<const T *>(a.k_plane) + (int64_t)kvh * a.capacity * D;
     const T *Vp = reinterpret_cast<const T *>(a.v_plane) + (int64_t)kvh * a.capacity * D;
@@ -60,7 +60,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_simt_kernel(const AttnArgs a
     // key-tile range of this split; the row tile needs keys below P + (last token + 1)
     const int row0 = tile * BM;
     const int tok_last = min(n - 1, (row0 + BM - 1) / G);
-    const int64_t need = P + tok_last + 1;
+    const int64_t need = P + (tok_last + 1) * a.self_rows;
     // (virtual key tiles: without a window they are the key tiles themselves)
     const WindowTiles wt(a.win_lo, a.n_sink, BN);
     const int nt_need = (int)((need + BN - 1) / BN) - wt.skip;
@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_simt_kernel(const AttnArgs a
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         int tok = (row0 + 4 * ty + i) / G;
-        limit[i] = tok < n ? P + tok + 1 : 0;
+        limit[i] = tok < n ? P + (tok + 1) * a.self_rows : 0;
     }
 
     float m[4], l[4], acc[4][NC * 4];

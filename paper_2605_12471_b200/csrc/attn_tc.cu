@@ -168,7 +168,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     // tokens this cache folds; a.n is the longest chunk of the launch and the stride of the caches' blocks
     const int n = a.ns ? (int)a.ns[cb] : a.n, nmax = a.n;
     if (blockIdx.x * 2 * kRows >= n * G) return;          // a shorter member of a batch: no row of this row pair exists
-    const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix, L = P + n;
+    const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix, L = P + n * a.self_rows;
     // streams == 2 (chunks of at most 128 / G tokens, i.e. one row tile): the two tile slots work on
     // the SAME 128 rows and take alternate key tiles, so that one stream's softmax still runs under
     // the other stream's MMAs; each stream leaves its own partial result.
@@ -186,7 +186,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
     const int tok_last = min(n - 1, ((kPair ? (qpair | 1) * 2 * kRows : row0) + 2 * kRows - 1) / G);
     // (virtual key tiles: without a window they are the key tiles themselves)
     const WindowTiles wt(kWindow ? a.win_lo : 0, kWindow ? a.n_sink : 0, kRows);
-    const int nt_need = (int)((P + tok_last + 1 + kRows - 1) / kRows) - wt.skip;
+    const int nt_need = (int)((P + (tok_last + 1) * a.self_rows + kRows - 1) / kRows) - wt.skip;
     const int nt_all = (int)((L + kRows - 1) / kRows) - wt.skip;
     // (the line holds a.piece_cost virtual tiles in front of every KV head's key tiles: a range that runs into the
     // next head spends them on what its second piece costs and takes that many key tiles fewer)
@@ -545,7 +545,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_q, cons
         const int j0 = streams == 2 ? i : 0, jstep = streams;        // my key tiles of a piece
         // keys below `limit` are visible; a row past the chunk's end is never written, and each
         // row of S, P and O depends on that row alone, so such rows are left unmasked
-        const int64_t limit = valid ? P + tok + 1 : ((int64_t)1 << 62);
+        const int64_t limit = valid ? P + (tok + 1) * a.self_rows : ((int64_t)1 << 62);
         const float sl2 = a.scale_log2;
         const float2 sl2v = make_float2(sl2, sl2);
         const int64_t nG = (int64_t)nmax * G;                 // rows of a partial slot
@@ -789,7 +789,7 @@ __global__ void __launch_bounds__(256, kFew ? 4 : 2) combine_groups_kernel(const
         if (n_b == 0) return;         // this cache sat the step out
         if (threadIdx.x == 0) {
             const int64_t P = a.prefixes ? a.prefixes[cb] : a.prefix;
-            const int nt_all = (int)((P + n_b + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
+            const int nt_all = (int)((P + n_b * a.self_rows + kRows - 1) / kRows) - WindowTiles(a.win_lo, a.n_sink, kRows).skip;
             group_range(a.Hkv, nt_all + a.piece_cost, a.ngroups, kvh, g_range[0], g_range[1]);
         }
         __syncthreads();

@@ -164,13 +164,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
     const int rblock = blockIdx.x, group = blockIdx.y;
     const uint32_t rank = kPair ? cluster_cta_rank() : 0u;
     const int G = a.Gp, Gq = a.G, n = a.n;      // rows per token in the row layout (a power of two), query heads per KV head
-    const int64_t P = a.prefix, L = P + n;
+    const int64_t P = a.prefix, L = P + n * a.self_rows;
     const bool direct = a.ngroups == a.Hkv;
     const int row0 = rblock * kRows;
     // (paired variant: both CTAs of a cluster take the steps the later row block needs; the earlier one finds
     // nothing visible in the last of them, and its rows' limits mask those keys out)
     const int tok_last = min(n - 1, ((kPair ? (rblock | 1) * kRows : row0) + kRows - 1) / G);
-    const int64_t need = P + tok_last + 1;            // keys below `need` are visible to some row of this CTA
+    const int64_t need = P + (tok_last + 1) * a.self_rows;            // keys below `need` are visible to some row of this CTA
     // (virtual key tiles: without a window they are the key tiles themselves)
     const WindowTiles wt(kWindow ? a.win_lo : 0, kWindow ? a.n_sink : 0, kTileKeys);
     const int nt_need = (int)((need + kTileKeys - 1) / kTileKeys) - wt.skip;
@@ -404,7 +404,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc32_kernel(const AttnArgs a
         const bool valid = tok < n && gi < Gq;       // (gi >= Gq: padding of a group that is no power of two)
         // keys below `limit` are visible; a row past the chunk's end is never written, and each
         // row of S, P and O depends on that row alone, so such rows are left unmasked
-        const int64_t limit = valid ? P + tok + 1 : ((int64_t)1 << 62);
+        const int64_t limit = valid ? P + (tok + 1) * a.self_rows : ((int64_t)1 << 62);
         const float sl2 = a.scale_log2;
         const int64_t nG = (int64_t)n * G;
         const uint32_t t_o = tmem + lane_addr + kColO;

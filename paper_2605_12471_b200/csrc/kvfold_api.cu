@@ -519,7 +519,10 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
                      int64_t pos0, void *out, float *lse, cudaStream_t st) {
     const kvf_config &f = c->cfg;
     const int64_t P = c->len;
-    const Plan plan = make_plan(c, n, P);
+    // k_new == null: queries only (kvf_attend) - nothing is appended, every query row sees the P rows held
+    const bool attend = k_new == nullptr;
+    const int64_t L = attend ? P : P + n;                     // rows the step's queries can see at most
+    const Plan plan = make_plan(c, n, L - n);
     const bool behind = c->comb_stream != nullptr;
     unsigned long long capture = 0;
     if (behind) {
@@ -536,10 +539,9 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     ra.capacity = f.capacity; ra.prefix = P; ra.pos0 = pos0;
     ra.n = n; ra.H = f.n_q_heads; ra.Hkv = f.n_kv_heads; ra.d = f.head_dim;
     {
-        int64_t L = P + n;
         int64_t pad_end = (L + kKvTile - 1) / kKvTile * kKvTile;
         if (pad_end > f.capacity && !c->page_table) pad_end = f.capacity;   // a page always has its 128 rows
-        ra.zero_rows = (int32_t)(pad_end - L);
+        ra.zero_rows = attend ? 0 : (int32_t)(pad_end - L);
     }
     ra.page_table = c->page_table;
     ra.page_elems = c->page_elems;
@@ -577,8 +579,9 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     aa.scale_log2 = c->scale_log2;
     aa.range_valid = 0;
     aa.piece_cost = piece_cost_of(c, plan, aa.streams);
+    aa.self_rows = attend ? 0 : 1;
     if (plan.tc && plan.kernels > 2)
-        fill_group_ranges(aa, (P + n + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip + aa.piece_cost);
+        fill_group_ranges(aa, (L + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip + aa.piece_cost);
 
     cudaError_t e;
     if (c->quant) {
@@ -630,7 +633,7 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
             c->part_set ^= 1;
         }
     }
-    c->len = P + n;
+    c->len = L;
     return KVF_OK;
 }
 
@@ -814,6 +817,29 @@ kvf_status kvf_fold_step(kvf_cache *c, const void *q, const void *k_new, const v
     if (check_ptr(q) || check_ptr(k_new) || check_ptr(v_new) || check_ptr(out)) return KVF_ERR_INVALID_ARG;
     if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return KVF_ERR_INVALID_ARG;
     return step_impl(c, q, k_new, v_new, n_tokens, pos0, out, lse, static_cast<cudaStream_t>(cuda_stream));
+}
+
+kvf_status kvf_attend(kvf_cache *c, const void *q, int32_t n_tokens, int64_t pos0, void *out, float *lse,
+                      void *cuda_stream) {
+    if (!c) return KVF_ERR_INVALID_ARG;
+    if (n_tokens < 1 || n_tokens > c->cfg.max_chunk || pos0 < 0) return KVF_ERR_INVALID_ARG;
+    if (c->len < 1) return KVF_ERR_INVALID_ARG;               // nothing to attend to
+    if (c->window > 0) return KVF_ERR_UNSUPPORTED;
+    if (check_ptr(q) || check_ptr(out)) return KVF_ERR_INVALID_ARG;
+    if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return KVF_ERR_INVALID_ARG;
+    return step_impl(c, q, nullptr, nullptr, n_tokens, pos0, out, lse, static_cast<cudaStream_t>(cuda_stream));
+}
+
+kvf_status kvf_merge_partials(int32_t n_parts, int64_t n_rows, int32_t head_dim, kvf_dtype dtype, const void *parts_out,
+                              const float *parts_lse, void *out, float *lse, void *cuda_stream) {
+    if (n_parts < 1 || n_parts > 1024 || n_rows < 1) return KVF_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return KVF_ERR_UNSUPPORTED;
+    if (dtype != KVF_BF16 && dtype != KVF_F32) return KVF_ERR_UNSUPPORTED;
+    if (check_ptr(parts_out) || check_ptr(out) || !parts_lse) return KVF_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(parts_lse) & 3u) || (lse && (reinterpret_cast<uintptr_t>(lse) & 3u))) return KVF_ERR_INVALID_ARG;
+    cudaError_t e = launch_merge_parts(n_parts, n_rows, head_dim, dtype == KVF_F32, parts_out, parts_lse, out, lse,
+                                       static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? KVF_OK : cuda_fail(e, "merge_parts launch");
 }
 
 kvf_status kvf_fold_step_host(kvf_cache *c, const void *q_host, const void *k_host, const void *v_host,
@@ -1233,6 +1259,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     aa.scale_log2 = c0->scale_log2;
     aa.range_valid = 0;
     aa.piece_cost = piece_cost_of(c0, plan, aa.streams);
+    aa.self_rows = 1;
     if (!ragged && plan.kernels > 2)
         fill_group_ranges(aa, (P + n + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip + aa.piece_cost);
 

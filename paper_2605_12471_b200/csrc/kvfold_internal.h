@@ -100,7 +100,8 @@ struct RowMap {
 
 // Arguments of the fused rotate + append kernel (one launch per step).
 struct RopeAppendArgs {
-    const void *q, *k_new, *v_new;   // [n][H][d], [n][Hkv][d], [n][Hkv][d]
+    const void *q, *k_new, *v_new;   // [n][H][d], [n][Hkv][d], [n][Hkv][d]; k_new = v_new = null: only the queries
+                                     // are rotated, nothing is appended (kvf_attend)
     void *q_rot;                     // [n][H][d]
     void *k_plane, *v_plane;         // [Hkv][capacity][d]
     int64_t capacity, prefix, pos0;  // prefix = rows already held
@@ -167,6 +168,8 @@ struct AttnArgs {
                                      // (another Q load, another drain and set of partial rows): a CTA whose range
                                      // runs into the next KV head gets that many key tiles fewer (0: plain line)
     int32_t out_f32;
+    int32_t self_rows;               // 1: a fold step - the chunk's own rows are in the cache, token i sees rows < prefix + i + 1;
+                                     // 0: queries only (kvf_attend) - nothing was appended, every token sees rows < prefix
     float scale_log2;                // softmax scale * log2(e)
     // tensor-core paths, when the host knows the row count (no ragged batch): first and last group whose
     // range of the (KV head, key tile) line touches KV head h, for h < kRangeHeads (see group_range)
@@ -244,6 +247,10 @@ cudaError_t launch_attn_q8_decode(const AttnArgs &a, const TcMaps &maps, cudaStr
 
 // Tensor-core path for fp32 caches (head_dim 128): operands split into fp16 halves, three MMAs per
 // product; contiguous planes, read straight from global memory (no tensor maps).
+// Merge of attention results over disjoint sets of cache rows (merge_parts.cu).
+cudaError_t launch_merge_parts(int n_parts, int64_t n_rows, int d, bool f32, const void *parts_out, const float *parts_lse,
+                               void *out, float *lse, cudaStream_t s);
+
 bool attn_tc32_supported(int dtype, int d, int G);
 int attn_tc32_row_blocks(int n, int G);   // 128-row blocks per KV head = grid.x
 cudaError_t launch_attn_tc32(const AttnArgs &a, cudaStream_t s);                     // grid (row blocks, ngroups)

@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
     // Rows between the new end of the cache and the next key-tile boundary get value scale 0: the
     // attention expands them to zeros whatever their codes are, so a zero probability never
     // multiplies non-finite bits.
-    if (blockIdx.x == 0 && n > 0) {
+    if (blockIdx.x == 0 && n > 0 && a.k_new) {
         const int zero_rows = a.prefixes ? (int)((kKvTile - (prefix + n) % kKvTile) % kKvTile) : a.zero_rows;
         for (int i = threadIdx.x; i < zero_rows * a.Hkv; i += kThreads)
             qp.v_scales[scale_idx(i / zero_rows, prefix + n + i % zero_rows)] = 0.f;
@@ -102,7 +102,7 @@ __global__ void __launch_bounds__(kThreads) rope_append_q8_kernel(const RopeAppe
     const __nv_bfloat16 *k = reinterpret_cast<const __nv_bfloat16 *>(a.k_new) + koff;
     const __nv_bfloat16 *v = reinterpret_cast<const __nv_bfloat16 *>(a.v_new) + koff;
     __nv_bfloat16 *qr = reinterpret_cast<__nv_bfloat16 *>(a.q_rot) + qoff;
-    const int heads = a.H + 2 * a.Hkv;         // query rows, key rows, value rows
+    const int heads = a.H + (a.k_new ? 2 * a.Hkv : 0);     // query rows, key rows, value rows (queries only: kvf_attend)
     for (int row = warp; row < ntok * heads; row += kThreads / 32) {
         const int t = row / heads, hh = row % heads;
         const int64_t tok = tok0 + t;

@@ -117,14 +117,14 @@ __global__ void __launch_bounds__(kThreads) rope_append_kernel(const RopeAppendA
     T *qr = reinterpret_cast<T *>(a.q_rot) + qoff;
     T *kp = reinterpret_cast<T *>(a.k_plane);
     T *vp = reinterpret_cast<T *>(a.v_plane);
-    const int heads = a.H + a.Hkv;
+    const int heads = a.H + (a.k_new ? a.Hkv : 0);     // (queries only when no keys are given: kvf_attend)
 
     // One loop over the rotated segments of q and k and, behind them, the value segments (verbatim
     // 16-byte copies): a thread's items are independent, so their loads go out back to back.
     const int rot_chunks = INTERLEAVED ? d / VEC : half / VEC;       // vectors per row (interleaved) or per half row
     const int rot_items = ntok * heads * rot_chunks;
     const int v_chunks = d / VEC;
-    const int items = rot_items + ntok * a.Hkv * v_chunks;
+    const int items = rot_items + (a.v_new ? ntok * a.Hkv * v_chunks : 0);
     float amax = 0.f;               // largest magnitude written (tracked only under a range limit, fp32 caches)
     const bool ranged = sizeof(T) == 4 && a.range_limit > 0.f;
     for (int idx = threadIdx.x; idx < items; idx += kThreads) {

@@ -5,8 +5,16 @@ One process per GPU.  By sequence: rank r folds sequence r into its own cache.  
 r keeps the cache planes of its block of KV heads and is given the matching query heads; since a
 query head reads one KV head only, every rank's output is a disjoint slice of the heads.  Either
 way there is no exchange on the data path (a cache never leaves its GPU), so the only collectives
-are a barrier around the timed region and the max-over-ranks of the elapsed time.  Works on any
-torch.distributed backend (NCCL on GPUs, gloo on CPU for tests).
+are a barrier around the timed region and the max-over-ranks of the elapsed time.
+
+By row range (one sequence longer than one GPU's memory): chunk t is appended on rank t % world
+(chunk_owner), so every rank holds the rows of some chunks; each step, the owner runs the fold
+step (its earlier rows plus the chunk itself, causally) and every other rank lets the same
+queries attend to what it holds (kvf_attend); ONE exchange - an all-gather of every rank's
+normalised output and log-sum-exp, [n, H, d + 1] values per rank - and the merge kernel
+(kvf_merge_partials) give the step's output on every rank (row_range_fold_step).
+
+Works on any torch.distributed backend (NCCL on GPUs, gloo on CPU for tests).
 """
 from __future__ import annotations
 
@@ -59,3 +67,41 @@ def max_over_ranks(value: float, device: str | torch.device = "cpu") -> float:
 def whole_job_tokens_per_s(tokens_per_rank_step: int, steps: int, world: int, elapsed_ms_max: float) -> float:
     """Aggregate throughput: tokens all ranks folded / the slowest rank's time."""
     return world * steps * tokens_per_rank_step / (elapsed_ms_max * 1e-3)
+
+
+def chunk_owner(step: int, world: int) -> int:
+    """Rank that appends chunk `step` when one sequence's rows are dealt to the ranks chunk by chunk."""
+    return step % world
+
+
+def gather_partials(out: torch.Tensor, lse: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+    """All-gather of every rank's (out [n, H, d], lse [n, H]) into ([world, n, H, d], [world, n, H]): the one
+    exchange of a step under the row-range split.  Without a process group: the rank's own part, as world 1."""
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return out.unsqueeze(0).contiguous(), lse.unsqueeze(0).contiguous()
+    world = dist.get_world_size()
+    outs = torch.empty((world,) + tuple(out.shape), dtype=out.dtype, device=out.device)
+    lses = torch.empty((world,) + tuple(lse.shape), dtype=lse.dtype, device=lse.device)
+    # (slices of the two result tensors as the per-rank receive buffers: works on gloo and NCCL alike)
+    dist.all_gather(list(outs.unbind(0)), out.contiguous())
+    dist.all_gather(list(lses.unbind(0)), lse.contiguous())
+    return outs, lses
+
+
+def row_range_fold_step(cache, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, step: int, pos0: int,
+                        rank: int, world: int) -> Tuple[torch.Tensor, torch.Tensor]:
+    """One fold step of a sequence whose cache rows are dealt to the ranks chunk by chunk (`cache` is this
+    rank's binding.Cache).  Returns the step's (out [n, H, d], lse [n, H]) - the same on every rank."""
+    from . import binding
+    n, h = q.shape[0], q.shape[1]
+    lse = torch.empty((n, h), dtype=torch.float32, device=q.device)
+    if chunk_owner(step, world) == rank:
+        out = cache.fold_step(q, k, v, pos0=pos0, lse=lse)
+    elif len(cache) > 0:
+        out = cache.attend(q, pos0=pos0, lse=lse)
+    else:
+        # nothing held yet: a part that saw no row
+        out = torch.zeros((n, h, q.shape[2]), dtype=cache.out_dtype, device=q.device)
+        lse.fill_(float("-inf"))
+    outs, lses = gather_partials(out, lse)
+    return binding.merge_partials(outs, lses)

@@ -106,6 +106,15 @@ def test_null_handles_are_harmless(binding):
     assert lib.kvf_cache_len(None) == -1
     assert lib.kvf_cache_reset(None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_cache_set_len(None, 0) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_attend(None, 4096, 1, 0, 4096, None, None) == binding.KVF_ERR_INVALID_ARG
+    # the merge of partial results checks its arguments before any CUDA call
+    assert lib.kvf_merge_partials(0, 8, 128, binding.KVF_BF16, 4096, 4096, 4096, None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_merge_partials(2, 0, 128, binding.KVF_BF16, 4096, 4096, 4096, None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_merge_partials(2, 8, 96, binding.KVF_BF16, 4096, 4096, 4096, None, None) == binding.KVF_ERR_UNSUPPORTED
+    assert lib.kvf_merge_partials(2, 8, 128, 7, 4096, 4096, 4096, None, None) == binding.KVF_ERR_UNSUPPORTED
+    assert lib.kvf_merge_partials(2, 8, 128, binding.KVF_BF16, None, 4096, 4096, None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_merge_partials(2, 8, 128, binding.KVF_BF16, 4096, None, 4096, None, None) == binding.KVF_ERR_INVALID_ARG
+    assert lib.kvf_merge_partials(2, 8, 128, binding.KVF_BF16, 4096, 4096, 4096 + 8, None, None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_fold_step(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_fold_step_host(None, None, None, None, 1, 0, None, None, None) == binding.KVF_ERR_INVALID_ARG
     assert lib.kvf_cache_launch_count(None) == 0
