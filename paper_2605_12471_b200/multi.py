@@ -56,8 +56,9 @@ def shard_heads(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rank: int, wo
             v[..., kvh.start:kvh.stop, :].contiguous())
 
 
-def max_over_ranks(value: float, device: str | torch.device = "cpu") -> float:
-    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+def max_over_ranks(value: float, device: str | torch.device = "cpu", always: bool = False) -> float:
+    """Largest value over the ranks (`always`: run the collective even in a group of one rank)."""
+    if not (dist.is_available() and dist.is_initialized()) or (dist.get_world_size() == 1 and not always):
         return float(value)
     t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -74,10 +75,11 @@ def chunk_owner(step: int, world: int) -> int:
     return step % world
 
 
-def gather_partials(out: torch.Tensor, lse: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+def gather_partials(out: torch.Tensor, lse: torch.Tensor, always: bool = False) -> Tuple[torch.Tensor, torch.Tensor]:
     """All-gather of every rank's (out [n, H, d], lse [n, H]) into ([world, n, H, d], [world, n, H]): the one
-    exchange of a step under the row-range split.  Without a process group: the rank's own part, as world 1."""
-    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+    exchange of a step under the row-range split.  Without a process group: the rank's own part, as world 1
+    (`always`: run the collective even in a group of one rank)."""
+    if not (dist.is_available() and dist.is_initialized()) or (dist.get_world_size() == 1 and not always):
         return out.unsqueeze(0).contiguous(), lse.unsqueeze(0).contiguous()
     world = dist.get_world_size()
     outs = torch.empty((world,) + tuple(out.shape), dtype=out.dtype, device=out.device)
