@@ -482,6 +482,17 @@ int piece_cost_of(const kvf_cache *c, const Plan &plan, int streams) {
     return KVF_PIECE_COST;
 }
 
+// A step whose attention kernel is long enough for a chain of such steps to run at the power cap: full row
+// tiles on the tensor cores and at least KVF_PDL_MAX_TILES key tiles per CTA.
+#ifndef KVF_PDL_MAX_TILES
+#define KVF_PDL_MAX_TILES 32
+#endif
+bool long_step(const kvf_cache *c, const Plan &plan, int streams, int64_t L) {
+    if (!plan.tc || plan.qdec || streams != 1 || plan.ngroups <= 0 || c->window > 0) return false;
+    const int64_t nt = (L + kKvTile - 1) / kKvTile;
+    return nt * c->cfg.n_kv_heads >= (int64_t)KVF_PDL_MAX_TILES * plan.ngroups;
+}
+
 // The groups that touch each KV head, worked out once on the host for the combine kernel.
 void fill_group_ranges(AttnArgs &aa, int64_t nt_all) {
     aa.range_valid = 0;
@@ -583,6 +594,8 @@ kvf_status step_impl(kvf_cache *c, const void *q, const void *k_new, const void 
     if (plan.tc && plan.kernels > 2)
         fill_group_ranges(aa, (L + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip + aa.piece_cost);
 
+    // plain launches for long tensor-bound steps, dependent launches for short ones (see g_pdl_allowed)
+    const PdlScope pdl(!long_step(c, plan, aa.streams, L));
     cudaError_t e;
     if (c->quant) {
         // int8 storage: rotate + quantise + append (the attention kernel expands the code tiles itself)
@@ -1263,6 +1276,7 @@ kvf_status batch_step(kvf_batch *b, const void *q, const void *k_new, const void
     if (!ragged && plan.kernels > 2)
         fill_group_ranges(aa, (P + n + kKvTile - 1) / kKvTile - WindowTiles(aa.win_lo, aa.n_sink, kKvTile).skip + aa.piece_cost);
 
+    const PdlScope pdl(!long_step(c0, plan, aa.streams, P + n));
     cudaError_t e = c0->quant ? launch_rope_append_q8(ra, c0->qp, (f.flags & KVF_ROPE_INTERLEAVED) != 0, B, st)
                               : launch_rope_append(ra, f.dtype, (f.flags & KVF_ROPE_INTERLEAVED) != 0, B, st);
     if (e != cudaSuccess) return cuda_fail(e, "rope_append launch (batch)");

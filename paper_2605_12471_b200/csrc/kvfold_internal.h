@@ -19,6 +19,18 @@ namespace kvf {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Whether the launches of the calling thread ask for it.  Overlapping a kernel's set-up with the tail of the one
+// before pays where a step is short (decode-shaped steps, short prefixes, the sink + window chain: 1.5 - 5 %);
+// a long chain of long tensor-bound steps runs at the power cap, where the idle gap between plain launches comes
+// back as clock (measured on the 131 072-token chain: 148.3 ms with plain launches against 150.1 ms, the
+// attention kernels at 1.53 instead of 1.505 GHz).  The host layer sets this per step (PdlScope).
+inline thread_local bool g_pdl_allowed = true;
+struct PdlScope {
+    bool saved;
+    explicit PdlScope(bool allow) : saved(g_pdl_allowed) { g_pdl_allowed = allow; }
+    ~PdlScope() { g_pdl_allowed = saved; }
+};
+
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args &&...args) {
     cudaLaunchConfig_t cfg = {};
@@ -28,7 +40,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = g_pdl_allowed ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
@@ -43,7 +55,7 @@ cudaError_t launch_pdl_cluster2(void (*kernel)(KArgs...), dim3 grid, dim3 block,
     cfg.stream = s;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = g_pdl_allowed ? 1 : 0;
     attr[1].id = cudaLaunchAttributeClusterDimension;
     attr[1].val.clusterDim.x = 2;
     attr[1].val.clusterDim.y = 1;
