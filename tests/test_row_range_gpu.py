@@ -21,6 +21,13 @@ def make_cache(kind, w, total, max_chunk, flags=0):
         cfg = binding.make_config(w.n_q_heads, w.n_kv_heads, w.head_dim, "bf16", total, max_chunk, rope_base=w.rope_base,
                                   flags=flags)
         return binding.Cache(cfg)
+    if kind == "paged":
+        cfg = binding.make_config(w.n_q_heads, w.n_kv_heads, w.head_dim, "bf16", total, max_chunk, rope_base=w.rope_base,
+                                  flags=flags)
+        n_pages = (total + 127) // 128
+        pool = torch.empty(binding.paged_pool_bytes(cfg, n_pages), dtype=torch.uint8, device="cuda")
+        table = torch.arange(n_pages - 1, -1, -1, dtype=torch.int32, device="cuda")      # pages in reverse order
+        return binding.PagedCache(cfg, pool, n_pages, table)
     return binding.cache_for(w, capacity=total, max_chunk=max_chunk, flags=flags)
 
 
@@ -63,7 +70,7 @@ CHUNKS = [256, 256, 100, 256, 1, 1, 2, 33, 256, 512, 7, 1]
 
 
 @pytest.mark.parametrize("world", [2, 3])
-@pytest.mark.parametrize("kind", ["bf16", "f32", "int8", "int4"])
+@pytest.mark.parametrize("kind", ["bf16", "f32", "int8", "int4", "paged"])
 def test_rows_dealt_to_several_caches_give_the_plain_fold(kind, world):
     w = LLAMA.with_(name=f"row_range_{kind}", dtype="f32" if kind == "f32" else "bf16")
     worst, worst_lse = run_split(w, kind, CHUNKS, world, seed=41)
