@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdio>
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -488,6 +489,12 @@ int piece_cost_of(const kvf_cache *c, const Plan &plan, int streams) {
 #define KVF_PDL_MAX_TILES 32
 #endif
 bool long_step(const kvf_cache *c, const Plan &plan, int streams, int64_t L) {
+    // KVF_DEPENDENT_LAUNCH=always / never in the environment overrides the rule (read once; for measurements)
+    static const int forced = [] {
+        const char *e = std::getenv("KVF_DEPENDENT_LAUNCH");
+        return !e ? 0 : std::strcmp(e, "always") == 0 ? 1 : std::strcmp(e, "never") == 0 ? 2 : 0;
+    }();
+    if (forced) return forced == 2;
     if (!plan.tc || plan.qdec || streams != 1 || plan.ngroups <= 0 || c->window > 0) return false;
     const int64_t nt = (L + kKvTile - 1) / kKvTile;
     return nt * c->cfg.n_kv_heads >= (int64_t)KVF_PDL_MAX_TILES * plan.ngroups;
