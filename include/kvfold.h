@@ -210,6 +210,11 @@ kvf_status kvf_paged_cache_create(const kvf_config *cfg, void *dev_pool, size_t 
  * Effects, in stream order: rotate q into the workspace; write rotated k and v as rows
  * [len, len+n_tokens); attention; then the host-side length becomes len + n_tokens.
  * Errors: INVALID_ARG, CAPACITY (cache full), POS, CUDA (launch failure; length unchanged).
+ * A step is two or three kernels on cuda_stream.  Short steps launch them with programmatic stream
+ * serialisation (a kernel's set-up overlaps the tail of the one before); steps with long
+ * tensor-bound attention kernels launch them plainly, which on a power-capped board is the faster
+ * of the two.  KVF_DEPENDENT_LAUNCH=always or =never in the environment (read once) overrides the
+ * choice; results do not depend on it.
  */
 kvf_status kvf_fold_step(kvf_cache *c, const void *q, const void *k_new, const void *v_new,
                          int32_t n_tokens, int64_t pos0, void *out, float *lse, void *cuda_stream);
