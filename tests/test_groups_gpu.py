@@ -116,3 +116,18 @@ def test_batch_of_paged_caches_with_groups_of_seven():
     torch.cuda.synchronize()
     assert batch.status_word() == 0
     assert worst <= TOL["bf16"][0], worst
+
+
+def test_qwen_heads_on_the_deep_chain_at_full_size():
+    """28 / 4 heads through the benchmark's launch configuration (`bench.py --q-heads 28 --kv-heads 4`): 512 steps
+    of 256 tokens to 131 072, sampled steps and rows against the oracle, the final cache in full."""
+    w = workloads.DEEP_CHAIN.with_(name="deep_chain_qwen_28_4", n_q_heads=28, n_kv_heads=4)
+    chunks = [w.chunk] * w.n_steps
+    rng = np.random.default_rng(7)
+    steps = sorted({0, 1, w.n_steps // 2, w.n_steps - 2, w.n_steps - 1} | {int(x) for x in rng.integers(0, w.n_steps, size=4)})
+    res, cache, _, _ = run_chain(w, chunks, seed=37, check_steps=steps, rows_per_step=4)
+    assert len(cache) == 131072
+    assert_within(res, "bf16", "deep chain, groups of 7")
+    assert res.rel_rms <= 2e-2, res.rel_rms
+    bits = assert_chain_cache_bits(cache, w, chunks, seed=37, what="deep chain, groups of 7: cache")
+    assert bits.elements == 131072 * 4 * 128
