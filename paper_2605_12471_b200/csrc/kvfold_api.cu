@@ -483,8 +483,8 @@ int piece_cost_of(const kvf_cache *c, const Plan &plan, int streams) {
     return KVF_PIECE_COST;
 }
 
-// A step whose attention kernel is long enough for a chain of such steps to run at the power cap: full row
-// tiles on the tensor cores and at least KVF_PDL_MAX_TILES key tiles per CTA.
+// A step whose attention kernel is long enough for a chain of such steps to run at the power cap: bf16 rows, full
+// row tiles on the tensor cores and at least KVF_PDL_MAX_TILES key tiles per CTA.
 #ifndef KVF_PDL_MAX_TILES
 #define KVF_PDL_MAX_TILES 32
 #endif
@@ -495,7 +495,9 @@ bool long_step(const kvf_cache *c, const Plan &plan, int streams, int64_t L) {
         return !e ? 0 : std::strcmp(e, "always") == 0 ? 1 : std::strcmp(e, "never") == 0 ? 2 : 0;
     }();
     if (forced) return forced == 2;
-    if (!plan.tc || plan.qdec || streams != 1 || plan.ngroups <= 0 || c->window > 0) return false;
+    // (bf16 rows only: the quantised kernels are bound by issue slots and the fp32 kernel by its softmax thread,
+    // not by the power cap - measured, they keep 0.2 - 0.5 % with dependent launches)
+    if (!c->tc || c->quant || plan.qdec || streams != 1 || plan.ngroups <= 0 || c->window > 0) return false;
     const int64_t nt = (L + kKvTile - 1) / kKvTile;
     return nt * c->cfg.n_kv_heads >= (int64_t)KVF_PDL_MAX_TILES * plan.ngroups;
 }
