@@ -65,6 +65,12 @@ def test_static_scratch_step_fp32_on_the_tensor_cores():
     _same_chain(w, [256, 256, 256, 256, 100, 1, 64], seed=33)
 
 
+def test_static_scratch_step_with_groups_of_seven():
+    """28 / 4 heads: the fixed scratch holds the partial rows in the padded-group layout as well."""
+    w = workloads.Workload("static_qwen", 28, 4, 128, "bf16", 256, 4096, 500000.0)
+    _same_chain(w, [512, 512, 256, 256, 19, 2, 1, 100], seed=34)
+
+
 def test_static_scratch_rejects_sizes_beyond_its_fixed_maximum():
     lib = binding.load()
     cfg = binding.make_config(32, 8, 128, "bf16", 4096, 1024, rope_base=5e5)      # 1024 x 32 x 128 x 2 B = 8 MiB > 4 MiB
